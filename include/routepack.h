@@ -1,0 +1,172 @@
+/*
+ * routepack.h -- C ABI of the B200 (sm_100a) RoutePack planner hot path.
+ *
+ * The library plans one optimizer-step window at a time on one GPU: it reduces the
+ * routing-replay counts to per-layer expert loads, places experts on EP ranks with the
+ * layer-local LPT rule, projects every sample's demand onto physical ranks, picks the
+ * row count and a length-only seed layout, scores layouts with the EDP-shard-aware
+ * objective and refines a population of layouts by population annealing.  Every step
+ * runs in CUDA kernels of this library; there is no CPU fallback.
+ *
+ * Conventions
+ *  - All functions return RP_OK (0) or a negative rp_status; none throws, prints, aborts
+ *    or traps.  rp_strerror() names a status.  Calling out of order gives RP_ERR_STATE.
+ *  - Array arguments are plain pointers to HOST or DEVICE memory (either is accepted for
+ *    every array, resolved with the CUDA unified-addressing rules).  The caller owns every
+ *    buffer it passes.  Output arrays are complete when the call returns (each call
+ *    synchronises its stream before returning).
+ *  - Scalars and structs are passed from host memory.
+ *  - A context belongs to the device that was current in rp_window_load and to the
+ *    stream given there; calls on one context must not overlap.
+ *  - Layouts are int32 arrays cell_of[N] with cell = row * dp_width + dp_slot.
+ *  - Scores are int64 triples in fixed point: (max_g U_g, sum_g U_g, max_{r,g} J_{r,g})
+ *    multiplied by 2^8 * token_cap^2, and the same triple as doubles divided by that scale.
+ */
+#ifndef ROUTEPACK_H_
+#define ROUTEPACK_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    RP_OK = 0,
+    RP_ERR_ARG = -1,           /* NULL or out-of-range scalar argument                    */
+    RP_ERR_SHAPE = -2,         /* E not a multiple of P, N < D, bad EDP partition, ...     */
+    RP_ERR_CONSERVATION = -3,  /* some t_i outside [1,C], negative count, or sum_e a != k*t */
+    RP_ERR_INFEASIBLE = -4,    /* no row count R <= N/D admits the length-only packing      */
+    RP_ERR_RANGE = -5,         /* fixed-point range or on-chip memory budget exceeded       */
+    RP_ERR_CUDA = -6,          /* a CUDA call failed; see rp_last_cuda_error()              */
+    RP_ERR_STATE = -7,         /* call out of order                                         */
+    RP_ERR_TIMEOUT = -8,       /* reserved: a bounded device-side wait ran out              */
+    RP_ERR_INVALID_PLAN = -9   /* rp_best: the incumbent failed validation                  */
+} rp_status;
+
+typedef struct rp_ctx rp_ctx;  /* opaque; owns all device state of one window */
+
+#define RP_MAX_STAGES 8
+
+/* Problem statement (Sections 3.1-3.4 of the paper). */
+typedef struct {
+    int32_t n_samples;          /* N                                                        */
+    int32_t n_layers;           /* L  MoE layers                                            */
+    int32_t n_experts;          /* E  logical experts per layer                             */
+    int32_t top_k;              /* k  assignments per token per layer                       */
+    int32_t token_cap;          /* C  tokens per cell                                       */
+    int32_t dp_width;           /* D  controller DP slots per execution row                 */
+    int32_t ep_width;           /* P  physical EP ranks; E % P == 0                         */
+    const int32_t *edp_of_dp;   /* HOST [D]: DP slot -> EDP shard g in [0,G), every g used;
+                                   NULL = identity (G = D)                                  */
+    int32_t n_stages;           /* attention stage types, 1..RP_MAX_STAGES                  */
+    const double *alpha;        /* HOST [n_stages] token-linear coefficients  (>= 0)        */
+    const double *beta;         /* HOST [n_stages] token-pair coefficients    (>= 0)        */
+    int32_t pop_size;           /* P_pop population members                                 */
+    int32_t min_rows;           /* optional lower bound on the row count; 0 = none          */
+    uint64_t seed;              /* Philox key of the annealing random streams               */
+} rp_config;
+
+/* Search budget (Section 4.1.2, Algorithm 3). T_n = t0 * t_ratio^n. */
+typedef struct {
+    int32_t n_levels;           /* temperature levels N                                     */
+    int32_t steps_per_level;    /* proposals K per chain per level                          */
+    double t0;                  /* first temperature, in relative-energy units              */
+    double t_ratio;             /* geometric ratio in (0,1]                                 */
+    double p_reloc;             /* relocation probability rho in [0,1]                      */
+    double p_guide;             /* guided-proposal probability in [0,1] (paper: 0.8)        */
+} rp_anneal_params;
+
+typedef struct {
+    int64_t proposed, feasible, accepted, improved;  /* summed over chains and levels       */
+    double ms_chains;           /* device time in the per-level chain kernels               */
+    double ms_barrier;          /* device time in incumbent update + resampling             */
+} rp_anneal_stats;
+
+/* Routing-replay input (Eq. routing-replay-input): creates a context, copies host arrays
+ * to the device (device arrays are adopted without a copy and must stay valid until
+ * rp_place_experts returns) and checks 1 <= t_i <= C, a >= 0 and sum_e a[i][l][e] == k*t_i.
+ *   lengths [N] int32; demand [N][L][E] int32, expert index fastest.
+ *   cuda_stream: a cudaStream_t (NULL = default stream).
+ * On failure *out is NULL. */
+int rp_window_load(rp_ctx **out, const rp_config *cfg, const int32_t *lengths,
+                   const int32_t *demand, void *cuda_stream);
+
+/* Layer-wise expert placement (Section 3.3, Algorithm 1) and demand projection
+ * (Eq. physical-rank-demand).  Aggregates L[l][e] = sum_i a[i][l][e], places each layer's
+ * experts by decreasing load on the least-loaded rank with a free slot (ties: lower expert
+ * id, lower rank id; exactly E/P experts per rank; slot = rank*(E/P) + arrival index), then
+ * computes q[i][l][p].
+ *   pi [L][E] int32 out, nullable: physical slot of logical expert e.
+ *   rank_load [L][P] int64 out, nullable: aggregate load G[l][p] under pi. */
+int rp_place_experts(rp_ctx *ctx, int32_t *pi, int64_t *rank_load);
+
+/* Row count and seed population (Section 3.2; Algorithm 2, first line and last loop).
+ * R_lb = max(1, min_rows, ceil(sum t / (C*D))); for R = R_lb, R_lb+1, ... first-fit-decreasing
+ * into R*D cells (the R*D longest samples open the cells, each later sample goes to the
+ * lowest-numbered cell it fits); the first R that packs is R*.  certified = 1 iff R* == R_lb
+ * (then it is the minimum).  Every population member starts as this layout.
+ *   n_rows, certified: HOST scalars out (nullable). */
+int rp_pack_rows(rp_ctx *ctx, int32_t *n_rows, int32_t *certified);
+
+/* Full evaluation of layouts (Section 3.4-3.5: Eqs. cell-token-statistics,
+ * stage-aware-attention, row-expert-load, row-expert-cost, lexicographic-score).
+ *   layouts [n][N] int32 cell ids, or NULL to score the current population (n = pop_size).
+ *   score_fx [n][3] int64 out, nullable; score_f64 [n][3] double out, nullable.
+ * Layouts with a cell id outside [0, R*D) give RP_ERR_ARG. */
+int rp_eval_population(rp_ctx *ctx, const int32_t *layouts, int32_t n, int64_t *score_fx,
+                       double *score_f64);
+
+/* Fixed-row population annealing (Algorithm 3): n_levels temperature levels; at each level
+ * every member runs steps_per_level guided swap/relocation proposals with incremental
+ * rescoring and the Metropolis rule, the incumbent takes any strictly better
+ * trajectory-best plan, and (except after the last level) the population is resampled
+ * systematically with Boltzmann weights.  May be called again to continue from the
+ * current population; level indices of the random streams restart at 0 on each call.
+ *   stats: HOST out, nullable. */
+int rp_anneal(rp_ctx *ctx, const rp_anneal_params *params, rp_anneal_stats *stats);
+
+/* Validate the incumbent (coverage, capacity, non-empty cells, cached score equals a full
+ * rescoring, not worse than the seed) and return it.
+ *   cell_of_sample [N] int32 out, nullable; score_fx [3], score_f64 [3] out, nullable. */
+int rp_best(rp_ctx *ctx, int32_t *cell_of_sample, int64_t *score_fx, double *score_f64);
+
+void rp_destroy(rp_ctx *ctx);
+const char *rp_strerror(int status);
+/* cudaError_t value of the last failed CUDA call on this thread (0 if none). */
+int rp_last_cuda_error(void);
+
+/* ---- inspection hooks (the paper has no counterpart; used by the parity tests) -------- */
+typedef enum {
+    RP_DUMP_LAGG = 1,        /* int64 [L][E]                                               */
+    RP_DUMP_Q = 2,           /* int32 [N][L][P]                                            */
+    RP_DUMP_SEED_LAYOUT = 3, /* int32 [N]                                                  */
+    RP_DUMP_POPULATION = 4,  /* int32 [P_pop][N]  current layouts                          */
+    RP_DUMP_W = 5,           /* int32 [R][G][L][P] of population member `index`            */
+    RP_DUMP_CELL_T = 6,      /* int64 [R*D] token sums of member `index` (recomputed)      */
+    RP_DUMP_CELL_Q = 7,      /* int64 [R*D] squared-length sums of member `index`          */
+    RP_DUMP_CELL_CNT = 8,    /* int32 [R*D]                                                */
+    RP_DUMP_ESUM = 9,        /* int64 [R][G]  sum_l max_p W of member `index`              */
+    RP_DUMP_TRACE_TERM = 10, /* int64 [n_levels][P_pop][3] terminal scores, last rp_anneal */
+    RP_DUMP_TRACE_BEST = 11, /* int64 [n_levels][P_pop][3] trajectory-best scores          */
+    RP_DUMP_TRACE_BEST_STEP = 12, /* int32 [n_levels][P_pop], 0 = level start              */
+    RP_DUMP_TRACE_DIGEST = 13,    /* uint64 [n_levels][P_pop] digest of accepted moves     */
+    RP_DUMP_TRACE_ANC = 14,       /* int32 [n_levels-1][P_pop] resampling ancestors        */
+    RP_DUMP_TRACE_INCUMBENT = 15, /* int64 [n_levels][3]                                   */
+    RP_DUMP_EVAL_W = 16      /* int32 [R][G][L][P] of layout `index` of the last
+                                rp_eval_population call with explicit layouts (n <= 64)    */
+} rp_dump_what;
+/* Copies the named array into buf (host or device); bytes must equal its size. */
+int rp_debug_dump(rp_ctx *ctx, int what, int32_t index, void *buf, int64_t bytes);
+/* Element-wise device evaluation of the integer functions used by the accept test and the
+ * resampling weights: out[i] = -log2((x[i]+1)/2^32) in Q32, and out[i] = 2^(-z[i]) in Q32.
+ * x, z, out: host or device arrays of n elements. */
+int rp_debug_nl2(const uint32_t *x, uint64_t *out, int64_t n);
+int rp_debug_exp2neg(const uint64_t *z, uint64_t *out, int64_t n);
+/* out[i][0..3] = Philox4x32-10(counter ctr[i][0..3], key) on the device. */
+int rp_debug_philox(const uint32_t *ctr, const uint32_t key[2], uint32_t *out, int64_t n);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ROUTEPACK_H_ */

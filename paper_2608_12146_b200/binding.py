@@ -1,0 +1,237 @@
+"""Thin ctypes binding of the C-ABI library (argument marshalling only).
+
+Function names and argument order follow ``include/routepack.h``.  Arrays may be numpy
+arrays (host memory) or torch tensors (host or CUDA); outputs are allocated here when the
+caller passes none.  Nothing in this module computes any step of the method: if the CUDA
+library cannot be loaded, every call raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence, Tuple
+
+import numpy as np
+
+from . import build as _build
+
+_lib = None
+
+STATUS_NAMES = {0: "RP_OK", -1: "RP_ERR_ARG", -2: "RP_ERR_SHAPE", -3: "RP_ERR_CONSERVATION",
+                -4: "RP_ERR_INFEASIBLE", -5: "RP_ERR_RANGE", -6: "RP_ERR_CUDA", -7: "RP_ERR_STATE",
+                -8: "RP_ERR_TIMEOUT", -9: "RP_ERR_INVALID_PLAN"}
+RP_OK = 0
+
+EXPORTS = ("rp_window_load", "rp_place_experts", "rp_pack_rows", "rp_eval_population", "rp_anneal",
+           "rp_best", "rp_destroy", "rp_strerror", "rp_last_cuda_error", "rp_debug_dump",
+           "rp_debug_nl2", "rp_debug_exp2neg", "rp_debug_philox")
+
+
+class RpError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().rp_strerror(status).decode()
+        extra = f" (cudaError {lib().rp_last_cuda_error()})" if status == -6 else ""
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)}: {msg}{extra}")
+
+
+class rp_config(C.Structure):
+    _fields_ = [("n_samples", C.c_int32), ("n_layers", C.c_int32), ("n_experts", C.c_int32),
+                ("top_k", C.c_int32), ("token_cap", C.c_int32), ("dp_width", C.c_int32),
+                ("ep_width", C.c_int32), ("edp_of_dp", C.c_void_p), ("n_stages", C.c_int32),
+                ("alpha", C.c_void_p), ("beta", C.c_void_p), ("pop_size", C.c_int32),
+                ("min_rows", C.c_int32), ("seed", C.c_uint64)]
+
+
+class rp_anneal_params(C.Structure):
+    _fields_ = [("n_levels", C.c_int32), ("steps_per_level", C.c_int32), ("t0", C.c_double),
+                ("t_ratio", C.c_double), ("p_reloc", C.c_double), ("p_guide", C.c_double)]
+
+
+class rp_anneal_stats(C.Structure):
+    _fields_ = [("proposed", C.c_int64), ("feasible", C.c_int64), ("accepted", C.c_int64),
+                ("improved", C.c_int64), ("ms_chains", C.c_double), ("ms_barrier", C.c_double)]
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def lib():
+    """Load the CUDA library; raises if it has not been built (there is no fallback)."""
+    global _lib
+    if _lib is None:
+        path = library_path()
+        if not os.path.exists(path):
+            raise RuntimeError(f"{path} is missing: run paper_2608_12146_b200.build.build() (needs nvcc)")
+        L = C.CDLL(path)
+        L.rp_strerror.restype = C.c_char_p
+        L.rp_strerror.argtypes = [C.c_int]
+        L.rp_last_cuda_error.restype = C.c_int
+        L.rp_destroy.restype = None
+        L.rp_destroy.argtypes = [C.c_void_p]
+        L.rp_window_load.argtypes = [C.POINTER(C.c_void_p), C.POINTER(rp_config), C.c_void_p, C.c_void_p, C.c_void_p]
+        L.rp_place_experts.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+        L.rp_pack_rows.argtypes = [C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+        L.rp_eval_population.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
+        L.rp_anneal.argtypes = [C.c_void_p, C.POINTER(rp_anneal_params), C.POINTER(rp_anneal_stats)]
+        L.rp_best.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.rp_debug_dump.argtypes = [C.c_void_p, C.c_int, C.c_int32, C.c_void_p, C.c_int64]
+        L.rp_debug_nl2.argtypes = [C.c_void_p, C.c_void_p, C.c_int64]
+        L.rp_debug_exp2neg.argtypes = [C.c_void_p, C.c_void_p, C.c_int64]
+        L.rp_debug_philox.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64]
+        _lib = L
+    return _lib
+
+
+def _ptr(a) -> Optional[int]:
+    """Address of a numpy array or torch tensor (host or device); None stays NULL."""
+    if a is None:
+        return None
+    if isinstance(a, np.ndarray):
+        if not a.flags["C_CONTIGUOUS"]:
+            raise ValueError("array must be C-contiguous")
+        return a.ctypes.data
+    if hasattr(a, "data_ptr"):
+        if not a.is_contiguous():
+            raise ValueError("tensor must be contiguous")
+        return a.data_ptr()
+    raise TypeError(f"unsupported array type {type(a)}")
+
+
+def _check(status: int, where: str):
+    if status != RP_OK:
+        raise RpError(status, where)
+
+
+def _stream_handle(stream) -> Optional[int]:
+    if stream is None:
+        return None
+    if isinstance(stream, int):
+        return stream
+    return int(stream.cuda_stream)           # torch.cuda.Stream
+
+
+class Context:
+    """Owner of one rp_ctx*; destroyed with close() or at garbage collection."""
+
+    def __init__(self, handle: int, cfg: rp_config, keep: tuple):
+        self.handle = C.c_void_p(handle)
+        self.cfg = cfg
+        self._keep = keep                    # input arrays adopted by the library must stay alive
+        self.n_rows = 0
+        self.n_shards = 0
+
+    def close(self):
+        if self.handle:
+            lib().rp_destroy(self.handle)
+            self.handle = C.c_void_p(None)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def rp_window_load(lengths, demand, *, top_k: int, token_cap: int, dp_width: int, ep_width: int,
+                   pop_size: int, edp_of_dp: Optional[Sequence[int]] = None,
+                   alpha: Sequence[float] = (1.0, 1.0), beta: Sequence[float] = (0.0, 1.0),
+                   min_rows: int = 0, seed: int = 0, stream=None) -> Context:
+    n, l, e = tuple(demand.shape)
+    al = np.ascontiguousarray(alpha, dtype=np.float64)
+    be = np.ascontiguousarray(beta, dtype=np.float64)
+    edp = None if edp_of_dp is None else np.ascontiguousarray(edp_of_dp, dtype=np.int32)
+    cfg = rp_config(n, l, e, top_k, token_cap, dp_width, ep_width, _ptr(edp), len(al), _ptr(al), _ptr(be),
+                    pop_size, min_rows, seed)
+    out = C.c_void_p(None)
+    st = lib().rp_window_load(C.byref(out), C.byref(cfg), _ptr(lengths), _ptr(demand), _stream_handle(stream))
+    _check(st, "rp_window_load")
+    ctx = Context(out.value, cfg, (lengths, demand, al, be, edp))
+    ctx.n_shards = dp_width if edp is None else int(edp.max()) + 1
+    return ctx
+
+
+def rp_place_experts(ctx: Context, pi=None, rank_load=None):
+    c = ctx.cfg
+    if pi is None:
+        pi = np.empty((c.n_layers, c.n_experts), np.int32)
+    if rank_load is None:
+        rank_load = np.empty((c.n_layers, c.ep_width), np.int64)
+    _check(lib().rp_place_experts(ctx.handle, _ptr(pi), _ptr(rank_load)), "rp_place_experts")
+    return pi, rank_load
+
+
+def rp_pack_rows(ctx: Context) -> Tuple[int, int]:
+    r, cert = C.c_int32(0), C.c_int32(0)
+    _check(lib().rp_pack_rows(ctx.handle, C.byref(r), C.byref(cert)), "rp_pack_rows")
+    ctx.n_rows = r.value
+    return r.value, cert.value
+
+
+def rp_eval_population(ctx: Context, layouts=None, score_fx=None, score_f64=None):
+    n = ctx.cfg.pop_size if layouts is None else int(layouts.shape[0])
+    if score_fx is None:
+        score_fx = np.empty((n, 3), np.int64)
+    if score_f64 is None:
+        score_f64 = np.empty((n, 3), np.float64)
+    _check(lib().rp_eval_population(ctx.handle, _ptr(layouts), n, _ptr(score_fx), _ptr(score_f64)),
+           "rp_eval_population")
+    return score_fx, score_f64
+
+
+def rp_anneal(ctx: Context, *, n_levels: int, steps_per_level: int, t0: float, t_ratio: float,
+              p_reloc: float, p_guide: float, want_stats: bool = True) -> Optional[rp_anneal_stats]:
+    prm = rp_anneal_params(n_levels, steps_per_level, t0, t_ratio, p_reloc, p_guide)
+    stats = rp_anneal_stats() if want_stats else None
+    _check(lib().rp_anneal(ctx.handle, C.byref(prm), C.byref(stats) if want_stats else None), "rp_anneal")
+    return stats
+
+
+def rp_best(ctx: Context, cell_of_sample=None, score_fx=None, score_f64=None):
+    if cell_of_sample is None:
+        cell_of_sample = np.empty(ctx.cfg.n_samples, np.int32)
+    if score_fx is None:
+        score_fx = np.empty(3, np.int64)
+    if score_f64 is None:
+        score_f64 = np.empty(3, np.float64)
+    _check(lib().rp_best(ctx.handle, _ptr(cell_of_sample), _ptr(score_fx), _ptr(score_f64)), "rp_best")
+    return cell_of_sample, score_fx, score_f64
+
+
+def rp_destroy(ctx: Context):
+    ctx.close()
+
+
+# ---- inspection hooks -------------------------------------------------------------------
+DUMP = dict(LAGG=1, Q=2, SEED_LAYOUT=3, POPULATION=4, W=5, CELL_T=6, CELL_Q=7, CELL_CNT=8, ESUM=9,
+            TRACE_TERM=10, TRACE_BEST=11, TRACE_BEST_STEP=12, TRACE_DIGEST=13, TRACE_ANC=14,
+            TRACE_INCUMBENT=15, EVAL_W=16)
+
+
+def rp_debug_dump(ctx: Context, what: str, shape, dtype, index: int = 0) -> np.ndarray:
+    out = np.empty(shape, dtype)
+    _check(lib().rp_debug_dump(ctx.handle, DUMP[what], index, _ptr(out), out.nbytes), f"rp_debug_dump({what})")
+    return out
+
+
+def rp_debug_nl2(x) -> np.ndarray:
+    x = np.ascontiguousarray(x, np.uint32)
+    out = np.empty(x.shape, np.uint64)
+    _check(lib().rp_debug_nl2(_ptr(x), _ptr(out), x.size), "rp_debug_nl2")
+    return out
+
+
+def rp_debug_exp2neg(z) -> np.ndarray:
+    z = np.ascontiguousarray(z, np.uint64)
+    out = np.empty(z.shape, np.uint64)
+    _check(lib().rp_debug_exp2neg(_ptr(z), _ptr(out), z.size), "rp_debug_exp2neg")
+    return out
+
+
+def rp_debug_philox(ctr, key) -> np.ndarray:
+    ctr = np.ascontiguousarray(ctr, np.uint32)
+    key = np.ascontiguousarray(key, np.uint32)
+    out = np.empty(ctr.shape, np.uint32)
+    _check(lib().rp_debug_philox(_ptr(ctr), _ptr(key), _ptr(out), ctr.shape[0]), "rp_debug_philox")
+    return out

@@ -1,0 +1,618 @@
+// Fixed-row population annealing (Algorithm 3 of the paper): the per-level chain kernel
+// (K5: GuidedProposal, feasibility, IncrementalScore, Metropolis), the level barrier
+// (K6 incumbent update + K7 Boltzmann weights and systematic resampling) and the final
+// validation (K8).
+//
+// Mapping.  One CTA runs one chain for all K steps of a level.  The chain's small state
+// (assignment, cell statistics, per-row-shard costs, shard work) lives in shared memory;
+// its rank-load tensor W[R][G][L][P] lives in global memory (L2/HBM) and is touched two
+// slices per feasible move.  The sample demand rows q[i][L][P] are shared by all chains and
+// stay L2-resident.  Resampling is folded into the next level's prologue: slot j starts
+// from the terminal state of its ancestor in the other population buffer, so no separate
+// gather pass runs.  Trajectory-best layouts are not copied: every accepted move is logged
+// (8 bytes) and the level barrier rebuilds the one winning layout from the chain's start
+// layout and its log prefix.
+//
+// Algorithmic bytes per feasible move: reads 2 W slices + the moved samples' q rows
+// ((3 or 4) * L*P*4 bytes), writes 2 W slices when accepted.
+#include "rp_score.cuh"
+
+struct AnnealArgs {
+    RpDims dm;
+    const int *t, *q, *edp, *dp_list, *dp_off;
+    const unsigned short *cell_src;  unsigned short *cell_dst;
+    const int *W_src;                int *W_dst;
+    const i64 *Esum_src;             i64 *Esum_dst;
+    const int *anc;
+    int level, steps, t_in_smem, log_cap;
+    u64 tau, rho_q32, guide_q32;
+    u32 key0, key1;
+    i64 *term, *best;
+    int *best_step, *best_nlog;
+    u64 *digest;
+    uint2 *log;
+    i64 *counters;
+};
+
+struct MoveRec {
+    int feasible, reloc, i, i2, c1, c2, rg1, rg2, accept;
+};
+
+template <int NT>
+__device__ __forceinline__ void block_sync()
+{
+    if (NT == 32) __syncwarp(); else __syncthreads();
+}
+
+template <int NT>
+__global__ void __launch_bounds__(NT)
+k_anneal_level(const AnnealArgs A)
+{
+    const RpDims &dm = A.dm;
+    extern __shared__ __align__(16) unsigned char smraw[];
+    // Q[K] | Esum[RG] | Afx[RG] | Jfx[RG] | U[G] | red[2*NT/32] | T[K] | cnt[K] | scratch[2*LP] | t_s[N]? | cell_of[N] | mv
+    u64 *Q = (u64 *)smraw;
+    i64 *Esum = (i64 *)(Q + dm.K);
+    i64 *Afx = Esum + dm.RG;
+    i64 *Jfx = Afx + dm.RG;
+    i64 *U = Jfx + dm.RG;
+    i64 *red = U + dm.G;
+    int *T = (int *)(red + 2 * (NT / 32));
+    int *cnt = T + dm.K;
+    int *scratch = cnt + dm.K;
+    int *t_s = scratch + 2 * dm.LP;
+    unsigned short *cell_of = (unsigned short *)(t_s + (A.t_in_smem ? dm.N : 0));
+    MoveRec *mv = (MoveRec *)(((uintptr_t)(cell_of + dm.N) + 15) & ~(uintptr_t)15);
+    RpSmemState st = { cell_of, T, Q, cnt, Esum, Afx, U };
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int j = blockIdx.x;
+    const int src = A.anc[j];
+    const int *tt = A.t_in_smem ? t_s : A.t;
+
+    // ---- prologue: adopt the ancestor's terminal state -------------------------------
+    {
+        const unsigned short *cs = A.cell_src + (size_t)src * dm.N;
+        for (int i = tid; i < dm.N; i += NT) cell_of[i] = cs[i];
+        if (A.t_in_smem) for (int i = tid; i < dm.N; i += NT) t_s[i] = A.t[i];
+        for (int c = tid; c < dm.K; c += NT) { T[c] = 0; Q[c] = 0; cnt[c] = 0; }
+        const i64 *es = A.Esum_src + (size_t)src * dm.RG;
+        for (int rg = tid; rg < dm.RG; rg += NT) Esum[rg] = es[rg];
+        const size_t wn = (size_t)dm.RG * dm.LP;
+        const int *ws = A.W_src + (size_t)src * wn;
+        int *wd = A.W_dst + (size_t)j * wn;
+        if ((wn & 3) == 0) {
+            const int4 *ws4 = (const int4 *)ws;
+            int4 *wd4 = (int4 *)wd;
+            for (size_t x = tid; x < wn / 4; x += NT) wd4[x] = ws4[x];
+        } else {
+            for (size_t x = tid; x < wn; x += NT) wd[x] = ws[x];
+        }
+    }
+    __syncthreads();
+    rp_accumulate_cells(dm, st, A.t, tid, NT);
+    __syncthreads();
+    i64 S[3];
+    rp_rows_to_score(dm, st, A.dp_list, A.dp_off, tid, NT, S);
+    for (int rg = tid; rg < dm.RG; rg += NT) Jfx[rg] = Afx[rg] + dm.EC * Esum[rg];
+    __syncthreads();
+
+    int *Wj = A.W_dst + (size_t)j * dm.RG * dm.LP;
+    // chain bookkeeping (thread 0 only)
+    i64 B0 = S[0], B1 = S[1], B2 = S[2];
+    int best_step = 0, best_nlog = 0, nlog = 0;
+    u64 dig = 0;
+    i64 n_feas = 0, n_acc = 0, n_imp = 0;
+    uint2 *logj = A.log + (size_t)j * A.log_cap;
+
+    for (int k = 0; k < A.steps; ++k) {
+        // ---- phase 1: proposal and feasibility (thread 0) -----------------------------
+        if (tid == 0) {
+            const uint4 a = rp_philox((u32)k, (u32)A.level, (u32)j, 0u, A.key0, A.key1);
+            const bool reloc = (u64)a.x < A.rho_q32;
+            const bool guided = (u64)a.y < A.guide_q32;
+            int i, i2 = -1, c1, c2;
+            if (!guided) {
+                i = rp_pick(a.z, dm.N);
+                c1 = cell_of[i];
+                if (reloc) c2 = rp_pick(a.w, dm.K);
+                else { i2 = rp_pick(a.w, dm.N); c2 = cell_of[i2]; }
+            } else {
+                const uint4 b = rp_philox((u32)k, (u32)A.level, (u32)j, 1u, A.key0, A.key1);
+                const int sa = rp_pick(a.z, dm.N), sb = rp_pick(a.w, dm.N);
+                const int ca = cell_of[sa], cb = cell_of[sb];
+                const int rga = rp_rowshard(dm, A.edp, ca);
+                const u64 Ja = (u64)Jfx[rga], Aa = (u64)Afx[rga];
+                // attention key with probability Afx/Jfx:  b.z * Ja < Aa * 2^32  (128-bit compare)
+                const u64 lh = __umul64hi((u64)b.z, Ja), ll = (u64)b.z * Ja;
+                const u64 rh = Aa >> 32, rl = Aa << 32;
+                const bool use_att = (lh < rh) || (lh == rh && ll < rl);
+                i64 ka, kb;
+                if (use_att) {
+                    ka = dm.asum * dm.C * (i64)T[ca] + dm.bsum * (i64)Q[ca];
+                    kb = dm.asum * dm.C * (i64)T[cb] + dm.bsum * (i64)Q[cb];
+                } else {
+                    ka = (i64)Ja;
+                    kb = Jfx[rp_rowshard(dm, A.edp, cb)];
+                }
+                i = (kb > ka) ? sb : sa;
+                c1 = (kb > ka) ? cb : ca;
+                if (reloc) {
+                    const int xa = rp_pick(b.x, dm.K), xb = rp_pick(b.y, dm.K);
+                    i64 ta, tb;
+                    if (use_att) {
+                        ta = dm.asum * dm.C * (i64)T[xa] + dm.bsum * (i64)Q[xa];
+                        tb = dm.asum * dm.C * (i64)T[xb] + dm.bsum * (i64)Q[xb];
+                    } else {
+                        ta = Jfx[rp_rowshard(dm, A.edp, xa)];
+                        tb = Jfx[rp_rowshard(dm, A.edp, xb)];
+                    }
+                    c2 = (tb < ta) ? xb : xa;
+                } else {
+                    const int ya = rp_pick(b.x, dm.N), yb = rp_pick(b.y, dm.N);
+                    const int xa = cell_of[ya], xb = cell_of[yb];
+                    i64 ta, tb;
+                    if (use_att) {
+                        ta = dm.asum * dm.C * (i64)T[xa] + dm.bsum * (i64)Q[xa];
+                        tb = dm.asum * dm.C * (i64)T[xb] + dm.bsum * (i64)Q[xb];
+                    } else {
+                        ta = Jfx[rp_rowshard(dm, A.edp, xa)];
+                        tb = Jfx[rp_rowshard(dm, A.edp, xb)];
+                    }
+                    i2 = (tb < ta) ? yb : ya;
+                    c2 = (tb < ta) ? xb : xa;
+                }
+            }
+            bool ok = (c1 != c2);
+            if (ok) {
+                const int ti = tt[i];
+                if (reloc) ok = (cnt[c1] > 1) && (T[c2] + ti <= dm.C);
+                else {
+                    const int t2 = tt[i2];
+                    ok = (T[c1] - ti + t2 <= dm.C) && (T[c2] - t2 + ti <= dm.C);
+                }
+            }
+            mv->feasible = ok; mv->reloc = reloc; mv->i = i; mv->i2 = i2; mv->c1 = c1; mv->c2 = c2;
+            if (ok) {
+                mv->rg1 = rp_rowshard(dm, A.edp, c1);
+                mv->rg2 = rp_rowshard(dm, A.edp, c2);
+            }
+        }
+        block_sync<NT>();
+        if (!mv->feasible) { block_sync<NT>(); continue; }
+        const int mi = mv->i, mi2 = mv->i2, rg1 = mv->rg1, rg2 = mv->rg2;
+        const bool swap = !mv->reloc;
+        const bool touchW = (rg1 != rg2);
+
+        // ---- phase 2: tentative rank loads of the two row-shards and their layer maxima ----
+        i64 e1 = 0, e2 = 0;
+        if (touchW) {
+            const int *qi = A.q + (size_t)mi * dm.LP;
+            const int *q2 = swap ? A.q + (size_t)mi2 * dm.LP : nullptr;
+            const int *w1 = Wj + (size_t)rg1 * dm.LP, *w2 = Wj + (size_t)rg2 * dm.LP;
+            const int P = dm.P, LP = dm.LP;
+            if (P <= 32 && (P & (P - 1)) == 0) {
+                for (int x0 = 0; x0 < LP; x0 += NT) {
+                    const int x = x0 + tid;
+                    int v1 = 0, v2 = 0;
+                    if (x < LP) {
+                        int d = __ldg(qi + x);
+                        if (swap) d -= __ldg(q2 + x);
+                        v1 = w1[x] - d;
+                        v2 = w2[x] + d;
+                        scratch[x] = v1;
+                        scratch[LP + x] = v2;
+                    }
+                    for (int o = P >> 1; o; o >>= 1) {
+                        v1 = max(v1, __shfl_xor_sync(0xffffffffu, v1, o));
+                        v2 = max(v2, __shfl_xor_sync(0xffffffffu, v2, o));
+                    }
+                    if ((lane & (P - 1)) == 0 && x < LP) { e1 += v1; e2 += v2; }
+                }
+            } else {
+                for (int x = tid; x < LP; x += NT) {
+                    int d = __ldg(qi + x);
+                    if (swap) d -= __ldg(q2 + x);
+                    scratch[x] = w1[x] - d;
+                    scratch[LP + x] = w2[x] + d;
+                }
+                block_sync<NT>();
+                for (int l = warp; l < dm.L; l += NT / 32) {
+                    int v1 = 0, v2 = 0;
+                    for (int p = lane; p < P; p += 32) {
+                        v1 = max(v1, scratch[l * P + p]);
+                        v2 = max(v2, scratch[LP + l * P + p]);
+                    }
+                    for (int o = 16; o; o >>= 1) {
+                        v1 = max(v1, __shfl_xor_sync(0xffffffffu, v1, o));
+                        v2 = max(v2, __shfl_xor_sync(0xffffffffu, v2, o));
+                    }
+                    if (lane == 0) { e1 += v1; e2 += v2; }
+                }
+            }
+            for (int o = 16; o; o >>= 1) {
+                e1 += __shfl_xor_sync(0xffffffffu, e1, o);
+                e2 += __shfl_xor_sync(0xffffffffu, e2, o);
+            }
+            if (NT > 32) {
+                if (lane == 0) { red[2 * warp] = e1; red[2 * warp + 1] = e2; }
+                __syncthreads();
+                if (tid == 0) {
+                    e1 = 0; e2 = 0;
+                    for (int w = 0; w < NT / 32; ++w) { e1 += red[2 * w]; e2 += red[2 * w + 1]; }
+                }
+            }
+        }
+
+        // ---- phase 3: exact new score, Metropolis, commit of the scalar state (thread 0) ----
+        if (tid == 0) {
+            const int c1 = mv->c1, c2 = mv->c2;
+            const i64 ti = tt[mi], t2 = swap ? tt[mi2] : 0;
+            const i64 Ta = (i64)T[c1] - ti + t2, Qa = (i64)Q[c1] - ti * ti + t2 * t2;
+            const i64 Tb = (i64)T[c2] + ti - t2, Qb = (i64)Q[c2] + ti * ti - t2 * t2;
+            const int r1 = c1 / dm.D, g1 = A.edp[c1 % dm.D], r2 = c2 / dm.D, g2 = A.edp[c2 % dm.D];
+            if (!touchW) { e1 = Esum[rg1]; e2 = e1; }
+            const i64 A1 = rp_attention(dm, st, A.dp_list, A.dp_off, r1, g1, c1, Ta, Qa, c2, Tb, Qb);
+            const i64 A2 = touchW ? rp_attention(dm, st, A.dp_list, A.dp_off, r2, g2, c1, Ta, Qa, c2, Tb, Qb) : A1;
+            const i64 J1o = Jfx[rg1], J2o = Jfx[rg2];
+            const i64 J1n = A1 + dm.EC * e1, J2n = touchW ? A2 + dm.EC * e2 : J1n;
+            const i64 dJ1 = J1n - J1o, dJ2 = touchW ? J2n - J2o : 0;
+            const i64 U1o = U[g1], U2o = U[g2];
+            i64 U1n, U2n;
+            if (g1 == g2) { U1n = U1o + dJ1 + dJ2; U2n = U1n; }
+            else { U1n = U1o + dJ1; U2n = U2o + dJ2; }
+            const i64 n1 = S[1] + dJ1 + dJ2;
+            // s0 = max_g U: only U[g1], U[g2] changed
+            i64 n0;
+            {
+                const i64 newmax = U1n > U2n ? U1n : U2n, oldmax = U1o > U2o ? U1o : U2o;
+                if (newmax >= S[0]) n0 = newmax;
+                else if (oldmax < S[0]) n0 = S[0];
+                else {
+                    n0 = newmax;
+                    for (int g = 0; g < dm.G; ++g) if (g != g1 && g != g2 && U[g] > n0) n0 = U[g];
+                }
+            }
+            // s2 = max_{r,g} J: only J[rg1], J[rg2] changed
+            i64 n2;
+            {
+                const i64 newmax = J1n > J2n ? J1n : J2n, oldmax = J1o > J2o ? J1o : J2o;
+                if (newmax >= S[2]) n2 = newmax;
+                else if (oldmax < S[2]) n2 = S[2];
+                else {
+                    n2 = newmax;
+                    for (int rg = 0; rg < dm.RG; ++rg) if (rg != rg1 && rg != rg2 && Jfx[rg] > n2) n2 = Jfx[rg];
+                }
+            }
+            bool acc = rp_lex_less(n0, n1, n2, S[0], S[1], S[2]);
+            if (!acc) {
+                const i64 eo = rp_energy(S[0], S[1], S[2]), en = rp_energy(n0, n1, n2);
+                if (en <= eo) acc = true;
+                else {
+                    const uint4 xw = rp_philox((u32)k, (u32)A.level, (u32)j, 2u, A.key0, A.key1);
+                    acc = rp_accept_uphill(eo, en - eo, dm.SC, A.tau, xw.x);
+                }
+            }
+            ++n_feas;
+            if (acc) {
+                ++n_acc;
+                cell_of[mi] = (unsigned short)c2;
+                if (swap) cell_of[mi2] = (unsigned short)c1;
+                T[c1] = (int)Ta; Q[c1] = (u64)Qa; T[c2] = (int)Tb; Q[c2] = (u64)Qb;
+                if (!swap) { cnt[c1] -= 1; cnt[c2] += 1; }
+                Esum[rg1] = e1; Afx[rg1] = A1; Jfx[rg1] = J1n;
+                if (touchW) { Esum[rg2] = e2; Afx[rg2] = A2; Jfx[rg2] = J2n; }
+                U[g1] = U1n; U[g2] = U2n;
+                S[0] = n0; S[1] = n1; S[2] = n2;
+                const u32 second = swap ? (u32)mi2 : (u32)c2;
+                if (nlog < A.log_cap) logj[nlog] = make_uint2((u32)mi, second | (swap ? 0u : 0x80000000u));
+                ++nlog;
+                const u64 code = ((u64)(swap ? 0 : 1) << 63) ^ ((u64)(u32)k << 40) ^ ((u64)(u32)mi << 20) ^ (u64)second;
+                dig = (dig ^ code) * 0x100000001B3ull;
+                if (rp_lex_less(n0, n1, n2, B0, B1, B2)) {
+                    B0 = n0; B1 = n1; B2 = n2;
+                    best_step = k + 1; best_nlog = nlog;
+                    ++n_imp;
+                }
+            }
+            mv->accept = acc;
+        }
+        block_sync<NT>();
+        // ---- phase 4: commit the two W slices ---------------------------------------------
+        if (mv->accept && touchW) {
+            int *w1 = Wj + (size_t)rg1 * dm.LP, *w2 = Wj + (size_t)rg2 * dm.LP;
+            for (int x = tid; x < dm.LP; x += NT) { w1[x] = scratch[x]; w2[x] = scratch[dm.LP + x]; }
+        }
+        block_sync<NT>();
+    }
+
+    // ---- epilogue: terminal state and chain report ------------------------------------------
+    {
+        unsigned short *cd = A.cell_dst + (size_t)j * dm.N;
+        for (int i = tid; i < dm.N; i += NT) cd[i] = cell_of[i];
+        i64 *ed = A.Esum_dst + (size_t)j * dm.RG;
+        for (int rg = tid; rg < dm.RG; rg += NT) ed[rg] = Esum[rg];
+        if (tid == 0) {
+            A.term[3 * (size_t)j + 0] = S[0]; A.term[3 * (size_t)j + 1] = S[1]; A.term[3 * (size_t)j + 2] = S[2];
+            A.best[3 * (size_t)j + 0] = B0; A.best[3 * (size_t)j + 1] = B1; A.best[3 * (size_t)j + 2] = B2;
+            A.best_step[j] = best_step;
+            A.best_nlog[j] = best_nlog;
+            A.digest[j] = dig;
+            atomicAdd((u64 *)&A.counters[0], (u64)A.steps);
+            atomicAdd((u64 *)&A.counters[1], (u64)n_feas);
+            atomicAdd((u64 *)&A.counters[2], (u64)n_acc);
+            atomicAdd((u64 *)&A.counters[3], (u64)n_imp);
+        }
+    }
+}
+
+static int anneal_threads(const RpDims &dm)
+{
+    if (dm.LP <= 128) return 32;
+    if (dm.LP <= 512) return 128;
+    return 256;
+}
+
+int rp_anneal_smem_bytes(const rp_ctx *c, int *threads, size_t *bytes)
+{
+    const RpDims &dm = c->dm;
+    int nt = anneal_threads(dm);
+    int t_in_smem = dm.N <= 2048;
+    size_t b = sizeof(u64) * dm.K + sizeof(i64) * (3 * (size_t)dm.RG + dm.G + 2 * (nt / 32));
+    b += sizeof(int) * (2 * (size_t)dm.K + 2 * (size_t)dm.LP + (t_in_smem ? dm.N : 0));
+    b += sizeof(unsigned short) * dm.N;
+    b = (b + 15) & ~(size_t)15;
+    b += sizeof(MoveRec) + 16;
+    *threads = nt;
+    *bytes = b;
+    return t_in_smem;
+}
+
+int rp_launch_anneal_level(rp_ctx *c, int level, const rp_anneal_params *prm, u64 rho_q32, u64 guide_q32)
+{
+    AnnealArgs A;
+    A.dm = c->dm;
+    A.t = c->d_t; A.q = c->d_q; A.edp = c->d_edp; A.dp_list = c->d_dp_list; A.dp_off = c->d_dp_off;
+    const RpPopBuf &s = c->buf[c->cur], &d = c->buf[1 - c->cur];
+    A.cell_src = s.cell_of; A.cell_dst = d.cell_of;
+    A.W_src = s.W; A.W_dst = d.W;
+    A.Esum_src = s.Esum; A.Esum_dst = d.Esum;
+    A.anc = c->d_anc;
+    A.level = level; A.steps = prm->steps_per_level; A.log_cap = c->log_cap;
+    int nt; size_t smem;
+    A.t_in_smem = rp_anneal_smem_bytes(c, &nt, &smem);
+    if (smem > 220 * 1024) return RP_ERR_RANGE;
+    A.rho_q32 = rho_q32; A.guide_q32 = guide_q32;
+    A.key0 = (u32)c->cfg.seed; A.key1 = (u32)(c->cfg.seed >> 32);
+    A.term = c->d_term; A.best = c->d_best; A.best_step = c->d_best_step; A.best_nlog = c->d_best_nlog;
+    A.digest = c->d_digest; A.log = c->d_log; A.counters = c->d_counters;
+    A.tau = c->h_levels[level].tau;
+#define LAUNCH(NT_)                                                                                   \
+    do {                                                                                              \
+        if (smem > 48 * 1024)                                                                         \
+            RP_CUDA(cudaFuncSetAttribute(k_anneal_level<NT_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+        k_anneal_level<NT_><<<c->Ppop, NT_, smem, c->stream>>>(A);                                    \
+    } while (0)
+    if (nt == 32) LAUNCH(32);
+    else if (nt == 128) LAUNCH(128);
+    else LAUNCH(256);
+#undef LAUNCH
+    RP_CUDA(cudaGetLastError());
+    return RP_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Level barrier: incumbent update (strictly better trajectory-best, lowest slot on ties) and,
+// unless this was the last level, Boltzmann weights + systematic resampling -> ancestors.
+// One CTA; the population has at most a few tens of thousands of members.
+// ---------------------------------------------------------------------------------------------
+#define LE_THREADS 1024
+
+struct LevelEndArgs {
+    RpDims dm;
+    int Ppop, level, last, log_cap;
+    u64 cq;
+    u32 key0, key1;
+    const i64 *term, *best;
+    const int *best_step, *best_nlog;
+    const u64 *digest;
+    const uint2 *log;
+    const unsigned short *cell_src;   // layouts the level started from (indexed through anc)
+    int *anc;
+    u64 *F;
+    int *inc_layout;
+    i64 *inc_score;
+    // trace (nullable)
+    i64 *tr_term, *tr_best, *tr_inc;
+    int *tr_best_step, *tr_anc;
+    u64 *tr_digest;
+};
+
+__global__ void __launch_bounds__(LE_THREADS)
+k_level_end(const LevelEndArgs A)
+{
+    __shared__ i64 r0[LE_THREADS / 32], r1[LE_THREADS / 32], r2[LE_THREADS / 32];
+    __shared__ int rj[LE_THREADS / 32];
+    __shared__ u64 rsum[LE_THREADS / 32];
+    __shared__ int win_j, do_update;
+    __shared__ i64 Emin_s;
+    __shared__ u64 carry_s;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int P = A.Ppop;
+
+    // trace copies of the per-chain reports
+    if (A.tr_term) {
+        const size_t o = (size_t)A.level * P;
+        for (int x = tid; x < 3 * P; x += LE_THREADS) { A.tr_term[o * 3 + x] = A.term[x]; A.tr_best[o * 3 + x] = A.best[x]; }
+        for (int x = tid; x < P; x += LE_THREADS) { A.tr_best_step[o + x] = A.best_step[x]; A.tr_digest[o + x] = A.digest[x]; }
+    }
+
+    // ---- incumbent: lexicographic argmin of the trajectory-best scores, lowest slot first ----
+    i64 b0 = 0x7fffffffffffffffll, b1 = b0, b2 = b0;
+    int bj = 0x7fffffff;
+    for (int j = tid; j < P; j += LE_THREADS) {
+        i64 s0 = A.best[3 * (size_t)j], s1 = A.best[3 * (size_t)j + 1], s2 = A.best[3 * (size_t)j + 2];
+        if (rp_lex_less(s0, s1, s2, b0, b1, b2)) { b0 = s0; b1 = s1; b2 = s2; bj = j; }   // ascending j: first wins
+    }
+    for (int o = 16; o; o >>= 1) {
+        i64 o0 = __shfl_xor_sync(0xffffffffu, b0, o), o1 = __shfl_xor_sync(0xffffffffu, b1, o);
+        i64 o2 = __shfl_xor_sync(0xffffffffu, b2, o);
+        int oj = __shfl_xor_sync(0xffffffffu, bj, o);
+        bool take = rp_lex_less(o0, o1, o2, b0, b1, b2) || (o0 == b0 && o1 == b1 && o2 == b2 && oj < bj);
+        if (take) { b0 = o0; b1 = o1; b2 = o2; bj = oj; }
+    }
+    if (lane == 0) { r0[warp] = b0; r1[warp] = b1; r2[warp] = b2; rj[warp] = bj; }
+    __syncthreads();
+    if (tid == 0) {
+        for (int w = 1; w < LE_THREADS / 32; ++w) {
+            bool take = rp_lex_less(r0[w], r1[w], r2[w], b0, b1, b2) ||
+                        (r0[w] == b0 && r1[w] == b1 && r2[w] == b2 && rj[w] < bj);
+            if (take) { b0 = r0[w]; b1 = r1[w]; b2 = r2[w]; bj = rj[w]; }
+        }
+        win_j = bj;
+        do_update = rp_lex_less(b0, b1, b2, A.inc_score[0], A.inc_score[1], A.inc_score[2]);
+        if (do_update) { A.inc_score[0] = b0; A.inc_score[1] = b1; A.inc_score[2] = b2; }
+    }
+    __syncthreads();
+    if (do_update) {
+        const int w = win_j;
+        const unsigned short *cs = A.cell_src + (size_t)A.anc[w] * A.dm.N;
+        for (int i = tid; i < A.dm.N; i += LE_THREADS) A.inc_layout[i] = cs[i];
+        __syncthreads();
+        if (tid == 0) {      // replay the accepted moves up to the trajectory-best step
+            const uint2 *lg = A.log + (size_t)w * A.log_cap;
+            const int n = A.best_nlog[w];
+            for (int x = 0; x < n; ++x) {
+                const uint2 m = lg[x];
+                const int i = (int)m.x;
+                if (m.y & 0x80000000u) A.inc_layout[i] = (int)(m.y & 0x7fffffffu);
+                else {
+                    const int i2 = (int)m.y;
+                    const int c = A.inc_layout[i];
+                    A.inc_layout[i] = A.inc_layout[i2];
+                    A.inc_layout[i2] = c;
+                }
+            }
+        }
+    }
+    __syncthreads();
+    if (A.tr_inc && tid < 3) A.tr_inc[(size_t)A.level * 3 + tid] = A.inc_score[tid];
+
+    if (A.last) {            // the terminal states are the population as they stand
+        for (int m = tid; m < P; m += LE_THREADS) A.anc[m] = m;
+        return;
+    }
+
+    // ---- resampling -------------------------------------------------------------------------
+    i64 emin = 0x7fffffffffffffffll;
+    for (int j = tid; j < P; j += LE_THREADS) {
+        i64 e = rp_energy(A.term[3 * (size_t)j], A.term[3 * (size_t)j + 1], A.term[3 * (size_t)j + 2]);
+        emin = e < emin ? e : emin;
+    }
+    for (int o = 16; o; o >>= 1) { i64 x = __shfl_xor_sync(0xffffffffu, emin, o); emin = x < emin ? x : emin; }
+    if (lane == 0) r0[warp] = emin;
+    __syncthreads();
+    if (tid == 0) {
+        for (int w = 1; w < LE_THREADS / 32; ++w) emin = r0[w] < emin ? r0[w] : emin;
+        Emin_s = emin;
+        carry_s = 0;
+    }
+    __syncthreads();
+    emin = Emin_s;
+    const u64 M = (u64)(emin > A.dm.SC ? emin : A.dm.SC);
+    // inclusive prefix sums of the weights, 1024 members per round
+    for (int base = 0; base < P; base += LE_THREADS) {
+        const int j = base + tid;
+        u64 w = 0;
+        if (j < P) {
+            const i64 e = rp_energy(A.term[3 * (size_t)j], A.term[3 * (size_t)j + 1], A.term[3 * (size_t)j + 2]);
+            unsigned __int128 eq = ((unsigned __int128)(u64)(e - emin) << 32) / (unsigned __int128)M;
+            const unsigned __int128 cap = (((unsigned __int128)1) << 48) - 1;
+            if (eq > cap) eq = cap;
+            unsigned __int128 z = (eq * (unsigned __int128)A.cq) >> 16;
+            const unsigned __int128 zcap = ((unsigned __int128)1) << 40;
+            if (z > zcap) z = zcap;
+            w = rp_exp2neg((u64)z);
+        }
+        u64 v = w;
+        for (int o = 1; o < 32; o <<= 1) { u64 x = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += x; }
+        if (lane == 31) rsum[warp] = v;
+        __syncthreads();
+        if (warp == 0) {
+            u64 s = rsum[lane];
+            for (int o = 1; o < 32; o <<= 1) { u64 x = __shfl_up_sync(0xffffffffu, s, o); if (lane >= o) s += x; }
+            rsum[lane] = s;
+        }
+        __syncthreads();
+        const u64 before = carry_s + (warp ? rsum[warp - 1] : 0);
+        if (j < P) A.F[j] = before + v;
+        __syncthreads();
+        if (tid == LE_THREADS - 1) carry_s = before + v;
+        __syncthreads();
+    }
+    const u64 Ftot = A.F[P - 1];
+    const uint4 xw = rp_philox(0u, (u32)A.level, 0u, 3u, A.key0, A.key1);
+    const u64 u0 = (u64)(((unsigned __int128)xw.x * Ftot) >> 32);
+    for (int m = tid; m < P; m += LE_THREADS) {
+        const unsigned __int128 pos = (unsigned __int128)u0 + (unsigned __int128)m * Ftot;
+        int lo = 0, hi = P - 1;                 // smallest j with P*F[j] > pos
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if ((unsigned __int128)P * A.F[mid] > pos) hi = mid; else lo = mid + 1;
+        }
+        A.anc[m] = lo;
+        if (A.tr_anc) A.tr_anc[(size_t)A.level * P + m] = lo;
+    }
+}
+
+int rp_launch_level_end(rp_ctx *c, int level, int n_levels)
+{
+    LevelEndArgs A;
+    A.dm = c->dm; A.Ppop = c->Ppop; A.level = level; A.last = (level == n_levels - 1); A.log_cap = c->log_cap;
+    A.cq = c->h_levels[level].cq;
+    A.key0 = (u32)c->cfg.seed; A.key1 = (u32)(c->cfg.seed >> 32);
+    A.term = c->d_term; A.best = c->d_best; A.best_step = c->d_best_step; A.best_nlog = c->d_best_nlog;
+    A.digest = c->d_digest; A.log = c->d_log;
+    A.cell_src = c->buf[c->cur].cell_of;
+    A.anc = c->d_anc; A.F = c->d_F;
+    A.inc_layout = c->d_inc_layout; A.inc_score = c->d_inc_score;
+    A.tr_term = c->d_tr_term; A.tr_best = c->d_tr_best; A.tr_inc = c->d_tr_inc;
+    A.tr_best_step = c->d_tr_best_step; A.tr_anc = c->d_tr_anc; A.tr_digest = c->d_tr_digest;
+    k_level_end<<<1, LE_THREADS, 0, c->stream>>>(A);
+    RP_CUDA(cudaGetLastError());
+    return RP_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Validate(x*): every sample in a real cell, no empty cell, no cell over the token cap.
+// (Score consistency and non-regression are checked by the caller from a full rescoring.)
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024)
+k_validate(const int *__restrict__ layout, const int *__restrict__ t, RpDims dm, int *__restrict__ fill,
+           int *__restrict__ cnt, int *__restrict__ status)
+{
+    const int tid = threadIdx.x;
+    for (int c = tid; c < dm.K; c += 1024) { fill[c] = 0; cnt[c] = 0; }
+    __syncthreads();
+    int bad = 0;
+    for (int i = tid; i < dm.N; i += 1024) {
+        int c = layout[i];
+        if (c < 0 || c >= dm.K) { bad |= 1; continue; }
+        atomicAdd(&fill[c], t[i]);
+        atomicAdd(&cnt[c], 1);
+    }
+    __syncthreads();
+    for (int c = tid; c < dm.K; c += 1024) {
+        if (cnt[c] < 1) bad |= 2;
+        if (fill[c] > dm.C) bad |= 4;
+    }
+    if (bad) atomicOr(&status[RP_SW_VALIDATE], bad);
+}
+
+int rp_launch_validate(rp_ctx *c)
+{
+    int *fill = (int *)c->d_sort_keys;                 // scratch: 2*K ints fit (K <= N)
+    k_validate<<<1, 1024, 0, c->stream>>>(c->d_inc_layout, c->d_t, c->dm, fill, fill + c->dm.K, c->d_status);
+    RP_CUDA(cudaGetLastError());
+    return RP_OK;
+}

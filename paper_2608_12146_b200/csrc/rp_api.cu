@@ -1,0 +1,623 @@
+// C-ABI entry points of the RoutePack B200 library: argument checks, device memory
+// ownership, kernel sequencing.  All arithmetic of the method runs in the kernels.
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+
+#include "rp_common.cuh"
+
+thread_local int g_rp_last_cuda_error = 0;
+
+extern "C" int rp_last_cuda_error(void) { return g_rp_last_cuda_error; }
+
+extern "C" const char *rp_strerror(int s)
+{
+    switch (s) {
+        case RP_OK: return "ok";
+        case RP_ERR_ARG: return "bad argument";
+        case RP_ERR_SHAPE: return "inconsistent shapes";
+        case RP_ERR_CONSERVATION: return "window fails the input checks (length range, negative count, or sum_e a != k*t)";
+        case RP_ERR_INFEASIBLE: return "no feasible row count";
+        case RP_ERR_RANGE: return "fixed-point range or on-chip memory budget exceeded";
+        case RP_ERR_CUDA: return "CUDA error";
+        case RP_ERR_STATE: return "call out of order";
+        case RP_ERR_TIMEOUT: return "device-side wait timed out";
+        case RP_ERR_INVALID_PLAN: return "incumbent failed validation";
+        default: return "unknown status";
+    }
+}
+
+template <class T>
+static int dev_alloc(T **p, size_t n)
+{
+    *p = nullptr;
+    if (n == 0) n = 1;
+    RP_CUDA(cudaMalloc((void **)p, n * sizeof(T)));
+    return RP_OK;
+}
+static void dev_free(void *p) { if (p) cudaFree(p); }
+
+static bool is_device_ptr(const void *p)
+{
+    cudaPointerAttributes at;
+    cudaError_t e = cudaPointerGetAttributes(&at, p);
+    if (e != cudaSuccess) { cudaGetLastError(); return false; }
+    return at.type == cudaMemoryTypeDevice || at.type == cudaMemoryTypeManaged;
+}
+
+static int copy_out(rp_ctx *c, void *dst, const void *src, size_t bytes)
+{
+    if (!dst || !bytes) return RP_OK;
+    RP_CUDA(cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDefault, c->stream));
+    return RP_OK;
+}
+
+static void free_population(rp_ctx *c)
+{
+    for (int b = 0; b < 2; ++b) {
+        dev_free(c->buf[b].cell_of); dev_free(c->buf[b].W); dev_free(c->buf[b].Esum);
+        c->buf[b].cell_of = nullptr; c->buf[b].W = nullptr; c->buf[b].Esum = nullptr;
+    }
+    dev_free(c->d_anc); dev_free(c->d_term); dev_free(c->d_best); dev_free(c->d_best_step);
+    dev_free(c->d_best_nlog); dev_free(c->d_digest); dev_free(c->d_log); dev_free(c->d_F);
+    c->d_anc = nullptr; c->d_term = nullptr; c->d_best = nullptr; c->d_best_step = nullptr;
+    c->d_best_nlog = nullptr; c->d_digest = nullptr; c->d_log = nullptr; c->d_F = nullptr;
+    c->log_cap = 0;
+}
+
+static void free_trace(rp_ctx *c)
+{
+    dev_free(c->d_tr_term); dev_free(c->d_tr_best); dev_free(c->d_tr_inc);
+    dev_free(c->d_tr_best_step); dev_free(c->d_tr_anc); dev_free(c->d_tr_digest);
+    c->d_tr_term = c->d_tr_best = c->d_tr_inc = nullptr;
+    c->d_tr_best_step = c->d_tr_anc = nullptr;
+    c->d_tr_digest = nullptr;
+    c->trace_levels = 0;
+}
+
+static void free_eval(rp_ctx *c)
+{
+    dev_free(c->d_eval_score); dev_free(c->d_eval_f64); dev_free(c->d_eval_W);
+    dev_free(c->d_eval_cells); dev_free(c->d_eval_Esum);
+    c->d_eval_score = nullptr; c->d_eval_f64 = nullptr; c->d_eval_W = nullptr;
+    c->d_eval_cells = nullptr; c->d_eval_Esum = nullptr;
+    c->eval_cap = 0; c->eval_W_n = 0;
+}
+
+extern "C" void rp_destroy(rp_ctx *c)
+{
+    if (!c) return;
+    cudaStreamSynchronize(c->stream);
+    free_population(c); free_trace(c); free_eval(c);
+    dev_free(c->own_t); dev_free(c->own_a); dev_free(c->d_edp); dev_free(c->d_dp_list); dev_free(c->d_dp_off);
+    dev_free(c->d_Lagg); dev_free(c->d_pi); dev_free(c->d_inv); dev_free(c->d_rank_load); dev_free(c->d_q);
+    dev_free(c->d_status); dev_free(c->d_sort_keys); dev_free(c->d_seed_layout); dev_free(c->d_pack_out);
+    dev_free(c->d_counters); dev_free(c->d_inc_layout); dev_free(c->d_inc_score);
+    free(c->h_levels); free(c->h_t);
+    free(c);
+}
+
+static int reset_status(rp_ctx *c)
+{
+    int init[RP_SW_COUNT];
+    for (int x = 0; x < RP_SW_COUNT; ++x) init[x] = 0;
+    init[RP_SW_BAD_SAMPLE] = 0x7fffffff;
+    RP_CUDA(cudaMemcpyAsync(c->d_status, init, sizeof init, cudaMemcpyHostToDevice, c->stream));
+    RP_CUDA(cudaStreamSynchronize(c->stream));   // init[] is a stack array
+    return RP_OK;
+}
+
+static int read_status(rp_ctx *c, int out[RP_SW_COUNT])
+{
+    RP_CUDA(cudaMemcpyAsync(out, c->d_status, sizeof(int) * RP_SW_COUNT, cudaMemcpyDeviceToHost, c->stream));
+    RP_CUDA(cudaStreamSynchronize(c->stream));
+    return RP_OK;
+}
+
+static int window_load_impl(rp_ctx *c, const rp_config *cfg, const int32_t *lengths, const int32_t *demand)
+{
+    RpDims &dm = c->dm;
+    const int N = cfg->n_samples, L = cfg->n_layers, E = cfg->n_experts, D = cfg->dp_width, P = cfg->ep_width;
+    // EDP partition
+    int *edp = (int *)malloc(sizeof(int) * D);
+    int G = 0;
+    for (int d = 0; d < D; ++d) {
+        edp[d] = cfg->edp_of_dp ? cfg->edp_of_dp[d] : d;
+        if (edp[d] < 0 || edp[d] >= D) { free(edp); return RP_ERR_SHAPE; }
+        if (edp[d] + 1 > G) G = edp[d] + 1;
+    }
+    int *off = (int *)calloc(G + 1, sizeof(int)), *list = (int *)malloc(sizeof(int) * D);
+    for (int d = 0; d < D; ++d) off[edp[d] + 1]++;
+    int maxshard = 0;
+    for (int g = 0; g < G; ++g) {
+        if (off[g + 1] == 0) { free(edp); free(off); free(list); return RP_ERR_SHAPE; }   // unused shard id
+        if (off[g + 1] > maxshard) maxshard = off[g + 1];
+        off[g + 1] += off[g];
+    }
+    {
+        int *cursor = (int *)malloc(sizeof(int) * G);
+        for (int g = 0; g < G; ++g) cursor[g] = off[g];
+        for (int d = 0; d < D; ++d) list[cursor[edp[d]]++] = d;
+        free(cursor);
+    }
+    dm.N = N; dm.L = L; dm.E = E; dm.k = cfg->top_k; dm.C = cfg->token_cap; dm.D = D; dm.P = P; dm.G = G;
+    dm.H = E / P; dm.S = cfg->n_stages;
+    dm.R = 0; dm.K = 0; dm.RG = 0; dm.LP = L * P;
+    dm.asum = 0; dm.bsum = 0;
+    for (int s = 0; s < RP_MAX_STAGES; ++s) { dm.ahat[s] = 0; dm.bhat[s] = 0; }
+    for (int s = 0; s < dm.S; ++s) {
+        dm.ahat[s] = (i64)floor(cfg->alpha[s] * 256.0 + 0.5);
+        dm.bhat[s] = (i64)floor(cfg->beta[s] * 256.0 + 0.5);
+        dm.asum += dm.ahat[s]; dm.bsum += dm.bhat[s];
+    }
+    dm.SC = ((i64)dm.C * dm.C) << RP_FBITS;
+    dm.EC = (i64)dm.C << RP_FBITS;
+    int st = RP_OK;
+    do {
+        // rank loads must fit int32: W <= k * C * |D_g|
+        if ((double)dm.k * dm.C * maxshard >= 2147483648.0) { st = RP_ERR_RANGE; break; }
+        if ((st = dev_alloc(&c->d_edp, D)) != RP_OK) break;
+        if ((st = dev_alloc(&c->d_dp_list, D)) != RP_OK) break;
+        if ((st = dev_alloc(&c->d_dp_off, G + 1)) != RP_OK) break;
+        cudaMemcpyAsync(c->d_edp, edp, sizeof(int) * D, cudaMemcpyHostToDevice, c->stream);
+        cudaMemcpyAsync(c->d_dp_list, list, sizeof(int) * D, cudaMemcpyHostToDevice, c->stream);
+        cudaMemcpyAsync(c->d_dp_off, off, sizeof(int) * (G + 1), cudaMemcpyHostToDevice, c->stream);
+        if (cudaStreamSynchronize(c->stream) != cudaSuccess) { st = RP_ERR_CUDA; break; }
+    } while (0);
+    free(edp); free(off); free(list);
+    RP_TRY(st);
+
+    // inputs: adopt device arrays, copy host arrays
+    const size_t n_a = (size_t)N * L * E;
+    c->h_t = (int *)malloc(sizeof(int) * N);
+    if (is_device_ptr(lengths)) {
+        c->d_t = lengths;
+        RP_CUDA(cudaMemcpyAsync(c->h_t, lengths, sizeof(int) * N, cudaMemcpyDeviceToHost, c->stream));
+    } else {
+        RP_TRY(dev_alloc(&c->own_t, N));
+        RP_CUDA(cudaMemcpyAsync(c->own_t, lengths, sizeof(int) * N, cudaMemcpyHostToDevice, c->stream));
+        memcpy(c->h_t, lengths, sizeof(int) * N);
+        c->d_t = c->own_t;
+    }
+    if (is_device_ptr(demand)) c->d_a = demand;
+    else {
+        RP_TRY(dev_alloc(&c->own_a, n_a));
+        RP_CUDA(cudaMemcpyAsync(c->own_a, demand, sizeof(int) * n_a, cudaMemcpyHostToDevice, c->stream));
+        c->d_a = c->own_a;
+    }
+    RP_TRY(dev_alloc(&c->d_Lagg, (size_t)L * E));
+    RP_TRY(dev_alloc(&c->d_pi, (size_t)L * E));
+    RP_TRY(dev_alloc(&c->d_inv, (size_t)L * E));
+    RP_TRY(dev_alloc(&c->d_rank_load, (size_t)L * P));
+    RP_TRY(dev_alloc(&c->d_q, (size_t)N * L * P));
+    RP_TRY(dev_alloc(&c->d_status, RP_SW_COUNT));
+    int n_pow2 = 1;
+    while (n_pow2 < N) n_pow2 <<= 1;
+    RP_TRY(dev_alloc(&c->d_sort_keys, (size_t)2 * n_pow2));
+    RP_TRY(dev_alloc(&c->d_seed_layout, N));
+    RP_TRY(dev_alloc(&c->d_pack_out, 4));
+    RP_TRY(dev_alloc(&c->d_counters, 4));
+    RP_TRY(dev_alloc(&c->d_inc_layout, N));
+    RP_TRY(dev_alloc(&c->d_inc_score, 3));
+    RP_TRY(reset_status(c));
+
+    // input checks + aggregate expert load in one pass over the demand tensor
+    RP_TRY(rp_launch_check_reduce(c));
+    int sw[RP_SW_COUNT];
+    RP_TRY(read_status(c, sw));
+    if (sw[RP_SW_BAD_SAMPLE] != 0x7fffffff) return RP_ERR_CONSERVATION;
+
+    // fixed-point range of the score: s1 <= (2^8*C*L*k + (asum+bsum)*C) * sum t  must stay below 2^62
+    double total = 0.0;
+    for (int i = 0; i < N; ++i) total += (double)c->h_t[i];
+    double bound = ((double)dm.EC * L * dm.k + (double)(dm.asum + dm.bsum) * dm.C) * total;
+    if (bound >= 4.0e18) return RP_ERR_RANGE;
+    return RP_OK;
+}
+
+extern "C" int rp_window_load(rp_ctx **out, const rp_config *cfg, const int32_t *lengths,
+                              const int32_t *demand, void *cuda_stream)
+{
+    if (!out) return RP_ERR_ARG;
+    *out = nullptr;
+    if (!cfg || !lengths || !demand) return RP_ERR_ARG;
+    if (cfg->n_samples < 1 || cfg->n_layers < 1 || cfg->n_experts < 1 || cfg->top_k < 1 || cfg->token_cap < 1 ||
+        cfg->dp_width < 1 || cfg->ep_width < 1 || cfg->pop_size < 1 || cfg->min_rows < 0)
+        return RP_ERR_ARG;
+    if (cfg->n_stages < 1 || cfg->n_stages > RP_MAX_STAGES || !cfg->alpha || !cfg->beta) return RP_ERR_ARG;
+    for (int s = 0; s < cfg->n_stages; ++s)
+        if (!(cfg->alpha[s] >= 0.0) || !(cfg->beta[s] >= 0.0) || cfg->alpha[s] > 1e6 || cfg->beta[s] > 1e6) return RP_ERR_ARG;
+    if (cfg->n_experts % cfg->ep_width != 0 || cfg->n_samples < cfg->dp_width) return RP_ERR_SHAPE;
+    if (cfg->ep_width > RP_MAX_EP || cfg->dp_width > 4096 || cfg->n_experts > 1024) return RP_ERR_RANGE;
+    if (cfg->token_cap > (1 << 24) || cfg->n_samples > (1 << 20) || cfg->pop_size > (1 << 20)) return RP_ERR_RANGE;
+    if ((long long)cfg->n_layers * cfg->ep_width > (1 << 20)) return RP_ERR_RANGE;
+
+    rp_ctx *c = (rp_ctx *)calloc(1, sizeof(rp_ctx));
+    if (!c) return RP_ERR_ARG;
+    if (cudaGetDevice(&c->device) != cudaSuccess) { free(c); return RP_ERR_CUDA; }
+    c->stream = (cudaStream_t)cuda_stream;
+    c->cfg = *cfg;
+    c->cfg.edp_of_dp = nullptr; c->cfg.alpha = nullptr; c->cfg.beta = nullptr;
+    c->Ppop = cfg->pop_size;
+    int st = window_load_impl(c, cfg, lengths, demand);
+    if (st != RP_OK) { rp_destroy(c); return st; }
+    c->stage = 1;
+    *out = c;
+    return RP_OK;
+}
+
+extern "C" int rp_place_experts(rp_ctx *c, int32_t *pi, int64_t *rank_load)
+{
+    if (!c) return RP_ERR_ARG;
+    if (c->stage < 1) return RP_ERR_STATE;
+    const RpDims &dm = c->dm;
+    RP_TRY(rp_launch_lpt(c));
+    RP_TRY(rp_launch_project(c));
+    RP_TRY(copy_out(c, pi, c->d_pi, sizeof(int) * (size_t)dm.L * dm.E));
+    RP_TRY(copy_out(c, rank_load, c->d_rank_load, sizeof(i64) * (size_t)dm.L * dm.P));
+    RP_CUDA(cudaStreamSynchronize(c->stream));
+    if (c->stage < 2) c->stage = 2;
+    return RP_OK;
+}
+
+static int ensure_eval_scratch(rp_ctx *c, size_t n, bool want_W)
+{
+    const RpDims &dm = c->dm;
+    if (n > c->eval_cap) {
+        dev_free(c->d_eval_score); dev_free(c->d_eval_f64); dev_free(c->d_eval_cells); dev_free(c->d_eval_Esum);
+        c->d_eval_score = nullptr; c->d_eval_f64 = nullptr; c->d_eval_cells = nullptr; c->d_eval_Esum = nullptr;
+        c->eval_cap = 0;
+        RP_TRY(dev_alloc(&c->d_eval_score, n * 3));
+        RP_TRY(dev_alloc(&c->d_eval_f64, n * 3));
+        RP_TRY(dev_alloc(&c->d_eval_cells, n * dm.N));
+        RP_TRY(dev_alloc(&c->d_eval_Esum, n * dm.RG));
+        c->eval_cap = n;
+    }
+    if (want_W && (int)n > c->eval_W_n) {
+        dev_free(c->d_eval_W);
+        c->d_eval_W = nullptr; c->eval_W_n = 0;
+        RP_TRY(dev_alloc(&c->d_eval_W, n * dm.RG * dm.LP));
+        c->eval_W_n = (int)n;
+    }
+    return RP_OK;
+}
+
+extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
+{
+    if (!c) return RP_ERR_ARG;
+    if (c->stage < 2) return RP_ERR_STATE;
+    RpDims &dm = c->dm;
+    RP_TRY(rp_launch_pack(c, 0));
+    int po[4];
+    RP_CUDA(cudaMemcpyAsync(po, c->d_pack_out, sizeof po, cudaMemcpyDeviceToHost, c->stream));
+    RP_CUDA(cudaStreamSynchronize(c->stream));
+    if (po[3] || po[0] <= 0) return RP_ERR_INFEASIBLE;
+    c->Rstar = po[0]; c->certified = po[1];
+    dm.R = po[0]; dm.K = dm.R * dm.D; dm.RG = dm.R * dm.G;
+    if (dm.K > 65535) return RP_ERR_RANGE;
+    int nt; size_t smem;
+    rp_anneal_smem_bytes(c, &nt, &smem);
+    if (smem > 220 * 1024) return RP_ERR_RANGE;
+
+    // population buffers
+    free_population(c); free_eval(c);
+    const size_t P = (size_t)c->Ppop, wn = (size_t)dm.RG * dm.LP;
+    for (int b = 0; b < 2; ++b) {
+        RP_TRY(dev_alloc(&c->buf[b].cell_of, P * dm.N));
+        RP_TRY(dev_alloc(&c->buf[b].W, P * wn));
+        RP_TRY(dev_alloc(&c->buf[b].Esum, P * dm.RG));
+    }
+    RP_TRY(dev_alloc(&c->d_anc, P));
+    RP_TRY(dev_alloc(&c->d_term, P * 3));
+    RP_TRY(dev_alloc(&c->d_best, P * 3));
+    RP_TRY(dev_alloc(&c->d_best_step, P));
+    RP_TRY(dev_alloc(&c->d_best_nlog, P));
+    RP_TRY(dev_alloc(&c->d_digest, P));
+    RP_TRY(dev_alloc(&c->d_F, P));
+    c->cur = 0;
+    // every member starts as the length-only seed: evaluate it once into slot 0 and let all
+    // slots descend from slot 0
+    RP_TRY(rp_launch_cells_from_layouts(c, c->d_seed_layout, 1, c->buf[0].cell_of));
+    RP_TRY(rp_launch_eval(c, c->buf[0].cell_of, 1, c->buf[0].W, c->buf[0].Esum, c->d_inc_score, nullptr));
+    RP_CUDA(cudaMemsetAsync(c->d_anc, 0, sizeof(int) * P, c->stream));
+    RP_CUDA(cudaMemcpyAsync(c->d_inc_layout, c->d_seed_layout, sizeof(int) * dm.N, cudaMemcpyDeviceToDevice, c->stream));
+    RP_CUDA(cudaMemcpyAsync(c->seed_score, c->d_inc_score, sizeof(i64) * 3, cudaMemcpyDeviceToHost, c->stream));
+    RP_CUDA(cudaStreamSynchronize(c->stream));
+    if (n_rows) *n_rows = c->Rstar;
+    if (certified) *certified = c->certified;
+    c->stage = 3;
+    return RP_OK;
+}
+
+__global__ void k_gather_cells(const unsigned short *__restrict__ src, const int *__restrict__ anc, int N,
+                               unsigned short *__restrict__ dst16, int *__restrict__ dst32)
+{
+    const int j = blockIdx.x;
+    const unsigned short *s = src + (size_t)anc[j] * N;
+    for (int i = threadIdx.x; i < N; i += blockDim.x) {
+        if (dst16) dst16[(size_t)j * N + i] = s[i];
+        if (dst32) dst32[(size_t)j * N + i] = s[i];
+    }
+}
+
+extern "C" int rp_eval_population(rp_ctx *c, const int32_t *layouts, int32_t n, int64_t *score_fx, double *score_f64)
+{
+    if (!c) return RP_ERR_ARG;
+    if (c->stage < 3) return RP_ERR_STATE;
+    const RpDims &dm = c->dm;
+    if (!layouts) n = c->Ppop;
+    if (n < 1) return RP_ERR_ARG;
+    const bool keepW = layouts && n <= 64;
+    RP_TRY(ensure_eval_scratch(c, (size_t)n, keepW));
+    if (layouts) {
+        const int *dl = layouts;
+        int *tmp = nullptr;
+        if (!is_device_ptr(layouts)) {
+            RP_TRY(dev_alloc(&tmp, (size_t)n * dm.N));
+            cudaError_t e = cudaMemcpyAsync(tmp, layouts, sizeof(int) * (size_t)n * dm.N, cudaMemcpyHostToDevice, c->stream);
+            if (e != cudaSuccess) { dev_free(tmp); g_rp_last_cuda_error = (int)e; return RP_ERR_CUDA; }
+            dl = tmp;
+        }
+        RP_TRY(reset_status(c));
+        int st = rp_launch_cells_from_layouts(c, dl, n, c->d_eval_cells);
+        int sw[RP_SW_COUNT];
+        if (st == RP_OK) st = read_status(c, sw);
+        dev_free(tmp);
+        RP_TRY(st);
+        if (sw[RP_SW_BAD_LAYOUT]) return RP_ERR_ARG;
+    } else {
+        k_gather_cells<<<n, 256, 0, c->stream>>>(c->buf[c->cur].cell_of, c->d_anc, dm.N, c->d_eval_cells, nullptr);
+        RP_CUDA(cudaGetLastError());
+    }
+    RP_TRY(rp_launch_eval(c, c->d_eval_cells, n, keepW ? c->d_eval_W : nullptr, c->d_eval_Esum, c->d_eval_score,
+                          c->d_eval_f64));
+    RP_TRY(copy_out(c, score_fx, c->d_eval_score, sizeof(i64) * 3 * (size_t)n));
+    RP_TRY(copy_out(c, score_f64, c->d_eval_f64, sizeof(double) * 3 * (size_t)n));
+    RP_CUDA(cudaStreamSynchronize(c->stream));
+    return RP_OK;
+}
+
+// Per-level integers of the geometric schedule, from IEEE double operations only.
+static void make_schedule(const rp_anneal_params *p, RpLevel *lv)
+{
+    const double LN2 = 0.6931471805599453094;
+    volatile double T = p->t0;
+    for (int n = 0; n < p->n_levels; ++n) {
+        volatile double Tn = T * p->t_ratio;
+        volatile double x = T * LN2;
+        x = x * 4294967296.0;
+        lv[n].tau = (x >= 1.8e19) ? ~0ull : (u64)floor(x);
+        volatile double inv_next = 1.0 / Tn, inv_cur = 1.0 / T;
+        volatile double db = inv_next - inv_cur;
+        volatile double y = db * (1.0 / LN2);
+        y = y * 65536.0;
+        lv[n].cq = (y > 0.0) ? ((y >= 1.8e19) ? ~0ull : (u64)floor(y)) : 0ull;
+        T = Tn;
+    }
+}
+
+extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *stats)
+{
+    if (!c || !p) return RP_ERR_ARG;
+    if (c->stage < 3) return RP_ERR_STATE;
+    if (p->n_levels < 1 || p->steps_per_level < 1 || p->n_levels > 100000 || p->steps_per_level > (1 << 22)) return RP_ERR_ARG;
+    if (!(p->t0 > 0.0) || !(p->t_ratio > 0.0) || p->t_ratio > 1.0) return RP_ERR_ARG;
+    if (!(p->p_reloc >= 0.0) || p->p_reloc > 1.0 || !(p->p_guide >= 0.0) || p->p_guide > 1.0) return RP_ERR_ARG;
+    const size_t P = (size_t)c->Ppop;
+    const int NL = p->n_levels;
+    // schedule
+    free(c->h_levels);
+    c->h_levels = (RpLevel *)malloc(sizeof(RpLevel) * NL);
+    make_schedule(p, c->h_levels);
+    const u64 rho_q32 = (u64)floor(p->p_reloc * 4294967296.0);
+    const u64 guide_q32 = (u64)floor(p->p_guide * 4294967296.0);
+    // accepted-move log
+    if (c->log_cap < p->steps_per_level) {
+        dev_free(c->d_log); c->d_log = nullptr; c->log_cap = 0;
+        RP_TRY(dev_alloc(&c->d_log, P * (size_t)p->steps_per_level));
+        c->log_cap = p->steps_per_level;
+    }
+    // trace
+    free_trace(c);
+    RP_TRY(dev_alloc(&c->d_tr_term, (size_t)NL * P * 3));
+    RP_TRY(dev_alloc(&c->d_tr_best, (size_t)NL * P * 3));
+    RP_TRY(dev_alloc(&c->d_tr_inc, (size_t)NL * 3));
+    RP_TRY(dev_alloc(&c->d_tr_best_step, (size_t)NL * P));
+    RP_TRY(dev_alloc(&c->d_tr_digest, (size_t)NL * P));
+    RP_TRY(dev_alloc(&c->d_tr_anc, (size_t)(NL > 1 ? NL - 1 : 1) * P));
+    c->trace_levels = NL;
+    RP_CUDA(cudaMemsetAsync(c->d_counters, 0, sizeof(i64) * 4, c->stream));
+
+    cudaEvent_t ev[3];
+    for (int x = 0; x < 3; ++x) RP_CUDA(cudaEventCreate(&ev[x]));
+    float ms_chains = 0.f, ms_barrier = 0.f;
+    int st = RP_OK;
+    for (int n = 0; n < NL && st == RP_OK; ++n) {
+        cudaEventRecord(ev[0], c->stream);
+        st = rp_launch_anneal_level(c, n, p, rho_q32, guide_q32);
+        cudaEventRecord(ev[1], c->stream);
+        if (st == RP_OK) st = rp_launch_level_end(c, n, NL);
+        cudaEventRecord(ev[2], c->stream);
+        c->cur = 1 - c->cur;          // the terminal states are the next level's sources
+        if (stats) {
+            if (cudaEventSynchronize(ev[2]) != cudaSuccess) { st = RP_ERR_CUDA; break; }
+            float a = 0.f, b = 0.f;
+            cudaEventElapsedTime(&a, ev[0], ev[1]);
+            cudaEventElapsedTime(&b, ev[1], ev[2]);
+            ms_chains += a; ms_barrier += b;
+        }
+    }
+    cudaError_t e = cudaStreamSynchronize(c->stream);
+    for (int x = 0; x < 3; ++x) cudaEventDestroy(ev[x]);
+    if (st == RP_OK && e != cudaSuccess) { g_rp_last_cuda_error = (int)e; st = RP_ERR_CUDA; }
+    RP_TRY(st);
+    if (stats) {
+        i64 cn[4];
+        RP_CUDA(cudaMemcpy(cn, c->d_counters, sizeof cn, cudaMemcpyDeviceToHost));
+        stats->proposed = cn[0]; stats->feasible = cn[1]; stats->accepted = cn[2]; stats->improved = cn[3];
+        stats->ms_chains = ms_chains; stats->ms_barrier = ms_barrier;
+    }
+    c->stage = 4;
+    return RP_OK;
+}
+
+extern "C" int rp_best(rp_ctx *c, int32_t *cell_of_sample, int64_t *score_fx, double *score_f64)
+{
+    if (!c) return RP_ERR_ARG;
+    if (c->stage < 3) return RP_ERR_STATE;
+    const RpDims &dm = c->dm;
+    RP_TRY(reset_status(c));
+    RP_TRY(rp_launch_validate(c));
+    // full rescoring of the incumbent
+    RP_TRY(ensure_eval_scratch(c, 1, false));
+    RP_TRY(rp_launch_cells_from_layouts(c, c->d_inc_layout, 1, c->d_eval_cells));
+    RP_TRY(rp_launch_eval(c, c->d_eval_cells, 1, nullptr, c->d_eval_Esum, c->d_eval_score, c->d_eval_f64));
+    i64 inc[3], full[3];
+    int sw[RP_SW_COUNT];
+    RP_CUDA(cudaMemcpyAsync(inc, c->d_inc_score, sizeof inc, cudaMemcpyDeviceToHost, c->stream));
+    RP_CUDA(cudaMemcpyAsync(full, c->d_eval_score, sizeof full, cudaMemcpyDeviceToHost, c->stream));
+    RP_TRY(read_status(c, sw));
+    bool ok = !sw[RP_SW_VALIDATE] && !sw[RP_SW_BAD_LAYOUT];
+    ok = ok && inc[0] == full[0] && inc[1] == full[1] && inc[2] == full[2];
+    // non-regression: not worse than the best seed
+    const i64 *s = c->seed_score;
+    bool worse = (s[0] != inc[0]) ? (s[0] < inc[0]) : (s[1] != inc[1]) ? (s[1] < inc[1]) : (s[2] < inc[2]);
+    ok = ok && !worse;
+    RP_TRY(copy_out(c, cell_of_sample, c->d_inc_layout, sizeof(int) * (size_t)dm.N));
+    RP_TRY(copy_out(c, score_fx, c->d_inc_score, sizeof(i64) * 3));
+    RP_TRY(copy_out(c, score_f64, c->d_eval_f64, sizeof(double) * 3));
+    RP_CUDA(cudaStreamSynchronize(c->stream));
+    return ok ? RP_OK : RP_ERR_INVALID_PLAN;
+}
+
+// ---------------------------------------------------------------------------------------
+// inspection hooks
+// ---------------------------------------------------------------------------------------
+__global__ void k_cell_stats(const unsigned short *__restrict__ cells, const int *__restrict__ t, int N, int K,
+                             i64 *__restrict__ T, i64 *__restrict__ Q, int *__restrict__ cnt)
+{
+    for (int c = threadIdx.x; c < K; c += blockDim.x) { T[c] = 0; Q[c] = 0; cnt[c] = 0; }
+    __syncthreads();
+    for (int i = threadIdx.x; i < N; i += blockDim.x) {
+        int c = cells[i];
+        atomicAdd((u64 *)&T[c], (u64)t[i]);
+        atomicAdd((u64 *)&Q[c], (u64)t[i] * (u64)t[i]);
+        atomicAdd(&cnt[c], 1);
+    }
+}
+
+extern "C" int rp_debug_dump(rp_ctx *c, int what, int32_t index, void *buf, int64_t bytes)
+{
+    if (!c || !buf) return RP_ERR_ARG;
+    const RpDims &dm = c->dm;
+    const size_t P = (size_t)c->Ppop;
+    const void *src = nullptr;
+    size_t need = 0;
+    void *tmp = nullptr;
+    int st = RP_OK;
+    int member = -1;
+    if (what >= RP_DUMP_POPULATION && what <= RP_DUMP_ESUM) {
+        if (c->stage < 3) return RP_ERR_STATE;
+        if (what != RP_DUMP_POPULATION) {
+            if (index < 0 || index >= c->Ppop) return RP_ERR_ARG;
+            RP_CUDA(cudaMemcpyAsync(&member, c->d_anc + index, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+            RP_CUDA(cudaStreamSynchronize(c->stream));
+        }
+    }
+    switch (what) {
+        case RP_DUMP_LAGG: if (c->stage < 1) return RP_ERR_STATE; src = c->d_Lagg; need = sizeof(i64) * dm.L * dm.E; break;
+        case RP_DUMP_Q: if (c->stage < 2) return RP_ERR_STATE; src = c->d_q; need = sizeof(int) * (size_t)dm.N * dm.LP; break;
+        case RP_DUMP_SEED_LAYOUT: if (c->stage < 3) return RP_ERR_STATE; src = c->d_seed_layout; need = sizeof(int) * dm.N; break;
+        case RP_DUMP_POPULATION: {
+            need = sizeof(int) * P * dm.N;
+            if ((st = dev_alloc((int **)&tmp, P * dm.N)) != RP_OK) return st;
+            k_gather_cells<<<c->Ppop, 256, 0, c->stream>>>(c->buf[c->cur].cell_of, c->d_anc, dm.N, nullptr, (int *)tmp);
+            src = tmp;
+            break;
+        }
+        case RP_DUMP_W: src = c->buf[c->cur].W + (size_t)member * dm.RG * dm.LP; need = sizeof(int) * (size_t)dm.RG * dm.LP; break;
+        case RP_DUMP_ESUM: src = c->buf[c->cur].Esum + (size_t)member * dm.RG; need = sizeof(i64) * dm.RG; break;
+        case RP_DUMP_CELL_T: case RP_DUMP_CELL_Q: case RP_DUMP_CELL_CNT: {
+            size_t K = dm.K;
+            if ((st = dev_alloc((i64 **)&tmp, 3 * K)) != RP_OK) return st;
+            i64 *T = (i64 *)tmp, *Q = T + K;
+            int *cnt = (int *)(Q + K);
+            k_cell_stats<<<1, 256, 0, c->stream>>>(c->buf[c->cur].cell_of + (size_t)member * dm.N, c->d_t, dm.N, dm.K, T, Q, cnt);
+            if (what == RP_DUMP_CELL_T) { src = T; need = sizeof(i64) * K; }
+            else if (what == RP_DUMP_CELL_Q) { src = Q; need = sizeof(i64) * K; }
+            else { src = cnt; need = sizeof(int) * K; }
+            break;
+        }
+        case RP_DUMP_TRACE_TERM: src = c->d_tr_term; need = sizeof(i64) * 3 * P * c->trace_levels; break;
+        case RP_DUMP_TRACE_BEST: src = c->d_tr_best; need = sizeof(i64) * 3 * P * c->trace_levels; break;
+        case RP_DUMP_TRACE_BEST_STEP: src = c->d_tr_best_step; need = sizeof(int) * P * c->trace_levels; break;
+        case RP_DUMP_TRACE_DIGEST: src = c->d_tr_digest; need = sizeof(u64) * P * c->trace_levels; break;
+        case RP_DUMP_TRACE_ANC: src = c->d_tr_anc; need = sizeof(int) * P * (c->trace_levels > 1 ? c->trace_levels - 1 : 0); break;
+        case RP_DUMP_TRACE_INCUMBENT: src = c->d_tr_inc; need = sizeof(i64) * 3 * c->trace_levels; break;
+        case RP_DUMP_EVAL_W:
+            if (index < 0 || index >= c->eval_W_n) return RP_ERR_ARG;
+            src = c->d_eval_W + (size_t)index * dm.RG * dm.LP; need = sizeof(int) * (size_t)dm.RG * dm.LP; break;
+        default: return RP_ERR_ARG;
+    }
+    if (what >= RP_DUMP_TRACE_TERM && what <= RP_DUMP_TRACE_INCUMBENT && c->trace_levels == 0) { dev_free(tmp); return RP_ERR_STATE; }
+    if ((int64_t)need != bytes) { dev_free(tmp); return RP_ERR_ARG; }
+    cudaError_t e = cudaSuccess;
+    if (need) e = cudaMemcpyAsync(buf, src, need, cudaMemcpyDefault, c->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+    dev_free(tmp);
+    if (e != cudaSuccess) { g_rp_last_cuda_error = (int)e; return RP_ERR_CUDA; }
+    return RP_OK;
+}
+
+__global__ void k_dbg_nl2(const u32 *x, u64 *out, long long n)
+{
+    long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) out[i] = rp_nl2(x[i]);
+}
+__global__ void k_dbg_exp2neg(const u64 *z, u64 *out, long long n)
+{
+    long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) out[i] = rp_exp2neg(z[i]);
+}
+__global__ void k_dbg_philox(const u32 *ctr, u32 k0, u32 k1, u32 *out, long long n)
+{
+    long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) {
+        uint4 r = rp_philox(ctr[4 * i], ctr[4 * i + 1], ctr[4 * i + 2], ctr[4 * i + 3], k0, k1);
+        out[4 * i] = r.x; out[4 * i + 1] = r.y; out[4 * i + 2] = r.z; out[4 * i + 3] = r.w;
+    }
+}
+
+template <class TI, class TO, class F>
+static int dbg_map(const TI *in, size_t in_per, TO *out, size_t out_per, int64_t n, F launch)
+{
+    if (!in || !out || n < 0) return RP_ERR_ARG;
+    if (n == 0) return RP_OK;
+    TI *din = nullptr; TO *dout = nullptr;
+    RP_TRY(dev_alloc(&din, (size_t)n * in_per));
+    int st = dev_alloc(&dout, (size_t)n * out_per);
+    if (st != RP_OK) { dev_free(din); return st; }
+    cudaError_t e = cudaMemcpy(din, in, sizeof(TI) * n * in_per, cudaMemcpyDefault);
+    if (e == cudaSuccess) { launch(din, dout); e = cudaGetLastError(); }
+    if (e == cudaSuccess) e = cudaMemcpy(out, dout, sizeof(TO) * n * out_per, cudaMemcpyDefault);
+    dev_free(din); dev_free(dout);
+    if (e != cudaSuccess) { g_rp_last_cuda_error = (int)e; return RP_ERR_CUDA; }
+    return RP_OK;
+}
+
+extern "C" int rp_debug_nl2(const uint32_t *x, uint64_t *out, int64_t n)
+{
+    return dbg_map<u32, u64>(x, 1, (u64 *)out, 1, n, [&](u32 *a, u64 *b) { k_dbg_nl2<<<(unsigned)((n + 255) / 256), 256>>>(a, b, n); });
+}
+extern "C" int rp_debug_exp2neg(const uint64_t *z, uint64_t *out, int64_t n)
+{
+    return dbg_map<u64, u64>((const u64 *)z, 1, (u64 *)out, 1, n, [&](u64 *a, u64 *b) { k_dbg_exp2neg<<<(unsigned)((n + 255) / 256), 256>>>(a, b, n); });
+}
+extern "C" int rp_debug_philox(const uint32_t *ctr, const uint32_t key[2], uint32_t *out, int64_t n)
+{
+    if (!key) return RP_ERR_ARG;
+    const u32 k0 = key[0], k1 = key[1];
+    return dbg_map<u32, u32>(ctr, 4, out, 4, n, [&](u32 *a, u32 *b) { k_dbg_philox<<<(unsigned)((n + 255) / 256), 256>>>(a, k0, k1, b, n); });
+}

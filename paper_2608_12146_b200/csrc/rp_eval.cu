@@ -1,0 +1,112 @@
+// Full evaluation of layouts (K4): cell statistics, per-row-shard rank loads W, expert and
+// attention costs, shard work and the score tuple (Sections 3.4-3.5 of the paper).
+//
+// One CTA per layout.  Samples are bucketed by row-shard in shared memory; each warp then
+// owns whole row-shards and adds up the q rows of its members with coalesced loads (q is
+// shared by all layouts and stays L2-resident), so W is produced without atomics and is
+// written at most once.  Algorithmic bytes per layout: N*2 (assignment) + N*L*P*4 (q rows,
+// L2-served) read, R*G*L*P*4 written when W is kept.
+#include "rp_score.cuh"
+
+#define EVAL_THREADS 256
+
+__global__ void k_layouts_to_cells(const int *__restrict__ layouts, long long total, int K,
+                                   unsigned short *__restrict__ cells, int *__restrict__ status)
+{
+    long long x = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (x >= total) return;
+    int c = layouts[x];
+    if (c < 0 || c >= K) { atomicExch(&status[RP_SW_BAD_LAYOUT], 1); c = 0; }
+    cells[x] = (unsigned short)c;
+}
+
+int rp_launch_cells_from_layouts(rp_ctx *c, const int *layouts, int n, unsigned short *cells)
+{
+    long long total = (long long)n * c->dm.N;
+    int grid = (int)((total + 255) / 256);
+    k_layouts_to_cells<<<grid, 256, 0, c->stream>>>(layouts, total, c->dm.K, cells, c->d_status);
+    RP_CUDA(cudaGetLastError());
+    return RP_OK;
+}
+
+__global__ void __launch_bounds__(EVAL_THREADS)
+k_eval(const unsigned short *__restrict__ cells, const int *__restrict__ t, const int *__restrict__ q,
+       const int *__restrict__ edp, const int *__restrict__ dp_list, const int *__restrict__ dp_off,
+       RpDims dm, int *__restrict__ W_out, i64 *__restrict__ Esum_out, i64 *__restrict__ score_out,
+       double *__restrict__ f64_out)
+{
+    extern __shared__ __align__(16) unsigned char smraw[];
+    // layout: Q[K] u64 | Esum[RG] | Afx[RG] | U[G] | T[K] | cnt[K] | off[RG+1] | cur[RG] | members[N] | cell_of[N]
+    u64 *Q = (u64 *)smraw;
+    i64 *Esum = (i64 *)(Q + dm.K);
+    i64 *Afx = Esum + dm.RG;
+    i64 *U = Afx + dm.RG;
+    int *T = (int *)(U + dm.G);
+    int *cnt = T + dm.K;
+    int *off = cnt + dm.K;
+    int *cur = off + dm.RG + 1;
+    int *members = cur + dm.RG;
+    unsigned short *cell_of = (unsigned short *)(members + dm.N);
+    RpSmemState st = { cell_of, T, Q, cnt, Esum, Afx, U };
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = EVAL_THREADS / 32;
+    const int lay = blockIdx.x;
+    const unsigned short *src = cells + (size_t)lay * dm.N;
+    for (int i = tid; i < dm.N; i += EVAL_THREADS) cell_of[i] = src[i];
+    for (int c = tid; c < dm.K; c += EVAL_THREADS) { T[c] = 0; Q[c] = 0; cnt[c] = 0; }
+    for (int x = tid; x <= dm.RG; x += EVAL_THREADS) { off[x] = 0; if (x < dm.RG) cur[x] = 0; }
+    __syncthreads();
+    rp_accumulate_cells(dm, st, t, tid, EVAL_THREADS);
+    for (int i = tid; i < dm.N; i += EVAL_THREADS) atomicAdd(&off[rp_rowshard(dm, edp, cell_of[i]) + 1], 1);
+    __syncthreads();
+    if (tid == 0) for (int x = 0; x < dm.RG; ++x) off[x + 1] += off[x];
+    __syncthreads();
+    for (int i = tid; i < dm.N; i += EVAL_THREADS) {
+        int rg = rp_rowshard(dm, edp, cell_of[i]);
+        members[off[rg] + atomicAdd(&cur[rg], 1)] = i;
+    }
+    __syncthreads();
+    for (int rg = warp; rg < dm.RG; rg += nwarps) {
+        const int m0 = off[rg], m1 = off[rg + 1];
+        int *wout = W_out ? W_out + ((size_t)lay * dm.RG + rg) * dm.LP : nullptr;
+        i64 es = rp_warp_layer_max_sum(dm, lane, [&](int x) {
+            int s = 0;
+            for (int m = m0; m < m1; ++m) s += __ldg(q + (size_t)members[m] * dm.LP + x);
+            if (wout) wout[x] = s;
+            return s;
+        });
+        if (lane == 0) Esum[rg] = es;
+    }
+    __syncthreads();
+    i64 sc[3];
+    rp_rows_to_score(dm, st, dp_list, dp_off, tid, EVAL_THREADS, sc);
+    if (Esum_out) for (int rg = tid; rg < dm.RG; rg += EVAL_THREADS) Esum_out[(size_t)lay * dm.RG + rg] = Esum[rg];
+    if (tid == 0) {
+        for (int x = 0; x < 3; ++x) {
+            if (score_out) score_out[(size_t)lay * 3 + x] = sc[x];
+            if (f64_out) f64_out[(size_t)lay * 3 + x] = (double)sc[x] / (double)dm.SC;
+        }
+    }
+}
+
+static size_t eval_smem_bytes(const RpDims &dm)
+{
+    size_t b = sizeof(u64) * dm.K + sizeof(i64) * (2 * (size_t)dm.RG + dm.G);
+    b += sizeof(int) * (2 * (size_t)dm.K + 2 * (size_t)dm.RG + 1 + dm.N);
+    b += sizeof(unsigned short) * dm.N;
+    return (b + 15) & ~(size_t)15;
+}
+
+int rp_launch_eval(rp_ctx *c, const unsigned short *cells, int n, int *W_out, i64 *Esum_out,
+                   i64 *score_out, double *f64_out)
+{
+    const RpDims &dm = c->dm;
+    size_t smem = eval_smem_bytes(dm);
+    if (smem > 220 * 1024) return RP_ERR_RANGE;
+    if (smem > 48 * 1024)
+        RP_CUDA(cudaFuncSetAttribute(k_eval, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    k_eval<<<n, EVAL_THREADS, smem, c->stream>>>(cells, c->d_t, c->d_q, c->d_edp, c->d_dp_list, c->d_dp_off, dm,
+                                                W_out, Esum_out, score_out, f64_out);
+    RP_CUDA(cudaGetLastError());
+    return RP_OK;
+}

@@ -1,0 +1,108 @@
+// Row count R* and the length-only seed layout (Section 3.2 of the paper; first line of
+// Algorithm 2), as one CTA on the GPU so that the whole plan stays stream-ordered.
+//
+// The samples are sorted by (-t_i, i) with a bitonic sort on 64-bit keys, then for
+// R = R_lb, R_lb+1, ... first-fit-decreasing is tried into K = R*D cells: the K longest
+// samples open the cells, each later sample goes to the lowest-numbered cell it still fits
+// in.  The fit search is done by one warp, 32 cells per ballot.
+#include "rp_common.cuh"
+
+#define PACK_THREADS 1024
+
+__global__ void __launch_bounds__(PACK_THREADS)
+k_pack_ffd(const int *__restrict__ t, RpDims dm, int min_rows, u64 *__restrict__ keys_g, int n_pow2,
+           int *__restrict__ fill_g, int *__restrict__ cell_of, int *__restrict__ out)
+{
+    extern __shared__ u64 keys_s[];
+    u64 *keys = keys_g ? keys_g : keys_s;
+    __shared__ i64 total_s;
+    __shared__ int fail_s;
+    const int tid = threadIdx.x;
+    if (tid == 0) total_s = 0;
+    __syncthreads();
+    i64 part = 0;
+    for (int i = tid; i < n_pow2; i += PACK_THREADS) {
+        if (i < dm.N) {
+            int ti = t[i];
+            part += ti;
+            keys[i] = ((u64)(u32)(dm.C - ti) << 32) | (u32)i;     // ascending = longest first, then id
+        } else {
+            keys[i] = ~0ull;
+        }
+    }
+    atomicAdd((u64 *)&total_s, (u64)part);
+    __syncthreads();
+    for (int k = 2; k <= n_pow2; k <<= 1)
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int i = tid; i < n_pow2; i += PACK_THREADS) {
+                int ixj = i ^ j;
+                if (ixj > i) {
+                    u64 a = keys[i], b = keys[ixj];
+                    bool up = ((i & k) == 0);
+                    if ((a > b) == up) { keys[i] = b; keys[ixj] = a; }
+                }
+            }
+            __syncthreads();
+        }
+    const i64 cap_row = (i64)dm.C * dm.D;
+    i64 Rlb = (total_s + cap_row - 1) / cap_row;
+    if (Rlb < 1) Rlb = 1;
+    if (Rlb < min_rows) Rlb = min_rows;
+    int Rstar = 0;
+    for (i64 R = Rlb; R * dm.D <= dm.N && !Rstar; ++R) {
+        const int K = (int)(R * dm.D);
+        for (int b = tid; b < K; b += PACK_THREADS) fill_g[b] = 0;
+        if (tid == 0) fail_s = 0;
+        __syncthreads();
+        // the K longest samples open the cells
+        for (int x = tid; x < K; x += PACK_THREADS) {
+            int s = (int)(u32)keys[x];
+            fill_g[x] = t[s];
+            cell_of[s] = x;
+        }
+        __syncthreads();
+        if (tid < 32) {
+            for (int x = K; x < dm.N; ++x) {
+                const int s = (int)(u32)keys[x];
+                const int ts = t[s];
+                int found = -1;
+                for (int b0 = 0; b0 < K && found < 0; b0 += 32) {
+                    int b = b0 + tid;
+                    bool ok = (b < K) && (fill_g[b] + ts <= dm.C);
+                    unsigned m = __ballot_sync(0xffffffffu, ok);
+                    if (m) found = b0 + __ffs(m) - 1;
+                }
+                if (found < 0) { if (tid == 0) fail_s = 1; break; }
+                if (tid == 0) { fill_g[found] += ts; cell_of[s] = found; }
+                __syncwarp();
+            }
+        }
+        __syncthreads();
+        if (!fail_s) Rstar = (int)R;
+        __syncthreads();
+    }
+    if (tid == 0) {
+        out[0] = Rstar;
+        out[1] = (Rstar != 0 && Rstar == Rlb) ? 1 : 0;
+        out[2] = (int)(Rlb > 0x7fffffff ? 0x7fffffff : Rlb);
+        out[3] = (Rstar == 0);
+    }
+}
+
+int rp_launch_pack(rp_ctx *c, int /*unused*/)
+{
+    const RpDims &dm = c->dm;
+    int n_pow2 = 1;
+    while (n_pow2 < dm.N) n_pow2 <<= 1;
+    size_t smem = (size_t)n_pow2 * sizeof(u64);
+    u64 *keys_g = nullptr;
+    if (smem > 128 * 1024) { keys_g = c->d_sort_keys; smem = 0; }
+    if (smem > 48 * 1024)
+        RP_CUDA(cudaFuncSetAttribute(k_pack_ffd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    // fill scratch: reuse the front of the sort-key buffer's tail (allocated 2*n_pow2 u64)
+    int *fill_g = (int *)(c->d_sort_keys + n_pow2);
+    k_pack_ffd<<<1, PACK_THREADS, smem, c->stream>>>(c->d_t, dm, c->cfg.min_rows, keys_g, n_pow2, fill_g,
+                                                    c->d_seed_layout, c->d_pack_out);
+    RP_CUDA(cudaGetLastError());
+    return RP_OK;
+}

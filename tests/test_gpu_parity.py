@@ -1,0 +1,331 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element.
+
+Integers, indices, placements, layouts and the whole annealing trajectory must be bit-exact;
+the reported fp64 objective must agree with the oracle's real-valued evaluation to 1e-9
+relative (the tolerance the benchmark spec states).
+"""
+import numpy as np
+import pytest
+
+import oracle
+import paper_2608_12146_b200.binding as rp
+from paper_2608_12146_b200.windows import custom_spec, make_window
+
+pytestmark = pytest.mark.gpu
+F64_RTOL = 1e-9
+
+
+def load(w, pop=None, edp=None, min_rows=0, device_inputs=False):
+    s = w.spec
+    t, a = w.lengths, w.demand
+    if device_inputs:
+        import torch
+        t, a = torch.from_numpy(t).cuda(), torch.from_numpy(a).cuda()
+    return rp.rp_window_load(t, a, top_k=s.top_k, token_cap=s.token_cap, dp_width=s.dp_width,
+                             ep_width=s.ep_width, pop_size=pop or s.pop_size, edp_of_dp=edp,
+                             alpha=s.alpha, beta=s.beta, min_rows=min_rows, seed=s.anneal_seed)
+
+
+def oracle_front(w, edp=None, min_rows=0):
+    s = w.spec
+    Lagg = oracle.aggregate(w.demand)
+    pi, G = oracle.lpt(Lagg, s.ep_width)
+    q = oracle.project(w.demand, pi, s.ep_width)
+    R, cert, seed = oracle.pack_ffd(w.lengths, s.token_cap, s.dp_width, min_rows)
+    return dict(Lagg=Lagg, pi=pi, G=G, q=q, R=R, cert=cert, seed=seed)
+
+
+def check_front(w, ctx, ref):
+    s = w.spec
+    pi, load_ = rp.rp_place_experts(ctx)
+    assert (rp.rp_debug_dump(ctx, "LAGG", (s.n_layers, s.n_experts), np.int64) == ref["Lagg"]).all()
+    assert (pi == ref["pi"]).all()
+    assert (load_ == ref["G"]).all()
+    q = rp.rp_debug_dump(ctx, "Q", (s.n_samples, s.n_layers, s.ep_width), np.int32)
+    assert (q == ref["q"]).all()
+    R, cert = rp.rp_pack_rows(ctx)
+    assert (R, cert) == (ref["R"], ref["cert"])
+    assert (rp.rp_debug_dump(ctx, "SEED_LAYOUT", (s.n_samples,), np.int32) == ref["seed"]).all()
+    return R
+
+
+def check_eval(w, ctx, ref, edp, n=6, seed=0):
+    s = w.spec
+    R, D = ref["R"], s.dp_width
+    rng = np.random.default_rng(seed)
+    lays = rng.integers(0, R * D, (n, s.n_samples)).astype(np.int32)
+    lays[0] = ref["seed"]
+    fx, f64 = rp.rp_eval_population(ctx, lays)
+    ev = oracle.eval_layouts(w.lengths, ref["q"], lays, R, s.token_cap, D, edp, s.alpha, s.beta)
+    assert (fx == ev["score"]).all()
+    G = 1 + (max(edp) if edp is not None else D - 1)
+    for j in range(n):
+        Wj = rp.rp_debug_dump(ctx, "EVAL_W", (R, G, s.n_layers, s.ep_width), np.int32, index=j)
+        assert (Wj == ev["W"][j]).all()
+        real = oracle.eval_f64(w.lengths, ref["q"], lays[j], R, s.token_cap, D, edp, s.alpha, s.beta)
+        np.testing.assert_allclose(f64[j], real, rtol=F64_RTOL, atol=0)
+
+
+def check_anneal(w, ctx, ref, edp, pop, levels, steps, threads=8, t_ratio=None, check_members=3):
+    s = w.spec
+    R, D = ref["R"], s.dp_width
+    ratio = s.t_ratio if t_ratio is None else t_ratio
+    init = np.tile(ref["seed"], (pop, 1))
+    want = oracle.anneal(w.lengths, ref["q"], init, R, s.token_cap, D, n_levels=levels, steps=steps, t0=s.t0,
+                         t_ratio=ratio, p_reloc=s.p_reloc, p_guide=s.p_guide, seed=s.anneal_seed,
+                         edp_of_dp=edp, alpha=s.alpha, beta=s.beta, n_threads=threads)
+    assert want["status"] == 0
+    stats = rp.rp_anneal(ctx, n_levels=levels, steps_per_level=steps, t0=s.t0, t_ratio=ratio,
+                         p_reloc=s.p_reloc, p_guide=s.p_guide)
+    got_counters = [stats.proposed, stats.feasible, stats.accepted, stats.improved]
+    assert got_counters == want["counters"].tolist()
+    # the whole trajectory, level by level
+    assert (rp.rp_debug_dump(ctx, "TRACE_DIGEST", (levels, pop), np.uint64) == want["digest"]).all()
+    assert (rp.rp_debug_dump(ctx, "TRACE_TERM", (levels, pop, 3), np.int64) == want["term"]).all()
+    assert (rp.rp_debug_dump(ctx, "TRACE_BEST", (levels, pop, 3), np.int64) == want["best"]).all()
+    assert (rp.rp_debug_dump(ctx, "TRACE_BEST_STEP", (levels, pop), np.int32) == want["best_step"]).all()
+    if levels > 1:
+        assert (rp.rp_debug_dump(ctx, "TRACE_ANC", (levels - 1, pop), np.int32) == want["anc"]).all()
+    assert (rp.rp_debug_dump(ctx, "TRACE_INCUMBENT", (levels, 3), np.int64) == want["incumbent"]).all()
+    # final population and the incumbent
+    popl = rp.rp_debug_dump(ctx, "POPULATION", (pop, s.n_samples), np.int32)
+    assert (popl == want["final_pop"]).all()
+    layout, fx, f64 = rp.rp_best(ctx)
+    assert (layout == want["best_layout"]).all() and (fx == want["best_score"]).all()
+    real = oracle.eval_f64(w.lengths, ref["q"], layout, R, s.token_cap, D, edp, s.alpha, s.beta)
+    np.testing.assert_allclose(f64, real, rtol=F64_RTOL, atol=0)
+    # incrementally maintained state of a few members equals the oracle's full evaluation
+    G = 1 + (max(edp) if edp is not None else D - 1)
+    for j in sorted(set([0, pop // 2, pop - 1]))[:check_members]:
+        ev = oracle.eval_layouts(w.lengths, ref["q"], popl[j], R, s.token_cap, D, edp, s.alpha, s.beta)
+        assert (rp.rp_debug_dump(ctx, "W", (R, G, s.n_layers, s.ep_width), np.int32, index=j) == ev["W"][0]).all()
+        assert (rp.rp_debug_dump(ctx, "CELL_T", (R * D,), np.int64, index=j) == ev["T"][0]).all()
+        assert (rp.rp_debug_dump(ctx, "CELL_Q", (R * D,), np.int64, index=j) == ev["Q"][0]).all()
+        assert (rp.rp_debug_dump(ctx, "CELL_CNT", (R * D,), np.int32, index=j) == ev["cnt"][0]).all()
+        assert (rp.rp_debug_dump(ctx, "ESUM", (R, G), np.int64, index=j) * (256 * s.token_cap) == ev["Efx"][0]).all()
+    # scoring the current population from scratch agrees with the last terminal scores
+    fx_pop, _ = rp.rp_eval_population(ctx)
+    assert (fx_pop == want["term"][-1]).all()
+    return want, stats
+
+
+# ---------------------------------------------------------------------------------------------
+def test_device_integer_functions_bit_exact():
+    rng = np.random.default_rng(0)
+    ctr = rng.integers(0, 2 ** 32, (4096, 4), dtype=np.uint64).astype(np.uint32)
+    ctr[0] = 0
+    ctr[1] = 0xFFFFFFFF
+    key = np.array([0xA4093822, 0x299F31D0], np.uint32)
+    got = rp.rp_debug_philox(ctr, key)
+    for i in list(range(64)) + [4095]:
+        assert (got[i] == oracle.philox4x32_10(ctr[i], key)).all()
+    x = np.concatenate([rng.integers(0, 2 ** 32, 20000, dtype=np.uint64).astype(np.uint32),
+                        np.array([0, 1, 2, 3, 2 ** 31 - 1, 2 ** 31, 2 ** 32 - 2, 2 ** 32 - 1], np.uint32),
+                        (2 ** np.arange(1, 32, dtype=np.uint64) - 1).astype(np.uint32)])
+    got = rp.rp_debug_nl2(x)
+    assert got.tolist() == [oracle.nl2(int(v)) for v in x]
+    z = np.concatenate([rng.integers(0, 34 << 32, 20000, dtype=np.uint64),
+                        np.array([0, 1, 255, 256, 2 ** 32 - 1, 2 ** 32, 32 << 32, (32 << 32) - 1, 2 ** 40, 2 ** 63], np.uint64)])
+    got = rp.rp_debug_exp2neg(z)
+    assert got.tolist() == [oracle.exp2neg(int(v)) for v in z]
+
+
+@pytest.mark.parametrize("name", ["tiny", "medium"])
+def test_named_window_full_budget(name):
+    """The two windows the oracle finishes in seconds, at their full population and sweeps."""
+    w = make_window(name)
+    s = w.spec
+    ref = oracle_front(w)
+    ctx = load(w, device_inputs=(name == "medium"))
+    check_front(w, ctx, ref)
+    check_eval(w, ctx, ref, None)
+    check_anneal(w, ctx, ref, None, s.pop_size, s.n_levels, s.steps_per_level)
+    rp.rp_destroy(ctx)
+
+
+EDGE_SPECS = [
+    # name, N, L, E, k, C, D, P, edp, min_rows   (ragged sizes, non-power-of-two ranks, shared shards)
+    ("ragged", 77, 3, 12, 2, 3000, 3, 3, None, 4),
+    ("shared_shards", 96, 5, 16, 2, 4096, 4, 4, [0, 0, 1, 1], 3),
+    ("one_shard", 64, 2, 8, 1, 2048, 4, 8, [0, 0, 0, 0], 3),
+    ("interleaved", 120, 7, 24, 3, 4096, 6, 6, [0, 1, 2, 0, 1, 2], 2),
+    ("one_rank", 50, 4, 5, 2, 2048, 2, 1, None, 4),
+    ("wide_ranks", 90, 2, 96, 2, 4096, 2, 48, None, 5),
+    ("single_slot", 40, 3, 8, 2, 2048, 1, 4, None, 6),
+    ("vector_tail", 130, 9, 40, 2, 8192, 5, 20, [0, 1, 1, 2, 2], 3),
+]
+
+
+@pytest.mark.parametrize("spec", EDGE_SPECS, ids=[e[0] for e in EDGE_SPECS])
+def test_edge_shapes(spec):
+    name, N, L, E, k, C, D, P, edp, min_rows = spec
+    w = make_window(custom_spec(name, N, L, E, k, C, D, P, 24, 400, data_seed=len(name) * 7 + N))
+    ref = oracle_front(w, edp, min_rows)
+    ctx = load(w, pop=24, edp=edp, min_rows=min_rows)
+    check_front(w, ctx, ref)
+    check_eval(w, ctx, ref, edp)
+    want, stats = check_anneal(w, ctx, ref, edp, 24, 8, 50, t_ratio=0.6)
+    assert stats.accepted > 50
+    rp.rp_destroy(ctx)
+
+
+def test_three_attention_stages_and_resume():
+    """Three stage types with fractional coefficients; a second rp_anneal call continues from
+    the population the first one left (the oracle is restarted from that population)."""
+    w = make_window(custom_spec("stages", 100, 4, 16, 2, 4096, 4, 4, 16, 300, data_seed=99,
+                                alpha=(0.5, 2.25, 1.0), beta=(0.0, 0.75, 3.0)))
+    s = w.spec
+    edp = [0, 0, 1, 1]
+    ref = oracle_front(w, edp, 3)
+    ctx = load(w, pop=16, edp=edp, min_rows=3)
+    check_front(w, ctx, ref)
+    check_eval(w, ctx, ref, edp)
+    want, _ = check_anneal(w, ctx, ref, edp, 16, 5, 40, t_ratio=0.5)
+    # resume
+    again = oracle.anneal(w.lengths, ref["q"], want["final_pop"], ref["R"], s.token_cap, s.dp_width, n_levels=3,
+                          steps=30, t0=1e-4, t_ratio=0.5, p_reloc=0.5, p_guide=0.3, seed=s.anneal_seed,
+                          edp_of_dp=edp, alpha=s.alpha, beta=s.beta)
+    rp.rp_anneal(ctx, n_levels=3, steps_per_level=30, t0=1e-4, t_ratio=0.5, p_reloc=0.5, p_guide=0.3)
+    assert (rp.rp_debug_dump(ctx, "TRACE_TERM", (3, 16, 3), np.int64) == again["term"]).all()
+    assert (rp.rp_debug_dump(ctx, "POPULATION", (16, s.n_samples), np.int32) == again["final_pop"]).all()
+    _, fx, _ = rp.rp_best(ctx)
+    assert tuple(fx) == min(tuple(want["best_score"]), tuple(again["best_score"]))
+    rp.rp_destroy(ctx)
+
+
+@pytest.mark.parametrize("name,pop,levels,steps", [("large", 96, 3, 60), ("wide", 48, 2, 40), ("heavy", 64, 2, 80)])
+def test_large_windows_full_shapes_reduced_budget(name, pop, levels, steps):
+    """Full N, L, E, P, C, D of the three big windows (so the kernels run in the launch
+    configuration of the full-size runs), with a population and step budget the oracle finishes
+    quickly; every trajectory is still compared bit for bit."""
+    w = make_window(name)
+    ref = oracle_front(w)
+    ctx = load(w, pop=pop, device_inputs=True)
+    check_front(w, ctx, ref)
+    check_eval(w, ctx, ref, None, n=2)
+    check_anneal(w, ctx, ref, None, pop, levels, steps, check_members=2)
+    rp.rp_destroy(ctx)
+
+
+def test_full_size_properties_large():
+    """Large at its full population and sweeps: properties that hold at any size (feasibility
+    of every member, cached scores equal to a full rescoring, monotone incumbent, conserved
+    rank loads), plus the oracle's evaluation of sampled members."""
+    w = make_window("large")
+    s = w.spec
+    ref = oracle_front(w)
+    ctx = load(w, device_inputs=True)
+    R = check_front(w, ctx, ref)
+    stats = rp.rp_anneal(ctx, n_levels=s.n_levels, steps_per_level=s.steps_per_level, t0=s.t0, t_ratio=s.t_ratio,
+                         p_reloc=s.p_reloc, p_guide=s.p_guide)
+    assert stats.proposed == s.pop_size * s.sweeps
+    K = R * s.dp_width
+    popl = rp.rp_debug_dump(ctx, "POPULATION", (s.pop_size, s.n_samples), np.int32)
+    assert popl.min() >= 0 and popl.max() < K
+    for j in range(0, s.pop_size, 37):
+        assert (np.bincount(popl[j], minlength=K) >= 1).all()
+        assert (np.bincount(popl[j], weights=w.lengths, minlength=K) <= s.token_cap).all()
+    term = rp.rp_debug_dump(ctx, "TRACE_TERM", (s.n_levels, s.pop_size, 3), np.int64)
+    fx_pop, _ = rp.rp_eval_population(ctx)
+    assert (fx_pop == term[-1]).all()
+    inc = [tuple(x) for x in rp.rp_debug_dump(ctx, "TRACE_INCUMBENT", (s.n_levels, 3), np.int64)]
+    assert all(b <= a for a, b in zip(inc, inc[1:]))
+    for j in (0, 511, 1023):
+        ev = oracle.eval_layouts(w.lengths, ref["q"], popl[j], R, s.token_cap, s.dp_width)
+        assert tuple(ev["score"][0]) == tuple(term[-1, j])
+        Wj = rp.rp_debug_dump(ctx, "W", (R, s.dp_width, s.n_layers, s.ep_width), np.int32, index=j)
+        assert (Wj == ev["W"][0]).all()
+        assert (Wj.sum(axis=(0, 1)) == ref["G"]).all()          # aggregate invariance
+    layout, fx, f64 = rp.rp_best(ctx)
+    ev = oracle.eval_layouts(w.lengths, ref["q"], layout, R, s.token_cap, s.dp_width)
+    assert tuple(ev["score"][0]) == tuple(fx) == inc[-1]
+    seed_score = oracle.eval_layouts(w.lengths, ref["q"], ref["seed"], R, s.token_cap, s.dp_width)["score"][0]
+    assert tuple(fx) <= tuple(seed_score)
+    rp.rp_destroy(ctx)
+
+
+def test_bad_inputs_are_host_side_errors():
+    w = make_window("tiny")
+    s = w.spec
+    kw = dict(top_k=s.top_k, token_cap=s.token_cap, dp_width=s.dp_width, ep_width=s.ep_width, pop_size=4)
+    bad = w.demand.copy()
+    bad[7, 2, 3] += 1
+    with pytest.raises(rp.RpError) as e:
+        rp.rp_window_load(w.lengths, bad, **kw)
+    assert e.value.status == -3
+    neg = w.demand.copy()
+    neg[3, 0, 0] -= 5
+    neg[3, 0, 1] += 5
+    if neg[3, 0, 0] < 0:
+        with pytest.raises(rp.RpError) as e:
+            rp.rp_window_load(w.lengths, neg, **kw)
+        assert e.value.status == -3
+    long_ = w.lengths.copy()
+    long_[0] = s.token_cap + 1
+    with pytest.raises(rp.RpError) as e:
+        rp.rp_window_load(long_, w.demand, **kw)
+    assert e.value.status == -3
+    with pytest.raises(rp.RpError) as e:
+        rp.rp_window_load(w.lengths, w.demand, **dict(kw, ep_width=3))
+    assert e.value.status == -2
+    with pytest.raises(rp.RpError) as e:
+        rp.rp_window_load(w.lengths[:1], w.demand[:1], **kw)
+    assert e.value.status == -2
+    with pytest.raises(rp.RpError) as e:
+        rp.rp_window_load(w.lengths, w.demand, edp_of_dp=[0, 2], **kw)      # shard 1 unused
+    assert e.value.status == -2
+    ctx = rp.rp_window_load(w.lengths, w.demand, **kw)
+    with pytest.raises(rp.RpError) as e:
+        rp.rp_pack_rows(ctx)                                                 # before rp_place_experts
+    assert e.value.status == -7
+    rp.rp_place_experts(ctx)
+    with pytest.raises(rp.RpError) as e:
+        rp.rp_anneal(ctx, n_levels=1, steps_per_level=1, t0=1e-3, t_ratio=0.5, p_reloc=0.2, p_guide=0.8)
+    assert e.value.status == -7
+    R, _ = rp.rp_pack_rows(ctx)
+    lay = np.zeros((1, s.n_samples), np.int32)
+    lay[0, 5] = R * s.dp_width
+    with pytest.raises(rp.RpError) as e:
+        rp.rp_eval_population(ctx, lay)
+    assert e.value.status == -1
+    with pytest.raises(rp.RpError) as e:
+        rp.rp_anneal(ctx, n_levels=0, steps_per_level=1, t0=1e-3, t_ratio=0.5, p_reloc=0.2, p_guide=0.8)
+    assert e.value.status == -1
+    rp.rp_destroy(ctx)
+    # infeasible: more DP slots than one-sample cells can fill at this cap is fine, but a window
+    # whose samples cannot be split into non-empty cells within the cap is reported, not trapped
+    t = np.full(6, 10, np.int32)
+    a = np.zeros((6, 1, 2), np.int32)
+    a[:, 0, 0] = 10
+    ctx = rp.rp_window_load(t, a, top_k=1, token_cap=10, dp_width=4, ep_width=2, pop_size=2)
+    rp.rp_place_experts(ctx)
+    with pytest.raises(rp.RpError) as e:
+        rp.rp_pack_rows(ctx)          # 6 samples of a full cell each need 6 cells; 4 and 8 are the only shapes
+    assert e.value.status == -4
+    rp.rp_destroy(ctx)
+
+
+def test_smallest_window_and_empty_moves():
+    """N == D, one row, one sample per cell: every proposal is infeasible (same cell, or a
+    relocation that would empty a cell, or a swap over the cap) or a legal swap."""
+    t = np.array([5, 9, 3, 7], np.int32)
+    a = np.zeros((4, 2, 4), np.int32)
+    rng = np.random.default_rng(5)
+    for i in range(4):
+        for l in range(2):
+            a[i, l] = rng.multinomial(2 * t[i], [0.1, 0.2, 0.3, 0.4])
+    pi, G = oracle.lpt(oracle.aggregate(a), 2)
+    q = oracle.project(a, pi, 2)
+    R, cert, seed = oracle.pack_ffd(t, 16, 4)
+    assert R == 1
+    ctx = rp.rp_window_load(t, a, top_k=2, token_cap=16, dp_width=4, ep_width=2, pop_size=3, seed=11)
+    rp.rp_place_experts(ctx)
+    assert rp.rp_pack_rows(ctx) == (R, cert)
+    want = oracle.anneal(t, q, np.tile(seed, (3, 1)), R, 16, 4, n_levels=4, steps=30, t0=1e-2, t_ratio=0.5,
+                         p_reloc=0.3, p_guide=0.8, seed=11)
+    stats = rp.rp_anneal(ctx, n_levels=4, steps_per_level=30, t0=1e-2, t_ratio=0.5, p_reloc=0.3, p_guide=0.8)
+    assert [stats.proposed, stats.feasible, stats.accepted, stats.improved] == want["counters"].tolist()
+    assert (rp.rp_debug_dump(ctx, "TRACE_DIGEST", (4, 3), np.uint64) == want["digest"]).all()
+    layout, fx, _ = rp.rp_best(ctx)
+    assert (layout == want["best_layout"]).all() and (fx == want["best_score"]).all()
+    rp.rp_destroy(ctx)
