@@ -1,0 +1,346 @@
+#!/usr/bin/env python
+"""Benchmark of the RoutePack planner hot path on B200.
+
+A "step" is one complete plan of one synthetic optimizer-step window: input checks and
+aggregate demand, LPT placement, demand projection, row count + seed, population annealing
+over all temperature levels, validation and return of the best layout.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload medium] [--impl reference]
+
+Prints ONE JSON line.  `value` = replica-moves evaluated per second over the whole timed
+region (all stages, inputs resident in HBM); `e2e` = the same with host buffers in and out
+through the C ABI; `roofline` = the per-level chain kernel against the measured HBM peak;
+`cpu_baseline` = the C oracle on this machine's host cores.  With N > 1 every rank plans its own
+copy of the window (replicas only, no collective on the data path).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+from paper_2608_12146_b200.windows import SPECS, make_window
+
+METRIC = "annealing replica-moves evaluated/sec"
+UNIT = "moves/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def hbm_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+def workload_config(spec, extra=None):
+    cfg = {"workload": spec.name, "n_samples": spec.n_samples, "n_layers": spec.n_layers,
+           "n_experts": spec.n_experts, "top_k": spec.top_k, "token_cap": spec.token_cap,
+           "dp_shards": spec.dp_width, "ep_ranks": spec.ep_width, "population": spec.pop_size,
+           "sweeps": spec.sweeps, "n_levels": spec.n_levels, "steps_per_level": spec.steps_per_level,
+           "l2": "flushed between steps (256 MiB write)"}
+    if extra:
+        cfg.update(extra)
+    return cfg
+
+
+# ---------------------------------------------------------------------------------------------
+# reference arm: the oracle on the host cores
+# ---------------------------------------------------------------------------------------------
+def oracle_sample(w, threads, budget_moves=3.0e6):
+    """Run the oracle on a bounded sample of the workload: the whole front end once, then
+    annealing at the full population for as many whole levels as fit the move budget."""
+    import oracle
+    s = w.spec
+    per_level = s.pop_size * s.steps_per_level
+    levels = int(max(1, min(s.n_levels, budget_moves // per_level)))
+    t0 = time.perf_counter()
+    res = oracle.plan(w, n_levels=levels, n_threads=threads, trace=False)
+    dt = time.perf_counter() - t0
+    moves = int(res["counters"][0])
+    sample = (f"whole front end + {levels} of {s.n_levels} temperature levels at the full population "
+              f"({moves} replica-moves)")
+    return moves, dt, sample
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import oracle
+    oracle.build()
+    spec = SPECS[args.workload]
+    w = make_window(spec)
+    threads = os.cpu_count() or 1
+    budget = {"tiny": 1e5, "medium": 3e6, "large": 6e6, "wide": 3e6, "heavy": 8e6}[spec.name]
+    for _ in range(args.warmup):
+        oracle_sample(w, threads, budget)
+    moves = 0
+    dt = 0.0
+    sample = ""
+    for _ in range(args.steps):
+        m, d, sample = oracle_sample(w, threads, budget)
+        moves += m
+        dt += d
+    value = moves / dt
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
+            "data": "synthetic", "config": workload_config(spec),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+# ---------------------------------------------------------------------------------------------
+# CUDA arm
+# ---------------------------------------------------------------------------------------------
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index):
+        self.idx = device_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.idx)],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        for line in out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def plan_once(rp, torch, w, t_in, a_in, outs, stream, want_stats=True):
+    """One pass of the whole hot path through the C ABI; returns the annealing stats."""
+    s = w.spec
+    ctx = rp.rp_window_load(t_in, a_in, top_k=s.top_k, token_cap=s.token_cap, dp_width=s.dp_width,
+                            ep_width=s.ep_width, pop_size=s.pop_size, alpha=s.alpha, beta=s.beta,
+                            seed=s.anneal_seed, stream=stream)
+    rp.rp_place_experts(ctx, outs["pi"], outs["rank_load"])
+    rp.rp_pack_rows(ctx)
+    stats = rp.rp_anneal(ctx, n_levels=s.n_levels, steps_per_level=s.steps_per_level, t0=s.t0,
+                         t_ratio=s.t_ratio, p_reloc=s.p_reloc, p_guide=s.p_guide, want_stats=want_stats)
+    rp.rp_best(ctx, outs["layout"], outs["score_fx"], outs["score_f64"])
+    rp.rp_destroy(ctx)
+    return stats
+
+
+def run_cuda(args):
+    import torch
+    import paper_2608_12146_b200.binding as rp
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path); use --impl reference for the oracle")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    rp.lib()
+
+    spec = SPECS[args.workload]
+    w = make_window(spec)
+    s = spec
+    moves_per_step = s.pop_size * s.n_levels * s.steps_per_level
+    stream = torch.cuda.current_stream()
+    dev = torch.device("cuda", local)
+    t_dev = torch.from_numpy(w.lengths).to(dev)
+    a_dev = torch.from_numpy(w.demand).to(dev)
+    t_pin = torch.from_numpy(w.lengths).pin_memory()
+    a_pin = torch.from_numpy(w.demand).pin_memory()
+    outs_dev = dict(pi=torch.empty((s.n_layers, s.n_experts), dtype=torch.int32, device=dev),
+                    rank_load=torch.empty((s.n_layers, s.ep_width), dtype=torch.int64, device=dev),
+                    layout=torch.empty(s.n_samples, dtype=torch.int32, device=dev),
+                    score_fx=torch.empty(3, dtype=torch.int64, device=dev),
+                    score_f64=torch.empty(3, dtype=torch.float64, device=dev))
+    outs_host = dict(pi=torch.empty((s.n_layers, s.n_experts), dtype=torch.int32).pin_memory(),
+                     rank_load=torch.empty((s.n_layers, s.ep_width), dtype=torch.int64).pin_memory(),
+                     layout=torch.empty(s.n_samples, dtype=torch.int32).pin_memory(),
+                     score_fx=torch.empty(3, dtype=torch.int64).pin_memory(),
+                     score_f64=torch.empty(3, dtype=torch.float64).pin_memory())
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed_loop(t_in, a_in, outs, steps):
+        """K steps, each timed with CUDA events on the launching stream; L2 flushed in between."""
+        total_ms, chain_ms, barrier_ms = 0.0, 0.0, 0.0
+        move_bytes = gather_bytes = feasible = accepted = chain_launches = 0
+        barrier()
+        wall0 = time.perf_counter()
+        for _ in range(steps):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            st = plan_once(rp, torch, w, t_in, a_in, outs, stream)
+            e1.record(stream)
+            e1.synchronize()
+            total_ms += e0.elapsed_time(e1)
+            chain_ms += st.ms_chains
+            barrier_ms += st.ms_barrier
+            move_bytes += st.move_bytes
+            gather_bytes += st.gather_bytes
+            feasible += st.feasible
+            accepted += st.accepted
+            chain_launches += s.n_levels
+        barrier()
+        wall = time.perf_counter() - wall0
+        return dict(ms=total_ms, wall=wall, chain_ms=chain_ms, barrier_ms=barrier_ms, move_bytes=move_bytes,
+                    gather_bytes=gather_bytes, feasible=feasible, accepted=accepted, chain_launches=chain_launches)
+
+    for _ in range(args.warmup):
+        plan_once(rp, torch, w, t_dev, a_dev, outs_dev, stream)
+        plan_once(rp, torch, w, t_pin, a_pin, outs_host, stream)
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+    vis_ids = [x for x in vis.split(",") if x]
+    sampler = ClockSampler(vis_ids[local] if local < len(vis_ids) else local)
+    sampler.start()
+    launches0 = rp.rp_debug_launch_count()
+    res = timed_loop(t_dev, a_dev, outs_dev, args.steps)
+    launches = rp.rp_debug_launch_count() - launches0
+    clocks = sampler.stop()
+    e2e = timed_loop(t_pin, a_pin, outs_host, args.steps)
+
+    def max_over_ranks(x):
+        if dist is None:
+            return x
+        tt = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        return float(tt.item())
+
+    ms = max_over_ranks(res["ms"])
+    ms_e2e = max_over_ranks(e2e["ms"])
+    total_moves = moves_per_step * args.steps * world
+    value = total_moves / (ms * 1e-3)
+    e2e_value = total_moves / (ms_e2e * 1e-3)
+
+    peak, peak_kind = hbm_peak()
+    per_launch_s = res["chain_ms"] * 1e-3 / res["chain_launches"]
+    alg_bytes_per_launch = (res["move_bytes"] + res["gather_bytes"]) / res["chain_launches"]
+    achieved = alg_bytes_per_launch / per_launch_s / 1e9
+    roofline = {"bound": "hbm", "kernel": "k_anneal_level", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_source": peak_kind, "traffic": None,
+                "algorithmic_bytes_per_launch": alg_bytes_per_launch,
+                "move_bytes_per_launch": res["move_bytes"] / res["chain_launches"],
+                "gather_bytes_per_launch": res["gather_bytes"] / res["chain_launches"],
+                "launch_ms": per_launch_s * 1e3,
+                "share_of_step": res["chain_ms"] / res["ms"]}
+    traffic_file = os.path.join(ROOT, "profiles", f"traffic_{spec.name}.json")
+    if os.path.exists(traffic_file):
+        try:
+            roofline["traffic"] = json.load(open(traffic_file))["dram_bytes_per_launch"]
+        except Exception:
+            pass
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return 0
+
+    # CPU baseline: the oracle as it stands on this machine's cores (rank 0, N=1 only)
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        threads = os.cpu_count() or 1
+        budget = {"tiny": 1e5, "medium": 2e7, "large": 2e7, "wide": 6e6, "heavy": 2e7}[spec.name]
+        oracle_sample(w, threads, min(budget, 1e6))           # warm the page cache and the thread pool
+        m, d, reps = 0, 0.0, 0
+        while d < 2.0 and reps < 64:                          # a few seconds of wall time on all cores
+            mi, di, sample = oracle_sample(w, threads, budget)
+            m, d, reps = m + mi, d + di, reps + 1
+        cpu = {"value": m / d, "unit": UNIT, "cores": threads, "kind": "oracle",
+               "sample": f"{reps} x ({sample})", "seconds": d}
+
+    h2d = int(w.lengths.nbytes + w.demand.nbytes)
+    d2h = int(sum(v.numel() * v.element_size() for v in outs_host.values()))
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+            "config": workload_config(spec, {"parallelism": "replicas only" if world > 1 else "1 gpu"}),
+            "plans_per_s": args.steps * world / (ms * 1e-3),
+            "anneal_only_moves_per_s": moves_per_step * args.steps / ((res["chain_ms"] + res["barrier_ms"]) * 1e-3),
+            "feasible_fraction": res["feasible"] / (moves_per_step * args.steps),
+            "accepted_fraction": res["accepted"] / (moves_per_step * args.steps),
+            "stage_ms_per_step": {"chains": res["chain_ms"] / args.steps, "level_barrier": res["barrier_ms"] / args.steps,
+                                  "other": (res["ms"] - res["chain_ms"] - res["barrier_ms"]) / args.steps},
+            "roofline": roofline,
+            "cpu_baseline": cpu,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": ms_e2e / args.steps},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+            "wall_s": res["wall"]}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="medium", choices=list(SPECS))
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "cuda":
+        args.warmup = 3
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_cuda(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

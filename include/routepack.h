@@ -81,6 +81,11 @@ typedef struct {
     int64_t proposed, feasible, accepted, improved;  /* summed over chains and levels       */
     double ms_chains;           /* device time in the per-level chain kernels               */
     double ms_barrier;          /* device time in incumbent update + resampling             */
+    int64_t move_bytes;         /* algorithmic bytes of the feasible moves: rank-load slices
+                                   and demand rows read, slices written on accept           */
+    int64_t gather_bytes;       /* rank-load bytes read+written for members that resampling
+                                   replaced by another member's state                       */
+    int64_t kernel_launches;    /* kernels this call launched                                */
 } rp_anneal_stats;
 
 /* Routing-replay input (Eq. routing-replay-input): creates a context, copies host arrays
@@ -165,6 +170,8 @@ int rp_debug_nl2(const uint32_t *x, uint64_t *out, int64_t n);
 int rp_debug_exp2neg(const uint64_t *z, uint64_t *out, int64_t n);
 /* out[i][0..3] = Philox4x32-10(counter ctr[i][0..3], key) on the device. */
 int rp_debug_philox(const uint32_t *ctr, const uint32_t key[2], uint32_t *out, int64_t n);
+/* Number of kernels this library has launched in this process so far. */
+int64_t rp_debug_launch_count(void);
 
 #ifdef __cplusplus
 }

@@ -24,7 +24,7 @@ RP_OK = 0
 
 EXPORTS = ("rp_window_load", "rp_place_experts", "rp_pack_rows", "rp_eval_population", "rp_anneal",
            "rp_best", "rp_destroy", "rp_strerror", "rp_last_cuda_error", "rp_debug_dump",
-           "rp_debug_nl2", "rp_debug_exp2neg", "rp_debug_philox")
+           "rp_debug_nl2", "rp_debug_exp2neg", "rp_debug_philox", "rp_debug_launch_count")
 
 
 class RpError(RuntimeError):
@@ -50,7 +50,8 @@ class rp_anneal_params(C.Structure):
 
 class rp_anneal_stats(C.Structure):
     _fields_ = [("proposed", C.c_int64), ("feasible", C.c_int64), ("accepted", C.c_int64),
-                ("improved", C.c_int64), ("ms_chains", C.c_double), ("ms_barrier", C.c_double)]
+                ("improved", C.c_int64), ("ms_chains", C.c_double), ("ms_barrier", C.c_double),
+                ("move_bytes", C.c_int64), ("gather_bytes", C.c_int64), ("kernel_launches", C.c_int64)]
 
 
 def library_path() -> str:
@@ -80,6 +81,7 @@ def lib():
         L.rp_debug_nl2.argtypes = [C.c_void_p, C.c_void_p, C.c_int64]
         L.rp_debug_exp2neg.argtypes = [C.c_void_p, C.c_void_p, C.c_int64]
         L.rp_debug_philox.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64]
+        L.rp_debug_launch_count.restype = C.c_int64
         _lib = L
     return _lib
 
@@ -227,6 +229,10 @@ def rp_debug_exp2neg(z) -> np.ndarray:
     out = np.empty(z.shape, np.uint64)
     _check(lib().rp_debug_exp2neg(_ptr(z), _ptr(out), z.size), "rp_debug_exp2neg")
     return out
+
+
+def rp_debug_launch_count() -> int:
+    return int(lib().rp_debug_launch_count())
 
 
 def rp_debug_philox(ctr, key) -> np.ndarray:

@@ -4,39 +4,31 @@
 // validation (K8).
 //
 // Mapping.  One CTA runs one chain for all K steps of a level.  The chain's small state
-// (assignment, cell statistics, per-row-shard costs, shard work) lives in shared memory;
-// its rank-load tensor W[R][G][L][P] lives in global memory (L2/HBM) and is touched two
-// slices per feasible move.  The sample demand rows q[i][L][P] are shared by all chains and
-// stay L2-resident.  Resampling is folded into the next level's prologue: slot j starts
-// from the terminal state of its ancestor in the other population buffer, so no separate
-// gather pass runs.  Trajectory-best layouts are not copied: every accepted move is logged
-// (8 bytes) and the level barrier rebuilds the one winning layout from the chain's start
-// layout and its log prefix.
+// (assignment, cell statistics, per-row-shard costs, shard work) lives in shared memory.
+// Its rank-load tensor W[R][G][L][P] lives in shared memory too when it fits beside a
+// second CTA on the SM (small windows: the chain is latency-bound), else in global memory
+// (L2/HBM; large windows: the chain is bandwidth-bound and many CTAs per SM hide latency).
+// The sample demand rows q[i][L][P] are shared by all chains and stay L2-resident.
+//
+// A chain is a sequential process, but three things about it are not:
+//  * every random number is a pure function of (step, level, slot), so the proposal words
+//    and the accept threshold -log2(u)*T of the next 32 steps are computed by 32 lanes at once;
+//  * a proposal depends on the chain state, which changes only when a move is ACCEPTED, so
+//    32 lanes evaluate the proposals and feasibility of the next 32 steps against the current
+//    state at once; infeasible steps are skipped in bulk, feasible ones are scored in step
+//    order, and the speculation is redone only after an acceptance (the result is identical
+//    to stepping one by one);
+//  * scoring a move is a data-parallel pass over two L*P slices.
+// Resampling is folded into the next level's prologue: slot j starts from the terminal
+// state of its ancestor in the other population buffer, so no separate gather pass runs.
+// Trajectory-best layouts are not copied: every accepted move is logged (8 bytes) and the
+// level barrier rebuilds the one winning layout from the chain's start layout and its log.
 //
 // Algorithmic bytes per feasible move: reads 2 W slices + the moved samples' q rows
 // ((3 or 4) * L*P*4 bytes), writes 2 W slices when accepted.
-#include "rp_score.cuh"
+#include "rp_anneal.cuh"
 
-struct AnnealArgs {
-    RpDims dm;
-    const int *t, *q, *edp, *dp_list, *dp_off;
-    const unsigned short *cell_src;  unsigned short *cell_dst;
-    const int *W_src;                int *W_dst;
-    const i64 *Esum_src;             i64 *Esum_dst;
-    const int *anc;
-    int level, steps, t_in_smem, log_cap;
-    u64 tau, rho_q32, guide_q32;
-    u32 key0, key1;
-    i64 *term, *best;
-    int *best_step, *best_nlog;
-    u64 *digest;
-    uint2 *log;
-    i64 *counters;
-};
-
-struct MoveRec {
-    int feasible, reloc, i, i2, c1, c2, rg1, rg2, accept;
-};
+struct RoundS { unsigned fmask; int accept; int fallback; };
 
 template <int NT>
 __device__ __forceinline__ void block_sync()
@@ -44,286 +36,273 @@ __device__ __forceinline__ void block_sync()
     if (NT == 32) __syncwarp(); else __syncthreads();
 }
 
-template <int NT>
+template <int NT, bool WS>
 __global__ void __launch_bounds__(NT)
 k_anneal_level(const AnnealArgs A)
 {
     const RpDims &dm = A.dm;
     extern __shared__ __align__(16) unsigned char smraw[];
-    // Q[K] | Esum[RG] | Afx[RG] | Jfx[RG] | U[G] | red[2*NT/32] | T[K] | cnt[K] | scratch[2*LP] | t_s[N]? | cell_of[N] | mv
+    // 8-byte: Q[K] Esum[RG] Afx[RG] Jfx[RG] U[G] red[2*NT/32] recs[SPEC]
+    // 4-byte: T[K] cnt[K] scratch[2*LP] dp_list[D] dp_off[G+1] mvs[SPEC] round t_s[N]? W[RG*LP]?
+    // 2-byte: cell_of[N] rg_of[K] g_of[K] rowbase[K]
     u64 *Q = (u64 *)smraw;
     i64 *Esum = (i64 *)(Q + dm.K);
     i64 *Afx = Esum + dm.RG;
     i64 *Jfx = Afx + dm.RG;
     i64 *U = Jfx + dm.RG;
     i64 *red = U + dm.G;
-    int *T = (int *)(red + 2 * (NT / 32));
+    StepRec *recs = (StepRec *)(red + 2 * (NT / 32));
+    int *scratch = (int *)(((uintptr_t)(recs + SPEC) + 15) & ~(uintptr_t)15);     // 16-byte aligned slices
+    const size_t slice_pad = ((size_t)dm.LP + 3) & ~(size_t)3;
+    int *Wsm = scratch + 2 * slice_pad;
+    int *T = Wsm + (WS ? (((size_t)dm.RG * dm.LP + 3) & ~(size_t)3) : 0);
     int *cnt = T + dm.K;
-    int *scratch = cnt + dm.K;
-    int *t_s = scratch + 2 * dm.LP;
+    int *dpl = cnt + dm.K;
+    int *dpo = dpl + dm.D;
+    MoveS *mvs = (MoveS *)(dpo + dm.G + 1);
+    RoundS *rnd = (RoundS *)(mvs + SPEC);
+    int *t_s = (int *)(rnd + 1);
     unsigned short *cell_of = (unsigned short *)(t_s + (A.t_in_smem ? dm.N : 0));
-    MoveRec *mv = (MoveRec *)(((uintptr_t)(cell_of + dm.N) + 15) & ~(uintptr_t)15);
+    unsigned short *rg_of = cell_of + dm.N;
+    unsigned short *g_of = rg_of + dm.K;
+    unsigned short *rowbase = g_of + dm.K;
     RpSmemState st = { cell_of, T, Q, cnt, Esum, Afx, U };
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int j = blockIdx.x;
     const int src = A.anc[j];
     const int *tt = A.t_in_smem ? t_s : A.t;
+    const bool identity_edp = (dm.G == dm.D);
+    const size_t wn = (size_t)dm.RG * dm.LP;
+    int *Wj = WS ? Wsm : A.W_dst + (size_t)j * wn;
 
     // ---- prologue: adopt the ancestor's terminal state -------------------------------
     {
         const unsigned short *cs = A.cell_src + (size_t)src * dm.N;
         for (int i = tid; i < dm.N; i += NT) cell_of[i] = cs[i];
         if (A.t_in_smem) for (int i = tid; i < dm.N; i += NT) t_s[i] = A.t[i];
-        for (int c = tid; c < dm.K; c += NT) { T[c] = 0; Q[c] = 0; cnt[c] = 0; }
+        for (int c = tid; c < dm.K; c += NT) {
+            T[c] = 0; Q[c] = 0; cnt[c] = 0;
+            const int r = c / dm.D, g = A.edp[c % dm.D];
+            rg_of[c] = (unsigned short)(r * dm.G + g);
+            g_of[c] = (unsigned short)g;
+            rowbase[c] = (unsigned short)(r * dm.D);
+        }
+        for (int d = tid; d < dm.D; d += NT) dpl[d] = A.dp_list[d];
+        for (int g = tid; g <= dm.G; g += NT) dpo[g] = A.dp_off[g];
         const i64 *es = A.Esum_src + (size_t)src * dm.RG;
         for (int rg = tid; rg < dm.RG; rg += NT) Esum[rg] = es[rg];
-        const size_t wn = (size_t)dm.RG * dm.LP;
         const int *ws = A.W_src + (size_t)src * wn;
-        int *wd = A.W_dst + (size_t)j * wn;
         if ((wn & 3) == 0) {
             const int4 *ws4 = (const int4 *)ws;
-            int4 *wd4 = (int4 *)wd;
+            int4 *wd4 = (int4 *)Wj;
+#pragma unroll 8
             for (size_t x = tid; x < wn / 4; x += NT) wd4[x] = ws4[x];
         } else {
-            for (size_t x = tid; x < wn; x += NT) wd[x] = ws[x];
+            for (size_t x = tid; x < wn; x += NT) Wj[x] = ws[x];
         }
     }
     __syncthreads();
     rp_accumulate_cells(dm, st, A.t, tid, NT);
     __syncthreads();
     i64 S[3];
-    rp_rows_to_score(dm, st, A.dp_list, A.dp_off, tid, NT, S);
+    rp_rows_to_score(dm, st, dpl, dpo, tid, NT, S);
     for (int rg = tid; rg < dm.RG; rg += NT) Jfx[rg] = Afx[rg] + dm.EC * Esum[rg];
     __syncthreads();
 
-    int *Wj = A.W_dst + (size_t)j * dm.RG * dm.LP;
     // chain bookkeeping (thread 0 only)
     i64 B0 = S[0], B1 = S[1], B2 = S[2];
+    i64 Ecur = (tid == 0) ? rp_energy(S[0], S[1], S[2]) : 0;
     int best_step = 0, best_nlog = 0, nlog = 0;
     u64 dig = 0;
-    i64 n_feas = 0, n_acc = 0, n_imp = 0;
+    i64 n_feas = 0, n_acc = 0, n_imp = 0, n_bytes = 0;
     uint2 *logj = A.log + (size_t)j * A.log_cap;
+    const i64 aC = dm.asum * dm.C, bS = dm.bsum;
+    const RpChainView view = { cell_of, rg_of, T, cnt, tt, Q, Jfx, Afx };
+    const bool vec = (dm.P >= 4) && (dm.P <= 128) && ((dm.P & (dm.P - 1)) == 0);
 
-    for (int k = 0; k < A.steps; ++k) {
-        // ---- phase 1: proposal and feasibility (thread 0) -----------------------------
-        if (tid == 0) {
-            const uint4 a = rp_philox((u32)k, (u32)A.level, (u32)j, 0u, A.key0, A.key1);
-            const bool reloc = (u64)a.x < A.rho_q32;
-            const bool guided = (u64)a.y < A.guide_q32;
-            int i, i2 = -1, c1, c2;
-            if (!guided) {
-                i = rp_pick(a.z, dm.N);
-                c1 = cell_of[i];
-                if (reloc) c2 = rp_pick(a.w, dm.K);
-                else { i2 = rp_pick(a.w, dm.N); c2 = cell_of[i2]; }
-            } else {
-                const uint4 b = rp_philox((u32)k, (u32)A.level, (u32)j, 1u, A.key0, A.key1);
-                const int sa = rp_pick(a.z, dm.N), sb = rp_pick(a.w, dm.N);
-                const int ca = cell_of[sa], cb = cell_of[sb];
-                const int rga = rp_rowshard(dm, A.edp, ca);
-                const u64 Ja = (u64)Jfx[rga], Aa = (u64)Afx[rga];
-                // attention key with probability Afx/Jfx:  b.z * Ja < Aa * 2^32  (128-bit compare)
-                const u64 lh = __umul64hi((u64)b.z, Ja), ll = (u64)b.z * Ja;
-                const u64 rh = Aa >> 32, rl = Aa << 32;
-                const bool use_att = (lh < rh) || (lh == rh && ll < rl);
-                i64 ka, kb;
-                if (use_att) {
-                    ka = dm.asum * dm.C * (i64)T[ca] + dm.bsum * (i64)Q[ca];
-                    kb = dm.asum * dm.C * (i64)T[cb] + dm.bsum * (i64)Q[cb];
-                } else {
-                    ka = (i64)Ja;
-                    kb = Jfx[rp_rowshard(dm, A.edp, cb)];
-                }
-                i = (kb > ka) ? sb : sa;
-                c1 = (kb > ka) ? cb : ca;
-                if (reloc) {
-                    const int xa = rp_pick(b.x, dm.K), xb = rp_pick(b.y, dm.K);
-                    i64 ta, tb;
-                    if (use_att) {
-                        ta = dm.asum * dm.C * (i64)T[xa] + dm.bsum * (i64)Q[xa];
-                        tb = dm.asum * dm.C * (i64)T[xb] + dm.bsum * (i64)Q[xb];
-                    } else {
-                        ta = Jfx[rp_rowshard(dm, A.edp, xa)];
-                        tb = Jfx[rp_rowshard(dm, A.edp, xb)];
-                    }
-                    c2 = (tb < ta) ? xb : xa;
-                } else {
-                    const int ya = rp_pick(b.x, dm.N), yb = rp_pick(b.y, dm.N);
-                    const int xa = cell_of[ya], xb = cell_of[yb];
-                    i64 ta, tb;
-                    if (use_att) {
-                        ta = dm.asum * dm.C * (i64)T[xa] + dm.bsum * (i64)Q[xa];
-                        tb = dm.asum * dm.C * (i64)T[xb] + dm.bsum * (i64)Q[xb];
-                    } else {
-                        ta = Jfx[rp_rowshard(dm, A.edp, xa)];
-                        tb = Jfx[rp_rowshard(dm, A.edp, xb)];
-                    }
-                    i2 = (tb < ta) ? yb : ya;
-                    c2 = (tb < ta) ? xb : xa;
-                }
-            }
-            bool ok = (c1 != c2);
-            if (ok) {
-                const int ti = tt[i];
-                if (reloc) ok = (cnt[c1] > 1) && (T[c2] + ti <= dm.C);
-                else {
-                    const int t2 = tt[i2];
-                    ok = (T[c1] - ti + t2 <= dm.C) && (T[c2] - t2 + ti <= dm.C);
-                }
-            }
-            mv->feasible = ok; mv->reloc = reloc; mv->i = i; mv->i2 = i2; mv->c1 = c1; mv->c2 = c2;
-            if (ok) {
-                mv->rg1 = rp_rowshard(dm, A.edp, c1);
-                mv->rg2 = rp_rowshard(dm, A.edp, c2);
-            }
+    for (int kb = 0; kb < A.steps; kb += SPEC) {
+        const int nb = min(SPEC, A.steps - kb);
+        // ---- state-independent part of the next steps: one step per lane ------------------
+        if (warp == 0 && lane < nb) {
+            const StepRec r = rp_make_step_rec(A, (u32)(kb + lane), (u32)j);
+            recs[lane] = r;
         }
         block_sync<NT>();
-        if (!mv->feasible) { block_sync<NT>(); continue; }
-        const int mi = mv->i, mi2 = mv->i2, rg1 = mv->rg1, rg2 = mv->rg2;
-        const bool swap = !mv->reloc;
-        const bool touchW = (rg1 != rg2);
 
-        // ---- phase 2: tentative rank loads of the two row-shards and their layer maxima ----
-        i64 e1 = 0, e2 = 0;
-        if (touchW) {
-            const int *qi = A.q + (size_t)mi * dm.LP;
-            const int *q2 = swap ? A.q + (size_t)mi2 * dm.LP : nullptr;
-            const int *w1 = Wj + (size_t)rg1 * dm.LP, *w2 = Wj + (size_t)rg2 * dm.LP;
-            const int P = dm.P, LP = dm.LP;
-            if (P <= 32 && (P & (P - 1)) == 0) {
-                for (int x0 = 0; x0 < LP; x0 += NT) {
-                    const int x = x0 + tid;
-                    int v1 = 0, v2 = 0;
-                    if (x < LP) {
-                        int d = __ldg(qi + x);
-                        if (swap) d -= __ldg(q2 + x);
-                        v1 = w1[x] - d;
-                        v2 = w2[x] + d;
-                        scratch[x] = v1;
-                        scratch[LP + x] = v2;
-                    }
-                    for (int o = P >> 1; o; o >>= 1) {
-                        v1 = max(v1, __shfl_xor_sync(0xffffffffu, v1, o));
-                        v2 = max(v2, __shfl_xor_sync(0xffffffffu, v2, o));
-                    }
-                    if ((lane & (P - 1)) == 0 && x < LP) { e1 += v1; e2 += v2; }
+        int pos = 0;
+        while (pos < nb) {
+            // ---- speculation: proposals of steps kb+pos .. kb+nb-1 against the current state ----
+            if (warp == 0) {
+                bool ok = false;
+                if (lane >= pos && lane < nb) {
+                    MoveS m;
+                    ok = rp_propose(dm, view, recs[lane], aC, bS, m);
+                    if (ok) mvs[lane] = m;
                 }
-            } else {
-                for (int x = tid; x < LP; x += NT) {
-                    int d = __ldg(qi + x);
-                    if (swap) d -= __ldg(q2 + x);
-                    scratch[x] = w1[x] - d;
-                    scratch[LP + x] = w2[x] + d;
-                }
-                block_sync<NT>();
-                for (int l = warp; l < dm.L; l += NT / 32) {
-                    int v1 = 0, v2 = 0;
-                    for (int p = lane; p < P; p += 32) {
-                        v1 = max(v1, scratch[l * P + p]);
-                        v2 = max(v2, scratch[LP + l * P + p]);
+                const unsigned fm = __ballot_sync(0xffffffffu, ok);
+                if (lane == 0) { rnd->fmask = fm; rnd->accept = 0; }
+            }
+            block_sync<NT>();
+            unsigned fmask = rnd->fmask;
+            int next_pos = nb;
+            // ---- feasible steps in order, until one is accepted ---------------------------------
+            while (fmask) {
+                const int ls = __ffs(fmask) - 1;
+                fmask &= fmask - 1;
+                const MoveS m = mvs[ls];
+                const bool swap = !m.reloc;
+                const int rg1 = rg_of[m.c1], rg2 = rg_of[m.c2];
+                const bool touchW = (rg1 != rg2);
+                // tentative rank loads of the two row-shards and their layer maxima
+                i64 e1 = 0, e2 = 0;
+                if (touchW) {
+                    const int *qi = A.q + (size_t)m.i * dm.LP;
+                    const int *q2 = swap ? A.q + (size_t)m.i2 * dm.LP : nullptr;
+                    const int *w1 = Wj + (size_t)rg1 * dm.LP, *w2 = Wj + (size_t)rg2 * dm.LP;
+                    const int P = dm.P, LP = dm.LP;
+                    if (vec) {
+                        rp_slices_vec<2, NT>(LP >> 2, P >> 2, (const int4 *)qi, (const int4 *)q2, (const int4 *)w1,
+                                             (const int4 *)w2, (int4 *)scratch, (int4 *)(scratch + slice_pad), tid, e1, e2);
+                    } else {
+                        for (int x = tid; x < LP; x += NT) {
+                            int d = __ldg(qi + x);
+                            if (swap) d -= __ldg(q2 + x);
+                            scratch[x] = w1[x] - d;
+                            scratch[slice_pad + x] = w2[x] + d;
+                        }
+                        block_sync<NT>();
+                        for (int l = warp; l < dm.L; l += NT / 32) {
+                            int v1 = 0, v2 = 0;
+                            for (int p = lane; p < P; p += 32) {
+                                v1 = max(v1, scratch[l * P + p]);
+                                v2 = max(v2, scratch[slice_pad + l * P + p]);
+                            }
+                            for (int o = 16; o; o >>= 1) {
+                                v1 = max(v1, __shfl_xor_sync(0xffffffffu, v1, o));
+                                v2 = max(v2, __shfl_xor_sync(0xffffffffu, v2, o));
+                            }
+                            if (lane == 0) { e1 += v1; e2 += v2; }
+                        }
                     }
                     for (int o = 16; o; o >>= 1) {
-                        v1 = max(v1, __shfl_xor_sync(0xffffffffu, v1, o));
-                        v2 = max(v2, __shfl_xor_sync(0xffffffffu, v2, o));
+                        e1 += __shfl_xor_sync(0xffffffffu, e1, o);
+                        e2 += __shfl_xor_sync(0xffffffffu, e2, o);
                     }
-                    if (lane == 0) { e1 += v1; e2 += v2; }
+                    if (NT > 32) {
+                        if (lane == 0) { red[2 * warp] = e1; red[2 * warp + 1] = e2; }
+                        __syncthreads();
+                        if (warp == 0) {
+                            e1 = 0; e2 = 0;
+                            for (int w = 0; w < NT / 32; ++w) { e1 += red[2 * w]; e2 += red[2 * w + 1]; }
+                        }
+                    }
                 }
-            }
-            for (int o = 16; o; o >>= 1) {
-                e1 += __shfl_xor_sync(0xffffffffu, e1, o);
-                e2 += __shfl_xor_sync(0xffffffffu, e2, o);
-            }
-            if (NT > 32) {
-                if (lane == 0) { red[2 * warp] = e1; red[2 * warp + 1] = e2; }
-                __syncthreads();
-                if (tid == 0) {
-                    e1 = 0; e2 = 0;
-                    for (int w = 0; w < NT / 32; ++w) { e1 += red[2 * w]; e2 += red[2 * w + 1]; }
-                }
-            }
-        }
 
-        // ---- phase 3: exact new score, Metropolis, commit of the scalar state (thread 0) ----
-        if (tid == 0) {
-            const int c1 = mv->c1, c2 = mv->c2;
-            const i64 ti = tt[mi], t2 = swap ? tt[mi2] : 0;
-            const i64 Ta = (i64)T[c1] - ti + t2, Qa = (i64)Q[c1] - ti * ti + t2 * t2;
-            const i64 Tb = (i64)T[c2] + ti - t2, Qb = (i64)Q[c2] + ti * ti - t2 * t2;
-            const int r1 = c1 / dm.D, g1 = A.edp[c1 % dm.D], r2 = c2 / dm.D, g2 = A.edp[c2 % dm.D];
-            if (!touchW) { e1 = Esum[rg1]; e2 = e1; }
-            const i64 A1 = rp_attention(dm, st, A.dp_list, A.dp_off, r1, g1, c1, Ta, Qa, c2, Tb, Qb);
-            const i64 A2 = touchW ? rp_attention(dm, st, A.dp_list, A.dp_off, r2, g2, c1, Ta, Qa, c2, Tb, Qb) : A1;
-            const i64 J1o = Jfx[rg1], J2o = Jfx[rg2];
-            const i64 J1n = A1 + dm.EC * e1, J2n = touchW ? A2 + dm.EC * e2 : J1n;
-            const i64 dJ1 = J1n - J1o, dJ2 = touchW ? J2n - J2o : 0;
-            const i64 U1o = U[g1], U2o = U[g2];
-            i64 U1n, U2n;
-            if (g1 == g2) { U1n = U1o + dJ1 + dJ2; U2n = U1n; }
-            else { U1n = U1o + dJ1; U2n = U2o + dJ2; }
-            const i64 n1 = S[1] + dJ1 + dJ2;
-            // s0 = max_g U: only U[g1], U[g2] changed
-            i64 n0;
-            {
-                const i64 newmax = U1n > U2n ? U1n : U2n, oldmax = U1o > U2o ? U1o : U2o;
-                if (newmax >= S[0]) n0 = newmax;
-                else if (oldmax < S[0]) n0 = S[0];
-                else {
-                    n0 = newmax;
-                    for (int g = 0; g < dm.G; ++g) if (g != g1 && g != g2 && U[g] > n0) n0 = U[g];
+                // exact new score, Metropolis, commit of the scalar state (leading warp)
+                if (warp == 0) {
+                    const int c1 = m.c1, c2 = m.c2;
+                    const int g1 = g_of[c1], g2 = g_of[c2];
+                    i64 n0 = 0, n1 = 0, n2 = 0, A1 = 0, A2 = 0, J1n = 0, J2n = 0, U1n = 0, U2n = 0;
+                    i64 Ta = 0, Qa = 0, Tb = 0, Qb = 0;
+                    int fb0 = 0, fb2 = 0;
+                    if (lane == 0) {
+                        const i64 ti = tt[m.i], t2 = swap ? tt[m.i2] : 0;
+                        Ta = (i64)T[c1] - ti + t2; Qa = (i64)Q[c1] - ti * ti + t2 * t2;
+                        Tb = (i64)T[c2] + ti - t2; Qb = (i64)Q[c2] + ti * ti - t2 * t2;
+                        if (!touchW) { e1 = Esum[rg1]; e2 = e1; }
+                        if (identity_edp) { A1 = aC * Ta + bS * Qa; A2 = aC * Tb + bS * Qb; }
+                        else {
+                            A1 = rp_attention(dm, st, dpl, dpo, rowbase[c1] / dm.D, g1, c1, Ta, Qa, c2, Tb, Qb);
+                            A2 = touchW ? rp_attention(dm, st, dpl, dpo, rowbase[c2] / dm.D, g2, c1, Ta, Qa, c2, Tb, Qb) : A1;
+                        }
+                        const i64 J1o = Jfx[rg1], J2o = Jfx[rg2];
+                        J1n = A1 + dm.EC * e1; J2n = touchW ? A2 + dm.EC * e2 : J1n;
+                        const i64 dJ1 = J1n - J1o, dJ2 = touchW ? J2n - J2o : 0;
+                        const i64 U1o = U[g1], U2o = U[g2];
+                        if (g1 == g2) { U1n = U1o + dJ1 + dJ2; U2n = U1n; }
+                        else { U1n = U1o + dJ1; U2n = U2o + dJ2; }
+                        n1 = S[1] + dJ1 + dJ2;
+                        {   // s0 = max_g U: only U[g1], U[g2] changed
+                            const i64 newmax = U1n > U2n ? U1n : U2n, oldmax = U1o > U2o ? U1o : U2o;
+                            if (newmax >= S[0]) n0 = newmax;
+                            else if (oldmax < S[0]) n0 = S[0];
+                            else { n0 = newmax; fb0 = 1; }
+                        }
+                        {   // s2 = max_{r,g} J: only J[rg1], J[rg2] changed
+                            const i64 newmax = J1n > J2n ? J1n : J2n, oldmax = J1o > J2o ? J1o : J2o;
+                            if (newmax >= S[2]) n2 = newmax;
+                            else if (oldmax < S[2]) n2 = S[2];
+                            else { n2 = newmax; fb2 = 1; }
+                        }
+                    }
+                    // rare: the previous maximum sat on a changed entry and fell -> rescan in parallel
+                    const int fb = __shfl_sync(0xffffffffu, fb0 | (fb2 << 1), 0);
+                    if (fb & 1) {
+                        i64 v = 0;
+                        for (int g = lane; g < dm.G; g += 32) if (g != g1 && g != g2 && U[g] > v) v = U[g];
+                        v = warp_max_i64(v);
+                        if (lane == 0 && v > n0) n0 = v;
+                    }
+                    if (fb & 2) {
+                        i64 v = 0;
+                        for (int rg = lane; rg < dm.RG; rg += 32) if (rg != rg1 && rg != rg2 && Jfx[rg] > v) v = Jfx[rg];
+                        v = warp_max_i64(v);
+                        if (lane == 0 && v > n2) n2 = v;
+                    }
+                    if (lane == 0) {
+                        const StepRec rr = recs[ls];
+                        bool acc = rp_lex_less(n0, n1, n2, S[0], S[1], S[2]);
+                        const i64 en = rp_energy(n0, n1, n2);
+                        if (!acc) {
+                            if (en <= Ecur || (rr.flags & 4u)) acc = true;
+                            else {
+                                const u64 M = (u64)(Ecur > dm.SC ? Ecur : dm.SC);
+                                const u64 bh = __umul64hi(rr.thr, M), bl = rr.thr * M;
+                                acc = (bh >> 31) ? true : ((u64)(en - Ecur) < ((bh << 32) | (bl >> 32)));
+                            }
+                        }
+                        ++n_feas;
+                        if (touchW) n_bytes += (i64)((swap ? 4 : 3) + (acc ? 2 : 0)) * dm.LP * 4;
+                        if (acc) {
+                            ++n_acc;
+                            const int k = kb + ls;
+                            cell_of[m.i] = (unsigned short)c2;
+                            if (swap) cell_of[m.i2] = (unsigned short)c1;
+                            T[c1] = (int)Ta; Q[c1] = (u64)Qa; T[c2] = (int)Tb; Q[c2] = (u64)Qb;
+                            if (!swap) { cnt[c1] -= 1; cnt[c2] += 1; }
+                            Esum[rg1] = e1; Afx[rg1] = A1; Jfx[rg1] = J1n;
+                            if (touchW) { Esum[rg2] = e2; Afx[rg2] = A2; Jfx[rg2] = J2n; }
+                            U[g1] = U1n; U[g2] = U2n;
+                            S[0] = n0; S[1] = n1; S[2] = n2; Ecur = en;
+                            const u32 second = swap ? (u32)m.i2 : (u32)c2;
+                            if (nlog < A.log_cap) logj[nlog] = make_uint2((u32)m.i, second | (swap ? 0u : 0x80000000u));
+                            ++nlog;
+                            const u64 code = ((u64)(swap ? 0 : 1) << 63) ^ ((u64)(u32)k << 40) ^ ((u64)(u32)m.i << 20) ^ (u64)second;
+                            dig = (dig ^ code) * 0x100000001B3ull;
+                            if (rp_lex_less(n0, n1, n2, B0, B1, B2)) {
+                                B0 = n0; B1 = n1; B2 = n2;
+                                best_step = k + 1; best_nlog = nlog;
+                                ++n_imp;
+                            }
+                        }
+                        rnd->accept = acc;
+                    }
                 }
-            }
-            // s2 = max_{r,g} J: only J[rg1], J[rg2] changed
-            i64 n2;
-            {
-                const i64 newmax = J1n > J2n ? J1n : J2n, oldmax = J1o > J2o ? J1o : J2o;
-                if (newmax >= S[2]) n2 = newmax;
-                else if (oldmax < S[2]) n2 = S[2];
-                else {
-                    n2 = newmax;
-                    for (int rg = 0; rg < dm.RG; ++rg) if (rg != rg1 && rg != rg2 && Jfx[rg] > n2) n2 = Jfx[rg];
+                block_sync<NT>();
+                const int acc = rnd->accept;
+                if (acc) {
+                    if (touchW) {
+                        int *w1 = Wj + (size_t)rg1 * dm.LP, *w2 = Wj + (size_t)rg2 * dm.LP;
+                        for (int x = tid; x < dm.LP; x += NT) { w1[x] = scratch[x]; w2[x] = scratch[slice_pad + x]; }
+                    }
+                    next_pos = ls + 1;
+                    fmask = 0;
                 }
+                block_sync<NT>();
             }
-            bool acc = rp_lex_less(n0, n1, n2, S[0], S[1], S[2]);
-            if (!acc) {
-                const i64 eo = rp_energy(S[0], S[1], S[2]), en = rp_energy(n0, n1, n2);
-                if (en <= eo) acc = true;
-                else {
-                    const uint4 xw = rp_philox((u32)k, (u32)A.level, (u32)j, 2u, A.key0, A.key1);
-                    acc = rp_accept_uphill(eo, en - eo, dm.SC, A.tau, xw.x);
-                }
-            }
-            ++n_feas;
-            if (acc) {
-                ++n_acc;
-                cell_of[mi] = (unsigned short)c2;
-                if (swap) cell_of[mi2] = (unsigned short)c1;
-                T[c1] = (int)Ta; Q[c1] = (u64)Qa; T[c2] = (int)Tb; Q[c2] = (u64)Qb;
-                if (!swap) { cnt[c1] -= 1; cnt[c2] += 1; }
-                Esum[rg1] = e1; Afx[rg1] = A1; Jfx[rg1] = J1n;
-                if (touchW) { Esum[rg2] = e2; Afx[rg2] = A2; Jfx[rg2] = J2n; }
-                U[g1] = U1n; U[g2] = U2n;
-                S[0] = n0; S[1] = n1; S[2] = n2;
-                const u32 second = swap ? (u32)mi2 : (u32)c2;
-                if (nlog < A.log_cap) logj[nlog] = make_uint2((u32)mi, second | (swap ? 0u : 0x80000000u));
-                ++nlog;
-                const u64 code = ((u64)(swap ? 0 : 1) << 63) ^ ((u64)(u32)k << 40) ^ ((u64)(u32)mi << 20) ^ (u64)second;
-                dig = (dig ^ code) * 0x100000001B3ull;
-                if (rp_lex_less(n0, n1, n2, B0, B1, B2)) {
-                    B0 = n0; B1 = n1; B2 = n2;
-                    best_step = k + 1; best_nlog = nlog;
-                    ++n_imp;
-                }
-            }
-            mv->accept = acc;
+            pos = next_pos;
         }
-        block_sync<NT>();
-        // ---- phase 4: commit the two W slices ---------------------------------------------
-        if (mv->accept && touchW) {
-            int *w1 = Wj + (size_t)rg1 * dm.LP, *w2 = Wj + (size_t)rg2 * dm.LP;
-            for (int x = tid; x < dm.LP; x += NT) { w1[x] = scratch[x]; w2[x] = scratch[dm.LP + x]; }
-        }
-        block_sync<NT>();
     }
 
     // ---- epilogue: terminal state and chain report ------------------------------------------
@@ -332,6 +311,16 @@ k_anneal_level(const AnnealArgs A)
         for (int i = tid; i < dm.N; i += NT) cd[i] = cell_of[i];
         i64 *ed = A.Esum_dst + (size_t)j * dm.RG;
         for (int rg = tid; rg < dm.RG; rg += NT) ed[rg] = Esum[rg];
+        if (WS) {
+            int *wd = A.W_dst + (size_t)j * wn;
+            if ((wn & 3) == 0) {
+                int4 *wd4 = (int4 *)wd;
+                const int4 *ws4 = (const int4 *)Wsm;
+                for (size_t x = tid; x < wn / 4; x += NT) wd4[x] = ws4[x];
+            } else {
+                for (size_t x = tid; x < wn; x += NT) wd[x] = Wsm[x];
+            }
+        }
         if (tid == 0) {
             A.term[3 * (size_t)j + 0] = S[0]; A.term[3 * (size_t)j + 1] = S[1]; A.term[3 * (size_t)j + 2] = S[2];
             A.best[3 * (size_t)j + 0] = B0; A.best[3 * (size_t)j + 1] = B1; A.best[3 * (size_t)j + 2] = B2;
@@ -342,27 +331,36 @@ k_anneal_level(const AnnealArgs A)
             atomicAdd((u64 *)&A.counters[1], (u64)n_feas);
             atomicAdd((u64 *)&A.counters[2], (u64)n_acc);
             atomicAdd((u64 *)&A.counters[3], (u64)n_imp);
+            atomicAdd((u64 *)&A.counters[4], (u64)n_bytes);
+            if (src != j) atomicAdd((u64 *)&A.counters[5], (u64)2 * dm.RG * dm.LP * 4);
         }
     }
 }
 
-static int anneal_threads(const RpDims &dm)
-{
-    if (dm.LP <= 128) return 32;
-    if (dm.LP <= 512) return 128;
-    return 256;
-}
+// Thread count and shared-memory plan of the chain kernels.  Windows with L*P <= 512 use the
+// warp-per-candidate kernel; larger ones this cooperative kernel with 256 threads.
+size_t rp_wpc_smem_bytes(const RpDims &dm, int t_in_smem, int *w_in_smem);
+int rp_launch_anneal_wpc(rp_ctx *c, const AnnealArgs &A0);
+
+static bool use_wpc(const RpDims &dm) { return dm.LP <= 512; }
 
 int rp_anneal_smem_bytes(const rp_ctx *c, int *threads, size_t *bytes)
 {
     const RpDims &dm = c->dm;
-    int nt = anneal_threads(dm);
-    int t_in_smem = dm.N <= 2048;
-    size_t b = sizeof(u64) * dm.K + sizeof(i64) * (3 * (size_t)dm.RG + dm.G + 2 * (nt / 32));
-    b += sizeof(int) * (2 * (size_t)dm.K + 2 * (size_t)dm.LP + (t_in_smem ? dm.N : 0));
-    b += sizeof(unsigned short) * dm.N;
+    const int t_in_smem = dm.N <= 2048;
+    if (use_wpc(dm)) {
+        int ws = 0;
+        *threads = 128;
+        *bytes = rp_wpc_smem_bytes(dm, t_in_smem, &ws);
+        return t_in_smem | (ws << 1);
+    }
+    const int nt = 256;
+    size_t b = sizeof(u64) * dm.K + sizeof(i64) * (3 * (size_t)dm.RG + dm.G + 2 * (nt / 32)) + sizeof(StepRec) * SPEC + 16;
+    const size_t slice_pad = ((size_t)dm.LP + 3) & ~(size_t)3;
+    b += sizeof(int) * (2 * slice_pad + 2 * (size_t)dm.K + dm.D + dm.G + 1) + sizeof(MoveS) * SPEC + sizeof(RoundS);
+    b += sizeof(int) * (t_in_smem ? dm.N : 0) + 16;
+    b += sizeof(unsigned short) * ((size_t)dm.N + 3 * (size_t)dm.K);
     b = (b + 15) & ~(size_t)15;
-    b += sizeof(MoveRec) + 16;
     *threads = nt;
     *bytes = b;
     return t_in_smem;
@@ -379,24 +377,19 @@ int rp_launch_anneal_level(rp_ctx *c, int level, const rp_anneal_params *prm, u6
     A.Esum_src = s.Esum; A.Esum_dst = d.Esum;
     A.anc = c->d_anc;
     A.level = level; A.steps = prm->steps_per_level; A.log_cap = c->log_cap;
-    int nt; size_t smem;
-    A.t_in_smem = rp_anneal_smem_bytes(c, &nt, &smem);
-    if (smem > 220 * 1024) return RP_ERR_RANGE;
     A.rho_q32 = rho_q32; A.guide_q32 = guide_q32;
     A.key0 = (u32)c->cfg.seed; A.key1 = (u32)(c->cfg.seed >> 32);
     A.term = c->d_term; A.best = c->d_best; A.best_step = c->d_best_step; A.best_nlog = c->d_best_nlog;
-    A.digest = c->d_digest; A.log = c->d_log; A.counters = c->d_counters;
+    A.digest = c->d_digest; A.log = c->d_log; A.counters = c->d_counters; A.status = c->d_status;
     A.tau = c->h_levels[level].tau;
-#define LAUNCH(NT_)                                                                                   \
-    do {                                                                                              \
-        if (smem > 48 * 1024)                                                                         \
-            RP_CUDA(cudaFuncSetAttribute(k_anneal_level<NT_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
-        k_anneal_level<NT_><<<c->Ppop, NT_, smem, c->stream>>>(A);                                    \
-    } while (0)
-    if (nt == 32) LAUNCH(32);
-    else if (nt == 128) LAUNCH(128);
-    else LAUNCH(256);
-#undef LAUNCH
+    if (use_wpc(c->dm)) return rp_launch_anneal_wpc(c, A);
+    int nt; size_t smem;
+    A.t_in_smem = rp_anneal_smem_bytes(c, &nt, &smem) & 1;
+    if (smem > 220 * 1024) return RP_ERR_RANGE;
+    if (smem > 48 * 1024)
+        RP_CUDA(cudaFuncSetAttribute(k_anneal_level<256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    k_anneal_level<256, false><<<c->Ppop, 256, smem, c->stream>>>(A);
+    ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
     return RP_OK;
 }
@@ -579,6 +572,7 @@ int rp_launch_level_end(rp_ctx *c, int level, int n_levels)
     A.tr_term = c->d_tr_term; A.tr_best = c->d_tr_best; A.tr_inc = c->d_tr_inc;
     A.tr_best_step = c->d_tr_best_step; A.tr_anc = c->d_tr_anc; A.tr_digest = c->d_tr_digest;
     k_level_end<<<1, LE_THREADS, 0, c->stream>>>(A);
+    ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
     return RP_OK;
 }
@@ -613,6 +607,7 @@ int rp_launch_validate(rp_ctx *c)
 {
     int *fill = (int *)c->d_sort_keys;                 // scratch: 2*K ints fit (K <= N)
     k_validate<<<1, 1024, 0, c->stream>>>(c->d_inc_layout, c->d_t, c->dm, fill, fill + c->dm.K, c->d_status);
+    ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
     return RP_OK;
 }

@@ -9,6 +9,9 @@
 #include "rp_common.cuh"
 
 thread_local int g_rp_last_cuda_error = 0;
+long long g_rp_launches = 0;      // kernels launched by this library in this process
+
+extern "C" int64_t rp_debug_launch_count(void) { return g_rp_launches; }
 
 extern "C" int rp_last_cuda_error(void) { return g_rp_last_cuda_error; }
 
@@ -198,7 +201,7 @@ static int window_load_impl(rp_ctx *c, const rp_config *cfg, const int32_t *leng
     RP_TRY(dev_alloc(&c->d_sort_keys, (size_t)2 * n_pow2));
     RP_TRY(dev_alloc(&c->d_seed_layout, N));
     RP_TRY(dev_alloc(&c->d_pack_out, 4));
-    RP_TRY(dev_alloc(&c->d_counters, 4));
+    RP_TRY(dev_alloc(&c->d_counters, 8));
     RP_TRY(dev_alloc(&c->d_inc_layout, N));
     RP_TRY(dev_alloc(&c->d_inc_score, 3));
     RP_TRY(reset_status(c));
@@ -369,7 +372,8 @@ extern "C" int rp_eval_population(rp_ctx *c, const int32_t *layouts, int32_t n, 
         if (sw[RP_SW_BAD_LAYOUT]) return RP_ERR_ARG;
     } else {
         k_gather_cells<<<n, 256, 0, c->stream>>>(c->buf[c->cur].cell_of, c->d_anc, dm.N, c->d_eval_cells, nullptr);
-        RP_CUDA(cudaGetLastError());
+        ++g_rp_launches;
+    RP_CUDA(cudaGetLastError());
     }
     RP_TRY(rp_launch_eval(c, c->d_eval_cells, n, keepW ? c->d_eval_W : nullptr, c->d_eval_Esum, c->d_eval_score,
                           c->d_eval_f64));
@@ -428,7 +432,8 @@ extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *
     RP_TRY(dev_alloc(&c->d_tr_digest, (size_t)NL * P));
     RP_TRY(dev_alloc(&c->d_tr_anc, (size_t)(NL > 1 ? NL - 1 : 1) * P));
     c->trace_levels = NL;
-    RP_CUDA(cudaMemsetAsync(c->d_counters, 0, sizeof(i64) * 4, c->stream));
+    RP_CUDA(cudaMemsetAsync(c->d_counters, 0, sizeof(i64) * 8, c->stream));
+    RP_TRY(reset_status(c));
 
     cudaEvent_t ev[3];
     for (int x = 0; x < 3; ++x) RP_CUDA(cudaEventCreate(&ev[x]));
@@ -453,10 +458,17 @@ extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *
     for (int x = 0; x < 3; ++x) cudaEventDestroy(ev[x]);
     if (st == RP_OK && e != cudaSuccess) { g_rp_last_cuda_error = (int)e; st = RP_ERR_CUDA; }
     RP_TRY(st);
+    {
+        int sw[RP_SW_COUNT];
+        RP_TRY(read_status(c, sw));
+        if (sw[RP_SW_TIMEOUT]) return RP_ERR_TIMEOUT;     // a bounded device-side wait ran out
+    }
     if (stats) {
-        i64 cn[4];
+        i64 cn[8];
         RP_CUDA(cudaMemcpy(cn, c->d_counters, sizeof cn, cudaMemcpyDeviceToHost));
         stats->proposed = cn[0]; stats->feasible = cn[1]; stats->accepted = cn[2]; stats->improved = cn[3];
+        stats->move_bytes = cn[4]; stats->gather_bytes = cn[5];
+        stats->kernel_launches = 2 * (int64_t)NL;
         stats->ms_chains = ms_chains; stats->ms_barrier = ms_barrier;
     }
     c->stage = 4;
@@ -534,6 +546,7 @@ extern "C" int rp_debug_dump(rp_ctx *c, int what, int32_t index, void *buf, int6
             need = sizeof(int) * P * dm.N;
             if ((st = dev_alloc((int **)&tmp, P * dm.N)) != RP_OK) return st;
             k_gather_cells<<<c->Ppop, 256, 0, c->stream>>>(c->buf[c->cur].cell_of, c->d_anc, dm.N, nullptr, (int *)tmp);
+            ++g_rp_launches;
             src = tmp;
             break;
         }
@@ -545,6 +558,7 @@ extern "C" int rp_debug_dump(rp_ctx *c, int what, int32_t index, void *buf, int6
             i64 *T = (i64 *)tmp, *Q = T + K;
             int *cnt = (int *)(Q + K);
             k_cell_stats<<<1, 256, 0, c->stream>>>(c->buf[c->cur].cell_of + (size_t)member * dm.N, c->d_t, dm.N, dm.K, T, Q, cnt);
+            ++g_rp_launches;
             if (what == RP_DUMP_CELL_T) { src = T; need = sizeof(i64) * K; }
             else if (what == RP_DUMP_CELL_Q) { src = Q; need = sizeof(i64) * K; }
             else { src = cnt; need = sizeof(int) * K; }
@@ -600,7 +614,7 @@ static int dbg_map(const TI *in, size_t in_per, TO *out, size_t out_per, int64_t
     int st = dev_alloc(&dout, (size_t)n * out_per);
     if (st != RP_OK) { dev_free(din); return st; }
     cudaError_t e = cudaMemcpy(din, in, sizeof(TI) * n * in_per, cudaMemcpyDefault);
-    if (e == cudaSuccess) { launch(din, dout); e = cudaGetLastError(); }
+    if (e == cudaSuccess) { launch(din, dout); ++g_rp_launches; e = cudaGetLastError(); }
     if (e == cudaSuccess) e = cudaMemcpy(out, dout, sizeof(TO) * n * out_per, cudaMemcpyDefault);
     dev_free(din); dev_free(dout);
     if (e != cudaSuccess) { g_rp_last_cuda_error = (int)e; return RP_ERR_CUDA; }

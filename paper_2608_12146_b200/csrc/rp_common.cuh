@@ -19,6 +19,7 @@ typedef unsigned int u32;
 // error plumbing
 // ---------------------------------------------------------------------------------------
 extern thread_local int g_rp_last_cuda_error;
+extern long long g_rp_launches;
 #define RP_CUDA(call)                                                    \
     do {                                                                 \
         cudaError_t e_ = (call);                                         \
@@ -120,7 +121,7 @@ struct rp_ctx {
     int *h_t;                  // host copy of the lengths (range checks)
 };
 
-enum RpStatusWord { RP_SW_BAD_SAMPLE = 0, RP_SW_BAD_LAYOUT = 1, RP_SW_VALIDATE = 2, RP_SW_COUNT = 8 };
+enum RpStatusWord { RP_SW_BAD_SAMPLE = 0, RP_SW_BAD_LAYOUT = 1, RP_SW_VALIDATE = 2, RP_SW_TIMEOUT = 3, RP_SW_COUNT = 8 };
 
 // ---------------------------------------------------------------------------------------
 // launch wrappers (each returns an rp_status; none synchronises)

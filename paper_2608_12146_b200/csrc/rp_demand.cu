@@ -69,6 +69,7 @@ int rp_launch_check_reduce(rp_ctx *c)
     else if (nc <= 32) K1_CASE(32);
     else return RP_ERR_RANGE;             // more than 1024 experts per layer
 #undef K1_CASE
+    ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
     return RP_OK;
 }
@@ -133,6 +134,7 @@ int rp_launch_lpt(rp_ctx *c)
     size_t smem = sizeof(i64) * (dm.E + dm.P) + sizeof(int) * (dm.E + dm.P);
     int threads = dm.E < 32 ? 32 : (dm.E > 1024 ? 1024 : ((dm.E + 31) / 32) * 32);
     k_lpt<<<dm.L, threads, smem, c->stream>>>(c->d_Lagg, dm, c->d_pi, c->d_inv, c->d_rank_load);
+    ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
     return RP_OK;
 }
@@ -187,6 +189,7 @@ int rp_launch_project(rp_ctx *c)
     int grid = (int)(want < 148 * 8 ? want : 148 * 8);
     if (grid < 1) grid = 1;
     k_project<<<grid, K3_WARPS * 32, smem, c->stream>>>(c->d_a, c->d_inv, dm, c->d_q);
+    ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
     return RP_OK;
 }

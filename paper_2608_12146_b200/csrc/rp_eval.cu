@@ -25,6 +25,7 @@ int rp_launch_cells_from_layouts(rp_ctx *c, const int *layouts, int n, unsigned 
     long long total = (long long)n * c->dm.N;
     int grid = (int)((total + 255) / 256);
     k_layouts_to_cells<<<grid, 256, 0, c->stream>>>(layouts, total, c->dm.K, cells, c->d_status);
+    ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
     return RP_OK;
 }
@@ -107,6 +108,7 @@ int rp_launch_eval(rp_ctx *c, const unsigned short *cells, int n, int *W_out, i6
         RP_CUDA(cudaFuncSetAttribute(k_eval, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     k_eval<<<n, EVAL_THREADS, smem, c->stream>>>(cells, c->d_t, c->d_q, c->d_edp, c->d_dp_list, c->d_dp_off, dm,
                                                 W_out, Esum_out, score_out, f64_out);
+    ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
     return RP_OK;
 }

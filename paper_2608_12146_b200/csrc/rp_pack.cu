@@ -103,6 +103,7 @@ int rp_launch_pack(rp_ctx *c, int /*unused*/)
     int *fill_g = (int *)(c->d_sort_keys + n_pow2);
     k_pack_ffd<<<1, PACK_THREADS, smem, c->stream>>>(c->d_t, dm, c->cfg.min_rows, keys_g, n_pow2, fill_g,
                                                     c->d_seed_layout, c->d_pack_out);
+    ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
     return RP_OK;
 }
