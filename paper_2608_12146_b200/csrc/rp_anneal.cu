@@ -28,125 +28,104 @@
 // ((3 or 4) * L*P*4 bytes), writes 2 W slices when accepted.
 #include "rp_anneal.cuh"
 
-struct RoundS { unsigned fmask; int accept; int fallback; };
+struct ChainB {                 // bookkeeping of the chain within this level
+    i64 B[3];
+    u64 dig;
+    int best_step, best_nlog, nlog, failed;
+    unsigned fmask;
+    int accept;
+};
 
+// Cooperative chain kernel for bandwidth-bound windows (L*P > 512): all NT threads score one
+// candidate at a time (two L*P slices of W from global memory plus the moved samples' demand
+// rows, 16-byte loads); the leading warp rebuilds the score and decides.
 template <int NT>
-__device__ __forceinline__ void block_sync()
-{
-    if (NT == 32) __syncwarp(); else __syncthreads();
-}
-
-template <int NT, bool WS>
 __global__ void __launch_bounds__(NT)
 k_anneal_level(const AnnealArgs A)
 {
     const RpDims &dm = A.dm;
     extern __shared__ __align__(16) unsigned char smraw[];
-    // 8-byte: Q[K] Esum[RG] Afx[RG] Jfx[RG] U[G] red[2*NT/32] recs[SPEC]
-    // 4-byte: T[K] cnt[K] scratch[2*LP] dp_list[D] dp_off[G+1] mvs[SPEC] round t_s[N]? W[RG*LP]?
-    // 2-byte: cell_of[N] rg_of[K] g_of[K] rowbase[K]
-    u64 *Q = (u64 *)smraw;
-    i64 *Esum = (i64 *)(Q + dm.K);
-    i64 *Afx = Esum + dm.RG;
-    i64 *Jfx = Afx + dm.RG;
-    i64 *U = Jfx + dm.RG;
-    i64 *red = U + dm.G;
-    StepRec *recs = (StepRec *)(red + 2 * (NT / 32));
-    int *scratch = (int *)(((uintptr_t)(recs + SPEC) + 15) & ~(uintptr_t)15);     // 16-byte aligned slices
+    const size_t wn = (size_t)dm.RG * dm.LP;
     const size_t slice_pad = ((size_t)dm.LP + 3) & ~(size_t)3;
-    int *Wsm = scratch + 2 * slice_pad;
-    int *T = Wsm + (WS ? (((size_t)dm.RG * dm.LP + 3) & ~(size_t)3) : 0);
-    int *cnt = T + dm.K;
-    int *dpl = cnt + dm.K;
-    int *dpo = dpl + dm.D;
-    MoveS *mvs = (MoveS *)(dpo + dm.G + 1);
-    RoundS *rnd = (RoundS *)(mvs + SPEC);
-    int *t_s = (int *)(rnd + 1);
-    unsigned short *cell_of = (unsigned short *)(t_s + (A.t_in_smem ? dm.N : 0));
-    unsigned short *rg_of = cell_of + dm.N;
-    unsigned short *g_of = rg_of + dm.K;
-    unsigned short *rowbase = g_of + dm.K;
+    char *sm_blob = (char *)smraw;
+    char *sm_static = sm_blob + A.bl.bytes;
+    int *scratch = (int *)(sm_static + A.sl.bytes);
+    i64 *attkey = (i64 *)(scratch + 2 * slice_pad);
+    i64 *Jcell = attkey + dm.K;
+    i64 *Acell = Jcell + dm.K;
+    i64 *red = Acell + dm.K;
+    StepRec *recs = (StepRec *)(red + 2 * (NT / 32));
+    ChainB *chain = (ChainB *)(recs + SPEC);
+    u64 *mbar = (u64 *)(chain + 1);
+    MoveS *mvs = (MoveS *)(mbar + 1);
+
+    u64 *Q = (u64 *)(sm_blob + A.bl.off_Q);
+    i64 *Esum = (i64 *)(sm_blob + A.bl.off_Esum);
+    i64 *Afx = (i64 *)(sm_blob + A.bl.off_Afx);
+    i64 *Jfx = (i64 *)(sm_blob + A.bl.off_Jfx);
+    i64 *U = (i64 *)(sm_blob + A.bl.off_U);
+    i64 *Sc = (i64 *)(sm_blob + A.bl.off_S);
+    int *T = (int *)(sm_blob + A.bl.off_T);
+    int *cnt = (int *)(sm_blob + A.bl.off_cnt);
+    unsigned short *cell_of = (unsigned short *)(sm_blob + A.bl.off_cell);
+    const int *dpl = (const int *)(sm_static + A.sl.off_dpl);
+    const int *dpo = (const int *)(sm_static + A.sl.off_dpo);
+    const int *tt = A.sl.t_staged ? (const int *)(sm_static + A.sl.off_t) : A.t;
+    const unsigned short *rg_of = (const unsigned short *)(sm_static + A.sl.off_rg);
+    const unsigned short *g_of = (const unsigned short *)(sm_static + A.sl.off_g);
+    const unsigned short *rowbase = (const unsigned short *)(sm_static + A.sl.off_row);
     RpSmemState st = { cell_of, T, Q, cnt, Esum, Afx, U };
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int j = blockIdx.x;
     const int src = A.anc[j];
-    const int *tt = A.t_in_smem ? t_s : A.t;
     const bool identity_edp = (dm.G == dm.D);
-    const size_t wn = (size_t)dm.RG * dm.LP;
-    int *Wj = WS ? Wsm : A.W_dst + (size_t)j * wn;
+    int *Wj = A.W_dst + (size_t)j * wn;
+    const bool vec = (dm.P >= 4) && (dm.P <= 128) && ((dm.P & (dm.P - 1)) == 0);
+    const i64 aC = dm.asum * dm.C, bS = dm.bsum;
 
-    // ---- prologue: adopt the ancestor's terminal state -------------------------------
-    {
-        const unsigned short *cs = A.cell_src + (size_t)src * dm.N;
-        for (int i = tid; i < dm.N; i += NT) cell_of[i] = cs[i];
-        if (A.t_in_smem) for (int i = tid; i < dm.N; i += NT) t_s[i] = A.t[i];
-        for (int c = tid; c < dm.K; c += NT) {
-            T[c] = 0; Q[c] = 0; cnt[c] = 0;
-            const int r = c / dm.D, g = A.edp[c % dm.D];
-            rg_of[c] = (unsigned short)(r * dm.G + g);
-            g_of[c] = (unsigned short)g;
-            rowbase[c] = (unsigned short)(r * dm.D);
-        }
-        for (int d = tid; d < dm.D; d += NT) dpl[d] = A.dp_list[d];
-        for (int g = tid; g <= dm.G; g += NT) dpo[g] = A.dp_off[g];
-        const i64 *es = A.Esum_src + (size_t)src * dm.RG;
-        for (int rg = tid; rg < dm.RG; rg += NT) Esum[rg] = es[rg];
-        const int *ws = A.W_src + (size_t)src * wn;
-        if ((wn & 3) == 0) {
-            const int4 *ws4 = (const int4 *)ws;
-            int4 *wd4 = (int4 *)Wj;
-#pragma unroll 8
-            for (size_t x = tid; x < wn / 4; x += NT) wd4[x] = ws4[x];
-        } else {
-            for (size_t x = tid; x < wn; x += NT) Wj[x] = ws[x];
-        }
+    if (tid == 0) chain->failed = 0;
+    const bool landed = rp_chain_load<NT, false>(A, src, j, sm_blob, sm_static, nullptr, mbar, tid);
+    if (!landed) chain->failed = 1;
+    __syncthreads();
+    if (chain->failed) {
+        if (tid == 0) atomicExch(&A.status[RP_SW_TIMEOUT], 1);
+        return;
+    }
+    for (int c = tid; c < dm.K; c += NT) {
+        attkey[c] = aC * (i64)T[c] + bS * (i64)Q[c];
+        Jcell[c] = Jfx[rg_of[c]];
+        Acell[c] = Afx[rg_of[c]];
+    }
+    if (tid == 0) {
+        chain->B[0] = Sc[0]; chain->B[1] = Sc[1]; chain->B[2] = Sc[2];
+        chain->dig = 0; chain->best_step = 0; chain->best_nlog = 0; chain->nlog = 0;
     }
     __syncthreads();
-    rp_accumulate_cells(dm, st, A.t, tid, NT);
-    __syncthreads();
-    i64 S[3];
-    rp_rows_to_score(dm, st, dpl, dpo, tid, NT, S);
-    for (int rg = tid; rg < dm.RG; rg += NT) Jfx[rg] = Afx[rg] + dm.EC * Esum[rg];
-    __syncthreads();
 
-    // chain bookkeeping (thread 0 only)
-    i64 B0 = S[0], B1 = S[1], B2 = S[2];
-    i64 Ecur = (tid == 0) ? rp_energy(S[0], S[1], S[2]) : 0;
-    int best_step = 0, best_nlog = 0, nlog = 0;
-    u64 dig = 0;
-    i64 n_feas = 0, n_acc = 0, n_imp = 0, n_bytes = 0;
     uint2 *logj = A.log + (size_t)j * A.log_cap;
-    const i64 aC = dm.asum * dm.C, bS = dm.bsum;
-    const RpChainView view = { cell_of, rg_of, T, cnt, tt, Q, Jfx, Afx };
-    const bool vec = (dm.P >= 4) && (dm.P <= 128) && ((dm.P & (dm.P - 1)) == 0);
+    const RpChainView view = { cell_of, T, cnt, tt, attkey, Jcell, Acell };
+    i64 n_feas = 0, n_acc = 0, n_imp = 0, n_bytes = 0;          // thread 0
 
     for (int kb = 0; kb < A.steps; kb += SPEC) {
         const int nb = min(SPEC, A.steps - kb);
-        // ---- state-independent part of the next steps: one step per lane ------------------
-        if (warp == 0 && lane < nb) {
-            const StepRec r = rp_make_step_rec(A, (u32)(kb + lane), (u32)j);
-            recs[lane] = r;
-        }
-        block_sync<NT>();
-
+        if (tid < nb) recs[tid] = rp_make_step_rec(A, (u32)(kb + tid), (u32)j);
+        __syncthreads();
         int pos = 0;
         while (pos < nb) {
-            // ---- speculation: proposals of steps kb+pos .. kb+nb-1 against the current state ----
             if (warp == 0) {
                 bool ok = false;
                 if (lane >= pos && lane < nb) {
                     MoveS m;
-                    ok = rp_propose(dm, view, recs[lane], aC, bS, m);
+                    ok = rp_propose(dm, view, recs[lane], m);
                     if (ok) mvs[lane] = m;
                 }
                 const unsigned fm = __ballot_sync(0xffffffffu, ok);
-                if (lane == 0) { rnd->fmask = fm; rnd->accept = 0; }
+                if (lane == 0) { chain->fmask = fm; chain->accept = 0; }
             }
-            block_sync<NT>();
-            unsigned fmask = rnd->fmask;
+            __syncthreads();
+            unsigned fmask = chain->fmask;
             int next_pos = nb;
-            // ---- feasible steps in order, until one is accepted ---------------------------------
             while (fmask) {
                 const int ls = __ffs(fmask) - 1;
                 fmask &= fmask - 1;
@@ -154,7 +133,6 @@ k_anneal_level(const AnnealArgs A)
                 const bool swap = !m.reloc;
                 const int rg1 = rg_of[m.c1], rg2 = rg_of[m.c2];
                 const bool touchW = (rg1 != rg2);
-                // tentative rank loads of the two row-shards and their layer maxima
                 i64 e1 = 0, e2 = 0;
                 if (touchW) {
                     const int *qi = A.q + (size_t)m.i * dm.LP;
@@ -171,7 +149,7 @@ k_anneal_level(const AnnealArgs A)
                             scratch[x] = w1[x] - d;
                             scratch[slice_pad + x] = w2[x] + d;
                         }
-                        block_sync<NT>();
+                        __syncthreads();
                         for (int l = warp; l < dm.L; l += NT / 32) {
                             int v1 = 0, v2 = 0;
                             for (int p = lane; p < P; p += 32) {
@@ -185,21 +163,15 @@ k_anneal_level(const AnnealArgs A)
                             if (lane == 0) { e1 += v1; e2 += v2; }
                         }
                     }
-                    for (int o = 16; o; o >>= 1) {
-                        e1 += __shfl_xor_sync(0xffffffffu, e1, o);
-                        e2 += __shfl_xor_sync(0xffffffffu, e2, o);
-                    }
-                    if (NT > 32) {
-                        if (lane == 0) { red[2 * warp] = e1; red[2 * warp + 1] = e2; }
-                        __syncthreads();
-                        if (warp == 0) {
-                            e1 = 0; e2 = 0;
-                            for (int w = 0; w < NT / 32; ++w) { e1 += red[2 * w]; e2 += red[2 * w + 1]; }
-                        }
+                    e1 = warp_sum_i64(e1);
+                    e2 = warp_sum_i64(e2);
+                    if (lane == 0) { red[2 * warp] = e1; red[2 * warp + 1] = e2; }
+                    __syncthreads();
+                    if (warp == 0) {
+                        e1 = 0; e2 = 0;
+                        for (int w = 0; w < NT / 32; ++w) { e1 += red[2 * w]; e2 += red[2 * w + 1]; }
                     }
                 }
-
-                // exact new score, Metropolis, commit of the scalar state (leading warp)
                 if (warp == 0) {
                     const int c1 = m.c1, c2 = m.c2;
                     const int g1 = g_of[c1], g2 = g_of[c2];
@@ -207,6 +179,7 @@ k_anneal_level(const AnnealArgs A)
                     i64 Ta = 0, Qa = 0, Tb = 0, Qb = 0;
                     int fb0 = 0, fb2 = 0;
                     if (lane == 0) {
+                        const i64 S0 = Sc[0], S1 = Sc[1], S2 = Sc[2];
                         const i64 ti = tt[m.i], t2 = swap ? tt[m.i2] : 0;
                         Ta = (i64)T[c1] - ti + t2; Qa = (i64)Q[c1] - ti * ti + t2 * t2;
                         Tb = (i64)T[c2] + ti - t2; Qb = (i64)Q[c2] + ti * ti - t2 * t2;
@@ -222,21 +195,20 @@ k_anneal_level(const AnnealArgs A)
                         const i64 U1o = U[g1], U2o = U[g2];
                         if (g1 == g2) { U1n = U1o + dJ1 + dJ2; U2n = U1n; }
                         else { U1n = U1o + dJ1; U2n = U2o + dJ2; }
-                        n1 = S[1] + dJ1 + dJ2;
-                        {   // s0 = max_g U: only U[g1], U[g2] changed
+                        n1 = S1 + dJ1 + dJ2;
+                        {
                             const i64 newmax = U1n > U2n ? U1n : U2n, oldmax = U1o > U2o ? U1o : U2o;
-                            if (newmax >= S[0]) n0 = newmax;
-                            else if (oldmax < S[0]) n0 = S[0];
+                            if (newmax >= S0) n0 = newmax;
+                            else if (oldmax < S0) n0 = S0;
                             else { n0 = newmax; fb0 = 1; }
                         }
-                        {   // s2 = max_{r,g} J: only J[rg1], J[rg2] changed
+                        {
                             const i64 newmax = J1n > J2n ? J1n : J2n, oldmax = J1o > J2o ? J1o : J2o;
-                            if (newmax >= S[2]) n2 = newmax;
-                            else if (oldmax < S[2]) n2 = S[2];
+                            if (newmax >= S2) n2 = newmax;
+                            else if (oldmax < S2) n2 = S2;
                             else { n2 = newmax; fb2 = 1; }
                         }
                     }
-                    // rare: the previous maximum sat on a changed entry and fell -> rescan in parallel
                     const int fb = __shfl_sync(0xffffffffu, fb0 | (fb2 << 1), 0);
                     if (fb & 1) {
                         i64 v = 0;
@@ -252,7 +224,8 @@ k_anneal_level(const AnnealArgs A)
                     }
                     if (lane == 0) {
                         const StepRec rr = recs[ls];
-                        bool acc = rp_lex_less(n0, n1, n2, S[0], S[1], S[2]);
+                        const i64 Ecur = Sc[3];
+                        bool acc = rp_lex_less(n0, n1, n2, Sc[0], Sc[1], Sc[2]);
                         const i64 en = rp_energy(n0, n1, n2);
                         if (!acc) {
                             if (en <= Ecur || (rr.flags & 4u)) acc = true;
@@ -270,111 +243,103 @@ k_anneal_level(const AnnealArgs A)
                             cell_of[m.i] = (unsigned short)c2;
                             if (swap) cell_of[m.i2] = (unsigned short)c1;
                             T[c1] = (int)Ta; Q[c1] = (u64)Qa; T[c2] = (int)Tb; Q[c2] = (u64)Qb;
+                            attkey[c1] = aC * Ta + bS * Qa; attkey[c2] = aC * Tb + bS * Qb;
                             if (!swap) { cnt[c1] -= 1; cnt[c2] += 1; }
                             Esum[rg1] = e1; Afx[rg1] = A1; Jfx[rg1] = J1n;
                             if (touchW) { Esum[rg2] = e2; Afx[rg2] = A2; Jfx[rg2] = J2n; }
+                            if (identity_edp) { Jcell[c1] = J1n; Acell[c1] = A1; Jcell[c2] = J2n; Acell[c2] = A2; }
+                            else {
+                                for (int x = dpo[g1]; x < dpo[g1 + 1]; ++x) { const int c = rowbase[c1] + dpl[x]; Jcell[c] = J1n; Acell[c] = A1; }
+                                for (int x = dpo[g2]; x < dpo[g2 + 1]; ++x) { const int c = rowbase[c2] + dpl[x]; Jcell[c] = J2n; Acell[c] = A2; }
+                            }
                             U[g1] = U1n; U[g2] = U2n;
-                            S[0] = n0; S[1] = n1; S[2] = n2; Ecur = en;
+                            Sc[0] = n0; Sc[1] = n1; Sc[2] = n2; Sc[3] = en;
                             const u32 second = swap ? (u32)m.i2 : (u32)c2;
+                            int nlog = chain->nlog;
                             if (nlog < A.log_cap) logj[nlog] = make_uint2((u32)m.i, second | (swap ? 0u : 0x80000000u));
-                            ++nlog;
+                            chain->nlog = ++nlog;
                             const u64 code = ((u64)(swap ? 0 : 1) << 63) ^ ((u64)(u32)k << 40) ^ ((u64)(u32)m.i << 20) ^ (u64)second;
-                            dig = (dig ^ code) * 0x100000001B3ull;
-                            if (rp_lex_less(n0, n1, n2, B0, B1, B2)) {
-                                B0 = n0; B1 = n1; B2 = n2;
-                                best_step = k + 1; best_nlog = nlog;
+                            chain->dig = (chain->dig ^ code) * 0x100000001B3ull;
+                            if (rp_lex_less(n0, n1, n2, chain->B[0], chain->B[1], chain->B[2])) {
+                                chain->B[0] = n0; chain->B[1] = n1; chain->B[2] = n2;
+                                chain->best_step = k + 1; chain->best_nlog = nlog;
                                 ++n_imp;
                             }
                         }
-                        rnd->accept = acc;
+                        chain->accept = acc;
                     }
                 }
-                block_sync<NT>();
-                const int acc = rnd->accept;
+                __syncthreads();
+                const int acc = chain->accept;
                 if (acc) {
                     if (touchW) {
                         int *w1 = Wj + (size_t)rg1 * dm.LP, *w2 = Wj + (size_t)rg2 * dm.LP;
-                        for (int x = tid; x < dm.LP; x += NT) { w1[x] = scratch[x]; w2[x] = scratch[slice_pad + x]; }
+                        if (vec) {
+                            for (int c = tid; c < (dm.LP >> 2); c += NT) {
+                                ((int4 *)w1)[c] = ((const int4 *)scratch)[c];
+                                ((int4 *)w2)[c] = ((const int4 *)(scratch + slice_pad))[c];
+                            }
+                        } else {
+                            for (int x = tid; x < dm.LP; x += NT) { w1[x] = scratch[x]; w2[x] = scratch[slice_pad + x]; }
+                        }
                     }
                     next_pos = ls + 1;
                     fmask = 0;
                 }
-                block_sync<NT>();
+                __syncthreads();
             }
             pos = next_pos;
         }
     }
 
-    // ---- epilogue: terminal state and chain report ------------------------------------------
-    {
-        unsigned short *cd = A.cell_dst + (size_t)j * dm.N;
-        for (int i = tid; i < dm.N; i += NT) cd[i] = cell_of[i];
-        i64 *ed = A.Esum_dst + (size_t)j * dm.RG;
-        for (int rg = tid; rg < dm.RG; rg += NT) ed[rg] = Esum[rg];
-        if (WS) {
-            int *wd = A.W_dst + (size_t)j * wn;
-            if ((wn & 3) == 0) {
-                int4 *wd4 = (int4 *)wd;
-                const int4 *ws4 = (const int4 *)Wsm;
-                for (size_t x = tid; x < wn / 4; x += NT) wd4[x] = ws4[x];
-            } else {
-                for (size_t x = tid; x < wn; x += NT) wd[x] = Wsm[x];
-            }
-        }
-        if (tid == 0) {
-            A.term[3 * (size_t)j + 0] = S[0]; A.term[3 * (size_t)j + 1] = S[1]; A.term[3 * (size_t)j + 2] = S[2];
-            A.best[3 * (size_t)j + 0] = B0; A.best[3 * (size_t)j + 1] = B1; A.best[3 * (size_t)j + 2] = B2;
-            A.best_step[j] = best_step;
-            A.best_nlog[j] = best_nlog;
-            A.digest[j] = dig;
-            atomicAdd((u64 *)&A.counters[0], (u64)A.steps);
-            atomicAdd((u64 *)&A.counters[1], (u64)n_feas);
-            atomicAdd((u64 *)&A.counters[2], (u64)n_acc);
-            atomicAdd((u64 *)&A.counters[3], (u64)n_imp);
-            atomicAdd((u64 *)&A.counters[4], (u64)n_bytes);
-            if (src != j) atomicAdd((u64 *)&A.counters[5], (u64)2 * dm.RG * dm.LP * 4);
-        }
+    rp_chain_store<NT, false>(A, j, sm_blob, nullptr, tid);
+    if (tid == 0) {
+        for (int x = 0; x < 3; ++x) { A.term[3 * (size_t)j + x] = Sc[x]; A.best[3 * (size_t)j + x] = chain->B[x]; }
+        A.best_step[j] = chain->best_step;
+        A.best_nlog[j] = chain->best_nlog;
+        A.digest[j] = chain->dig;
+        atomicAdd((u64 *)&A.counters[0], (u64)A.steps);
+        atomicAdd((u64 *)&A.counters[1], (u64)n_feas);
+        atomicAdd((u64 *)&A.counters[2], (u64)n_acc);
+        atomicAdd((u64 *)&A.counters[3], (u64)n_imp);
+        atomicAdd((u64 *)&A.counters[4], (u64)n_bytes);
+        if (src != j) atomicAdd((u64 *)&A.counters[5], (u64)2 * dm.RG * dm.LP * 4);
     }
 }
 
 // Thread count and shared-memory plan of the chain kernels.  Windows with L*P <= 512 use the
-// warp-per-candidate kernel; larger ones this cooperative kernel with 256 threads.
-size_t rp_wpc_smem_bytes(const RpDims &dm, int t_in_smem, int *w_in_smem);
-int rp_launch_anneal_wpc(rp_ctx *c, const AnnealArgs &A0);
+// warp-per-candidate kernel; larger ones the cooperative kernel with 256 threads.
+size_t rp_wpc_smem_bytes(const RpDims &dm, const RpBlob &bl, const RpStatic &sl, int *w_in_smem);
+int rp_launch_anneal_wpc(rp_ctx *c, const AnnealArgs &A);
 
 static bool use_wpc(const RpDims &dm) { return dm.LP <= 512; }
 
 int rp_anneal_smem_bytes(const rp_ctx *c, int *threads, size_t *bytes)
 {
     const RpDims &dm = c->dm;
-    const int t_in_smem = dm.N <= 2048;
     if (use_wpc(dm)) {
         int ws = 0;
         *threads = 128;
-        *bytes = rp_wpc_smem_bytes(dm, t_in_smem, &ws);
-        return t_in_smem | (ws << 1);
+        *bytes = rp_wpc_smem_bytes(dm, c->bl, c->sl, &ws);
+        return ws;
     }
     const int nt = 256;
-    size_t b = sizeof(u64) * dm.K + sizeof(i64) * (3 * (size_t)dm.RG + dm.G + 2 * (nt / 32)) + sizeof(StepRec) * SPEC + 16;
     const size_t slice_pad = ((size_t)dm.LP + 3) & ~(size_t)3;
-    b += sizeof(int) * (2 * slice_pad + 2 * (size_t)dm.K + dm.D + dm.G + 1) + sizeof(MoveS) * SPEC + sizeof(RoundS);
-    b += sizeof(int) * (t_in_smem ? dm.N : 0) + 16;
-    b += sizeof(unsigned short) * ((size_t)dm.N + 3 * (size_t)dm.K);
-    b = (b + 15) & ~(size_t)15;
+    size_t b = (size_t)c->bl.bytes + c->sl.bytes + sizeof(int) * 2 * slice_pad + sizeof(i64) * (3 * (size_t)dm.K + 2 * (nt / 32)) +
+               sizeof(StepRec) * SPEC + sizeof(ChainB) + sizeof(u64) + sizeof(MoveS) * SPEC;
     *threads = nt;
-    *bytes = b;
-    return t_in_smem;
+    *bytes = (b + 15) & ~(size_t)15;
+    return 0;
 }
 
 int rp_launch_anneal_level(rp_ctx *c, int level, const rp_anneal_params *prm, u64 rho_q32, u64 guide_q32)
 {
     AnnealArgs A;
-    A.dm = c->dm;
-    A.t = c->d_t; A.q = c->d_q; A.edp = c->d_edp; A.dp_list = c->d_dp_list; A.dp_off = c->d_dp_off;
+    A.dm = c->dm; A.bl = c->bl; A.sl = c->sl;
+    A.t = c->d_t; A.q = c->d_q; A.static_blk = c->d_static;
     const RpPopBuf &s = c->buf[c->cur], &d = c->buf[1 - c->cur];
-    A.cell_src = s.cell_of; A.cell_dst = d.cell_of;
+    A.blob_src = s.blob; A.blob_dst = d.blob;
     A.W_src = s.W; A.W_dst = d.W;
-    A.Esum_src = s.Esum; A.Esum_dst = d.Esum;
     A.anc = c->d_anc;
     A.level = level; A.steps = prm->steps_per_level; A.log_cap = c->log_cap;
     A.rho_q32 = rho_q32; A.guide_q32 = guide_q32;
@@ -384,11 +349,11 @@ int rp_launch_anneal_level(rp_ctx *c, int level, const rp_anneal_params *prm, u6
     A.tau = c->h_levels[level].tau;
     if (use_wpc(c->dm)) return rp_launch_anneal_wpc(c, A);
     int nt; size_t smem;
-    A.t_in_smem = rp_anneal_smem_bytes(c, &nt, &smem) & 1;
+    rp_anneal_smem_bytes(c, &nt, &smem);
     if (smem > 220 * 1024) return RP_ERR_RANGE;
     if (smem > 48 * 1024)
-        RP_CUDA(cudaFuncSetAttribute(k_anneal_level<256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k_anneal_level<256, false><<<c->Ppop, 256, smem, c->stream>>>(A);
+        RP_CUDA(cudaFuncSetAttribute(k_anneal_level<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    k_anneal_level<256><<<c->Ppop, 256, smem, c->stream>>>(A);
     ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
     return RP_OK;
@@ -410,7 +375,8 @@ struct LevelEndArgs {
     const int *best_step, *best_nlog;
     const u64 *digest;
     const uint2 *log;
-    const unsigned short *cell_src;   // layouts the level started from (indexed through anc)
+    const char *blob_src;             // chain states the level started from (indexed through anc)
+    RpBlob bl;
     int *anc;
     u64 *F;
     int *inc_layout;
@@ -469,7 +435,7 @@ k_level_end(const LevelEndArgs A)
     __syncthreads();
     if (do_update) {
         const int w = win_j;
-        const unsigned short *cs = A.cell_src + (size_t)A.anc[w] * A.dm.N;
+        const unsigned short *cs = (const unsigned short *)(A.blob_src + (size_t)A.anc[w] * A.bl.bytes + A.bl.off_cell);
         for (int i = tid; i < A.dm.N; i += LE_THREADS) A.inc_layout[i] = cs[i];
         __syncthreads();
         if (tid == 0) {      // replay the accepted moves up to the trajectory-best step
@@ -566,7 +532,7 @@ int rp_launch_level_end(rp_ctx *c, int level, int n_levels)
     A.key0 = (u32)c->cfg.seed; A.key1 = (u32)(c->cfg.seed >> 32);
     A.term = c->d_term; A.best = c->d_best; A.best_step = c->d_best_step; A.best_nlog = c->d_best_nlog;
     A.digest = c->d_digest; A.log = c->d_log;
-    A.cell_src = c->buf[c->cur].cell_of;
+    A.blob_src = c->buf[c->cur].blob; A.bl = c->bl;
     A.anc = c->d_anc; A.F = c->d_F;
     A.inc_layout = c->d_inc_layout; A.inc_score = c->d_inc_score;
     A.tr_term = c->d_tr_term; A.tr_best = c->d_tr_best; A.tr_inc = c->d_tr_inc;

@@ -6,12 +6,14 @@
 
 struct AnnealArgs {
     RpDims dm;
-    const int *t, *q, *edp, *dp_list, *dp_off;
-    const unsigned short *cell_src;  unsigned short *cell_dst;
-    const int *W_src;                int *W_dst;
-    const i64 *Esum_src;             i64 *Esum_dst;
+    RpBlob bl;
+    RpStatic sl;
+    const int *t, *q;
+    const char *static_blk;
+    const char *blob_src;  char *blob_dst;
+    const int *W_src;      int *W_dst;
     const int *anc;
-    int level, steps, t_in_smem, log_cap;
+    int level, steps, log_cap;
     u64 tau, rho_q32, guide_q32;
     u32 key0, key1;
     i64 *term, *best;
@@ -34,6 +36,8 @@ struct MoveS { int reloc, i, i2, c1, c2; };
 
 // Random words of step k of chain slot j at this level -> the step record.
 // Purposes: 0 = proposal words A, 1 = proposal words B, 2 = accept word.
+// The uniform branch is stored as a tournament between a candidate and itself, so that the
+// proposal rule below needs no branch on it.
 __device__ __forceinline__ StepRec rp_make_step_rec(const AnnealArgs &A, u32 k, u32 j)
 {
     const RpDims &dm = A.dm;
@@ -43,8 +47,11 @@ __device__ __forceinline__ StepRec rp_make_step_rec(const AnnealArgs &A, u32 k, 
     const bool reloc = (u64)a.x < A.rho_q32, guided = (u64)a.y < A.guide_q32;
     StepRec r;
     r.i0 = rp_pick(a.z, dm.N);
-    if (!guided) { r.i1 = reloc ? rp_pick(a.w, dm.K) : rp_pick(a.w, dm.N); r.i2 = 0; r.i3 = 0; }
-    else {
+    if (!guided) {
+        r.i1 = r.i0;
+        r.i2 = reloc ? rp_pick(a.w, dm.K) : rp_pick(a.w, dm.N);
+        r.i3 = r.i2;
+    } else {
         r.i1 = rp_pick(a.w, dm.N);
         r.i2 = reloc ? rp_pick(b.x, dm.K) : rp_pick(b.x, dm.N);
         r.i3 = reloc ? rp_pick(b.y, dm.K) : rp_pick(b.y, dm.N);
@@ -58,60 +65,40 @@ __device__ __forceinline__ StepRec rp_make_step_rec(const AnnealArgs &A, u32 k, 
     return r;
 }
 
-// Tables of the chain state the proposal rule reads (all in shared memory).
+// Tables of the chain state the proposal rule reads (all in shared memory).  The three
+// per-cell arrays are caches kept in step with the state: the attention cost of the cell,
+// and the cost J and the attention part A of the row-shard the cell belongs to.
 struct RpChainView {
-    const unsigned short *cell_of, *rg_of;
+    const unsigned short *cell_of;
     const int *T, *cnt, *tt;
-    const u64 *Q;
-    const i64 *Jfx, *Afx;
+    const i64 *attkey, *Jcell, *Acell;
 };
 
 // GuidedProposal + feasibility of one step against the current state.
-//   uniform branch: sample i0, partner sample / destination cell i1.
-//   guided branch: tournament of two.  Source candidates i0, i1; the comparison key is the
-//   attention cost of the candidate's cell with probability Afx/Jfx of the first candidate's
-//   row-shard (bz * Jfx < Afx * 2^32), else the row-shard cost Jfx; source = larger key
-//   (tie: first).  Target candidates i2, i3 (samples for a swap, cells for a relocation);
-//   target = smaller key (tie: first).
+//   Tournament of two.  Source candidates i0, i1; the comparison key is the attention cost
+//   of the candidate's cell with probability Afx/Jfx of the first candidate's row-shard
+//   (bz * Jfx < Afx * 2^32), else the row-shard cost Jfx; source = larger key (tie: first).
+//   Target candidates i2, i3 (samples for a swap, cells for a relocation); target = smaller
+//   key (tie: first).  The uniform branch arrives as i1 == i0 and i3 == i2.
 // Feasible = distinct cells, both cells within the token cap afterwards, no cell emptied.
-__device__ __forceinline__ bool rp_propose(const RpDims &dm, const RpChainView &v, const StepRec &r,
-                                           i64 aC, i64 bS, MoveS &m)
+__device__ __forceinline__ bool rp_propose(const RpDims &dm, const RpChainView &v, const StepRec &r, MoveS &m)
 {
-    const bool reloc = r.flags & 1u, guided = r.flags & 2u;
-    m.reloc = reloc; m.i2 = -1;
-    if (!guided) {
-        m.i = r.i0;
-        m.c1 = v.cell_of[m.i];
-        if (reloc) m.c2 = r.i1;
-        else { m.i2 = r.i1; m.c2 = v.cell_of[m.i2]; }
-    } else {
-        const int sa = r.i0, sb = r.i1;
-        const int ca = v.cell_of[sa], cb = v.cell_of[sb];
-        const int rga = v.rg_of[ca];
-        const u64 Ja = (u64)v.Jfx[rga], Aa = (u64)v.Afx[rga];
-        const u64 lh = __umul64hi((u64)r.bz, Ja), ll = (u64)r.bz * Ja;
-        const u64 rh = Aa >> 32, rl = Aa << 32;
-        const bool use_att = (lh < rh) || (lh == rh && ll < rl);
-        int xa, xb, ya = -1, yb = -1;
-        if (reloc) { xa = r.i2; xb = r.i3; }
-        else { ya = r.i2; yb = r.i3; xa = v.cell_of[ya]; xb = v.cell_of[yb]; }
-        i64 ka, kb, ta, tb;
-        if (use_att) {
-            ka = aC * (i64)v.T[ca] + bS * (i64)v.Q[ca];
-            kb = aC * (i64)v.T[cb] + bS * (i64)v.Q[cb];
-            ta = aC * (i64)v.T[xa] + bS * (i64)v.Q[xa];
-            tb = aC * (i64)v.T[xb] + bS * (i64)v.Q[xb];
-        } else {
-            ka = (i64)Ja;
-            kb = v.Jfx[v.rg_of[cb]];
-            ta = v.Jfx[v.rg_of[xa]];
-            tb = v.Jfx[v.rg_of[xb]];
-        }
-        m.i = (kb > ka) ? sb : sa;
-        m.c1 = (kb > ka) ? cb : ca;
-        m.c2 = (tb < ta) ? xb : xa;
-        if (!reloc) m.i2 = (tb < ta) ? yb : ya;
-    }
+    const bool reloc = r.flags & 1u;
+    const int ca = v.cell_of[r.i0], cb = v.cell_of[r.i1];
+    const int xa = reloc ? r.i2 : (int)v.cell_of[r.i2];
+    const int xb = reloc ? r.i3 : (int)v.cell_of[r.i3];
+    const u64 Ja = (u64)v.Jcell[ca], Aa = (u64)v.Acell[ca];
+    const u64 lh = __umul64hi((u64)r.bz, Ja), ll = (u64)r.bz * Ja;
+    const u64 rh = Aa >> 32, rl = Aa << 32;
+    const bool use_att = (lh < rh) || (lh == rh && ll < rl);
+    const i64 *key = use_att ? v.attkey : v.Jcell;
+    const i64 ka = key[ca], kb = key[cb], ta = key[xa], tb = key[xb];
+    const bool src_b = kb > ka, dst_b = tb < ta;
+    m.reloc = reloc;
+    m.i = src_b ? r.i1 : r.i0;
+    m.c1 = src_b ? cb : ca;
+    m.c2 = dst_b ? xb : xa;
+    m.i2 = reloc ? -1 : (dst_b ? r.i3 : r.i2);
     if (m.c1 == m.c2) return false;
     const int ti = v.tt[m.i];
     if (reloc) return (v.cnt[m.c1] > 1) && (v.T[m.c2] + ti <= dm.C);
@@ -218,4 +205,68 @@ __device__ __forceinline__ void rp_bulk_commit_wait()
 __device__ __forceinline__ void rp_fence_async_smem()
 {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// ---- chain state in and out of shared memory ---------------------------------------------
+// Shared-memory front of both chain kernels: [blob][static tables][W when it lives on chip].
+// The blob of the ancestor, the static block and (on chip) the ancestor's W arrive by bulk
+// copies on one mbarrier; W kept in global memory is copied by all threads.
+template <int NT, bool WS>
+__device__ __forceinline__ bool rp_chain_load(const AnnealArgs &A, int src, int j, char *sm_blob, char *sm_static,
+                                              int *Wsm, u64 *mbar, int tid)
+{
+    const RpDims &dm = A.dm;
+    const size_t wn = (size_t)dm.RG * dm.LP;
+    const int *ws = A.W_src + (size_t)src * wn;
+    const bool w_bulk = WS && ((wn & 3) == 0);
+    if (tid == 0) {
+        rp_mbar_init(mbar, 1);
+        const u32 total = (u32)A.bl.bytes + (u32)A.sl.bytes + (w_bulk ? (u32)(wn * 4) : 0u);
+        rp_mbar_expect_tx(mbar, total);
+        rp_bulk_g2s(sm_blob, A.blob_src + (size_t)src * A.bl.bytes, (u32)A.bl.bytes, mbar);
+        rp_bulk_g2s(sm_static, A.static_blk, (u32)A.sl.bytes, mbar);
+        if (w_bulk)
+            for (size_t off = 0; off < wn * 4; off += 32768) {
+                const u32 n = (u32)((wn * 4 - off) < 32768 ? (wn * 4 - off) : 32768);
+                rp_bulk_g2s((char *)Wsm + off, (const char *)ws + off, n, mbar);
+            }
+    }
+    if (!w_bulk) {
+        int *wd = WS ? Wsm : A.W_dst + (size_t)j * wn;
+        if ((wn & 3) == 0) {
+            const int4 *ws4 = (const int4 *)ws;
+            int4 *wd4 = (int4 *)wd;
+#pragma unroll 8
+            for (size_t x = tid; x < wn / 4; x += NT) wd4[x] = __ldg(ws4 + x);
+        } else {
+            for (size_t x = tid; x < wn; x += NT) wd[x] = ws[x];
+        }
+    }
+    __syncthreads();                       // the barrier's initialisation is visible to every waiter
+    return rp_mbar_wait(mbar, 0);
+}
+
+template <int NT, bool WS>
+__device__ __forceinline__ void rp_chain_store(const AnnealArgs &A, int j, const char *sm_blob, const int *Wsm, int tid)
+{
+    const RpDims &dm = A.dm;
+    const size_t wn = (size_t)dm.RG * dm.LP;
+    const bool w_bulk = WS && ((wn & 3) == 0);
+    rp_fence_async_smem();                 // generic-proxy writes to shared memory -> visible to the bulk engine
+    __syncthreads();
+    if (tid == 0) {
+        rp_bulk_s2g(A.blob_dst + (size_t)j * A.bl.bytes, sm_blob, (u32)A.bl.bytes);
+        if (w_bulk) {
+            int *wd = A.W_dst + (size_t)j * wn;
+            for (size_t off = 0; off < wn * 4; off += 32768) {
+                const u32 n = (u32)((wn * 4 - off) < 32768 ? (wn * 4 - off) : 32768);
+                rp_bulk_s2g((char *)wd + off, (const char *)Wsm + off, n);
+            }
+        }
+        rp_bulk_commit_wait();
+    }
+    if (WS && !w_bulk) {
+        int *wd = A.W_dst + (size_t)j * wn;
+        for (size_t x = tid; x < wn; x += NT) wd[x] = Wsm[x];
+    }
 }

@@ -1,31 +1,24 @@
 // Chain kernel of the population annealing for latency-bound windows (L*P <= 512):
 // "warp per candidate".
 //
-// One CTA of NW warps runs one chain.  The random words and accept thresholds of the next
-// NW*32 steps are computed one step per thread.  The leading warp then evaluates the
-// proposals of the next 32 steps against the current state, one step per lane (a proposal
-// depends on the state, and the state changes only when a move is accepted).  The feasible
-// ones are scored NW at a time, one candidate per warp, all against the same state: each
-// warp builds the two tentative rank-load slices with 16-byte loads, reduces the busiest
-// rank per layer with shuffles, rebuilds the exact score and takes the Metropolis decision.
-// The first accepted candidate in step order is committed by its warp and everything
-// speculated after it is discarded and redone; if none is accepted the next NW follow.
-// This is step-for-step the sequential chain of Algorithm 3: a later step is only ever
-// scored against the state it would have seen.
-//
-// The rank-load tensor W of the chain sits in shared memory when it fits (moved in and out
-// with bulk asynchronous copies), so a scoring pass reads only the moved samples' demand
-// rows from L2.
+// One CTA of NW warps runs one chain.  The chain's small state arrives as one blob, and
+// its rank-load tensor W (when it fits on chip) as a second bulk asynchronous copy, both
+// signalled on one mbarrier; they leave the same way.  The random words and accept
+// thresholds of the next NW*32 steps are computed one step per thread.  The leading warp
+// then evaluates the proposals of the next 32 steps against the current state, one step
+// per lane (a proposal depends on the state, and the state changes only when a move is
+// accepted).  The feasible ones are scored NW at a time, one candidate per warp, all
+// against the same state: each warp builds the two tentative rank-load slices with 16-byte
+// loads, reduces the busiest rank per layer with shuffles, rebuilds the exact score and
+// takes the Metropolis decision.  The first accepted candidate in step order is committed
+// by its warp straight from its registers, and everything speculated after it is discarded
+// and redone; if none is accepted the next NW follow.  This is step-for-step the sequential
+// chain of Algorithm 3: a later step is only ever scored against the state it would have seen.
 #include "rp_anneal.cuh"
 
-struct EvalRes {
-    int acc, touchW, rg1, rg2, g1, g2, pad0, pad1;
-    i64 e1, e2, A1, A2, J1n, J2n, U1n, U2n, n0, n1, n2, en, Ta, Qa, Tb, Qb, bytes;
-};
-struct ChainS {
-    i64 S[3], Ecur, B[3];
-    u64 dig;
-    i64 n_feas, n_acc, n_imp, n_bytes;
+struct ChainS {                 // bookkeeping of the chain within this level
+    i64 B[3];                   // trajectory-best score
+    u64 dig;                    // digest of the accepted moves
     int best_step, best_nlog, nlog, failed;
 };
 
@@ -36,105 +29,71 @@ k_anneal_wpc(const AnnealArgs A)
     constexpr int NT = NW * 32;
     const RpDims &dm = A.dm;
     extern __shared__ __align__(16) unsigned char smraw[];
-    u64 *Q = (u64 *)smraw;
-    i64 *Esum = (i64 *)(Q + dm.K);
-    i64 *Afx = Esum + dm.RG;
-    i64 *Jfx = Afx + dm.RG;
-    i64 *U = Jfx + dm.RG;
-    StepRec *recs = (StepRec *)(U + dm.G);
-    EvalRes *res = (EvalRes *)(recs + NT);
-    ChainS *chain = (ChainS *)(res + NW);
-    u64 *mbar = (u64 *)(chain + 1);
-    int *scratch = (int *)(((uintptr_t)(mbar + 1) + 15) & ~(uintptr_t)15);
     const size_t wn = (size_t)dm.RG * dm.LP;
     const size_t slice_pad = ((size_t)dm.LP + 3) & ~(size_t)3;           // keeps every slice 16-byte aligned
-    int *Wsm = scratch + (size_t)NW * 2 * slice_pad;
-    int *T = Wsm + (WS ? ((wn + 3) & ~(size_t)3) : 0);
-    int *cnt = T + dm.K;
-    int *dpl = cnt + dm.K;
-    int *dpo = dpl + dm.D;
-    MoveS *mvs = (MoveS *)(dpo + dm.G + 1);
-    int *rnd = (int *)(mvs + SPEC);                                     // [0] feasible mask
-    int *t_s = rnd + 2;
-    unsigned short *cell_of = (unsigned short *)(t_s + (A.t_in_smem ? dm.N : 0));
-    unsigned short *rg_of = cell_of + dm.N;
-    unsigned short *g_of = rg_of + dm.K;
-    unsigned short *rowbase = g_of + dm.K;
+    char *sm_blob = (char *)smraw;
+    char *sm_static = sm_blob + A.bl.bytes;
+    int *Wsm = (int *)(sm_static + A.sl.bytes);
+    int *scratch = Wsm + (WS ? ((wn + 3) & ~(size_t)3) : 0);
+    i64 *attkey = (i64 *)(scratch + (size_t)NW * 2 * slice_pad);
+    i64 *Jcell = attkey + dm.K;
+    i64 *Acell = Jcell + dm.K;
+    StepRec *recs = (StepRec *)(Acell + dm.K);
+    ChainS *chain = (ChainS *)(recs + NT);
+    u64 *mbar = (u64 *)(chain + 1);
+    MoveS *mvs = (MoveS *)(mbar + 1);
+    int *vote = (int *)(mvs + SPEC);                                    // [NW] accept flags of a wave
+    int *rnd = vote + NW;                                               // [0] feasible mask, [1] next position
+
+    u64 *Q = (u64 *)(sm_blob + A.bl.off_Q);
+    i64 *Esum = (i64 *)(sm_blob + A.bl.off_Esum);
+    i64 *Afx = (i64 *)(sm_blob + A.bl.off_Afx);
+    i64 *Jfx = (i64 *)(sm_blob + A.bl.off_Jfx);
+    i64 *U = (i64 *)(sm_blob + A.bl.off_U);
+    i64 *Sc = (i64 *)(sm_blob + A.bl.off_S);                            // S0, S1, S2, energy
+    int *T = (int *)(sm_blob + A.bl.off_T);
+    int *cnt = (int *)(sm_blob + A.bl.off_cnt);
+    unsigned short *cell_of = (unsigned short *)(sm_blob + A.bl.off_cell);
+    const int *dpl = (const int *)(sm_static + A.sl.off_dpl);
+    const int *dpo = (const int *)(sm_static + A.sl.off_dpo);
+    const int *tt = A.sl.t_staged ? (const int *)(sm_static + A.sl.off_t) : A.t;
+    const unsigned short *rg_of = (const unsigned short *)(sm_static + A.sl.off_rg);
+    const unsigned short *g_of = (const unsigned short *)(sm_static + A.sl.off_g);
+    const unsigned short *rowbase = (const unsigned short *)(sm_static + A.sl.off_row);
     RpSmemState st = { cell_of, T, Q, cnt, Esum, Afx, U };
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int j = blockIdx.x;
     const int src = A.anc[j];
-    const int *tt = A.t_in_smem ? t_s : A.t;
     const bool identity_edp = (dm.G == dm.D);
     int *Wj = WS ? Wsm : A.W_dst + (size_t)j * wn;
-    const bool bulk_ok = WS && ((wn & 3) == 0);
     const bool vec = (dm.P >= 4) && (dm.P <= 128) && ((dm.P & (dm.P - 1)) == 0);
     const i64 aC = dm.asum * dm.C, bS = dm.bsum;
 
     // ---- prologue: adopt the ancestor's terminal state -------------------------------
-    {
-        const int *ws = A.W_src + (size_t)src * wn;
-        if (tid == 0) chain->failed = 0;
-        if (bulk_ok) {
-            if (tid == 0) {
-                rp_mbar_init(mbar, 1);
-                rp_mbar_expect_tx(mbar, (u32)(wn * 4));
-                for (size_t off = 0; off < wn * 4; off += 32768) {
-                    const u32 n = (u32)((wn * 4 - off) < 32768 ? (wn * 4 - off) : 32768);
-                    rp_bulk_g2s((char *)Wsm + off, (const char *)ws + off, n, mbar);
-                }
-            }
-        } else if ((wn & 3) == 0) {
-            const int4 *ws4 = (const int4 *)ws;
-            int4 *wd4 = (int4 *)Wj;
-#pragma unroll 8
-            for (size_t x = tid; x < wn / 4; x += NT) wd4[x] = ws4[x];
-        } else {
-            for (size_t x = tid; x < wn; x += NT) Wj[x] = ws[x];
-        }
-        const unsigned short *cs = A.cell_src + (size_t)src * dm.N;
-        for (int i = tid; i < dm.N; i += NT) cell_of[i] = cs[i];
-        if (A.t_in_smem) for (int i = tid; i < dm.N; i += NT) t_s[i] = A.t[i];
-        for (int c = tid; c < dm.K; c += NT) {
-            T[c] = 0; Q[c] = 0; cnt[c] = 0;
-            const int r = c / dm.D, g = A.edp[c % dm.D];
-            rg_of[c] = (unsigned short)(r * dm.G + g);
-            g_of[c] = (unsigned short)g;
-            rowbase[c] = (unsigned short)(r * dm.D);
-        }
-        for (int d = tid; d < dm.D; d += NT) dpl[d] = A.dp_list[d];
-        for (int g = tid; g <= dm.G; g += NT) dpo[g] = A.dp_off[g];
-        const i64 *es = A.Esum_src + (size_t)src * dm.RG;
-        for (int rg = tid; rg < dm.RG; rg += NT) Esum[rg] = es[rg];
-    }
+    if (tid == 0) chain->failed = 0;
+    const bool landed = rp_chain_load<NT, WS>(A, src, j, sm_blob, sm_static, Wsm, mbar, tid);
+    if (!landed) chain->failed = 1;
     __syncthreads();
-    rp_accumulate_cells(dm, st, tt, tid, NT);
-    __syncthreads();
-    {
-        i64 S[3];
-        rp_rows_to_score(dm, st, dpl, dpo, tid, NT, S);
-        for (int rg = tid; rg < dm.RG; rg += NT) Jfx[rg] = Afx[rg] + dm.EC * Esum[rg];
-        if (tid == 0) {
-            chain->S[0] = S[0]; chain->S[1] = S[1]; chain->S[2] = S[2];
-            chain->B[0] = S[0]; chain->B[1] = S[1]; chain->B[2] = S[2];
-            chain->Ecur = rp_energy(S[0], S[1], S[2]);
-            chain->dig = 0; chain->n_feas = 0; chain->n_acc = 0; chain->n_imp = 0; chain->n_bytes = 0;
-            chain->best_step = 0; chain->best_nlog = 0; chain->nlog = 0;
-        }
-    }
-    bool copy_ok = true;
-    if (bulk_ok) copy_ok = rp_mbar_wait(mbar, 0);
-    if (!copy_ok) chain->failed = 1;
-    __syncthreads();
-    if (chain->failed) {                 // the bulk copy never landed: report and leave
+    if (chain->failed) {                 // a bulk copy never landed: report and leave
         if (tid == 0) atomicExch(&A.status[RP_SW_TIMEOUT], 1);
         return;
     }
+    for (int c = tid; c < dm.K; c += NT) {
+        attkey[c] = aC * (i64)T[c] + bS * (i64)Q[c];
+        Jcell[c] = Jfx[rg_of[c]];
+        Acell[c] = Afx[rg_of[c]];
+    }
+    if (tid == 0) {
+        chain->B[0] = Sc[0]; chain->B[1] = Sc[1]; chain->B[2] = Sc[2];
+        chain->dig = 0; chain->best_step = 0; chain->best_nlog = 0; chain->nlog = 0;
+    }
+    __syncthreads();
 
     uint2 *logj = A.log + (size_t)j * A.log_cap;
-    const RpChainView view = { cell_of, rg_of, T, cnt, tt, Q, Jfx, Afx };
+    const RpChainView view = { cell_of, T, cnt, tt, attkey, Jcell, Acell };
     int *my_s1 = scratch + (size_t)warp * 2 * slice_pad, *my_s2 = my_s1 + slice_pad;
+    i64 w_feas = 0, w_acc = 0, w_imp = 0, w_bytes = 0;          // this warp's share of the counters (lane 0)
 
     for (int kb = 0; kb < A.steps; kb += NT) {
         const int nb = min(NT, A.steps - kb);
@@ -148,7 +107,7 @@ k_anneal_wpc(const AnnealArgs A)
                 bool ok = false;
                 if (pos + lane < nb) {
                     MoveS m;
-                    ok = rp_propose(dm, view, recs[pos + lane], aC, bS, m);
+                    ok = rp_propose(dm, view, recs[pos + lane], m);
                     if (ok) mvs[lane] = m;
                 }
                 const unsigned fm = __ballot_sync(0xffffffffu, ok);
@@ -162,12 +121,19 @@ k_anneal_wpc(const AnnealArgs A)
                 unsigned f = fmask;
                 for (int w = 0; w < warp; ++w) f &= f - 1;
                 const int my = f ? (__ffs(f) - 1) : -1;
+                // results of this warp's candidate stay in lane 0's registers until the vote
+                MoveS m;
+                m.reloc = 0; m.i = 0; m.i2 = -1; m.c1 = 0; m.c2 = 0;
+                int rg1 = 0, rg2 = 0, g1 = 0, g2 = 0;
+                bool touchW = false, acc = false;
+                i64 e1 = 0, e2 = 0, A1 = 0, A2 = 0, J1n = 0, J2n = 0, U1n = 0, U2n = 0;
+                i64 n0 = 0, n1 = 0, n2 = 0, en = 0, Ta = 0, Qa = 0, Tb = 0, Qb = 0, my_bytes = 0;
                 if (my >= 0) {
-                    const MoveS m = mvs[my];
+                    m = mvs[my];
                     const bool swap = !m.reloc;
-                    const int rg1 = rg_of[m.c1], rg2 = rg_of[m.c2];
-                    const bool touchW = (rg1 != rg2);
-                    i64 e1 = 0, e2 = 0;
+                    rg1 = rg_of[m.c1]; rg2 = rg_of[m.c2];
+                    g1 = g_of[m.c1]; g2 = g_of[m.c2];
+                    touchW = (rg1 != rg2);
                     if (touchW) {
                         const int *qi = A.q + (size_t)m.i * dm.LP;
                         const int *q2 = swap ? A.q + (size_t)m.i2 * dm.LP : nullptr;
@@ -201,36 +167,33 @@ k_anneal_wpc(const AnnealArgs A)
                     }
                     // exact new score and the Metropolis decision
                     const int c1 = m.c1, c2 = m.c2;
-                    const int g1 = g_of[c1], g2 = g_of[c2];
-                    EvalRes R;
                     int fb0 = 0, fb2 = 0;
-                    i64 n0 = 0, n2 = 0;
                     if (lane == 0) {
-                        const i64 S0 = chain->S[0], S1 = chain->S[1], S2 = chain->S[2];
+                        const i64 S0 = Sc[0], S1 = Sc[1], S2 = Sc[2];
                         const i64 ti = tt[m.i], t2 = swap ? tt[m.i2] : 0;
-                        R.Ta = (i64)T[c1] - ti + t2; R.Qa = (i64)Q[c1] - ti * ti + t2 * t2;
-                        R.Tb = (i64)T[c2] + ti - t2; R.Qb = (i64)Q[c2] + ti * ti - t2 * t2;
+                        Ta = (i64)T[c1] - ti + t2; Qa = (i64)Q[c1] - ti * ti + t2 * t2;
+                        Tb = (i64)T[c2] + ti - t2; Qb = (i64)Q[c2] + ti * ti - t2 * t2;
                         if (!touchW) { e1 = Esum[rg1]; e2 = e1; }
-                        if (identity_edp) { R.A1 = aC * R.Ta + bS * R.Qa; R.A2 = aC * R.Tb + bS * R.Qb; }
+                        if (identity_edp) { A1 = aC * Ta + bS * Qa; A2 = aC * Tb + bS * Qb; }
                         else {
-                            R.A1 = rp_attention(dm, st, dpl, dpo, rowbase[c1] / dm.D, g1, c1, R.Ta, R.Qa, c2, R.Tb, R.Qb);
-                            R.A2 = touchW ? rp_attention(dm, st, dpl, dpo, rowbase[c2] / dm.D, g2, c1, R.Ta, R.Qa, c2, R.Tb, R.Qb) : R.A1;
+                            A1 = rp_attention(dm, st, dpl, dpo, rowbase[c1] / dm.D, g1, c1, Ta, Qa, c2, Tb, Qb);
+                            A2 = touchW ? rp_attention(dm, st, dpl, dpo, rowbase[c2] / dm.D, g2, c1, Ta, Qa, c2, Tb, Qb) : A1;
                         }
                         const i64 J1o = Jfx[rg1], J2o = Jfx[rg2];
-                        R.J1n = R.A1 + dm.EC * e1; R.J2n = touchW ? R.A2 + dm.EC * e2 : R.J1n;
-                        const i64 dJ1 = R.J1n - J1o, dJ2 = touchW ? R.J2n - J2o : 0;
+                        J1n = A1 + dm.EC * e1; J2n = touchW ? A2 + dm.EC * e2 : J1n;
+                        const i64 dJ1 = J1n - J1o, dJ2 = touchW ? J2n - J2o : 0;
                         const i64 U1o = U[g1], U2o = U[g2];
-                        if (g1 == g2) { R.U1n = U1o + dJ1 + dJ2; R.U2n = R.U1n; }
-                        else { R.U1n = U1o + dJ1; R.U2n = U2o + dJ2; }
-                        R.n1 = S1 + dJ1 + dJ2;
+                        if (g1 == g2) { U1n = U1o + dJ1 + dJ2; U2n = U1n; }
+                        else { U1n = U1o + dJ1; U2n = U2o + dJ2; }
+                        n1 = S1 + dJ1 + dJ2;
                         {
-                            const i64 newmax = R.U1n > R.U2n ? R.U1n : R.U2n, oldmax = U1o > U2o ? U1o : U2o;
+                            const i64 newmax = U1n > U2n ? U1n : U2n, oldmax = U1o > U2o ? U1o : U2o;
                             if (newmax >= S0) n0 = newmax;
                             else if (oldmax < S0) n0 = S0;
                             else { n0 = newmax; fb0 = 1; }
                         }
                         {
-                            const i64 newmax = R.J1n > R.J2n ? R.J1n : R.J2n, oldmax = J1o > J2o ? J1o : J2o;
+                            const i64 newmax = J1n > J2n ? J1n : J2n, oldmax = J1o > J2o ? J1o : J2o;
                             if (newmax >= S2) n2 = newmax;
                             else if (oldmax < S2) n2 = S2;
                             else { n2 = newmax; fb2 = 1; }
@@ -251,9 +214,9 @@ k_anneal_wpc(const AnnealArgs A)
                     }
                     if (lane == 0) {
                         const StepRec rr = recs[pos + my];
-                        const i64 Ecur = chain->Ecur;
-                        bool acc = rp_lex_less(n0, R.n1, n2, chain->S[0], chain->S[1], chain->S[2]);
-                        const i64 en = rp_energy(n0, R.n1, n2);
+                        const i64 Ecur = Sc[3];
+                        acc = rp_lex_less(n0, n1, n2, Sc[0], Sc[1], Sc[2]);
+                        en = rp_energy(n0, n1, n2);
                         if (!acc) {
                             if (en <= Ecur || (rr.flags & 4u)) acc = true;
                             else {
@@ -262,23 +225,21 @@ k_anneal_wpc(const AnnealArgs A)
                                 acc = (bh >> 31) ? true : ((u64)(en - Ecur) < ((bh << 32) | (bl >> 32)));
                             }
                         }
-                        R.acc = acc; R.touchW = touchW; R.rg1 = rg1; R.rg2 = rg2; R.g1 = g1; R.g2 = g2;
-                        R.e1 = e1; R.e2 = e2; R.n0 = n0; R.n2 = n2; R.en = en;
-                        R.bytes = touchW ? (i64)((swap ? 4 : 3) + (acc ? 2 : 0)) * dm.LP * 4 : 0;
-                        res[warp] = R;
+                        my_bytes = touchW ? (i64)((swap ? 4 : 3) + (acc ? 2 : 0)) * dm.LP * 4 : 0;
+                        vote[warp] = acc;
                     }
                 }
                 __syncthreads();
                 const int wave = min(NW, __popc(fmask));
                 int win = -1;
-                for (int w = 0; w < wave; ++w) if (res[w].acc) { win = w; break; }
+#pragma unroll
+                for (int w = NW - 1; w >= 0; --w) if (w < wave && vote[w]) win = w;
+                if (my >= 0 && lane == 0 && (win < 0 || warp <= win)) { w_feas += 1; w_bytes += my_bytes; }
                 if (win >= 0) {
-                    if (warp == win) {
-                        const MoveS m = mvs[my];
-                        const EvalRes &R = res[win];
+                    if (warp == win) {        // commit from this warp's registers and scratch slices
                         const bool swap = !m.reloc;
-                        if (R.touchW) {
-                            int *w1 = Wj + (size_t)R.rg1 * dm.LP, *w2 = Wj + (size_t)R.rg2 * dm.LP;
+                        if (touchW) {
+                            int *w1 = Wj + (size_t)rg1 * dm.LP, *w2 = Wj + (size_t)rg2 * dm.LP;
                             if (vec) {
                                 for (int c = lane; c < (dm.LP >> 2); c += 32) {
                                     ((int4 *)w1)[c] = ((const int4 *)my_s1)[c];
@@ -293,37 +254,35 @@ k_anneal_wpc(const AnnealArgs A)
                             const int k = kb + pos + my;
                             cell_of[m.i] = (unsigned short)c2;
                             if (swap) cell_of[m.i2] = (unsigned short)c1;
-                            T[c1] = (int)R.Ta; Q[c1] = (u64)R.Qa; T[c2] = (int)R.Tb; Q[c2] = (u64)R.Qb;
+                            T[c1] = (int)Ta; Q[c1] = (u64)Qa; T[c2] = (int)Tb; Q[c2] = (u64)Qb;
+                            attkey[c1] = aC * Ta + bS * Qa; attkey[c2] = aC * Tb + bS * Qb;
                             if (!swap) { cnt[c1] -= 1; cnt[c2] += 1; }
-                            Esum[R.rg1] = R.e1; Afx[R.rg1] = R.A1; Jfx[R.rg1] = R.J1n;
-                            if (R.touchW) { Esum[R.rg2] = R.e2; Afx[R.rg2] = R.A2; Jfx[R.rg2] = R.J2n; }
-                            U[R.g1] = R.U1n; U[R.g2] = R.U2n;
-                            chain->S[0] = R.n0; chain->S[1] = R.n1; chain->S[2] = R.n2; chain->Ecur = R.en;
+                            Esum[rg1] = e1; Afx[rg1] = A1; Jfx[rg1] = J1n;
+                            if (touchW) { Esum[rg2] = e2; Afx[rg2] = A2; Jfx[rg2] = J2n; }
+                            if (identity_edp) { Jcell[c1] = J1n; Acell[c1] = A1; Jcell[c2] = J2n; Acell[c2] = A2; }
+                            else {
+                                for (int x = dpo[g1]; x < dpo[g1 + 1]; ++x) { const int c = rowbase[c1] + dpl[x]; Jcell[c] = J1n; Acell[c] = A1; }
+                                for (int x = dpo[g2]; x < dpo[g2 + 1]; ++x) { const int c = rowbase[c2] + dpl[x]; Jcell[c] = J2n; Acell[c] = A2; }
+                            }
+                            U[g1] = U1n; U[g2] = U2n;
+                            Sc[0] = n0; Sc[1] = n1; Sc[2] = n2; Sc[3] = en;
                             const u32 second = swap ? (u32)m.i2 : (u32)c2;
                             int nlog = chain->nlog;
                             if (nlog < A.log_cap) logj[nlog] = make_uint2((u32)m.i, second | (swap ? 0u : 0x80000000u));
                             chain->nlog = ++nlog;
                             const u64 code = ((u64)(swap ? 0 : 1) << 63) ^ ((u64)(u32)k << 40) ^ ((u64)(u32)m.i << 20) ^ (u64)second;
                             chain->dig = (chain->dig ^ code) * 0x100000001B3ull;
-                            if (rp_lex_less(R.n0, R.n1, R.n2, chain->B[0], chain->B[1], chain->B[2])) {
-                                chain->B[0] = R.n0; chain->B[1] = R.n1; chain->B[2] = R.n2;
+                            w_acc += 1;
+                            if (rp_lex_less(n0, n1, n2, chain->B[0], chain->B[1], chain->B[2])) {
+                                chain->B[0] = n0; chain->B[1] = n1; chain->B[2] = n2;
                                 chain->best_step = k + 1; chain->best_nlog = nlog;
-                                chain->n_imp += 1;
+                                w_imp += 1;
                             }
-                            i64 by = 0;
-                            for (int w = 0; w <= win; ++w) by += res[w].bytes;
-                            chain->n_feas += win + 1; chain->n_acc += 1; chain->n_bytes += by;
+                            rnd[1] = pos + my + 1;
                         }
-                        next_pos = pos + my + 1;      // warp-local; published below
-                        if (lane == 0) rnd[1] = next_pos;
                     }
                     fmask = 0;
                 } else {
-                    if (tid == 0) {
-                        i64 by = 0;
-                        for (int w = 0; w < wave; ++w) by += res[w].bytes;
-                        chain->n_feas += wave; chain->n_bytes += by;
-                    }
                     for (int w = 0; w < wave; ++w) fmask &= fmask - 1;
                 }
                 __syncthreads();
@@ -334,39 +293,20 @@ k_anneal_wpc(const AnnealArgs A)
     }
 
     // ---- epilogue: terminal state and chain report ------------------------------------------
-    {
-        unsigned short *cd = A.cell_dst + (size_t)j * dm.N;
-        for (int i = tid; i < dm.N; i += NT) cd[i] = cell_of[i];
-        i64 *ed = A.Esum_dst + (size_t)j * dm.RG;
-        for (int rg = tid; rg < dm.RG; rg += NT) ed[rg] = Esum[rg];
-        if (WS) {
-            int *wd = A.W_dst + (size_t)j * wn;
-            if (bulk_ok) {
-                rp_fence_async_smem();
-                __syncthreads();
-                if (tid == 0) {
-                    for (size_t off = 0; off < wn * 4; off += 32768) {
-                        const u32 n = (u32)((wn * 4 - off) < 32768 ? (wn * 4 - off) : 32768);
-                        rp_bulk_s2g((char *)wd + off, (const char *)Wsm + off, n);
-                    }
-                    rp_bulk_commit_wait();
-                }
-            } else {
-                for (size_t x = tid; x < wn; x += NT) wd[x] = Wsm[x];
-            }
-        }
-        if (tid == 0) {
-            for (int x = 0; x < 3; ++x) { A.term[3 * (size_t)j + x] = chain->S[x]; A.best[3 * (size_t)j + x] = chain->B[x]; }
-            A.best_step[j] = chain->best_step;
-            A.best_nlog[j] = chain->best_nlog;
-            A.digest[j] = chain->dig;
-            atomicAdd((u64 *)&A.counters[0], (u64)A.steps);
-            atomicAdd((u64 *)&A.counters[1], (u64)chain->n_feas);
-            atomicAdd((u64 *)&A.counters[2], (u64)chain->n_acc);
-            atomicAdd((u64 *)&A.counters[3], (u64)chain->n_imp);
-            atomicAdd((u64 *)&A.counters[4], (u64)chain->n_bytes);
-            if (src != j) atomicAdd((u64 *)&A.counters[5], (u64)2 * dm.RG * dm.LP * 4);
-        }
+    rp_chain_store<NT, WS>(A, j, sm_blob, Wsm, tid);
+    if (lane == 0) {
+        if (w_feas) atomicAdd((u64 *)&A.counters[1], (u64)w_feas);
+        if (w_acc) atomicAdd((u64 *)&A.counters[2], (u64)w_acc);
+        if (w_imp) atomicAdd((u64 *)&A.counters[3], (u64)w_imp);
+        if (w_bytes) atomicAdd((u64 *)&A.counters[4], (u64)w_bytes);
+    }
+    if (tid == 0) {
+        for (int x = 0; x < 3; ++x) { A.term[3 * (size_t)j + x] = Sc[x]; A.best[3 * (size_t)j + x] = chain->B[x]; }
+        A.best_step[j] = chain->best_step;
+        A.best_nlog[j] = chain->best_nlog;
+        A.digest[j] = chain->dig;
+        atomicAdd((u64 *)&A.counters[0], (u64)A.steps);
+        if (src != j) atomicAdd((u64 *)&A.counters[5], (u64)2 * dm.RG * dm.LP * 4);
     }
 }
 
@@ -374,29 +314,23 @@ k_anneal_wpc(const AnnealArgs A)
 
 // Shared-memory bytes of the warp-per-candidate kernel; *w_in_smem says whether W fits on chip
 // beside a second CTA.
-size_t rp_wpc_smem_bytes(const RpDims &dm, int t_in_smem, int *w_in_smem)
+size_t rp_wpc_smem_bytes(const RpDims &dm, const RpBlob &bl, const RpStatic &sl, int *w_in_smem)
 {
     const int NT = WPC_WARPS * 32;
-    size_t b = sizeof(u64) * dm.K + sizeof(i64) * (3 * (size_t)dm.RG + dm.G) + sizeof(StepRec) * NT +
-               sizeof(EvalRes) * WPC_WARPS + sizeof(ChainS) + sizeof(u64) + 16;
     const size_t slice_pad = ((size_t)dm.LP + 3) & ~(size_t)3;
-    b += sizeof(int) * WPC_WARPS * 2 * slice_pad;
-    size_t small = sizeof(int) * (2 * (size_t)dm.K + dm.D + dm.G + 1 + 2 + (t_in_smem ? dm.N : 0)) + sizeof(MoveS) * SPEC;
-    small += sizeof(unsigned short) * ((size_t)dm.N + 3 * (size_t)dm.K) + 16;
-    b += small;
+    size_t b = (size_t)bl.bytes + sl.bytes + sizeof(int) * WPC_WARPS * 2 * slice_pad + sizeof(i64) * 3 * dm.K +
+               sizeof(StepRec) * NT + sizeof(ChainS) + sizeof(u64) + sizeof(MoveS) * SPEC + sizeof(int) * (WPC_WARPS + 2);
     const size_t wbytes = sizeof(int) * ((((size_t)dm.RG * dm.LP) + 3) & ~(size_t)3);
     *w_in_smem = (b + wbytes <= 110 * 1024);
     if (*w_in_smem) b += wbytes;
     return (b + 15) & ~(size_t)15;
 }
 
-int rp_launch_anneal_wpc(rp_ctx *c, const AnnealArgs &A0)
+int rp_launch_anneal_wpc(rp_ctx *c, const AnnealArgs &A)
 {
-    AnnealArgs A = A0;
     const RpDims &dm = c->dm;
-    A.t_in_smem = dm.N <= 2048;
     int ws = 0;
-    const size_t smem = rp_wpc_smem_bytes(dm, A.t_in_smem, &ws);
+    const size_t smem = rp_wpc_smem_bytes(dm, c->bl, c->sl, &ws);
     if (smem > 220 * 1024) return RP_ERR_RANGE;
     const int chunks = ((dm.LP >> 2) + 31) / 32;
 #define LAUNCH(WS_, CH_)                                                                              \

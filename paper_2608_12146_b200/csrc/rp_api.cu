@@ -60,8 +60,8 @@ static int copy_out(rp_ctx *c, void *dst, const void *src, size_t bytes)
 static void free_population(rp_ctx *c)
 {
     for (int b = 0; b < 2; ++b) {
-        dev_free(c->buf[b].cell_of); dev_free(c->buf[b].W); dev_free(c->buf[b].Esum);
-        c->buf[b].cell_of = nullptr; c->buf[b].W = nullptr; c->buf[b].Esum = nullptr;
+        dev_free(c->buf[b].blob); dev_free(c->buf[b].W);
+        c->buf[b].blob = nullptr; c->buf[b].W = nullptr;
     }
     dev_free(c->d_anc); dev_free(c->d_term); dev_free(c->d_best); dev_free(c->d_best_step);
     dev_free(c->d_best_nlog); dev_free(c->d_digest); dev_free(c->d_log); dev_free(c->d_F);
@@ -83,9 +83,9 @@ static void free_trace(rp_ctx *c)
 static void free_eval(rp_ctx *c)
 {
     dev_free(c->d_eval_score); dev_free(c->d_eval_f64); dev_free(c->d_eval_W);
-    dev_free(c->d_eval_cells); dev_free(c->d_eval_Esum);
+    dev_free(c->d_eval_cells);
     c->d_eval_score = nullptr; c->d_eval_f64 = nullptr; c->d_eval_W = nullptr;
-    c->d_eval_cells = nullptr; c->d_eval_Esum = nullptr;
+    c->d_eval_cells = nullptr;
     c->eval_cap = 0; c->eval_W_n = 0;
 }
 
@@ -97,7 +97,7 @@ extern "C" void rp_destroy(rp_ctx *c)
     dev_free(c->own_t); dev_free(c->own_a); dev_free(c->d_edp); dev_free(c->d_dp_list); dev_free(c->d_dp_off);
     dev_free(c->d_Lagg); dev_free(c->d_pi); dev_free(c->d_inv); dev_free(c->d_rank_load); dev_free(c->d_q);
     dev_free(c->d_status); dev_free(c->d_sort_keys); dev_free(c->d_seed_layout); dev_free(c->d_pack_out);
-    dev_free(c->d_counters); dev_free(c->d_inc_layout); dev_free(c->d_inc_score);
+    dev_free(c->d_counters); dev_free(c->d_inc_layout); dev_free(c->d_inc_score); dev_free(c->d_static);
     free(c->h_levels); free(c->h_t);
     free(c);
 }
@@ -269,13 +269,12 @@ static int ensure_eval_scratch(rp_ctx *c, size_t n, bool want_W)
 {
     const RpDims &dm = c->dm;
     if (n > c->eval_cap) {
-        dev_free(c->d_eval_score); dev_free(c->d_eval_f64); dev_free(c->d_eval_cells); dev_free(c->d_eval_Esum);
-        c->d_eval_score = nullptr; c->d_eval_f64 = nullptr; c->d_eval_cells = nullptr; c->d_eval_Esum = nullptr;
+        dev_free(c->d_eval_score); dev_free(c->d_eval_f64); dev_free(c->d_eval_cells);
+        c->d_eval_score = nullptr; c->d_eval_f64 = nullptr; c->d_eval_cells = nullptr;
         c->eval_cap = 0;
         RP_TRY(dev_alloc(&c->d_eval_score, n * 3));
         RP_TRY(dev_alloc(&c->d_eval_f64, n * 3));
         RP_TRY(dev_alloc(&c->d_eval_cells, n * dm.N));
-        RP_TRY(dev_alloc(&c->d_eval_Esum, n * dm.RG));
         c->eval_cap = n;
     }
     if (want_W && (int)n > c->eval_W_n) {
@@ -300,6 +299,7 @@ extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
     c->Rstar = po[0]; c->certified = po[1];
     dm.R = po[0]; dm.K = dm.R * dm.D; dm.RG = dm.R * dm.G;
     if (dm.K > 65535) return RP_ERR_RANGE;
+    rp_make_layouts(dm, &c->bl, &c->sl);
     int nt; size_t smem;
     rp_anneal_smem_bytes(c, &nt, &smem);
     if (smem > 220 * 1024) return RP_ERR_RANGE;
@@ -308,9 +308,8 @@ extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
     free_population(c); free_eval(c);
     const size_t P = (size_t)c->Ppop, wn = (size_t)dm.RG * dm.LP;
     for (int b = 0; b < 2; ++b) {
-        RP_TRY(dev_alloc(&c->buf[b].cell_of, P * dm.N));
+        RP_TRY(dev_alloc(&c->buf[b].blob, P * (size_t)c->bl.bytes));
         RP_TRY(dev_alloc(&c->buf[b].W, P * wn));
-        RP_TRY(dev_alloc(&c->buf[b].Esum, P * dm.RG));
     }
     RP_TRY(dev_alloc(&c->d_anc, P));
     RP_TRY(dev_alloc(&c->d_term, P * 3));
@@ -322,8 +321,12 @@ extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
     c->cur = 0;
     // every member starts as the length-only seed: evaluate it once into slot 0 and let all
     // slots descend from slot 0
-    RP_TRY(rp_launch_cells_from_layouts(c, c->d_seed_layout, 1, c->buf[0].cell_of));
-    RP_TRY(rp_launch_eval(c, c->buf[0].cell_of, 1, c->buf[0].W, c->buf[0].Esum, c->d_inc_score, nullptr));
+    dev_free(c->d_static); c->d_static = nullptr;
+    RP_TRY(dev_alloc(&c->d_static, (size_t)c->sl.bytes));
+    RP_TRY(rp_launch_build_static(c));
+    RP_TRY(ensure_eval_scratch(c, 1, false));
+    RP_TRY(rp_launch_cells_from_layouts(c, c->d_seed_layout, 1, c->d_eval_cells));
+    RP_TRY(rp_launch_eval(c, c->d_eval_cells, 1, c->buf[0].W, c->buf[0].blob, c->d_inc_score, nullptr));
     RP_CUDA(cudaMemsetAsync(c->d_anc, 0, sizeof(int) * P, c->stream));
     RP_CUDA(cudaMemcpyAsync(c->d_inc_layout, c->d_seed_layout, sizeof(int) * dm.N, cudaMemcpyDeviceToDevice, c->stream));
     RP_CUDA(cudaMemcpyAsync(c->seed_score, c->d_inc_score, sizeof(i64) * 3, cudaMemcpyDeviceToHost, c->stream));
@@ -334,11 +337,11 @@ extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
     return RP_OK;
 }
 
-__global__ void k_gather_cells(const unsigned short *__restrict__ src, const int *__restrict__ anc, int N,
+__global__ void k_gather_cells(const char *__restrict__ blobs, RpBlob bl, const int *__restrict__ anc, int N,
                                unsigned short *__restrict__ dst16, int *__restrict__ dst32)
 {
     const int j = blockIdx.x;
-    const unsigned short *s = src + (size_t)anc[j] * N;
+    const unsigned short *s = (const unsigned short *)(blobs + (size_t)anc[j] * bl.bytes + bl.off_cell);
     for (int i = threadIdx.x; i < N; i += blockDim.x) {
         if (dst16) dst16[(size_t)j * N + i] = s[i];
         if (dst32) dst32[(size_t)j * N + i] = s[i];
@@ -371,11 +374,11 @@ extern "C" int rp_eval_population(rp_ctx *c, const int32_t *layouts, int32_t n, 
         RP_TRY(st);
         if (sw[RP_SW_BAD_LAYOUT]) return RP_ERR_ARG;
     } else {
-        k_gather_cells<<<n, 256, 0, c->stream>>>(c->buf[c->cur].cell_of, c->d_anc, dm.N, c->d_eval_cells, nullptr);
+        k_gather_cells<<<n, 256, 0, c->stream>>>(c->buf[c->cur].blob, c->bl, c->d_anc, dm.N, c->d_eval_cells, nullptr);
         ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
     }
-    RP_TRY(rp_launch_eval(c, c->d_eval_cells, n, keepW ? c->d_eval_W : nullptr, c->d_eval_Esum, c->d_eval_score,
+    RP_TRY(rp_launch_eval(c, c->d_eval_cells, n, keepW ? c->d_eval_W : nullptr, nullptr, c->d_eval_score,
                           c->d_eval_f64));
     RP_TRY(copy_out(c, score_fx, c->d_eval_score, sizeof(i64) * 3 * (size_t)n));
     RP_TRY(copy_out(c, score_f64, c->d_eval_f64, sizeof(double) * 3 * (size_t)n));
@@ -485,7 +488,7 @@ extern "C" int rp_best(rp_ctx *c, int32_t *cell_of_sample, int64_t *score_fx, do
     // full rescoring of the incumbent
     RP_TRY(ensure_eval_scratch(c, 1, false));
     RP_TRY(rp_launch_cells_from_layouts(c, c->d_inc_layout, 1, c->d_eval_cells));
-    RP_TRY(rp_launch_eval(c, c->d_eval_cells, 1, nullptr, c->d_eval_Esum, c->d_eval_score, c->d_eval_f64));
+    RP_TRY(rp_launch_eval(c, c->d_eval_cells, 1, nullptr, nullptr, c->d_eval_score, c->d_eval_f64));
     i64 inc[3], full[3];
     int sw[RP_SW_COUNT];
     RP_CUDA(cudaMemcpyAsync(inc, c->d_inc_score, sizeof inc, cudaMemcpyDeviceToHost, c->stream));
@@ -545,19 +548,20 @@ extern "C" int rp_debug_dump(rp_ctx *c, int what, int32_t index, void *buf, int6
         case RP_DUMP_POPULATION: {
             need = sizeof(int) * P * dm.N;
             if ((st = dev_alloc((int **)&tmp, P * dm.N)) != RP_OK) return st;
-            k_gather_cells<<<c->Ppop, 256, 0, c->stream>>>(c->buf[c->cur].cell_of, c->d_anc, dm.N, nullptr, (int *)tmp);
+            k_gather_cells<<<c->Ppop, 256, 0, c->stream>>>(c->buf[c->cur].blob, c->bl, c->d_anc, dm.N, nullptr, (int *)tmp);
             ++g_rp_launches;
             src = tmp;
             break;
         }
         case RP_DUMP_W: src = c->buf[c->cur].W + (size_t)member * dm.RG * dm.LP; need = sizeof(int) * (size_t)dm.RG * dm.LP; break;
-        case RP_DUMP_ESUM: src = c->buf[c->cur].Esum + (size_t)member * dm.RG; need = sizeof(i64) * dm.RG; break;
+        case RP_DUMP_ESUM: src = c->buf[c->cur].blob + (size_t)member * c->bl.bytes + c->bl.off_Esum; need = sizeof(i64) * dm.RG; break;
         case RP_DUMP_CELL_T: case RP_DUMP_CELL_Q: case RP_DUMP_CELL_CNT: {
             size_t K = dm.K;
             if ((st = dev_alloc((i64 **)&tmp, 3 * K)) != RP_OK) return st;
             i64 *T = (i64 *)tmp, *Q = T + K;
             int *cnt = (int *)(Q + K);
-            k_cell_stats<<<1, 256, 0, c->stream>>>(c->buf[c->cur].cell_of + (size_t)member * dm.N, c->d_t, dm.N, dm.K, T, Q, cnt);
+            k_cell_stats<<<1, 256, 0, c->stream>>>((const unsigned short *)(c->buf[c->cur].blob + (size_t)member * c->bl.bytes + c->bl.off_cell),
+                                                   c->d_t, dm.N, dm.K, T, Q, cnt);
             ++g_rp_launches;
             if (what == RP_DUMP_CELL_T) { src = T; need = sizeof(i64) * K; }
             else if (what == RP_DUMP_CELL_Q) { src = Q; need = sizeof(i64) * K; }

@@ -52,11 +52,37 @@ struct RpLevel {
     u64 cq;         // floor((1/T_{n+1} - 1/T_n) / ln2 * 2^16)
 };
 
+// Small state of one chain as one contiguous blob, laid out the same way in global and in
+// shared memory so that a single bulk copy moves it.  Offsets in bytes from a 16-byte
+// aligned base; `bytes` is a multiple of 16.
+struct RpBlob {
+    int off_Q;      // u64 [K]   squared-length sum per cell
+    int off_Esum;   // i64 [RG]  sum_l max_p W
+    int off_Afx;    // i64 [RG]  attention cost of the row-shard
+    int off_Jfx;    // i64 [RG]  Afx + 2^8*C*Esum
+    int off_U;      // i64 [G]   shard work
+    int off_S;      // i64 [4]   score tuple and energy
+    int off_T;      // int [K]   token sum per cell
+    int off_cnt;    // int [K]   samples per cell
+    int off_cell;   // u16 [N]   sample -> cell
+    int bytes;
+};
+// Tables that are the same for every chain of a plan (one block in global memory).
+struct RpStatic {
+    int off_dpl;    // int [D]   DP slots grouped by shard
+    int off_dpo;    // int [G+1] start of each shard's group
+    int off_t;      // int [N]   sample lengths (present when t_staged)
+    int off_rg;     // u16 [K]   cell -> row-shard
+    int off_g;      // u16 [K]   cell -> shard
+    int off_row;    // u16 [K]   cell -> first cell of its row
+    int bytes;
+    int t_staged;
+};
+
 // one population buffer set (two of them: the level reads one and writes the other)
 struct RpPopBuf {
-    unsigned short *cell_of;   // [P_pop][N]
+    char *blob;                // [P_pop][blob.bytes]
     int *W;                    // [P_pop][RG][LP]
-    i64 *Esum;                 // [P_pop][RG]   sum_l max_p W
 };
 
 struct rp_ctx {
@@ -88,6 +114,9 @@ struct rp_ctx {
     i64 seed_score[3];
     // population
     RpPopBuf buf[2];
+    RpBlob bl;
+    RpStatic sl;
+    char *d_static;            // static tables block
     int cur;                   // buffer holding the current population
     int *d_anc;                // [P_pop] which member of buf[cur] each slot continues from
     // per-level results
@@ -114,7 +143,6 @@ struct rp_ctx {
     int *d_eval_W;             // W of explicitly evaluated layouts (n <= 64), for inspection
     int eval_W_n;
     unsigned short *d_eval_cells;
-    i64 *d_eval_Esum;
     size_t eval_cap;
     RpLevel *h_levels;         // host copy of the per-level schedule integers
     int levels_cap;
@@ -130,8 +158,10 @@ int rp_launch_check_reduce(rp_ctx *c);
 int rp_launch_lpt(rp_ctx *c);
 int rp_launch_project(rp_ctx *c);
 int rp_launch_pack(rp_ctx *c, int Rlb_hint);
-int rp_launch_eval(rp_ctx *c, const unsigned short *cells, int n, int *W_out, i64 *Esum_out,
+int rp_launch_eval(rp_ctx *c, const unsigned short *cells, int n, int *W_out, char *blob_out,
                    i64 *score_out, double *f64_out);
+int rp_launch_build_static(rp_ctx *c);
+void rp_make_layouts(const RpDims &dm, RpBlob *bl, RpStatic *sl);
 int rp_launch_cells_from_layouts(rp_ctx *c, const int *layouts, int n, unsigned short *cells);
 int rp_launch_anneal_level(rp_ctx *c, int level, const rp_anneal_params *prm, u64 rho_q32, u64 guide_q32);
 int rp_launch_level_end(rp_ctx *c, int level, int n_levels);

@@ -33,8 +33,8 @@ int rp_launch_cells_from_layouts(rp_ctx *c, const int *layouts, int n, unsigned 
 __global__ void __launch_bounds__(EVAL_THREADS)
 k_eval(const unsigned short *__restrict__ cells, const int *__restrict__ t, const int *__restrict__ q,
        const int *__restrict__ edp, const int *__restrict__ dp_list, const int *__restrict__ dp_off,
-       RpDims dm, int *__restrict__ W_out, i64 *__restrict__ Esum_out, i64 *__restrict__ score_out,
-       double *__restrict__ f64_out)
+       RpDims dm, RpBlob bl, int *__restrict__ W_out, char *__restrict__ blob_out,
+       i64 *__restrict__ score_out, double *__restrict__ f64_out)
 {
     extern __shared__ __align__(16) unsigned char smraw[];
     // layout: Q[K] u64 | Esum[RG] | Afx[RG] | U[G] | T[K] | cnt[K] | off[RG+1] | cur[RG] | members[N] | cell_of[N]
@@ -81,7 +81,25 @@ k_eval(const unsigned short *__restrict__ cells, const int *__restrict__ t, cons
     __syncthreads();
     i64 sc[3];
     rp_rows_to_score(dm, st, dp_list, dp_off, tid, EVAL_THREADS, sc);
-    if (Esum_out) for (int rg = tid; rg < dm.RG; rg += EVAL_THREADS) Esum_out[(size_t)lay * dm.RG + rg] = Esum[rg];
+    if (blob_out) {      // the chain-state blob of this layout (see RpBlob)
+        char *b = blob_out + (size_t)lay * bl.bytes;
+        for (int c = tid; c < dm.K; c += EVAL_THREADS) {
+            ((u64 *)(b + bl.off_Q))[c] = Q[c];
+            ((int *)(b + bl.off_T))[c] = T[c];
+            ((int *)(b + bl.off_cnt))[c] = cnt[c];
+        }
+        for (int rg = tid; rg < dm.RG; rg += EVAL_THREADS) {
+            ((i64 *)(b + bl.off_Esum))[rg] = Esum[rg];
+            ((i64 *)(b + bl.off_Afx))[rg] = Afx[rg];
+            ((i64 *)(b + bl.off_Jfx))[rg] = Afx[rg] + dm.EC * Esum[rg];
+        }
+        for (int g = tid; g < dm.G; g += EVAL_THREADS) ((i64 *)(b + bl.off_U))[g] = U[g];
+        for (int i = tid; i < dm.N; i += EVAL_THREADS) ((unsigned short *)(b + bl.off_cell))[i] = cell_of[i];
+        if (tid == 0) {
+            i64 *S = (i64 *)(b + bl.off_S);
+            S[0] = sc[0]; S[1] = sc[1]; S[2] = sc[2]; S[3] = rp_energy(sc[0], sc[1], sc[2]);
+        }
+    }
     if (tid == 0) {
         for (int x = 0; x < 3; ++x) {
             if (score_out) score_out[(size_t)lay * 3 + x] = sc[x];
@@ -98,7 +116,7 @@ static size_t eval_smem_bytes(const RpDims &dm)
     return (b + 15) & ~(size_t)15;
 }
 
-int rp_launch_eval(rp_ctx *c, const unsigned short *cells, int n, int *W_out, i64 *Esum_out,
+int rp_launch_eval(rp_ctx *c, const unsigned short *cells, int n, int *W_out, char *blob_out,
                    i64 *score_out, double *f64_out)
 {
     const RpDims &dm = c->dm;
@@ -107,7 +125,57 @@ int rp_launch_eval(rp_ctx *c, const unsigned short *cells, int n, int *W_out, i6
     if (smem > 48 * 1024)
         RP_CUDA(cudaFuncSetAttribute(k_eval, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     k_eval<<<n, EVAL_THREADS, smem, c->stream>>>(cells, c->d_t, c->d_q, c->d_edp, c->d_dp_list, c->d_dp_off, dm,
-                                                W_out, Esum_out, score_out, f64_out);
+                                                c->bl, W_out, blob_out, score_out, f64_out);
+    ++g_rp_launches;
+    RP_CUDA(cudaGetLastError());
+    return RP_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Layout of the chain-state blob and of the per-plan static tables; the static block itself.
+// ---------------------------------------------------------------------------------------------
+void rp_make_layouts(const RpDims &dm, RpBlob *bl, RpStatic *sl)
+{
+    int o = 0;
+    bl->off_Q = o;    o += 8 * dm.K;
+    bl->off_Esum = o; o += 8 * dm.RG;
+    bl->off_Afx = o;  o += 8 * dm.RG;
+    bl->off_Jfx = o;  o += 8 * dm.RG;
+    bl->off_U = o;    o += 8 * dm.G;
+    bl->off_S = o;    o += 8 * 4;
+    bl->off_T = o;    o += 4 * dm.K;
+    bl->off_cnt = o;  o += 4 * dm.K;
+    bl->off_cell = o; o += 2 * dm.N;
+    bl->bytes = (o + 15) & ~15;
+    sl->t_staged = dm.N <= 2048;
+    o = 0;
+    sl->off_dpl = o;  o += 4 * dm.D;
+    sl->off_dpo = o;  o += 4 * (dm.G + 1);
+    sl->off_t = o;    o += sl->t_staged ? 4 * dm.N : 0;
+    sl->off_rg = o;   o += 2 * dm.K;
+    sl->off_g = o;    o += 2 * dm.K;
+    sl->off_row = o;  o += 2 * dm.K;
+    sl->bytes = (o + 15) & ~15;
+}
+
+__global__ void k_build_static(const int *__restrict__ t, const int *__restrict__ edp, const int *__restrict__ dp_list,
+                               const int *__restrict__ dp_off, RpDims dm, RpStatic sl, char *__restrict__ blk)
+{
+    const int tid = blockIdx.x * blockDim.x + threadIdx.x, nt = gridDim.x * blockDim.x;
+    for (int d = tid; d < dm.D; d += nt) ((int *)(blk + sl.off_dpl))[d] = dp_list[d];
+    for (int g = tid; g <= dm.G; g += nt) ((int *)(blk + sl.off_dpo))[g] = dp_off[g];
+    if (sl.t_staged) for (int i = tid; i < dm.N; i += nt) ((int *)(blk + sl.off_t))[i] = t[i];
+    for (int c = tid; c < dm.K; c += nt) {
+        const int r = c / dm.D, g = edp[c % dm.D];
+        ((unsigned short *)(blk + sl.off_rg))[c] = (unsigned short)(r * dm.G + g);
+        ((unsigned short *)(blk + sl.off_g))[c] = (unsigned short)g;
+        ((unsigned short *)(blk + sl.off_row))[c] = (unsigned short)(r * dm.D);
+    }
+}
+
+int rp_launch_build_static(rp_ctx *c)
+{
+    k_build_static<<<4, 256, 0, c->stream>>>(c->d_t, c->d_edp, c->d_dp_list, c->d_dp_off, c->dm, c->sl, c->d_static);
     ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
     return RP_OK;
