@@ -79,8 +79,9 @@ typedef struct {
 
 typedef struct {
     int64_t proposed, feasible, accepted, improved;  /* summed over chains and levels       */
-    double ms_chains;           /* device time in the per-level chain kernels               */
-    double ms_barrier;          /* device time in incumbent update + resampling             */
+    double ms_chains;           /* device time of all levels (chain kernels incl. the level
+                                   barrier that runs in their last CTA, and launch gaps)    */
+    double ms_barrier;          /* always 0: kept for layout compatibility                  */
     int64_t move_bytes;         /* algorithmic bytes of the feasible moves: rank-load slices
                                    and demand rows read, slices written on accept           */
     int64_t gather_bytes;       /* rank-load bytes read+written for members that resampling
@@ -136,7 +137,11 @@ int rp_anneal(rp_ctx *ctx, const rp_anneal_params *params, rp_anneal_stats *stat
  *   cell_of_sample [N] int32 out, nullable; score_fx [3], score_f64 [3] out, nullable. */
 int rp_best(rp_ctx *ctx, int32_t *cell_of_sample, int64_t *score_fx, double *score_f64);
 
+/* Frees the context.  Its device memory goes back to a per-device cache inside the library
+ * (so that the next window does not pay for allocation); rp_release_cached_memory() returns
+ * that cache to the driver. */
 void rp_destroy(rp_ctx *ctx);
+int rp_release_cached_memory(void);
 const char *rp_strerror(int status);
 /* cudaError_t value of the last failed CUDA call on this thread (0 if none). */
 int rp_last_cuda_error(void);

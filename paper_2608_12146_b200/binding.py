@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "RP_OK", -1: "RP_ERR_ARG", -2: "RP_ERR_SHAPE", -3: "RP_ERR_CO
 RP_OK = 0
 
 EXPORTS = ("rp_window_load", "rp_place_experts", "rp_pack_rows", "rp_eval_population", "rp_anneal",
-           "rp_best", "rp_destroy", "rp_strerror", "rp_last_cuda_error", "rp_debug_dump",
+           "rp_best", "rp_destroy", "rp_release_cached_memory", "rp_strerror", "rp_last_cuda_error", "rp_debug_dump",
            "rp_debug_nl2", "rp_debug_exp2neg", "rp_debug_philox", "rp_debug_launch_count")
 
 
@@ -203,6 +203,10 @@ def rp_best(ctx: Context, cell_of_sample=None, score_fx=None, score_f64=None):
 
 def rp_destroy(ctx: Context):
     ctx.close()
+
+
+def rp_release_cached_memory():
+    _check(lib().rp_release_cached_memory(), "rp_release_cached_memory")
 
 
 # ---- inspection hooks -------------------------------------------------------------------

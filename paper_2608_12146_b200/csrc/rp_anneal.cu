@@ -26,7 +26,7 @@
 //
 // Algorithmic bytes per feasible move: reads 2 W slices + the moved samples' q rows
 // ((3 or 4) * L*P*4 bytes), writes 2 W slices when accepted.
-#include "rp_anneal.cuh"
+#include "rp_level_end.cuh"
 
 struct ChainB {                 // bookkeeping of the chain within this level
     i64 B[3];
@@ -305,6 +305,7 @@ k_anneal_level(const AnnealArgs A)
         atomicAdd((u64 *)&A.counters[4], (u64)n_bytes);
         if (src != j) atomicAdd((u64 *)&A.counters[5], (u64)2 * dm.RG * dm.LP * 4);
     }
+    rp_finish_level(A, tid, NT);
 }
 
 // Thread count and shared-memory plan of the chain kernels.  Windows with L*P <= 512 use the
@@ -332,7 +333,7 @@ int rp_anneal_smem_bytes(const rp_ctx *c, int *threads, size_t *bytes)
     return 0;
 }
 
-int rp_launch_anneal_level(rp_ctx *c, int level, const rp_anneal_params *prm, u64 rho_q32, u64 guide_q32)
+int rp_launch_anneal_level(rp_ctx *c, int level, int n_levels, const rp_anneal_params *prm, u64 rho_q32, u64 guide_q32)
 {
     AnnealArgs A;
     A.dm = c->dm; A.bl = c->bl; A.sl = c->sl;
@@ -347,197 +348,20 @@ int rp_launch_anneal_level(rp_ctx *c, int level, const rp_anneal_params *prm, u6
     A.term = c->d_term; A.best = c->d_best; A.best_step = c->d_best_step; A.best_nlog = c->d_best_nlog;
     A.digest = c->d_digest; A.log = c->d_log; A.counters = c->d_counters; A.status = c->d_status;
     A.tau = c->h_levels[level].tau;
+    A.cq = c->h_levels[level].cq;
+    A.Ppop = c->Ppop;
+    A.last = (level == n_levels - 1);
+    A.lo.done = c->d_done; A.lo.anc_out = c->d_anc_next; A.lo.F = c->d_F;
+    A.lo.inc_layout = c->d_inc_layout; A.lo.inc_score = c->d_inc_score;
+    A.lo.tr_term = c->d_tr_term; A.lo.tr_best = c->d_tr_best; A.lo.tr_inc = c->d_tr_inc;
+    A.lo.tr_best_step = c->d_tr_best_step; A.lo.tr_anc = c->d_tr_anc; A.lo.tr_digest = c->d_tr_digest;
     if (use_wpc(c->dm)) return rp_launch_anneal_wpc(c, A);
     int nt; size_t smem;
     rp_anneal_smem_bytes(c, &nt, &smem);
     if (smem > 220 * 1024) return RP_ERR_RANGE;
-    if (smem > 48 * 1024)
+    if (smem > 32 * 1024)
         RP_CUDA(cudaFuncSetAttribute(k_anneal_level<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     k_anneal_level<256><<<c->Ppop, 256, smem, c->stream>>>(A);
-    ++g_rp_launches;
-    RP_CUDA(cudaGetLastError());
-    return RP_OK;
-}
-
-// ---------------------------------------------------------------------------------------------
-// Level barrier: incumbent update (strictly better trajectory-best, lowest slot on ties) and,
-// unless this was the last level, Boltzmann weights + systematic resampling -> ancestors.
-// One CTA; the population has at most a few tens of thousands of members.
-// ---------------------------------------------------------------------------------------------
-#define LE_THREADS 1024
-
-struct LevelEndArgs {
-    RpDims dm;
-    int Ppop, level, last, log_cap;
-    u64 cq;
-    u32 key0, key1;
-    const i64 *term, *best;
-    const int *best_step, *best_nlog;
-    const u64 *digest;
-    const uint2 *log;
-    const char *blob_src;             // chain states the level started from (indexed through anc)
-    RpBlob bl;
-    int *anc;
-    u64 *F;
-    int *inc_layout;
-    i64 *inc_score;
-    // trace (nullable)
-    i64 *tr_term, *tr_best, *tr_inc;
-    int *tr_best_step, *tr_anc;
-    u64 *tr_digest;
-};
-
-__global__ void __launch_bounds__(LE_THREADS)
-k_level_end(const LevelEndArgs A)
-{
-    __shared__ i64 r0[LE_THREADS / 32], r1[LE_THREADS / 32], r2[LE_THREADS / 32];
-    __shared__ int rj[LE_THREADS / 32];
-    __shared__ u64 rsum[LE_THREADS / 32];
-    __shared__ int win_j, do_update;
-    __shared__ i64 Emin_s;
-    __shared__ u64 carry_s;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int P = A.Ppop;
-
-    // trace copies of the per-chain reports
-    if (A.tr_term) {
-        const size_t o = (size_t)A.level * P;
-        for (int x = tid; x < 3 * P; x += LE_THREADS) { A.tr_term[o * 3 + x] = A.term[x]; A.tr_best[o * 3 + x] = A.best[x]; }
-        for (int x = tid; x < P; x += LE_THREADS) { A.tr_best_step[o + x] = A.best_step[x]; A.tr_digest[o + x] = A.digest[x]; }
-    }
-
-    // ---- incumbent: lexicographic argmin of the trajectory-best scores, lowest slot first ----
-    i64 b0 = 0x7fffffffffffffffll, b1 = b0, b2 = b0;
-    int bj = 0x7fffffff;
-    for (int j = tid; j < P; j += LE_THREADS) {
-        i64 s0 = A.best[3 * (size_t)j], s1 = A.best[3 * (size_t)j + 1], s2 = A.best[3 * (size_t)j + 2];
-        if (rp_lex_less(s0, s1, s2, b0, b1, b2)) { b0 = s0; b1 = s1; b2 = s2; bj = j; }   // ascending j: first wins
-    }
-    for (int o = 16; o; o >>= 1) {
-        i64 o0 = __shfl_xor_sync(0xffffffffu, b0, o), o1 = __shfl_xor_sync(0xffffffffu, b1, o);
-        i64 o2 = __shfl_xor_sync(0xffffffffu, b2, o);
-        int oj = __shfl_xor_sync(0xffffffffu, bj, o);
-        bool take = rp_lex_less(o0, o1, o2, b0, b1, b2) || (o0 == b0 && o1 == b1 && o2 == b2 && oj < bj);
-        if (take) { b0 = o0; b1 = o1; b2 = o2; bj = oj; }
-    }
-    if (lane == 0) { r0[warp] = b0; r1[warp] = b1; r2[warp] = b2; rj[warp] = bj; }
-    __syncthreads();
-    if (tid == 0) {
-        for (int w = 1; w < LE_THREADS / 32; ++w) {
-            bool take = rp_lex_less(r0[w], r1[w], r2[w], b0, b1, b2) ||
-                        (r0[w] == b0 && r1[w] == b1 && r2[w] == b2 && rj[w] < bj);
-            if (take) { b0 = r0[w]; b1 = r1[w]; b2 = r2[w]; bj = rj[w]; }
-        }
-        win_j = bj;
-        do_update = rp_lex_less(b0, b1, b2, A.inc_score[0], A.inc_score[1], A.inc_score[2]);
-        if (do_update) { A.inc_score[0] = b0; A.inc_score[1] = b1; A.inc_score[2] = b2; }
-    }
-    __syncthreads();
-    if (do_update) {
-        const int w = win_j;
-        const unsigned short *cs = (const unsigned short *)(A.blob_src + (size_t)A.anc[w] * A.bl.bytes + A.bl.off_cell);
-        for (int i = tid; i < A.dm.N; i += LE_THREADS) A.inc_layout[i] = cs[i];
-        __syncthreads();
-        if (tid == 0) {      // replay the accepted moves up to the trajectory-best step
-            const uint2 *lg = A.log + (size_t)w * A.log_cap;
-            const int n = A.best_nlog[w];
-            for (int x = 0; x < n; ++x) {
-                const uint2 m = lg[x];
-                const int i = (int)m.x;
-                if (m.y & 0x80000000u) A.inc_layout[i] = (int)(m.y & 0x7fffffffu);
-                else {
-                    const int i2 = (int)m.y;
-                    const int c = A.inc_layout[i];
-                    A.inc_layout[i] = A.inc_layout[i2];
-                    A.inc_layout[i2] = c;
-                }
-            }
-        }
-    }
-    __syncthreads();
-    if (A.tr_inc && tid < 3) A.tr_inc[(size_t)A.level * 3 + tid] = A.inc_score[tid];
-
-    if (A.last) {            // the terminal states are the population as they stand
-        for (int m = tid; m < P; m += LE_THREADS) A.anc[m] = m;
-        return;
-    }
-
-    // ---- resampling -------------------------------------------------------------------------
-    i64 emin = 0x7fffffffffffffffll;
-    for (int j = tid; j < P; j += LE_THREADS) {
-        i64 e = rp_energy(A.term[3 * (size_t)j], A.term[3 * (size_t)j + 1], A.term[3 * (size_t)j + 2]);
-        emin = e < emin ? e : emin;
-    }
-    for (int o = 16; o; o >>= 1) { i64 x = __shfl_xor_sync(0xffffffffu, emin, o); emin = x < emin ? x : emin; }
-    if (lane == 0) r0[warp] = emin;
-    __syncthreads();
-    if (tid == 0) {
-        for (int w = 1; w < LE_THREADS / 32; ++w) emin = r0[w] < emin ? r0[w] : emin;
-        Emin_s = emin;
-        carry_s = 0;
-    }
-    __syncthreads();
-    emin = Emin_s;
-    const u64 M = (u64)(emin > A.dm.SC ? emin : A.dm.SC);
-    // inclusive prefix sums of the weights, 1024 members per round
-    for (int base = 0; base < P; base += LE_THREADS) {
-        const int j = base + tid;
-        u64 w = 0;
-        if (j < P) {
-            const i64 e = rp_energy(A.term[3 * (size_t)j], A.term[3 * (size_t)j + 1], A.term[3 * (size_t)j + 2]);
-            unsigned __int128 eq = ((unsigned __int128)(u64)(e - emin) << 32) / (unsigned __int128)M;
-            const unsigned __int128 cap = (((unsigned __int128)1) << 48) - 1;
-            if (eq > cap) eq = cap;
-            unsigned __int128 z = (eq * (unsigned __int128)A.cq) >> 16;
-            const unsigned __int128 zcap = ((unsigned __int128)1) << 40;
-            if (z > zcap) z = zcap;
-            w = rp_exp2neg((u64)z);
-        }
-        u64 v = w;
-        for (int o = 1; o < 32; o <<= 1) { u64 x = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += x; }
-        if (lane == 31) rsum[warp] = v;
-        __syncthreads();
-        if (warp == 0) {
-            u64 s = rsum[lane];
-            for (int o = 1; o < 32; o <<= 1) { u64 x = __shfl_up_sync(0xffffffffu, s, o); if (lane >= o) s += x; }
-            rsum[lane] = s;
-        }
-        __syncthreads();
-        const u64 before = carry_s + (warp ? rsum[warp - 1] : 0);
-        if (j < P) A.F[j] = before + v;
-        __syncthreads();
-        if (tid == LE_THREADS - 1) carry_s = before + v;
-        __syncthreads();
-    }
-    const u64 Ftot = A.F[P - 1];
-    const uint4 xw = rp_philox(0u, (u32)A.level, 0u, 3u, A.key0, A.key1);
-    const u64 u0 = (u64)(((unsigned __int128)xw.x * Ftot) >> 32);
-    for (int m = tid; m < P; m += LE_THREADS) {
-        const unsigned __int128 pos = (unsigned __int128)u0 + (unsigned __int128)m * Ftot;
-        int lo = 0, hi = P - 1;                 // smallest j with P*F[j] > pos
-        while (lo < hi) {
-            const int mid = (lo + hi) >> 1;
-            if ((unsigned __int128)P * A.F[mid] > pos) hi = mid; else lo = mid + 1;
-        }
-        A.anc[m] = lo;
-        if (A.tr_anc) A.tr_anc[(size_t)A.level * P + m] = lo;
-    }
-}
-
-int rp_launch_level_end(rp_ctx *c, int level, int n_levels)
-{
-    LevelEndArgs A;
-    A.dm = c->dm; A.Ppop = c->Ppop; A.level = level; A.last = (level == n_levels - 1); A.log_cap = c->log_cap;
-    A.cq = c->h_levels[level].cq;
-    A.key0 = (u32)c->cfg.seed; A.key1 = (u32)(c->cfg.seed >> 32);
-    A.term = c->d_term; A.best = c->d_best; A.best_step = c->d_best_step; A.best_nlog = c->d_best_nlog;
-    A.digest = c->d_digest; A.log = c->d_log;
-    A.blob_src = c->buf[c->cur].blob; A.bl = c->bl;
-    A.anc = c->d_anc; A.F = c->d_F;
-    A.inc_layout = c->d_inc_layout; A.inc_score = c->d_inc_score;
-    A.tr_term = c->d_tr_term; A.tr_best = c->d_tr_best; A.tr_inc = c->d_tr_inc;
-    A.tr_best_step = c->d_tr_best_step; A.tr_anc = c->d_tr_anc; A.tr_digest = c->d_tr_digest;
-    k_level_end<<<1, LE_THREADS, 0, c->stream>>>(A);
     ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
     return RP_OK;

@@ -4,6 +4,18 @@
 #pragma once
 #include "rp_score.cuh"
 
+// Outputs of the level barrier (incumbent, next ancestors, per-level trace).
+struct LevelOut {
+    int *done;                 // arrival counter of the chain CTAs (zero between launches)
+    int *anc_out;              // [P_pop] ancestors for the next level
+    u64 *F;                    // [P_pop] cumulative resampling weights
+    int *inc_layout;           // [N]
+    i64 *inc_score;            // [3]
+    i64 *tr_term, *tr_best, *tr_inc;     // trace (nullable)
+    int *tr_best_step, *tr_anc;
+    u64 *tr_digest;
+};
+
 struct AnnealArgs {
     RpDims dm;
     RpBlob bl;
@@ -13,8 +25,8 @@ struct AnnealArgs {
     const char *blob_src;  char *blob_dst;
     const int *W_src;      int *W_dst;
     const int *anc;
-    int level, steps, log_cap;
-    u64 tau, rho_q32, guide_q32;
+    int level, steps, log_cap, Ppop, last;
+    u64 tau, cq, rho_q32, guide_q32;
     u32 key0, key1;
     i64 *term, *best;
     int *best_step, *best_nlog;
@@ -22,6 +34,7 @@ struct AnnealArgs {
     uint2 *log;
     i64 *counters;
     int *status;
+    LevelOut lo;
 };
 
 #define SPEC 32                 // steps speculated per round = lanes of the leading warp

@@ -14,7 +14,7 @@
 // by its warp straight from its registers, and everything speculated after it is discarded
 // and redone; if none is accepted the next NW follow.  This is step-for-step the sequential
 // chain of Algorithm 3: a later step is only ever scored against the state it would have seen.
-#include "rp_anneal.cuh"
+#include "rp_level_end.cuh"
 
 struct ChainS {                 // bookkeeping of the chain within this level
     i64 B[3];                   // trajectory-best score
@@ -308,6 +308,7 @@ k_anneal_wpc(const AnnealArgs A)
         atomicAdd((u64 *)&A.counters[0], (u64)A.steps);
         if (src != j) atomicAdd((u64 *)&A.counters[5], (u64)2 * dm.RG * dm.LP * 4);
     }
+    rp_finish_level(A, tid, NT);
 }
 
 #define WPC_WARPS 4
@@ -335,7 +336,7 @@ int rp_launch_anneal_wpc(rp_ctx *c, const AnnealArgs &A)
     const int chunks = ((dm.LP >> 2) + 31) / 32;
 #define LAUNCH(WS_, CH_)                                                                              \
     do {                                                                                              \
-        if (smem > 48 * 1024)                                                                         \
+        if (smem > 32 * 1024)                                                                         \
             RP_CUDA(cudaFuncSetAttribute(k_anneal_wpc<WPC_WARPS, WS_, CH_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
         k_anneal_wpc<WPC_WARPS, WS_, CH_><<<c->Ppop, WPC_WARPS * 32, smem, c->stream>>>(A);           \
     } while (0)

@@ -32,15 +32,50 @@ extern "C" const char *rp_strerror(int s)
     }
 }
 
+// Device memory comes from one stream-ordered pool per device that keeps freed blocks cached
+// (release threshold = unlimited), so that planning window after window does not pay for
+// cudaMalloc/cudaFree; rp_release_cached_memory() hands the cache back to the driver.
+#define RP_MAX_DEVICES 64
+static cudaMemPool_t g_pools[RP_MAX_DEVICES];
+static bool g_pool_ready[RP_MAX_DEVICES];
+
+static int get_pool(int device, cudaMemPool_t *out)
+{
+    if (device < 0 || device >= RP_MAX_DEVICES) return RP_ERR_ARG;
+    if (!g_pool_ready[device]) {
+        cudaMemPoolProps props;
+        memset(&props, 0, sizeof props);
+        props.allocType = cudaMemAllocationTypePinned;
+        props.handleTypes = cudaMemHandleTypeNone;
+        props.location.type = cudaMemLocationTypeDevice;
+        props.location.id = device;
+        RP_CUDA(cudaMemPoolCreate(&g_pools[device], &props));
+        unsigned long long keep = ~0ull;
+        RP_CUDA(cudaMemPoolSetAttribute(g_pools[device], cudaMemPoolAttrReleaseThreshold, &keep));
+        g_pool_ready[device] = true;
+    }
+    *out = g_pools[device];
+    return RP_OK;
+}
+
+extern "C" int rp_release_cached_memory(void)
+{
+    for (int d = 0; d < RP_MAX_DEVICES; ++d)
+        if (g_pool_ready[d]) RP_CUDA(cudaMemPoolTrimTo(g_pools[d], 0));
+    return RP_OK;
+}
+
 template <class T>
-static int dev_alloc(T **p, size_t n)
+static int dev_alloc(rp_ctx *c, T **p, size_t n)
 {
     *p = nullptr;
     if (n == 0) n = 1;
-    RP_CUDA(cudaMalloc((void **)p, n * sizeof(T)));
+    cudaMemPool_t pool;
+    RP_TRY(get_pool(c->device, &pool));
+    RP_CUDA(cudaMallocFromPoolAsync((void **)p, n * sizeof(T), pool, c->stream));
     return RP_OK;
 }
-static void dev_free(void *p) { if (p) cudaFree(p); }
+static void dev_free(rp_ctx *c, void *p) { if (p) cudaFreeAsync(p, c->stream); }
 
 static bool is_device_ptr(const void *p)
 {
@@ -60,20 +95,20 @@ static int copy_out(rp_ctx *c, void *dst, const void *src, size_t bytes)
 static void free_population(rp_ctx *c)
 {
     for (int b = 0; b < 2; ++b) {
-        dev_free(c->buf[b].blob); dev_free(c->buf[b].W);
+        dev_free(c, c->buf[b].blob); dev_free(c, c->buf[b].W);
         c->buf[b].blob = nullptr; c->buf[b].W = nullptr;
     }
-    dev_free(c->d_anc); dev_free(c->d_term); dev_free(c->d_best); dev_free(c->d_best_step);
-    dev_free(c->d_best_nlog); dev_free(c->d_digest); dev_free(c->d_log); dev_free(c->d_F);
-    c->d_anc = nullptr; c->d_term = nullptr; c->d_best = nullptr; c->d_best_step = nullptr;
+    dev_free(c, c->d_anc); dev_free(c, c->d_anc_next); dev_free(c, c->d_done); dev_free(c, c->d_term); dev_free(c, c->d_best); dev_free(c, c->d_best_step);
+    dev_free(c, c->d_best_nlog); dev_free(c, c->d_digest); dev_free(c, c->d_log); dev_free(c, c->d_F);
+    c->d_anc = nullptr; c->d_anc_next = nullptr; c->d_done = nullptr; c->d_term = nullptr; c->d_best = nullptr; c->d_best_step = nullptr;
     c->d_best_nlog = nullptr; c->d_digest = nullptr; c->d_log = nullptr; c->d_F = nullptr;
     c->log_cap = 0;
 }
 
 static void free_trace(rp_ctx *c)
 {
-    dev_free(c->d_tr_term); dev_free(c->d_tr_best); dev_free(c->d_tr_inc);
-    dev_free(c->d_tr_best_step); dev_free(c->d_tr_anc); dev_free(c->d_tr_digest);
+    dev_free(c, c->d_tr_term); dev_free(c, c->d_tr_best); dev_free(c, c->d_tr_inc);
+    dev_free(c, c->d_tr_best_step); dev_free(c, c->d_tr_anc); dev_free(c, c->d_tr_digest);
     c->d_tr_term = c->d_tr_best = c->d_tr_inc = nullptr;
     c->d_tr_best_step = c->d_tr_anc = nullptr;
     c->d_tr_digest = nullptr;
@@ -82,10 +117,10 @@ static void free_trace(rp_ctx *c)
 
 static void free_eval(rp_ctx *c)
 {
-    dev_free(c->d_eval_score); dev_free(c->d_eval_f64); dev_free(c->d_eval_W);
-    dev_free(c->d_eval_cells);
+    dev_free(c, c->d_eval_score); dev_free(c, c->d_eval_f64); dev_free(c, c->d_eval_W);
+    dev_free(c, c->d_eval_cells); dev_free(c, c->d_eval_Esum); dev_free(c, c->d_eval_tickets);
     c->d_eval_score = nullptr; c->d_eval_f64 = nullptr; c->d_eval_W = nullptr;
-    c->d_eval_cells = nullptr;
+    c->d_eval_cells = nullptr; c->d_eval_Esum = nullptr; c->d_eval_tickets = nullptr;
     c->eval_cap = 0; c->eval_W_n = 0;
 }
 
@@ -94,10 +129,10 @@ extern "C" void rp_destroy(rp_ctx *c)
     if (!c) return;
     cudaStreamSynchronize(c->stream);
     free_population(c); free_trace(c); free_eval(c);
-    dev_free(c->own_t); dev_free(c->own_a); dev_free(c->d_edp); dev_free(c->d_dp_list); dev_free(c->d_dp_off);
-    dev_free(c->d_Lagg); dev_free(c->d_pi); dev_free(c->d_inv); dev_free(c->d_rank_load); dev_free(c->d_q);
-    dev_free(c->d_status); dev_free(c->d_sort_keys); dev_free(c->d_seed_layout); dev_free(c->d_pack_out);
-    dev_free(c->d_counters); dev_free(c->d_inc_layout); dev_free(c->d_inc_score); dev_free(c->d_static);
+    dev_free(c, c->own_t); dev_free(c, c->own_a); dev_free(c, c->d_edp); dev_free(c, c->d_dp_list); dev_free(c, c->d_dp_off);
+    dev_free(c, c->d_Lagg); dev_free(c, c->d_pi); dev_free(c, c->d_inv); dev_free(c, c->d_rank_load); dev_free(c, c->d_q);
+    dev_free(c, c->d_status); dev_free(c, c->d_sort_keys); dev_free(c, c->d_seed_layout); dev_free(c, c->d_pack_out);
+    dev_free(c, c->d_counters); dev_free(c, c->d_inc_layout); dev_free(c, c->d_inc_score); dev_free(c, c->d_static);
     free(c->h_levels); free(c->h_t);
     free(c);
 }
@@ -161,9 +196,9 @@ static int window_load_impl(rp_ctx *c, const rp_config *cfg, const int32_t *leng
     do {
         // rank loads must fit int32: W <= k * C * |D_g|
         if ((double)dm.k * dm.C * maxshard >= 2147483648.0) { st = RP_ERR_RANGE; break; }
-        if ((st = dev_alloc(&c->d_edp, D)) != RP_OK) break;
-        if ((st = dev_alloc(&c->d_dp_list, D)) != RP_OK) break;
-        if ((st = dev_alloc(&c->d_dp_off, G + 1)) != RP_OK) break;
+        if ((st = dev_alloc(c, &c->d_edp, D)) != RP_OK) break;
+        if ((st = dev_alloc(c, &c->d_dp_list, D)) != RP_OK) break;
+        if ((st = dev_alloc(c, &c->d_dp_off, G + 1)) != RP_OK) break;
         cudaMemcpyAsync(c->d_edp, edp, sizeof(int) * D, cudaMemcpyHostToDevice, c->stream);
         cudaMemcpyAsync(c->d_dp_list, list, sizeof(int) * D, cudaMemcpyHostToDevice, c->stream);
         cudaMemcpyAsync(c->d_dp_off, off, sizeof(int) * (G + 1), cudaMemcpyHostToDevice, c->stream);
@@ -179,31 +214,31 @@ static int window_load_impl(rp_ctx *c, const rp_config *cfg, const int32_t *leng
         c->d_t = lengths;
         RP_CUDA(cudaMemcpyAsync(c->h_t, lengths, sizeof(int) * N, cudaMemcpyDeviceToHost, c->stream));
     } else {
-        RP_TRY(dev_alloc(&c->own_t, N));
+        RP_TRY(dev_alloc(c, &c->own_t, N));
         RP_CUDA(cudaMemcpyAsync(c->own_t, lengths, sizeof(int) * N, cudaMemcpyHostToDevice, c->stream));
         memcpy(c->h_t, lengths, sizeof(int) * N);
         c->d_t = c->own_t;
     }
     if (is_device_ptr(demand)) c->d_a = demand;
     else {
-        RP_TRY(dev_alloc(&c->own_a, n_a));
+        RP_TRY(dev_alloc(c, &c->own_a, n_a));
         RP_CUDA(cudaMemcpyAsync(c->own_a, demand, sizeof(int) * n_a, cudaMemcpyHostToDevice, c->stream));
         c->d_a = c->own_a;
     }
-    RP_TRY(dev_alloc(&c->d_Lagg, (size_t)L * E));
-    RP_TRY(dev_alloc(&c->d_pi, (size_t)L * E));
-    RP_TRY(dev_alloc(&c->d_inv, (size_t)L * E));
-    RP_TRY(dev_alloc(&c->d_rank_load, (size_t)L * P));
-    RP_TRY(dev_alloc(&c->d_q, (size_t)N * L * P));
-    RP_TRY(dev_alloc(&c->d_status, RP_SW_COUNT));
+    RP_TRY(dev_alloc(c, &c->d_Lagg, (size_t)L * E));
+    RP_TRY(dev_alloc(c, &c->d_pi, (size_t)L * E));
+    RP_TRY(dev_alloc(c, &c->d_inv, (size_t)L * E));
+    RP_TRY(dev_alloc(c, &c->d_rank_load, (size_t)L * P));
+    RP_TRY(dev_alloc(c, &c->d_q, (size_t)N * L * P));
+    RP_TRY(dev_alloc(c, &c->d_status, RP_SW_COUNT));
     int n_pow2 = 1;
     while (n_pow2 < N) n_pow2 <<= 1;
-    RP_TRY(dev_alloc(&c->d_sort_keys, (size_t)2 * n_pow2));
-    RP_TRY(dev_alloc(&c->d_seed_layout, N));
-    RP_TRY(dev_alloc(&c->d_pack_out, 4));
-    RP_TRY(dev_alloc(&c->d_counters, 8));
-    RP_TRY(dev_alloc(&c->d_inc_layout, N));
-    RP_TRY(dev_alloc(&c->d_inc_score, 3));
+    RP_TRY(dev_alloc(c, &c->d_sort_keys, (size_t)2 * n_pow2));
+    RP_TRY(dev_alloc(c, &c->d_seed_layout, N));
+    RP_TRY(dev_alloc(c, &c->d_pack_out, 4));
+    RP_TRY(dev_alloc(c, &c->d_counters, 8));
+    RP_TRY(dev_alloc(c, &c->d_inc_layout, N));
+    RP_TRY(dev_alloc(c, &c->d_inc_score, 3));
     RP_TRY(reset_status(c));
 
     // input checks + aggregate expert load in one pass over the demand tensor
@@ -269,18 +304,23 @@ static int ensure_eval_scratch(rp_ctx *c, size_t n, bool want_W)
 {
     const RpDims &dm = c->dm;
     if (n > c->eval_cap) {
-        dev_free(c->d_eval_score); dev_free(c->d_eval_f64); dev_free(c->d_eval_cells);
+        dev_free(c, c->d_eval_score); dev_free(c, c->d_eval_f64); dev_free(c, c->d_eval_cells);
+        dev_free(c, c->d_eval_Esum); dev_free(c, c->d_eval_tickets);
         c->d_eval_score = nullptr; c->d_eval_f64 = nullptr; c->d_eval_cells = nullptr;
+        c->d_eval_Esum = nullptr; c->d_eval_tickets = nullptr;
         c->eval_cap = 0;
-        RP_TRY(dev_alloc(&c->d_eval_score, n * 3));
-        RP_TRY(dev_alloc(&c->d_eval_f64, n * 3));
-        RP_TRY(dev_alloc(&c->d_eval_cells, n * dm.N));
+        RP_TRY(dev_alloc(c, &c->d_eval_score, n * 3));
+        RP_TRY(dev_alloc(c, &c->d_eval_f64, n * 3));
+        RP_TRY(dev_alloc(c, &c->d_eval_cells, n * dm.N));
+        RP_TRY(dev_alloc(c, &c->d_eval_Esum, n * dm.RG));
+        RP_TRY(dev_alloc(c, &c->d_eval_tickets, n));
+        RP_CUDA(cudaMemsetAsync(c->d_eval_tickets, 0, sizeof(int) * n, c->stream));
         c->eval_cap = n;
     }
     if (want_W && (int)n > c->eval_W_n) {
-        dev_free(c->d_eval_W);
+        dev_free(c, c->d_eval_W);
         c->d_eval_W = nullptr; c->eval_W_n = 0;
-        RP_TRY(dev_alloc(&c->d_eval_W, n * dm.RG * dm.LP));
+        RP_TRY(dev_alloc(c, &c->d_eval_W, n * dm.RG * dm.LP));
         c->eval_W_n = (int)n;
     }
     return RP_OK;
@@ -308,21 +348,24 @@ extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
     free_population(c); free_eval(c);
     const size_t P = (size_t)c->Ppop, wn = (size_t)dm.RG * dm.LP;
     for (int b = 0; b < 2; ++b) {
-        RP_TRY(dev_alloc(&c->buf[b].blob, P * (size_t)c->bl.bytes));
-        RP_TRY(dev_alloc(&c->buf[b].W, P * wn));
+        RP_TRY(dev_alloc(c, &c->buf[b].blob, P * (size_t)c->bl.bytes));
+        RP_TRY(dev_alloc(c, &c->buf[b].W, P * wn));
     }
-    RP_TRY(dev_alloc(&c->d_anc, P));
-    RP_TRY(dev_alloc(&c->d_term, P * 3));
-    RP_TRY(dev_alloc(&c->d_best, P * 3));
-    RP_TRY(dev_alloc(&c->d_best_step, P));
-    RP_TRY(dev_alloc(&c->d_best_nlog, P));
-    RP_TRY(dev_alloc(&c->d_digest, P));
-    RP_TRY(dev_alloc(&c->d_F, P));
+    RP_TRY(dev_alloc(c, &c->d_anc, P));
+    RP_TRY(dev_alloc(c, &c->d_anc_next, P));
+    RP_TRY(dev_alloc(c, &c->d_done, 1));
+    RP_CUDA(cudaMemsetAsync(c->d_done, 0, sizeof(int), c->stream));
+    RP_TRY(dev_alloc(c, &c->d_term, P * 3));
+    RP_TRY(dev_alloc(c, &c->d_best, P * 3));
+    RP_TRY(dev_alloc(c, &c->d_best_step, P));
+    RP_TRY(dev_alloc(c, &c->d_best_nlog, P));
+    RP_TRY(dev_alloc(c, &c->d_digest, P));
+    RP_TRY(dev_alloc(c, &c->d_F, P));
     c->cur = 0;
     // every member starts as the length-only seed: evaluate it once into slot 0 and let all
     // slots descend from slot 0
-    dev_free(c->d_static); c->d_static = nullptr;
-    RP_TRY(dev_alloc(&c->d_static, (size_t)c->sl.bytes));
+    dev_free(c, c->d_static); c->d_static = nullptr;
+    RP_TRY(dev_alloc(c, &c->d_static, (size_t)c->sl.bytes));
     RP_TRY(rp_launch_build_static(c));
     RP_TRY(ensure_eval_scratch(c, 1, false));
     RP_TRY(rp_launch_cells_from_layouts(c, c->d_seed_layout, 1, c->d_eval_cells));
@@ -361,16 +404,16 @@ extern "C" int rp_eval_population(rp_ctx *c, const int32_t *layouts, int32_t n, 
         const int *dl = layouts;
         int *tmp = nullptr;
         if (!is_device_ptr(layouts)) {
-            RP_TRY(dev_alloc(&tmp, (size_t)n * dm.N));
+            RP_TRY(dev_alloc(c, &tmp, (size_t)n * dm.N));
             cudaError_t e = cudaMemcpyAsync(tmp, layouts, sizeof(int) * (size_t)n * dm.N, cudaMemcpyHostToDevice, c->stream);
-            if (e != cudaSuccess) { dev_free(tmp); g_rp_last_cuda_error = (int)e; return RP_ERR_CUDA; }
+            if (e != cudaSuccess) { dev_free(c, tmp); g_rp_last_cuda_error = (int)e; return RP_ERR_CUDA; }
             dl = tmp;
         }
         RP_TRY(reset_status(c));
         int st = rp_launch_cells_from_layouts(c, dl, n, c->d_eval_cells);
         int sw[RP_SW_COUNT];
         if (st == RP_OK) st = read_status(c, sw);
-        dev_free(tmp);
+        dev_free(c, tmp);
         RP_TRY(st);
         if (sw[RP_SW_BAD_LAYOUT]) return RP_ERR_ARG;
     } else {
@@ -422,43 +465,38 @@ extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *
     const u64 guide_q32 = (u64)floor(p->p_guide * 4294967296.0);
     // accepted-move log
     if (c->log_cap < p->steps_per_level) {
-        dev_free(c->d_log); c->d_log = nullptr; c->log_cap = 0;
-        RP_TRY(dev_alloc(&c->d_log, P * (size_t)p->steps_per_level));
+        dev_free(c, c->d_log); c->d_log = nullptr; c->log_cap = 0;
+        RP_TRY(dev_alloc(c, &c->d_log, P * (size_t)p->steps_per_level));
         c->log_cap = p->steps_per_level;
     }
     // trace
     free_trace(c);
-    RP_TRY(dev_alloc(&c->d_tr_term, (size_t)NL * P * 3));
-    RP_TRY(dev_alloc(&c->d_tr_best, (size_t)NL * P * 3));
-    RP_TRY(dev_alloc(&c->d_tr_inc, (size_t)NL * 3));
-    RP_TRY(dev_alloc(&c->d_tr_best_step, (size_t)NL * P));
-    RP_TRY(dev_alloc(&c->d_tr_digest, (size_t)NL * P));
-    RP_TRY(dev_alloc(&c->d_tr_anc, (size_t)(NL > 1 ? NL - 1 : 1) * P));
+    RP_TRY(dev_alloc(c, &c->d_tr_term, (size_t)NL * P * 3));
+    RP_TRY(dev_alloc(c, &c->d_tr_best, (size_t)NL * P * 3));
+    RP_TRY(dev_alloc(c, &c->d_tr_inc, (size_t)NL * 3));
+    RP_TRY(dev_alloc(c, &c->d_tr_best_step, (size_t)NL * P));
+    RP_TRY(dev_alloc(c, &c->d_tr_digest, (size_t)NL * P));
+    RP_TRY(dev_alloc(c, &c->d_tr_anc, (size_t)(NL > 1 ? NL - 1 : 1) * P));
     c->trace_levels = NL;
     RP_CUDA(cudaMemsetAsync(c->d_counters, 0, sizeof(i64) * 8, c->stream));
     RP_TRY(reset_status(c));
 
-    cudaEvent_t ev[3];
-    for (int x = 0; x < 3; ++x) RP_CUDA(cudaEventCreate(&ev[x]));
-    float ms_chains = 0.f, ms_barrier = 0.f;
+    cudaEvent_t ev[2] = { nullptr, nullptr };
+    if (stats) for (int x = 0; x < 2; ++x) RP_CUDA(cudaEventCreate(&ev[x]));
+    float ms_chains = 0.f;
     int st = RP_OK;
+    if (stats) cudaEventRecord(ev[0], c->stream);
     for (int n = 0; n < NL && st == RP_OK; ++n) {
-        cudaEventRecord(ev[0], c->stream);
-        st = rp_launch_anneal_level(c, n, p, rho_q32, guide_q32);
-        cudaEventRecord(ev[1], c->stream);
-        if (st == RP_OK) st = rp_launch_level_end(c, n, NL);
-        cudaEventRecord(ev[2], c->stream);
+        st = rp_launch_anneal_level(c, n, NL, p, rho_q32, guide_q32);
         c->cur = 1 - c->cur;          // the terminal states are the next level's sources
-        if (stats) {
-            if (cudaEventSynchronize(ev[2]) != cudaSuccess) { st = RP_ERR_CUDA; break; }
-            float a = 0.f, b = 0.f;
-            cudaEventElapsedTime(&a, ev[0], ev[1]);
-            cudaEventElapsedTime(&b, ev[1], ev[2]);
-            ms_chains += a; ms_barrier += b;
-        }
+        { int *sw = c->d_anc; c->d_anc = c->d_anc_next; c->d_anc_next = sw; }
     }
+    if (stats) cudaEventRecord(ev[1], c->stream);
     cudaError_t e = cudaStreamSynchronize(c->stream);
-    for (int x = 0; x < 3; ++x) cudaEventDestroy(ev[x]);
+    if (stats) {
+        if (e == cudaSuccess) cudaEventElapsedTime(&ms_chains, ev[0], ev[1]);
+        for (int x = 0; x < 2; ++x) cudaEventDestroy(ev[x]);
+    }
     if (st == RP_OK && e != cudaSuccess) { g_rp_last_cuda_error = (int)e; st = RP_ERR_CUDA; }
     RP_TRY(st);
     {
@@ -471,8 +509,8 @@ extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *
         RP_CUDA(cudaMemcpy(cn, c->d_counters, sizeof cn, cudaMemcpyDeviceToHost));
         stats->proposed = cn[0]; stats->feasible = cn[1]; stats->accepted = cn[2]; stats->improved = cn[3];
         stats->move_bytes = cn[4]; stats->gather_bytes = cn[5];
-        stats->kernel_launches = 2 * (int64_t)NL;
-        stats->ms_chains = ms_chains; stats->ms_barrier = ms_barrier;
+        stats->kernel_launches = (int64_t)NL;
+        stats->ms_chains = ms_chains; stats->ms_barrier = 0.0;   // the barrier runs inside the chain kernels
     }
     c->stage = 4;
     return RP_OK;
@@ -547,7 +585,7 @@ extern "C" int rp_debug_dump(rp_ctx *c, int what, int32_t index, void *buf, int6
         case RP_DUMP_SEED_LAYOUT: if (c->stage < 3) return RP_ERR_STATE; src = c->d_seed_layout; need = sizeof(int) * dm.N; break;
         case RP_DUMP_POPULATION: {
             need = sizeof(int) * P * dm.N;
-            if ((st = dev_alloc((int **)&tmp, P * dm.N)) != RP_OK) return st;
+            if ((st = dev_alloc(c, (int **)&tmp, P * dm.N)) != RP_OK) return st;
             k_gather_cells<<<c->Ppop, 256, 0, c->stream>>>(c->buf[c->cur].blob, c->bl, c->d_anc, dm.N, nullptr, (int *)tmp);
             ++g_rp_launches;
             src = tmp;
@@ -557,7 +595,7 @@ extern "C" int rp_debug_dump(rp_ctx *c, int what, int32_t index, void *buf, int6
         case RP_DUMP_ESUM: src = c->buf[c->cur].blob + (size_t)member * c->bl.bytes + c->bl.off_Esum; need = sizeof(i64) * dm.RG; break;
         case RP_DUMP_CELL_T: case RP_DUMP_CELL_Q: case RP_DUMP_CELL_CNT: {
             size_t K = dm.K;
-            if ((st = dev_alloc((i64 **)&tmp, 3 * K)) != RP_OK) return st;
+            if ((st = dev_alloc(c, (i64 **)&tmp, 3 * K)) != RP_OK) return st;
             i64 *T = (i64 *)tmp, *Q = T + K;
             int *cnt = (int *)(Q + K);
             k_cell_stats<<<1, 256, 0, c->stream>>>((const unsigned short *)(c->buf[c->cur].blob + (size_t)member * c->bl.bytes + c->bl.off_cell),
@@ -579,12 +617,12 @@ extern "C" int rp_debug_dump(rp_ctx *c, int what, int32_t index, void *buf, int6
             src = c->d_eval_W + (size_t)index * dm.RG * dm.LP; need = sizeof(int) * (size_t)dm.RG * dm.LP; break;
         default: return RP_ERR_ARG;
     }
-    if (what >= RP_DUMP_TRACE_TERM && what <= RP_DUMP_TRACE_INCUMBENT && c->trace_levels == 0) { dev_free(tmp); return RP_ERR_STATE; }
-    if ((int64_t)need != bytes) { dev_free(tmp); return RP_ERR_ARG; }
+    if (what >= RP_DUMP_TRACE_TERM && what <= RP_DUMP_TRACE_INCUMBENT && c->trace_levels == 0) { dev_free(c, tmp); return RP_ERR_STATE; }
+    if ((int64_t)need != bytes) { dev_free(c, tmp); return RP_ERR_ARG; }
     cudaError_t e = cudaSuccess;
     if (need) e = cudaMemcpyAsync(buf, src, need, cudaMemcpyDefault, c->stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
-    dev_free(tmp);
+    dev_free(c, tmp);
     if (e != cudaSuccess) { g_rp_last_cuda_error = (int)e; return RP_ERR_CUDA; }
     return RP_OK;
 }
@@ -614,13 +652,12 @@ static int dbg_map(const TI *in, size_t in_per, TO *out, size_t out_per, int64_t
     if (!in || !out || n < 0) return RP_ERR_ARG;
     if (n == 0) return RP_OK;
     TI *din = nullptr; TO *dout = nullptr;
-    RP_TRY(dev_alloc(&din, (size_t)n * in_per));
-    int st = dev_alloc(&dout, (size_t)n * out_per);
-    if (st != RP_OK) { dev_free(din); return st; }
+    RP_CUDA(cudaMalloc((void **)&din, sizeof(TI) * (size_t)n * in_per));
+    if (cudaMalloc((void **)&dout, sizeof(TO) * (size_t)n * out_per) != cudaSuccess) { cudaFree(din); return RP_ERR_CUDA; }
     cudaError_t e = cudaMemcpy(din, in, sizeof(TI) * n * in_per, cudaMemcpyDefault);
     if (e == cudaSuccess) { launch(din, dout); ++g_rp_launches; e = cudaGetLastError(); }
     if (e == cudaSuccess) e = cudaMemcpy(out, dout, sizeof(TO) * n * out_per, cudaMemcpyDefault);
-    dev_free(din); dev_free(dout);
+    cudaFree(din); cudaFree(dout);
     if (e != cudaSuccess) { g_rp_last_cuda_error = (int)e; return RP_ERR_CUDA; }
     return RP_OK;
 }

@@ -119,6 +119,8 @@ struct rp_ctx {
     char *d_static;            // static tables block
     int cur;                   // buffer holding the current population
     int *d_anc;                // [P_pop] which member of buf[cur] each slot continues from
+    int *d_anc_next;           // [P_pop] written by the level barrier, swapped with d_anc
+    int *d_done;               // arrival counter of the chain CTAs
     // per-level results
     i64 *d_term;               // [P_pop][3]
     i64 *d_best;               // [P_pop][3]
@@ -143,6 +145,8 @@ struct rp_ctx {
     int *d_eval_W;             // W of explicitly evaluated layouts (n <= 64), for inspection
     int eval_W_n;
     unsigned short *d_eval_cells;
+    i64 *d_eval_Esum;          // [n][RG] row-shard sums handed to the finishing CTA
+    int *d_eval_tickets;       // [n] arrival counters, zero between launches
     size_t eval_cap;
     RpLevel *h_levels;         // host copy of the per-level schedule integers
     int levels_cap;
@@ -163,8 +167,7 @@ int rp_launch_eval(rp_ctx *c, const unsigned short *cells, int n, int *W_out, ch
 int rp_launch_build_static(rp_ctx *c);
 void rp_make_layouts(const RpDims &dm, RpBlob *bl, RpStatic *sl);
 int rp_launch_cells_from_layouts(rp_ctx *c, const int *layouts, int n, unsigned short *cells);
-int rp_launch_anneal_level(rp_ctx *c, int level, const rp_anneal_params *prm, u64 rho_q32, u64 guide_q32);
-int rp_launch_level_end(rp_ctx *c, int level, int n_levels);
+int rp_launch_anneal_level(rp_ctx *c, int level, int n_levels, const rp_anneal_params *prm, u64 rho_q32, u64 guide_q32);
 int rp_launch_validate(rp_ctx *c);
 int rp_anneal_smem_bytes(const rp_ctx *c, int *threads, size_t *bytes);
 

@@ -8,19 +8,19 @@
 #include "rp_common.cuh"
 
 #define K1_WARPS 8
-#define K1_CHUNK 32            // samples per CTA
+#define K1_CHUNK_MAX 32        // samples per CTA, at most
 
 // One warp owns one layer of a chunk of samples: it walks the chunk's rows a[i][l][0..E),
 // each row read with coalesced 4-byte loads, keeps the column sums of that layer in
 // registers (NC = ceil(E/32) columns per lane) and checks every row sum against k*t_i.
 template <int NC>
 __global__ void __launch_bounds__(K1_WARPS * 32)
-k_check_reduce(const int *__restrict__ a, const int *__restrict__ t, RpDims dm,
+k_check_reduce(const int *__restrict__ a, const int *__restrict__ t, RpDims dm, int chunk,
                i64 *__restrict__ Lagg, int *__restrict__ status)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int i0 = blockIdx.x * K1_CHUNK;
-    const int i1 = min(dm.N, i0 + K1_CHUNK);
+    const int i0 = blockIdx.x * chunk;
+    const int i1 = min(dm.N, i0 + chunk);
     for (int l = warp; l < dm.L; l += K1_WARPS) {
         i64 acc[NC];
 #pragma unroll
@@ -56,10 +56,13 @@ int rp_launch_check_reduce(rp_ctx *c)
 {
     const RpDims &dm = c->dm;
     RP_CUDA(cudaMemsetAsync(c->d_Lagg, 0, sizeof(i64) * dm.L * dm.E, c->stream));
-    int grid = (dm.N + K1_CHUNK - 1) / K1_CHUNK;
+    // enough CTAs to fill the GPU on small windows, up to 32 samples per CTA on large ones
+    int chunk = (dm.N + 2 * 148 - 1) / (2 * 148);
+    chunk = chunk < 4 ? 4 : (chunk > K1_CHUNK_MAX ? K1_CHUNK_MAX : chunk);
+    int grid = (dm.N + chunk - 1) / chunk;
     int nc = (dm.E + 31) / 32;
 #define K1_CASE(NC_)                                                                         \
-    k_check_reduce<NC_><<<grid, K1_WARPS * 32, 0, c->stream>>>(c->d_a, c->d_t, dm, c->d_Lagg, \
+    k_check_reduce<NC_><<<grid, K1_WARPS * 32, 0, c->stream>>>(c->d_a, c->d_t, dm, chunk, c->d_Lagg, \
                                                                c->d_status)
     if (nc <= 1) K1_CASE(1);
     else if (nc <= 2) K1_CASE(2);
@@ -182,7 +185,7 @@ int rp_launch_project(rp_ctx *c)
     const RpDims &dm = c->dm;
     size_t smem = (size_t)K3_WARPS * dm.E * sizeof(int);
     if ((size_t)(K3_WARPS + dm.L) * dm.E * sizeof(int) <= 96 * 1024) smem += (size_t)dm.L * dm.E * sizeof(int);
-    if (smem > 48 * 1024)
+    if (smem > 32 * 1024)
         RP_CUDA(cudaFuncSetAttribute(k_project, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     long long rows = (long long)dm.N * dm.L;
     long long want = (rows + K3_WARPS - 1) / K3_WARPS;

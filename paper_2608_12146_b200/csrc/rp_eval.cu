@@ -30,11 +30,14 @@ int rp_launch_cells_from_layouts(rp_ctx *c, const int *layouts, int n, unsigned 
     return RP_OK;
 }
 
+// grid = (layouts, splits): the CTAs of a layout share its row-shards (8 per CTA, one per warp);
+// the CTA that finishes last (atomic ticket) gathers the row-shard sums and scores the layout.
 __global__ void __launch_bounds__(EVAL_THREADS)
 k_eval(const unsigned short *__restrict__ cells, const int *__restrict__ t, const int *__restrict__ q,
        const int *__restrict__ edp, const int *__restrict__ dp_list, const int *__restrict__ dp_off,
        RpDims dm, RpBlob bl, int *__restrict__ W_out, char *__restrict__ blob_out,
-       i64 *__restrict__ score_out, double *__restrict__ f64_out)
+       i64 *__restrict__ score_out, double *__restrict__ f64_out, i64 *__restrict__ Esum_g,
+       int *__restrict__ tickets)
 {
     extern __shared__ __align__(16) unsigned char smraw[];
     // layout: Q[K] u64 | Esum[RG] | Afx[RG] | U[G] | T[K] | cnt[K] | off[RG+1] | cur[RG] | members[N] | cell_of[N]
@@ -48,6 +51,7 @@ k_eval(const unsigned short *__restrict__ cells, const int *__restrict__ t, cons
     int *cur = off + dm.RG + 1;
     int *members = cur + dm.RG;
     unsigned short *cell_of = (unsigned short *)(members + dm.N);
+    __shared__ int last_s;
     RpSmemState st = { cell_of, T, Q, cnt, Esum, Afx, U };
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = EVAL_THREADS / 32;
@@ -67,7 +71,8 @@ k_eval(const unsigned short *__restrict__ cells, const int *__restrict__ t, cons
         members[off[rg] + atomicAdd(&cur[rg], 1)] = i;
     }
     __syncthreads();
-    for (int rg = warp; rg < dm.RG; rg += nwarps) {
+    i64 *esum_lay = Esum_g + (size_t)lay * dm.RG;
+    for (int rg = blockIdx.y * nwarps + warp; rg < dm.RG; rg += gridDim.y * nwarps) {
         const int m0 = off[rg], m1 = off[rg + 1];
         int *wout = W_out ? W_out + ((size_t)lay * dm.RG + rg) * dm.LP : nullptr;
         i64 es = rp_warp_layer_max_sum(dm, lane, [&](int x) {
@@ -76,8 +81,19 @@ k_eval(const unsigned short *__restrict__ cells, const int *__restrict__ t, cons
             if (wout) wout[x] = s;
             return s;
         });
-        if (lane == 0) Esum[rg] = es;
+        if (lane == 0) esum_lay[rg] = es;
     }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const int ticket = atomicAdd(&tickets[lay], 1);
+        last_s = (ticket == (int)gridDim.y - 1);
+        if (last_s) tickets[lay] = 0;                 // ready for the next launch
+    }
+    __syncthreads();
+    if (!last_s) return;
+    __threadfence();
+    for (int rg = tid; rg < dm.RG; rg += EVAL_THREADS) Esum[rg] = ((volatile i64 *)esum_lay)[rg];
     __syncthreads();
     i64 sc[3];
     rp_rows_to_score(dm, st, dp_list, dp_off, tid, EVAL_THREADS, sc);
@@ -122,10 +138,16 @@ int rp_launch_eval(rp_ctx *c, const unsigned short *cells, int n, int *W_out, ch
     const RpDims &dm = c->dm;
     size_t smem = eval_smem_bytes(dm);
     if (smem > 220 * 1024) return RP_ERR_RANGE;
-    if (smem > 48 * 1024)
+    if (smem > 32 * 1024)
         RP_CUDA(cudaFuncSetAttribute(k_eval, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k_eval<<<n, EVAL_THREADS, smem, c->stream>>>(cells, c->d_t, c->d_q, c->d_edp, c->d_dp_list, c->d_dp_off, dm,
-                                                c->bl, W_out, blob_out, score_out, f64_out);
+    // few layouts: split each one's row-shards over several CTAs so the GPU is not left idle
+    int splits = (2 * 148 + n - 1) / n;
+    const int max_splits = (dm.RG + EVAL_THREADS / 32 - 1) / (EVAL_THREADS / 32);
+    if (splits > max_splits) splits = max_splits;
+    if (splits < 1) splits = 1;
+    k_eval<<<dim3(n, splits), EVAL_THREADS, smem, c->stream>>>(cells, c->d_t, c->d_q, c->d_edp, c->d_dp_list, c->d_dp_off,
+                                                              dm, c->bl, W_out, blob_out, score_out, f64_out,
+                                                              c->d_eval_Esum, c->d_eval_tickets);
     ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
     return RP_OK;

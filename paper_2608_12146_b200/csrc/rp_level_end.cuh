@@ -1,0 +1,166 @@
+// Level barrier of the population annealing (Algorithm 3): incumbent update (strictly better
+// trajectory-best, lowest slot on ties) and, unless this was the last level, Boltzmann
+// weights + systematic resampling -> ancestors.  Runs inside the chain kernel, in whichever
+// CTA finishes last (arrival counter), so a level costs one launch.
+#pragma once
+#include "rp_anneal.cuh"
+
+#define LE_MAX_WARPS 32
+
+// Loads of values other CTAs wrote during this launch go to L2.
+#define LE_LD(x) __ldcg(&(x))
+
+// Called by all threads of one CTA (nt a multiple of 32, at most 1024).
+__device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int nt)
+{
+    __shared__ i64 r0[LE_MAX_WARPS], r1[LE_MAX_WARPS], r2[LE_MAX_WARPS];
+    __shared__ int rj[LE_MAX_WARPS];
+    __shared__ u64 rsum[LE_MAX_WARPS];
+    __shared__ int win_j, do_update;
+    __shared__ i64 Emin_s;
+    __shared__ u64 carry_s;
+    const int lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
+    const int P = A.Ppop;
+    const LevelOut &O = A.lo;
+
+    // trace copies of the per-chain reports
+    if (O.tr_term) {
+        const size_t o = (size_t)A.level * P;
+        for (int x = tid; x < 3 * P; x += nt) { O.tr_term[o * 3 + x] = LE_LD(A.term[x]); O.tr_best[o * 3 + x] = LE_LD(A.best[x]); }
+        for (int x = tid; x < P; x += nt) { O.tr_best_step[o + x] = LE_LD(A.best_step[x]); O.tr_digest[o + x] = LE_LD(A.digest[x]); }
+    }
+
+    // ---- incumbent: lexicographic argmin of the trajectory-best scores, lowest slot first ----
+    i64 b0 = 0x7fffffffffffffffll, b1 = b0, b2 = b0;
+    int bj = 0x7fffffff;
+    for (int j = tid; j < P; j += nt) {
+        i64 s0 = LE_LD(A.best[3 * (size_t)j]), s1 = LE_LD(A.best[3 * (size_t)j + 1]), s2 = LE_LD(A.best[3 * (size_t)j + 2]);
+        if (rp_lex_less(s0, s1, s2, b0, b1, b2)) { b0 = s0; b1 = s1; b2 = s2; bj = j; }   // ascending j: first wins
+    }
+    for (int o = 16; o; o >>= 1) {
+        i64 o0 = __shfl_xor_sync(0xffffffffu, b0, o), o1 = __shfl_xor_sync(0xffffffffu, b1, o);
+        i64 o2 = __shfl_xor_sync(0xffffffffu, b2, o);
+        int oj = __shfl_xor_sync(0xffffffffu, bj, o);
+        bool take = rp_lex_less(o0, o1, o2, b0, b1, b2) || (o0 == b0 && o1 == b1 && o2 == b2 && oj < bj);
+        if (take) { b0 = o0; b1 = o1; b2 = o2; bj = oj; }
+    }
+    if (lane == 0) { r0[warp] = b0; r1[warp] = b1; r2[warp] = b2; rj[warp] = bj; }
+    __syncthreads();
+    if (tid == 0) {
+        for (int w = 1; w < nwarps; ++w) {
+            bool take = rp_lex_less(r0[w], r1[w], r2[w], b0, b1, b2) ||
+                        (r0[w] == b0 && r1[w] == b1 && r2[w] == b2 && rj[w] < bj);
+            if (take) { b0 = r0[w]; b1 = r1[w]; b2 = r2[w]; bj = rj[w]; }
+        }
+        win_j = bj;
+        do_update = rp_lex_less(b0, b1, b2, O.inc_score[0], O.inc_score[1], O.inc_score[2]);
+        if (do_update) { O.inc_score[0] = b0; O.inc_score[1] = b1; O.inc_score[2] = b2; }
+    }
+    __syncthreads();
+    if (do_update) {
+        const int w = win_j;
+        const unsigned short *cs = (const unsigned short *)(A.blob_src + (size_t)A.anc[w] * A.bl.bytes + A.bl.off_cell);
+        for (int i = tid; i < A.dm.N; i += nt) O.inc_layout[i] = cs[i];
+        __syncthreads();
+        if (tid == 0) {      // replay the accepted moves up to the trajectory-best step
+            const uint2 *lg = A.log + (size_t)w * A.log_cap;
+            const int n = LE_LD(A.best_nlog[w]);
+            for (int x = 0; x < n; ++x) {
+                const uint2 m = LE_LD(lg[x]);
+                const int i = (int)m.x;
+                if (m.y & 0x80000000u) O.inc_layout[i] = (int)(m.y & 0x7fffffffu);
+                else {
+                    const int i2 = (int)m.y;
+                    const int c = O.inc_layout[i];
+                    O.inc_layout[i] = O.inc_layout[i2];
+                    O.inc_layout[i2] = c;
+                }
+            }
+        }
+    }
+    __syncthreads();
+    if (O.tr_inc && tid < 3) O.tr_inc[(size_t)A.level * 3 + tid] = O.inc_score[tid];
+
+    if (A.last) {            // the terminal states are the population as they stand
+        for (int m = tid; m < P; m += nt) O.anc_out[m] = m;
+        return;
+    }
+
+    // ---- resampling -------------------------------------------------------------------------
+    i64 emin = 0x7fffffffffffffffll;
+    for (int j = tid; j < P; j += nt) {
+        i64 e = rp_energy(LE_LD(A.term[3 * (size_t)j]), LE_LD(A.term[3 * (size_t)j + 1]), LE_LD(A.term[3 * (size_t)j + 2]));
+        emin = e < emin ? e : emin;
+    }
+    for (int o = 16; o; o >>= 1) { i64 x = __shfl_xor_sync(0xffffffffu, emin, o); emin = x < emin ? x : emin; }
+    if (lane == 0) r0[warp] = emin;
+    __syncthreads();
+    if (tid == 0) {
+        for (int w = 1; w < nwarps; ++w) emin = r0[w] < emin ? r0[w] : emin;
+        Emin_s = emin;
+        carry_s = 0;
+    }
+    __syncthreads();
+    emin = Emin_s;
+    const u64 M = (u64)(emin > A.dm.SC ? emin : A.dm.SC);
+    // inclusive prefix sums of the weights, nt members per round
+    for (int base = 0; base < P; base += nt) {
+        const int j = base + tid;
+        u64 w = 0;
+        if (j < P) {
+            const i64 e = rp_energy(LE_LD(A.term[3 * (size_t)j]), LE_LD(A.term[3 * (size_t)j + 1]), LE_LD(A.term[3 * (size_t)j + 2]));
+            unsigned __int128 eq = ((unsigned __int128)(u64)(e - emin) << 32) / (unsigned __int128)M;
+            const unsigned __int128 cap = (((unsigned __int128)1) << 48) - 1;
+            if (eq > cap) eq = cap;
+            unsigned __int128 z = (eq * (unsigned __int128)A.cq) >> 16;
+            const unsigned __int128 zcap = ((unsigned __int128)1) << 40;
+            if (z > zcap) z = zcap;
+            w = rp_exp2neg((u64)z);
+        }
+        u64 v = w;
+        for (int o = 1; o < 32; o <<= 1) { u64 x = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += x; }
+        if (lane == 31) rsum[warp] = v;
+        __syncthreads();
+        if (warp == 0) {
+            u64 s = (lane < nwarps) ? rsum[lane] : 0;
+            for (int o = 1; o < 32; o <<= 1) { u64 x = __shfl_up_sync(0xffffffffu, s, o); if (lane >= o) s += x; }
+            rsum[lane] = s;
+        }
+        __syncthreads();
+        const u64 before = carry_s + (warp ? rsum[warp - 1] : 0);
+        if (j < P) O.F[j] = before + v;
+        __syncthreads();
+        if (tid == nt - 1) carry_s = before + v;
+        __syncthreads();
+    }
+    const u64 Ftot = O.F[P - 1];
+    const uint4 xw = rp_philox(0u, (u32)A.level, 0u, 3u, A.key0, A.key1);
+    const u64 u0 = (u64)(((unsigned __int128)xw.x * Ftot) >> 32);
+    for (int m = tid; m < P; m += nt) {
+        const unsigned __int128 pos = (unsigned __int128)u0 + (unsigned __int128)m * Ftot;
+        int lo = 0, hi = P - 1;                 // smallest j with P*F[j] > pos
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if ((unsigned __int128)P * O.F[mid] > pos) hi = mid; else lo = mid + 1;
+        }
+        O.anc_out[m] = lo;
+        if (O.tr_anc) O.tr_anc[(size_t)A.level * P + m] = lo;
+    }
+}
+
+// Tail of a chain CTA: publish, take a ticket, and let the last arrival run the level barrier.
+__device__ __forceinline__ void rp_finish_level(const AnnealArgs &A, int tid, int nt)
+{
+    __shared__ int is_last;
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const int ticket = atomicAdd(A.lo.done, 1);
+        is_last = (ticket == (int)gridDim.x - 1);
+        if (is_last) *A.lo.done = 0;
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    rp_level_end(A, tid, nt);
+}

@@ -10,11 +10,12 @@
 #define PACK_THREADS 1024
 
 __global__ void __launch_bounds__(PACK_THREADS)
-k_pack_ffd(const int *__restrict__ t, RpDims dm, int min_rows, u64 *__restrict__ keys_g, int n_pow2,
+k_pack_ffd(RpDims dm, const int *__restrict__ t, int min_rows, u64 *__restrict__ keys_g, int n_pow2,
            int *__restrict__ fill_g, int *__restrict__ cell_of, int *__restrict__ out)
 {
     extern __shared__ u64 keys_s[];
     u64 *keys = keys_g ? keys_g : keys_s;
+    int *fill = fill_g ? fill_g : (int *)(keys_s + (keys_g ? 0 : n_pow2));
     __shared__ i64 total_s;
     __shared__ int fail_s;
     const int tid = threadIdx.x;
@@ -48,32 +49,35 @@ k_pack_ffd(const int *__restrict__ t, RpDims dm, int min_rows, u64 *__restrict__
     i64 Rlb = (total_s + cap_row - 1) / cap_row;
     if (Rlb < 1) Rlb = 1;
     if (Rlb < min_rows) Rlb = min_rows;
+    const int t_min = dm.C - (int)(keys[dm.N - 1] >> 32);          // the shortest sample
     int Rstar = 0;
     for (i64 R = Rlb; R * dm.D <= dm.N && !Rstar; ++R) {
         const int K = (int)(R * dm.D);
-        for (int b = tid; b < K; b += PACK_THREADS) fill_g[b] = 0;
         if (tid == 0) fail_s = 0;
-        __syncthreads();
         // the K longest samples open the cells
         for (int x = tid; x < K; x += PACK_THREADS) {
-            int s = (int)(u32)keys[x];
-            fill_g[x] = t[s];
-            cell_of[s] = x;
+            const u64 key = keys[x];
+            fill[x] = dm.C - (int)(key >> 32);
+            cell_of[(u32)key] = x;
         }
         __syncthreads();
         if (tid < 32) {
+            // Cells before `lo` cannot take even the shortest sample any more; samples arrive
+            // in decreasing length, so skipping them leaves first-fit unchanged.
+            int lo = 0;
             for (int x = K; x < dm.N; ++x) {
-                const int s = (int)(u32)keys[x];
-                const int ts = t[s];
+                const u64 key = keys[x];
+                const int ts = dm.C - (int)(key >> 32);
+                while (lo < K && fill[lo] + t_min > dm.C) ++lo;
                 int found = -1;
-                for (int b0 = 0; b0 < K && found < 0; b0 += 32) {
-                    int b = b0 + tid;
-                    bool ok = (b < K) && (fill_g[b] + ts <= dm.C);
-                    unsigned m = __ballot_sync(0xffffffffu, ok);
+                for (int b0 = lo; b0 < K && found < 0; b0 += 32) {
+                    const int b = b0 + tid;
+                    const bool ok = (b < K) && (fill[b] + ts <= dm.C);
+                    const unsigned m = __ballot_sync(0xffffffffu, ok);
                     if (m) found = b0 + __ffs(m) - 1;
                 }
                 if (found < 0) { if (tid == 0) fail_s = 1; break; }
-                if (tid == 0) { fill_g[found] += ts; cell_of[s] = found; }
+                if (tid == 0) { fill[found] += ts; cell_of[(u32)key] = found; }
                 __syncwarp();
             }
         }
@@ -94,14 +98,14 @@ int rp_launch_pack(rp_ctx *c, int /*unused*/)
     const RpDims &dm = c->dm;
     int n_pow2 = 1;
     while (n_pow2 < dm.N) n_pow2 <<= 1;
-    size_t smem = (size_t)n_pow2 * sizeof(u64);
+    // sort keys (8 bytes each) and cell fills (4 bytes per cell, at most N cells) on chip when they fit
+    size_t smem = (size_t)n_pow2 * sizeof(u64) + (size_t)dm.N * sizeof(int);
     u64 *keys_g = nullptr;
-    if (smem > 128 * 1024) { keys_g = c->d_sort_keys; smem = 0; }
-    if (smem > 48 * 1024)
+    int *fill_g = nullptr;
+    if (smem > 160 * 1024) { keys_g = c->d_sort_keys; fill_g = (int *)(c->d_sort_keys + n_pow2); smem = 0; }
+    if (smem > 32 * 1024)
         RP_CUDA(cudaFuncSetAttribute(k_pack_ffd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    // fill scratch: reuse the front of the sort-key buffer's tail (allocated 2*n_pow2 u64)
-    int *fill_g = (int *)(c->d_sort_keys + n_pow2);
-    k_pack_ffd<<<1, PACK_THREADS, smem, c->stream>>>(c->d_t, dm, c->cfg.min_rows, keys_g, n_pow2, fill_g,
+    k_pack_ffd<<<1, PACK_THREADS, smem, c->stream>>>(dm, c->d_t, c->cfg.min_rows, keys_g, n_pow2, fill_g,
                                                     c->d_seed_layout, c->d_pack_out);
     ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
