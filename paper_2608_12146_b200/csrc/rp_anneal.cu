@@ -40,7 +40,7 @@ struct ChainB {                 // bookkeeping of the chain within this level
 // candidate at a time (two L*P slices of W from global memory plus the moved samples' demand
 // rows, 16-byte loads); the leading warp rebuilds the score and decides.
 template <int NT>
-__global__ void __launch_bounds__(NT)
+__global__ void __launch_bounds__(NT, 768 / NT)
 k_anneal_level(const AnnealArgs A)
 {
     const RpDims &dm = A.dm;
@@ -140,8 +140,13 @@ k_anneal_level(const AnnealArgs A)
                     const int *w1 = Wj + (size_t)rg1 * dm.LP, *w2 = Wj + (size_t)rg2 * dm.LP;
                     const int P = dm.P, LP = dm.LP;
                     if (vec) {
-                        rp_slices_vec<2, NT>(LP >> 2, P >> 2, (const int4 *)qi, (const int4 *)q2, (const int4 *)w1,
-                                             (const int4 *)w2, (int4 *)scratch, (int4 *)(scratch + slice_pad), tid, e1, e2);
+                        RpSliceRegs<2> regs;
+                        for (int base = 0; base < (LP >> 2); base += 2 * NT) {
+                            rp_slices_load<2, NT>(regs, base, LP >> 2, (const int4 *)qi, (const int4 *)q2, (const int4 *)w1,
+                                                  (const int4 *)w2, tid);
+                            rp_slices_reduce<2, NT>(regs, base, LP >> 2, P >> 2, (int4 *)scratch, (int4 *)(scratch + slice_pad),
+                                                    tid, e1, e2);
+                        }
                     } else {
                         for (int x = tid; x < LP; x += NT) {
                             int d = __ldg(qi + x);
@@ -310,7 +315,8 @@ k_anneal_level(const AnnealArgs A)
 
 // Thread count and shared-memory plan of the chain kernels.  Windows with L*P <= 512 use the
 // warp-per-candidate kernel; larger ones the cooperative kernel with 256 threads.
-size_t rp_wpc_smem_bytes(const RpDims &dm, const RpBlob &bl, const RpStatic &sl, int *w_in_smem);
+size_t rp_wpc_smem_bytes(const RpDims &dm, const RpBlob &bl, const RpStatic &sl, int nw, int *w_in_smem);
+int rp_wpc_warps(int pop_size);
 int rp_launch_anneal_wpc(rp_ctx *c, const AnnealArgs &A);
 
 static bool use_wpc(const RpDims &dm) { return dm.LP <= 512; }
@@ -320,11 +326,12 @@ int rp_anneal_smem_bytes(const rp_ctx *c, int *threads, size_t *bytes)
     const RpDims &dm = c->dm;
     if (use_wpc(dm)) {
         int ws = 0;
-        *threads = 128;
-        *bytes = rp_wpc_smem_bytes(dm, c->bl, c->sl, &ws);
+        const int nw = rp_wpc_warps(c->Ppop);
+        *threads = nw * 32;
+        *bytes = rp_wpc_smem_bytes(dm, c->bl, c->sl, nw, &ws);
         return ws;
     }
-    const int nt = 256;
+    const int nt = 128;
     const size_t slice_pad = ((size_t)dm.LP + 3) & ~(size_t)3;
     size_t b = (size_t)c->bl.bytes + c->sl.bytes + sizeof(int) * 2 * slice_pad + sizeof(i64) * (3 * (size_t)dm.K + 2 * (nt / 32)) +
                sizeof(StepRec) * SPEC + sizeof(ChainB) + sizeof(u64) + sizeof(MoveS) * SPEC;
@@ -360,8 +367,8 @@ int rp_launch_anneal_level(rp_ctx *c, int level, int n_levels, const rp_anneal_p
     rp_anneal_smem_bytes(c, &nt, &smem);
     if (smem > 220 * 1024) return RP_ERR_RANGE;
     if (smem > 32 * 1024)
-        RP_CUDA(cudaFuncSetAttribute(k_anneal_level<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k_anneal_level<256><<<c->Ppop, 256, smem, c->stream>>>(A);
+        RP_CUDA(cudaFuncSetAttribute(k_anneal_level<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    k_anneal_level<128><<<c->Ppop, 128, smem, c->stream>>>(A);
     ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
     return RP_OK;

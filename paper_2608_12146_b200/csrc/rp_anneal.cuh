@@ -122,46 +122,50 @@ __device__ __forceinline__ bool rp_propose(const RpDims &dm, const RpChainView &
 __device__ __forceinline__ int max4(const int4 &v) { return max(max(v.x, v.y), max(v.z, v.w)); }
 
 // Tentative rank loads of the two touched row-shards, W1' = W1 - d and W2' = W2 + d with
-// d = q[i] - q[i2] (relocation: d = q[i]), written to s1/s2, together with this thread's
-// share of sum_l max_p W' for both.  NTH threads cooperate (tid in [0,NTH)); whole warps must
-// call.  Vector form: 16-byte loads, CH chunks per thread in flight, ranks of a layer reduced
-// by segmented shuffles; needs P a power of two, 4 <= P <= 128.
+// d = q[i] - q[i2] (relocation: d = q[i]), in two halves: all loads of a pass are issued before any is consumed.  NTH threads cooperate (tid in
+// [0,NTH)); whole warps must call.  16-byte loads, CH chunks per thread in flight per pass;
+// ranks of a layer are reduced by segmented shuffles; needs P a power of two, 4 <= P <= 128.
+template <int CH>
+struct RpSliceRegs { int4 d[CH], a[CH], b[CH]; };
+
 template <int CH, int NTH>
-__device__ __forceinline__ void rp_slices_vec(int nchunks, int lanes_per_layer, const int4 *__restrict__ qi,
-                                              const int4 *__restrict__ q2, const int4 *w1, const int4 *w2,
-                                              int4 *s1, int4 *s2, int tid, i64 &e1, i64 &e2)
+__device__ __forceinline__ void rp_slices_load(RpSliceRegs<CH> &r, int base, int nchunks, const int4 *__restrict__ qi,
+                                               const int4 *__restrict__ q2, const int4 *w1, const int4 *w2, int tid)
+{
+#pragma unroll
+    for (int u = 0; u < CH; ++u) {
+        const int c = base + u * NTH + tid;
+        if (c < nchunks) {
+            r.d[u] = __ldg(qi + c);
+            if (q2) { const int4 o = __ldg(q2 + c); r.d[u].x -= o.x; r.d[u].y -= o.y; r.d[u].z -= o.z; r.d[u].w -= o.w; }
+            r.a[u] = w1[c];
+            r.b[u] = w2[c];
+        }
+    }
+}
+
+template <int CH, int NTH>
+__device__ __forceinline__ void rp_slices_reduce(const RpSliceRegs<CH> &r, int base, int nchunks, int lanes_per_layer,
+                                                 int4 *s1, int4 *s2, int tid, i64 &e1, i64 &e2)
 {
     const int lane = tid & 31;
-    for (int base = 0; base < nchunks; base += CH * NTH) {
-        int4 d[CH], a[CH], b[CH];
 #pragma unroll
-        for (int u = 0; u < CH; ++u) {
-            const int c = base + u * NTH + tid;
-            if (c < nchunks) {
-                d[u] = __ldg(qi + c);
-                if (q2) { const int4 o = __ldg(q2 + c); d[u].x -= o.x; d[u].y -= o.y; d[u].z -= o.z; d[u].w -= o.w; }
-                a[u] = w1[c];
-                b[u] = w2[c];
-            }
+    for (int u = 0; u < CH; ++u) {
+        const int c = base + u * NTH + tid;
+        int m1 = 0, m2 = 0;
+        if (c < nchunks) {
+            const int4 v1 = make_int4(r.a[u].x - r.d[u].x, r.a[u].y - r.d[u].y, r.a[u].z - r.d[u].z, r.a[u].w - r.d[u].w);
+            const int4 v2 = make_int4(r.b[u].x + r.d[u].x, r.b[u].y + r.d[u].y, r.b[u].z + r.d[u].z, r.b[u].w + r.d[u].w);
+            s1[c] = v1;
+            s2[c] = v2;
+            m1 = max4(v1);
+            m2 = max4(v2);
         }
-#pragma unroll
-        for (int u = 0; u < CH; ++u) {
-            const int c = base + u * NTH + tid;
-            int m1 = 0, m2 = 0;
-            if (c < nchunks) {
-                const int4 v1 = make_int4(a[u].x - d[u].x, a[u].y - d[u].y, a[u].z - d[u].z, a[u].w - d[u].w);
-                const int4 v2 = make_int4(b[u].x + d[u].x, b[u].y + d[u].y, b[u].z + d[u].z, b[u].w + d[u].w);
-                s1[c] = v1;
-                s2[c] = v2;
-                m1 = max4(v1);
-                m2 = max4(v2);
-            }
-            for (int o = lanes_per_layer >> 1; o; o >>= 1) {
-                m1 = max(m1, __shfl_xor_sync(0xffffffffu, m1, o));
-                m2 = max(m2, __shfl_xor_sync(0xffffffffu, m2, o));
-            }
-            if ((lane & (lanes_per_layer - 1)) == 0 && c < nchunks) { e1 += m1; e2 += m2; }
+        for (int o = lanes_per_layer >> 1; o; o >>= 1) {
+            m1 = max(m1, __shfl_xor_sync(0xffffffffu, m1, o));
+            m2 = max(m2, __shfl_xor_sync(0xffffffffu, m2, o));
         }
+        if ((lane & (lanes_per_layer - 1)) == 0 && c < nchunks) { e1 += m1; e2 += m2; }
     }
 }
 

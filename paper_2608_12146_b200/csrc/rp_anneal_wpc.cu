@@ -23,7 +23,7 @@ struct ChainS {                 // bookkeeping of the chain within this level
 };
 
 template <int NW, bool WS, int CH>
-__global__ void __launch_bounds__(NW * 32)
+__global__ void __launch_bounds__(NW * 32, 16 / NW)
 k_anneal_wpc(const AnnealArgs A)
 {
     constexpr int NT = NW * 32;
@@ -131,16 +131,28 @@ k_anneal_wpc(const AnnealArgs A)
                 if (my >= 0) {
                     m = mvs[my];
                     const bool swap = !m.reloc;
-                    rg1 = rg_of[m.c1]; rg2 = rg_of[m.c2];
-                    g1 = g_of[m.c1]; g2 = g_of[m.c2];
+                    const int c1 = m.c1, c2 = m.c2;
+                    rg1 = rg_of[c1]; rg2 = rg_of[c2];
+                    g1 = g_of[c1]; g2 = g_of[c2];
                     touchW = (rg1 != rg2);
+                    const int *qi = A.q + (size_t)m.i * dm.LP;
+                    const int *q2 = swap ? A.q + (size_t)m.i2 * dm.LP : nullptr;
+                    const int *w1 = Wj + (size_t)rg1 * dm.LP, *w2 = Wj + (size_t)rg2 * dm.LP;
+                    const int nchunks = dm.LP >> 2;
+                    RpSliceRegs<CH> regs;
+                    // (a) put the loads of the two slices and the demand rows in flight
+                    if (touchW && vec)
+                        rp_slices_load<CH, 32>(regs, 0, nchunks, (const int4 *)qi, (const int4 *)q2, (const int4 *)w1,
+                                               (const int4 *)w2, lane);
+                    // (b) tentative slices, busiest rank per layer, sum over layers
                     if (touchW) {
-                        const int *qi = A.q + (size_t)m.i * dm.LP;
-                        const int *q2 = swap ? A.q + (size_t)m.i2 * dm.LP : nullptr;
-                        const int *w1 = Wj + (size_t)rg1 * dm.LP, *w2 = Wj + (size_t)rg2 * dm.LP;
                         if (vec) {
-                            rp_slices_vec<CH, 32>(dm.LP >> 2, dm.P >> 2, (const int4 *)qi, (const int4 *)q2, (const int4 *)w1,
-                                                  (const int4 *)w2, (int4 *)my_s1, (int4 *)my_s2, lane, e1, e2);
+                            rp_slices_reduce<CH, 32>(regs, 0, nchunks, dm.P >> 2, (int4 *)my_s1, (int4 *)my_s2, lane, e1, e2);
+                            for (int base = CH * 32; base < nchunks; base += CH * 32) {
+                                rp_slices_load<CH, 32>(regs, base, nchunks, (const int4 *)qi, (const int4 *)q2,
+                                                       (const int4 *)w1, (const int4 *)w2, lane);
+                                rp_slices_reduce<CH, 32>(regs, base, nchunks, dm.P >> 2, (int4 *)my_s1, (int4 *)my_s2, lane, e1, e2);
+                            }
                         } else {
                             for (int x = lane; x < dm.LP; x += 32) {
                                 int d = __ldg(qi + x);
@@ -165,24 +177,31 @@ k_anneal_wpc(const AnnealArgs A)
                         e1 = warp_sum_i64(e1);
                         e2 = warp_sum_i64(e2);
                     }
-                    // exact new score and the Metropolis decision
-                    const int c1 = m.c1, c2 = m.c2;
-                    int fb0 = 0, fb2 = 0;
+                    // (c) the part of the new score that does not need the rank loads
+                    i64 S0 = 0, S1 = 0, S2 = 0, Ecur = 0, J1o = 0, J2o = 0, U1o = 0, U2o = 0;
+                    u64 thr = 0;
+                    u32 rflags = 0;
                     if (lane == 0) {
-                        const i64 S0 = Sc[0], S1 = Sc[1], S2 = Sc[2];
+                        S0 = Sc[0]; S1 = Sc[1]; S2 = Sc[2]; Ecur = Sc[3];
+                        const StepRec rr = recs[pos + my];
+                        thr = rr.thr; rflags = rr.flags;
                         const i64 ti = tt[m.i], t2 = swap ? tt[m.i2] : 0;
                         Ta = (i64)T[c1] - ti + t2; Qa = (i64)Q[c1] - ti * ti + t2 * t2;
                         Tb = (i64)T[c2] + ti - t2; Qb = (i64)Q[c2] + ti * ti - t2 * t2;
-                        if (!touchW) { e1 = Esum[rg1]; e2 = e1; }
                         if (identity_edp) { A1 = aC * Ta + bS * Qa; A2 = aC * Tb + bS * Qb; }
                         else {
                             A1 = rp_attention(dm, st, dpl, dpo, rowbase[c1] / dm.D, g1, c1, Ta, Qa, c2, Tb, Qb);
                             A2 = touchW ? rp_attention(dm, st, dpl, dpo, rowbase[c2] / dm.D, g2, c1, Ta, Qa, c2, Tb, Qb) : A1;
                         }
-                        const i64 J1o = Jfx[rg1], J2o = Jfx[rg2];
+                        J1o = Jfx[rg1]; J2o = Jfx[rg2];
+                        U1o = U[g1]; U2o = U[g2];
+                    }
+                    // (d) exact new score and the Metropolis decision
+                    int fb0 = 0, fb2 = 0;
+                    if (lane == 0) {
+                        if (!touchW) { e1 = Esum[rg1]; e2 = e1; }
                         J1n = A1 + dm.EC * e1; J2n = touchW ? A2 + dm.EC * e2 : J1n;
                         const i64 dJ1 = J1n - J1o, dJ2 = touchW ? J2n - J2o : 0;
-                        const i64 U1o = U[g1], U2o = U[g2];
                         if (g1 == g2) { U1n = U1o + dJ1 + dJ2; U2n = U1n; }
                         else { U1n = U1o + dJ1; U2n = U2o + dJ2; }
                         n1 = S1 + dJ1 + dJ2;
@@ -213,15 +232,13 @@ k_anneal_wpc(const AnnealArgs A)
                         if (lane == 0 && v > n2) n2 = v;
                     }
                     if (lane == 0) {
-                        const StepRec rr = recs[pos + my];
-                        const i64 Ecur = Sc[3];
-                        acc = rp_lex_less(n0, n1, n2, Sc[0], Sc[1], Sc[2]);
+                        acc = rp_lex_less(n0, n1, n2, S0, S1, S2);
                         en = rp_energy(n0, n1, n2);
                         if (!acc) {
-                            if (en <= Ecur || (rr.flags & 4u)) acc = true;
+                            if (en <= Ecur || (rflags & 4u)) acc = true;
                             else {
                                 const u64 M = (u64)(Ecur > dm.SC ? Ecur : dm.SC);
-                                const u64 bh = __umul64hi(rr.thr, M), bl = rr.thr * M;
+                                const u64 bh = __umul64hi(thr, M), bl = thr * M;
                                 acc = (bh >> 31) ? true : ((u64)(en - Ecur) < ((bh << 32) | (bl >> 32)));
                             }
                         }
@@ -311,34 +328,37 @@ k_anneal_wpc(const AnnealArgs A)
     rp_finish_level(A, tid, NT);
 }
 
-#define WPC_WARPS 4
+// Warps per chain: more warps score more candidates of a round at once (good when few chains
+// must hide a lot of latency), fewer warps let more chains be resident per SM.  Register use is
+// capped at 128 per thread, so NW warps per chain allow 16/NW chains per SM.
+int rp_wpc_warps(int pop_size)
+{
+    return pop_size <= 2 * 148 ? 8 : 4;
+}
 
 // Shared-memory bytes of the warp-per-candidate kernel; *w_in_smem says whether W fits on chip
-// beside a second CTA.
-size_t rp_wpc_smem_bytes(const RpDims &dm, const RpBlob &bl, const RpStatic &sl, int *w_in_smem)
+// while still leaving room for the 16/NW chains per SM that the register budget allows.
+size_t rp_wpc_smem_bytes(const RpDims &dm, const RpBlob &bl, const RpStatic &sl, int nw, int *w_in_smem)
 {
-    const int NT = WPC_WARPS * 32;
+    const int NT = nw * 32;
     const size_t slice_pad = ((size_t)dm.LP + 3) & ~(size_t)3;
-    size_t b = (size_t)bl.bytes + sl.bytes + sizeof(int) * WPC_WARPS * 2 * slice_pad + sizeof(i64) * 3 * dm.K +
-               sizeof(StepRec) * NT + sizeof(ChainS) + sizeof(u64) + sizeof(MoveS) * SPEC + sizeof(int) * (WPC_WARPS + 2);
+    size_t b = (size_t)bl.bytes + sl.bytes + sizeof(int) * nw * 2 * slice_pad + sizeof(i64) * 3 * dm.K +
+               sizeof(StepRec) * NT + sizeof(ChainS) + sizeof(u64) + sizeof(MoveS) * SPEC + sizeof(int) * (nw + 2);
     const size_t wbytes = sizeof(int) * ((((size_t)dm.RG * dm.LP) + 3) & ~(size_t)3);
-    *w_in_smem = (b + wbytes <= 110 * 1024);
+    const size_t per_cta = (size_t)220 * 1024 / (16 / nw);
+    *w_in_smem = (b + wbytes <= per_cta);
     if (*w_in_smem) b += wbytes;
     return (b + 15) & ~(size_t)15;
 }
 
-int rp_launch_anneal_wpc(rp_ctx *c, const AnnealArgs &A)
+template <int NW>
+static int launch_wpc(rp_ctx *c, const AnnealArgs &A, int ws, size_t smem, int chunks)
 {
-    const RpDims &dm = c->dm;
-    int ws = 0;
-    const size_t smem = rp_wpc_smem_bytes(dm, c->bl, c->sl, &ws);
-    if (smem > 220 * 1024) return RP_ERR_RANGE;
-    const int chunks = ((dm.LP >> 2) + 31) / 32;
 #define LAUNCH(WS_, CH_)                                                                              \
     do {                                                                                              \
         if (smem > 32 * 1024)                                                                         \
-            RP_CUDA(cudaFuncSetAttribute(k_anneal_wpc<WPC_WARPS, WS_, CH_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
-        k_anneal_wpc<WPC_WARPS, WS_, CH_><<<c->Ppop, WPC_WARPS * 32, smem, c->stream>>>(A);           \
+            RP_CUDA(cudaFuncSetAttribute(k_anneal_wpc<NW, WS_, CH_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+        k_anneal_wpc<NW, WS_, CH_><<<c->Ppop, NW * 32, smem, c->stream>>>(A);                         \
     } while (0)
     if (ws) { if (chunks <= 1) LAUNCH(true, 1); else if (chunks <= 2) LAUNCH(true, 2); else LAUNCH(true, 4); }
     else { if (chunks <= 1) LAUNCH(false, 1); else if (chunks <= 2) LAUNCH(false, 2); else LAUNCH(false, 4); }
@@ -346,4 +366,16 @@ int rp_launch_anneal_wpc(rp_ctx *c, const AnnealArgs &A)
     ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
     return RP_OK;
+}
+
+int rp_launch_anneal_wpc(rp_ctx *c, const AnnealArgs &A)
+{
+    const RpDims &dm = c->dm;
+    const int nw = rp_wpc_warps(c->Ppop);
+    int ws = 0;
+    const size_t smem = rp_wpc_smem_bytes(dm, c->bl, c->sl, nw, &ws);
+    if (smem > 220 * 1024) return RP_ERR_RANGE;
+    const int chunks = ((dm.LP >> 2) + 31) / 32;
+    if (nw == 8) return launch_wpc<8>(c, A, ws, smem, chunks);
+    return launch_wpc<4>(c, A, ws, smem, chunks);
 }
