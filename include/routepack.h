@@ -123,6 +123,27 @@ int rp_pack_rows(rp_ctx *ctx, int32_t *n_rows, int32_t *certified);
 int rp_eval_population(rp_ctx *ctx, const int32_t *layouts, int32_t n, int64_t *score_fx,
                        double *score_f64);
 
+/* The same scores as rp_eval_population, for callers that must not allocate device memory
+ * once they are running: a planner called from inside a training or serving loop whose
+ * framework has already handed all free device memory to its own pool, or from a section
+ * where an allocation would stall the whole device (cudaMalloc and cudaFree synchronise it).
+ * The paper has no counterpart; this is a deployment variant of the full evaluation.
+ * It calls no cudaMalloc/cudaFree or any allocating routine: its working memory (16-bit cell
+ * ids, row-shard sums, arrival counters; about 1.3 MiB) is a fixed array inside the library
+ * image, present on every GPU that loads the library until the process exits.
+ *   layouts [n][N] int32, score_fx [n][3] int64 (nullable), score_f64 [n][3] double
+ *   (nullable): all three must be DEVICE pointers (a host array would need a staging buffer).
+ *   Limits: n <= 1024, n*N <= 524288, n*R*G <= 32768; beyond them the call returns
+ *   RP_ERR_RANGE and does nothing (use rp_eval_population).
+ * The first call on a device looks up the device address of the fixed array
+ * (cudaGetSymbolAddress); make that first call before any stream capture.  The context's
+ * device must be the current device (RP_ERR_STATE otherwise).  All calls in the process share
+ * the one array and it keeps the previous call's contents (the call clears the part that must
+ * start at zero): two calls whose kernels overlap on the GPU, from different contexts or
+ * streams, race on it, so issue them one after the other. */
+int rp_eval_layouts_noalloc(rp_ctx *ctx, const int32_t *layouts, int32_t n, int64_t *score_fx,
+                            double *score_f64);
+
 /* Fixed-row population annealing (Algorithm 3): n_levels temperature levels; at each level
  * every member runs steps_per_level guided swap/relocation proposals with incremental
  * rescoring and the Metropolis rule, the incumbent takes any strictly better

@@ -22,7 +22,7 @@ STATUS_NAMES = {0: "RP_OK", -1: "RP_ERR_ARG", -2: "RP_ERR_SHAPE", -3: "RP_ERR_CO
                 -8: "RP_ERR_TIMEOUT", -9: "RP_ERR_INVALID_PLAN"}
 RP_OK = 0
 
-EXPORTS = ("rp_window_load", "rp_place_experts", "rp_pack_rows", "rp_eval_population", "rp_anneal",
+EXPORTS = ("rp_window_load", "rp_place_experts", "rp_pack_rows", "rp_eval_population", "rp_eval_layouts_noalloc", "rp_anneal",
            "rp_best", "rp_destroy", "rp_release_cached_memory", "rp_strerror", "rp_last_cuda_error", "rp_debug_dump",
            "rp_debug_nl2", "rp_debug_exp2neg", "rp_debug_philox", "rp_debug_launch_count")
 
@@ -75,6 +75,7 @@ def lib():
         L.rp_place_experts.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         L.rp_pack_rows.argtypes = [C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         L.rp_eval_population.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
+        L.rp_eval_layouts_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
         L.rp_anneal.argtypes = [C.c_void_p, C.POINTER(rp_anneal_params), C.POINTER(rp_anneal_stats)]
         L.rp_best.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.rp_debug_dump.argtypes = [C.c_void_p, C.c_int, C.c_int32, C.c_void_p, C.c_int64]
@@ -179,6 +180,19 @@ def rp_eval_population(ctx: Context, layouts=None, score_fx=None, score_f64=None
         score_f64 = np.empty((n, 3), np.float64)
     _check(lib().rp_eval_population(ctx.handle, _ptr(layouts), n, _ptr(score_fx), _ptr(score_f64)),
            "rp_eval_population")
+    return score_fx, score_f64
+
+
+def rp_eval_layouts_noalloc(ctx: Context, layouts, score_fx, score_f64):
+    """Scores of device-resident layouts into device-resident outputs without any allocation.
+
+    For callers that may not allocate once running (all device memory already belongs to a
+    framework's pool, or an allocation would stall the device).  ``layouts`` [n][N] int32 and
+    the outputs [n][3] int64 / float64 must be CUDA tensors; nothing is allocated here either.
+    """
+    n = int(layouts.shape[0])
+    _check(lib().rp_eval_layouts_noalloc(ctx.handle, _ptr(layouts), n, _ptr(score_fx), _ptr(score_f64)),
+           "rp_eval_layouts_noalloc")
     return score_fx, score_f64
 
 

@@ -202,3 +202,75 @@ int rp_launch_build_static(rp_ctx *c)
     RP_CUDA(cudaGetLastError());
     return RP_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Scoring layouts without allocating: the kernels above, with their scratch (16-bit cell ids,
+// row-shard sums, arrival counters) taken from a fixed array that is part of the library image
+// instead of from the context's allocator.
+// ---------------------------------------------------------------------------------------------
+#define RP_NOALLOC_MAX_LAYOUTS 1024            // layouts per call
+#define RP_NOALLOC_MAX_CELLS (1 << 19)         // n * N          (1 MiB of 16-bit cell ids)
+#define RP_NOALLOC_MAX_ROWSHARDS (1 << 15)     // n * R * G      (256 KiB of 64-bit sums)
+
+struct RpNoAllocScratch {
+    i64 esum[RP_NOALLOC_MAX_ROWSHARDS];
+    int tickets[RP_NOALLOC_MAX_LAYOUTS];
+    unsigned short cells[RP_NOALLOC_MAX_CELLS];
+};
+// About 1.3 MiB on every GPU that loads the library, held until the process exits.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(RpNoAllocScratch)];
+// Device address of the array above, per device (in host code the symbol itself is only a
+// stand-in, never a device address).
+static void *g_noalloc_addr[64];
+
+extern "C" int rp_eval_layouts_noalloc(rp_ctx *c, const int32_t *layouts, int32_t n, int64_t *score_fx,
+                                       double *score_f64)
+{
+    if (!c || !layouts || n < 1) return RP_ERR_ARG;
+    if (c->stage < 3) return RP_ERR_STATE;
+    const RpDims &dm = c->dm;
+    if (n > RP_NOALLOC_MAX_LAYOUTS || (long long)n * dm.N > RP_NOALLOC_MAX_CELLS ||
+        (long long)n * dm.RG > RP_NOALLOC_MAX_ROWSHARDS)
+        return RP_ERR_RANGE;                  // beyond the fixed scratch: use rp_eval_population
+    int cur = -1;
+    RP_CUDA(cudaGetDevice(&cur));
+    if (cur != c->device || cur < 0 || cur >= 64) return RP_ERR_STATE;
+    // every array must already be on the device: staging a host array would need memory
+    const void *ptrs[3] = { layouts, score_fx, score_f64 };
+    for (int x = 0; x < 3; ++x) {
+        if (!ptrs[x]) continue;
+        cudaPointerAttributes at;
+        if (cudaPointerGetAttributes(&at, ptrs[x]) != cudaSuccess) { cudaGetLastError(); return RP_ERR_ARG; }
+        if (at.type != cudaMemoryTypeDevice && at.type != cudaMemoryTypeManaged) return RP_ERR_ARG;
+    }
+    if (!g_noalloc_addr[cur]) {               // set-up, once per device, with that device current
+        void *p = nullptr;
+        RP_CUDA(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+        g_noalloc_addr[cur] = p;
+    }
+    RpNoAllocScratch *sc = (RpNoAllocScratch *)g_noalloc_addr[cur];
+    // the array keeps what the previous call left: the arrival counters must start at zero
+    RP_CUDA(cudaMemsetAsync(sc->tickets, 0, sizeof(int) * n, c->stream));
+    RP_CUDA(cudaMemsetAsync(c->d_status + RP_SW_BAD_LAYOUT, 0, sizeof(int), c->stream));
+    const long long total = (long long)n * dm.N;
+    k_layouts_to_cells<<<(int)((total + 255) / 256), 256, 0, c->stream>>>(layouts, total, dm.K, sc->cells, c->d_status);
+    ++g_rp_launches;
+    RP_CUDA(cudaGetLastError());
+    const size_t smem = eval_smem_bytes(dm);
+    if (smem > 220 * 1024) return RP_ERR_RANGE;
+    if (smem > 32 * 1024)
+        RP_CUDA(cudaFuncSetAttribute(k_eval, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    int splits = (2 * 148 + n - 1) / n;
+    const int max_splits = (dm.RG + EVAL_THREADS / 32 - 1) / (EVAL_THREADS / 32);
+    if (splits > max_splits) splits = max_splits;
+    if (splits < 1) splits = 1;
+    k_eval<<<dim3(n, splits), EVAL_THREADS, smem, c->stream>>>(sc->cells, c->d_t, c->d_q, c->d_edp, c->d_dp_list, c->d_dp_off,
+                                                              dm, c->bl, nullptr, nullptr, (i64 *)score_fx, score_f64, sc->esum,
+                                                              sc->tickets);
+    ++g_rp_launches;
+    RP_CUDA(cudaGetLastError());
+    int bad = 0;
+    RP_CUDA(cudaMemcpyAsync(&bad, c->d_status + RP_SW_BAD_LAYOUT, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+    RP_CUDA(cudaStreamSynchronize(c->stream));
+    return bad ? RP_ERR_ARG : RP_OK;
+}
