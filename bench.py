@@ -185,7 +185,14 @@ def run_cuda(args):
     rp.lib()
 
     spec = SPECS[args.workload]
-    w = make_window(spec)
+    overrides = {}
+    if args.pop:
+        overrides["pop_size"] = args.pop          # profiling aid: a smaller population of the same window
+    if args.levels:
+        overrides["n_levels"] = args.levels
+        overrides["sweeps"] = spec.steps_per_level * args.levels
+    w = make_window(spec, **overrides)
+    spec = w.spec
     s = spec
     moves_per_step = s.pop_size * s.n_levels * s.steps_per_level
     stream = torch.cuda.current_stream()
@@ -267,7 +274,8 @@ def run_cuda(args):
     per_launch_s = res["chain_ms"] * 1e-3 / res["chain_launches"]
     alg_bytes_per_launch = (res["move_bytes"] + res["gather_bytes"]) / res["chain_launches"]
     achieved = alg_bytes_per_launch / per_launch_s / 1e9
-    roofline = {"bound": "hbm", "kernel": "k_anneal_level", "achieved": achieved, "peak": peak, "unit": "GB/s",
+    chain_kernel = "k_anneal_wpc" if s.n_layers * s.ep_width <= 512 else "k_anneal_level"
+    roofline = {"bound": "hbm", "kernel": chain_kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_source": peak_kind, "traffic": None,
                 "algorithmic_bytes_per_launch": alg_bytes_per_launch,
                 "move_bytes_per_launch": res["move_bytes"] / res["chain_launches"],
@@ -334,6 +342,8 @@ def main():
     ap.add_argument("--workload", default="medium", choices=list(SPECS))
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--pop", type=int, default=0, help="override the population size (profiling aid)")
+    ap.add_argument("--levels", type=int, default=0, help="override the number of temperature levels (profiling aid)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "cuda":
         args.warmup = 3
