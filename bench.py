@@ -153,6 +153,21 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def reduce_job(ms_local, moves_local, dist=None, device="cpu"):
+    """Whole-job figures from one rank's: the slowest rank's time and the moves of all ranks.
+
+    With a process group (N > 1, replicas only) the time is the MAX over ranks and the moves
+    the SUM; without one the local values stand."""
+    if dist is None:
+        return float(ms_local), int(moves_local)
+    import torch
+    tmax = torch.tensor([float(ms_local)], dtype=torch.float64, device=device)
+    tsum = torch.tensor([float(moves_local)], dtype=torch.float64, device=device)
+    dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+    dist.all_reduce(tsum, op=dist.ReduceOp.SUM)
+    return float(tmax.item()), int(round(tsum.item()))
+
+
 def plan_once(rp, torch, w, t_in, a_in, outs, stream, want_stats=True):
     """One pass of the whole hot path through the C ABI; returns the annealing stats."""
     s = w.spec
@@ -257,16 +272,8 @@ def run_cuda(args):
     clocks = sampler.stop()
     e2e = timed_loop(t_pin, a_pin, outs_host, args.steps)
 
-    def max_over_ranks(x):
-        if dist is None:
-            return x
-        tt = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        return float(tt.item())
-
-    ms = max_over_ranks(res["ms"])
-    ms_e2e = max_over_ranks(e2e["ms"])
-    total_moves = moves_per_step * args.steps * world
+    ms, total_moves = reduce_job(res["ms"], moves_per_step * args.steps, dist, dev)
+    ms_e2e, _ = reduce_job(e2e["ms"], moves_per_step * args.steps, dist, dev)
     value = total_moves / (ms * 1e-3)
     e2e_value = total_moves / (ms_e2e * 1e-3)
 
