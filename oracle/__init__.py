@@ -191,6 +191,30 @@ def eval_f64(lengths, q, layout, R: int, C_cap: int, D: int, edp_of_dp=None,
     return out
 
 
+def diagnostics(lengths, q, Lagg, pi, layout, R: int, C_cap: int, D: int, edp_of_dp=None,
+                alpha=(1.0, 1.0), beta=(0.0, 1.0)) -> Dict[str, float]:
+    """CV_global before/after placement, S_EP, T_EP, eta_EP, attention and joint proxies of a layout."""
+    t = _i32(lengths)
+    q = _i32(q)
+    Lagg = np.ascontiguousarray(Lagg, np.int64)
+    pi = _i32(pi)
+    lay = _i32(layout)
+    _, L, P = q.shape
+    E = Lagg.shape[1]
+    edp = _edp(D, edp_of_dp)
+    G = int(edp.max()) + 1
+    al, be = _f64(alpha), _f64(beta)
+    cv = np.zeros(2)
+    peaks = np.zeros(3, np.int64)
+    aj = np.zeros(2)
+    eta = C.c_double(0.0)
+    lib().orc_diagnostics(C.c_int32(t.shape[0]), C.c_int32(L), C.c_int32(E), C.c_int32(P), C.c_int32(D), C.c_int32(G),
+                          C.c_int32(R), C.c_int32(C_cap), _p(edp), C.c_int32(al.shape[0]), _p(al), _p(be), _p(t), _p(q),
+                          _p(Lagg), _p(pi), _p(lay), _p(cv), _p(peaks), _p(aj), C.byref(eta))
+    return dict(cv_identity=float(cv[0]), cv_placed=float(cv[1]), s_ep=int(peaks[0]), t_ep=int(peaks[1]),
+                n_ep=int(peaks[2]), eta_ep=float(eta.value), attention=float(aj[0]), joint=float(aj[1]))
+
+
 def score_scale(C_cap: int) -> int:
     """SC: the integer that stands for 1.0 of the paper's normalised cost."""
     return (C_cap * C_cap) << 8

@@ -892,3 +892,76 @@ int32_t orc_anneal(int32_t N, int32_t L, int32_t P, int32_t D, int32_t G, int32_
     free(pop); free(nxt); free(best); free(tau); free(cq); free(Eterm); free(anc); free(bstep); free(dig);
     return status;
 }
+
+/* ------------------------------------------------------------------------------------ */
+/* Load-balance diagnostics of the evaluation section (Eq. global-ep-cv, the EP peak     */
+/* sum and tail peak, Eq. ep-efficiency) for one layout.                                 */
+/*   cv[0]: CV_global under the identity placement (expert e on rank e / H),            */
+/*   cv[1]: CV_global under the given placement pi.                                      */
+/*   peaks[0] = S_EP = sum_{r,l} max_{g,p} W,  peaks[1] = T_EP = max W,                  */
+/*   peaks[2] = sum_{r,l} max_g sum_p W  (eta_EP = peaks[2] / (P * peaks[0])).           */
+/*   att_joint[0] = sum_{r,g} A_{r,g}, att_joint[1] = max_g sum_r J_{r,g} (real units).  */
+/* ------------------------------------------------------------------------------------ */
+static double cv_of_loads(int32_t L, int32_t P, const int64_t *G)
+{
+    double acc = 0.0;
+    for (int32_t l = 0; l < L; ++l) {
+        double mean = 0.0;
+        for (int32_t p = 0; p < P; ++p) mean += (double)G[(size_t)l * P + p];
+        mean /= (double)P;
+        double var = 0.0;
+        for (int32_t p = 0; p < P; ++p) {
+            double d = (double)G[(size_t)l * P + p] - mean;
+            var += d * d;
+        }
+        var /= (double)P;
+        acc += (mean > 0.0) ? sqrt(var) / mean : 0.0;
+    }
+    return acc / (double)L;
+}
+
+void orc_diagnostics(int32_t N, int32_t L, int32_t E, int32_t P, int32_t D, int32_t G, int32_t R, int32_t C,
+                     const int32_t *edp_of_dp, int32_t S, const double *alpha, const double *beta,
+                     const int32_t *t, const int32_t *q, const int64_t *Lagg, const int32_t *pi,
+                     const int32_t *cell_of, double cv[2], int64_t peaks[3], double att_joint[2], double *eta)
+{
+    int32_t H = E / P;
+    int64_t *Gid = (int64_t *)calloc((size_t)L * P, sizeof(int64_t));
+    int64_t *Gpi = (int64_t *)calloc((size_t)L * P, sizeof(int64_t));
+    for (int32_t l = 0; l < L; ++l)
+        for (int32_t e = 0; e < E; ++e) {
+            Gid[(size_t)l * P + e / H] += Lagg[(size_t)l * E + e];
+            Gpi[(size_t)l * P + pi[(size_t)l * E + e] / H] += Lagg[(size_t)l * E + e];
+        }
+    cv[0] = cv_of_loads(L, P, Gid);
+    cv[1] = cv_of_loads(L, P, Gpi);
+    free(Gid); free(Gpi);
+
+    orc_problem pb;
+    fill_problem(&pb, N, L, P, D, G, R, C, edp_of_dp, S, alpha, beta, t, q);
+    orc_state *st = state_new(&pb);
+    memcpy(st->cell_of, cell_of, sizeof(int32_t) * N);
+    evaluate(&pb, st);
+    int64_t s_ep = 0, t_ep = 0, n_ep = 0;
+    for (int32_t r = 0; r < R; ++r)
+        for (int32_t l = 0; l < L; ++l) {
+            int64_t peak = 0, best_sum = 0;
+            for (int32_t g = 0; g < G; ++g) {
+                const int32_t *w = st->W + (((size_t)r * G + g) * L + l) * P;
+                int64_t sum = 0;
+                for (int32_t p = 0; p < P; ++p) { sum += w[p]; if (w[p] > peak) peak = w[p]; }
+                if (sum > best_sum) best_sum = sum;
+            }
+            s_ep += peak;
+            n_ep += best_sum;
+            if (peak > t_ep) t_ep = peak;
+        }
+    peaks[0] = s_ep; peaks[1] = t_ep; peaks[2] = n_ep;
+    *eta = s_ep > 0 ? (double)n_ep / ((double)P * (double)s_ep) : 1.0;
+    const double SC = (double)(((int64_t)C * C) << ORC_FBITS);
+    int64_t asum = 0;
+    for (size_t x = 0; x < (size_t)R * G; ++x) asum += st->Afx[x];
+    att_joint[0] = (double)asum / SC;
+    att_joint[1] = (double)st->s[0] / SC;
+    state_free(st);
+}

@@ -530,3 +530,44 @@ def test_named_tiny_window_end_to_end():
     assert res["status"] == 0 and res["n_rows"] >= 13
     assert res["counters"][0] == 8 * 200
     assert res["counters"][1] <= res["counters"][0] and res["counters"][2] <= res["counters"][1]
+
+
+# ----------------------------------------------------------------------------------------
+# diagnostics (Section 5.2: Eq. global-ep-cv, EP peak sum, tail peak, Eq. ep-efficiency)
+# ----------------------------------------------------------------------------------------
+def test_diagnostics_on_the_fig2_instance():
+    """Window loads 12/4 -> mean 8, deviation 4, CV 0.5; after the permutation 8/8 -> CV 0.
+    Packing A (row peaks 8, 8): S_EP 16, T_EP 8, each row's mean rank load is 4 -> eta 0.5.
+    Packing B (row peaks 4, 4): S_EP 8, T_EP 4, eta 1."""
+    a, m = read_fig2()
+    Lagg = oracle.aggregate(a)
+    pi, _ = oracle.lpt(Lagg, 2)
+    q = oracle.project(a, pi, 2)
+    t = np.full(4, 4, np.int32)
+    dA = oracle.diagnostics(t, q, Lagg, pi, np.array(m["packing_A_rows"], np.int32), R=2, C_cap=8, D=1)
+    dB = oracle.diagnostics(t, q, Lagg, pi, np.array(m["packing_B_rows"], np.int32), R=2, C_cap=8, D=1)
+    assert dA["cv_identity"] == 0.5 and dA["cv_placed"] == 0.0
+    assert (dA["s_ep"], dA["t_ep"], dA["eta_ep"]) == (16, 8, 0.5)
+    assert (dB["s_ep"], dB["t_ep"], dB["eta_ep"]) == (8, 4, 1.0)
+    assert dA["attention"] == 5.0 and dA["joint"] == 7.0 and dB["joint"] == 6.0
+
+
+def test_diagnostics_against_numpy_and_placement_effect():
+    w = hetero_window(N=80, L=4, E=16, k=2, C=4096, D=4, P=4, seed=31)
+    s = w.spec
+    Lagg = oracle.aggregate(w.demand)
+    pi, G, q = placed(w)
+    R, _, seed = oracle.pack_ffd(w.lengths, s.token_cap, s.dp_width, min_rows=3)
+    edp = [0, 0, 1, 1]
+    d = oracle.diagnostics(w.lengths, q, Lagg, pi, seed, R, s.token_cap, s.dp_width, edp)
+    ev = oracle.eval_layouts(w.lengths, q, seed, R, s.token_cap, s.dp_width, edp)
+    W = ev["W"][0].astype(np.int64)                      # [R][G][L][P]
+    assert d["s_ep"] == W.max(axis=(1, 3)).sum() and d["t_ep"] == W.max()
+    assert d["n_ep"] == W.sum(axis=3).max(axis=1).sum()
+    assert abs(d["eta_ep"] - d["n_ep"] / (s.ep_width * d["s_ep"])) < 1e-15 and 0 < d["eta_ep"] <= 1
+    Gf = G.astype(np.float64)
+    want = np.mean(Gf.std(axis=1) / Gf.mean(axis=1))
+    assert abs(d["cv_placed"] - want) < 1e-12
+    assert d["cv_placed"] < d["cv_identity"]             # LPT lowers the aggregate skew
+    SC = oracle.score_scale(s.token_cap)
+    assert abs(d["attention"] - ev["Afx"][0].sum() / SC) < 1e-12 and abs(d["joint"] - ev["score"][0][0] / SC) < 1e-12
