@@ -158,6 +158,21 @@ int rp_anneal(rp_ctx *ctx, const rp_anneal_params *params, rp_anneal_stats *stat
  *   cell_of_sample [N] int32 out, nullable; score_fx [3], score_f64 [3] out, nullable. */
 int rp_best(rp_ctx *ctx, int32_t *cell_of_sample, int64_t *score_fx, double *score_f64);
 
+/* Load-balance diagnostics of the paper's evaluation section for one layout (Eq. global-ep-cv,
+ * the EP peak sum and tail peak, Eq. ep-efficiency, and the attention / joint proxies of its
+ * mechanism table).  W is the rank-load tensor of the layout under the committed placement.
+ *   cv_identity / cv_placed: mean over layers of std_p(G[l][p]) / mean_p(G[l][p]) of the
+ *     aggregate rank loads, with expert e on rank e/(E/P), and under the LPT placement;
+ *   s_ep = sum_{r,l} max_{g,p} W;  t_ep = max W;  n_ep = sum_{r,l} max_g sum_p W;
+ *   eta_ep = n_ep / (P * s_ep);  attention = sum_{r,g} A_{r,g};  joint = max_g sum_r J_{r,g}.
+ *   layout [N] int32 (host or device), NULL = the incumbent.  out: HOST struct. */
+typedef struct {
+    double cv_identity, cv_placed;
+    int64_t s_ep, t_ep, n_ep;
+    double eta_ep, attention, joint;
+} rp_diag;
+int rp_diagnostics(rp_ctx *ctx, const int32_t *layout, rp_diag *out);
+
 /* Frees the context.  Its device memory goes back to a per-device cache inside the library
  * (so that the next window does not pay for allocation); rp_release_cached_memory() returns
  * that cache to the driver. */

@@ -22,7 +22,7 @@ STATUS_NAMES = {0: "RP_OK", -1: "RP_ERR_ARG", -2: "RP_ERR_SHAPE", -3: "RP_ERR_CO
                 -8: "RP_ERR_TIMEOUT", -9: "RP_ERR_INVALID_PLAN"}
 RP_OK = 0
 
-EXPORTS = ("rp_window_load", "rp_place_experts", "rp_pack_rows", "rp_eval_population", "rp_eval_layouts_noalloc", "rp_anneal",
+EXPORTS = ("rp_window_load", "rp_place_experts", "rp_pack_rows", "rp_eval_population", "rp_eval_layouts_noalloc", "rp_diagnostics", "rp_anneal",
            "rp_best", "rp_destroy", "rp_release_cached_memory", "rp_strerror", "rp_last_cuda_error", "rp_debug_dump",
            "rp_debug_nl2", "rp_debug_exp2neg", "rp_debug_philox", "rp_debug_launch_count")
 
@@ -54,6 +54,11 @@ class rp_anneal_stats(C.Structure):
                 ("move_bytes", C.c_int64), ("gather_bytes", C.c_int64), ("kernel_launches", C.c_int64)]
 
 
+class rp_diag(C.Structure):
+    _fields_ = [("cv_identity", C.c_double), ("cv_placed", C.c_double), ("s_ep", C.c_int64), ("t_ep", C.c_int64),
+                ("n_ep", C.c_int64), ("eta_ep", C.c_double), ("attention", C.c_double), ("joint", C.c_double)]
+
+
 def library_path() -> str:
     return _build.LIB
 
@@ -76,6 +81,7 @@ def lib():
         L.rp_pack_rows.argtypes = [C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         L.rp_eval_population.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
         L.rp_eval_layouts_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
+        L.rp_diagnostics.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(rp_diag)]
         L.rp_anneal.argtypes = [C.c_void_p, C.POINTER(rp_anneal_params), C.POINTER(rp_anneal_stats)]
         L.rp_best.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.rp_debug_dump.argtypes = [C.c_void_p, C.c_int, C.c_int32, C.c_void_p, C.c_int64]
@@ -194,6 +200,13 @@ def rp_eval_layouts_noalloc(ctx: Context, layouts, score_fx, score_f64):
     _check(lib().rp_eval_layouts_noalloc(ctx.handle, _ptr(layouts), n, _ptr(score_fx), _ptr(score_f64)),
            "rp_eval_layouts_noalloc")
     return score_fx, score_f64
+
+
+def rp_diagnostics(ctx: Context, layout=None) -> dict:
+    """Load-balance diagnostics of a layout (None = the incumbent) as a dict."""
+    d = rp_diag()
+    _check(lib().rp_diagnostics(ctx.handle, _ptr(layout), C.byref(d)), "rp_diagnostics")
+    return {name: getattr(d, name) for name, _ in rp_diag._fields_}
 
 
 def rp_anneal(ctx: Context, *, n_levels: int, steps_per_level: int, t0: float, t_ratio: float,

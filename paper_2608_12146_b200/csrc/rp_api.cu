@@ -39,7 +39,7 @@ extern "C" const char *rp_strerror(int s)
 static cudaMemPool_t g_pools[RP_MAX_DEVICES];
 static bool g_pool_ready[RP_MAX_DEVICES];
 
-static int get_pool(int device, cudaMemPool_t *out)
+int rp_get_pool(int device, cudaMemPool_t *out)
 {
     if (device < 0 || device >= RP_MAX_DEVICES) return RP_ERR_ARG;
     if (!g_pool_ready[device]) {
@@ -71,7 +71,7 @@ static int dev_alloc(rp_ctx *c, T **p, size_t n)
     *p = nullptr;
     if (n == 0) n = 1;
     cudaMemPool_t pool;
-    RP_TRY(get_pool(c->device, &pool));
+    RP_TRY(rp_get_pool(c->device, &pool));
     RP_CUDA(cudaMallocFromPoolAsync((void **)p, n * sizeof(T), pool, c->stream));
     return RP_OK;
 }

@@ -204,6 +204,161 @@ int rp_launch_build_static(rp_ctx *c)
 }
 
 // ---------------------------------------------------------------------------------------------
+// Load-balance diagnostics (evaluation section of the paper): coefficient of variation of the
+// aggregate rank loads, EP peak sum, tail peak, EP balance efficiency, attention and joint proxies.
+// ---------------------------------------------------------------------------------------------
+struct RpDiagDev { double cv_identity, cv_placed; i64 s_ep, t_ep, n_ep; i64 afx_sum, s0; };
+
+// One thread per layer, each with plain sequential IEEE sums (no fused multiply-add), then
+// thread 0 averages the layers in order.
+__global__ void k_diag_cv(const i64 *__restrict__ Lagg, const i64 *__restrict__ rank_load, RpDims dm,
+                          RpDiagDev *__restrict__ out)
+{
+    extern __shared__ double cvs[];          // [2][L]
+    const int l = threadIdx.x;
+    if (l < dm.L) {
+        for (int which = 0; which < 2; ++which) {
+            double mean = 0.0;
+            for (int p = 0; p < dm.P; ++p) {
+                i64 g = 0;
+                if (which) g = rank_load[(size_t)l * dm.P + p];
+                else for (int n = 0; n < dm.H; ++n) g += Lagg[(size_t)l * dm.E + p * dm.H + n];
+                mean = __dadd_rn(mean, (double)g);
+            }
+            mean = __ddiv_rn(mean, (double)dm.P);
+            double var = 0.0;
+            for (int p = 0; p < dm.P; ++p) {
+                i64 g = 0;
+                if (which) g = rank_load[(size_t)l * dm.P + p];
+                else for (int n = 0; n < dm.H; ++n) g += Lagg[(size_t)l * dm.E + p * dm.H + n];
+                const double d = __dsub_rn((double)g, mean);
+                var = __dadd_rn(var, __dmul_rn(d, d));
+            }
+            var = __ddiv_rn(var, (double)dm.P);
+            cvs[which * dm.L + l] = (mean > 0.0) ? __ddiv_rn(__dsqrt_rn(var), mean) : 0.0;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double a = 0.0, b = 0.0;
+        for (int x = 0; x < dm.L; ++x) { a = __dadd_rn(a, cvs[x]); b = __dadd_rn(b, cvs[dm.L + x]); }
+        out->cv_identity = __ddiv_rn(a, (double)dm.L);
+        out->cv_placed = __ddiv_rn(b, (double)dm.L);
+    }
+}
+
+// One warp per (row, layer): lanes over ranks, loop over shards; integer results by atomics.
+__global__ void k_diag_peaks(const int *__restrict__ W, const char *__restrict__ blob, RpBlob bl, RpDims dm,
+                             RpDiagDev *__restrict__ out)
+{
+    const int lane = threadIdx.x & 31;
+    const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nw = (gridDim.x * blockDim.x) >> 5;
+    i64 s_ep = 0, n_ep = 0, t_ep = 0;
+    for (int rl = wid; rl < dm.R * dm.L; rl += nw) {
+        const int r = rl / dm.L, l = rl % dm.L;
+        i64 peak = 0, best_sum = 0;
+        for (int g = 0; g < dm.G; ++g) {
+            const int *w = W + (((size_t)r * dm.G + g) * dm.L + l) * dm.P;
+            i64 sum = 0, mx = 0;
+            for (int p = lane; p < dm.P; p += 32) { const i64 v = w[p]; sum += v; mx = v > mx ? v : mx; }
+            for (int o = 16; o; o >>= 1) {
+                sum += __shfl_xor_sync(0xffffffffu, sum, o);
+                const i64 x = __shfl_xor_sync(0xffffffffu, mx, o);
+                mx = x > mx ? x : mx;
+            }
+            peak = mx > peak ? mx : peak;
+            best_sum = sum > best_sum ? sum : best_sum;
+        }
+        s_ep += peak; n_ep += best_sum; t_ep = peak > t_ep ? peak : t_ep;
+    }
+    if (lane == 0) {
+        if (s_ep) atomicAdd((u64 *)&out->s_ep, (u64)s_ep);
+        if (n_ep) atomicAdd((u64 *)&out->n_ep, (u64)n_ep);
+        atomicMax((i64 *)&out->t_ep, t_ep);
+    }
+    if (blockIdx.x == 0 && threadIdx.x < 32) {      // attention total and joint from the layout's blob
+        const i64 *Afx = (const i64 *)(blob + bl.off_Afx);
+        i64 a = 0;
+        for (int x = lane; x < dm.RG; x += 32) a += Afx[x];
+        for (int o = 16; o; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+        if (lane == 0) { out->afx_sum = a; out->s0 = ((const i64 *)(blob + bl.off_S))[0]; }
+    }
+}
+
+extern "C" int rp_diagnostics(rp_ctx *c, const int32_t *layout, rp_diag *out)
+{
+    if (!c || !out) return RP_ERR_ARG;
+    if (c->stage < 3) return RP_ERR_STATE;
+    const RpDims &dm = c->dm;
+    if (dm.L > 1024) return RP_ERR_RANGE;
+    cudaMemPool_t pool;
+    RP_TRY(rp_get_pool(c->device, &pool));
+    // scratch: cells, W, one blob, the result record, and the row-shard sums / ticket of the scoring kernel
+    const size_t wn = (size_t)dm.RG * dm.LP;
+    size_t off_cells = 0, off_lay = off_cells + (((size_t)dm.N * 2 + 255) & ~(size_t)255);
+    size_t off_W = off_lay + (((size_t)dm.N * 4 + 255) & ~(size_t)255);
+    size_t off_blob = off_W + ((wn * 4 + 255) & ~(size_t)255);
+    size_t off_res = off_blob + (((size_t)c->bl.bytes + 255) & ~(size_t)255);
+    size_t off_es = off_res + 256, off_tk = off_es + (((size_t)dm.RG * 8 + 255) & ~(size_t)255);
+    size_t total = off_tk + 256;
+    char *buf = nullptr;
+    RP_CUDA(cudaMallocFromPoolAsync((void **)&buf, total, pool, c->stream));
+    int st = RP_OK;
+    cudaError_t e = cudaSuccess;
+    do {
+        const int *dl = c->d_inc_layout;
+        if (layout) {
+            e = cudaMemcpyAsync(buf + off_lay, layout, sizeof(int) * dm.N, cudaMemcpyDefault, c->stream);
+            if (e != cudaSuccess) break;
+            dl = (const int *)(buf + off_lay);
+        }
+        e = cudaMemsetAsync(buf + off_res, 0, 256 + (off_tk - off_es) + 256, c->stream);
+        if (e != cudaSuccess) break;
+        e = cudaMemsetAsync(c->d_status + RP_SW_BAD_LAYOUT, 0, sizeof(int), c->stream);
+        if (e != cudaSuccess) break;
+        k_layouts_to_cells<<<(dm.N + 255) / 256, 256, 0, c->stream>>>(dl, dm.N, dm.K, (unsigned short *)(buf + off_cells),
+                                                                     c->d_status);
+        ++g_rp_launches;
+        const size_t smem = eval_smem_bytes(dm);
+        if (smem > 220 * 1024) { st = RP_ERR_RANGE; break; }
+        if (smem > 32 * 1024) {
+            e = cudaFuncSetAttribute(k_eval, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) break;
+        }
+        int splits = 2 * 148;
+        const int max_splits = (dm.RG + EVAL_THREADS / 32 - 1) / (EVAL_THREADS / 32);
+        if (splits > max_splits) splits = max_splits;
+        k_eval<<<dim3(1, splits), EVAL_THREADS, smem, c->stream>>>((const unsigned short *)(buf + off_cells), c->d_t, c->d_q,
+                                                                  c->d_edp, c->d_dp_list, c->d_dp_off, dm, c->bl,
+                                                                  (int *)(buf + off_W), buf + off_blob, nullptr, nullptr,
+                                                                  (i64 *)(buf + off_es), (int *)(buf + off_tk));
+        ++g_rp_launches;
+        RpDiagDev *res = (RpDiagDev *)(buf + off_res);
+        k_diag_cv<<<1, ((dm.L + 31) / 32) * 32, sizeof(double) * 2 * dm.L, c->stream>>>(c->d_Lagg, c->d_rank_load, dm, res);
+        ++g_rp_launches;
+        k_diag_peaks<<<148, 256, 0, c->stream>>>((const int *)(buf + off_W), buf + off_blob, c->bl, dm, res);
+        ++g_rp_launches;
+        e = cudaGetLastError();
+        if (e != cudaSuccess) break;
+        RpDiagDev h;
+        int bad = 0;
+        e = cudaMemcpyAsync(&h, res, sizeof h, cudaMemcpyDeviceToHost, c->stream);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(&bad, c->d_status + RP_SW_BAD_LAYOUT, sizeof(int), cudaMemcpyDeviceToHost, c->stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+        if (e != cudaSuccess) break;
+        if (bad) { st = RP_ERR_ARG; break; }
+        out->cv_identity = h.cv_identity; out->cv_placed = h.cv_placed;
+        out->s_ep = h.s_ep; out->t_ep = h.t_ep; out->n_ep = h.n_ep;
+        out->eta_ep = h.s_ep > 0 ? (double)h.n_ep / ((double)dm.P * (double)h.s_ep) : 1.0;
+        out->attention = (double)h.afx_sum / (double)dm.SC;
+        out->joint = (double)h.s0 / (double)dm.SC;
+    } while (0);
+    cudaFreeAsync(buf, c->stream);
+    if (e != cudaSuccess) { g_rp_last_cuda_error = (int)e; return RP_ERR_CUDA; }
+    return st;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Scoring layouts without allocating: the kernels above, with their scratch (16-bit cell ids,
 // row-shard sums, arrival counters) taken from a fixed array that is part of the library image
 // instead of from the context's allocator.

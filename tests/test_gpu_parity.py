@@ -106,6 +106,15 @@ def check_anneal(w, ctx, ref, edp, pop, levels, steps, threads=8, t_ratio=None, 
     # scoring the current population from scratch agrees with the last terminal scores
     fx_pop, _ = rp.rp_eval_population(ctx)
     assert (fx_pop == want["term"][-1]).all()
+    # load-balance diagnostics of the incumbent and of the seed
+    pi = oracle.lpt(ref["Lagg"], s.ep_width)[0]
+    for lay, arg in ((want["best_layout"], None), (ref["seed"], ref["seed"])):
+        d_want = oracle.diagnostics(w.lengths, ref["q"], ref["Lagg"], pi, lay, R, s.token_cap, D, edp, s.alpha, s.beta)
+        d_got = rp.rp_diagnostics(ctx, arg)
+        for key in ("s_ep", "t_ep", "n_ep"):
+            assert d_got[key] == d_want[key], key
+        for key in ("cv_identity", "cv_placed", "eta_ep", "attention", "joint"):
+            assert abs(d_got[key] - d_want[key]) <= F64_RTOL * abs(d_want[key]), key
     return want, stats
 
 
