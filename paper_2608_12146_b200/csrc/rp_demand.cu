@@ -106,14 +106,15 @@ k_lpt(const i64 *__restrict__ Lagg, RpDims dm, int *__restrict__ pi, int *__rest
     __syncthreads();
     if (threadIdx.x < 32) {
         const int lane = threadIdx.x;
+        int width = 1;                               // lanes that hold ranks, rounded up to a power of two
+        while (width < dm.P && width < 32) width <<= 1;
         for (int x = 0; x < dm.E; ++x) {
             const int e = order[x];
             i64 bestG = 0x7fffffffffffffffll;
             int bestP = 0x7fffffff;
             for (int p = lane; p < dm.P; p += 32)
                 if (cnt[p] < dm.H && (G[p] < bestG || (G[p] == bestG && p < bestP))) { bestG = G[p]; bestP = p; }
-#pragma unroll
-            for (int o = 16; o; o >>= 1) {
+            for (int o = width >> 1; o; o >>= 1) {   // lane 0 ends up with the minimum over lanes 0..width-1
                 i64 og = __shfl_xor_sync(0xffffffffu, bestG, o);
                 int op = __shfl_xor_sync(0xffffffffu, bestP, o);
                 if (og < bestG || (og == bestG && op < bestP)) { bestG = og; bestP = op; }

@@ -49,7 +49,6 @@ k_pack_ffd(RpDims dm, const int *__restrict__ t, int min_rows, u64 *__restrict__
     i64 Rlb = (total_s + cap_row - 1) / cap_row;
     if (Rlb < 1) Rlb = 1;
     if (Rlb < min_rows) Rlb = min_rows;
-    const int t_min = dm.C - (int)(keys[dm.N - 1] >> 32);          // the shortest sample
     int Rstar = 0;
     for (i64 R = Rlb; R * dm.D <= dm.N && !Rstar; ++R) {
         const int K = (int)(R * dm.D);
@@ -62,23 +61,29 @@ k_pack_ffd(RpDims dm, const int *__restrict__ t, int min_rows, u64 *__restrict__
         }
         __syncthreads();
         if (tid < 32) {
-            // Cells before `lo` cannot take even the shortest sample any more; samples arrive
-            // in decreasing length, so skipping them leaves first-fit unchanged.
-            int lo = 0;
+            // First fit = the lowest cell whose remaining capacity takes the sample.  Each lane
+            // owns a block of B consecutive cells and keeps the largest remaining capacity of its
+            // block in a register: one ballot finds the lowest lane that can take the sample, and
+            // only that lane scans its block.
+            const int B = (K + 31) / 32;
+            const int b0 = tid * B, b1 = min(K, b0 + B);
+            int blockmax = -1;
+            for (int b = b0; b < b1; ++b) blockmax = max(blockmax, dm.C - fill[b]);
             for (int x = K; x < dm.N; ++x) {
                 const u64 key = keys[x];
                 const int ts = dm.C - (int)(key >> 32);
-                while (lo < K && fill[lo] + t_min > dm.C) ++lo;
-                int found = -1;
-                for (int b0 = lo; b0 < K && found < 0; b0 += 32) {
-                    const int b = b0 + tid;
-                    const bool ok = (b < K) && (fill[b] + ts <= dm.C);
-                    const unsigned m = __ballot_sync(0xffffffffu, ok);
-                    if (m) found = b0 + __ffs(m) - 1;
+                const unsigned m = __ballot_sync(0xffffffffu, blockmax >= ts);
+                if (!m) { if (tid == 0) fail_s = 1; break; }
+                if (tid == __ffs(m) - 1) {
+                    int found = -1, nm = -1;
+                    for (int b = b0; b < b1; ++b) {
+                        int rem = dm.C - fill[b];
+                        if (found < 0 && rem >= ts) { found = b; rem -= ts; fill[b] += ts; }
+                        nm = max(nm, rem);
+                    }
+                    blockmax = nm;
+                    cell_of[(u32)key] = found;
                 }
-                if (found < 0) { if (tid == 0) fail_s = 1; break; }
-                if (tid == 0) { fill[found] += ts; cell_of[(u32)key] = found; }
-                __syncwarp();
             }
         }
         __syncthreads();
