@@ -34,6 +34,9 @@ from paper_2608_12146_b200.windows import SPECS, make_window
 METRIC = "annealing replica-moves evaluated/sec"
 UNIT = "moves/s"
 FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes (read + write) per launch of the chain kernel from the ncu captures summarised under
+# profiles/ (k_anneal_wpc_medium.txt); None where no full-size capture exists.
+NCU_DRAM_BYTES_PER_LAUNCH = {"medium": 6.5e6}
 
 
 def hbm_peak():
@@ -122,7 +125,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.idx)],
+                                          "-lms", "20", "-i", str(self.idx)],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
@@ -183,6 +186,120 @@ def plan_once(rp, torch, w, t_in, a_in, outs, stream, want_stats=True):
     return stats
 
 
+def measure(rp, torch, args, name, steps, dist, dev, local, with_clocks, with_cpu):
+    """Time `steps` plans of the named workload on this rank; returns the pieces of the JSON line."""
+    spec = SPECS[name]
+    overrides = {}
+    if args.pop:
+        overrides["pop_size"] = args.pop          # profiling aid: a smaller population of the same window
+    if args.levels:
+        overrides["n_levels"] = args.levels
+        overrides["sweeps"] = spec.steps_per_level * args.levels
+    w = make_window(spec, **overrides)
+    s = spec = w.spec
+    moves_per_step = s.pop_size * s.n_levels * s.steps_per_level
+    stream = torch.cuda.current_stream()
+    t_dev = torch.from_numpy(w.lengths).to(dev)
+    a_dev = torch.from_numpy(w.demand).to(dev)
+    t_pin = torch.from_numpy(w.lengths).pin_memory()
+    a_pin = torch.from_numpy(w.demand).pin_memory()
+
+    def outputs(**kw):
+        return dict(pi=torch.empty((s.n_layers, s.n_experts), dtype=torch.int32, **kw),
+                    rank_load=torch.empty((s.n_layers, s.ep_width), dtype=torch.int64, **kw),
+                    layout=torch.empty(s.n_samples, dtype=torch.int32, **kw),
+                    score_fx=torch.empty(3, dtype=torch.int64, **kw),
+                    score_f64=torch.empty(3, dtype=torch.float64, **kw))
+
+    outs_dev = outputs(device=dev)
+    outs_host = {k: v.pin_memory() for k, v in outputs().items()}
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed_loop(t_in, a_in, outs, n):
+        """n plans, each timed with CUDA events on the launching stream; L2 flushed in between."""
+        acc = dict(ms=0.0, chain_ms=0.0, move_bytes=0, gather_bytes=0, feasible=0, accepted=0, chain_launches=0)
+        barrier()
+        wall0 = time.perf_counter()
+        for _ in range(n):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            st = plan_once(rp, torch, w, t_in, a_in, outs, stream)
+            e1.record(stream)
+            e1.synchronize()
+            acc["ms"] += e0.elapsed_time(e1)
+            acc["chain_ms"] += st.ms_chains
+            acc["move_bytes"] += st.move_bytes
+            acc["gather_bytes"] += st.gather_bytes
+            acc["feasible"] += st.feasible
+            acc["accepted"] += st.accepted
+            acc["chain_launches"] += s.n_levels
+        barrier()
+        acc["wall"] = time.perf_counter() - wall0
+        return acc
+
+    for _ in range(args.warmup):
+        plan_once(rp, torch, w, t_dev, a_dev, outs_dev, stream)
+        plan_once(rp, torch, w, t_pin, a_pin, outs_host, stream)
+    clocks = None
+    if with_clocks:
+        vis = [x for x in os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",") if x]
+        sampler = ClockSampler(vis[local] if local < len(vis) else local)
+        sampler.start()
+    launches0 = rp.rp_debug_launch_count()
+    res = timed_loop(t_dev, a_dev, outs_dev, steps)
+    launches = rp.rp_debug_launch_count() - launches0
+    if with_clocks:
+        clocks = sampler.stop()
+    e2e = timed_loop(t_pin, a_pin, outs_host, steps)
+
+    ms, total_moves = reduce_job(res["ms"], moves_per_step * steps, dist, dev)
+    ms_e2e, _ = reduce_job(e2e["ms"], moves_per_step * steps, dist, dev)
+    world = 1 if dist is None else dist.get_world_size()
+    peak, peak_kind = hbm_peak()
+    per_launch_s = res["chain_ms"] * 1e-3 / res["chain_launches"]
+    alg = (res["move_bytes"] + res["gather_bytes"]) / res["chain_launches"]
+    achieved = alg / per_launch_s / 1e9
+    chain_kernel = "k_anneal_wpc" if s.n_layers * s.ep_width <= 512 else "k_anneal_level"
+    roofline = {"bound": "hbm", "kernel": chain_kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_source": peak_kind, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(s.name),
+                "algorithmic_bytes_per_launch": alg,
+                "move_bytes_per_launch": res["move_bytes"] / res["chain_launches"],
+                "gather_bytes_per_launch": res["gather_bytes"] / res["chain_launches"],
+                "launch_ms": per_launch_s * 1e3, "share_of_step": res["chain_ms"] / res["ms"]}
+    cpu = None
+    if with_cpu:
+        import oracle
+        oracle.build()
+        threads = os.cpu_count() or 1
+        budget = {"tiny": 1e5, "medium": 2e7, "large": 2e7, "wide": 6e6, "heavy": 2e7}[s.name]
+        oracle_sample(w, threads, min(budget, 1e6))           # warm the page cache and the thread pool
+        m, d, reps = 0, 0.0, 0
+        while d < 2.0 and reps < 64:                          # a few seconds of wall time on all cores
+            mi, di, sample = oracle_sample(w, threads, budget)
+            m, d, reps = m + mi, d + di, reps + 1
+        cpu = {"value": m / d, "unit": UNIT, "cores": threads, "kind": "oracle",
+               "sample": f"{reps} x ({sample})", "seconds": d}
+    h2d = int(w.lengths.nbytes + w.demand.nbytes)
+    d2h = int(sum(v.numel() * v.element_size() for v in outs_host.values()))
+    n_all = moves_per_step * steps
+    return {"value": total_moves / (ms * 1e-3), "ms_per_step": ms / steps,
+            "config": workload_config(spec, {"parallelism": "replicas only" if world > 1 else "1 gpu"}),
+            "plans_per_s": steps * world / (ms * 1e-3),
+            "anneal_only_moves_per_s": n_all / (res["chain_ms"] * 1e-3),
+            "feasible_fraction": res["feasible"] / n_all, "accepted_fraction": res["accepted"] / n_all,
+            "stage_ms_per_step": {"anneal_levels": res["chain_ms"] / steps, "other": (res["ms"] - res["chain_ms"]) / steps},
+            "roofline": roofline, "cpu_baseline": cpu,
+            "e2e": {"value": total_moves / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / steps},
+            "gpu_launches": int(launches), "clocks": clocks, "wall_s": res["wall"]}
+
+
 def run_cuda(args):
     import torch
     import paper_2608_12146_b200.binding as rp
@@ -198,144 +315,29 @@ def run_cuda(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     rp.lib()
-
-    spec = SPECS[args.workload]
-    overrides = {}
-    if args.pop:
-        overrides["pop_size"] = args.pop          # profiling aid: a smaller population of the same window
-    if args.levels:
-        overrides["n_levels"] = args.levels
-        overrides["sweeps"] = spec.steps_per_level * args.levels
-    w = make_window(spec, **overrides)
-    spec = w.spec
-    s = spec
-    moves_per_step = s.pop_size * s.n_levels * s.steps_per_level
-    stream = torch.cuda.current_stream()
     dev = torch.device("cuda", local)
-    t_dev = torch.from_numpy(w.lengths).to(dev)
-    a_dev = torch.from_numpy(w.demand).to(dev)
-    t_pin = torch.from_numpy(w.lengths).pin_memory()
-    a_pin = torch.from_numpy(w.demand).pin_memory()
-    outs_dev = dict(pi=torch.empty((s.n_layers, s.n_experts), dtype=torch.int32, device=dev),
-                    rank_load=torch.empty((s.n_layers, s.ep_width), dtype=torch.int64, device=dev),
-                    layout=torch.empty(s.n_samples, dtype=torch.int32, device=dev),
-                    score_fx=torch.empty(3, dtype=torch.int64, device=dev),
-                    score_f64=torch.empty(3, dtype=torch.float64, device=dev))
-    outs_host = dict(pi=torch.empty((s.n_layers, s.n_experts), dtype=torch.int32).pin_memory(),
-                     rank_load=torch.empty((s.n_layers, s.ep_width), dtype=torch.int64).pin_memory(),
-                     layout=torch.empty(s.n_samples, dtype=torch.int32).pin_memory(),
-                     score_fx=torch.empty(3, dtype=torch.int64).pin_memory(),
-                     score_f64=torch.empty(3, dtype=torch.float64).pin_memory())
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
 
-    def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def timed_loop(t_in, a_in, outs, steps):
-        """K steps, each timed with CUDA events on the launching stream; L2 flushed in between."""
-        total_ms, chain_ms, barrier_ms = 0.0, 0.0, 0.0
-        move_bytes = gather_bytes = feasible = accepted = chain_launches = 0
-        barrier()
-        wall0 = time.perf_counter()
-        for _ in range(steps):
-            flush.fill_(1)
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(stream)
-            st = plan_once(rp, torch, w, t_in, a_in, outs, stream)
-            e1.record(stream)
-            e1.synchronize()
-            total_ms += e0.elapsed_time(e1)
-            chain_ms += st.ms_chains
-            barrier_ms += st.ms_barrier
-            move_bytes += st.move_bytes
-            gather_bytes += st.gather_bytes
-            feasible += st.feasible
-            accepted += st.accepted
-            chain_launches += s.n_levels
-        barrier()
-        wall = time.perf_counter() - wall0
-        return dict(ms=total_ms, wall=wall, chain_ms=chain_ms, barrier_ms=barrier_ms, move_bytes=move_bytes,
-                    gather_bytes=gather_bytes, feasible=feasible, accepted=accepted, chain_launches=chain_launches)
-
-    for _ in range(args.warmup):
-        plan_once(rp, torch, w, t_dev, a_dev, outs_dev, stream)
-        plan_once(rp, torch, w, t_pin, a_pin, outs_host, stream)
-    vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
-    vis_ids = [x for x in vis.split(",") if x]
-    sampler = ClockSampler(vis_ids[local] if local < len(vis_ids) else local)
-    sampler.start()
-    launches0 = rp.rp_debug_launch_count()
-    res = timed_loop(t_dev, a_dev, outs_dev, args.steps)
-    launches = rp.rp_debug_launch_count() - launches0
-    clocks = sampler.stop()
-    e2e = timed_loop(t_pin, a_pin, outs_host, args.steps)
-
-    ms, total_moves = reduce_job(res["ms"], moves_per_step * args.steps, dist, dev)
-    ms_e2e, _ = reduce_job(e2e["ms"], moves_per_step * args.steps, dist, dev)
-    value = total_moves / (ms * 1e-3)
-    e2e_value = total_moves / (ms_e2e * 1e-3)
-
-    peak, peak_kind = hbm_peak()
-    per_launch_s = res["chain_ms"] * 1e-3 / res["chain_launches"]
-    alg_bytes_per_launch = (res["move_bytes"] + res["gather_bytes"]) / res["chain_launches"]
-    achieved = alg_bytes_per_launch / per_launch_s / 1e9
-    chain_kernel = "k_anneal_wpc" if s.n_layers * s.ep_width <= 512 else "k_anneal_level"
-    roofline = {"bound": "hbm", "kernel": chain_kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_source": peak_kind, "traffic": None,
-                "algorithmic_bytes_per_launch": alg_bytes_per_launch,
-                "move_bytes_per_launch": res["move_bytes"] / res["chain_launches"],
-                "gather_bytes_per_launch": res["gather_bytes"] / res["chain_launches"],
-                "launch_ms": per_launch_s * 1e3,
-                "share_of_step": res["chain_ms"] / res["ms"]}
-    traffic_file = os.path.join(ROOT, "profiles", f"traffic_{spec.name}.json")
-    if os.path.exists(traffic_file):
-        try:
-            roofline["traffic"] = json.load(open(traffic_file))["dram_bytes_per_launch"]
-        except Exception:
-            pass
-
-    if rank != 0:
-        if dist is not None:
-            dist.destroy_process_group()
-        return 0
-
-    # CPU baseline: the oracle as it stands on this box's cores (rank 0, N=1 only)
-    cpu = None
-    if world == 1 and not args.no_cpu_baseline:
-        import oracle
-        oracle.build()
-        threads = os.cpu_count() or 1
-        budget = {"tiny": 1e5, "medium": 2e7, "large": 2e7, "wide": 6e6, "heavy": 2e7}[spec.name]
-        oracle_sample(w, threads, min(budget, 1e6))           # warm the page cache and the thread pool
-        m, d, reps = 0, 0.0, 0
-        while d < 2.0 and reps < 64:                          # a few seconds of wall time on all cores
-            mi, di, sample = oracle_sample(w, threads, budget)
-            m, d, reps = m + mi, d + di, reps + 1
-        cpu = {"value": m / d, "unit": UNIT, "cores": threads, "kind": "oracle",
-               "sample": f"{reps} x ({sample})", "seconds": d}
-
-    h2d = int(w.lengths.nbytes + w.demand.nbytes)
-    d2h = int(sum(v.numel() * v.element_size() for v in outs_host.values()))
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "int64", "data": "synthetic",
-            "config": workload_config(spec, {"parallelism": "replicas only" if world > 1 else "1 gpu"}),
-            "plans_per_s": args.steps * world / (ms * 1e-3),
-            "anneal_only_moves_per_s": moves_per_step * args.steps / ((res["chain_ms"] + res["barrier_ms"]) * 1e-3),
-            "feasible_fraction": res["feasible"] / (moves_per_step * args.steps),
-            "accepted_fraction": res["accepted"] / (moves_per_step * args.steps),
-            "stage_ms_per_step": {"chains": res["chain_ms"] / args.steps, "level_barrier": res["barrier_ms"] / args.steps,
-                                  "other": (res["ms"] - res["chain_ms"] - res["barrier_ms"]) / args.steps},
-            "roofline": roofline,
-            "cpu_baseline": cpu,
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "ms_per_step": ms_e2e / args.steps},
-            "gpu_launches": int(launches),
-            "clocks": clocks,
-            "wall_s": res["wall"]}
-    print(json.dumps(line))
+    main_res = measure(rp, torch, args, args.workload, args.steps, dist, dev, local, with_clocks=True,
+                       with_cpu=(world == 1 and rank == 0 and not args.no_cpu_baseline))
+    sweep = {}
+    if args.sweep and world == 1:
+        for name in SPECS:            # context beside the headline: the other windows, 3 plans each
+            if name == args.workload:
+                continue
+            r = measure(rp, torch, args, name, 3, None, dev, local, with_clocks=False, with_cpu=False)
+            sweep[name] = {"moves_per_s": r["value"], "plans_per_s": r["plans_per_s"], "ms_per_plan": r["ms_per_step"],
+                           "roofline_frac": r["roofline"]["frac"], "algorithmic_gbs": r["roofline"]["achieved"],
+                           "kernel": r["roofline"]["kernel"], "feasible_fraction": r["feasible_fraction"],
+                           "accepted_fraction": r["accepted_fraction"]}
+            rp.rp_release_cached_memory()
+    if rank == 0:
+        line = {"metric": METRIC, "value": main_res.pop("value"), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": main_res.pop("ms_per_step"), "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic"}
+        line.update(main_res)
+        if sweep:
+            line["other_workloads"] = sweep
+        print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
     return 0
@@ -349,6 +351,8 @@ def main():
     ap.add_argument("--workload", default="medium", choices=list(SPECS))
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", dest="sweep", action="store_false",
+                    help="skip the context sweep over the other four windows (3 plans each, N=1 only)")
     ap.add_argument("--pop", type=int, default=0, help="override the population size (profiling aid)")
     ap.add_argument("--levels", type=int, default=0, help="override the number of temperature levels (profiling aid)")
     args = ap.parse_args()
