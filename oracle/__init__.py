@@ -146,6 +146,17 @@ def pack_ffd(lengths, C_cap: int, D: int, min_rows: int = 0):
     return int(R), int(cert.value), cell
 
 
+def seed_trials(lengths, seed_layout, R: int, C_cap: int, D: int, pop_size: int, width: int, seed: int):
+    """Randomized fixed-row seeds, one trial per member: returns (layouts [P][N], ok [P])."""
+    t = _i32(lengths)
+    sl = _i32(seed_layout)
+    lay = np.zeros((pop_size, t.shape[0]), np.int32)
+    ok = np.zeros(pop_size, np.int32)
+    lib().orc_seed_trials(C.c_int32(t.shape[0]), C.c_int32(C_cap), C.c_int32(D), C.c_int32(R), C.c_int32(width),
+                          C.c_uint64(seed), _p(t), _p(sl), C.c_int32(pop_size), _p(lay), _p(ok))
+    return lay, ok
+
+
 # ---- scoring ----------------------------------------------------------------------------
 def _edp(D: int, edp_of_dp) -> np.ndarray:
     return np.arange(D, dtype=np.int32) if edp_of_dp is None else _i32(edp_of_dp)

@@ -965,3 +965,85 @@ void orc_diagnostics(int32_t N, int32_t L, int32_t E, int32_t P, int32_t D, int3
     att_joint[1] = (double)st->s[0] / SC;
     state_free(st);
 }
+
+/* ------------------------------------------------------------------------------------ */
+/* Randomized fixed-row seeds (Algorithm 2, the trial loop without the pairing and       */
+/* canonical-selection operators): one trial per population member.                      */
+/*                                                                                        */
+/* Reading of the two construction operators (the paper gives one sentence each):        */
+/*  WindowShuffle: walk the samples in order (-t_i, i); keep a window of the next w       */
+/*    not-yet-emitted samples; emit a uniformly chosen one of the window, close the gap   */
+/*    (order kept) and refill from the sorted list.  Draw: Philox(h, 0, trial, 4).x for   */
+/*    the h-th emitted sample, index = floor(x * window_size / 2^32).                     */
+/*  RandomizedBestFit: the first K emitted samples open the K cells in order; each later  */
+/*    sample looks at the cells it fits in, ranks them by (fuller first, then fewer       */
+/*    samples, then lower index) and takes a uniformly chosen one of the leading          */
+/*    min(w, #feasible).  Draw: Philox(h, 0, trial, 5).x.  No feasible cell: the trial    */
+/*    is aborted.                                                                          */
+/*  Cell b is (row b / D, slot b % D) (the pairing operator is not applied).              */
+/* Member 0 is always the length-only seed; member j >= 1 is trial j, or the length-only  */
+/* seed again when trial j aborted.  ok[j] = 1 when member j is its own trial's layout.   */
+/* ------------------------------------------------------------------------------------ */
+void orc_seed_trials(int32_t N, int32_t C, int32_t D, int32_t R, int32_t w, uint64_t seed, const int32_t *t,
+                     const int32_t *seed_layout, int32_t Ppop, int32_t *layouts, int32_t *ok)
+{
+    int32_t K = R * D;
+    int32_t *order = (int32_t *)malloc(sizeof(int32_t) * N);
+    for (int32_t i = 0; i < N; ++i) order[i] = i;
+    for (int32_t x = 1; x < N; ++x) {               /* insertion sort by (-t, i) */
+        int32_t s = order[x], y = x;
+        while (y > 0 && (t[order[y - 1]] < t[s] || (t[order[y - 1]] == t[s] && order[y - 1] > s))) {
+            order[y] = order[y - 1];
+            --y;
+        }
+        order[y] = s;
+    }
+    int32_t *win = (int32_t *)malloc(sizeof(int32_t) * (w > 0 ? w : 1));
+    int64_t *fill = (int64_t *)malloc(sizeof(int64_t) * K);
+    int32_t *cnt = (int32_t *)malloc(sizeof(int32_t) * K);
+    int32_t *cand = (int32_t *)malloc(sizeof(int32_t) * K);
+    for (int32_t j = 0; j < Ppop; ++j) {
+        int32_t *lay = layouts + (size_t)j * N;
+        memcpy(lay, seed_layout, sizeof(int32_t) * N);
+        ok[j] = (j == 0);
+        if (j == 0) continue;
+        int32_t nwin = 0, next = 0, good = 1;
+        for (int32_t b = 0; b < K; ++b) { fill[b] = 0; cnt[b] = 0; }
+        for (int32_t h = 0; h < N && good; ++h) {
+            while (nwin < w && next < N) win[nwin++] = order[next++];
+            uint32_t X[4];
+            draw(seed, (uint32_t)h, 0u, (uint32_t)j, 4u, X);
+            int32_t pos = pick(X[0], nwin);
+            int32_t s = win[pos];
+            for (int32_t x = pos; x + 1 < nwin; ++x) win[x] = win[x + 1];
+            --nwin;
+            int32_t b;
+            if (h < K) b = h;
+            else {
+                int32_t nc = 0;
+                for (int32_t c = 0; c < K; ++c) if (fill[c] + t[s] <= C) cand[nc++] = c;
+                if (nc == 0) { good = 0; break; }
+                /* order the feasible cells: fuller first, then fewer samples, then lower index */
+                for (int32_t x = 1; x < nc; ++x) {
+                    int32_t c = cand[x], y = x;
+                    while (y > 0) {
+                        int32_t p = cand[y - 1];
+                        int before = (fill[p] > fill[c]) || (fill[p] == fill[c] && (cnt[p] < cnt[c] || (cnt[p] == cnt[c] && p < c)));
+                        if (before) break;
+                        cand[y] = p;
+                        --y;
+                    }
+                    cand[y] = c;
+                }
+                draw(seed, (uint32_t)h, 0u, (uint32_t)j, 5u, X);
+                b = cand[pick(X[0], nc < w ? nc : w)];
+            }
+            fill[b] += t[s];
+            cnt[b] += 1;
+            lay[s] = b;
+        }
+        if (good) ok[j] = 1;
+        else memcpy(lay, seed_layout, sizeof(int32_t) * N);
+    }
+    free(order); free(win); free(fill); free(cnt); free(cand);
+}

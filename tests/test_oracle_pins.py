@@ -571,3 +571,56 @@ def test_diagnostics_against_numpy_and_placement_effect():
     assert d["cv_placed"] < d["cv_identity"]             # LPT lowers the aggregate skew
     SC = oracle.score_scale(s.token_cap)
     assert abs(d["attention"] - ev["Afx"][0].sum() / SC) < 1e-12 and abs(d["joint"] - ev["score"][0][0] / SC) < 1e-12
+
+
+# ----------------------------------------------------------------------------------------
+# randomized fixed-row seeds (Algorithm 2, trial loop)
+# ----------------------------------------------------------------------------------------
+def test_seed_trials_are_feasible_partitions_and_width_one_is_best_fit_decreasing():
+    w = hetero_window(N=90, L=2, E=8, k=1, C=4096, D=3, P=4, seed=41)
+    s = w.spec
+    t = w.lengths
+    R, _, seed = oracle.pack_ffd(t, s.token_cap, s.dp_width, min_rows=3)
+    K = R * s.dp_width
+    for width in (1, 4, 16):
+        lays, ok = oracle.seed_trials(t, seed, R, s.token_cap, s.dp_width, 24, width, seed=9)
+        assert ok[0] == 1 and (lays[0] == seed).all()
+        for j in range(24):
+            assert lays[j].min() >= 0 and lays[j].max() < K
+            assert (np.bincount(lays[j], minlength=K) >= 1).all()
+            assert (np.bincount(lays[j], weights=t, minlength=K) <= s.token_cap).all()
+            if not ok[j]:
+                assert (lays[j] == seed).all()
+        if width == 1:
+            # no randomness left: decreasing order, K longest open the cells, then the fullest
+            # feasible cell (ties: fewer samples, lower index) -- plain best-fit-decreasing
+            order = sorted(range(len(t)), key=lambda i: (-int(t[i]), i))
+            fill, cnt, want = [0] * K, [0] * K, [0] * len(t)
+            for h, i in enumerate(order):
+                if h < K:
+                    b = h
+                else:
+                    feas = [c for c in range(K) if fill[c] + t[i] <= s.token_cap]
+                    b = min(feas, key=lambda c: (-fill[c], cnt[c], c))
+                fill[b] += int(t[i]); cnt[b] += 1; want[i] = b
+            assert ok[1:].all() and all((lays[j] == want).all() for j in range(1, 24))
+        else:
+            assert len({lays[j].tobytes() for j in range(24)}) > 12      # the trials really differ
+
+
+def test_seed_trial_draws_are_uniform_over_the_window():
+    """With as many cells as samples every sample opens the cell of its emission position, so the
+    layout is the shuffle itself: the first emitted sample must be a uniform pick among the first
+    w samples of the sorted order, and no sample can be emitted more than w-1 places early."""
+    N, width = 64, 8
+    t = np.full(N, 10, np.int32)                       # equal lengths: sorted order = index order
+    seed = np.arange(N, dtype=np.int32)
+    lays, ok = oracle.seed_trials(t, seed, 16, 10, 4, 4000, width, seed=5)
+    assert ok.all()
+    first = np.array([int(np.where(lays[j] == 0)[0][0]) for j in range(1, 4000)])
+    counts = np.bincount(first, minlength=N)
+    assert counts[width:].sum() == 0
+    assert abs(counts[:width] - 3999 / width).max() < 5 * (3999 / width * (1 - 1 / width)) ** 0.5
+    for j in range(1, 200):
+        assert sorted(lays[j].tolist()) == list(range(N))            # a permutation
+        assert (lays[j] >= np.arange(N) - (width - 1)).all()         # sample i leaves no earlier than i-(w-1)
