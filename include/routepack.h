@@ -115,6 +115,17 @@ int rp_place_experts(rp_ctx *ctx, int32_t *pi, int64_t *rank_load);
  *   n_rows, certified: HOST scalars out (nullable). */
 int rp_pack_rows(rp_ctx *ctx, int32_t *n_rows, int32_t *certified);
 
+/* Randomized fixed-row seeds (Algorithm 2, the trial loop; the pairing and canonical-selection
+ * operators are not applied).  Optional, between rp_pack_rows and rp_anneal.  Member 0 keeps the
+ * length-only seed; member j >= 1 runs trial j: WindowShuffle (emit a uniformly chosen one of the
+ * next choice_width samples in decreasing-length order) feeds RandomizedBestFit (the first R*D
+ * emitted samples open the cells; each later one takes a uniformly chosen one of the leading
+ * choice_width cells it fits in, ranked fuller first, then fewer samples, then lower index);
+ * a trial with no feasible cell is dropped and its member keeps the length-only seed.  All
+ * members are scored from scratch; the incumbent becomes the best member (lowest index on ties).
+ *   choice_width in [1, 32]; n_own: HOST out, members that carry their own trial (nullable). */
+int rp_seed_population(rp_ctx *ctx, int32_t choice_width, int32_t *n_own);
+
 /* Full evaluation of layouts (Section 3.4-3.5: Eqs. cell-token-statistics,
  * stage-aware-attention, row-expert-load, row-expert-cost, lexicographic-score).
  *   layouts [n][N] int32 cell ids, or NULL to score the current population (n = pop_size).

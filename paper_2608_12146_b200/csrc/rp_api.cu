@@ -131,7 +131,7 @@ extern "C" void rp_destroy(rp_ctx *c)
     free_population(c); free_trace(c); free_eval(c);
     dev_free(c, c->own_t); dev_free(c, c->own_a); dev_free(c, c->d_edp); dev_free(c, c->d_dp_list); dev_free(c, c->d_dp_off);
     dev_free(c, c->d_Lagg); dev_free(c, c->d_pi); dev_free(c, c->d_inv); dev_free(c, c->d_rank_load); dev_free(c, c->d_q);
-    dev_free(c, c->d_status); dev_free(c, c->d_sort_keys); dev_free(c, c->d_seed_layout); dev_free(c, c->d_pack_out);
+    dev_free(c, c->d_status); dev_free(c, c->d_sort_keys); dev_free(c, c->d_seed_layout); dev_free(c, c->d_order); dev_free(c, c->d_pack_out);
     dev_free(c, c->d_counters); dev_free(c, c->d_inc_layout); dev_free(c, c->d_inc_score); dev_free(c, c->d_static);
     free(c->h_levels); free(c->h_t);
     free(c);
@@ -235,6 +235,7 @@ static int window_load_impl(rp_ctx *c, const rp_config *cfg, const int32_t *leng
     while (n_pow2 < N) n_pow2 <<= 1;
     RP_TRY(dev_alloc(c, &c->d_sort_keys, (size_t)2 * n_pow2));
     RP_TRY(dev_alloc(c, &c->d_seed_layout, N));
+    RP_TRY(dev_alloc(c, &c->d_order, N));
     RP_TRY(dev_alloc(c, &c->d_pack_out, 4));
     RP_TRY(dev_alloc(c, &c->d_counters, 8));
     RP_TRY(dev_alloc(c, &c->d_inc_layout, N));
@@ -426,6 +427,45 @@ extern "C" int rp_eval_population(rp_ctx *c, const int32_t *layouts, int32_t n, 
     RP_TRY(copy_out(c, score_fx, c->d_eval_score, sizeof(i64) * 3 * (size_t)n));
     RP_TRY(copy_out(c, score_f64, c->d_eval_f64, sizeof(double) * 3 * (size_t)n));
     RP_CUDA(cudaStreamSynchronize(c->stream));
+    return RP_OK;
+}
+
+// Randomized fixed-row seeds (Algorithm 2, trial loop): member 0 keeps the length-only seed, every
+// other member runs its own WindowShuffle + RandomizedBestFit trial; all members are then scored
+// from scratch and the incumbent becomes the best of them.
+extern "C" int rp_seed_population(rp_ctx *c, int32_t choice_width, int32_t *n_own)
+{
+    if (!c) return RP_ERR_ARG;
+    if (c->stage != 3) return RP_ERR_STATE;          // after rp_pack_rows, before rp_anneal
+    if (choice_width < 1 || choice_width > 32) return RP_ERR_ARG;
+    const RpDims &dm = c->dm;
+    if (dm.K > 2048) return RP_ERR_RANGE;            // per-warp cell tables live in shared memory
+    const size_t P = (size_t)c->Ppop;
+    int *lay = nullptr, *ok = nullptr;
+    i64 *best = nullptr;
+    RP_TRY(dev_alloc(c, &lay, P * dm.N));
+    int st = dev_alloc(c, &ok, P);
+    if (st == RP_OK) st = dev_alloc(c, &best, 3);
+    if (st == RP_OK) st = rp_launch_seed_trials(c, choice_width, lay, ok);
+    if (st == RP_OK) st = ensure_eval_scratch(c, P, false);
+    if (st == RP_OK) st = rp_launch_cells_from_layouts(c, lay, (int)P, c->d_eval_cells);
+    c->cur = 0;
+    if (st == RP_OK) st = rp_launch_eval(c, c->d_eval_cells, (int)P, c->buf[0].W, c->buf[0].blob, c->d_eval_score, nullptr);
+    if (st == RP_OK) st = rp_launch_pick_best(c, c->d_eval_score, lay, (int)P, best);
+    int *h_ok = (int *)malloc(sizeof(int) * P);
+    cudaError_t e = cudaSuccess;
+    if (st == RP_OK) {
+        e = cudaMemcpyAsync(h_ok, ok, sizeof(int) * P, cudaMemcpyDeviceToHost, c->stream);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(c->seed_score, best, sizeof(i64) * 3, cudaMemcpyDeviceToHost, c->stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+    }
+    int own = 0;
+    if (st == RP_OK && e == cudaSuccess) for (size_t j = 0; j < P; ++j) own += h_ok[j];
+    free(h_ok);
+    dev_free(c, lay); dev_free(c, ok); dev_free(c, best);
+    if (e != cudaSuccess) { g_rp_last_cuda_error = (int)e; return RP_ERR_CUDA; }
+    RP_TRY(st);
+    if (n_own) *n_own = own;
     return RP_OK;
 }
 

@@ -109,6 +109,7 @@ struct rp_ctx {
     // packing
     u64 *d_sort_keys;          // scratch for the length sort
     int *d_seed_layout;        // [N]
+    int *d_order;              // [N] samples sorted by (-t, i)
     int *d_pack_out;           // [4]: R*, certified, R_lb, failure flag
     int Rstar, certified;
     i64 seed_score[3];
@@ -165,6 +166,8 @@ int rp_launch_pack(rp_ctx *c, int Rlb_hint);
 int rp_launch_eval(rp_ctx *c, const unsigned short *cells, int n, int *W_out, char *blob_out,
                    i64 *score_out, double *f64_out);
 int rp_launch_build_static(rp_ctx *c);
+int rp_launch_seed_trials(rp_ctx *c, int width, int *layouts, int *ok);
+int rp_launch_pick_best(rp_ctx *c, const i64 *scores, const int *layouts, int n, i64 *best_score_out);
 int rp_get_pool(int device, cudaMemPool_t *out);     // the library's stream-ordered pool of a device
 void rp_make_layouts(const RpDims &dm, RpBlob *bl, RpStatic *sl);
 int rp_launch_cells_from_layouts(rp_ctx *c, const int *layouts, int n, unsigned short *cells);

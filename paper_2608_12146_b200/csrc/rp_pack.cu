@@ -11,7 +11,7 @@
 
 __global__ void __launch_bounds__(PACK_THREADS)
 k_pack_ffd(RpDims dm, const int *__restrict__ t, int min_rows, u64 *__restrict__ keys_g, int n_pow2,
-           int *__restrict__ fill_g, int *__restrict__ cell_of, int *__restrict__ out)
+           int *__restrict__ fill_g, int *__restrict__ cell_of, int *__restrict__ out, int *__restrict__ order_out)
 {
     extern __shared__ u64 keys_s[];
     u64 *keys = keys_g ? keys_g : keys_s;
@@ -45,6 +45,7 @@ k_pack_ffd(RpDims dm, const int *__restrict__ t, int min_rows, u64 *__restrict__
             }
             __syncthreads();
         }
+    for (int x = tid; x < dm.N; x += PACK_THREADS) order_out[x] = (int)(u32)keys[x];   // samples by (-t, i)
     const i64 cap_row = (i64)dm.C * dm.D;
     i64 Rlb = (total_s + cap_row - 1) / cap_row;
     if (Rlb < 1) Rlb = 1;
@@ -111,7 +112,7 @@ int rp_launch_pack(rp_ctx *c, int /*unused*/)
     if (smem > 32 * 1024)
         RP_CUDA(cudaFuncSetAttribute(k_pack_ffd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     k_pack_ffd<<<1, PACK_THREADS, smem, c->stream>>>(dm, c->d_t, c->cfg.min_rows, keys_g, n_pow2, fill_g,
-                                                    c->d_seed_layout, c->d_pack_out);
+                                                    c->d_seed_layout, c->d_pack_out, c->d_order);
     ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
     return RP_OK;

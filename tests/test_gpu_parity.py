@@ -66,11 +66,12 @@ def check_eval(w, ctx, ref, edp, n=6, seed=0):
         np.testing.assert_allclose(f64[j], real, rtol=F64_RTOL, atol=0)
 
 
-def check_anneal(w, ctx, ref, edp, pop, levels, steps, threads=8, t_ratio=None, check_members=3):
+def check_anneal(w, ctx, ref, edp, pop, levels, steps, threads=8, t_ratio=None, check_members=3, init=None):
     s = w.spec
     R, D = ref["R"], s.dp_width
     ratio = s.t_ratio if t_ratio is None else t_ratio
-    init = np.tile(ref["seed"], (pop, 1))
+    if init is None:
+        init = np.tile(ref["seed"], (pop, 1))
     want = oracle.anneal(w.lengths, ref["q"], init, R, s.token_cap, D, n_levels=levels, steps=steps, t0=s.t0,
                          t_ratio=ratio, p_reloc=s.p_reloc, p_guide=s.p_guide, seed=s.anneal_seed,
                          edp_of_dp=edp, alpha=s.alpha, beta=s.beta, n_threads=threads)
@@ -250,6 +251,39 @@ def test_full_size_properties_large():
     assert tuple(ev["score"][0]) == tuple(fx) == inc[-1]
     seed_score = oracle.eval_layouts(w.lengths, ref["q"], ref["seed"], R, s.token_cap, s.dp_width)["score"][0]
     assert tuple(fx) <= tuple(seed_score)
+    rp.rp_destroy(ctx)
+
+
+@pytest.mark.parametrize("case,width", [("medium", 4), ("shared", 8), ("ragged", 1), ("large", 3)])
+def test_randomized_seed_population(case, width):
+    """Algorithm 2's trial loop: every member's seed layout, which trials were dropped, the scores
+    of the seeded population and the annealing that starts from it, all against the oracle."""
+    edp, min_rows, pop = None, 0, 48
+    if case == "medium":
+        w = make_window("medium")
+    elif case == "large":
+        w = make_window("large")
+    elif case == "shared":
+        w = make_window(custom_spec("seeds_shared", 96, 5, 16, 2, 4096, 4, 4, pop, 400, data_seed=5))
+        edp, min_rows = [0, 0, 1, 1], 3
+    else:
+        w = make_window(custom_spec("seeds_ragged", 77, 3, 12, 2, 3000, 3, 3, pop, 400, data_seed=6))
+        min_rows = 4
+    s = w.spec
+    ref = oracle_front(w, edp, min_rows)
+    ctx = load(w, pop=pop, edp=edp, min_rows=min_rows)
+    check_front(w, ctx, ref)
+    lays, ok = oracle.seed_trials(w.lengths, ref["seed"], ref["R"], s.token_cap, s.dp_width, pop, width, s.anneal_seed)
+    own = rp.rp_seed_population(ctx, width)
+    assert own == int(ok.sum())
+    assert (rp.rp_debug_dump(ctx, "POPULATION", (pop, s.n_samples), np.int32) == lays).all()
+    ev = oracle.eval_layouts(w.lengths, ref["q"], lays, ref["R"], s.token_cap, s.dp_width, edp, s.alpha, s.beta)
+    fx, _ = rp.rp_eval_population(ctx)
+    assert (fx == ev["score"]).all()
+    best = min(range(pop), key=lambda j: (tuple(ev["score"][j]), j))
+    layout, bfx, _ = rp.rp_best(ctx)
+    assert (layout == lays[best]).all() and tuple(bfx) == tuple(ev["score"][best])
+    check_anneal(w, ctx, ref, edp, pop, 4, 40, t_ratio=0.5, check_members=2, init=lays)
     rp.rp_destroy(ctx)
 
 
