@@ -14,6 +14,8 @@
 // by its warp straight from its registers, and everything speculated after it is discarded
 // and redone; if none is accepted the next NW follow.  This is step-for-step the sequential
 // chain of Algorithm 3: a later step is only ever scored against the state it would have seen.
+#include <string.h>
+
 #include "rp_level_end.cuh"
 
 struct ChainS {                 // bookkeeping of the chain within this level
@@ -64,11 +66,20 @@ k_anneal_wpc(const AnnealArgs A)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int j = blockIdx.x;
-    const int src = A.anc[j];
     const bool identity_edp = (dm.G == dm.D);
     int *Wj = WS ? Wsm : A.W_dst + (size_t)j * wn;
     const bool vec = (dm.P >= 4) && (dm.P <= 128) && ((dm.P & (dm.P - 1)) == 0);
     const i64 aC = dm.asum * dm.C, bS = dm.bsum;
+
+    // The step records of the first batch depend on nothing the previous level wrote: compute
+    // them before waiting for it (this kernel is launched with programmatic stream
+    // serialisation, so it may start while the previous level's last CTA runs the barrier).
+    {
+        const int nb0 = min(NT, A.steps);
+        if (tid < nb0) recs[tid] = rp_make_step_rec(A, (u32)tid, (u32)blockIdx.x);
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int src = A.anc[j];
 
     // ---- prologue: adopt the ancestor's terminal state -------------------------------
     if (tid == 0) chain->failed = 0;
@@ -97,7 +108,7 @@ k_anneal_wpc(const AnnealArgs A)
 
     for (int kb = 0; kb < A.steps; kb += NT) {
         const int nb = min(NT, A.steps - kb);
-        if (tid < nb) recs[tid] = rp_make_step_rec(A, (u32)(kb + tid), (u32)j);
+        if (kb > 0 && tid < nb) recs[tid] = rp_make_step_rec(A, (u32)(kb + tid), (u32)j);
         __syncthreads();
 
         int pos = 0;
@@ -325,6 +336,7 @@ k_anneal_wpc(const AnnealArgs A)
         atomicAdd((u64 *)&A.counters[0], (u64)A.steps);
         if (src != j) atomicAdd((u64 *)&A.counters[5], (u64)2 * dm.RG * dm.LP * 4);
     }
+    asm volatile("griddepcontrol.launch_dependents;");     // the next level may start its own prologue
     rp_finish_level(A, tid, NT);
 }
 
@@ -358,7 +370,15 @@ static int launch_wpc(rp_ctx *c, const AnnealArgs &A, int ws, size_t smem, int c
     do {                                                                                              \
         if (smem > 32 * 1024)                                                                         \
             RP_CUDA(cudaFuncSetAttribute(k_anneal_wpc<NW, WS_, CH_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
-        k_anneal_wpc<NW, WS_, CH_><<<c->Ppop, NW * 32, smem, c->stream>>>(A);                         \
+        cudaLaunchConfig_t cfg;                                                                       \
+        memset(&cfg, 0, sizeof cfg);                                                                  \
+        cfg.gridDim = dim3(c->Ppop); cfg.blockDim = dim3(NW * 32);                                    \
+        cfg.dynamicSmemBytes = smem; cfg.stream = c->stream;                                          \
+        cudaLaunchAttribute at[1];                                                                    \
+        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;                                \
+        at[0].val.programmaticStreamSerializationAllowed = 1;                                         \
+        cfg.attrs = at; cfg.numAttrs = 1;                                                             \
+        RP_CUDA(cudaLaunchKernelEx(&cfg, k_anneal_wpc<NW, WS_, CH_>, A));                              \
     } while (0)
     if (ws) { if (chunks <= 1) LAUNCH(true, 1); else if (chunks <= 2) LAUNCH(true, 2); else LAUNCH(true, 4); }
     else { if (chunks <= 1) LAUNCH(false, 1); else if (chunks <= 2) LAUNCH(false, 2); else LAUNCH(false, 4); }
