@@ -80,7 +80,7 @@ k_anneal_level(const AnnealArgs A)
     const int j = blockIdx.x;
     const int src = A.anc[j];
     const bool identity_edp = (dm.G == dm.D);
-    int *Wj = A.W_dst + (size_t)j * wn;
+    int *Wj = A.W + (size_t)A.wloc_dst[j] * wn;
     const bool vec = (dm.P >= 4) && (dm.P <= 128) && ((dm.P & (dm.P - 1)) == 0);
     const i64 aC = dm.asum * dm.C, bS = dm.bsum;
 
@@ -308,7 +308,7 @@ k_anneal_level(const AnnealArgs A)
         atomicAdd((u64 *)&A.counters[2], (u64)n_acc);
         atomicAdd((u64 *)&A.counters[3], (u64)n_imp);
         atomicAdd((u64 *)&A.counters[4], (u64)n_bytes);
-        if (src != j) atomicAdd((u64 *)&A.counters[5], (u64)2 * dm.RG * dm.LP * 4);
+        if (A.wloc_src[src] != A.wloc_dst[j]) atomicAdd((u64 *)&A.counters[5], (u64)2 * dm.RG * dm.LP * 4);
     }
     rp_finish_level(A, tid, NT);
 }
@@ -347,7 +347,7 @@ int rp_launch_anneal_level(rp_ctx *c, int level, int n_levels, const rp_anneal_p
     A.t = c->d_t; A.q = c->d_q; A.static_blk = c->d_static;
     const RpPopBuf &s = c->buf[c->cur], &d = c->buf[1 - c->cur];
     A.blob_src = s.blob; A.blob_dst = d.blob;
-    A.W_src = s.W; A.W_dst = d.W;
+    A.W = c->d_W; A.wloc_src = c->d_wloc; A.wloc_dst = c->d_wloc_next;
     A.anc = c->d_anc;
     A.level = level; A.steps = prm->steps_per_level; A.log_cap = c->log_cap;
     A.rho_q32 = rho_q32; A.guide_q32 = guide_q32;
@@ -358,7 +358,9 @@ int rp_launch_anneal_level(rp_ctx *c, int level, int n_levels, const rp_anneal_p
     A.cq = c->h_levels[level].cq;
     A.Ppop = c->Ppop;
     A.last = (level == n_levels - 1);
+    A.w_on_chip = 0;
     A.lo.done = c->d_done; A.lo.anc_out = c->d_anc_next; A.lo.F = c->d_F;
+    A.lo.wloc_out = c->d_wloc; A.lo.scratch = c->d_le_scratch;   // the barrier rewrites the array the level read from
     A.lo.inc_layout = c->d_inc_layout; A.lo.inc_score = c->d_inc_score;
     A.lo.tr_term = c->d_tr_term; A.lo.tr_best = c->d_tr_best; A.lo.tr_inc = c->d_tr_inc;
     A.lo.tr_best_step = c->d_tr_best_step; A.lo.tr_anc = c->d_tr_anc; A.lo.tr_digest = c->d_tr_digest;

@@ -8,6 +8,8 @@
 struct LevelOut {
     int *done;                 // arrival counter of the chain CTAs (zero between launches)
     int *anc_out;              // [P_pop] ancestors for the next level
+    int *wloc_out;             // [P_pop] W cells for the next level
+    int *scratch;              // [6*P_pop] ints
     u64 *F;                    // [P_pop] cumulative resampling weights
     int *inc_layout;           // [N]
     i64 *inc_score;            // [3]
@@ -23,9 +25,12 @@ struct AnnealArgs {
     const int *t, *q;
     const char *static_blk;
     const char *blob_src;  char *blob_dst;
-    const int *W_src;      int *W_dst;
+    int *W;                          // rank-load cells [2*P_pop][RG][LP]
+    const int *wloc_src;             // [P_pop] cell of each member's W at the start of the level
+    int *wloc_dst;                   // [P_pop] cell each slot works in; rewritten by the level barrier for the next level
     const int *anc;
     int level, steps, log_cap, Ppop, last;
+    int w_on_chip;                   // W is staged in shared memory: every level moves it anyway
     u64 tau, cq, rho_q32, guide_q32;
     u32 key0, key1;
     i64 *term, *best;
@@ -234,7 +239,8 @@ __device__ __forceinline__ bool rp_chain_load(const AnnealArgs &A, int src, int 
 {
     const RpDims &dm = A.dm;
     const size_t wn = (size_t)dm.RG * dm.LP;
-    const int *ws = A.W_src + (size_t)src * wn;
+    const int src_cell = A.wloc_src[src], dst_cell = A.wloc_dst[j];
+    const int *ws = A.W + (size_t)src_cell * wn;
     const bool w_bulk = WS && ((wn & 3) == 0);
     if (tid == 0) {
         rp_mbar_init(mbar, 1);
@@ -248,8 +254,8 @@ __device__ __forceinline__ bool rp_chain_load(const AnnealArgs &A, int src, int 
                 rp_bulk_g2s((char *)Wsm + off, (const char *)ws + off, n, mbar);
             }
     }
-    if (!w_bulk) {
-        int *wd = WS ? Wsm : A.W_dst + (size_t)j * wn;
+    if (!w_bulk && (WS || src_cell != dst_cell)) {      // a sole child works on in its ancestor's cell
+        int *wd = WS ? Wsm : A.W + (size_t)dst_cell * wn;
         if ((wn & 3) == 0) {
             const int4 *ws4 = (const int4 *)ws;
             int4 *wd4 = (int4 *)wd;
@@ -274,7 +280,7 @@ __device__ __forceinline__ void rp_chain_store(const AnnealArgs &A, int j, const
     if (tid == 0) {
         rp_bulk_s2g(A.blob_dst + (size_t)j * A.bl.bytes, sm_blob, (u32)A.bl.bytes);
         if (w_bulk) {
-            int *wd = A.W_dst + (size_t)j * wn;
+            int *wd = A.W + (size_t)A.wloc_dst[j] * wn;
             for (size_t off = 0; off < wn * 4; off += 32768) {
                 const u32 n = (u32)((wn * 4 - off) < 32768 ? (wn * 4 - off) : 32768);
                 rp_bulk_s2g((char *)wd + off, (const char *)Wsm + off, n);
@@ -283,7 +289,7 @@ __device__ __forceinline__ void rp_chain_store(const AnnealArgs &A, int j, const
         rp_bulk_commit_wait();
     }
     if (WS && !w_bulk) {
-        int *wd = A.W_dst + (size_t)j * wn;
+        int *wd = A.W + (size_t)A.wloc_dst[j] * wn;
         for (size_t x = tid; x < wn; x += NT) wd[x] = Wsm[x];
     }
 }

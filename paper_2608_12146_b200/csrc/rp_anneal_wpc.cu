@@ -67,7 +67,6 @@ k_anneal_wpc(const AnnealArgs A)
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int j = blockIdx.x;
     const bool identity_edp = (dm.G == dm.D);
-    int *Wj = WS ? Wsm : A.W_dst + (size_t)j * wn;
     const bool vec = (dm.P >= 4) && (dm.P <= 128) && ((dm.P & (dm.P - 1)) == 0);
     const i64 aC = dm.asum * dm.C, bS = dm.bsum;
 
@@ -80,6 +79,7 @@ k_anneal_wpc(const AnnealArgs A)
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const int src = A.anc[j];
+    int *Wj = WS ? Wsm : A.W + (size_t)A.wloc_dst[j] * wn;     // the previous level's barrier wrote wloc_dst
 
     // ---- prologue: adopt the ancestor's terminal state -------------------------------
     if (tid == 0) chain->failed = 0;
@@ -334,7 +334,7 @@ k_anneal_wpc(const AnnealArgs A)
         A.best_nlog[j] = chain->best_nlog;
         A.digest[j] = chain->dig;
         atomicAdd((u64 *)&A.counters[0], (u64)A.steps);
-        if (src != j) atomicAdd((u64 *)&A.counters[5], (u64)2 * dm.RG * dm.LP * 4);
+        if (A.wloc_src[src] != A.wloc_dst[j]) atomicAdd((u64 *)&A.counters[5], (u64)2 * dm.RG * dm.LP * 4);
     }
     asm volatile("griddepcontrol.launch_dependents;");     // the next level may start its own prologue
     rp_finish_level(A, tid, NT);
@@ -388,12 +388,14 @@ static int launch_wpc(rp_ctx *c, const AnnealArgs &A, int ws, size_t smem, int c
     return RP_OK;
 }
 
-int rp_launch_anneal_wpc(rp_ctx *c, const AnnealArgs &A)
+int rp_launch_anneal_wpc(rp_ctx *c, const AnnealArgs &A0)
 {
     const RpDims &dm = c->dm;
     const int nw = rp_wpc_warps(c->Ppop);
     int ws = 0;
     const size_t smem = rp_wpc_smem_bytes(dm, c->bl, c->sl, nw, &ws);
+    AnnealArgs A = A0;
+    A.w_on_chip = ws;
     if (smem > 220 * 1024) return RP_ERR_RANGE;
     const int chunks = ((dm.LP >> 2) + 31) / 32;
     if (nw == 8) return launch_wpc<8>(c, A, ws, smem, chunks);

@@ -95,9 +95,11 @@ static int copy_out(rp_ctx *c, void *dst, const void *src, size_t bytes)
 static void free_population(rp_ctx *c)
 {
     for (int b = 0; b < 2; ++b) {
-        dev_free(c, c->buf[b].blob); dev_free(c, c->buf[b].W);
-        c->buf[b].blob = nullptr; c->buf[b].W = nullptr;
+        dev_free(c, c->buf[b].blob);
+        c->buf[b].blob = nullptr;
     }
+    dev_free(c, c->d_W); dev_free(c, c->d_wloc); dev_free(c, c->d_wloc_next); dev_free(c, c->d_le_scratch);
+    c->d_W = nullptr; c->d_wloc = nullptr; c->d_wloc_next = nullptr; c->d_le_scratch = nullptr;
     dev_free(c, c->d_anc); dev_free(c, c->d_anc_next); dev_free(c, c->d_done); dev_free(c, c->d_term); dev_free(c, c->d_best); dev_free(c, c->d_best_step);
     dev_free(c, c->d_best_nlog); dev_free(c, c->d_digest); dev_free(c, c->d_log); dev_free(c, c->d_F);
     c->d_anc = nullptr; c->d_anc_next = nullptr; c->d_done = nullptr; c->d_term = nullptr; c->d_best = nullptr; c->d_best_step = nullptr;
@@ -327,6 +329,12 @@ static int ensure_eval_scratch(rp_ctx *c, size_t n, bool want_W)
     return RP_OK;
 }
 
+__global__ void k_iota(int *out, int n, int first)
+{
+    const int x = blockIdx.x * blockDim.x + threadIdx.x;
+    if (x < n) out[x] = first + x;
+}
+
 extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
 {
     if (!c) return RP_ERR_ARG;
@@ -350,8 +358,11 @@ extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
     const size_t P = (size_t)c->Ppop, wn = (size_t)dm.RG * dm.LP;
     for (int b = 0; b < 2; ++b) {
         RP_TRY(dev_alloc(c, &c->buf[b].blob, P * (size_t)c->bl.bytes));
-        RP_TRY(dev_alloc(c, &c->buf[b].W, P * wn));
     }
+    RP_TRY(dev_alloc(c, &c->d_W, 2 * P * wn));
+    RP_TRY(dev_alloc(c, &c->d_wloc, P));
+    RP_TRY(dev_alloc(c, &c->d_wloc_next, P));
+    RP_TRY(dev_alloc(c, &c->d_le_scratch, 6 * P));
     RP_TRY(dev_alloc(c, &c->d_anc, P));
     RP_TRY(dev_alloc(c, &c->d_anc_next, P));
     RP_TRY(dev_alloc(c, &c->d_done, 1));
@@ -370,8 +381,12 @@ extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
     RP_TRY(rp_launch_build_static(c));
     RP_TRY(ensure_eval_scratch(c, 1, false));
     RP_TRY(rp_launch_cells_from_layouts(c, c->d_seed_layout, 1, c->d_eval_cells));
-    RP_TRY(rp_launch_eval(c, c->d_eval_cells, 1, c->buf[0].W, c->buf[0].blob, c->d_inc_score, nullptr));
+    RP_TRY(rp_launch_eval(c, c->d_eval_cells, 1, c->d_W, c->buf[0].blob, c->d_inc_score, nullptr));
     RP_CUDA(cudaMemsetAsync(c->d_anc, 0, sizeof(int) * P, c->stream));
+    // the seed's W sits in cell 0; every member copies it into a cell of its own (P + m) at level 0
+    RP_CUDA(cudaMemsetAsync(c->d_wloc, 0, sizeof(int) * P, c->stream));
+    k_iota<<<(int)((P + 255) / 256), 256, 0, c->stream>>>(c->d_wloc_next, (int)P, (int)P);
+    ++g_rp_launches;
     RP_CUDA(cudaMemcpyAsync(c->d_inc_layout, c->d_seed_layout, sizeof(int) * dm.N, cudaMemcpyDeviceToDevice, c->stream));
     RP_CUDA(cudaMemcpyAsync(c->seed_score, c->d_inc_score, sizeof(i64) * 3, cudaMemcpyDeviceToHost, c->stream));
     RP_CUDA(cudaStreamSynchronize(c->stream));
@@ -450,7 +465,12 @@ extern "C" int rp_seed_population(rp_ctx *c, int32_t choice_width, int32_t *n_ow
     if (st == RP_OK) st = ensure_eval_scratch(c, P, false);
     if (st == RP_OK) st = rp_launch_cells_from_layouts(c, lay, (int)P, c->d_eval_cells);
     c->cur = 0;
-    if (st == RP_OK) st = rp_launch_eval(c, c->d_eval_cells, (int)P, c->buf[0].W, c->buf[0].blob, c->d_eval_score, nullptr);
+    if (st == RP_OK) st = rp_launch_eval(c, c->d_eval_cells, (int)P, c->d_W, c->buf[0].blob, c->d_eval_score, nullptr);
+    if (st == RP_OK) {           // member m owns cell m and works on in it
+        k_iota<<<(int)((P + 255) / 256), 256, 0, c->stream>>>(c->d_wloc, (int)P, 0);
+        k_iota<<<(int)((P + 255) / 256), 256, 0, c->stream>>>(c->d_wloc_next, (int)P, 0);
+        g_rp_launches += 2;
+    }
     if (st == RP_OK) st = rp_launch_pick_best(c, c->d_eval_score, lay, (int)P, best);
     int *h_ok = (int *)malloc(sizeof(int) * P);
     cudaError_t e = cudaSuccess;
@@ -530,6 +550,7 @@ extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *
         st = rp_launch_anneal_level(c, n, NL, p, rho_q32, guide_q32);
         c->cur = 1 - c->cur;          // the terminal states are the next level's sources
         { int *sw = c->d_anc; c->d_anc = c->d_anc_next; c->d_anc_next = sw; }
+        { int *sw = c->d_wloc; c->d_wloc = c->d_wloc_next; c->d_wloc_next = sw; }
     }
     if (stats) cudaEventRecord(ev[1], c->stream);
     cudaError_t e = cudaStreamSynchronize(c->stream);
@@ -631,7 +652,12 @@ extern "C" int rp_debug_dump(rp_ctx *c, int what, int32_t index, void *buf, int6
             src = tmp;
             break;
         }
-        case RP_DUMP_W: src = c->buf[c->cur].W + (size_t)member * dm.RG * dm.LP; need = sizeof(int) * (size_t)dm.RG * dm.LP; break;
+        case RP_DUMP_W: {
+            int cell = 0;
+            RP_CUDA(cudaMemcpyAsync(&cell, c->d_wloc + member, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+            RP_CUDA(cudaStreamSynchronize(c->stream));
+            src = c->d_W + (size_t)cell * dm.RG * dm.LP; need = sizeof(int) * (size_t)dm.RG * dm.LP; break;
+        }
         case RP_DUMP_ESUM: src = c->buf[c->cur].blob + (size_t)member * c->bl.bytes + c->bl.off_Esum; need = sizeof(i64) * dm.RG; break;
         case RP_DUMP_CELL_T: case RP_DUMP_CELL_Q: case RP_DUMP_CELL_CNT: {
             size_t K = dm.K;

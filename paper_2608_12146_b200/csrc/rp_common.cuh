@@ -82,7 +82,6 @@ struct RpStatic {
 // one population buffer set (two of them: the level reads one and writes the other)
 struct RpPopBuf {
     char *blob;                // [P_pop][blob.bytes]
-    int *W;                    // [P_pop][RG][LP]
 };
 
 struct rp_ctx {
@@ -115,6 +114,10 @@ struct rp_ctx {
     i64 seed_score[3];
     // population
     RpPopBuf buf[2];
+    int *d_W;                  // [2*P_pop][RG][LP] rank-load cells; a member's W sits in the cell wloc says
+    int *d_wloc;               // [P_pop] cell of each member's current W (read through d_anc)
+    int *d_wloc_next;          // [P_pop] cell each member works in during the next level
+    int *d_le_scratch;         // [6*P_pop] ints for the level barrier's cell bookkeeping
     RpBlob bl;
     RpStatic sl;
     char *d_static;            // static tables block

@@ -82,7 +82,7 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
     if (O.tr_inc && tid < 3) O.tr_inc[(size_t)A.level * 3 + tid] = O.inc_score[tid];
 
     if (A.last) {            // the terminal states are the population as they stand
-        for (int m = tid; m < P; m += nt) O.anc_out[m] = m;
+        for (int m = tid; m < P; m += nt) { O.anc_out[m] = m; O.wloc_out[m] = A.wloc_dst[m]; }
         return;
     }
 
@@ -146,6 +146,59 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
         O.anc_out[m] = lo;
         if (O.tr_anc) O.tr_anc[(size_t)A.level * P + m] = lo;
     }
+    __syncthreads();
+
+    // ---- W cells of the next level.  A member that is its ancestor's only child works on in the
+    // ancestor's cell; children of an ancestor with several children each get a free cell and
+    // copy.  Cells: 2*P of them; the ones no surviving ancestor holds are free.
+    int *kids = O.scratch;                 // [P]   children per ancestor
+    int *need = kids + P;                  // [P]   1 = this member needs a fresh cell -> exclusive ranks
+    int *isfree = need + P;                // [2P]  1 = free cell -> exclusive ranks
+    int *freelist = isfree + 2 * P;        // [2P]  k-th free cell
+    const int *now = A.wloc_dst;           // cells the terminal states of this level sit in
+    if (A.w_on_chip) {      // W goes through shared memory every level anyway: alternate between the two halves
+        for (int m = tid; m < P; m += nt) O.wloc_out[m] = (now[m] >= P) ? m : P + m;
+        return;
+    }
+    for (int a = tid; a < P; a += nt) kids[a] = 0;
+    for (int c2 = tid; c2 < 2 * P; c2 += nt) isfree[c2] = 1;
+    __syncthreads();
+    for (int m = tid; m < P; m += nt) atomicAdd(&kids[O.anc_out[m]], 1);
+    __syncthreads();
+    for (int a = tid; a < P; a += nt) if (kids[a] >= 1) isfree[now[a]] = 0;
+    for (int m = tid; m < P; m += nt) need[m] = (kids[O.anc_out[m]] != 1);
+    __syncthreads();
+    for (int pass = 0; pass < 2; ++pass) {          // exclusive prefix sums of need[P] and isfree[2P], in place
+        int *arr = pass ? isfree : need;
+        const int n = pass ? 2 * P : P;
+        if (tid == 0) carry_s = 0;
+        __syncthreads();
+        for (int base = 0; base < n; base += nt) {
+            const int x = base + tid;
+            const int flag = (x < n) ? arr[x] : 0;
+            int v = flag;
+            for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += y; }
+            if (lane == 31) rj[warp] = v;
+            __syncthreads();
+            if (warp == 0) {
+                int s2 = (lane < nwarps) ? rj[lane] : 0;
+                for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, s2, o); if (lane >= o) s2 += y; }
+                rj[lane] = s2;
+            }
+            __syncthreads();
+            const int before = (int)carry_s + (warp ? rj[warp - 1] : 0);
+            if (x < n) {
+                const int rank = before + v - flag;          // exclusive
+                if (pass) { if (flag) freelist[rank] = x; }
+                else arr[x] = flag ? rank : -1;
+            }
+            __syncthreads();
+            if (tid == nt - 1) carry_s = (u64)(before + v);
+            __syncthreads();
+        }
+    }
+    for (int m = tid; m < P; m += nt)
+        O.wloc_out[m] = (need[m] >= 0) ? freelist[need[m]] : now[O.anc_out[m]];
 }
 
 // Tail of a chain CTA: publish, take a ticket, and let the last arrival run the level barrier.
