@@ -287,6 +287,43 @@ def test_randomized_seed_population(case, width):
     rp.rp_destroy(ctx)
 
 
+def test_fuzz_random_small_windows():
+    """Random shapes and search parameters (rank counts 1..48 including non powers of two, shared
+    and interleaved shards, swap-only and relocation-only proposals, unguided and fully guided,
+    one to four attention stages, hot and cold schedules): every trajectory against the oracle."""
+    rng = np.random.default_rng(2024)
+    for trial in range(24):
+        P = int(rng.choice([1, 2, 3, 4, 6, 8, 16, 24, 32, 48]))
+        H = int(rng.choice([1, 2, 3]))
+        E = P * H
+        L = int(rng.integers(1, 7))
+        D = int(rng.choice([1, 2, 3, 4, 6]))
+        N = int(rng.integers(max(12, 4 * D), 160))
+        k = int(rng.choice([1, 2, 4]))
+        C = int(rng.choice([512, 3000, 8192]))
+        G = int(rng.integers(1, D + 1))
+        edp = None if G == D else sorted(int(x) for x in np.concatenate([np.arange(G), rng.integers(0, G, D - G)]))
+        if edp is not None and trial % 2:
+            edp = [int(x) for x in rng.permutation(edp)]
+        S = int(rng.integers(1, 5))
+        alpha = tuple(float(x) for x in np.round(rng.uniform(0, 3, S) * 256) / 256)
+        beta = tuple(float(x) for x in np.round(rng.uniform(0, 3, S) * 256) / 256)
+        pop = int(rng.choice([1, 2, 5, 9, 33]))
+        spec = custom_spec(f"fuzz{trial}", N, L, E, k, C, D, P, pop, 0, data_seed=1000 + trial, alpha=alpha, beta=beta,
+                           p_reloc=float(rng.choice([0.0, 0.25, 0.6, 1.0])), p_guide=float(rng.choice([0.0, 0.5, 0.8, 1.0])),
+                           t0=float(rng.choice([1e-5, 1e-3, 5e-2])), anneal_seed=int(rng.integers(0, 2 ** 62)))
+        w = make_window(spec)
+        min_rows = int(rng.integers(1, 4))
+        ref = oracle_front(w, edp, min_rows)
+        if ref["R"] == 0:
+            continue
+        ctx = load(w, pop=pop, edp=edp, min_rows=min_rows)
+        check_front(w, ctx, ref)
+        levels, steps = int(rng.integers(1, 5)), int(rng.choice([1, 7, 33, 130]))
+        check_anneal(w, ctx, ref, edp, pop, levels, steps, t_ratio=float(rng.choice([0.3, 0.7, 1.0])), check_members=1)
+        rp.rp_destroy(ctx)
+
+
 def test_bad_inputs_are_host_side_errors():
     w = make_window("tiny")
     s = w.spec
