@@ -65,6 +65,29 @@ extern "C" int rp_release_cached_memory(void)
     return RP_OK;
 }
 
+// Pinned staging blocks (512 bytes) for reading scalars back without a synchronous pageable copy;
+// recycled across contexts because pinning memory is slow.
+#include <mutex>
+#include <vector>
+static std::mutex g_pin_mutex;
+static std::vector<void *> g_pin_free;
+static void *pin_take()
+{
+    {
+        std::lock_guard<std::mutex> lk(g_pin_mutex);
+        if (!g_pin_free.empty()) { void *p = g_pin_free.back(); g_pin_free.pop_back(); return p; }
+    }
+    void *p = nullptr;
+    if (cudaHostAlloc(&p, 512, cudaHostAllocDefault) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    return p;
+}
+static void pin_give(void *p)
+{
+    if (!p) return;
+    std::lock_guard<std::mutex> lk(g_pin_mutex);
+    g_pin_free.push_back(p);
+}
+
 template <class T>
 static int dev_alloc(rp_ctx *c, T **p, size_t n)
 {
@@ -135,24 +158,24 @@ extern "C" void rp_destroy(rp_ctx *c)
     dev_free(c, c->d_Lagg); dev_free(c, c->d_pi); dev_free(c, c->d_inv); dev_free(c, c->d_rank_load); dev_free(c, c->d_q);
     dev_free(c, c->d_status); dev_free(c, c->d_sort_keys); dev_free(c, c->d_seed_layout); dev_free(c, c->d_order); dev_free(c, c->d_pack_out);
     dev_free(c, c->d_counters); dev_free(c, c->d_inc_layout); dev_free(c, c->d_inc_score); dev_free(c, c->d_static);
+    dev_free(c, c->d_seed_score);
+    pin_give(c->h_pin);
     free(c->h_levels); free(c->h_t);
     free(c);
 }
 
 static int reset_status(rp_ctx *c)
 {
-    int init[RP_SW_COUNT];
-    for (int x = 0; x < RP_SW_COUNT; ++x) init[x] = 0;
-    init[RP_SW_BAD_SAMPLE] = 0x7fffffff;
-    RP_CUDA(cudaMemcpyAsync(c->d_status, init, sizeof init, cudaMemcpyHostToDevice, c->stream));
-    RP_CUDA(cudaStreamSynchronize(c->stream));   // init[] is a stack array
+    RP_CUDA(cudaMemsetAsync(c->d_status, 0, sizeof(int) * RP_SW_COUNT, c->stream));
     return RP_OK;
 }
 
 static int read_status(rp_ctx *c, int out[RP_SW_COUNT])
 {
-    RP_CUDA(cudaMemcpyAsync(out, c->d_status, sizeof(int) * RP_SW_COUNT, cudaMemcpyDeviceToHost, c->stream));
+    int *stage = (int *)(c->h_pin + 56);
+    RP_CUDA(cudaMemcpyAsync(stage, c->d_status, sizeof(int) * RP_SW_COUNT, cudaMemcpyDeviceToHost, c->stream));
     RP_CUDA(cudaStreamSynchronize(c->stream));
+    memcpy(out, stage, sizeof(int) * RP_SW_COUNT);
     return RP_OK;
 }
 
@@ -204,8 +227,7 @@ static int window_load_impl(rp_ctx *c, const rp_config *cfg, const int32_t *leng
         cudaMemcpyAsync(c->d_edp, edp, sizeof(int) * D, cudaMemcpyHostToDevice, c->stream);
         cudaMemcpyAsync(c->d_dp_list, list, sizeof(int) * D, cudaMemcpyHostToDevice, c->stream);
         cudaMemcpyAsync(c->d_dp_off, off, sizeof(int) * (G + 1), cudaMemcpyHostToDevice, c->stream);
-        if (cudaStreamSynchronize(c->stream) != cudaSuccess) { st = RP_ERR_CUDA; break; }
-    } while (0);
+    } while (0);      // (copies from pageable memory are staged before the call returns)
     free(edp); free(off); free(list);
     RP_TRY(st);
 
@@ -242,13 +264,14 @@ static int window_load_impl(rp_ctx *c, const rp_config *cfg, const int32_t *leng
     RP_TRY(dev_alloc(c, &c->d_counters, 8));
     RP_TRY(dev_alloc(c, &c->d_inc_layout, N));
     RP_TRY(dev_alloc(c, &c->d_inc_score, 3));
+    RP_TRY(dev_alloc(c, &c->d_seed_score, 3));
     RP_TRY(reset_status(c));
 
     // input checks + aggregate expert load in one pass over the demand tensor
     RP_TRY(rp_launch_check_reduce(c));
     int sw[RP_SW_COUNT];
     RP_TRY(read_status(c, sw));
-    if (sw[RP_SW_BAD_SAMPLE] != 0x7fffffff) return RP_ERR_CONSERVATION;
+    if (sw[RP_SW_BAD_SAMPLE]) return RP_ERR_CONSERVATION;
 
     // fixed-point range of the score: s1 <= (2^8*C*L*k + (asum+bsum)*C) * sum t  must stay below 2^62
     double total = 0.0;
@@ -282,6 +305,8 @@ extern "C" int rp_window_load(rp_ctx **out, const rp_config *cfg, const int32_t 
     c->cfg = *cfg;
     c->cfg.edp_of_dp = nullptr; c->cfg.alpha = nullptr; c->cfg.beta = nullptr;
     c->Ppop = cfg->pop_size;
+    c->h_pin = (i64 *)pin_take();
+    if (!c->h_pin) { free(c); return RP_ERR_CUDA; }
     int st = window_load_impl(c, cfg, lengths, demand);
     if (st != RP_OK) { rp_destroy(c); return st; }
     c->stage = 1;
@@ -341,8 +366,8 @@ extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
     if (c->stage < 2) return RP_ERR_STATE;
     RpDims &dm = c->dm;
     RP_TRY(rp_launch_pack(c, 0));
-    int po[4];
-    RP_CUDA(cudaMemcpyAsync(po, c->d_pack_out, sizeof po, cudaMemcpyDeviceToHost, c->stream));
+    int *po = (int *)c->h_pin;
+    RP_CUDA(cudaMemcpyAsync(po, c->d_pack_out, sizeof(int) * 4, cudaMemcpyDeviceToHost, c->stream));
     RP_CUDA(cudaStreamSynchronize(c->stream));
     if (po[3] || po[0] <= 0) return RP_ERR_INFEASIBLE;
     c->Rstar = po[0]; c->certified = po[1];
@@ -388,8 +413,7 @@ extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
     k_iota<<<(int)((P + 255) / 256), 256, 0, c->stream>>>(c->d_wloc_next, (int)P, (int)P);
     ++g_rp_launches;
     RP_CUDA(cudaMemcpyAsync(c->d_inc_layout, c->d_seed_layout, sizeof(int) * dm.N, cudaMemcpyDeviceToDevice, c->stream));
-    RP_CUDA(cudaMemcpyAsync(c->seed_score, c->d_inc_score, sizeof(i64) * 3, cudaMemcpyDeviceToHost, c->stream));
-    RP_CUDA(cudaStreamSynchronize(c->stream));
+    RP_CUDA(cudaMemcpyAsync(c->d_seed_score, c->d_inc_score, sizeof(i64) * 3, cudaMemcpyDeviceToDevice, c->stream));
     if (n_rows) *n_rows = c->Rstar;
     if (certified) *certified = c->certified;
     c->stage = 3;
@@ -476,7 +500,7 @@ extern "C" int rp_seed_population(rp_ctx *c, int32_t choice_width, int32_t *n_ow
     cudaError_t e = cudaSuccess;
     if (st == RP_OK) {
         e = cudaMemcpyAsync(h_ok, ok, sizeof(int) * P, cudaMemcpyDeviceToHost, c->stream);
-        if (e == cudaSuccess) e = cudaMemcpyAsync(c->seed_score, best, sizeof(i64) * 3, cudaMemcpyDeviceToHost, c->stream);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(c->d_seed_score, best, sizeof(i64) * 3, cudaMemcpyDeviceToDevice, c->stream);
         if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
     }
     int own = 0;
@@ -553,21 +577,20 @@ extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *
         { int *sw = c->d_wloc; c->d_wloc = c->d_wloc_next; c->d_wloc_next = sw; }
     }
     if (stats) cudaEventRecord(ev[1], c->stream);
-    cudaError_t e = cudaStreamSynchronize(c->stream);
+    // one synchronisation: the counters and the status words ride back in the pinned block
+    i64 *cn = c->h_pin;                       // [8] counters
+    int *sw = (int *)(c->h_pin + 56);         // status words
+    cudaError_t e = cudaMemcpyAsync(cn, c->d_counters, sizeof(i64) * 8, cudaMemcpyDeviceToHost, c->stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(sw, c->d_status, sizeof(int) * RP_SW_COUNT, cudaMemcpyDeviceToHost, c->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
     if (stats) {
         if (e == cudaSuccess) cudaEventElapsedTime(&ms_chains, ev[0], ev[1]);
         for (int x = 0; x < 2; ++x) cudaEventDestroy(ev[x]);
     }
     if (st == RP_OK && e != cudaSuccess) { g_rp_last_cuda_error = (int)e; st = RP_ERR_CUDA; }
     RP_TRY(st);
-    {
-        int sw[RP_SW_COUNT];
-        RP_TRY(read_status(c, sw));
-        if (sw[RP_SW_TIMEOUT]) return RP_ERR_TIMEOUT;     // a bounded device-side wait ran out
-    }
+    if (sw[RP_SW_TIMEOUT]) return RP_ERR_TIMEOUT;         // a bounded device-side wait ran out
     if (stats) {
-        i64 cn[8];
-        RP_CUDA(cudaMemcpy(cn, c->d_counters, sizeof cn, cudaMemcpyDeviceToHost));
         stats->proposed = cn[0]; stats->feasible = cn[1]; stats->accepted = cn[2]; stats->improved = cn[3];
         stats->move_bytes = cn[4]; stats->gather_bytes = cn[5];
         stats->kernel_launches = (int64_t)NL;
@@ -588,21 +611,22 @@ extern "C" int rp_best(rp_ctx *c, int32_t *cell_of_sample, int64_t *score_fx, do
     RP_TRY(ensure_eval_scratch(c, 1, false));
     RP_TRY(rp_launch_cells_from_layouts(c, c->d_inc_layout, 1, c->d_eval_cells));
     RP_TRY(rp_launch_eval(c, c->d_eval_cells, 1, nullptr, nullptr, c->d_eval_score, c->d_eval_f64));
-    i64 inc[3], full[3];
-    int sw[RP_SW_COUNT];
-    RP_CUDA(cudaMemcpyAsync(inc, c->d_inc_score, sizeof inc, cudaMemcpyDeviceToHost, c->stream));
-    RP_CUDA(cudaMemcpyAsync(full, c->d_eval_score, sizeof full, cudaMemcpyDeviceToHost, c->stream));
-    RP_TRY(read_status(c, sw));
-    bool ok = !sw[RP_SW_VALIDATE] && !sw[RP_SW_BAD_LAYOUT];
-    ok = ok && inc[0] == full[0] && inc[1] == full[1] && inc[2] == full[2];
-    // non-regression: not worse than the best seed
-    const i64 *s = c->seed_score;
-    bool worse = (s[0] != inc[0]) ? (s[0] < inc[0]) : (s[1] != inc[1]) ? (s[1] < inc[1]) : (s[2] < inc[2]);
-    ok = ok && !worse;
+    // inc score, full rescoring, seed score and status words ride back in the pinned block
+    i64 *inc = c->h_pin, *full = c->h_pin + 3, *seed = c->h_pin + 6;
+    int *sw = (int *)(c->h_pin + 56);
+    RP_CUDA(cudaMemcpyAsync(inc, c->d_inc_score, sizeof(i64) * 3, cudaMemcpyDeviceToHost, c->stream));
+    RP_CUDA(cudaMemcpyAsync(full, c->d_eval_score, sizeof(i64) * 3, cudaMemcpyDeviceToHost, c->stream));
+    RP_CUDA(cudaMemcpyAsync(seed, c->d_seed_score, sizeof(i64) * 3, cudaMemcpyDeviceToHost, c->stream));
+    RP_CUDA(cudaMemcpyAsync(sw, c->d_status, sizeof(int) * RP_SW_COUNT, cudaMemcpyDeviceToHost, c->stream));
     RP_TRY(copy_out(c, cell_of_sample, c->d_inc_layout, sizeof(int) * (size_t)dm.N));
     RP_TRY(copy_out(c, score_fx, c->d_inc_score, sizeof(i64) * 3));
     RP_TRY(copy_out(c, score_f64, c->d_eval_f64, sizeof(double) * 3));
     RP_CUDA(cudaStreamSynchronize(c->stream));
+    bool ok = !sw[RP_SW_VALIDATE] && !sw[RP_SW_BAD_LAYOUT];
+    ok = ok && inc[0] == full[0] && inc[1] == full[1] && inc[2] == full[2];
+    // non-regression: not worse than the best member of the initial population
+    const bool worse = (seed[0] != inc[0]) ? (seed[0] < inc[0]) : (seed[1] != inc[1]) ? (seed[1] < inc[1]) : (seed[2] < inc[2]);
+    ok = ok && !worse;
     return ok ? RP_OK : RP_ERR_INVALID_PLAN;
 }
 

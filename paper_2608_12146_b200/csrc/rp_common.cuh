@@ -155,6 +155,8 @@ struct rp_ctx {
     RpLevel *h_levels;         // host copy of the per-level schedule integers
     int levels_cap;
     int *h_t;                  // host copy of the lengths (range checks)
+    i64 *h_pin;                // small pinned staging block for device->host scalars (64 x 8 bytes)
+    i64 *d_seed_score;         // [3] best score of the initial population
 };
 
 enum RpStatusWord { RP_SW_BAD_SAMPLE = 0, RP_SW_BAD_LAYOUT = 1, RP_SW_VALIDATE = 2, RP_SW_TIMEOUT = 3, RP_SW_COUNT = 8 };

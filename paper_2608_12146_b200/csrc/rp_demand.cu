@@ -42,7 +42,7 @@ k_check_reduce(const int *__restrict__ a, const int *__restrict__ t, RpDims dm, 
             for (int o = 16; o; o >>= 1) rs += __shfl_xor_sync(0xffffffffu, rs, o);
             neg = __any_sync(0xffffffffu, neg);
             bool bad = neg || rs != (i64)dm.k * ti || ti < 1 || ti > dm.C;
-            if (bad && lane == 0) atomicMin(&status[RP_SW_BAD_SAMPLE], i);
+            if (bad && lane == 0) atomicExch(&status[RP_SW_BAD_SAMPLE], 1);
         }
 #pragma unroll
         for (int c = 0; c < NC; ++c) {
