@@ -310,7 +310,7 @@ k_anneal_level(const AnnealArgs A)
         atomicAdd((u64 *)&A.counters[4], (u64)n_bytes);
         if (A.wloc_src[src] != A.wloc_dst[j]) atomicAdd((u64 *)&A.counters[5], (u64)2 * dm.RG * dm.LP * 4);
     }
-    rp_finish_level(A, tid, NT);
+    rp_finish_level(A, tid, NT, smraw, A.smem_bytes);
 }
 
 // Thread count and shared-memory plan of the chain kernels.  Windows with L*P <= 512 use the
@@ -368,6 +368,7 @@ int rp_launch_anneal_level(rp_ctx *c, int level, int n_levels, const rp_anneal_p
     int nt; size_t smem;
     rp_anneal_smem_bytes(c, &nt, &smem);
     if (smem > 220 * 1024) return RP_ERR_RANGE;
+    A.smem_bytes = (unsigned)smem;
     if (smem > 32 * 1024)
         RP_CUDA(cudaFuncSetAttribute(k_anneal_level<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     k_anneal_level<128><<<c->Ppop, 128, smem, c->stream>>>(A);

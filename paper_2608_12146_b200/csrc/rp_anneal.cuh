@@ -31,6 +31,7 @@ struct AnnealArgs {
     const int *anc;
     int level, steps, log_cap, Ppop, last;
     int w_on_chip;                   // W is staged in shared memory: every level moves it anyway
+    unsigned smem_bytes;             // dynamic shared memory of the launch
     u64 tau, cq, rho_q32, guide_q32;
     u32 key0, key1;
     i64 *term, *best;

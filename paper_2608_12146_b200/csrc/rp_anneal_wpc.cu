@@ -337,7 +337,7 @@ k_anneal_wpc(const AnnealArgs A)
         if (A.wloc_src[src] != A.wloc_dst[j]) atomicAdd((u64 *)&A.counters[5], (u64)2 * dm.RG * dm.LP * 4);
     }
     asm volatile("griddepcontrol.launch_dependents;");     // the next level may start its own prologue
-    rp_finish_level(A, tid, NT);
+    rp_finish_level(A, tid, NT, smraw, A.smem_bytes);
 }
 
 // Warps per chain: more warps score more candidates of a round at once (good when few chains
@@ -396,6 +396,7 @@ int rp_launch_anneal_wpc(rp_ctx *c, const AnnealArgs &A0)
     const size_t smem = rp_wpc_smem_bytes(dm, c->bl, c->sl, nw, &ws);
     AnnealArgs A = A0;
     A.w_on_chip = ws;
+    A.smem_bytes = (unsigned)smem;
     if (smem > 220 * 1024) return RP_ERR_RANGE;
     const int chunks = ((dm.LP >> 2) + 31) / 32;
     if (nw == 8) return launch_wpc<8>(c, A, ws, smem, chunks);

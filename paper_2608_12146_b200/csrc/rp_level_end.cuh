@@ -10,8 +10,11 @@
 // Loads of values other CTAs wrote during this launch go to L2.
 #define LE_LD(x) __ldcg(&(x))
 
-// Called by all threads of one CTA (nt a multiple of 32, at most 1024).
-__device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int nt)
+// Called by all threads of one CTA (nt a multiple of 32, at most 1024).  `ws` is the CTA's
+// dynamic shared memory, free once the chain has been stored: the cumulative weights and the
+// replayed layout live there when they fit (global memory otherwise), which keeps the
+// dependent accesses of the binary search and of the replay off the L2 round trip.
+__device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int nt, unsigned char *ws, size_t ws_bytes)
 {
     __shared__ i64 r0[LE_MAX_WARPS], r1[LE_MAX_WARPS], r2[LE_MAX_WARPS];
     __shared__ int rj[LE_MAX_WARPS];
@@ -22,6 +25,10 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
     const int lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
     const int P = A.Ppop;
     const LevelOut &O = A.lo;
+    const bool F_on_chip = (size_t)P * 8 <= ws_bytes / 2;
+    const bool lay_on_chip = (size_t)A.dm.N * 2 <= ws_bytes / 2;
+    u64 *F = F_on_chip ? (u64 *)ws : O.F;
+    unsigned short *lay_s = (unsigned short *)(ws + ws_bytes / 2);
 
     // trace copies of the per-chain reports
     if (O.tr_term) {
@@ -60,20 +67,40 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
     if (do_update) {
         const int w = win_j;
         const unsigned short *cs = (const unsigned short *)(A.blob_src + (size_t)A.anc[w] * A.bl.bytes + A.bl.off_cell);
-        for (int i = tid; i < A.dm.N; i += nt) O.inc_layout[i] = cs[i];
-        __syncthreads();
-        if (tid == 0) {      // replay the accepted moves up to the trajectory-best step
-            const uint2 *lg = A.log + (size_t)w * A.log_cap;
-            const int n = LE_LD(A.best_nlog[w]);
-            for (int x = 0; x < n; ++x) {
-                const uint2 m = LE_LD(lg[x]);
-                const int i = (int)m.x;
-                if (m.y & 0x80000000u) O.inc_layout[i] = (int)(m.y & 0x7fffffffu);
-                else {
-                    const int i2 = (int)m.y;
-                    const int c = O.inc_layout[i];
-                    O.inc_layout[i] = O.inc_layout[i2];
-                    O.inc_layout[i2] = c;
+        const uint2 *lg = A.log + (size_t)w * A.log_cap;
+        const int n = LE_LD(A.best_nlog[w]);
+        if (lay_on_chip) {
+            for (int i = tid; i < A.dm.N; i += nt) lay_s[i] = cs[i];
+            __syncthreads();
+            if (tid == 0) {      // replay the accepted moves up to the trajectory-best step
+                for (int x = 0; x < n; ++x) {
+                    const uint2 m = LE_LD(lg[x]);
+                    const int i = (int)m.x;
+                    if (m.y & 0x80000000u) lay_s[i] = (unsigned short)(m.y & 0x7fffffffu);
+                    else {
+                        const int i2 = (int)m.y;
+                        const unsigned short c = lay_s[i];
+                        lay_s[i] = lay_s[i2];
+                        lay_s[i2] = c;
+                    }
+                }
+            }
+            __syncthreads();
+            for (int i = tid; i < A.dm.N; i += nt) O.inc_layout[i] = lay_s[i];
+        } else {
+            for (int i = tid; i < A.dm.N; i += nt) O.inc_layout[i] = cs[i];
+            __syncthreads();
+            if (tid == 0) {
+                for (int x = 0; x < n; ++x) {
+                    const uint2 m = LE_LD(lg[x]);
+                    const int i = (int)m.x;
+                    if (m.y & 0x80000000u) O.inc_layout[i] = (int)(m.y & 0x7fffffffu);
+                    else {
+                        const int i2 = (int)m.y;
+                        const int c = O.inc_layout[i];
+                        O.inc_layout[i] = O.inc_layout[i2];
+                        O.inc_layout[i2] = c;
+                    }
                 }
             }
         }
@@ -128,12 +155,12 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
         }
         __syncthreads();
         const u64 before = carry_s + (warp ? rsum[warp - 1] : 0);
-        if (j < P) O.F[j] = before + v;
+        if (j < P) F[j] = before + v;
         __syncthreads();
         if (tid == nt - 1) carry_s = before + v;
         __syncthreads();
     }
-    const u64 Ftot = O.F[P - 1];
+    const u64 Ftot = F[P - 1];
     const uint4 xw = rp_philox(0u, (u32)A.level, 0u, 3u, A.key0, A.key1);
     const u64 u0 = (u64)(((unsigned __int128)xw.x * Ftot) >> 32);
     for (int m = tid; m < P; m += nt) {
@@ -141,7 +168,7 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
         int lo = 0, hi = P - 1;                 // smallest j with P*F[j] > pos
         while (lo < hi) {
             const int mid = (lo + hi) >> 1;
-            if ((unsigned __int128)P * O.F[mid] > pos) hi = mid; else lo = mid + 1;
+            if ((unsigned __int128)P * F[mid] > pos) hi = mid; else lo = mid + 1;
         }
         O.anc_out[m] = lo;
         if (O.tr_anc) O.tr_anc[(size_t)A.level * P + m] = lo;
@@ -202,7 +229,7 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
 }
 
 // Tail of a chain CTA: publish, take a ticket, and let the last arrival run the level barrier.
-__device__ __forceinline__ void rp_finish_level(const AnnealArgs &A, int tid, int nt)
+__device__ __forceinline__ void rp_finish_level(const AnnealArgs &A, int tid, int nt, unsigned char *ws, size_t ws_bytes)
 {
     __shared__ int is_last;
     __threadfence();
@@ -215,5 +242,5 @@ __device__ __forceinline__ void rp_finish_level(const AnnealArgs &A, int tid, in
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    rp_level_end(A, tid, nt);
+    rp_level_end(A, tid, nt, ws, ws_bytes);
 }
