@@ -213,6 +213,9 @@ typedef enum {
     RP_DUMP_EVAL_W = 16      /* int32 [R][G][L][P] of layout `index` of the last
                                 rp_eval_population call with explicit layouts (n <= 64)    */
 } rp_dump_what;
+/* Per-level traces (RP_DUMP_TRACE_*) are recorded by rp_anneal calls made after
+ * rp_debug_set_trace(ctx, 1); off by default (the copies cost a few microseconds per level). */
+int rp_debug_set_trace(rp_ctx *ctx, int on);
 /* Copies the named array into buf (host or device); bytes must equal its size. */
 int rp_debug_dump(rp_ctx *ctx, int what, int32_t index, void *buf, int64_t bytes);
 /* Element-wise device evaluation of the integer functions used by the accept test and the

@@ -24,6 +24,7 @@ RP_OK = 0
 
 EXPORTS = ("rp_window_load", "rp_place_experts", "rp_pack_rows", "rp_seed_population", "rp_eval_population", "rp_eval_layouts_noalloc", "rp_diagnostics", "rp_anneal",
            "rp_best", "rp_destroy", "rp_release_cached_memory", "rp_strerror", "rp_last_cuda_error", "rp_debug_dump",
+           "rp_debug_set_trace",
            "rp_debug_nl2", "rp_debug_exp2neg", "rp_debug_philox", "rp_debug_launch_count")
 
 
@@ -86,6 +87,7 @@ def lib():
         L.rp_anneal.argtypes = [C.c_void_p, C.POINTER(rp_anneal_params), C.POINTER(rp_anneal_stats)]
         L.rp_best.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.rp_debug_dump.argtypes = [C.c_void_p, C.c_int, C.c_int32, C.c_void_p, C.c_int64]
+        L.rp_debug_set_trace.argtypes = [C.c_void_p, C.c_int]
         L.rp_debug_nl2.argtypes = [C.c_void_p, C.c_void_p, C.c_int64]
         L.rp_debug_exp2neg.argtypes = [C.c_void_p, C.c_void_p, C.c_int64]
         L.rp_debug_philox.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64]
@@ -248,6 +250,10 @@ def rp_release_cached_memory():
 DUMP = dict(LAGG=1, Q=2, SEED_LAYOUT=3, POPULATION=4, W=5, CELL_T=6, CELL_Q=7, CELL_CNT=8, ESUM=9,
             TRACE_TERM=10, TRACE_BEST=11, TRACE_BEST_STEP=12, TRACE_DIGEST=13, TRACE_ANC=14,
             TRACE_INCUMBENT=15, EVAL_W=16)
+
+
+def rp_debug_set_trace(ctx: Context, on: bool = True):
+    _check(lib().rp_debug_set_trace(ctx.handle, int(on)), "rp_debug_set_trace")
 
 
 def rp_debug_dump(ctx: Context, what: str, shape, dtype, index: int = 0) -> np.ndarray:

@@ -553,15 +553,17 @@ extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *
         RP_TRY(dev_alloc(c, &c->d_log, P * (size_t)p->steps_per_level));
         c->log_cap = p->steps_per_level;
     }
-    // trace
+    // per-level trace (only when the inspection hook asked for it)
     free_trace(c);
-    RP_TRY(dev_alloc(c, &c->d_tr_term, (size_t)NL * P * 3));
-    RP_TRY(dev_alloc(c, &c->d_tr_best, (size_t)NL * P * 3));
-    RP_TRY(dev_alloc(c, &c->d_tr_inc, (size_t)NL * 3));
-    RP_TRY(dev_alloc(c, &c->d_tr_best_step, (size_t)NL * P));
-    RP_TRY(dev_alloc(c, &c->d_tr_digest, (size_t)NL * P));
-    RP_TRY(dev_alloc(c, &c->d_tr_anc, (size_t)(NL > 1 ? NL - 1 : 1) * P));
-    c->trace_levels = NL;
+    if (c->trace_on) {
+        RP_TRY(dev_alloc(c, &c->d_tr_term, (size_t)NL * P * 3));
+        RP_TRY(dev_alloc(c, &c->d_tr_best, (size_t)NL * P * 3));
+        RP_TRY(dev_alloc(c, &c->d_tr_inc, (size_t)NL * 3));
+        RP_TRY(dev_alloc(c, &c->d_tr_best_step, (size_t)NL * P));
+        RP_TRY(dev_alloc(c, &c->d_tr_digest, (size_t)NL * P));
+        RP_TRY(dev_alloc(c, &c->d_tr_anc, (size_t)(NL > 1 ? NL - 1 : 1) * P));
+        c->trace_levels = NL;
+    }
     RP_CUDA(cudaMemsetAsync(c->d_counters, 0, sizeof(i64) * 8, c->stream));
     RP_TRY(reset_status(c));
 
@@ -644,6 +646,13 @@ __global__ void k_cell_stats(const unsigned short *__restrict__ cells, const int
         atomicAdd((u64 *)&Q[c], (u64)t[i] * (u64)t[i]);
         atomicAdd(&cnt[c], 1);
     }
+}
+
+extern "C" int rp_debug_set_trace(rp_ctx *c, int on)
+{
+    if (!c) return RP_ERR_ARG;
+    c->trace_on = on ? 1 : 0;
+    return RP_OK;
 }
 
 extern "C" int rp_debug_dump(rp_ctx *c, int what, int32_t index, void *buf, int64_t bytes)

@@ -140,6 +140,7 @@ struct rp_ctx {
     i64 *d_inc_score;          // [3]
     // trace of the last rp_anneal call
     int trace_levels;
+    int trace_on;              // keep per-level traces (inspection hook; off by default)
     i64 *d_tr_term, *d_tr_best, *d_tr_inc;
     int *d_tr_best_step, *d_tr_anc;
     u64 *d_tr_digest;

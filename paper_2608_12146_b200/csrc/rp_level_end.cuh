@@ -38,12 +38,15 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
     }
 
     // ---- incumbent: lexicographic argmin of the trajectory-best scores, lowest slot first ----
-    i64 b0 = 0x7fffffffffffffffll, b1 = b0, b2 = b0;
+    // Only chains that beat the incumbent matter; late in the schedule there are usually none.
+    const i64 i0 = O.inc_score[0], i1 = O.inc_score[1], i2 = O.inc_score[2];
+    i64 b0 = i0, b1 = i1, b2 = i2;
     int bj = 0x7fffffff;
     for (int j = tid; j < P; j += nt) {
         i64 s0 = LE_LD(A.best[3 * (size_t)j]), s1 = LE_LD(A.best[3 * (size_t)j + 1]), s2 = LE_LD(A.best[3 * (size_t)j + 2]);
         if (rp_lex_less(s0, s1, s2, b0, b1, b2)) { b0 = s0; b1 = s1; b2 = s2; bj = j; }   // ascending j: first wins
     }
+    if (__syncthreads_or(bj != 0x7fffffff)) {
     for (int o = 16; o; o >>= 1) {
         i64 o0 = __shfl_xor_sync(0xffffffffu, b0, o), o1 = __shfl_xor_sync(0xffffffffu, b1, o);
         i64 o2 = __shfl_xor_sync(0xffffffffu, b2, o);
@@ -60,7 +63,7 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
             if (take) { b0 = r0[w]; b1 = r1[w]; b2 = r2[w]; bj = rj[w]; }
         }
         win_j = bj;
-        do_update = rp_lex_less(b0, b1, b2, O.inc_score[0], O.inc_score[1], O.inc_score[2]);
+        do_update = rp_lex_less(b0, b1, b2, i0, i1, i2);
         if (do_update) { O.inc_score[0] = b0; O.inc_score[1] = b1; O.inc_score[2] = b2; }
     }
     __syncthreads();
@@ -105,6 +108,7 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
             }
         }
     }
+    }     // some chain beat the incumbent
     __syncthreads();
     if (O.tr_inc && tid < 3) O.tr_inc[(size_t)A.level * 3 + tid] = O.inc_score[tid];
 
@@ -136,13 +140,28 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
         u64 w = 0;
         if (j < P) {
             const i64 e = rp_energy(LE_LD(A.term[3 * (size_t)j]), LE_LD(A.term[3 * (size_t)j + 1]), LE_LD(A.term[3 * (size_t)j + 2]));
-            unsigned __int128 eq = ((unsigned __int128)(u64)(e - emin) << 32) / (unsigned __int128)M;
-            const unsigned __int128 cap = (((unsigned __int128)1) << 48) - 1;
-            if (eq > cap) eq = cap;
-            unsigned __int128 z = (eq * (unsigned __int128)A.cq) >> 16;
-            const unsigned __int128 zcap = ((unsigned __int128)1) << 40;
-            if (z > zcap) z = zcap;
-            w = rp_exp2neg((u64)z);
+            // eq = min(2^48 - 1, floor((e - emin) * 2^32 / M)): a 64-bit quotient for the integer part
+            // and 32 restoring steps for the fraction (M < 2^63, so the shifted remainder fits)
+            const u64 Dd = (u64)(e - emin);
+            u64 eq;
+            if ((Dd >> 16) >= M) eq = (1ull << 48) - 1;
+            else {
+                u64 q = Dd / M, r = Dd - q * M;
+                u32 fr = 0;
+#pragma unroll 4
+                for (int it = 0; it < 32; ++it) {
+                    r <<= 1;
+                    const bool ge = r >= M;
+                    r -= ge ? M : 0;
+                    fr = (fr << 1) | (ge ? 1u : 0u);
+                }
+                eq = (q << 32) | fr;
+            }
+            // z = min(2^40, (eq * cq) >> 16) with a 128-bit product
+            const u64 zh = __umul64hi(eq, A.cq), zl = eq * A.cq;
+            u64 z = (zh >> 16) ? (1ull << 40) : ((zh << 48) | (zl >> 16));
+            if (z > (1ull << 40)) z = 1ull << 40;
+            w = rp_exp2neg(z);
         }
         u64 v = w;
         for (int o = 1; o < 32; o <<= 1) { u64 x = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += x; }

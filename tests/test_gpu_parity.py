@@ -21,9 +21,11 @@ def load(w, pop=None, edp=None, min_rows=0, device_inputs=False):
     if device_inputs:
         import torch
         t, a = torch.from_numpy(t).cuda(), torch.from_numpy(a).cuda()
-    return rp.rp_window_load(t, a, top_k=s.top_k, token_cap=s.token_cap, dp_width=s.dp_width,
-                             ep_width=s.ep_width, pop_size=pop or s.pop_size, edp_of_dp=edp,
-                             alpha=s.alpha, beta=s.beta, min_rows=min_rows, seed=s.anneal_seed)
+    ctx = rp.rp_window_load(t, a, top_k=s.top_k, token_cap=s.token_cap, dp_width=s.dp_width,
+                            ep_width=s.ep_width, pop_size=pop or s.pop_size, edp_of_dp=edp,
+                            alpha=s.alpha, beta=s.beta, min_rows=min_rows, seed=s.anneal_seed)
+    rp.rp_debug_set_trace(ctx, True)          # the parity checks read the per-level traces
+    return ctx
 
 
 def oracle_front(w, edp=None, min_rows=0):
@@ -399,6 +401,7 @@ def test_smallest_window_and_empty_moves():
     R, cert, seed = oracle.pack_ffd(t, 16, 4)
     assert R == 1
     ctx = rp.rp_window_load(t, a, top_k=2, token_cap=16, dp_width=4, ep_width=2, pop_size=3, seed=11)
+    rp.rp_debug_set_trace(ctx, True)
     rp.rp_place_experts(ctx)
     assert rp.rp_pack_rows(ctx) == (R, cert)
     want = oracle.anneal(t, q, np.tile(seed, (3, 1)), R, 16, 4, n_levels=4, steps=30, t0=1e-2, t_ratio=0.5,
