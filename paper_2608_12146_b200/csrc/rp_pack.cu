@@ -9,6 +9,64 @@
 
 #define PACK_THREADS 1024
 
+// First fit of the samples keys[K..N) into K cells by one warp; lane `tid` owns cells
+// [tid*B, tid*B+B).  Returns true when some sample fits nowhere.  BR >= B cells per lane are
+// kept in registers (statically indexed); the shared-memory variant handles any B.
+template <int BR>
+__device__ __forceinline__ bool first_fit_regs(const RpDims &dm, const u64 *keys, int *fill, int *cell_of, int K, int B, int tid)
+{
+    const int b0 = tid * B;
+    int rem[BR];
+    int blockmax = -1;
+#pragma unroll
+    for (int u = 0; u < BR; ++u) {
+        rem[u] = (u < B && b0 + u < K) ? dm.C - fill[b0 + u] : -1;
+        blockmax = max(blockmax, rem[u]);
+    }
+    for (int x = K; x < dm.N; ++x) {
+        const u64 key = keys[x];
+        const int ts = dm.C - (int)(key >> 32);
+        const unsigned m = __ballot_sync(0xffffffffu, blockmax >= ts);
+        if (!m) return true;
+        if (tid == __ffs(m) - 1) {
+            int found = -1, nm = -1;
+#pragma unroll
+            for (int u = 0; u < BR; ++u) {
+                const bool take = (found < 0) && (rem[u] >= ts);
+                if (take) { found = b0 + u; rem[u] -= ts; }
+                nm = max(nm, rem[u]);
+            }
+            blockmax = nm;
+            cell_of[(u32)key] = found;
+        }
+    }
+    return false;
+}
+
+__device__ __forceinline__ bool first_fit_smem(const RpDims &dm, const u64 *keys, int *fill, int *cell_of, int K, int B, int tid)
+{
+    const int b0 = tid * B, b1 = min(K, b0 + B);
+    int blockmax = -1;
+    for (int b = b0; b < b1; ++b) blockmax = max(blockmax, dm.C - fill[b]);
+    for (int x = K; x < dm.N; ++x) {
+        const u64 key = keys[x];
+        const int ts = dm.C - (int)(key >> 32);
+        const unsigned m = __ballot_sync(0xffffffffu, blockmax >= ts);
+        if (!m) return true;
+        if (tid == __ffs(m) - 1) {
+            int found = -1, nm = -1;
+            for (int b = b0; b < b1; ++b) {
+                int rem = dm.C - fill[b];
+                if (found < 0 && rem >= ts) { found = b; rem -= ts; fill[b] += ts; }
+                nm = max(nm, rem);
+            }
+            blockmax = nm;
+            cell_of[(u32)key] = found;
+        }
+    }
+    return false;
+}
+
 __global__ void __launch_bounds__(PACK_THREADS)
 k_pack_ffd(RpDims dm, const int *__restrict__ t, int min_rows, u64 *__restrict__ keys_g, int n_pow2,
            int *__restrict__ fill_g, int *__restrict__ cell_of, int *__restrict__ out, int *__restrict__ order_out)
@@ -65,27 +123,14 @@ k_pack_ffd(RpDims dm, const int *__restrict__ t, int min_rows, u64 *__restrict__
             // First fit = the lowest cell whose remaining capacity takes the sample.  Each lane
             // owns a block of B consecutive cells and keeps the largest remaining capacity of its
             // block in a register: one ballot finds the lowest lane that can take the sample, and
-            // only that lane scans its block.
+            // only that lane scans its block (held in registers when B <= 16).
             const int B = (K + 31) / 32;
-            const int b0 = tid * B, b1 = min(K, b0 + B);
-            int blockmax = -1;
-            for (int b = b0; b < b1; ++b) blockmax = max(blockmax, dm.C - fill[b]);
-            for (int x = K; x < dm.N; ++x) {
-                const u64 key = keys[x];
-                const int ts = dm.C - (int)(key >> 32);
-                const unsigned m = __ballot_sync(0xffffffffu, blockmax >= ts);
-                if (!m) { if (tid == 0) fail_s = 1; break; }
-                if (tid == __ffs(m) - 1) {
-                    int found = -1, nm = -1;
-                    for (int b = b0; b < b1; ++b) {
-                        int rem = dm.C - fill[b];
-                        if (found < 0 && rem >= ts) { found = b; rem -= ts; fill[b] += ts; }
-                        nm = max(nm, rem);
-                    }
-                    blockmax = nm;
-                    cell_of[(u32)key] = found;
-                }
-            }
+            bool failed;
+            if (B <= 4) failed = first_fit_regs<4>(dm, keys, fill, cell_of, K, B, tid);
+            else if (B <= 8) failed = first_fit_regs<8>(dm, keys, fill, cell_of, K, B, tid);
+            else if (B <= 16) failed = first_fit_regs<16>(dm, keys, fill, cell_of, K, B, tid);
+            else failed = first_fit_smem(dm, keys, fill, cell_of, K, B, tid);
+            if (failed && tid == 0) fail_s = 1;
         }
         __syncthreads();
         if (!fail_s) Rstar = (int)R;
