@@ -86,6 +86,8 @@ k_anneal_level(const AnnealArgs A)
 
     if (tid == 0) chain->failed = 0;
     const bool landed = rp_chain_load<NT, false>(A, src, j, sm_blob, sm_static, nullptr, mbar, tid);
+    if (tid == 0 && A.wloc_src[src] != A.wloc_dst[j])      // bytes of the W gather (counted here: off the level's tail)
+        atomicAdd((u64 *)&A.counters[5], (u64)2 * dm.RG * dm.LP * 4);
     if (!landed) chain->failed = 1;
     __syncthreads();
     if (chain->failed) {
@@ -308,7 +310,6 @@ k_anneal_level(const AnnealArgs A)
         atomicAdd((u64 *)&A.counters[2], (u64)n_acc);
         atomicAdd((u64 *)&A.counters[3], (u64)n_imp);
         atomicAdd((u64 *)&A.counters[4], (u64)n_bytes);
-        if (A.wloc_src[src] != A.wloc_dst[j]) atomicAdd((u64 *)&A.counters[5], (u64)2 * dm.RG * dm.LP * 4);
     }
     rp_finish_level(A, tid, NT, smraw, A.smem_bytes);
 }

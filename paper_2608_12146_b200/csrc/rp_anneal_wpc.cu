@@ -84,6 +84,8 @@ k_anneal_wpc(const AnnealArgs A)
     // ---- prologue: adopt the ancestor's terminal state -------------------------------
     if (tid == 0) chain->failed = 0;
     const bool landed = rp_chain_load<NT, WS>(A, src, j, sm_blob, sm_static, Wsm, mbar, tid);
+    if (tid == 0 && A.wloc_src[src] != A.wloc_dst[j])      // bytes of the W gather (counted here: off the level's tail)
+        atomicAdd((u64 *)&A.counters[5], (u64)2 * dm.RG * dm.LP * 4);
     if (!landed) chain->failed = 1;
     __syncthreads();
     if (chain->failed) {                 // a bulk copy never landed: report and leave
@@ -334,7 +336,6 @@ k_anneal_wpc(const AnnealArgs A)
         A.best_nlog[j] = chain->best_nlog;
         A.digest[j] = chain->dig;
         atomicAdd((u64 *)&A.counters[0], (u64)A.steps);
-        if (A.wloc_src[src] != A.wloc_dst[j]) atomicAdd((u64 *)&A.counters[5], (u64)2 * dm.RG * dm.LP * 4);
     }
     asm volatile("griddepcontrol.launch_dependents;");     // the next level may start its own prologue
     rp_finish_level(A, tid, NT, smraw, A.smem_bytes);

@@ -10,6 +10,92 @@
 // Loads of values other CTAs wrote during this launch go to L2.
 #define LE_LD(x) __ldcg(&(x))
 
+// min(2^48 - 1, floor(Dd * 2^32 / M)) for 0 < M < 2^63.  A double-precision estimate is within
+// one of the quotient (it is below 2^48 and the estimate's relative error below 2^-50); the exact
+// 128-bit remainder then corrects it, so the result is the exact floor.
+__device__ __forceinline__ u64 le_scaled_quotient(u64 Dd, u64 M)
+{
+    if ((Dd >> 16) >= M) return (1ull << 48) - 1;
+    u64 q = (u64)(((double)Dd * 4294967296.0) / (double)M);
+    const u64 ph = __umul64hi(q, M), pl = q * M;
+    const u64 nh = Dd >> 32, nl = Dd << 32;
+    u64 rl = nl - pl, rh = nh - ph - (nl < pl ? 1ull : 0ull);        // remainder, signed 128-bit
+    for (int it = 0; it < 4 && (i64)rh < 0; ++it) { --q; const u64 t = rl + M; rh += (t < rl) ? 1ull : 0ull; rl = t; }
+    for (int it = 0; it < 4 && (rh != 0 || rl >= M); ++it) { ++q; rh -= (rl < M) ? 1ull : 0ull; rl -= M; }
+    return q;
+}
+
+// Boltzmann weights of U members at once (independent dependency chains interleave):
+// w = exp2neg(min(2^40, (eq * cq) >> 16)), eq the scaled energy gap above.
+template <int U>
+__device__ __forceinline__ void le_weights(const i64 (&e)[U], i64 emin, u64 M, u64 cq, u64 (&w)[U])
+{
+    u64 z[U], acc[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const u64 eq = le_scaled_quotient((u64)(e[u] - emin), M);
+        const u64 zh = __umul64hi(eq, cq), zl = eq * cq;
+        u64 zz = (zh >> 16) ? (1ull << 40) : ((zh << 48) | (zl >> 16));
+        z[u] = zz > (1ull << 40) ? (1ull << 40) : zz;
+        acc[u] = 1ull << 63;
+    }
+    // the fraction bits in the order of rp_exp2neg; a clear bit multiplies by one (2^63 in Q63), which is exact
+#pragma unroll 1
+    for (int i = 1; i <= 24; ++i) {
+        const u64 c = RP_EXP2_Q63[i - 1];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const u64 cc = ((z[u] >> (32 - i)) & 1ull) ? c : (1ull << 63);
+            acc[u] = (__umul64hi(acc[u], cc) << 1) | ((acc[u] * cc) >> 63);
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const u64 ip = z[u] >> 32;
+        w[u] = ip >= 32 ? 0 : (acc[u] >> 31) >> ip;
+    }
+}
+
+// Inclusive prefix sums F[j] of the weights, U consecutive members per thread and round.
+template <int U>
+__device__ __forceinline__ void le_prefix_weights(const AnnealArgs &A, int tid, int nt, i64 emin, u64 M, u64 *F,
+                                                  u64 *rsum, u64 *carry_s)
+{
+    const int lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
+    const int P = A.Ppop;
+    for (int base = 0; base < P; base += nt * U) {
+        const int j0 = base + tid * U;
+        i64 e[U];
+        u64 w[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int j = j0 + u;
+            e[u] = (j < P) ? rp_energy(LE_LD(A.term[3 * (size_t)j]), LE_LD(A.term[3 * (size_t)j + 1]), LE_LD(A.term[3 * (size_t)j + 2]))
+                           : emin;
+        }
+        le_weights<U>(e, emin, M, A.cq, w);
+        u64 v = 0;
+#pragma unroll
+        for (int u = 0; u < U; ++u) { if (j0 + u >= P) w[u] = 0; v += w[u]; w[u] = v; }     // thread-local inclusive sums
+        for (int o = 1; o < 32; o <<= 1) { u64 x = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += x; }
+        if (lane == 31) rsum[warp] = v;
+        __syncthreads();
+        if (warp == 0) {
+            u64 s2 = (lane < nwarps) ? rsum[lane] : 0;
+            for (int o = 1; o < 32; o <<= 1) { u64 x = __shfl_up_sync(0xffffffffu, s2, o); if (lane >= o) s2 += x; }
+            rsum[lane] = s2;
+        }
+        __syncthreads();
+        const u64 upto = *carry_s + (warp ? rsum[warp - 1] : 0) + v;       // through this thread's last member
+        const u64 mine = w[U - 1];
+#pragma unroll
+        for (int u = 0; u < U; ++u) if (j0 + u < P) F[j0 + u] = upto - mine + w[u];
+        __syncthreads();
+        if (tid == nt - 1) *carry_s = upto;
+        __syncthreads();
+    }
+}
+
 // Called by all threads of one CTA (nt a multiple of 32, at most 1024).  `ws` is the CTA's
 // dynamic shared memory, free once the chain has been stored: the cumulative weights and the
 // replayed layout live there when they fit (global memory otherwise), which keeps the
@@ -17,10 +103,10 @@
 __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int nt, unsigned char *ws, size_t ws_bytes)
 {
     __shared__ i64 r0[LE_MAX_WARPS], r1[LE_MAX_WARPS], r2[LE_MAX_WARPS];
-    __shared__ int rj[LE_MAX_WARPS];
+    __shared__ int rj[LE_MAX_WARPS], rn[LE_MAX_WARPS], ra[LE_MAX_WARPS];
     __shared__ u64 rsum[LE_MAX_WARPS];
-    __shared__ int win_j, do_update;
-    __shared__ i64 Emin_s;
+    __shared__ int win_j, win_n, win_a, do_update;
+    __shared__ i64 rmin[LE_MAX_WARPS];
     __shared__ u64 carry_s;
     const int lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
     const int P = A.Ppop;
@@ -41,43 +127,58 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
     // Only chains that beat the incumbent matter; late in the schedule there are usually none.
     const i64 i0 = O.inc_score[0], i1 = O.inc_score[1], i2 = O.inc_score[2];
     i64 b0 = i0, b1 = i1, b2 = i2;
-    int bj = 0x7fffffff;
+    int bj = 0x7fffffff, bn = 0, ba = 0;
+    i64 emin = 0x7fffffffffffffffll;         // smallest terminal energy, for the weights further down
+#pragma unroll 2
     for (int j = tid; j < P; j += nt) {
-        i64 s0 = LE_LD(A.best[3 * (size_t)j]), s1 = LE_LD(A.best[3 * (size_t)j + 1]), s2 = LE_LD(A.best[3 * (size_t)j + 2]);
-        if (rp_lex_less(s0, s1, s2, b0, b1, b2)) { b0 = s0; b1 = s1; b2 = s2; bj = j; }   // ascending j: first wins
+        const i64 s0 = LE_LD(A.best[3 * (size_t)j]), s1 = LE_LD(A.best[3 * (size_t)j + 1]), s2 = LE_LD(A.best[3 * (size_t)j + 2]);
+        const i64 t0 = LE_LD(A.term[3 * (size_t)j]), t1 = LE_LD(A.term[3 * (size_t)j + 1]), t2 = LE_LD(A.term[3 * (size_t)j + 2]);
+        if (rp_lex_less(s0, s1, s2, b0, b1, b2)) {    // ascending j: first wins
+            b0 = s0; b1 = s1; b2 = s2; bj = j;
+            bn = LE_LD(A.best_nlog[j]); ba = A.anc[j];       // what the replay needs, fetched with the rest
+        }
+        const i64 e = rp_energy(t0, t1, t2);
+        emin = e < emin ? e : emin;
     }
+    for (int o = 16; o; o >>= 1) { const i64 x = __shfl_xor_sync(0xffffffffu, emin, o); emin = x < emin ? x : emin; }
+    if (lane == 0) rmin[warp] = emin;
     if (__syncthreads_or(bj != 0x7fffffff)) {
     for (int o = 16; o; o >>= 1) {
         i64 o0 = __shfl_xor_sync(0xffffffffu, b0, o), o1 = __shfl_xor_sync(0xffffffffu, b1, o);
         i64 o2 = __shfl_xor_sync(0xffffffffu, b2, o);
         int oj = __shfl_xor_sync(0xffffffffu, bj, o);
+        const int on = __shfl_xor_sync(0xffffffffu, bn, o), oa = __shfl_xor_sync(0xffffffffu, ba, o);
         bool take = rp_lex_less(o0, o1, o2, b0, b1, b2) || (o0 == b0 && o1 == b1 && o2 == b2 && oj < bj);
-        if (take) { b0 = o0; b1 = o1; b2 = o2; bj = oj; }
+        if (take) { b0 = o0; b1 = o1; b2 = o2; bj = oj; bn = on; ba = oa; }
     }
-    if (lane == 0) { r0[warp] = b0; r1[warp] = b1; r2[warp] = b2; rj[warp] = bj; }
+    if (lane == 0) { r0[warp] = b0; r1[warp] = b1; r2[warp] = b2; rj[warp] = bj; rn[warp] = bn; ra[warp] = ba; }
     __syncthreads();
     if (tid == 0) {
         for (int w = 1; w < nwarps; ++w) {
             bool take = rp_lex_less(r0[w], r1[w], r2[w], b0, b1, b2) ||
                         (r0[w] == b0 && r1[w] == b1 && r2[w] == b2 && rj[w] < bj);
-            if (take) { b0 = r0[w]; b1 = r1[w]; b2 = r2[w]; bj = rj[w]; }
+            if (take) { b0 = r0[w]; b1 = r1[w]; b2 = r2[w]; bj = rj[w]; bn = rn[w]; ba = ra[w]; }
         }
-        win_j = bj;
+        win_j = bj; win_n = bn; win_a = ba;
         do_update = rp_lex_less(b0, b1, b2, i0, i1, i2);
         if (do_update) { O.inc_score[0] = b0; O.inc_score[1] = b1; O.inc_score[2] = b2; }
     }
     __syncthreads();
     if (do_update) {
         const int w = win_j;
-        const unsigned short *cs = (const unsigned short *)(A.blob_src + (size_t)A.anc[w] * A.bl.bytes + A.bl.off_cell);
+        const unsigned short *cs = (const unsigned short *)(A.blob_src + (size_t)win_a * A.bl.bytes + A.bl.off_cell);
         const uint2 *lg = A.log + (size_t)w * A.log_cap;
-        const int n = LE_LD(A.best_nlog[w]);
+        const int n = win_n;
         if (lay_on_chip) {
+            // the log goes through the other half of the workspace when it fits (no dependent L2 round trips)
+            uint2 *lg_s = (uint2 *)ws;
+            const bool log_on_chip = (size_t)n * sizeof(uint2) <= ws_bytes / 2;
             for (int i = tid; i < A.dm.N; i += nt) lay_s[i] = cs[i];
+            if (log_on_chip) for (int x = tid; x < n; x += nt) lg_s[x] = LE_LD(lg[x]);
             __syncthreads();
             if (tid == 0) {      // replay the accepted moves up to the trajectory-best step
                 for (int x = 0; x < n; ++x) {
-                    const uint2 m = LE_LD(lg[x]);
+                    const uint2 m = log_on_chip ? lg_s[x] : LE_LD(lg[x]);
                     const int i = (int)m.x;
                     if (m.y & 0x80000000u) lay_s[i] = (unsigned short)(m.y & 0x7fffffffu);
                     else {
@@ -118,79 +219,45 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
     }
 
     // ---- resampling -------------------------------------------------------------------------
-    i64 emin = 0x7fffffffffffffffll;
-    for (int j = tid; j < P; j += nt) {
-        i64 e = rp_energy(LE_LD(A.term[3 * (size_t)j]), LE_LD(A.term[3 * (size_t)j + 1]), LE_LD(A.term[3 * (size_t)j + 2]));
-        emin = e < emin ? e : emin;
-    }
-    for (int o = 16; o; o >>= 1) { i64 x = __shfl_xor_sync(0xffffffffu, emin, o); emin = x < emin ? x : emin; }
-    if (lane == 0) r0[warp] = emin;
+    for (int w = 0; w < nwarps; ++w) emin = rmin[w] < emin ? rmin[w] : emin;
+    if (tid == 0) carry_s = 0;
     __syncthreads();
-    if (tid == 0) {
-        for (int w = 1; w < nwarps; ++w) emin = r0[w] < emin ? r0[w] : emin;
-        Emin_s = emin;
-        carry_s = 0;
-    }
-    __syncthreads();
-    emin = Emin_s;
     const u64 M = (u64)(emin > A.dm.SC ? emin : A.dm.SC);
-    // inclusive prefix sums of the weights, nt members per round
-    for (int base = 0; base < P; base += nt) {
-        const int j = base + tid;
-        u64 w = 0;
-        if (j < P) {
-            const i64 e = rp_energy(LE_LD(A.term[3 * (size_t)j]), LE_LD(A.term[3 * (size_t)j + 1]), LE_LD(A.term[3 * (size_t)j + 2]));
-            // eq = min(2^48 - 1, floor((e - emin) * 2^32 / M)): a 64-bit quotient for the integer part
-            // and 32 restoring steps for the fraction (M < 2^63, so the shifted remainder fits)
-            const u64 Dd = (u64)(e - emin);
-            u64 eq;
-            if ((Dd >> 16) >= M) eq = (1ull << 48) - 1;
-            else {
-                u64 q = Dd / M, r = Dd - q * M;
-                u32 fr = 0;
-#pragma unroll 4
-                for (int it = 0; it < 32; ++it) {
-                    r <<= 1;
-                    const bool ge = r >= M;
-                    r -= ge ? M : 0;
-                    fr = (fr << 1) | (ge ? 1u : 0u);
-                }
-                eq = (q << 32) | fr;
-            }
-            // z = min(2^40, (eq * cq) >> 16) with a 128-bit product
-            const u64 zh = __umul64hi(eq, A.cq), zl = eq * A.cq;
-            u64 z = (zh >> 16) ? (1ull << 40) : ((zh << 48) | (zl >> 16));
-            if (z > (1ull << 40)) z = 1ull << 40;
-            w = rp_exp2neg(z);
-        }
-        u64 v = w;
-        for (int o = 1; o < 32; o <<= 1) { u64 x = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += x; }
-        if (lane == 31) rsum[warp] = v;
-        __syncthreads();
-        if (warp == 0) {
-            u64 s = (lane < nwarps) ? rsum[lane] : 0;
-            for (int o = 1; o < 32; o <<= 1) { u64 x = __shfl_up_sync(0xffffffffu, s, o); if (lane >= o) s += x; }
-            rsum[lane] = s;
-        }
-        __syncthreads();
-        const u64 before = carry_s + (warp ? rsum[warp - 1] : 0);
-        if (j < P) F[j] = before + v;
-        __syncthreads();
-        if (tid == nt - 1) carry_s = before + v;
-        __syncthreads();
-    }
+    if (P <= nt) le_prefix_weights<1>(A, tid, nt, emin, M, F, rsum, &carry_s);
+    else if (P <= 2 * nt) le_prefix_weights<2>(A, tid, nt, emin, M, F, rsum, &carry_s);
+    else le_prefix_weights<4>(A, tid, nt, emin, M, F, rsum, &carry_s);
     const u64 Ftot = F[P - 1];
     const uint4 xw = rp_philox(0u, (u32)A.level, 0u, 3u, A.key0, A.key1);
     const u64 u0 = (u64)(((unsigned __int128)xw.x * Ftot) >> 32);
-    for (int m = tid; m < P; m += nt) {
-        const unsigned __int128 pos = (unsigned __int128)u0 + (unsigned __int128)m * Ftot;
-        int lo = 0, hi = P - 1;                 // smallest j with P*F[j] > pos
-        while (lo < hi) {
-            const int mid = (lo + hi) >> 1;
-            if ((unsigned __int128)P * F[mid] > pos) hi = mid; else lo = mid + 1;
+    int depth = 0;
+    while ((1 << depth) < P) ++depth;
+    constexpr int SU = 4;                       // searches per thread in flight
+    for (int base = 0; base < P; base += nt * SU) {
+        unsigned __int128 pos[SU];
+        int lo[SU], hi[SU];
+#pragma unroll
+        for (int u = 0; u < SU; ++u) {
+            const int m = base + u * nt + tid;
+            pos[u] = (unsigned __int128)u0 + (unsigned __int128)(m < P ? m : 0) * Ftot;
+            lo[u] = 0; hi[u] = (m < P) ? P - 1 : 0;      // smallest j with P*F[j] > pos (nothing to search past the end)
         }
-        O.anc_out[m] = lo;
-        if (O.tr_anc) O.tr_anc[(size_t)A.level * P + m] = lo;
+        for (int it = 0; it < depth; ++it) {
+#pragma unroll
+            for (int u = 0; u < SU; ++u) {
+                if (lo[u] < hi[u]) {
+                    const int mid = (lo[u] + hi[u]) >> 1;
+                    if ((unsigned __int128)P * F[mid] > pos[u]) hi[u] = mid; else lo[u] = mid + 1;
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < SU; ++u) {
+            const int m = base + u * nt + tid;
+            if (m < P) {
+                O.anc_out[m] = lo[u];
+                if (O.tr_anc) O.tr_anc[(size_t)A.level * P + m] = lo[u];
+            }
+        }
     }
     __syncthreads();
 
