@@ -18,6 +18,13 @@
 
 #include "rp_level_end.cuh"
 
+struct CandS {                  // a feasible proposal and the cell statistics it would leave behind
+    MoveS m;
+    int pad;
+    i64 Ta, Qa, Tb, Qb;         // token count and sum of squares of the source and target cells after the move
+    i64 A1, A2;                 // their attention terms (identity shard map only)
+};
+
 struct ChainS {                 // bookkeeping of the chain within this level
     i64 B[3];                   // trajectory-best score
     u64 dig;                    // digest of the accepted moves
@@ -43,8 +50,8 @@ k_anneal_wpc(const AnnealArgs A)
     StepRec *recs = (StepRec *)(Acell + dm.K);
     ChainS *chain = (ChainS *)(recs + NT);
     u64 *mbar = (u64 *)(chain + 1);
-    MoveS *mvs = (MoveS *)(mbar + 1);
-    int *vote = (int *)(mvs + SPEC);                                    // [NW] accept flags of a wave
+    CandS *cand = (CandS *)(mbar + 1);
+    int *vote = (int *)(cand + SPEC);                                    // [NW] accept flags of a wave
     int *rnd = vote + NW;                                               // [0] feasible mask, [1] next position
 
     u64 *Q = (u64 *)(sm_blob + A.bl.off_Q);
@@ -106,6 +113,7 @@ k_anneal_wpc(const AnnealArgs A)
     uint2 *logj = A.log + (size_t)j * A.log_cap;
     const RpChainView view = { cell_of, T, cnt, tt, attkey, Jcell, Acell };
     int *my_s1 = scratch + (size_t)warp * 2 * slice_pad, *my_s2 = my_s1 + slice_pad;
+    int proposer = 0;                                           // warp that evaluates the next proposals
     i64 w_feas = 0, w_acc = 0, w_imp = 0, w_bytes = 0;          // this warp's share of the counters (lane 0)
 
     for (int kb = 0; kb < A.steps; kb += NT) {
@@ -115,13 +123,24 @@ k_anneal_wpc(const AnnealArgs A)
 
         int pos = 0;
         while (pos < nb) {
-            // ---- proposals of steps kb+pos .. kb+pos+31 against the current state ----
-            if (warp == 0) {
+            // ---- proposals of steps kb+pos .. kb+pos+31 against the current state, one per lane,
+            // with the part of the scoring that needs only the cell statistics.  The warp that
+            // proposes is the one after the last winner, whose own warp is still writing the
+            // score-side state of its move (nothing read here).
+            if (warp == proposer) {
                 bool ok = false;
                 if (pos + lane < nb) {
-                    MoveS m;
-                    ok = rp_propose(dm, view, recs[pos + lane], m);
-                    if (ok) mvs[lane] = m;
+                    CandS cd;
+                    ok = rp_propose(dm, view, recs[pos + lane], cd.m);
+                    if (ok) {
+                        const bool swap = !cd.m.reloc;
+                        const i64 ti = tt[cd.m.i], t2 = swap ? tt[cd.m.i2] : 0;
+                        cd.pad = 0;
+                        cd.Ta = (i64)T[cd.m.c1] - ti + t2; cd.Qa = (i64)Q[cd.m.c1] - ti * ti + t2 * t2;
+                        cd.Tb = (i64)T[cd.m.c2] + ti - t2; cd.Qb = (i64)Q[cd.m.c2] + ti * ti - t2 * t2;
+                        cd.A1 = aC * cd.Ta + bS * cd.Qa; cd.A2 = aC * cd.Tb + bS * cd.Qb;
+                        cand[lane] = cd;
+                    }
                 }
                 const unsigned fm = __ballot_sync(0xffffffffu, ok);
                 if (lane == 0) rnd[0] = (int)fm;
@@ -142,7 +161,7 @@ k_anneal_wpc(const AnnealArgs A)
                 i64 e1 = 0, e2 = 0, A1 = 0, A2 = 0, J1n = 0, J2n = 0, U1n = 0, U2n = 0;
                 i64 n0 = 0, n1 = 0, n2 = 0, en = 0, Ta = 0, Qa = 0, Tb = 0, Qb = 0, my_bytes = 0;
                 if (my >= 0) {
-                    m = mvs[my];
+                    m = cand[my].m;
                     const bool swap = !m.reloc;
                     const int c1 = m.c1, c2 = m.c2;
                     rg1 = rg_of[c1]; rg2 = rg_of[c2];
@@ -198,10 +217,9 @@ k_anneal_wpc(const AnnealArgs A)
                         S0 = Sc[0]; S1 = Sc[1]; S2 = Sc[2]; Ecur = Sc[3];
                         const StepRec rr = recs[pos + my];
                         thr = rr.thr; rflags = rr.flags;
-                        const i64 ti = tt[m.i], t2 = swap ? tt[m.i2] : 0;
-                        Ta = (i64)T[c1] - ti + t2; Qa = (i64)Q[c1] - ti * ti + t2 * t2;
-                        Tb = (i64)T[c2] + ti - t2; Qb = (i64)Q[c2] + ti * ti - t2 * t2;
-                        if (identity_edp) { A1 = aC * Ta + bS * Qa; A2 = aC * Tb + bS * Qb; }
+                        const CandS &cd = cand[my];
+                        Ta = cd.Ta; Qa = cd.Qa; Tb = cd.Tb; Qb = cd.Qb;
+                        if (identity_edp) { A1 = cd.A1; A2 = cd.A2; }
                         else {
                             A1 = rp_attention(dm, st, dpl, dpo, rowbase[c1] / dm.D, g1, c1, Ta, Qa, c2, Tb, Qb);
                             A2 = touchW ? rp_attention(dm, st, dpl, dpo, rowbase[c2] / dm.D, g2, c1, Ta, Qa, c2, Tb, Qb) : A1;
@@ -266,7 +284,34 @@ k_anneal_wpc(const AnnealArgs A)
                 for (int w = NW - 1; w >= 0; --w) if (w < wave && vote[w]) win = w;
                 if (my >= 0 && lane == 0 && (win < 0 || warp <= win)) { w_feas += 1; w_bytes += my_bytes; }
                 if (win >= 0) {
-                    if (warp == win) {        // commit from this warp's registers and scratch slices
+                    // commit, first half: what the next proposals read (cells, their statistics and keys)
+                    if (warp == win && lane == 0) {
+                        const bool swap = !m.reloc;
+                        const int c1 = m.c1, c2 = m.c2;
+                        cell_of[m.i] = (unsigned short)c2;
+                        if (swap) cell_of[m.i2] = (unsigned short)c1;
+                        T[c1] = (int)Ta; Q[c1] = (u64)Qa; T[c2] = (int)Tb; Q[c2] = (u64)Qb;
+                        attkey[c1] = aC * Ta + bS * Qa; attkey[c2] = aC * Tb + bS * Qb;
+                        if (!swap) { cnt[c1] -= 1; cnt[c2] += 1; }
+                        if (identity_edp) { Jcell[c1] = J1n; Acell[c1] = A1; Jcell[c2] = J2n; Acell[c2] = A2; }
+                        else {
+                            for (int x = dpo[g1]; x < dpo[g1 + 1]; ++x) { const int c = rowbase[c1] + dpl[x]; Jcell[c] = J1n; Acell[c] = A1; }
+                            for (int x = dpo[g2]; x < dpo[g2 + 1]; ++x) { const int c = rowbase[c2] + dpl[x]; Jcell[c] = J2n; Acell[c] = A2; }
+                        }
+                        rnd[1] = pos + my + 1;
+                    }
+                    fmask = 0;
+                } else {
+                    for (int w = 0; w < wave; ++w) fmask &= fmask - 1;
+                }
+                __syncthreads();
+                if (win >= 0) {
+                    next_pos = rnd[1];
+                    proposer = win + 1 == NW ? 0 : win + 1;
+                    // commit, second half, by the winner's warp while another warp proposes: rank
+                    // loads, row-shard and shard costs, score, move log and trajectory best (read
+                    // again only after the block-wide barrier that follows the proposals)
+                    if (warp == win) {
                         const bool swap = !m.reloc;
                         if (touchW) {
                             int *w1 = Wj + (size_t)rg1 * dm.LP, *w2 = Wj + (size_t)rg2 * dm.LP;
@@ -282,18 +327,8 @@ k_anneal_wpc(const AnnealArgs A)
                         if (lane == 0) {
                             const int c1 = m.c1, c2 = m.c2;
                             const int k = kb + pos + my;
-                            cell_of[m.i] = (unsigned short)c2;
-                            if (swap) cell_of[m.i2] = (unsigned short)c1;
-                            T[c1] = (int)Ta; Q[c1] = (u64)Qa; T[c2] = (int)Tb; Q[c2] = (u64)Qb;
-                            attkey[c1] = aC * Ta + bS * Qa; attkey[c2] = aC * Tb + bS * Qb;
-                            if (!swap) { cnt[c1] -= 1; cnt[c2] += 1; }
                             Esum[rg1] = e1; Afx[rg1] = A1; Jfx[rg1] = J1n;
                             if (touchW) { Esum[rg2] = e2; Afx[rg2] = A2; Jfx[rg2] = J2n; }
-                            if (identity_edp) { Jcell[c1] = J1n; Acell[c1] = A1; Jcell[c2] = J2n; Acell[c2] = A2; }
-                            else {
-                                for (int x = dpo[g1]; x < dpo[g1 + 1]; ++x) { const int c = rowbase[c1] + dpl[x]; Jcell[c] = J1n; Acell[c] = A1; }
-                                for (int x = dpo[g2]; x < dpo[g2 + 1]; ++x) { const int c = rowbase[c2] + dpl[x]; Jcell[c] = J2n; Acell[c] = A2; }
-                            }
                             U[g1] = U1n; U[g2] = U2n;
                             Sc[0] = n0; Sc[1] = n1; Sc[2] = n2; Sc[3] = en;
                             const u32 second = swap ? (u32)m.i2 : (u32)c2;
@@ -308,15 +343,9 @@ k_anneal_wpc(const AnnealArgs A)
                                 chain->best_step = k + 1; chain->best_nlog = nlog;
                                 w_imp += 1;
                             }
-                            rnd[1] = pos + my + 1;
                         }
                     }
-                    fmask = 0;
-                } else {
-                    for (int w = 0; w < wave; ++w) fmask &= fmask - 1;
                 }
-                __syncthreads();
-                if (win >= 0) next_pos = rnd[1];
             }
             pos = next_pos;
         }
@@ -356,7 +385,7 @@ size_t rp_wpc_smem_bytes(const RpDims &dm, const RpBlob &bl, const RpStatic &sl,
     const int NT = nw * 32;
     const size_t slice_pad = ((size_t)dm.LP + 3) & ~(size_t)3;
     size_t b = (size_t)bl.bytes + sl.bytes + sizeof(int) * nw * 2 * slice_pad + sizeof(i64) * 3 * dm.K +
-               sizeof(StepRec) * NT + sizeof(ChainS) + sizeof(u64) + sizeof(MoveS) * SPEC + sizeof(int) * (nw + 2);
+               sizeof(StepRec) * NT + sizeof(ChainS) + sizeof(u64) + sizeof(CandS) * SPEC + sizeof(int) * (nw + 2);
     const size_t wbytes = sizeof(int) * ((((size_t)dm.RG * dm.LP) + 3) & ~(size_t)3);
     const size_t per_cta = (size_t)220 * 1024 / (16 / nw);
     *w_in_smem = (b + wbytes <= per_cta);
