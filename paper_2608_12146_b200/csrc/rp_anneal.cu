@@ -321,6 +321,7 @@ int rp_wpc_warps(int pop_size);
 int rp_launch_anneal_wpc(rp_ctx *c, const AnnealArgs &A);
 
 static bool use_wpc(const RpDims &dm) { return dm.LP <= 512; }
+bool rp_uses_wpc(const RpDims &dm) { return use_wpc(dm); }
 
 int rp_anneal_smem_bytes(const rp_ctx *c, int *threads, size_t *bytes)
 {
@@ -363,6 +364,8 @@ int rp_launch_anneal_level(rp_ctx *c, int level, int n_levels, const rp_anneal_p
     A.lo.done = c->d_done; A.lo.anc_out = c->d_anc_next; A.lo.F = c->d_F;
     A.lo.wloc_out = c->d_wloc; A.lo.scratch = c->d_le_scratch;   // the barrier rewrites the array the level read from
     A.lo.inc_layout = c->d_inc_layout; A.lo.inc_score = c->d_inc_score;
+    A.lo.cand_layout = use_wpc(c->dm) ? c->d_cand_layout : nullptr;
+    A.lo.inc_slot = c->d_inc_slot;
     A.lo.tr_term = c->d_tr_term; A.lo.tr_best = c->d_tr_best; A.lo.tr_inc = c->d_tr_inc;
     A.lo.tr_best_step = c->d_tr_best_step; A.lo.tr_anc = c->d_tr_anc; A.lo.tr_digest = c->d_tr_digest;
     if (use_wpc(c->dm)) return rp_launch_anneal_wpc(c, A);

@@ -13,6 +13,12 @@ struct LevelOut {
     u64 *F;                    // [P_pop] cumulative resampling weights
     int *inc_layout;           // [N]
     i64 *inc_score;            // [3]
+    // Chains that keep a snapshot of their trajectory-best layout (null otherwise: the barrier then
+    // rebuilds the winner's layout from its move log).  A chain writes its row only when it
+    // strictly beats the incumbent, and then the barrier of that level names a new incumbent
+    // among the writers: the row of the current incumbent's slot is never overwritten unnoticed.
+    unsigned short *cand_layout;   // [P_pop][N]
+    int *inc_slot;                 // slot whose row holds the incumbent, -1 = inc_layout is current
     i64 *tr_term, *tr_best, *tr_inc;     // trace (nullable)
     int *tr_best_step, *tr_anc;
     u64 *tr_digest;

@@ -29,6 +29,8 @@ struct ChainS {                 // bookkeeping of the chain within this level
     i64 B[3];                   // trajectory-best score
     u64 dig;                    // digest of the accepted moves
     int best_step, best_nlog, nlog, failed;
+    i64 I[3];                   // incumbent score when the level started
+    int has_snap;               // best_lay holds a layout that beats it
 };
 
 template <int NW, bool WS, int CH>
@@ -53,6 +55,7 @@ k_anneal_wpc(const AnnealArgs A)
     CandS *cand = (CandS *)(mbar + 1);
     int *vote = (int *)(cand + SPEC);                                    // [NW] accept flags of a wave
     int *rnd = vote + NW;                                               // [0] feasible mask, [1] next position
+    unsigned short *best_lay = (unsigned short *)(((size_t)(rnd + 2) + 15) & ~(size_t)15);   // [N] trajectory-best layout
 
     u64 *Q = (u64 *)(sm_blob + A.bl.off_Q);
     i64 *Esum = (i64 *)(sm_blob + A.bl.off_Esum);
@@ -107,6 +110,8 @@ k_anneal_wpc(const AnnealArgs A)
     if (tid == 0) {
         chain->B[0] = Sc[0]; chain->B[1] = Sc[1]; chain->B[2] = Sc[2];
         chain->dig = 0; chain->best_step = 0; chain->best_nlog = 0; chain->nlog = 0;
+        chain->I[0] = A.lo.inc_score[0]; chain->I[1] = A.lo.inc_score[1]; chain->I[2] = A.lo.inc_score[2];
+        chain->has_snap = 0;
     }
     __syncthreads();
 
@@ -324,6 +329,7 @@ k_anneal_wpc(const AnnealArgs A)
                                 for (int x = lane; x < dm.LP; x += 32) { w1[x] = my_s1[x]; w2[x] = my_s2[x]; }
                             }
                         }
+                        int snap = 0;
                         if (lane == 0) {
                             const int c1 = m.c1, c2 = m.c2;
                             const int k = kb + pos + my;
@@ -342,7 +348,20 @@ k_anneal_wpc(const AnnealArgs A)
                                 chain->B[0] = n0; chain->B[1] = n1; chain->B[2] = n2;
                                 chain->best_step = k + 1; chain->best_nlog = nlog;
                                 w_imp += 1;
+                                snap = rp_lex_less(n0, n1, n2, chain->I[0], chain->I[1], chain->I[2]);
                             }
+                        }
+                        // a new trajectory best that also beats the incumbent: keep its layout (the first
+                        // half of the commit is already in cell_of; the proposing warp only reads it)
+                        if (__shfl_sync(0xffffffffu, snap, 0)) {
+                            if ((((size_t)cell_of & 15) | ((size_t)dm.N & 7)) == 0) {
+                                const uint4 *sv = (const uint4 *)cell_of;
+                                uint4 *dv = (uint4 *)best_lay;
+                                for (int x = lane; x < (dm.N >> 3); x += 32) dv[x] = sv[x];
+                            } else {
+                                for (int x = lane; x < dm.N; x += 32) best_lay[x] = cell_of[x];
+                            }
+                            if (lane == 0) chain->has_snap = 1;
                         }
                     }
                 }
@@ -353,6 +372,10 @@ k_anneal_wpc(const AnnealArgs A)
 
     // ---- epilogue: terminal state and chain report ------------------------------------------
     rp_chain_store<NT, WS>(A, j, sm_blob, Wsm, tid);
+    if (chain->has_snap) {
+        unsigned short *row = A.lo.cand_layout + (size_t)j * dm.N;
+        for (int x = tid; x < dm.N; x += NT) row[x] = best_lay[x];
+    }
     if (lane == 0) {
         if (w_feas) atomicAdd((u64 *)&A.counters[1], (u64)w_feas);
         if (w_acc) atomicAdd((u64 *)&A.counters[2], (u64)w_acc);
@@ -385,7 +408,8 @@ size_t rp_wpc_smem_bytes(const RpDims &dm, const RpBlob &bl, const RpStatic &sl,
     const int NT = nw * 32;
     const size_t slice_pad = ((size_t)dm.LP + 3) & ~(size_t)3;
     size_t b = (size_t)bl.bytes + sl.bytes + sizeof(int) * nw * 2 * slice_pad + sizeof(i64) * 3 * dm.K +
-               sizeof(StepRec) * NT + sizeof(ChainS) + sizeof(u64) + sizeof(CandS) * SPEC + sizeof(int) * (nw + 2);
+               sizeof(StepRec) * NT + sizeof(ChainS) + sizeof(u64) + sizeof(CandS) * SPEC + sizeof(int) * (nw + 2) +
+               16 + ((sizeof(unsigned short) * dm.N + 15) & ~(size_t)15);
     const size_t wbytes = sizeof(int) * ((((size_t)dm.RG * dm.LP) + 3) & ~(size_t)3);
     const size_t per_cta = (size_t)220 * 1024 / (16 / nw);
     *w_in_smem = (b + wbytes <= per_cta);

@@ -123,6 +123,8 @@ static void free_population(rp_ctx *c)
     }
     dev_free(c, c->d_W); dev_free(c, c->d_wloc); dev_free(c, c->d_wloc_next); dev_free(c, c->d_le_scratch);
     c->d_W = nullptr; c->d_wloc = nullptr; c->d_wloc_next = nullptr; c->d_le_scratch = nullptr;
+    dev_free(c, c->d_cand_layout); dev_free(c, c->d_inc_slot);
+    c->d_cand_layout = nullptr; c->d_inc_slot = nullptr;
     dev_free(c, c->d_anc); dev_free(c, c->d_anc_next); dev_free(c, c->d_done); dev_free(c, c->d_term); dev_free(c, c->d_best); dev_free(c, c->d_best_step);
     dev_free(c, c->d_best_nlog); dev_free(c, c->d_digest); dev_free(c, c->d_log); dev_free(c, c->d_F);
     c->d_anc = nullptr; c->d_anc_next = nullptr; c->d_done = nullptr; c->d_term = nullptr; c->d_best = nullptr; c->d_best_step = nullptr;
@@ -388,6 +390,8 @@ extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
     RP_TRY(dev_alloc(c, &c->d_wloc, P));
     RP_TRY(dev_alloc(c, &c->d_wloc_next, P));
     RP_TRY(dev_alloc(c, &c->d_le_scratch, 6 * P));
+    RP_TRY(dev_alloc(c, &c->d_inc_slot, 1));
+    if (rp_uses_wpc(c->dm)) RP_TRY(dev_alloc(c, &c->d_cand_layout, P * (size_t)c->dm.N));
     RP_TRY(dev_alloc(c, &c->d_anc, P));
     RP_TRY(dev_alloc(c, &c->d_anc_next, P));
     RP_TRY(dev_alloc(c, &c->d_done, 1));
@@ -565,6 +569,7 @@ extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *
         c->trace_levels = NL;
     }
     RP_CUDA(cudaMemsetAsync(c->d_counters, 0, sizeof(i64) * 8, c->stream));
+    RP_CUDA(cudaMemsetAsync(c->d_inc_slot, 0xff, sizeof(int), c->stream));      // -1: the incumbent is in d_inc_layout
     RP_TRY(reset_status(c));
 
     cudaEvent_t ev[2] = { nullptr, nullptr };

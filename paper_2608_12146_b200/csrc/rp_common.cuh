@@ -137,6 +137,8 @@ struct rp_ctx {
     i64 *d_counters;           // [4]
     // incumbent
     int *d_inc_layout;         // [N]
+    unsigned short *d_cand_layout;   // [P_pop][N] trajectory-best snapshots of the chains (warp-per-candidate kernel)
+    int *d_inc_slot;           // [1]
     i64 *d_inc_score;          // [3]
     // trace of the last rp_anneal call
     int trace_levels;
@@ -177,6 +179,7 @@ int rp_launch_pick_best(rp_ctx *c, const i64 *scores, const int *layouts, int n,
 int rp_get_pool(int device, cudaMemPool_t *out);     // the library's stream-ordered pool of a device
 void rp_make_layouts(const RpDims &dm, RpBlob *bl, RpStatic *sl);
 int rp_launch_cells_from_layouts(rp_ctx *c, const int *layouts, int n, unsigned short *cells);
+bool rp_uses_wpc(const RpDims &dm);
 int rp_launch_anneal_level(rp_ctx *c, int level, int n_levels, const rp_anneal_params *prm, u64 rho_q32, u64 guide_q32);
 int rp_launch_validate(rp_ctx *c);
 int rp_anneal_smem_bytes(const rp_ctx *c, int *threads, size_t *bytes);

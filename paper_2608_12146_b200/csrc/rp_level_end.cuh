@@ -135,7 +135,7 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
         const i64 t0 = LE_LD(A.term[3 * (size_t)j]), t1 = LE_LD(A.term[3 * (size_t)j + 1]), t2 = LE_LD(A.term[3 * (size_t)j + 2]);
         if (rp_lex_less(s0, s1, s2, b0, b1, b2)) {    // ascending j: first wins
             b0 = s0; b1 = s1; b2 = s2; bj = j;
-            bn = LE_LD(A.best_nlog[j]); ba = A.anc[j];       // what the replay needs, fetched with the rest
+            if (!O.cand_layout) { bn = LE_LD(A.best_nlog[j]); ba = A.anc[j]; }     // what the replay needs, fetched with the rest
         }
         const i64 e = rp_energy(t0, t1, t2);
         emin = e < emin ? e : emin;
@@ -161,10 +161,13 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
         }
         win_j = bj; win_n = bn; win_a = ba;
         do_update = rp_lex_less(b0, b1, b2, i0, i1, i2);
-        if (do_update) { O.inc_score[0] = b0; O.inc_score[1] = b1; O.inc_score[2] = b2; }
+        if (do_update) {
+            O.inc_score[0] = b0; O.inc_score[1] = b1; O.inc_score[2] = b2;
+            if (O.cand_layout) *O.inc_slot = bj;         // the winner stored its best layout itself
+        }
     }
     __syncthreads();
-    if (do_update) {
+    if (do_update && !O.cand_layout) {
         const int w = win_j;
         const unsigned short *cs = (const unsigned short *)(A.blob_src + (size_t)win_a * A.bl.bytes + A.bl.off_cell);
         const uint2 *lg = A.log + (size_t)w * A.log_cap;
@@ -214,6 +217,13 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
     if (O.tr_inc && tid < 3) O.tr_inc[(size_t)A.level * 3 + tid] = O.inc_score[tid];
 
     if (A.last) {            // the terminal states are the population as they stand
+        if (O.cand_layout) {
+            const int sl = *O.inc_slot;
+            if (sl >= 0) {
+                const unsigned short *row = O.cand_layout + (size_t)sl * A.dm.N;
+                for (int i = tid; i < A.dm.N; i += nt) O.inc_layout[i] = LE_LD(row[i]);
+            }
+        }
         for (int m = tid; m < P; m += nt) { O.anc_out[m] = m; O.wloc_out[m] = A.wloc_dst[m]; }
         return;
     }
