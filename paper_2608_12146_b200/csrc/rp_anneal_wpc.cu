@@ -79,6 +79,10 @@ k_anneal_wpc(const AnnealArgs A)
     const bool identity_edp = (dm.G == dm.D);
     const bool vec = (dm.P >= 4) && (dm.P <= 128) && ((dm.P & (dm.P - 1)) == 0);
     const i64 aC = dm.asum * dm.C, bS = dm.bsum;
+    // A rank load is at most k*C tokens per cell of the row-shard (conservation of the demand
+    // rows, token cap), so the sum over layers of the busiest ranks usually fits 32 bits and
+    // the warp can add it up with one reduction instruction.
+    const bool sum32 = (i64)dm.L * dm.k * dm.C * ((dm.D + dm.G - 1) / dm.G) < (1ll << 31);
 
     // The step records of the first batch depend on nothing the previous level wrote: compute
     // them before waiting for it (this kernel is launched with programmatic stream
@@ -211,8 +215,13 @@ k_anneal_wpc(const AnnealArgs A)
                                 if (lane == 0) { e1 += v1; e2 += v2; }
                             }
                         }
-                        e1 = warp_sum_i64(e1);
-                        e2 = warp_sum_i64(e2);
+                        if (sum32) {
+                            e1 = (i64)__reduce_add_sync(0xffffffffu, (unsigned)e1);
+                            e2 = (i64)__reduce_add_sync(0xffffffffu, (unsigned)e2);
+                        } else {
+                            e1 = warp_sum_i64(e1);
+                            e2 = warp_sum_i64(e2);
+                        }
                     }
                     // (c) the part of the new score that does not need the rank loads
                     i64 S0 = 0, S1 = 0, S2 = 0, Ecur = 0, J1o = 0, J2o = 0, U1o = 0, U2o = 0;
@@ -296,7 +305,8 @@ k_anneal_wpc(const AnnealArgs A)
                         cell_of[m.i] = (unsigned short)c2;
                         if (swap) cell_of[m.i2] = (unsigned short)c1;
                         T[c1] = (int)Ta; Q[c1] = (u64)Qa; T[c2] = (int)Tb; Q[c2] = (u64)Qb;
-                        attkey[c1] = aC * Ta + bS * Qa; attkey[c2] = aC * Tb + bS * Qb;
+                        if (identity_edp) { attkey[c1] = A1; attkey[c2] = A2; }      // the same expression
+                        else { attkey[c1] = aC * Ta + bS * Qa; attkey[c2] = aC * Tb + bS * Qb; }
                         if (!swap) { cnt[c1] -= 1; cnt[c2] += 1; }
                         if (identity_edp) { Jcell[c1] = J1n; Acell[c1] = A1; Jcell[c2] = J2n; Acell[c2] = A2; }
                         else {

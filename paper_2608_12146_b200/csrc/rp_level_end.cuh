@@ -251,12 +251,27 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
             pos[u] = (unsigned __int128)u0 + (unsigned __int128)(m < P ? m : 0) * Ftot;
             lo[u] = 0; hi[u] = (m < P) ? P - 1 : 0;      // smallest j with P*F[j] > pos (nothing to search past the end)
         }
-        for (int it = 0; it < depth; ++it) {
+        if ((P & (P - 1)) == 0) {       // P = 2^depth: P*F > pos  <=>  F > floor(pos / P), a 64-bit comparison
+            u64 thr[SU];
 #pragma unroll
-            for (int u = 0; u < SU; ++u) {
-                if (lo[u] < hi[u]) {
-                    const int mid = (lo[u] + hi[u]) >> 1;
-                    if ((unsigned __int128)P * F[mid] > pos[u]) hi[u] = mid; else lo[u] = mid + 1;
+            for (int u = 0; u < SU; ++u) thr[u] = (u64)(pos[u] >> depth);
+            for (int it = 0; it < depth; ++it) {
+#pragma unroll
+                for (int u = 0; u < SU; ++u) {
+                    if (lo[u] < hi[u]) {
+                        const int mid = (lo[u] + hi[u]) >> 1;
+                        if (F[mid] > thr[u]) hi[u] = mid; else lo[u] = mid + 1;
+                    }
+                }
+            }
+        } else {
+            for (int it = 0; it < depth; ++it) {
+#pragma unroll
+                for (int u = 0; u < SU; ++u) {
+                    if (lo[u] < hi[u]) {
+                        const int mid = (lo[u] + hi[u]) >> 1;
+                        if ((unsigned __int128)P * F[mid] > pos[u]) hi[u] = mid; else lo[u] = mid + 1;
+                    }
                 }
             }
         }
