@@ -165,6 +165,8 @@ EDGE_SPECS = [
     ("wide_ranks", 90, 2, 96, 2, 4096, 2, 48, None, 5),
     ("single_slot", 40, 3, 8, 2, 2048, 1, 4, None, 6),
     ("vector_tail", 130, 9, 40, 2, 8192, 5, 20, [0, 1, 1, 2, 2], 3),
+    # L*k*C*(cells per row-shard) >= 2^31: the sums over layers of the busiest ranks need 64 bits
+    ("wide_sums", 72, 64, 16, 8, 1 << 20, 4, 4, [0, 0, 0, 0], 3),
 ]
 
 
