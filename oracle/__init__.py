@@ -157,6 +157,19 @@ def seed_trials(lengths, seed_layout, R: int, C_cap: int, D: int, pop_size: int,
     return lay, ok
 
 
+def edp_pair(q, layouts, R: int, D: int, width: int, seed: int, edp_of_dp=None) -> np.ndarray:
+    """EDPAwarePair on every member j >= 1 of `layouts` [P][N]; returns the re-paired layouts."""
+    q = _i32(q)
+    lay = _i32(layouts).copy()
+    Ppop, N = lay.shape
+    _, L, P = q.shape
+    edp = np.arange(D, dtype=np.int32) if edp_of_dp is None else _i32(edp_of_dp)
+    G = int(edp.max()) + 1
+    lib().orc_edp_pair(C.c_int32(N), C.c_int32(L), C.c_int32(P), C.c_int32(D), C.c_int32(G), C.c_int32(R),
+                       C.c_int32(width), C.c_uint64(seed), _p(q), _p(edp), C.c_int32(Ppop), _p(lay))
+    return lay
+
+
 # ---- scoring ----------------------------------------------------------------------------
 def _edp(D: int, edp_of_dp) -> np.ndarray:
     return np.arange(D, dtype=np.int32) if edp_of_dp is None else _i32(edp_of_dp)

@@ -1047,3 +1047,106 @@ void orc_seed_trials(int32_t N, int32_t C, int32_t D, int32_t R, int32_t w, uint
     }
     free(order); free(win); free(fill); free(cnt); free(cand);
 }
+
+/* ------------------------------------------------------------------------------------ */
+/* EDPAwarePair (Section 4.1.1, the third construction operator of Algorithm 2): keeps   */
+/* every completed cell as a set of samples and only changes which (row, DP slot) it     */
+/* occupies.                                                                              */
+/*                                                                                        */
+/* Reading (the paper gives one sentence; "parity unpinned" against the paper for the     */
+/* sampling law, the rest is pinned by a worked example and closed forms):                */
+/*  * profile of a cell b: w_b[l][p] = sum of q[i][l][p] over its samples; its            */
+/*    routed-token peak is max_{l,p} w_b[l][p].  Cells are taken in order of decreasing   */
+/*    peak, ties by lower cell index.                                                     */
+/*  * V[r][g][l][p] is the rank load of row-shard (r, g) from the cells placed so far.    */
+/*    For the cell in hand every still-empty slot s = r*D + d (shard g = edp(d)) gets the */
+/*    insertion key (sum_l max_p (V+w) - sum_l max_p V,  max_{l,p} (V+w)); slots are      */
+/*    ranked by ascending key, ties by lower slot index.                                  */
+/*  * rank-decaying top-w sampling: with m = min(w, #empty), rank rho = min(m-1, number   */
+/*    of leading zero bits of the draw) - rank 0 with probability 1/2, rank 1 with 1/4,   */
+/*    ..., the remainder on rank m-1.  Draw: Philox(h, 0, trial, 6).x for the h-th cell   */
+/*    placed.                                                                             */
+/* Member 0 is left untouched (the length-only seed); member j >= 1 is trial j.           */
+/* ------------------------------------------------------------------------------------ */
+void orc_edp_pair(int32_t N, int32_t L, int32_t P, int32_t D, int32_t G, int32_t R, int32_t w, uint64_t seed,
+                  const int32_t *q, const int32_t *edp_of_dp, int32_t Ppop, int32_t *layouts)
+{
+    const int32_t K = R * D;
+    const size_t LP = (size_t)L * P;
+    int64_t *prof = (int64_t *)malloc(sizeof(int64_t) * K * LP);
+    int64_t *V = (int64_t *)malloc(sizeof(int64_t) * (size_t)R * G * LP);
+    int64_t *peak = (int64_t *)malloc(sizeof(int64_t) * K);
+    int32_t *order = (int32_t *)malloc(sizeof(int32_t) * K);
+    int32_t *slot_of = (int32_t *)malloc(sizeof(int32_t) * K);
+    int32_t *empty = (int32_t *)malloc(sizeof(int32_t) * K);
+    int32_t *rank = (int32_t *)malloc(sizeof(int32_t) * K);
+    int64_t *kd = (int64_t *)malloc(sizeof(int64_t) * K), *kp = (int64_t *)malloc(sizeof(int64_t) * K);
+    for (int32_t j = 1; j < Ppop; ++j) {
+        int32_t *lay = layouts + (size_t)j * N;
+        memset(prof, 0, sizeof(int64_t) * K * LP);
+        memset(V, 0, sizeof(int64_t) * (size_t)R * G * LP);
+        for (int32_t i = 0; i < N; ++i)
+            for (size_t x = 0; x < LP; ++x) prof[(size_t)lay[i] * LP + x] += q[(size_t)i * LP + x];
+        for (int32_t b = 0; b < K; ++b) {
+            int64_t m = 0;
+            for (size_t x = 0; x < LP; ++x) if (prof[(size_t)b * LP + x] > m) m = prof[(size_t)b * LP + x];
+            peak[b] = m;
+            order[b] = b;
+            empty[b] = 1;
+        }
+        for (int32_t x = 1; x < K; ++x) {                /* insertion sort by (-peak, b) */
+            int32_t s = order[x], y = x;
+            while (y > 0 && (peak[order[y - 1]] < peak[s] || (peak[order[y - 1]] == peak[s] && order[y - 1] > s))) {
+                order[y] = order[y - 1];
+                --y;
+            }
+            order[y] = s;
+        }
+        for (int32_t h = 0; h < K; ++h) {
+            const int32_t b = order[h];
+            const int64_t *wb = prof + (size_t)b * LP;
+            int32_t ne = 0;
+            for (int32_t s = 0; s < K; ++s) {
+                if (!empty[s]) continue;
+                const int32_t r = s / D, g = edp_of_dp[s % D];
+                const int64_t *v = V + ((size_t)r * G + g) * LP;
+                int64_t e_old = 0, e_new = 0, pk = 0;
+                for (int32_t l = 0; l < L; ++l) {
+                    int64_t mo = 0, mn = 0;
+                    for (int32_t p = 0; p < P; ++p) {
+                        const int64_t a = v[(size_t)l * P + p], c = a + wb[(size_t)l * P + p];
+                        if (a > mo) mo = a;
+                        if (c > mn) mn = c;
+                    }
+                    e_old += mo;
+                    e_new += mn;
+                    if (mn > pk) pk = mn;
+                }
+                kd[s] = e_new - e_old;
+                kp[s] = pk;
+                /* insert s into the ranking: ascending (kd, kp, s) */
+                int32_t y = ne++;
+                while (y > 0) {
+                    const int32_t o = rank[y - 1];
+                    if (kd[o] < kd[s] || (kd[o] == kd[s] && (kp[o] < kp[s] || (kp[o] == kp[s] && o < s)))) break;
+                    rank[y] = o;
+                    --y;
+                }
+                rank[y] = s;
+            }
+            uint32_t X[4];
+            draw(seed, (uint32_t)h, 0u, (uint32_t)j, 6u, X);
+            int32_t lz = 0;
+            while (lz < 32 && !((X[0] >> (31 - lz)) & 1u)) ++lz;
+            const int32_t m = ne < w ? ne : w;
+            const int32_t rho = lz < m - 1 ? lz : m - 1;
+            const int32_t s = rank[rho];
+            slot_of[b] = s;
+            empty[s] = 0;
+            int64_t *v = V + ((size_t)(s / D) * G + edp_of_dp[s % D]) * LP;
+            for (size_t x = 0; x < LP; ++x) v[x] += wb[x];
+        }
+        for (int32_t i = 0; i < N; ++i) lay[i] = slot_of[lay[i]];
+    }
+    free(prof); free(V); free(peak); free(order); free(slot_of); free(empty); free(rank); free(kd); free(kp);
+}

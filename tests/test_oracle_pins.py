@@ -624,3 +624,118 @@ def test_seed_trial_draws_are_uniform_over_the_window():
     for j in range(1, 200):
         assert sorted(lays[j].tolist()) == list(range(N))            # a permutation
         assert (lays[j] >= np.arange(N) - (width - 1)).all()         # sample i leaves no earlier than i-(w-1)
+
+
+# ---- EDPAwarePair (Section 4.1.1, Algorithm 2) ---------------------------------------------
+def _pair_inputs(profiles):
+    """One sample per cell whose demand row is the given profile [K][L][P]."""
+    prof = np.asarray(profiles, np.int32)
+    K = prof.shape[0]
+    q = prof.copy()
+    lay = np.arange(K, dtype=np.int32)
+    return q, lay
+
+
+def test_edp_pair_worked_example_balances_the_shared_shard():
+    """Two rows of two DP slots that share one EDP shard; one layer, two ranks.  Cells a, c load
+    rank 0 with 10 tokens, cells b, d load rank 1.  Greedy pairing (width 1): a opens row 0; b adds
+    nothing to the peak sum of row 0 (key (0, 10)) but 10 to row 1, so it joins a; c then only has
+    row 1 left, d follows.  Rows {a, b}, {c, d}: each row peaks at 10 instead of 20 for {a, c}."""
+    prof = [[[10, 0]], [[0, 10]], [[10, 0]], [[0, 10]]]
+    q, lay = _pair_inputs(prof)
+    pop = np.stack([lay, lay])
+    out = oracle.edp_pair(q, pop, R=2, D=2, width=1, seed=3, edp_of_dp=[0, 0])
+    assert (out[0] == lay).all()                     # member 0 is never touched
+    assert out[1].tolist() == [0, 1, 2, 3]
+    # same cells listed as a, c, b, d: the pairing must undo the bad order (a with b, c with d)
+    prof2 = [prof[0], prof[2], prof[1], prof[3]]
+    q2, lay2 = _pair_inputs(prof2)
+    out2 = oracle.edp_pair(q2, np.stack([lay2, lay2]), R=2, D=2, width=1, seed=3, edp_of_dp=[0, 0])
+    rows = out2[1] // 2
+    assert rows[0] == rows[2] and rows[1] == rows[3] and rows[0] != rows[1]
+
+
+def test_edp_pair_second_key_breaks_equal_increases():
+    """One shard, two rows of two slots, two layers, one rank.  a = (10, 0) opens row 0.  b = (0, 8)
+    raises the peak sum by 8 in either row, but the largest peak would be 10 in row 0 and 8 in row 1:
+    the second key sends it to row 1 (slot 2) although slot 1 has the lower index.  c = (1, 0) adds 1
+    anywhere; the peak is 11 beside a and 8 beside b, so it joins b (slot 3); d = (0, 1) takes slot 1."""
+    prof = [[[10], [0]], [[0], [8]], [[1], [0]], [[0], [1]]]
+    q, lay = _pair_inputs(prof)
+    out = oracle.edp_pair(q, np.stack([lay, lay]), R=2, D=2, width=1, seed=11, edp_of_dp=[0, 0])
+    assert out[1].tolist() == [0, 2, 3, 1]
+
+
+def test_edp_pair_identity_shards_sorts_cells_by_peak():
+    """With one shard per DP slot every empty slot has an empty row-shard, so all keys tie and the
+    lowest slot wins: greedy pairing lists the cells by decreasing peak (ties: lower index)."""
+    rng = np.random.default_rng(4)
+    K, L, P = 12, 3, 4
+    prof = rng.integers(0, 50, (K, L, P))
+    prof[5] = prof[2]                                   # a tie
+    q, lay = _pair_inputs(prof)
+    out = oracle.edp_pair(q, np.stack([lay, lay]), R=3, D=4, width=1, seed=1)
+    peaks = prof.reshape(K, -1).max(1)
+    order = sorted(range(K), key=lambda b: (-int(peaks[b]), b))
+    want = np.empty(K, np.int64)
+    for h, b in enumerate(order):
+        want[b] = h
+    assert out[1].tolist() == want.tolist()
+
+
+def test_edp_pair_keeps_cells_and_its_greedy_step_is_the_smallest_key():
+    w = hetero_window(N=80, L=3, E=8, k=2, C=4096, D=4, P=4, seed=17)
+    s, t = w.spec, w.lengths
+    edp = [0, 0, 1, 1]
+    pi, _ = oracle.lpt(oracle.aggregate(w.demand), s.ep_width)
+    q = oracle.project(w.demand, pi, s.ep_width)
+    R, _, seed_lay = oracle.pack_ffd(t, s.token_cap, s.dp_width, min_rows=3)
+    K = R * s.dp_width
+    lays, ok = oracle.seed_trials(t, seed_lay, R, s.token_cap, s.dp_width, 16, 4, seed=9)
+    for width in (1, 3):
+        out = oracle.edp_pair(q, lays, R, s.dp_width, width, seed=9, edp_of_dp=edp)
+        assert (out[0] == lays[0]).all()
+        for j in range(1, 16):
+            # a bijection of cells onto slots: samples that shared a cell still do, nothing else does
+            m = {}
+            for i in range(len(t)):
+                assert m.setdefault(int(lays[j][i]), int(out[j][i])) == int(out[j][i])
+            assert sorted(m.values()) == sorted(set(m.values())) and len(m) == K
+    # width 1, member 1: replay the greedy rule with plain numpy and compare slot by slot
+    out = oracle.edp_pair(q, lays, R, s.dp_width, 1, seed=9, edp_of_dp=edp)
+    lay = lays[1]
+    prof = np.zeros((K,) + q.shape[1:], np.int64)
+    np.add.at(prof, lay, q)
+    V = np.zeros((R, 2) + q.shape[1:], np.int64)
+    empty = [True] * K
+    slot_of = {}
+    for b in sorted(range(K), key=lambda b: (-int(prof[b].max()), b)):
+        best = None
+        for sl in range(K):
+            if not empty[sl]:
+                continue
+            v = V[sl // 4, edp[sl % 4]]
+            key = (int((v + prof[b]).max(1).sum() - v.max(1).sum()), int((v + prof[b]).max()), sl)
+            if best is None or key < best:
+                best = key
+        sl = best[2]
+        empty[sl] = False
+        slot_of[b] = sl
+        V[sl // 4, edp[sl % 4]] += prof[b]
+    assert [slot_of[int(b)] for b in lay] == out[1].tolist()
+
+
+def test_edp_pair_sampling_ranks_decay_by_halves():
+    """Identity shards, so the ranking of the empty slots is the slot order itself and the cell with
+    the largest peak lands on slot rho of the first draw: rho = 0, 1, 2 with probability 1/2, 1/4 and
+    (width 3) the remaining 1/4."""
+    K, L, P = 6, 1, 2
+    prof = np.zeros((K, L, P), np.int64)
+    prof[:, 0, 0] = [60, 50, 40, 30, 20, 10]
+    q, lay = _pair_inputs(prof)
+    n = 4001
+    out = oracle.edp_pair(q, np.tile(lay, (n, 1)), R=2, D=3, width=3, seed=77)
+    first = out[1:, 0]                                   # slot of the cell with the largest peak
+    freq = np.bincount(first, minlength=K) / (n - 1)
+    assert freq[3:].sum() == 0
+    assert abs(freq[0] - 0.5) < 0.03 and abs(freq[1] - 0.25) < 0.03 and abs(freq[2] - 0.25) < 0.03
