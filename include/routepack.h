@@ -126,6 +126,23 @@ int rp_pack_rows(rp_ctx *ctx, int32_t *n_rows, int32_t *certified);
  *   choice_width in [1, 32]; n_own: HOST out, members that carry their own trial (nullable). */
 int rp_seed_population(rp_ctx *ctx, int32_t choice_width, int32_t *n_own);
 
+/* EDPAwarePair on the current population (Section 4.1.1; Algorithm 2, third construction
+ * operator).  Optional, between rp_pack_rows and rp_anneal (after rp_seed_population when both are
+ * used).  Member 0 is left as it is; in every member j >= 1 each completed cell keeps its samples
+ * and moves to a new (row, DP slot):
+ *   - profile w_b[l][p] = sum of q[i][l][p] over the cell's samples; cells are taken by decreasing
+ *     routed-token peak max w_b (ties: lower cell index);
+ *   - every empty slot gets the insertion key (increase of sum_l max_p of its row-shard's rank
+ *     load, largest such peak afterwards); slots are ranked by ascending key, ties by lower index;
+ *   - rank-decaying sampling among the leading min(choice_width, #empty) slots: rank 0 with
+ *     probability 1/2, rank 1 with 1/4, ..., the remainder on the last rank (the paper names the
+ *     rule without giving its law; this is one reading of it).  Draw: Philox(h, 0, j, 6) for the
+ *     h-th cell placed.
+ * All members are scored from scratch; the incumbent becomes the best member (lowest index on ties).
+ *   choice_width in [1, 32]; n_changed: HOST out, members whose layout changed (nullable).
+ * RP_ERR_STATE outside stage 3, RP_ERR_RANGE when the per-member tables exceed shared memory. */
+int rp_pair_population(rp_ctx *ctx, int32_t choice_width, int32_t *n_changed);
+
 /* Full evaluation of layouts (Section 3.4-3.5: Eqs. cell-token-statistics,
  * stage-aware-attention, row-expert-load, row-expert-cost, lexicographic-score).
  *   layouts [n][N] int32 cell ids, or NULL to score the current population (n = pop_size).

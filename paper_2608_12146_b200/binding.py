@@ -22,7 +22,7 @@ STATUS_NAMES = {0: "RP_OK", -1: "RP_ERR_ARG", -2: "RP_ERR_SHAPE", -3: "RP_ERR_CO
                 -8: "RP_ERR_TIMEOUT", -9: "RP_ERR_INVALID_PLAN"}
 RP_OK = 0
 
-EXPORTS = ("rp_window_load", "rp_place_experts", "rp_pack_rows", "rp_seed_population", "rp_eval_population", "rp_eval_layouts_noalloc", "rp_diagnostics", "rp_anneal",
+EXPORTS = ("rp_window_load", "rp_place_experts", "rp_pack_rows", "rp_seed_population", "rp_pair_population", "rp_eval_population", "rp_eval_layouts_noalloc", "rp_diagnostics", "rp_anneal",
            "rp_best", "rp_destroy", "rp_release_cached_memory", "rp_strerror", "rp_last_cuda_error", "rp_debug_dump",
            "rp_debug_set_trace",
            "rp_debug_nl2", "rp_debug_exp2neg", "rp_debug_philox", "rp_debug_launch_count")
@@ -81,6 +81,7 @@ def lib():
         L.rp_place_experts.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         L.rp_pack_rows.argtypes = [C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         L.rp_seed_population.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_int32)]
+        L.rp_pair_population.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_int32)]
         L.rp_eval_population.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
         L.rp_eval_layouts_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
         L.rp_diagnostics.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(rp_diag)]
@@ -186,6 +187,13 @@ def rp_seed_population(ctx: Context, choice_width: int) -> int:
     own = C.c_int32(0)
     _check(lib().rp_seed_population(ctx.handle, choice_width, C.byref(own)), "rp_seed_population")
     return own.value
+
+
+def rp_pair_population(ctx: Context, choice_width: int) -> int:
+    """EDPAwarePair on every member but the first; returns how many layouts changed."""
+    changed = C.c_int32(0)
+    _check(lib().rp_pair_population(ctx.handle, choice_width, C.byref(changed)), "rp_pair_population")
+    return int(changed.value)
 
 
 def rp_eval_population(ctx: Context, layouts=None, score_fx=None, score_f64=None):

@@ -476,6 +476,31 @@ extern "C" int rp_eval_population(rp_ctx *c, const int32_t *layouts, int32_t n, 
 // Randomized fixed-row seeds (Algorithm 2, trial loop): member 0 keeps the length-only seed, every
 // other member runs its own WindowShuffle + RandomizedBestFit trial; all members are then scored
 // from scratch and the incumbent becomes the best of them.
+// Scores `lay` [P_pop][N] from scratch, makes it the population (member m owns rank-load cell m)
+// and makes the best member the incumbent (lowest index on ties).
+static int install_population(rp_ctx *c, const int *lay)
+{
+    const size_t P = (size_t)c->Ppop;
+    i64 *best = nullptr;
+    RP_TRY(dev_alloc(c, &best, 3));
+    int st = ensure_eval_scratch(c, P, false);
+    if (st == RP_OK) st = rp_launch_cells_from_layouts(c, lay, (int)P, c->d_eval_cells);
+    c->cur = 0;
+    if (st == RP_OK) st = rp_launch_eval(c, c->d_eval_cells, (int)P, c->d_W, c->buf[0].blob, c->d_eval_score, nullptr);
+    if (st == RP_OK) {
+        k_iota<<<(int)((P + 255) / 256), 256, 0, c->stream>>>(c->d_wloc, (int)P, 0);
+        k_iota<<<(int)((P + 255) / 256), 256, 0, c->stream>>>(c->d_wloc_next, (int)P, 0);
+        k_iota<<<(int)((P + 255) / 256), 256, 0, c->stream>>>(c->d_anc, (int)P, 0);
+        g_rp_launches += 3;
+    }
+    if (st == RP_OK) st = rp_launch_pick_best(c, c->d_eval_score, lay, (int)P, best);
+    cudaError_t e = cudaSuccess;
+    if (st == RP_OK) e = cudaMemcpyAsync(c->d_seed_score, best, sizeof(i64) * 3, cudaMemcpyDeviceToDevice, c->stream);
+    dev_free(c, best);
+    if (e != cudaSuccess) { g_rp_last_cuda_error = (int)e; return RP_ERR_CUDA; }
+    return st;
+}
+
 extern "C" int rp_seed_population(rp_ctx *c, int32_t choice_width, int32_t *n_own)
 {
     if (!c) return RP_ERR_ARG;
@@ -485,35 +510,76 @@ extern "C" int rp_seed_population(rp_ctx *c, int32_t choice_width, int32_t *n_ow
     if (dm.K > 2048) return RP_ERR_RANGE;            // per-warp cell tables live in shared memory
     const size_t P = (size_t)c->Ppop;
     int *lay = nullptr, *ok = nullptr;
-    i64 *best = nullptr;
     RP_TRY(dev_alloc(c, &lay, P * dm.N));
     int st = dev_alloc(c, &ok, P);
-    if (st == RP_OK) st = dev_alloc(c, &best, 3);
     if (st == RP_OK) st = rp_launch_seed_trials(c, choice_width, lay, ok);
-    if (st == RP_OK) st = ensure_eval_scratch(c, P, false);
-    if (st == RP_OK) st = rp_launch_cells_from_layouts(c, lay, (int)P, c->d_eval_cells);
-    c->cur = 0;
-    if (st == RP_OK) st = rp_launch_eval(c, c->d_eval_cells, (int)P, c->d_W, c->buf[0].blob, c->d_eval_score, nullptr);
-    if (st == RP_OK) {           // member m owns cell m and works on in it
-        k_iota<<<(int)((P + 255) / 256), 256, 0, c->stream>>>(c->d_wloc, (int)P, 0);
-        k_iota<<<(int)((P + 255) / 256), 256, 0, c->stream>>>(c->d_wloc_next, (int)P, 0);
-        g_rp_launches += 2;
-    }
-    if (st == RP_OK) st = rp_launch_pick_best(c, c->d_eval_score, lay, (int)P, best);
+    if (st == RP_OK) st = install_population(c, lay);
     int *h_ok = (int *)malloc(sizeof(int) * P);
     cudaError_t e = cudaSuccess;
     if (st == RP_OK) {
         e = cudaMemcpyAsync(h_ok, ok, sizeof(int) * P, cudaMemcpyDeviceToHost, c->stream);
-        if (e == cudaSuccess) e = cudaMemcpyAsync(c->d_seed_score, best, sizeof(i64) * 3, cudaMemcpyDeviceToDevice, c->stream);
         if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
     }
     int own = 0;
     if (st == RP_OK && e == cudaSuccess) for (size_t j = 0; j < P; ++j) own += h_ok[j];
     free(h_ok);
-    dev_free(c, lay); dev_free(c, ok); dev_free(c, best);
+    dev_free(c, lay); dev_free(c, ok);
     if (e != cudaSuccess) { g_rp_last_cuda_error = (int)e; return RP_ERR_CUDA; }
     RP_TRY(st);
     if (n_own) *n_own = own;
+    return RP_OK;
+}
+
+__global__ void k_count_changed(const int *__restrict__ a, const int *__restrict__ b, int N, int *__restrict__ out)
+{
+    __shared__ int diff;
+    if (threadIdx.x == 0) diff = 0;
+    __syncthreads();
+    int d = 0;
+    for (int i = threadIdx.x; i < N; i += blockDim.x) d |= (a[(size_t)blockIdx.x * N + i] != b[(size_t)blockIdx.x * N + i]);
+    if (d) diff = 1;
+    __syncthreads();
+    if (threadIdx.x == 0 && diff) atomicAdd(out, 1);
+}
+
+extern "C" int rp_pair_population(rp_ctx *c, int32_t choice_width, int32_t *n_changed)
+{
+    if (!c) return RP_ERR_ARG;
+    if (c->stage != 3) return RP_ERR_STATE;          // after rp_pack_rows, before rp_anneal
+    if (choice_width < 1 || choice_width > 32) return RP_ERR_ARG;
+    const RpDims &dm = c->dm;
+    const size_t P = (size_t)c->Ppop;
+    int *lay = nullptr, *out = nullptr, *prof = nullptr, *cnt = nullptr;
+    RP_TRY(dev_alloc(c, &lay, P * dm.N));
+    int st = dev_alloc(c, &out, P * dm.N);
+    if (st == RP_OK) st = dev_alloc(c, &cnt, 1);
+    const int batch = (int)(P - 1 < 1024 ? P - 1 : 1024);          // members paired per launch (bounds the scratch)
+    if (st == RP_OK && batch > 0) st = dev_alloc(c, &prof, (size_t)batch * dm.K * dm.LP);
+    cudaError_t e = cudaSuccess;
+    if (st == RP_OK) {
+        k_gather_cells<<<c->Ppop, 256, 0, c->stream>>>(c->buf[c->cur].blob, c->bl, c->d_anc, dm.N, nullptr, lay);
+        ++g_rp_launches;
+        e = cudaMemcpyAsync(out, lay, sizeof(int) * dm.N, cudaMemcpyDeviceToDevice, c->stream);     // member 0 stays
+        if (e == cudaSuccess) e = cudaMemsetAsync(cnt, 0, sizeof(int), c->stream);
+    }
+    for (int first = 1; st == RP_OK && e == cudaSuccess && first < (int)P; first += batch) {
+        const int count = (int)P - first < batch ? (int)P - first : batch;
+        st = rp_launch_edp_pair(c, lay, out, prof, first, count, choice_width);
+    }
+    if (st == RP_OK && e == cudaSuccess) {
+        k_count_changed<<<c->Ppop, 256, 0, c->stream>>>(lay, out, dm.N, cnt);
+        ++g_rp_launches;
+        st = install_population(c, out);
+    }
+    int h_cnt = 0;
+    if (st == RP_OK && e == cudaSuccess) {
+        e = cudaMemcpyAsync(&h_cnt, cnt, sizeof(int), cudaMemcpyDeviceToHost, c->stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+    }
+    dev_free(c, lay); dev_free(c, out); dev_free(c, prof); dev_free(c, cnt);
+    if (e != cudaSuccess) { g_rp_last_cuda_error = (int)e; return RP_ERR_CUDA; }
+    RP_TRY(st);
+    if (n_changed) *n_changed = h_cnt;
     return RP_OK;
 }
 

@@ -175,6 +175,7 @@ int rp_launch_eval(rp_ctx *c, const unsigned short *cells, int n, int *W_out, ch
                    i64 *score_out, double *f64_out);
 int rp_launch_build_static(rp_ctx *c);
 int rp_launch_seed_trials(rp_ctx *c, int width, int *layouts, int *ok);
+int rp_launch_edp_pair(rp_ctx *c, const int *lay_in, int *lay_out, int *prof, int first, int count, int width);
 int rp_launch_pick_best(rp_ctx *c, const i64 *scores, const int *layouts, int n, i64 *best_score_out);
 int rp_get_pool(int device, cudaMemPool_t *out);     // the library's stream-ordered pool of a device
 void rp_make_layouts(const RpDims &dm, RpBlob *bl, RpStatic *sl);

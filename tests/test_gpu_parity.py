@@ -291,6 +291,50 @@ def test_randomized_seed_population(case, width):
     rp.rp_destroy(ctx)
 
 
+@pytest.mark.parametrize("case,width", [("shared", 1), ("shared", 4), ("interleaved", 3), ("one_shard", 8),
+                                        ("identity", 4), ("medium", 4), ("no_trials", 2)])
+def test_edp_aware_pairing(case, width):
+    """Algorithm 2's pairing operator on a randomized seed population: every member's re-paired
+    layout, the scores, the incumbent and the annealing that starts from it, against the oracle."""
+    pop, edp, min_rows = 40, None, 3
+    if case == "medium":
+        w = make_window("medium")
+        min_rows = 0
+    elif case in ("shared", "no_trials"):
+        w = make_window(custom_spec("pair_shared", 96, 5, 16, 2, 4096, 4, 4, pop, 400, data_seed=15))
+        edp = [0, 0, 1, 1]
+    elif case == "interleaved":
+        w = make_window(custom_spec("pair_inter", 120, 7, 24, 3, 4096, 6, 6, pop, 400, data_seed=16))
+        edp, min_rows = [0, 1, 2, 0, 1, 2], 2
+    elif case == "one_shard":
+        w = make_window(custom_spec("pair_one", 64, 2, 8, 1, 2048, 4, 8, pop, 400, data_seed=17))
+        edp = [0, 0, 0, 0]
+    else:
+        w = make_window(custom_spec("pair_ident", 77, 3, 12, 2, 3000, 3, 3, pop, 400, data_seed=18))
+        min_rows = 4
+    s = w.spec
+    ref = oracle_front(w, edp, min_rows)
+    ctx = load(w, pop=pop, edp=edp, min_rows=min_rows)
+    check_front(w, ctx, ref)
+    if case == "no_trials":                 # straight on the length-only seed: the x_paired candidates
+        lays = np.tile(ref["seed"], (pop, 1)).astype(np.int32)
+    else:
+        lays, _ = oracle.seed_trials(w.lengths, ref["seed"], ref["R"], s.token_cap, s.dp_width, pop, 4, s.anneal_seed)
+        rp.rp_seed_population(ctx, 4)
+    want = oracle.edp_pair(ref["q"], lays, ref["R"], s.dp_width, width, s.anneal_seed, edp)
+    changed = rp.rp_pair_population(ctx, width)
+    assert changed == int((want != lays).any(axis=1).sum())
+    assert (rp.rp_debug_dump(ctx, "POPULATION", (pop, s.n_samples), np.int32) == want).all()
+    ev = oracle.eval_layouts(w.lengths, ref["q"], want, ref["R"], s.token_cap, s.dp_width, edp, s.alpha, s.beta)
+    fx, _ = rp.rp_eval_population(ctx)
+    assert (fx == ev["score"]).all()
+    best = min(range(pop), key=lambda j: (tuple(ev["score"][j]), j))
+    layout, bfx, _ = rp.rp_best(ctx)
+    assert (layout == want[best]).all() and tuple(bfx) == tuple(ev["score"][best])
+    check_anneal(w, ctx, ref, edp, pop, 3, 40, t_ratio=0.5, check_members=2, init=want)
+    rp.rp_destroy(ctx)
+
+
 def test_fuzz_random_small_windows():
     """Random shapes and search parameters (rank counts 1..48 including non powers of two, shared
     and interleaved shards, swap-only and relocation-only proposals, unguided and fully guided,
