@@ -40,6 +40,7 @@ def lib():
         _lib.orc_check_window.restype = C.c_int64
         _lib.orc_pack_ffd.restype = C.c_int32
         _lib.orc_anneal.restype = C.c_int32
+        _lib.orc_coassign_q20.restype = C.c_int64
         _lib.orc_accept_uphill.restype = C.c_int32
         _lib.orc_accept_uphill.argtypes = [C.c_int64, C.c_int64, C.c_int64, C.c_uint64, C.c_uint32]
     return _lib
@@ -168,6 +169,54 @@ def edp_pair(q, layouts, R: int, D: int, width: int, seed: int, edp_of_dp=None) 
     lib().orc_edp_pair(C.c_int32(N), C.c_int32(L), C.c_int32(P), C.c_int32(D), C.c_int32(G), C.c_int32(R),
                        C.c_int32(width), C.c_uint64(seed), _p(q), _p(edp), C.c_int32(Ppop), _p(lay))
     return lay
+
+
+def canonicalize(layout, R: int, D: int, edp_of_dp=None) -> np.ndarray:
+    lay = _i32(layout)
+    edp = np.arange(D, dtype=np.int32) if edp_of_dp is None else _i32(edp_of_dp)
+    out = np.zeros_like(lay)
+    lib().orc_canonicalize(C.c_int32(lay.shape[0]), C.c_int32(D), C.c_int32(int(edp.max()) + 1), C.c_int32(R),
+                           _p(edp), _p(lay), _p(out))
+    return out
+
+
+def coassign_q20(la, lb) -> int:
+    la, lb = _i32(la), _i32(lb)
+    return int(lib().orc_coassign_q20(C.c_int32(la.shape[0]), _p(la), _p(lb)))
+
+
+def sw_sketch(lengths, q, layout, R: int, C_cap: int, D: int, top_k: int, nproj: int, seed: int, edp_of_dp=None):
+    """Sorted projections [nproj][R] of the row features."""
+    t, q, lay = _i32(lengths), _i32(q), _i32(layout)
+    _, L, P = q.shape
+    edp = np.arange(D, dtype=np.int32) if edp_of_dp is None else _i32(edp_of_dp)
+    phi = np.zeros((nproj, R), np.int64)
+    lib().orc_sw_sketch(C.c_int32(t.shape[0]), C.c_int32(L), C.c_int32(P), C.c_int32(D), C.c_int32(int(edp.max()) + 1),
+                        C.c_int32(R), C.c_int32(C_cap), C.c_int32(top_k), C.c_int32(nproj), C.c_uint64(seed),
+                        _p(t), _p(q), _p(edp), _p(lay), _p(phi))
+    return phi
+
+
+def select_population(lengths, q, layouts, scores, R: int, C_cap: int, D: int, top_k: int, nproj: int, eta_q16: int,
+                      seed: int, edp_of_dp=None, want_dist: bool = False):
+    """CanonicalMap + QualityDiversitySelect: returns dict(layouts, n_distinct, order[, dist])."""
+    t, q = _i32(lengths), _i32(q)
+    lay = _i32(layouts).copy()
+    sc = np.ascontiguousarray(scores, dtype=np.int64)
+    Ppop, N = lay.shape
+    _, L, P = q.shape
+    edp = np.arange(D, dtype=np.int32) if edp_of_dp is None else _i32(edp_of_dp)
+    nd = C.c_int32(0)
+    order = np.zeros(Ppop, np.int32)
+    dist = np.zeros((Ppop, Ppop), np.int64) if want_dist else None
+    lib().orc_select_population(C.c_int32(N), C.c_int32(L), C.c_int32(P), C.c_int32(D), C.c_int32(int(edp.max()) + 1),
+                                C.c_int32(R), C.c_int32(C_cap), C.c_int32(top_k), C.c_int32(nproj), C.c_int64(eta_q16),
+                                C.c_uint64(seed), _p(t), _p(q), _p(edp), C.c_int32(Ppop), _p(sc), _p(lay),
+                                C.byref(nd), _p(order), _p(dist))
+    out = dict(layouts=lay, n_distinct=int(nd.value), order=order)
+    if want_dist:
+        out["dist"] = dist
+    return out
 
 
 # ---- scoring ----------------------------------------------------------------------------

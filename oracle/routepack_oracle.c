@@ -1150,3 +1150,208 @@ void orc_edp_pair(int32_t N, int32_t L, int32_t P, int32_t D, int32_t G, int32_t
     }
     free(prof); free(V); free(peak); free(order); free(slot_of); free(empty); free(rank); free(kd); free(kp);
 }
+
+/* ------------------------------------------------------------------------------------ */
+/* Canonicalize / CanonicalMap / QualityDiversitySelect (Section 4.1.1, Algorithm 2).    */
+/*                                                                                        */
+/* Canonicalize: layouts that differ only by the order of rows, or by which of the       */
+/* exchangeable DP slots of one EDP shard a cell sits in, get the same signature.  A cell */
+/* is named by its smallest sample id (sample order inside a cell is not represented at   */
+/* all); inside a row the cells of one shard are listed by that name over the shard's     */
+/* slots in increasing slot order; rows are listed by their smallest sample id.  Any      */
+/* other total order would give the same classes.                                         */
+/* ------------------------------------------------------------------------------------ */
+void orc_canonicalize(int32_t N, int32_t D, int32_t G, int32_t R, const int32_t *edp_of_dp,
+                      const int32_t *lay, int32_t *canon)
+{
+    const int32_t K = R * D;
+    int32_t *name = (int32_t *)malloc(sizeof(int32_t) * K);       /* smallest sample of the cell */
+    int32_t *new_d = (int32_t *)malloc(sizeof(int32_t) * K);      /* slot inside the row */
+    int32_t *rname = (int32_t *)malloc(sizeof(int32_t) * R);
+    int32_t *new_r = (int32_t *)malloc(sizeof(int32_t) * R);
+    for (int32_t c = 0; c < K; ++c) name[c] = N;
+    for (int32_t i = N - 1; i >= 0; --i) name[lay[i]] = i;
+    for (int32_t r = 0; r < R; ++r) {
+        rname[r] = N;
+        for (int32_t d = 0; d < D; ++d) if (name[r * D + d] < rname[r]) rname[r] = name[r * D + d];
+        for (int32_t g = 0; g < G; ++g)
+            for (int32_t d = 0; d < D; ++d) {
+                if (edp_of_dp[d] != g) continue;
+                /* position of cell (r, d) among the cells of shard g in this row, by name */
+                int32_t pos = 0;
+                for (int32_t d2 = 0; d2 < D; ++d2)
+                    if (edp_of_dp[d2] == g && name[r * D + d2] < name[r * D + d]) ++pos;
+                /* the pos-th slot of the shard */
+                int32_t seen = 0, target = -1;
+                for (int32_t d2 = 0; d2 < D && target < 0; ++d2)
+                    if (edp_of_dp[d2] == g) { if (seen == pos) target = d2; ++seen; }
+                new_d[r * D + d] = target;
+            }
+    }
+    for (int32_t r = 0; r < R; ++r) {
+        int32_t pos = 0;
+        for (int32_t r2 = 0; r2 < R; ++r2) if (rname[r2] < rname[r]) ++pos;
+        new_r[r] = pos;
+    }
+    for (int32_t i = 0; i < N; ++i) canon[i] = new_r[lay[i] / D] * D + new_d[lay[i]];
+    free(name); free(new_d); free(rname); free(new_r);
+}
+
+/* Co-assignment distance of two labelings in Q20: 1 - |pairs together in both| / |pairs
+ * together in either| (0 when neither puts any two samples together). */
+int64_t orc_coassign_q20(int32_t N, const int32_t *la, const int32_t *lb)
+{
+    int64_t pa = 0, pb = 0, both = 0;
+    for (int32_t i = 0; i < N; ++i)
+        for (int32_t i2 = i + 1; i2 < N; ++i2) {
+            const int sa = la[i] == la[i2], sb = lb[i] == lb[i2];
+            pa += sa; pb += sb; both += (sa && sb);
+        }
+    const int64_t uni = pa + pb - both;
+    if (uni == 0) return 0;
+    return ((int64_t)1 << 20) - (both << 20) / uni;
+}
+
+/* Sorted projections of the row features (the Sliced-Wasserstein sketch), phi [nproj][R].
+ * Row features in Q16 (F = 2 + G*L of them):
+ *   tokens / (C*D),  sum of squared lengths / (C*C*D),  and for every shard g and layer l the
+ *   busiest rank of row-shard (r, g), max_p W[r][g][l][p] / (k * C * |D_g|).
+ * Projection k has entries +1 / -1: -1 where the top bit of Philox(f, 0, k, 7).x is set. */
+void orc_sw_sketch(int32_t N, int32_t L, int32_t P, int32_t D, int32_t G, int32_t R, int32_t C, int32_t k,
+                   int32_t nproj, uint64_t seed, const int32_t *t, const int32_t *q, const int32_t *edp_of_dp,
+                   const int32_t *lay, int64_t *phi)
+{
+    const int32_t F = 2 + G * L;
+    const size_t LP = (size_t)L * P;
+    int64_t *H = (int64_t *)calloc((size_t)R * F, sizeof(int64_t));
+    int64_t *W = (int64_t *)calloc((size_t)R * G * LP, sizeof(int64_t));
+    int64_t *Tr = (int64_t *)calloc(R, sizeof(int64_t)), *Qr = (int64_t *)calloc(R, sizeof(int64_t));
+    int32_t *ng = (int32_t *)calloc(G, sizeof(int32_t));
+    for (int32_t d = 0; d < D; ++d) ng[edp_of_dp[d]] += 1;
+    for (int32_t i = 0; i < N; ++i) {
+        const int32_t r = lay[i] / D, g = edp_of_dp[lay[i] % D];
+        Tr[r] += t[i];
+        Qr[r] += (int64_t)t[i] * t[i];
+        for (size_t x = 0; x < LP; ++x) W[((size_t)r * G + g) * LP + x] += q[(size_t)i * LP + x];
+    }
+    for (int32_t r = 0; r < R; ++r) {
+        H[(size_t)r * F + 0] = (int64_t)(((unsigned __int128)Tr[r] << 16) / ((unsigned __int128)C * D));
+        H[(size_t)r * F + 1] = (int64_t)(((unsigned __int128)Qr[r] << 16) / ((unsigned __int128)C * C * D));
+        for (int32_t g = 0; g < G; ++g)
+            for (int32_t l = 0; l < L; ++l) {
+                int64_t m = 0;
+                for (int32_t p = 0; p < P; ++p) {
+                    const int64_t v = W[((size_t)r * G + g) * LP + (size_t)l * P + p];
+                    if (v > m) m = v;
+                }
+                H[(size_t)r * F + 2 + g * L + l] = (m << 16) / ((int64_t)k * C * ng[g]);
+            }
+    }
+    for (int32_t kk = 0; kk < nproj; ++kk) {
+        int64_t *ph = phi + (size_t)kk * R;
+        for (int32_t r = 0; r < R; ++r) ph[r] = 0;
+        for (int32_t f = 0; f < F; ++f) {
+            uint32_t X[4];
+            draw(seed, (uint32_t)f, 0u, (uint32_t)kk, 7u, X);
+            const int64_t sgn = (X[0] >> 31) ? -1 : 1;
+            for (int32_t r = 0; r < R; ++r) ph[r] += sgn * H[(size_t)r * F + f];
+        }
+        for (int32_t x = 1; x < R; ++x) {              /* insertion sort, ascending */
+            int64_t v = ph[x];
+            int32_t y = x;
+            while (y > 0 && ph[y - 1] > v) { ph[y] = ph[y - 1]; --y; }
+            ph[y] = v;
+        }
+    }
+    free(H); free(W); free(Tr); free(Qr); free(ng);
+}
+
+/* Plan distance in Q20 units (0 .. about 3 * 2^20): cell co-assignment + row co-assignment +
+ * sketch distance floor(16 * sum_k sum_r |phi_k(x)[r] - phi_k(y)[r]| / (nproj * R * F)).
+ * The paper names the three ingredients but not how they are mixed: equal weights here. */
+int64_t orc_plan_distance(int32_t N, int32_t D, int32_t R, int32_t F, int32_t nproj, const int32_t *la,
+                          const int32_t *lb, const int64_t *phia, const int64_t *phib)
+{
+    int32_t *ra = (int32_t *)malloc(sizeof(int32_t) * N), *rb = (int32_t *)malloc(sizeof(int32_t) * N);
+    for (int32_t i = 0; i < N; ++i) { ra[i] = la[i] / D; rb[i] = lb[i] / D; }
+    int64_t d = orc_coassign_q20(N, la, lb) + orc_coassign_q20(N, ra, rb);
+    int64_t s = 0;
+    for (size_t x = 0; x < (size_t)nproj * R; ++x) s += phia[x] > phib[x] ? phia[x] - phib[x] : phib[x] - phia[x];
+    d += (s * 16) / ((int64_t)nproj * R * F);
+    free(ra); free(rb);
+    return d;
+}
+
+/* CanonicalMap + QualityDiversitySelect over the population as the candidate set.
+ *  - members with the same signature form one class; its representative has the lowest score
+ *    (lexicographic), ties by lower member index;
+ *  - the selection starts from the representative with the lowest score and then repeatedly
+ *    takes the representative x that maximises  min_{y selected} d(x, y) - (eta * delta0(x)),
+ *    delta0(x) = floor((S0(x) - S0*) * 2^20 / S0*) the primary-score gap to the winner in Q20,
+ *    eta given in Q16, ties by lower member index;
+ *  - new member m is the (m mod n_distinct)-th selected representative.
+ * order [Ppop]: selected member indices (first *n_distinct valid); layouts are rewritten.
+ * dist (nullable) [Ppop][Ppop]: plan distances between members (all pairs). */
+void orc_select_population(int32_t N, int32_t L, int32_t P, int32_t D, int32_t G, int32_t R, int32_t C, int32_t k,
+                           int32_t nproj, int64_t eta_q16, uint64_t seed, const int32_t *t, const int32_t *q,
+                           const int32_t *edp_of_dp, int32_t Ppop, const int64_t *scores, int32_t *layouts,
+                           int32_t *n_distinct, int32_t *order, int64_t *dist)
+{
+    const int32_t F = 2 + G * L;
+    int32_t *canon = (int32_t *)malloc(sizeof(int32_t) * (size_t)Ppop * N);
+    int64_t *phi = (int64_t *)malloc(sizeof(int64_t) * (size_t)Ppop * nproj * R);
+    int32_t *rep = (int32_t *)malloc(sizeof(int32_t) * Ppop), *sel = (int32_t *)calloc(Ppop, sizeof(int32_t));
+    int64_t *mind = (int64_t *)malloc(sizeof(int64_t) * Ppop), *pen = (int64_t *)malloc(sizeof(int64_t) * Ppop);
+    for (int32_t j = 0; j < Ppop; ++j) {
+        orc_canonicalize(N, D, G, R, edp_of_dp, layouts + (size_t)j * N, canon + (size_t)j * N);
+        orc_sw_sketch(N, L, P, D, G, R, C, k, nproj, seed, t, q, edp_of_dp, layouts + (size_t)j * N,
+                      phi + (size_t)j * nproj * R);
+    }
+#define LEXLT(a, b) ((a)[0] != (b)[0] ? (a)[0] < (b)[0] : ((a)[1] != (b)[1] ? (a)[1] < (b)[1] : (a)[2] < (b)[2]))
+    for (int32_t j = 0; j < Ppop; ++j) {
+        rep[j] = 1;
+        for (int32_t o = 0; o < Ppop && rep[j]; ++o) {
+            if (o == j || memcmp(canon + (size_t)j * N, canon + (size_t)o * N, sizeof(int32_t) * N) != 0) continue;
+            const int64_t *sj = scores + 3 * (size_t)j, *so = scores + 3 * (size_t)o;
+            if (LEXLT(so, sj) || (!LEXLT(sj, so) && o < j)) rep[j] = 0;
+        }
+    }
+    if (dist)
+        for (int32_t a = 0; a < Ppop; ++a)
+            for (int32_t b = 0; b < Ppop; ++b)
+                dist[(size_t)a * Ppop + b] = orc_plan_distance(N, D, R, F, nproj, layouts + (size_t)a * N, layouts + (size_t)b * N,
+                                                               phi + (size_t)a * nproj * R, phi + (size_t)b * nproj * R);
+    int32_t nd = 0, best = -1;
+    for (int32_t j = 0; j < Ppop; ++j) {
+        if (!rep[j]) continue;
+        ++nd;
+        if (best < 0 || LEXLT(scores + 3 * (size_t)j, scores + 3 * (size_t)best)) best = j;
+    }
+    const int64_t s0 = scores[3 * (size_t)best];
+    for (int32_t j = 0; j < Ppop; ++j)
+        pen[j] = s0 > 0 ? (int64_t)(((unsigned __int128)(((unsigned __int128)(uint64_t)(scores[3 * (size_t)j] - s0) << 20) / (uint64_t)s0)
+                                     * (unsigned __int128)(uint64_t)eta_q16) >> 16) : 0;
+    int32_t last = best;
+    for (int32_t n = 0; n < nd; ++n) {
+        order[n] = last;
+        sel[last] = 1;
+        int32_t nxt = -1;
+        int64_t bestv = 0;
+        for (int32_t j = 0; j < Ppop; ++j) {
+            if (!rep[j] || sel[j]) continue;
+            const int64_t dj = orc_plan_distance(N, D, R, F, nproj, layouts + (size_t)j * N, layouts + (size_t)last * N,
+                                                 phi + (size_t)j * nproj * R, phi + (size_t)last * nproj * R);
+            if (n == 0 || dj < mind[j]) mind[j] = dj;
+            const int64_t v = mind[j] - pen[j];
+            if (nxt < 0 || v > bestv) { nxt = j; bestv = v; }
+        }
+        last = nxt;
+    }
+#undef LEXLT
+    int32_t *old = (int32_t *)malloc(sizeof(int32_t) * (size_t)Ppop * N);
+    memcpy(old, layouts, sizeof(int32_t) * (size_t)Ppop * N);
+    for (int32_t m = 0; m < Ppop; ++m) memcpy(layouts + (size_t)m * N, old + (size_t)order[m % nd] * N, sizeof(int32_t) * N);
+    for (int32_t m = nd; m < Ppop; ++m) order[m] = order[m % nd];
+    *n_distinct = nd;
+    free(old); free(canon); free(phi); free(rep); free(sel); free(mind); free(pen);
+}

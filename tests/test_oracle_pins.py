@@ -739,3 +739,133 @@ def test_edp_pair_sampling_ranks_decay_by_halves():
     freq = np.bincount(first, minlength=K) / (n - 1)
     assert freq[3:].sum() == 0
     assert abs(freq[0] - 0.5) < 0.03 and abs(freq[1] - 0.25) < 0.03 and abs(freq[2] - 0.25) < 0.03
+
+
+# ---- Canonicalize / CanonicalMap / QualityDiversitySelect (Section 4.1.1) -------------------
+def _small_population(seed=23, pop=20, edp=(0, 0, 1, 1)):
+    w = hetero_window(N=60, L=3, E=8, k=2, C=4096, D=4, P=4, seed=seed)
+    s, t = w.spec, w.lengths
+    pi, _ = oracle.lpt(oracle.aggregate(w.demand), s.ep_width)
+    q = oracle.project(w.demand, pi, s.ep_width)
+    R, _, seed_lay = oracle.pack_ffd(t, s.token_cap, s.dp_width, min_rows=3)
+    lays, _ = oracle.seed_trials(t, seed_lay, R, s.token_cap, s.dp_width, pop, 4, seed=9)
+    return w, q, R, lays, list(edp)
+
+
+def test_canonicalize_by_hand_and_its_symmetries():
+    # two rows of two exchangeable slots; cells {0,4} {1,5} in row 1 and {2} {3} in row 0, listed backwards
+    assert oracle.canonicalize([3, 2, 1, 0, 3, 2], 2, 2, [0, 0]).tolist() == [0, 1, 2, 3, 0, 1]
+    # slots of different shards are not exchangeable: only the rows are reordered
+    assert oracle.canonicalize([3, 2, 1, 0, 3, 2], 2, 2, [0, 1]).tolist() == [1, 0, 3, 2, 1, 0]
+    w, q, R, lays, edp = _small_population()
+    s, t = w.spec, w.lengths
+    D = s.dp_width
+    rng = np.random.default_rng(1)
+    for j in range(6):
+        x = lays[j]
+        cx = oracle.canonicalize(x, R, D, edp)
+        assert (oracle.canonicalize(cx, R, D, edp) == cx).all()                   # idempotent
+        # the canonical form is the same plan: same co-assignment, same score
+        assert oracle.coassign_q20(x, cx) == 0 and oracle.coassign_q20(x // D, cx // D) == 0
+        ex = oracle.eval_layouts(t, q, np.stack([x, cx]), R, s.token_cap, D, edp, s.alpha, s.beta)["score"]
+        assert (ex[0] == ex[1]).all()
+        # every row permutation combined with swaps inside the shards gives the same signature
+        for _ in range(5):
+            rows = rng.permutation(R)
+            slot = np.arange(D)
+            for g in set(edp):
+                ds = [d for d in range(D) if edp[d] == g]
+                slot[ds] = rng.permutation(ds)
+            y = rows[x // D] * D + slot[x % D]
+            assert (oracle.canonicalize(y, R, D, edp) == cx).all()
+        # moving a cell across shards changes the plan, hence the signature
+        y = (x // D) * D + np.array([2, 1, 0, 3])[x % D]
+        assert (oracle.canonicalize(y, R, D, edp) != cx).any()
+
+
+def test_coassignment_distance_special_cases():
+    assert oracle.coassign_q20([0, 0, 1, 1], [0, 0, 0, 1]) == 786432        # 1 common pair of 4: 1 - 1/4
+    assert oracle.coassign_q20([0, 0, 1, 1], [5, 5, 9, 9]) == 0             # same partition, other names
+    assert oracle.coassign_q20([0, 0, 1, 1], [0, 1, 0, 1]) == 1 << 20       # no common pair
+    assert oracle.coassign_q20([0, 1, 2, 3], [3, 2, 1, 0]) == 0             # nobody together in either
+    rng = np.random.default_rng(3)
+    a, b = rng.integers(0, 5, 40), rng.integers(0, 7, 40)
+    assert oracle.coassign_q20(a, b) == oracle.coassign_q20(b, a)
+    # against the contingency-table form of the same count
+    tab = np.zeros((5, 7), np.int64)
+    np.add.at(tab, (a, b), 1)
+    both = int((tab * (tab - 1) // 2).sum())
+    pa = int((tab.sum(1) * (tab.sum(1) - 1) // 2).sum())
+    pb = int((tab.sum(0) * (tab.sum(0) - 1) // 2).sum())
+    assert oracle.coassign_q20(a, b) == (1 << 20) - (both << 20) // (pa + pb - both)
+
+
+def test_sketch_is_row_order_invariant_and_matches_a_plain_restatement():
+    w, q, R, lays, edp = _small_population()
+    s, t = w.spec, w.lengths
+    D, nproj = s.dp_width, 5
+    x = lays[3]
+    phi = oracle.sw_sketch(t, q, x, R, s.token_cap, D, s.top_k, nproj, 77, edp)
+    assert (np.diff(phi, axis=1) >= 0).all()
+    rows = np.random.default_rng(2).permutation(R)
+    y = rows[x // D] * D + x % D
+    assert (oracle.sw_sketch(t, q, y, R, s.token_cap, D, s.top_k, nproj, 77, edp) == phi).all()
+    # features and projections restated with numpy
+    G, L = max(edp) + 1, q.shape[1]
+    W = np.zeros((R, G, L, q.shape[2]), np.int64)
+    np.add.at(W, (x // D, np.asarray(edp)[x % D]), q)
+    Tr = np.bincount(x // D, weights=t, minlength=R).astype(np.int64)
+    Qr = np.bincount(x // D, weights=t.astype(np.int64) ** 2, minlength=R).astype(np.int64)
+    H = np.zeros((R, 2 + G * L), np.int64)
+    H[:, 0] = (Tr << 16) // (s.token_cap * D)
+    H[:, 1] = (Qr << 16) // (s.token_cap * s.token_cap * D)
+    ng = np.bincount(edp, minlength=G)
+    for g in range(G):
+        H[:, 2 + g * L: 2 + (g + 1) * L] = (W[:, g].max(-1) << 16) // (s.top_k * s.token_cap * ng[g])
+    for kk in range(nproj):
+        sign = np.array([-1 if oracle.philox4x32_10((f, 0, kk, 7), (77, 0))[0] >> 31 else 1 for f in range(H.shape[1])])
+        assert (np.sort(H @ sign) == phi[kk]).all()
+
+
+def test_canonical_map_and_quality_diversity_selection():
+    w, q, R, lays, edp = _small_population(pop=24)
+    s, t = w.spec, w.lengths
+    D = s.dp_width
+    rng = np.random.default_rng(8)
+    pop = lays.copy()
+    # members 20..23 are disguised copies (row order and exchangeable slots changed) of members 3, 3, 7, 0
+    for dst, src in ((20, 3), (21, 3), (22, 7), (23, 0)):
+        rows = rng.permutation(R)
+        pop[dst] = rows[lays[src] // D] * D + np.array([1, 0, 3, 2])[lays[src] % D]
+    sc = oracle.eval_layouts(t, q, pop, R, s.token_cap, D, edp, s.alpha, s.beta)["score"]
+    sig = [oracle.canonicalize(x, R, D, edp).tobytes() for x in pop]
+    classes = {}
+    for j, k in enumerate(sig):
+        classes.setdefault(k, []).append(j)
+    for eta in (0, 1 << 16, 1 << 26):
+        out = oracle.select_population(t, q, pop, sc, R, s.token_cap, D, s.top_k, 6, eta, 5, edp, want_dist=True)
+        nd, order, dist = out["n_distinct"], out["order"], out["dist"]
+        assert nd == len(classes) <= 20
+        # one representative per class: lowest score, then lowest index (a copy scores like its source)
+        reps = sorted(min(js, key=lambda j: (tuple(sc[j]), j)) for js in classes.values())
+        assert sorted(order[:nd].tolist()) == reps
+        assert all(j < 20 for j in reps)
+        # starts from the exact-score winner; members repeat cyclically once all are used
+        assert order[0] == min(reps, key=lambda j: (tuple(sc[j]), j))
+        assert (order[nd:] == np.resize(order[:nd], len(order))[nd:]).all()
+        assert all((out["layouts"][m] == pop[order[m]]).all() for m in range(len(order)))
+        # distances: symmetric, zero on the diagonal and between a plan and its disguised copy
+        assert (dist == dist.T).all() and (np.diag(dist) == 0).all() and dist[20, 3] == 0 and dist[23, 0] == 0
+        # every pick maximises (distance to the nearest selected - penalty) among the remaining ones
+        s0 = int(sc[order[0]][0])
+        pen = {j: ((((int(sc[j][0]) - s0) << 20) // s0) * eta) >> 16 for j in reps}
+        chosen = [int(order[0])]
+        for n in range(1, nd):
+            rest = [j for j in reps if j not in chosen]
+            val = {j: min(int(dist[j, y]) for y in chosen) - pen[j] for j in rest}
+            top = max(val.values())
+            assert int(order[n]) == min(j for j in rest if val[j] == top)
+            chosen.append(int(order[n]))
+    # a large eta turns the order into the score order (by primary score)
+    prim = [int(sc[j][0]) for j in order[:nd]]
+    assert prim == sorted(prim)
