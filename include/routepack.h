@@ -143,6 +143,29 @@ int rp_seed_population(rp_ctx *ctx, int32_t choice_width, int32_t *n_own);
  * RP_ERR_STATE outside stage 3, RP_ERR_RANGE when the per-member tables exceed shared memory. */
 int rp_pair_population(rp_ctx *ctx, int32_t choice_width, int32_t *n_changed);
 
+/* Canonicalize + CanonicalMap + QualityDiversitySelect with the current population as the
+ * candidate set (Section 4.1.1; Algorithm 2, last lines).  Optional, between rp_pack_rows and
+ * rp_anneal, after the seeding calls above.
+ *   - signature: a cell is named by its smallest sample; inside a row the cells of one EDP shard
+ *     are listed by name over the shard's slots, rows are listed by their smallest sample.  Members
+ *     with equal signatures are the same plan up to row order and exchangeable DP slots; the class
+ *     is represented by its lowest score, then lowest index.
+ *   - the selection starts from the representative with the lowest score and then repeatedly takes
+ *     the one that maximises  (distance to the nearest selected) - ((eta_q16 * gap) >> 16),
+ *     gap = floor((S0 - S0_best) * 2^20 / S0_best), ties by lower index.
+ *   - distance (Q20 units): cell co-assignment + row co-assignment (1 - pairs together in both /
+ *     pairs together in either) + a Sliced-Wasserstein sketch: L1 distance of the sorted projections
+ *     of the Q16 row features (tokens/(C*D), squared lengths/(C*C*D), busiest rank of every (shard,
+ *     layer)/(k*C*slots of the shard)) onto n_proj +-1 vectors (sign f of vector k = top bit of
+ *     Philox(f, 0, k, 7)), times 16 / (n_proj * R * F).
+ *   - new member m = the (m mod n_distinct)-th selected representative.
+ * The paper names the ingredients of the distance, eta, the feature matrix and the projections
+ * without fixing them: the mixing (equal weights), the features and the sign vectors are this
+ * library's reading.  Cost grows with the square of the number of distinct members.
+ *   n_proj in [1, 64]; eta_q16 >= 0; n_distinct HOST out (nullable); order HOST out [P_pop],
+ *   former member index of every new member (nullable). */
+int rp_select_population(rp_ctx *ctx, int32_t n_proj, int64_t eta_q16, int32_t *n_distinct, int32_t *order);
+
 /* Full evaluation of layouts (Section 3.4-3.5: Eqs. cell-token-statistics,
  * stage-aware-attention, row-expert-load, row-expert-cost, lexicographic-score).
  *   layouts [n][N] int32 cell ids, or NULL to score the current population (n = pop_size).
@@ -227,6 +250,8 @@ typedef enum {
     RP_DUMP_TRACE_DIGEST = 13,    /* uint64 [n_levels][P_pop] digest of accepted moves     */
     RP_DUMP_TRACE_ANC = 14,       /* int32 [n_levels-1][P_pop] resampling ancestors        */
     RP_DUMP_TRACE_INCUMBENT = 15, /* int64 [n_levels][3]                                   */
+    RP_DUMP_SELECT_DIST = 17, /* int64 [P_pop][P_pop] plan distances between the representatives
+                                 of the last rp_select_population (0 elsewhere); inspection hook on */
     RP_DUMP_EVAL_W = 16      /* int32 [R][G][L][P] of layout `index` of the last
                                 rp_eval_population call with explicit layouts (n <= 64)    */
 } rp_dump_what;

@@ -22,7 +22,7 @@ STATUS_NAMES = {0: "RP_OK", -1: "RP_ERR_ARG", -2: "RP_ERR_SHAPE", -3: "RP_ERR_CO
                 -8: "RP_ERR_TIMEOUT", -9: "RP_ERR_INVALID_PLAN"}
 RP_OK = 0
 
-EXPORTS = ("rp_window_load", "rp_place_experts", "rp_pack_rows", "rp_seed_population", "rp_pair_population", "rp_eval_population", "rp_eval_layouts_noalloc", "rp_diagnostics", "rp_anneal",
+EXPORTS = ("rp_window_load", "rp_place_experts", "rp_pack_rows", "rp_seed_population", "rp_pair_population", "rp_select_population", "rp_eval_population", "rp_eval_layouts_noalloc", "rp_diagnostics", "rp_anneal",
            "rp_best", "rp_destroy", "rp_release_cached_memory", "rp_strerror", "rp_last_cuda_error", "rp_debug_dump",
            "rp_debug_set_trace",
            "rp_debug_nl2", "rp_debug_exp2neg", "rp_debug_philox", "rp_debug_launch_count")
@@ -82,6 +82,7 @@ def lib():
         L.rp_pack_rows.argtypes = [C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         L.rp_seed_population.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_int32)]
         L.rp_pair_population.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_int32)]
+        L.rp_select_population.argtypes = [C.c_void_p, C.c_int32, C.c_int64, C.POINTER(C.c_int32), C.c_void_p]
         L.rp_eval_population.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
         L.rp_eval_layouts_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
         L.rp_diagnostics.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(rp_diag)]
@@ -196,6 +197,14 @@ def rp_pair_population(ctx: Context, choice_width: int) -> int:
     return int(changed.value)
 
 
+def rp_select_population(ctx: Context, n_proj: int = 8, eta_q16: int = 1 << 16):
+    """CanonicalMap + QualityDiversitySelect over the population; returns (n_distinct, order [P_pop])."""
+    nd = C.c_int32(0)
+    order = np.zeros(ctx.cfg.pop_size, np.int32)
+    _check(lib().rp_select_population(ctx.handle, n_proj, eta_q16, C.byref(nd), _ptr(order)), "rp_select_population")
+    return int(nd.value), order
+
+
 def rp_eval_population(ctx: Context, layouts=None, score_fx=None, score_f64=None):
     n = ctx.cfg.pop_size if layouts is None else int(layouts.shape[0])
     if score_fx is None:
@@ -257,7 +266,7 @@ def rp_release_cached_memory():
 # ---- inspection hooks -------------------------------------------------------------------
 DUMP = dict(LAGG=1, Q=2, SEED_LAYOUT=3, POPULATION=4, W=5, CELL_T=6, CELL_Q=7, CELL_CNT=8, ESUM=9,
             TRACE_TERM=10, TRACE_BEST=11, TRACE_BEST_STEP=12, TRACE_DIGEST=13, TRACE_ANC=14,
-            TRACE_INCUMBENT=15, EVAL_W=16)
+            TRACE_INCUMBENT=15, EVAL_W=16, SELECT_DIST=17)
 
 
 def rp_debug_set_trace(ctx: Context, on: bool = True):

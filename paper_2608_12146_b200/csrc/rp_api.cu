@@ -88,17 +88,6 @@ static void pin_give(void *p)
     g_pin_free.push_back(p);
 }
 
-template <class T>
-static int dev_alloc(rp_ctx *c, T **p, size_t n)
-{
-    *p = nullptr;
-    if (n == 0) n = 1;
-    cudaMemPool_t pool;
-    RP_TRY(rp_get_pool(c->device, &pool));
-    RP_CUDA(cudaMallocFromPoolAsync((void **)p, n * sizeof(T), pool, c->stream));
-    return RP_OK;
-}
-static void dev_free(rp_ctx *c, void *p) { if (p) cudaFreeAsync(p, c->stream); }
 
 static bool is_device_ptr(const void *p)
 {
@@ -123,8 +112,8 @@ static void free_population(rp_ctx *c)
     }
     dev_free(c, c->d_W); dev_free(c, c->d_wloc); dev_free(c, c->d_wloc_next); dev_free(c, c->d_le_scratch);
     c->d_W = nullptr; c->d_wloc = nullptr; c->d_wloc_next = nullptr; c->d_le_scratch = nullptr;
-    dev_free(c, c->d_cand_layout); dev_free(c, c->d_inc_slot);
-    c->d_cand_layout = nullptr; c->d_inc_slot = nullptr;
+    dev_free(c, c->d_cand_layout); dev_free(c, c->d_inc_slot); dev_free(c, c->d_sel_dist);
+    c->d_cand_layout = nullptr; c->d_inc_slot = nullptr; c->d_sel_dist = nullptr;
     dev_free(c, c->d_anc); dev_free(c, c->d_anc_next); dev_free(c, c->d_done); dev_free(c, c->d_term); dev_free(c, c->d_best); dev_free(c, c->d_best_step);
     dev_free(c, c->d_best_nlog); dev_free(c, c->d_digest); dev_free(c, c->d_log); dev_free(c, c->d_F);
     c->d_anc = nullptr; c->d_anc_next = nullptr; c->d_done = nullptr; c->d_term = nullptr; c->d_best = nullptr; c->d_best_step = nullptr;
@@ -583,6 +572,49 @@ extern "C" int rp_pair_population(rp_ctx *c, int32_t choice_width, int32_t *n_ch
     return RP_OK;
 }
 
+extern "C" int rp_select_population(rp_ctx *c, int32_t n_proj, int64_t eta_q16, int32_t *n_distinct, int32_t *order)
+{
+    if (!c) return RP_ERR_ARG;
+    if (c->stage != 3) return RP_ERR_STATE;          // after rp_pack_rows, before rp_anneal
+    if (n_proj < 1 || n_proj > 64 || eta_q16 < 0 || eta_q16 > ((int64_t)1 << 40)) return RP_ERR_ARG;
+    const RpDims &dm = c->dm;
+    if ((double)dm.C * dm.C * dm.D * 65536.0 >= 9.0e18) return RP_ERR_RANGE;      // Q16 row feature of the squared lengths
+    const size_t P = (size_t)c->Ppop;
+    int *lay = nullptr, *out = nullptr, *d_order = nullptr, *d_nd = nullptr;
+    dev_free(c, c->d_sel_dist); c->d_sel_dist = nullptr;
+    RP_TRY(dev_alloc(c, &lay, P * dm.N));
+    int st = dev_alloc(c, &out, P * dm.N);
+    if (st == RP_OK) st = dev_alloc(c, &d_order, P);
+    if (st == RP_OK) st = dev_alloc(c, &d_nd, 1);
+    if (st == RP_OK) st = dev_alloc(c, &c->d_sel_dist, P * P);
+    if (st == RP_OK) {
+        k_gather_cells<<<c->Ppop, 256, 0, c->stream>>>(c->buf[c->cur].blob, c->bl, c->d_anc, dm.N, nullptr, lay);
+        ++g_rp_launches;
+        // exact scores of the members as they stand
+        st = ensure_eval_scratch(c, P, false);
+    }
+    if (st == RP_OK) st = rp_launch_cells_from_layouts(c, lay, (int)P, c->d_eval_cells);
+    if (st == RP_OK) st = rp_launch_eval(c, c->d_eval_cells, (int)P, nullptr, nullptr, c->d_eval_score, nullptr);
+    if (st == RP_OK) st = rp_launch_select(c, lay, out, c->d_eval_score, n_proj, eta_q16, d_order, d_nd, c->d_sel_dist);
+    if (st == RP_OK) st = install_population(c, out);
+    int *h = (int *)malloc(sizeof(int) * (P + 1));
+    cudaError_t e = cudaSuccess;
+    if (st == RP_OK) {
+        e = cudaMemcpyAsync(h, d_order, sizeof(int) * P, cudaMemcpyDeviceToHost, c->stream);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(h + P, d_nd, sizeof(int), cudaMemcpyDeviceToHost, c->stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+    }
+    if (st == RP_OK && e == cudaSuccess) {
+        if (n_distinct) *n_distinct = h[P];
+        if (order) memcpy(order, h, sizeof(int) * P);
+    }
+    free(h);
+    dev_free(c, lay); dev_free(c, out); dev_free(c, d_order); dev_free(c, d_nd);
+    if (!c->trace_on) { dev_free(c, c->d_sel_dist); c->d_sel_dist = nullptr; }      // kept for inspection only
+    if (e != cudaSuccess) { g_rp_last_cuda_error = (int)e; return RP_ERR_CUDA; }
+    return st;
+}
+
 // Per-level integers of the geometric schedule, from IEEE double operations only.
 static void make_schedule(const rp_anneal_params *p, RpLevel *lv)
 {
@@ -785,6 +817,9 @@ extern "C" int rp_debug_dump(rp_ctx *c, int what, int32_t index, void *buf, int6
         case RP_DUMP_EVAL_W:
             if (index < 0 || index >= c->eval_W_n) return RP_ERR_ARG;
             src = c->d_eval_W + (size_t)index * dm.RG * dm.LP; need = sizeof(int) * (size_t)dm.RG * dm.LP; break;
+        case RP_DUMP_SELECT_DIST:
+            if (!c->d_sel_dist) return RP_ERR_STATE;
+            src = c->d_sel_dist; need = sizeof(i64) * P * P; break;
         default: return RP_ERR_ARG;
     }
     if (what >= RP_DUMP_TRACE_TERM && what <= RP_DUMP_TRACE_INCUMBENT && c->trace_levels == 0) { dev_free(c, tmp); return RP_ERR_STATE; }

@@ -139,6 +139,7 @@ struct rp_ctx {
     int *d_inc_layout;         // [N]
     unsigned short *d_cand_layout;   // [P_pop][N] trajectory-best snapshots of the chains (warp-per-candidate kernel)
     int *d_inc_slot;           // [1]
+    i64 *d_sel_dist;           // [P_pop][P_pop] plan distances of the last rp_select_population (inspection hook on)
     i64 *d_inc_score;          // [3]
     // trace of the last rp_anneal call
     int trace_levels;
@@ -180,6 +181,21 @@ int rp_launch_pick_best(rp_ctx *c, const i64 *scores, const int *layouts, int n,
 int rp_get_pool(int device, cudaMemPool_t *out);     // the library's stream-ordered pool of a device
 void rp_make_layouts(const RpDims &dm, RpBlob *bl, RpStatic *sl);
 int rp_launch_cells_from_layouts(rp_ctx *c, const int *layouts, int n, unsigned short *cells);
+// Stream-ordered device memory from the device's pool (n elements of T; freed on the context's stream).
+template <class T>
+static inline int dev_alloc(rp_ctx *c, T **p, size_t n)
+{
+    *p = nullptr;
+    if (n == 0) n = 1;
+    cudaMemPool_t pool;
+    RP_TRY(rp_get_pool(c->device, &pool));
+    RP_CUDA(cudaMallocFromPoolAsync((void **)p, n * sizeof(T), pool, c->stream));
+    return RP_OK;
+}
+static inline void dev_free(rp_ctx *c, void *p) { if (p) cudaFreeAsync(p, c->stream); }
+
+int rp_launch_select(rp_ctx *c, int *lay, int *out, const i64 *score, int n_proj, i64 eta_q16, int *order,
+                     int *n_distinct, i64 *dist);
 bool rp_uses_wpc(const RpDims &dm);
 int rp_launch_anneal_level(rp_ctx *c, int level, int n_levels, const rp_anneal_params *prm, u64 rho_q32, u64 guide_q32);
 int rp_launch_validate(rp_ctx *c);

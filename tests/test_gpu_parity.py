@@ -335,6 +335,60 @@ def test_edp_aware_pairing(case, width):
     rp.rp_destroy(ctx)
 
 
+@pytest.mark.parametrize("case,eta", [("shared", 1 << 16), ("shared", 0), ("interleaved", 1 << 18),
+                                      ("identity", 1 << 16), ("medium", 1 << 14), ("copies", 1 << 16)])
+def test_canonical_map_and_quality_diversity_selection(case, eta):
+    """Algorithm 2's last lines over a seeded and paired population: which members are one plan,
+    the order the selection takes the distinct ones in, the plan distances, the new population,
+    its scores, the incumbent and the annealing that starts from it, against the oracle."""
+    pop, edp, min_rows, n_proj = 40, None, 3, 6
+    if case == "medium":
+        w = make_window("medium")
+        min_rows = 0
+    elif case in ("shared", "copies"):
+        w = make_window(custom_spec("sel_shared", 96, 5, 16, 2, 4096, 4, 4, pop, 400, data_seed=25))
+        edp = [0, 0, 1, 1]
+    elif case == "interleaved":
+        w = make_window(custom_spec("sel_inter", 120, 7, 24, 3, 4096, 6, 6, pop, 400, data_seed=26))
+        edp, min_rows = [0, 1, 2, 0, 1, 2], 2
+    else:
+        w = make_window(custom_spec("sel_ident", 77, 3, 12, 2, 3000, 3, 3, pop, 400, data_seed=28))
+        min_rows = 4
+    s = w.spec
+    ref = oracle_front(w, edp, min_rows)
+    ctx = load(w, pop=pop, edp=edp, min_rows=min_rows)
+    check_front(w, ctx, ref)
+    if case == "copies":            # no trials: every member is the length-only seed, re-paired with width 1 -> few classes
+        lays = np.tile(ref["seed"], (pop, 1)).astype(np.int32)
+        width = 2
+    else:
+        lays, _ = oracle.seed_trials(w.lengths, ref["seed"], ref["R"], s.token_cap, s.dp_width, pop, 4, s.anneal_seed)
+        rp.rp_seed_population(ctx, 4)
+        width = 3
+    lays = oracle.edp_pair(ref["q"], lays, ref["R"], s.dp_width, width, s.anneal_seed, edp)
+    rp.rp_pair_population(ctx, width)
+    sc = oracle.eval_layouts(w.lengths, ref["q"], lays, ref["R"], s.token_cap, s.dp_width, edp, s.alpha, s.beta)["score"]
+    want = oracle.select_population(w.lengths, ref["q"], lays, sc, ref["R"], s.token_cap, s.dp_width, s.top_k, n_proj, eta,
+                                    s.anneal_seed, edp, want_dist=True)
+    nd, order = rp.rp_select_population(ctx, n_proj, eta)
+    assert nd == want["n_distinct"]
+    if case == "copies":
+        assert nd < pop
+    assert (order == want["order"]).all()
+    got = rp.rp_debug_dump(ctx, "POPULATION", (pop, s.n_samples), np.int32)
+    assert (got == want["layouts"]).all()
+    dist = rp.rp_debug_dump(ctx, "SELECT_DIST", (pop, pop), np.int64)
+    reps = sorted(set(order[:nd].tolist()))
+    assert (dist[np.ix_(reps, reps)] == want["dist"][np.ix_(reps, reps)]).all()
+    ev = oracle.eval_layouts(w.lengths, ref["q"], want["layouts"], ref["R"], s.token_cap, s.dp_width, edp, s.alpha, s.beta)
+    fx, _ = rp.rp_eval_population(ctx)
+    assert (fx == ev["score"]).all()
+    layout, bfx, _ = rp.rp_best(ctx)
+    assert (layout == want["layouts"][0]).all() and tuple(bfx) == tuple(ev["score"][0])     # the winner leads
+    check_anneal(w, ctx, ref, edp, pop, 3, 40, t_ratio=0.5, check_members=2, init=want["layouts"])
+    rp.rp_destroy(ctx)
+
+
 def test_fuzz_random_small_windows():
     """Random shapes and search parameters (rank counts 1..48 including non powers of two, shared
     and interleaved shards, swap-only and relocation-only proposals, unguided and fully guided,
