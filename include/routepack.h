@@ -91,7 +91,7 @@ typedef struct {
 
 /* Routing-replay input (Eq. routing-replay-input): creates a context, copies host arrays
  * to the device (device arrays are adopted without a copy and must stay valid until
- * rp_place_experts returns) and checks 1 <= t_i <= C, a >= 0 and sum_e a[i][l][e] == k*t_i.
+ * rp_pack_rows returns: rp_place_experts may leave its work queued on the stream) and checks 1 <= t_i <= C, a >= 0 and sum_e a[i][l][e] == k*t_i.
  *   lengths [N] int32; demand [N][L][E] int32, expert index fastest.
  *   cuda_stream: a cudaStream_t (NULL = default stream).
  * On failure *out is NULL. */
@@ -104,7 +104,9 @@ int rp_window_load(rp_ctx **out, const rp_config *cfg, const int32_t *lengths,
  * id, lower rank id; exactly E/P experts per rank; slot = rank*(E/P) + arrival index), then
  * computes q[i][l][p].
  *   pi [L][E] int32 out, nullable: physical slot of logical expert e.
- *   rank_load [L][P] int64 out, nullable: aggregate load G[l][p] under pi. */
+ *   rank_load [L][P] int64 out, nullable: aggregate load G[l][p] under pi.
+ * Host outputs are complete on return; outputs in device memory (and the call itself when both
+ * are NULL) are only ordered on the context's stream. */
 int rp_place_experts(rp_ctx *ctx, int32_t *pi, int64_t *rank_load);
 
 /* Row count and seed population (Section 3.2; Algorithm 2, first line and last loop).

@@ -314,7 +314,9 @@ extern "C" int rp_place_experts(rp_ctx *c, int32_t *pi, int64_t *rank_load)
     RP_TRY(rp_launch_project(c));
     RP_TRY(copy_out(c, pi, c->d_pi, sizeof(int) * (size_t)dm.L * dm.E));
     RP_TRY(copy_out(c, rank_load, c->d_rank_load, sizeof(i64) * (size_t)dm.L * dm.P));
-    RP_CUDA(cudaStreamSynchronize(c->stream));
+    // Host outputs are complete when the call returns; device outputs are ordered on the stream.
+    if ((pi && !is_device_ptr(pi)) || (rank_load && !is_device_ptr(rank_load)))
+        RP_CUDA(cudaStreamSynchronize(c->stream));
     if (c->stage < 2) c->stage = 2;
     return RP_OK;
 }
