@@ -23,21 +23,31 @@ __device__ __forceinline__ bool first_fit_regs(const RpDims &dm, const u64 *keys
         rem[u] = (u < B && b0 + u < K) ? dm.C - fill[b0 + u] : -1;
         blockmax = max(blockmax, rem[u]);
     }
-    for (int x = K; x < dm.N; ++x) {
-        const u64 key = keys[x];
-        const int ts = dm.C - (int)(key >> 32);
-        const unsigned m = __ballot_sync(0xffffffffu, blockmax >= ts);
-        if (!m) return true;
-        if (tid == __ffs(m) - 1) {
-            int found = -1, nm = -1;
+    for (int x0 = K; x0 < dm.N; x0 += 32) {
+        // the next 32 keys, one per lane, handed out by shuffles
+        const u64 mine = (x0 + tid < dm.N) ? keys[x0 + tid] : 0;
+        const int nx = min(32, dm.N - x0);
+        const int my_len = dm.C - (int)(mine >> 32), my_id = (int)(u32)mine;
+#pragma unroll 4
+        for (int y = 0; y < nx; ++y) {
+            const int ts = __shfl_sync(0xffffffffu, my_len, y), id = __shfl_sync(0xffffffffu, my_id, y);
+            // every lane works out what it would do if the sample fell to it; only the ballot and
+            // the selects that follow it are on the path from one sample to the next
+            int found = -1, nm = -1, nrem[BR];
 #pragma unroll
             for (int u = 0; u < BR; ++u) {
                 const bool take = (found < 0) && (rem[u] >= ts);
-                if (take) { found = b0 + u; rem[u] -= ts; }
-                nm = max(nm, rem[u]);
+                nrem[u] = take ? rem[u] - ts : rem[u];
+                found = take ? b0 + u : found;
+                nm = max(nm, nrem[u]);
             }
-            blockmax = nm;
-            cell_of[(u32)key] = found;
+            const unsigned m = __ballot_sync(0xffffffffu, blockmax >= ts);
+            if (!m) return true;
+            const bool win = (tid == __ffs(m) - 1);
+#pragma unroll
+            for (int u = 0; u < BR; ++u) rem[u] = win ? nrem[u] : rem[u];
+            blockmax = win ? nm : blockmax;
+            if (win) cell_of[id] = found;
         }
     }
     return false;
@@ -89,10 +99,17 @@ k_pack_ffd(RpDims dm, const int *__restrict__ t, int min_rows, u64 *__restrict__
             keys[i] = ~0ull;
         }
     }
-    atomicAdd((u64 *)&total_s, (u64)part);
+    for (int o = 16; o; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+    if ((tid & 31) == 0 && part) atomicAdd((u64 *)&total_s, (u64)part);
     __syncthreads();
-    for (int k = 2; k <= n_pow2; k <<= 1)
-        for (int j = k >> 1; j > 0; j >>= 1) {
+    // Bitonic sort.  Element i sits with thread i % PACK_THREADS, so partners closer than 32 are
+    // lanes of one warp: those exchanges run on registers with shuffles (no block-wide barrier),
+    // the wider ones through the key array.
+    constexpr int SORT_E = 8;                      // elements per thread at most (n_pow2 <= 8192 on this path)
+    const bool in_regs = n_pow2 <= SORT_E * PACK_THREADS;
+    for (int k = 2; k <= n_pow2; k <<= 1) {
+        int j = k >> 1;
+        for (; j >= 32 || (j > 0 && !in_regs); j >>= 1) {
             for (int i = tid; i < n_pow2; i += PACK_THREADS) {
                 int ixj = i ^ j;
                 if (ixj > i) {
@@ -103,6 +120,33 @@ k_pack_ffd(RpDims dm, const int *__restrict__ t, int min_rows, u64 *__restrict__
             }
             __syncthreads();
         }
+        if (j > 0) {
+            // all remaining distances of this k (and, while k <= 32, of the following k as well)
+            u64 r[SORT_E];
+#pragma unroll
+            for (int m = 0; m < SORT_E; ++m) { const int i = m * PACK_THREADS + tid; r[m] = i < n_pow2 ? keys[i] : ~0ull; }
+            int kk = k;
+            for (;;) {
+                for (int jj = min(kk >> 1, 16); jj > 0; jj >>= 1) {
+#pragma unroll
+                    for (int m = 0; m < SORT_E; ++m) {
+                        const int i = m * PACK_THREADS + tid;
+                        if (m * PACK_THREADS >= n_pow2) break;          // uniform: no element of this slot exists
+                        const u64 o = __shfl_xor_sync(0xffffffffu, r[m], jj);
+                        const bool up = ((i & kk) == 0), lower = ((tid & jj) == 0);
+                        const u64 lo = r[m] < o ? r[m] : o, hi = r[m] < o ? o : r[m];
+                        r[m] = (lower == up) ? lo : hi;
+                    }
+                }
+                if (kk >= 32 || (kk << 1) > n_pow2) break;
+                kk <<= 1;                                       // the next k still fits inside a warp
+            }
+            k = kk;
+#pragma unroll
+            for (int m = 0; m < SORT_E; ++m) { const int i = m * PACK_THREADS + tid; if (i < n_pow2) keys[i] = r[m]; }
+            __syncthreads();
+        }
+    }
     for (int x = tid; x < dm.N; x += PACK_THREADS) order_out[x] = (int)(u32)keys[x];   // samples by (-t, i)
     const i64 cap_row = (i64)dm.C * dm.D;
     i64 Rlb = (total_s + cap_row - 1) / cap_row;
