@@ -104,7 +104,45 @@ k_lpt(const i64 *__restrict__ Lagg, RpDims dm, int *__restrict__ pi, int *__rest
         order[before] = e;
     }
     __syncthreads();
-    if (threadIdx.x < 32) {
+    if (threadIdx.x < 32 && dm.P <= 128) {
+        // Rank p lives in lane p % 32 (registers: load and slot count).  The least-loaded rank with
+        // a free slot is found by three warp reductions: smallest high word of the load, smallest
+        // low word among those, lowest rank id among those.
+        const int lane = threadIdx.x;
+        i64 Gr[4] = { 0, 0, 0, 0 };
+        int cr[4] = { 0, 0, 0, 0 };
+        for (int x = 0; x < dm.E; ++x) {
+            const int e = order[x];
+            const i64 le = load[e];
+            i64 bG = 0x7fffffffffffffffll;
+            int bP = 0x7fffffff;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int p = lane + 32 * u;
+                if (p < dm.P && cr[u] < dm.H && Gr[u] < bG) { bG = Gr[u]; bP = p; }      // ascending p: first wins
+            }
+            const u32 hi = (u32)((u64)bG >> 32);
+            const u32 mh = __reduce_min_sync(0xffffffffu, hi);
+            const u32 lo = (hi == mh) ? (u32)bG : 0xffffffffu;
+            const u32 ml = __reduce_min_sync(0xffffffffu, lo);
+            const int cand = (hi == mh && lo == ml) ? bP : 0x7fffffff;
+            const int mp = __reduce_min_sync(0xffffffffu, cand);
+            if (lane == (mp & 31)) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (u == (mp >> 5)) {
+                        const int slot = mp * dm.H + cr[u];
+                        pi[(size_t)l * dm.E + e] = slot;
+                        inv[(size_t)l * dm.E + slot] = e;
+                        Gr[u] += le;
+                        cr[u] += 1;
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) { const int p = lane + 32 * u; if (p < dm.P) rank_load[(size_t)l * dm.P + p] = Gr[u]; }
+    } else if (threadIdx.x < 32) {
         const int lane = threadIdx.x;
         int width = 1;                               // lanes that hold ranks, rounded up to a power of two
         while (width < dm.P && width < 32) width <<= 1;

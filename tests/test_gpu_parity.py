@@ -167,6 +167,8 @@ EDGE_SPECS = [
     ("vector_tail", 130, 9, 40, 2, 8192, 5, 20, [0, 1, 1, 2, 2], 3),
     # L*k*C*(cells per row-shard) >= 2^31: the sums over layers of the busiest ranks need 64 bits
     ("wide_sums", 72, 64, 16, 8, 1 << 20, 4, 4, [0, 0, 0, 0], 3),
+    # more ranks than the register-resident placement holds (128): its shared-memory form
+    ("many_ranks", 60, 2, 160, 2, 4096, 2, 160, None, 4),
 ]
 
 
