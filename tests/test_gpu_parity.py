@@ -466,7 +466,17 @@ def test_bad_inputs_are_host_side_errors():
     with pytest.raises(rp.RpError) as e:
         rp.rp_anneal(ctx, n_levels=1, steps_per_level=1, t0=1e-3, t_ratio=0.5, p_reloc=0.2, p_guide=0.8)
     assert e.value.status == -7
+    for call in (lambda: rp.rp_seed_population(ctx, 4), lambda: rp.rp_pair_population(ctx, 4),
+                 lambda: rp.rp_select_population(ctx, 4, 1 << 16)):
+        with pytest.raises(rp.RpError) as e:
+            call()                                                           # before rp_pack_rows
+        assert e.value.status == -7
     R, _ = rp.rp_pack_rows(ctx)
+    for call in (lambda: rp.rp_seed_population(ctx, 0), lambda: rp.rp_pair_population(ctx, 33),
+                 lambda: rp.rp_select_population(ctx, 0, 1 << 16), lambda: rp.rp_select_population(ctx, 4, -1)):
+        with pytest.raises(rp.RpError) as e:
+            call()
+        assert e.value.status == -1
     lay = np.zeros((1, s.n_samples), np.int32)
     lay[0, 5] = R * s.dp_width
     with pytest.raises(rp.RpError) as e:
@@ -475,6 +485,10 @@ def test_bad_inputs_are_host_side_errors():
     with pytest.raises(rp.RpError) as e:
         rp.rp_anneal(ctx, n_levels=0, steps_per_level=1, t0=1e-3, t_ratio=0.5, p_reloc=0.2, p_guide=0.8)
     assert e.value.status == -1
+    rp.rp_anneal(ctx, n_levels=1, steps_per_level=4, t0=1e-3, t_ratio=0.5, p_reloc=0.2, p_guide=0.8)
+    with pytest.raises(rp.RpError) as e:
+        rp.rp_pair_population(ctx, 4)                                        # the seeding stages end with rp_anneal
+    assert e.value.status == -7
     rp.rp_destroy(ctx)
     # infeasible: more DP slots than one-sample cells can fill at this cap is fine, but a window
     # whose samples cannot be split into non-empty cells within the cap is reported, not trapped
