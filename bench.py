@@ -300,6 +300,36 @@ def measure(rp, torch, args, name, steps, dist, dev, local, with_clocks, with_cp
             "gpu_launches": int(launches), "clocks": clocks, "wall_s": res["wall"]}
 
 
+def seeding_stages(rp, torch, name, dev, reps=3):
+    """Context figure: device time of the optional seeding stages (trial loop, pairing, canonical
+    map + quality-diversity selection) on the named window, mean over `reps` fresh contexts."""
+    w = make_window(SPECS[name])
+    s = w.spec
+    t_dev = torch.from_numpy(w.lengths).to(dev)
+    a_dev = torch.from_numpy(w.demand).to(dev)
+    ms = {"seed_population": 0.0, "pair_population": 0.0, "select_population": 0.0}
+    n_distinct = 0
+    for _ in range(reps):
+        ctx = rp.rp_window_load(t_dev, a_dev, top_k=s.top_k, token_cap=s.token_cap, dp_width=s.dp_width,
+                                ep_width=s.ep_width, pop_size=s.pop_size, alpha=s.alpha, beta=s.beta, seed=s.anneal_seed)
+        rp.rp_place_experts(ctx)
+        rp.rp_pack_rows(ctx)
+        for key, call in (("seed_population", lambda: rp.rp_seed_population(ctx, 4)),
+                          ("pair_population", lambda: rp.rp_pair_population(ctx, 4)),
+                          ("select_population", lambda: rp.rp_select_population(ctx, 8, 1 << 16))):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            out = call()
+            e1.record()
+            e1.synchronize()
+            ms[key] += e0.elapsed_time(e1) / reps
+            if key == "select_population":
+                n_distinct = int(out[0])
+        rp.rp_destroy(ctx)
+    return {"workload": name, "ms": ms, "n_distinct": n_distinct, "population": s.pop_size,
+            "choice_width": 4, "n_proj": 8, "eta_q16": 1 << 16}
+
+
 def run_cuda(args):
     import torch
     import paper_2608_12146_b200.binding as rp
@@ -337,6 +367,8 @@ def run_cuda(args):
         line.update(main_res)
         if sweep:
             line["other_workloads"] = sweep
+        if args.sweep and world == 1 and not args.pop and not args.levels:
+            line["seeding_stages"] = seeding_stages(rp, torch, args.workload, dev)
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
