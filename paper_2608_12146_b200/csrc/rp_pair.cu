@@ -44,6 +44,7 @@ k_edp_pair(RpDims dm, const int *__restrict__ q, const unsigned short *__restric
     int *cstart = slot_of + K;                     // [K + 1] first entry of each cell in `list`
     int *fillp = cstart + K + 1;                   // [K] fill pointers / empty flags later
     int *list = fillp + K;                         // [N] samples grouped by cell
+    i64 *eself = (i64 *)(((size_t)(list + N) + 7) & ~(size_t)7);   // [K] sum_l max_p of the cell's own profile
     __shared__ PairKey red[PAIR_WARPS];
     __shared__ int picked[32];
     __shared__ int rho_s, chosen_s;
@@ -79,7 +80,15 @@ k_edp_pair(RpDims dm, const int *__restrict__ q, const unsigned short *__restric
             pk = max(pk, acc);
         }
         pk = __reduce_max_sync(0xffffffffu, pk);
-        if (lane == 0) peak[b] = pk;
+        __syncwarp();                              // the profile row is complete before it is read back per layer
+        i64 es = 0;
+        for (int l = lane; l < L; l += 32) {
+            int mn = 0;
+            for (int p = 0; p < P; ++p) mn = max(mn, prof[(size_t)b * LP + l * P + p]);
+            es += mn;
+        }
+        for (int o = 16; o; o >>= 1) es += __shfl_xor_sync(0xffffffffu, es, o);
+        if (lane == 0) { peak[b] = pk; eself[b] = es; }
     }
     __syncthreads();
     // ---- order by (-peak, index): rank by counting ---------------------------------------------
@@ -99,6 +108,10 @@ k_edp_pair(RpDims dm, const int *__restrict__ q, const unsigned short *__restric
         // keys of the row-shards that still have an empty slot
         for (int rg = warp; rg < RG; rg += PAIR_WARPS) {
             if (free_rg[rg] == 0) continue;
+            if (e_old[rg] == 0) {                  // nothing placed there yet (or only empty profiles): the cell's own sums
+                if (lane == 0) { kd[rg] = eself[b]; kp[rg] = peak[b]; }
+                continue;
+            }
             const int *v = V + (size_t)rg * LP;
             i64 en = 0;
             int pk = 0;
@@ -165,7 +178,8 @@ k_edp_pair(RpDims dm, const int *__restrict__ q, const unsigned short *__restric
 
 size_t rp_pair_smem_bytes(const RpDims &dm)
 {
-    return sizeof(i64) * 2 * dm.RG + sizeof(int) * 2 * dm.RG + sizeof(int) * ((size_t)5 * dm.K + 1) + sizeof(int) * dm.N + 16;
+    return sizeof(i64) * 2 * dm.RG + sizeof(int) * 2 * dm.RG + sizeof(int) * ((size_t)5 * dm.K + 1) + sizeof(int) * (dm.N + 1) +
+           sizeof(i64) * dm.K + 16;
 }
 
 // Pairs members [first, first + count) of lay_in into lay_out; prof is scratch for `count`
