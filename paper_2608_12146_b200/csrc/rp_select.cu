@@ -19,6 +19,7 @@
 #include "rp_common.cuh"
 
 #define SEL_THREADS 256
+#define SEL_TABLE 4096
 
 struct SelBuf {                 // per-member arrays in global memory
     int *lay;                   // [P][N] layouts
@@ -220,13 +221,24 @@ k_sel_dist(RpDims dm, int Ppop, int n_proj, const int *__restrict__ rep, SelBuf 
     if (b <= a) { if (a == b && threadIdx.x == 0) dist[(size_t)a * Ppop + a] = 0; return; }
     if (!rep[a] || !rep[b]) return;
     __shared__ i64 acc[3];
+    __shared__ int tab[SEL_TABLE];                 // row-by-row contingency counts when R*R fits
     const int tid = threadIdx.x;
     const int N = dm.N, K = dm.K, R = dm.R, D = dm.D;
+    const bool rows_by_table = R * R <= SEL_TABLE;
     if (tid < 3) acc[tid] = 0;
+    if (rows_by_table) for (int x = tid; x < R * R; x += SEL_THREADS) tab[x] = 0;
     __syncthreads();
-    const int *lb = B.lay + (size_t)b * N;
+    const int *la = B.lay + (size_t)a * N, *lb = B.lay + (size_t)b * N;
     i64 bc = sel_both(B.clist + (size_t)a * N, B.cstart + (size_t)a * (K + 1), K, lb, 1, tid);
-    i64 br = sel_both(B.rlist + (size_t)a * N, B.rstart + (size_t)a * (R + 1), R, lb, D, tid);
+    i64 br = 0;
+    if (rows_by_table) {
+        // pairs in the same row of both plans = sum over (row of a, row of b) of C(count, 2)
+        for (int i = tid; i < N; i += SEL_THREADS) atomicAdd(&tab[(la[i] / D) * R + lb[i] / D], 1);
+        __syncthreads();
+        for (int x = tid; x < R * R; x += SEL_THREADS) { const i64 n = tab[x]; br += n * (n - 1) / 2; }
+    } else {
+        br = sel_both(B.rlist + (size_t)a * N, B.rstart + (size_t)a * (R + 1), R, lb, D, tid);
+    }
     i64 sw = 0;
     const i64 *pa = B.phi + (size_t)a * n_proj * R, *pb = B.phi + (size_t)b * n_proj * R;
     for (int x = tid; x < n_proj * R; x += SEL_THREADS) { const i64 d = pa[x] - pb[x]; sw += d < 0 ? -d : d; }
