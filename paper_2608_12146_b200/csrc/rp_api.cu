@@ -145,13 +145,13 @@ extern "C" void rp_destroy(rp_ctx *c)
     if (!c) return;
     cudaStreamSynchronize(c->stream);
     free_population(c); free_trace(c); free_eval(c);
-    dev_free(c, c->own_t); dev_free(c, c->own_a); dev_free(c, c->d_edp); dev_free(c, c->d_dp_list); dev_free(c, c->d_dp_off);
+    dev_free(c, c->own_t); dev_free(c, c->own_a); dev_free(c, c->d_edp);      // d_dp_list and d_dp_off live in d_edp's block
     dev_free(c, c->d_Lagg); dev_free(c, c->d_pi); dev_free(c, c->d_inv); dev_free(c, c->d_rank_load); dev_free(c, c->d_q);
     dev_free(c, c->d_status); dev_free(c, c->d_sort_keys); dev_free(c, c->d_seed_layout); dev_free(c, c->d_order); dev_free(c, c->d_pack_out);
     dev_free(c, c->d_counters); dev_free(c, c->d_inc_layout); dev_free(c, c->d_inc_score); dev_free(c, c->d_static);
     dev_free(c, c->d_seed_score);
     pin_give(c->h_pin);
-    free(c->h_levels); free(c->h_t);
+    free(c->h_levels);
     free(c);
 }
 
@@ -208,65 +208,70 @@ static int window_load_impl(rp_ctx *c, const rp_config *cfg, const int32_t *leng
     }
     dm.SC = ((i64)dm.C * dm.C) << RP_FBITS;
     dm.EC = (i64)dm.C << RP_FBITS;
-    int st = RP_OK;
-    do {
-        // rank loads must fit int32: W <= k * C * |D_g|
-        if ((double)dm.k * dm.C * maxshard >= 2147483648.0) { st = RP_ERR_RANGE; break; }
-        if ((st = dev_alloc(c, &c->d_edp, D)) != RP_OK) break;
-        if ((st = dev_alloc(c, &c->d_dp_list, D)) != RP_OK) break;
-        if ((st = dev_alloc(c, &c->d_dp_off, G + 1)) != RP_OK) break;
-        cudaMemcpyAsync(c->d_edp, edp, sizeof(int) * D, cudaMemcpyHostToDevice, c->stream);
-        cudaMemcpyAsync(c->d_dp_list, list, sizeof(int) * D, cudaMemcpyHostToDevice, c->stream);
-        cudaMemcpyAsync(c->d_dp_off, off, sizeof(int) * (G + 1), cudaMemcpyHostToDevice, c->stream);
-    } while (0);      // (copies from pageable memory are staged before the call returns)
-    free(edp); free(off); free(list);
-    RP_TRY(st);
+    // rank loads must fit int32: W <= k * C * |D_g|
+    if ((double)dm.k * dm.C * maxshard >= 2147483648.0) { free(edp); free(off); free(list); return RP_ERR_RANGE; }
 
     // inputs: adopt device arrays, copy host arrays
     const size_t n_a = (size_t)N * L * E;
-    c->h_t = (int *)malloc(sizeof(int) * N);
-    if (is_device_ptr(lengths)) {
-        c->d_t = lengths;
-        RP_CUDA(cudaMemcpyAsync(c->h_t, lengths, sizeof(int) * N, cudaMemcpyDeviceToHost, c->stream));
-    } else {
-        RP_TRY(dev_alloc(c, &c->own_t, N));
-        RP_CUDA(cudaMemcpyAsync(c->own_t, lengths, sizeof(int) * N, cudaMemcpyHostToDevice, c->stream));
-        memcpy(c->h_t, lengths, sizeof(int) * N);
-        c->d_t = c->own_t;
-    }
-    if (is_device_ptr(demand)) c->d_a = demand;
-    else {
-        RP_TRY(dev_alloc(c, &c->own_a, n_a));
-        RP_CUDA(cudaMemcpyAsync(c->own_a, demand, sizeof(int) * n_a, cudaMemcpyHostToDevice, c->stream));
-        c->d_a = c->own_a;
-    }
-    RP_TRY(dev_alloc(c, &c->d_Lagg, (size_t)L * E));
+    int st = RP_OK;
+    do {
+        if (is_device_ptr(lengths)) c->d_t = lengths;
+        else {
+            if ((st = dev_alloc(c, &c->own_t, N)) != RP_OK) break;
+            if (cudaMemcpyAsync(c->own_t, lengths, sizeof(int) * N, cudaMemcpyHostToDevice, c->stream) != cudaSuccess) { st = RP_ERR_CUDA; break; }
+            c->d_t = c->own_t;
+        }
+        if (is_device_ptr(demand)) c->d_a = demand;
+        else {
+            if ((st = dev_alloc(c, &c->own_a, n_a)) != RP_OK) break;
+            if (cudaMemcpyAsync(c->own_a, demand, sizeof(int) * n_a, cudaMemcpyHostToDevice, c->stream) != cudaSuccess) { st = RP_ERR_CUDA; break; }
+            c->d_a = c->own_a;
+        }
+        // input checks + aggregate expert load + token total in one pass over the demand tensor,
+        // put in flight before the rest of the set-up
+        if ((st = dev_alloc(c, &c->d_Lagg, (size_t)L * E)) != RP_OK) break;
+        if ((st = dev_alloc(c, &c->d_status, RP_SW_COUNT)) != RP_OK) break;
+        if ((st = dev_alloc(c, &c->d_counters, 8)) != RP_OK) break;
+        if (cudaMemsetAsync(c->d_counters, 0, sizeof(i64) * 8, c->stream) != cudaSuccess) { st = RP_ERR_CUDA; break; }
+        if ((st = reset_status(c)) != RP_OK) break;
+        if ((st = rp_launch_check_reduce(c)) != RP_OK) break;
+        // the EDP tables: one allocation, one copy (pageable source: staged before the call returns)
+        const size_t n_tab = (size_t)2 * D + G + 1;
+        if ((st = dev_alloc(c, &c->d_edp, n_tab)) != RP_OK) break;
+        c->d_dp_list = c->d_edp + D;
+        c->d_dp_off = c->d_dp_list + D;
+        int *tab = (int *)malloc(sizeof(int) * n_tab);
+        memcpy(tab, edp, sizeof(int) * D);
+        memcpy(tab + D, list, sizeof(int) * D);
+        memcpy(tab + 2 * D, off, sizeof(int) * (G + 1));
+        const cudaError_t e = cudaMemcpyAsync(c->d_edp, tab, sizeof(int) * n_tab, cudaMemcpyHostToDevice, c->stream);
+        free(tab);
+        if (e != cudaSuccess) { g_rp_last_cuda_error = (int)e; st = RP_ERR_CUDA; break; }
+    } while (0);
+    free(edp); free(off); free(list);
+    RP_TRY(st);
     RP_TRY(dev_alloc(c, &c->d_pi, (size_t)L * E));
     RP_TRY(dev_alloc(c, &c->d_inv, (size_t)L * E));
     RP_TRY(dev_alloc(c, &c->d_rank_load, (size_t)L * P));
     RP_TRY(dev_alloc(c, &c->d_q, (size_t)N * L * P));
-    RP_TRY(dev_alloc(c, &c->d_status, RP_SW_COUNT));
     int n_pow2 = 1;
     while (n_pow2 < N) n_pow2 <<= 1;
     RP_TRY(dev_alloc(c, &c->d_sort_keys, (size_t)2 * n_pow2));
     RP_TRY(dev_alloc(c, &c->d_seed_layout, N));
     RP_TRY(dev_alloc(c, &c->d_order, N));
     RP_TRY(dev_alloc(c, &c->d_pack_out, 4));
-    RP_TRY(dev_alloc(c, &c->d_counters, 8));
     RP_TRY(dev_alloc(c, &c->d_inc_layout, N));
     RP_TRY(dev_alloc(c, &c->d_inc_score, 3));
     RP_TRY(dev_alloc(c, &c->d_seed_score, 3));
-    RP_TRY(reset_status(c));
 
-    // input checks + aggregate expert load in one pass over the demand tensor
-    RP_TRY(rp_launch_check_reduce(c));
+    // verdict of the checks and the token total ride back in the pinned block
+    RP_CUDA(cudaMemcpyAsync(c->h_pin + 8, c->d_counters + 7, sizeof(i64), cudaMemcpyDeviceToHost, c->stream));
     int sw[RP_SW_COUNT];
     RP_TRY(read_status(c, sw));
     if (sw[RP_SW_BAD_SAMPLE]) return RP_ERR_CONSERVATION;
 
     // fixed-point range of the score: s1 <= (2^8*C*L*k + (asum+bsum)*C) * sum t  must stay below 2^62
-    double total = 0.0;
-    for (int i = 0; i < N; ++i) total += (double)c->h_t[i];
+    const double total = (double)c->h_pin[8];
     double bound = ((double)dm.EC * L * dm.k + (double)(dm.asum + dm.bsum) * dm.C) * total;
     if (bound >= 4.0e18) return RP_ERR_RANGE;
     return RP_OK;

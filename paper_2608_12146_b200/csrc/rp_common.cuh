@@ -158,7 +158,6 @@ struct rp_ctx {
     size_t eval_cap;
     RpLevel *h_levels;         // host copy of the per-level schedule integers
     int levels_cap;
-    int *h_t;                  // host copy of the lengths (range checks)
     i64 *h_pin;                // small pinned staging block for device->host scalars (64 x 8 bytes)
     i64 *d_seed_score;         // [3] best score of the initial population
 };

@@ -16,11 +16,12 @@
 template <int NC>
 __global__ void __launch_bounds__(K1_WARPS * 32)
 k_check_reduce(const int *__restrict__ a, const int *__restrict__ t, RpDims dm, int chunk,
-               i64 *__restrict__ Lagg, int *__restrict__ status)
+               i64 *__restrict__ Lagg, int *__restrict__ status, i64 *__restrict__ t_sum)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int i0 = blockIdx.x * chunk;
     const int i1 = min(dm.N, i0 + chunk);
+    i64 tsum = 0;                  // tokens of this chunk (added up by the warp that owns layer 0)
     for (int l = warp; l < dm.L; l += K1_WARPS) {
         i64 acc[NC];
 #pragma unroll
@@ -28,6 +29,7 @@ k_check_reduce(const int *__restrict__ a, const int *__restrict__ t, RpDims dm, 
         for (int i = i0; i < i1; ++i) {
             const int *row = a + ((size_t)i * dm.L + l) * dm.E;
             const int ti = t[i];
+            if (l == 0) tsum += ti;
             i64 rs = 0;
             bool neg = false;
 #pragma unroll
@@ -50,6 +52,7 @@ k_check_reduce(const int *__restrict__ a, const int *__restrict__ t, RpDims dm, 
             if (e < dm.E && acc[c]) atomicAdd((u64 *)&Lagg[(size_t)l * dm.E + e], (u64)acc[c]);
         }
     }
+    if (warp == 0 && lane == 0 && tsum > 0) atomicAdd((u64 *)t_sum, (u64)tsum);
 }
 
 int rp_launch_check_reduce(rp_ctx *c)
@@ -63,7 +66,7 @@ int rp_launch_check_reduce(rp_ctx *c)
     int nc = (dm.E + 31) / 32;
 #define K1_CASE(NC_)                                                                         \
     k_check_reduce<NC_><<<grid, K1_WARPS * 32, 0, c->stream>>>(c->d_a, c->d_t, dm, chunk, c->d_Lagg, \
-                                                               c->d_status)
+                                                               c->d_status, c->d_counters + 7)
     if (nc <= 1) K1_CASE(1);
     else if (nc <= 2) K1_CASE(2);
     else if (nc <= 4) K1_CASE(4);
