@@ -18,6 +18,7 @@ __device__ __forceinline__ bool first_fit_regs(const RpDims &dm, const u64 *keys
     const int b0 = tid * B;
     int rem[BR];
     int blockmax = -1;
+    bool failed = false;                           // some sample fitted nowhere (the rest of the pass is then moot)
 #pragma unroll
     for (int u = 0; u < BR; ++u) {
         rem[u] = (u < B && b0 + u < K) ? dm.C - fill[b0 + u] : -1;
@@ -31,26 +32,28 @@ __device__ __forceinline__ bool first_fit_regs(const RpDims &dm, const u64 *keys
 #pragma unroll 4
         for (int y = 0; y < nx; ++y) {
             const int ts = __shfl_sync(0xffffffffu, my_len, y), id = __shfl_sync(0xffffffffu, my_id, y);
-            // every lane works out what it would do if the sample fell to it; only the ballot and
-            // the selects that follow it are on the path from one sample to the next
-            int found = -1, nm = -1, nrem[BR];
+            // every lane works out what it would do if the sample fell to it (first cell of its
+            // block that fits, block maximum afterwards), with no chain from cell to cell; only
+            // the ballot and the selects after it link one sample to the next
+            bool fits[BR];
 #pragma unroll
-            for (int u = 0; u < BR; ++u) {
-                const bool take = (found < 0) && (rem[u] >= ts);
-                nrem[u] = take ? rem[u] - ts : rem[u];
-                found = take ? b0 + u : found;
-                nm = max(nm, nrem[u]);
-            }
+            for (int u = 0; u < BR; ++u) fits[u] = rem[u] >= ts;
+            int first = BR;
+#pragma unroll
+            for (int u = BR - 1; u >= 0; --u) first = fits[u] ? u : first;
+            int nm = -1;
+#pragma unroll
+            for (int u = 0; u < BR; ++u) nm = max(nm, u == first ? rem[u] - ts : rem[u]);
             const unsigned m = __ballot_sync(0xffffffffu, blockmax >= ts);
-            if (!m) return true;
+            failed |= (m == 0);
             const bool win = (tid == __ffs(m) - 1);
 #pragma unroll
-            for (int u = 0; u < BR; ++u) rem[u] = win ? nrem[u] : rem[u];
+            for (int u = 0; u < BR; ++u) rem[u] = (win && u == first) ? rem[u] - ts : rem[u];
             blockmax = win ? nm : blockmax;
-            if (win) cell_of[id] = found;
+            if (win) cell_of[id] = b0 + first;
         }
     }
-    return false;
+    return failed;
 }
 
 __device__ __forceinline__ bool first_fit_smem(const RpDims &dm, const u64 *keys, int *fill, int *cell_of, int K, int B, int tid)
