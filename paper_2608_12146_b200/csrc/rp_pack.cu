@@ -89,11 +89,11 @@ k_pack_ffd(RpDims dm, const int *__restrict__ t, int min_rows, u64 *__restrict__
     int *fill = fill_g ? fill_g : (int *)(keys_s + (keys_g ? 0 : n_pow2));
     __shared__ i64 total_s;
     __shared__ int fail_s;
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, nt = (int)blockDim.x;
     if (tid == 0) total_s = 0;
     __syncthreads();
     i64 part = 0;
-    for (int i = tid; i < n_pow2; i += PACK_THREADS) {
+    for (int i = tid; i < n_pow2; i += nt) {
         if (i < dm.N) {
             int ti = t[i];
             part += ti;
@@ -105,15 +105,15 @@ k_pack_ffd(RpDims dm, const int *__restrict__ t, int min_rows, u64 *__restrict__
     for (int o = 16; o; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
     if ((tid & 31) == 0 && part) atomicAdd((u64 *)&total_s, (u64)part);
     __syncthreads();
-    // Bitonic sort.  Element i sits with thread i % PACK_THREADS, so partners closer than 32 are
+    // Bitonic sort.  Element i sits with thread i % nt, so partners closer than 32 are
     // lanes of one warp: those exchanges run on registers with shuffles (no block-wide barrier),
     // the wider ones through the key array.
     constexpr int SORT_E = 8;                      // elements per thread at most (n_pow2 <= 8192 on this path)
-    const bool in_regs = n_pow2 <= SORT_E * PACK_THREADS;
+    const bool in_regs = n_pow2 <= SORT_E * nt;
     for (int k = 2; k <= n_pow2; k <<= 1) {
         int j = k >> 1;
         for (; j >= 32 || (j > 0 && !in_regs); j >>= 1) {
-            for (int i = tid; i < n_pow2; i += PACK_THREADS) {
+            for (int i = tid; i < n_pow2; i += nt) {
                 int ixj = i ^ j;
                 if (ixj > i) {
                     u64 a = keys[i], b = keys[ixj];
@@ -127,14 +127,14 @@ k_pack_ffd(RpDims dm, const int *__restrict__ t, int min_rows, u64 *__restrict__
             // all remaining distances of this k (and, while k <= 32, of the following k as well)
             u64 r[SORT_E];
 #pragma unroll
-            for (int m = 0; m < SORT_E; ++m) { const int i = m * PACK_THREADS + tid; r[m] = i < n_pow2 ? keys[i] : ~0ull; }
+            for (int m = 0; m < SORT_E; ++m) { const int i = m * nt + tid; r[m] = i < n_pow2 ? keys[i] : ~0ull; }
             int kk = k;
             for (;;) {
                 for (int jj = min(kk >> 1, 16); jj > 0; jj >>= 1) {
 #pragma unroll
                     for (int m = 0; m < SORT_E; ++m) {
-                        const int i = m * PACK_THREADS + tid;
-                        if (m * PACK_THREADS >= n_pow2) break;          // uniform: no element of this slot exists
+                        const int i = m * nt + tid;
+                        if (m * nt >= n_pow2) break;          // uniform: no element of this slot exists
                         const u64 o = __shfl_xor_sync(0xffffffffu, r[m], jj);
                         const bool up = ((i & kk) == 0), lower = ((tid & jj) == 0);
                         const u64 lo = r[m] < o ? r[m] : o, hi = r[m] < o ? o : r[m];
@@ -146,11 +146,11 @@ k_pack_ffd(RpDims dm, const int *__restrict__ t, int min_rows, u64 *__restrict__
             }
             k = kk;
 #pragma unroll
-            for (int m = 0; m < SORT_E; ++m) { const int i = m * PACK_THREADS + tid; if (i < n_pow2) keys[i] = r[m]; }
+            for (int m = 0; m < SORT_E; ++m) { const int i = m * nt + tid; if (i < n_pow2) keys[i] = r[m]; }
             __syncthreads();
         }
     }
-    for (int x = tid; x < dm.N; x += PACK_THREADS) order_out[x] = (int)(u32)keys[x];   // samples by (-t, i)
+    for (int x = tid; x < dm.N; x += nt) order_out[x] = (int)(u32)keys[x];   // samples by (-t, i)
     const i64 cap_row = (i64)dm.C * dm.D;
     i64 Rlb = (total_s + cap_row - 1) / cap_row;
     if (Rlb < 1) Rlb = 1;
@@ -160,7 +160,7 @@ k_pack_ffd(RpDims dm, const int *__restrict__ t, int min_rows, u64 *__restrict__
         const int K = (int)(R * dm.D);
         if (tid == 0) fail_s = 0;
         // the K longest samples open the cells
-        for (int x = tid; x < K; x += PACK_THREADS) {
+        for (int x = tid; x < K; x += nt) {
             const u64 key = keys[x];
             fill[x] = dm.C - (int)(key >> 32);
             cell_of[(u32)key] = x;
@@ -203,7 +203,9 @@ int rp_launch_pack(rp_ctx *c, int /*unused*/)
     if (smem > 160 * 1024) { keys_g = c->d_sort_keys; fill_g = (int *)(c->d_sort_keys + n_pow2); smem = 0; }
     if (smem > 32 * 1024)
         RP_CUDA(cudaFuncSetAttribute(k_pack_ffd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k_pack_ffd<<<1, PACK_THREADS, smem, c->stream>>>(dm, c->d_t, c->cfg.min_rows, keys_g, n_pow2, fill_g,
+    // small windows: fewer warps make the block-wide barriers of the sort cheaper
+    const int threads = n_pow2 >= PACK_THREADS ? PACK_THREADS : (n_pow2 < 256 ? 256 : n_pow2);
+    k_pack_ffd<<<1, threads, smem, c->stream>>>(dm, c->d_t, c->cfg.min_rows, keys_g, n_pow2, fill_g,
                                                     c->d_seed_layout, c->d_pack_out, c->d_order);
     ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
