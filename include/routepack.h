@@ -203,12 +203,17 @@ int rp_eval_layouts_noalloc(rp_ctx *ctx, const int32_t *layouts, int32_t n, int6
  * trajectory-best plan, and (except after the last level) the population is resampled
  * systematically with Boltzmann weights.  May be called again to continue from the
  * current population; level indices of the random streams restart at 0 on each call.
+ * Before it returns the call also validates and fully rescores its incumbent (the checks of
+ * rp_best) in the same stream, so that a following rp_best has nothing left to compute.
  *   stats: HOST out, nullable. */
 int rp_anneal(rp_ctx *ctx, const rp_anneal_params *params, rp_anneal_stats *stats);
 
 /* Validate the incumbent (coverage, capacity, non-empty cells, cached score equals a full
  * rescoring, not worse than the seed) and return it.
- *   cell_of_sample [N] int32 out, nullable; score_fx [3], score_f64 [3] out, nullable. */
+ *   cell_of_sample [N] int32 out, nullable; score_fx [3], score_f64 [3] out, nullable.
+ * RP_ERR_INVALID_PLAN when a check fails.  Host outputs are complete on return; outputs in
+ * device memory are ordered on the context's stream.  Right after rp_anneal the checks are
+ * already done and the call only hands the results over. */
 int rp_best(rp_ctx *ctx, int32_t *cell_of_sample, int64_t *score_fx, double *score_f64);
 
 /* Load-balance diagnostics of the paper's evaluation section for one layout (Eq. global-ep-cv,

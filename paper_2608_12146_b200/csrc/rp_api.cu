@@ -149,7 +149,7 @@ extern "C" void rp_destroy(rp_ctx *c)
     dev_free(c, c->d_Lagg); dev_free(c, c->d_pi); dev_free(c, c->d_inv); dev_free(c, c->d_rank_load); dev_free(c, c->d_q);
     dev_free(c, c->d_status); dev_free(c, c->d_sort_keys); dev_free(c, c->d_seed_layout); dev_free(c, c->d_order); dev_free(c, c->d_pack_out);
     dev_free(c, c->d_counters); dev_free(c, c->d_inc_layout); dev_free(c, c->d_inc_score); dev_free(c, c->d_static);
-    dev_free(c, c->d_seed_score);
+    dev_free(c, c->d_seed_score); dev_free(c, c->d_best_score); dev_free(c, c->d_best_f64);
     pin_give(c->h_pin);
     free(c->h_levels);
     free(c);
@@ -263,6 +263,8 @@ static int window_load_impl(rp_ctx *c, const rp_config *cfg, const int32_t *leng
     RP_TRY(dev_alloc(c, &c->d_inc_layout, N));
     RP_TRY(dev_alloc(c, &c->d_inc_score, 3));
     RP_TRY(dev_alloc(c, &c->d_seed_score, 3));
+    RP_TRY(dev_alloc(c, &c->d_best_score, 3));
+    RP_TRY(dev_alloc(c, &c->d_best_f64, 3));
 
     // verdict of the checks and the token total ride back in the pinned block
     RP_CUDA(cudaMemcpyAsync(c->h_pin + 8, c->d_counters + 7, sizeof(i64), cudaMemcpyDeviceToHost, c->stream));
@@ -363,6 +365,7 @@ extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
     if (!c) return RP_ERR_ARG;
     if (c->stage < 2) return RP_ERR_STATE;
     RpDims &dm = c->dm;
+    c->best_ready = 0;
     RP_TRY(rp_launch_pack(c, 0));
     int *po = (int *)c->h_pin;
     RP_CUDA(cudaMemcpyAsync(po, c->d_pack_out, sizeof(int) * 4, cudaMemcpyDeviceToHost, c->stream));
@@ -477,6 +480,7 @@ extern "C" int rp_eval_population(rp_ctx *c, const int32_t *layouts, int32_t n, 
 static int install_population(rp_ctx *c, const int *lay)
 {
     const size_t P = (size_t)c->Ppop;
+    c->best_ready = 0;
     i64 *best = nullptr;
     RP_TRY(dev_alloc(c, &best, 3));
     int st = ensure_eval_scratch(c, P, false);
@@ -641,6 +645,9 @@ static void make_schedule(const rp_anneal_params *p, RpLevel *lv)
     }
 }
 
+static int launch_best_check(rp_ctx *c);
+static int best_verdict(const rp_ctx *c, const int *sw);
+
 extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *stats)
 {
     if (!c || !p) return RP_ERR_ARG;
@@ -689,6 +696,10 @@ extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *
         { int *sw = c->d_wloc; c->d_wloc = c->d_wloc_next; c->d_wloc_next = sw; }
     }
     if (stats) cudaEventRecord(ev[1], c->stream);
+    // Validate(x*) and the full rescoring of the incumbent follow in the same stream, so that
+    // rp_best finds them done
+    c->best_ready = 0;
+    if (st == RP_OK) st = launch_best_check(c);
     // one synchronisation: the counters and the status words ride back in the pinned block
     i64 *cn = c->h_pin;                       // [8] counters
     int *sw = (int *)(c->h_pin + 56);         // status words
@@ -708,8 +719,36 @@ extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *
         stats->kernel_launches = (int64_t)NL;
         stats->ms_chains = ms_chains; stats->ms_barrier = 0.0;   // the barrier runs inside the chain kernels
     }
+    c->best_verdict = best_verdict(c, sw);
+    c->best_ready = 1;
     c->stage = 4;
     return RP_OK;
+}
+
+// Validate(x*) on the device: coverage / capacity / non-empty cells, and a full rescoring of the
+// incumbent; the three score tuples the verdict needs are queued into the pinned block.
+static int launch_best_check(rp_ctx *c)
+{
+    RP_TRY(rp_launch_validate(c));
+    RP_TRY(ensure_eval_scratch(c, 1, false));
+    RP_TRY(rp_launch_cells_from_layouts(c, c->d_inc_layout, 1, c->d_eval_cells));
+    RP_TRY(rp_launch_eval(c, c->d_eval_cells, 1, nullptr, nullptr, c->d_best_score, c->d_best_f64));
+    RP_CUDA(cudaMemcpyAsync(c->h_pin + 16, c->d_inc_score, sizeof(i64) * 3, cudaMemcpyDeviceToHost, c->stream));
+    RP_CUDA(cudaMemcpyAsync(c->h_pin + 19, c->d_best_score, sizeof(i64) * 3, cudaMemcpyDeviceToHost, c->stream));
+    RP_CUDA(cudaMemcpyAsync(c->h_pin + 22, c->d_seed_score, sizeof(i64) * 3, cudaMemcpyDeviceToHost, c->stream));
+    return RP_OK;
+}
+
+// After the stream has been synchronised: the verdict from the pinned block and the status words.
+static int best_verdict(const rp_ctx *c, const int *sw)
+{
+    const i64 *inc = c->h_pin + 16, *full = c->h_pin + 19, *seed = c->h_pin + 22;
+    bool ok = !sw[RP_SW_VALIDATE] && !sw[RP_SW_BAD_LAYOUT];
+    ok = ok && inc[0] == full[0] && inc[1] == full[1] && inc[2] == full[2];
+    // non-regression: not worse than the best member of the initial population
+    const bool worse = (seed[0] != inc[0]) ? (seed[0] < inc[0]) : (seed[1] != inc[1]) ? (seed[1] < inc[1]) : (seed[2] < inc[2]);
+    ok = ok && !worse;
+    return ok ? RP_OK : RP_ERR_INVALID_PLAN;
 }
 
 extern "C" int rp_best(rp_ctx *c, int32_t *cell_of_sample, int64_t *score_fx, double *score_f64)
@@ -717,29 +756,21 @@ extern "C" int rp_best(rp_ctx *c, int32_t *cell_of_sample, int64_t *score_fx, do
     if (!c) return RP_ERR_ARG;
     if (c->stage < 3) return RP_ERR_STATE;
     const RpDims &dm = c->dm;
-    RP_TRY(reset_status(c));
-    RP_TRY(rp_launch_validate(c));
-    // full rescoring of the incumbent
-    RP_TRY(ensure_eval_scratch(c, 1, false));
-    RP_TRY(rp_launch_cells_from_layouts(c, c->d_inc_layout, 1, c->d_eval_cells));
-    RP_TRY(rp_launch_eval(c, c->d_eval_cells, 1, nullptr, nullptr, c->d_eval_score, c->d_eval_f64));
-    // inc score, full rescoring, seed score and status words ride back in the pinned block
-    i64 *inc = c->h_pin, *full = c->h_pin + 3, *seed = c->h_pin + 6;
     int *sw = (int *)(c->h_pin + 56);
-    RP_CUDA(cudaMemcpyAsync(inc, c->d_inc_score, sizeof(i64) * 3, cudaMemcpyDeviceToHost, c->stream));
-    RP_CUDA(cudaMemcpyAsync(full, c->d_eval_score, sizeof(i64) * 3, cudaMemcpyDeviceToHost, c->stream));
-    RP_CUDA(cudaMemcpyAsync(seed, c->d_seed_score, sizeof(i64) * 3, cudaMemcpyDeviceToHost, c->stream));
-    RP_CUDA(cudaMemcpyAsync(sw, c->d_status, sizeof(int) * RP_SW_COUNT, cudaMemcpyDeviceToHost, c->stream));
+    const bool fresh = !c->best_ready;          // rp_anneal validates its incumbent before it returns
+    if (fresh) {
+        RP_TRY(reset_status(c));
+        RP_TRY(launch_best_check(c));
+        RP_CUDA(cudaMemcpyAsync(sw, c->d_status, sizeof(int) * RP_SW_COUNT, cudaMemcpyDeviceToHost, c->stream));
+    }
     RP_TRY(copy_out(c, cell_of_sample, c->d_inc_layout, sizeof(int) * (size_t)dm.N));
     RP_TRY(copy_out(c, score_fx, c->d_inc_score, sizeof(i64) * 3));
-    RP_TRY(copy_out(c, score_f64, c->d_eval_f64, sizeof(double) * 3));
-    RP_CUDA(cudaStreamSynchronize(c->stream));
-    bool ok = !sw[RP_SW_VALIDATE] && !sw[RP_SW_BAD_LAYOUT];
-    ok = ok && inc[0] == full[0] && inc[1] == full[1] && inc[2] == full[2];
-    // non-regression: not worse than the best member of the initial population
-    const bool worse = (seed[0] != inc[0]) ? (seed[0] < inc[0]) : (seed[1] != inc[1]) ? (seed[1] < inc[1]) : (seed[2] < inc[2]);
-    ok = ok && !worse;
-    return ok ? RP_OK : RP_ERR_INVALID_PLAN;
+    RP_TRY(copy_out(c, score_f64, c->d_best_f64, sizeof(double) * 3));
+    const bool host_out = (cell_of_sample && !is_device_ptr(cell_of_sample)) || (score_fx && !is_device_ptr(score_fx)) ||
+                          (score_f64 && !is_device_ptr(score_f64));
+    if (fresh || host_out) RP_CUDA(cudaStreamSynchronize(c->stream));
+    if (fresh) { c->best_verdict = best_verdict(c, sw); c->best_ready = 1; }
+    return c->best_verdict;
 }
 
 // ---------------------------------------------------------------------------------------

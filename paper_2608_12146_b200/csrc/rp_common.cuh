@@ -141,6 +141,10 @@ struct rp_ctx {
     int *d_inc_slot;           // [1]
     i64 *d_sel_dist;           // [P_pop][P_pop] plan distances of the last rp_select_population (inspection hook on)
     i64 *d_inc_score;          // [3]
+    i64 *d_best_score;         // [3] full rescoring of the incumbent (validation)
+    double *d_best_f64;        // [3] the same as the real-valued objective
+    int best_ready;            // the incumbent has been validated and rescored since it last changed
+    int best_verdict;          // RP_OK or RP_ERR_INVALID_PLAN of that validation
     // trace of the last rp_anneal call
     int trace_levels;
     int trace_on;              // keep per-level traces (inspection hook; off by default)
