@@ -360,6 +360,20 @@ __global__ void k_iota(int *out, int n, int first)
     if (x < n) out[x] = first + x;
 }
 
+// Population bookkeeping of a fresh seed in one launch: every member descends from slot 0, whose
+// rank loads sit in cell 0 and are copied into a cell of the member's own (P + m) at level 0; the
+// seed is the incumbent.
+__global__ void k_init_population(int P, int N, int *__restrict__ anc, int *__restrict__ wloc, int *__restrict__ wloc_next,
+                                  int *__restrict__ done, const int *__restrict__ seed_layout, int *__restrict__ inc_layout,
+                                  const i64 *__restrict__ inc_score, i64 *__restrict__ seed_score)
+{
+    const int x = blockIdx.x * blockDim.x + threadIdx.x;
+    if (x < P) { anc[x] = 0; wloc[x] = 0; wloc_next[x] = P + x; }
+    if (x < N) inc_layout[x] = seed_layout[x];
+    if (x < 3) seed_score[x] = inc_score[x];
+    if (x == 0) *done = 0;
+}
+
 extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
 {
     if (!c) return RP_ERR_ARG;
@@ -394,7 +408,6 @@ extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
     RP_TRY(dev_alloc(c, &c->d_anc, P));
     RP_TRY(dev_alloc(c, &c->d_anc_next, P));
     RP_TRY(dev_alloc(c, &c->d_done, 1));
-    RP_CUDA(cudaMemsetAsync(c->d_done, 0, sizeof(int), c->stream));
     RP_TRY(dev_alloc(c, &c->d_term, P * 3));
     RP_TRY(dev_alloc(c, &c->d_best, P * 3));
     RP_TRY(dev_alloc(c, &c->d_best_step, P));
@@ -410,13 +423,14 @@ extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
     RP_TRY(ensure_eval_scratch(c, 1, false));
     RP_TRY(rp_launch_cells_from_layouts(c, c->d_seed_layout, 1, c->d_eval_cells));
     RP_TRY(rp_launch_eval(c, c->d_eval_cells, 1, c->d_W, c->buf[0].blob, c->d_inc_score, nullptr));
-    RP_CUDA(cudaMemsetAsync(c->d_anc, 0, sizeof(int) * P, c->stream));
-    // the seed's W sits in cell 0; every member copies it into a cell of its own (P + m) at level 0
-    RP_CUDA(cudaMemsetAsync(c->d_wloc, 0, sizeof(int) * P, c->stream));
-    k_iota<<<(int)((P + 255) / 256), 256, 0, c->stream>>>(c->d_wloc_next, (int)P, (int)P);
-    ++g_rp_launches;
-    RP_CUDA(cudaMemcpyAsync(c->d_inc_layout, c->d_seed_layout, sizeof(int) * dm.N, cudaMemcpyDeviceToDevice, c->stream));
-    RP_CUDA(cudaMemcpyAsync(c->d_seed_score, c->d_inc_score, sizeof(i64) * 3, cudaMemcpyDeviceToDevice, c->stream));
+    {
+        const size_t n = P > (size_t)dm.N ? P : (size_t)dm.N;
+        k_init_population<<<(int)((n + 255) / 256), 256, 0, c->stream>>>((int)P, dm.N, c->d_anc, c->d_wloc, c->d_wloc_next, c->d_done,
+                                                                          c->d_seed_layout, c->d_inc_layout, c->d_inc_score,
+                                                                          c->d_seed_score);
+        ++g_rp_launches;
+        RP_CUDA(cudaGetLastError());
+    }
     if (n_rows) *n_rows = c->Rstar;
     if (certified) *certified = c->certified;
     c->stage = 3;
