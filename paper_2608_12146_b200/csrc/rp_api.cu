@@ -662,6 +662,14 @@ static void make_schedule(const rp_anneal_params *p, RpLevel *lv)
 static int launch_best_check(rp_ctx *c);
 static int best_verdict(const rp_ctx *c, const int *sw);
 
+__global__ void k_reset_anneal(i64 *__restrict__ counters, int *__restrict__ status, int *__restrict__ inc_slot)
+{
+    const int x = threadIdx.x;
+    if (x < 8) counters[x] = 0;
+    if (x < RP_SW_COUNT) status[x] = 0;
+    if (x == 0) *inc_slot = -1;
+}
+
 extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *stats)
 {
     if (!c || !p) return RP_ERR_ARG;
@@ -694,9 +702,10 @@ extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *
         RP_TRY(dev_alloc(c, &c->d_tr_anc, (size_t)(NL > 1 ? NL - 1 : 1) * P));
         c->trace_levels = NL;
     }
-    RP_CUDA(cudaMemsetAsync(c->d_counters, 0, sizeof(i64) * 8, c->stream));
-    RP_CUDA(cudaMemsetAsync(c->d_inc_slot, 0xff, sizeof(int), c->stream));      // -1: the incumbent is in d_inc_layout
-    RP_TRY(reset_status(c));
+    // counters and status words to zero, incumbent slot to -1 (the incumbent is in d_inc_layout)
+    k_reset_anneal<<<1, 32, 0, c->stream>>>(c->d_counters, c->d_status, c->d_inc_slot);
+    ++g_rp_launches;
+    RP_CUDA(cudaGetLastError());
 
     cudaEvent_t ev[2] = { nullptr, nullptr };
     if (stats) for (int x = 0; x < 2; ++x) RP_CUDA(cudaEventCreate(&ev[x]));
