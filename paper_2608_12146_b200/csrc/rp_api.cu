@@ -106,18 +106,14 @@ static int copy_out(rp_ctx *c, void *dst, const void *src, size_t bytes)
 
 static void free_population(rp_ctx *c)
 {
-    for (int b = 0; b < 2; ++b) {
-        dev_free(c, c->buf[b].blob);
-        c->buf[b].blob = nullptr;
-    }
-    dev_free(c, c->d_W); dev_free(c, c->d_wloc); dev_free(c, c->d_wloc_next); dev_free(c, c->d_le_scratch);
+    dev_free(c, c->d_pop_slab); c->d_pop_slab = nullptr;           // every buffer below is a piece of it
+    c->buf[0].blob = nullptr; c->buf[1].blob = nullptr;
     c->d_W = nullptr; c->d_wloc = nullptr; c->d_wloc_next = nullptr; c->d_le_scratch = nullptr;
-    dev_free(c, c->d_cand_layout); dev_free(c, c->d_inc_slot); dev_free(c, c->d_sel_dist);
-    c->d_cand_layout = nullptr; c->d_inc_slot = nullptr; c->d_sel_dist = nullptr;
-    dev_free(c, c->d_anc); dev_free(c, c->d_anc_next); dev_free(c, c->d_done); dev_free(c, c->d_term); dev_free(c, c->d_best); dev_free(c, c->d_best_step);
-    dev_free(c, c->d_best_nlog); dev_free(c, c->d_digest); dev_free(c, c->d_log); dev_free(c, c->d_F);
+    c->d_cand_layout = nullptr; c->d_inc_slot = nullptr;
     c->d_anc = nullptr; c->d_anc_next = nullptr; c->d_done = nullptr; c->d_term = nullptr; c->d_best = nullptr; c->d_best_step = nullptr;
-    c->d_best_nlog = nullptr; c->d_digest = nullptr; c->d_log = nullptr; c->d_F = nullptr;
+    c->d_best_nlog = nullptr; c->d_digest = nullptr; c->d_F = nullptr;
+    dev_free(c, c->d_sel_dist); c->d_sel_dist = nullptr;
+    dev_free(c, c->d_log); c->d_log = nullptr;
     c->log_cap = 0;
 }
 
@@ -145,11 +141,7 @@ extern "C" void rp_destroy(rp_ctx *c)
     if (!c) return;
     cudaStreamSynchronize(c->stream);
     free_population(c); free_trace(c); free_eval(c);
-    dev_free(c, c->own_t); dev_free(c, c->own_a); dev_free(c, c->d_edp);      // d_dp_list and d_dp_off live in d_edp's block
-    dev_free(c, c->d_Lagg); dev_free(c, c->d_pi); dev_free(c, c->d_inv); dev_free(c, c->d_rank_load); dev_free(c, c->d_q);
-    dev_free(c, c->d_status); dev_free(c, c->d_sort_keys); dev_free(c, c->d_seed_layout); dev_free(c, c->d_order); dev_free(c, c->d_pack_out);
-    dev_free(c, c->d_counters); dev_free(c, c->d_inc_layout); dev_free(c, c->d_inc_score); dev_free(c, c->d_static);
-    dev_free(c, c->d_seed_score); dev_free(c, c->d_best_score); dev_free(c, c->d_best_f64);
+    dev_free(c, c->own_t); dev_free(c, c->own_a); dev_free(c, c->d_load_slab); dev_free(c, c->d_static);
     pin_give(c->h_pin);
     free(c->h_levels);
     free(c);
@@ -227,19 +219,41 @@ static int window_load_impl(rp_ctx *c, const rp_config *cfg, const int32_t *leng
             if (cudaMemcpyAsync(c->own_a, demand, sizeof(int) * n_a, cudaMemcpyHostToDevice, c->stream) != cudaSuccess) { st = RP_ERR_CUDA; break; }
             c->d_a = c->own_a;
         }
+        // everything sized by the window alone comes out of one allocation
+        int n_pow2 = 1;
+        while (n_pow2 < N) n_pow2 <<= 1;
+        const size_t n_tab = (size_t)2 * D + G + 1;
+        RpSlab slab = { nullptr, 0 };
+        for (int pass = 0; pass < 2 && st == RP_OK; ++pass) {
+            slab.off = 0;
+            slab.take(&c->d_Lagg, (size_t)L * E);
+            slab.take(&c->d_status, RP_SW_COUNT);
+            slab.take(&c->d_counters, 8);
+            slab.take(&c->d_edp, n_tab);
+            slab.take(&c->d_pi, (size_t)L * E);
+            slab.take(&c->d_inv, (size_t)L * E);
+            slab.take(&c->d_rank_load, (size_t)L * P);
+            slab.take(&c->d_q, (size_t)N * L * P);
+            slab.take(&c->d_sort_keys, (size_t)2 * n_pow2);
+            slab.take(&c->d_seed_layout, N);
+            slab.take(&c->d_order, N);
+            slab.take(&c->d_pack_out, 4);
+            slab.take(&c->d_inc_layout, N);
+            slab.take(&c->d_inc_score, 3);
+            slab.take(&c->d_seed_score, 3);
+            slab.take(&c->d_best_score, 3);
+            slab.take(&c->d_best_f64, 3);
+            if (pass == 0) { st = dev_alloc(c, &c->d_load_slab, slab.off); slab.base = c->d_load_slab; }
+        }
+        if (st != RP_OK) break;
+        c->d_dp_list = c->d_edp + D;
+        c->d_dp_off = c->d_dp_list + D;
         // input checks + aggregate expert load + token total in one pass over the demand tensor,
         // put in flight before the rest of the set-up
-        if ((st = dev_alloc(c, &c->d_Lagg, (size_t)L * E)) != RP_OK) break;
-        if ((st = dev_alloc(c, &c->d_status, RP_SW_COUNT)) != RP_OK) break;
-        if ((st = dev_alloc(c, &c->d_counters, 8)) != RP_OK) break;
         if (cudaMemsetAsync(c->d_counters, 0, sizeof(i64) * 8, c->stream) != cudaSuccess) { st = RP_ERR_CUDA; break; }
         if ((st = reset_status(c)) != RP_OK) break;
         if ((st = rp_launch_check_reduce(c)) != RP_OK) break;
-        // the EDP tables: one allocation, one copy (pageable source: staged before the call returns)
-        const size_t n_tab = (size_t)2 * D + G + 1;
-        if ((st = dev_alloc(c, &c->d_edp, n_tab)) != RP_OK) break;
-        c->d_dp_list = c->d_edp + D;
-        c->d_dp_off = c->d_dp_list + D;
+        // the EDP tables: one copy (pageable source: staged before the call returns)
         int *tab = (int *)malloc(sizeof(int) * n_tab);
         memcpy(tab, edp, sizeof(int) * D);
         memcpy(tab + D, list, sizeof(int) * D);
@@ -250,21 +264,6 @@ static int window_load_impl(rp_ctx *c, const rp_config *cfg, const int32_t *leng
     } while (0);
     free(edp); free(off); free(list);
     RP_TRY(st);
-    RP_TRY(dev_alloc(c, &c->d_pi, (size_t)L * E));
-    RP_TRY(dev_alloc(c, &c->d_inv, (size_t)L * E));
-    RP_TRY(dev_alloc(c, &c->d_rank_load, (size_t)L * P));
-    RP_TRY(dev_alloc(c, &c->d_q, (size_t)N * L * P));
-    int n_pow2 = 1;
-    while (n_pow2 < N) n_pow2 <<= 1;
-    RP_TRY(dev_alloc(c, &c->d_sort_keys, (size_t)2 * n_pow2));
-    RP_TRY(dev_alloc(c, &c->d_seed_layout, N));
-    RP_TRY(dev_alloc(c, &c->d_order, N));
-    RP_TRY(dev_alloc(c, &c->d_pack_out, 4));
-    RP_TRY(dev_alloc(c, &c->d_inc_layout, N));
-    RP_TRY(dev_alloc(c, &c->d_inc_score, 3));
-    RP_TRY(dev_alloc(c, &c->d_seed_score, 3));
-    RP_TRY(dev_alloc(c, &c->d_best_score, 3));
-    RP_TRY(dev_alloc(c, &c->d_best_f64, 3));
 
     // verdict of the checks and the token total ride back in the pinned block
     RP_CUDA(cudaMemcpyAsync(c->h_pin + 8, c->d_counters + 7, sizeof(i64), cudaMemcpyDeviceToHost, c->stream));
@@ -396,24 +395,30 @@ extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
     // population buffers
     free_population(c); free_eval(c);
     const size_t P = (size_t)c->Ppop, wn = (size_t)dm.RG * dm.LP;
-    for (int b = 0; b < 2; ++b) {
-        RP_TRY(dev_alloc(c, &c->buf[b].blob, P * (size_t)c->bl.bytes));
+    {
+        RpSlab slab = { nullptr, 0 };
+        for (int pass = 0; pass < 2; ++pass) {
+            slab.off = 0;
+            slab.take(&c->buf[0].blob, P * (size_t)c->bl.bytes);
+            slab.take(&c->buf[1].blob, P * (size_t)c->bl.bytes);
+            slab.take(&c->d_W, 2 * P * wn);
+            slab.take(&c->d_wloc, P);
+            slab.take(&c->d_wloc_next, P);
+            slab.take(&c->d_le_scratch, 6 * P);
+            slab.take(&c->d_inc_slot, 1);
+            if (rp_uses_wpc(c->dm)) slab.take(&c->d_cand_layout, P * (size_t)c->dm.N);
+            slab.take(&c->d_anc, P);
+            slab.take(&c->d_anc_next, P);
+            slab.take(&c->d_done, 1);
+            slab.take(&c->d_term, P * 3);
+            slab.take(&c->d_best, P * 3);
+            slab.take(&c->d_best_step, P);
+            slab.take(&c->d_best_nlog, P);
+            slab.take(&c->d_digest, P);
+            slab.take(&c->d_F, P);
+            if (pass == 0) { RP_TRY(dev_alloc(c, &c->d_pop_slab, slab.off)); slab.base = c->d_pop_slab; }
+        }
     }
-    RP_TRY(dev_alloc(c, &c->d_W, 2 * P * wn));
-    RP_TRY(dev_alloc(c, &c->d_wloc, P));
-    RP_TRY(dev_alloc(c, &c->d_wloc_next, P));
-    RP_TRY(dev_alloc(c, &c->d_le_scratch, 6 * P));
-    RP_TRY(dev_alloc(c, &c->d_inc_slot, 1));
-    if (rp_uses_wpc(c->dm)) RP_TRY(dev_alloc(c, &c->d_cand_layout, P * (size_t)c->dm.N));
-    RP_TRY(dev_alloc(c, &c->d_anc, P));
-    RP_TRY(dev_alloc(c, &c->d_anc_next, P));
-    RP_TRY(dev_alloc(c, &c->d_done, 1));
-    RP_TRY(dev_alloc(c, &c->d_term, P * 3));
-    RP_TRY(dev_alloc(c, &c->d_best, P * 3));
-    RP_TRY(dev_alloc(c, &c->d_best_step, P));
-    RP_TRY(dev_alloc(c, &c->d_best_nlog, P));
-    RP_TRY(dev_alloc(c, &c->d_digest, P));
-    RP_TRY(dev_alloc(c, &c->d_F, P));
     c->cur = 0;
     // every member starts as the length-only seed: evaluate it once into slot 0 and let all
     // slots descend from slot 0

@@ -95,6 +95,8 @@ struct rp_ctx {
     const int *d_t;            // [N]
     const int *d_a;            // [N][L][E]
     int *own_t, *own_a;        // non-null when this context allocated the copies
+    char *d_load_slab;         // one allocation behind the buffers sized by the window alone (freed by rp_destroy)
+    char *d_pop_slab;          // one allocation behind the population buffers (sized after packing)
     int *d_edp;                // [D]
     int *d_dp_list;            // [D] DP slots grouped by shard
     int *d_dp_off;             // [G+1]
@@ -196,6 +198,20 @@ static inline int dev_alloc(rp_ctx *c, T **p, size_t n)
     return RP_OK;
 }
 static inline void dev_free(rp_ctx *c, void *p) { if (p) cudaFreeAsync(p, c->stream); }
+
+// Carves 256-byte aligned pieces out of one allocation: first pass (base == nullptr) adds up the
+// sizes, second pass hands out the pointers.
+struct RpSlab {
+    char *base;
+    size_t off;
+    template <class T>
+    void take(T **p, size_t n)
+    {
+        if (n == 0) n = 1;
+        if (base) *p = (T *)(base + off);
+        off = (off + n * sizeof(T) + 255) & ~(size_t)255;
+    }
+};
 
 int rp_launch_select(rp_ctx *c, int *lay, int *out, const i64 *score, int n_proj, i64 eta_q16, int *order,
                      int *n_distinct, i64 *dist);
