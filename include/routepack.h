@@ -94,6 +94,10 @@ typedef struct {
  * rp_pack_rows returns: rp_place_experts may leave its work queued on the stream) and checks 1 <= t_i <= C, a >= 0 and sum_e a[i][l][e] == k*t_i.
  *   lengths [N] int32; demand [N][L][E] int32, expert index fastest.
  *   cuda_stream: a cudaStream_t (NULL = default stream).
+ * The placement, projection and packing kernels depend on nothing but these inputs and are queued
+ * on the stream right behind the checks, so the GPU is already working on them while the host
+ * waits for the verdict; rp_place_experts and rp_pack_rows then hand their results over (and
+ * compute them themselves when called again).
  * On failure *out is NULL. */
 int rp_window_load(rp_ctx **out, const rp_config *cfg, const int32_t *lengths,
                    const int32_t *demand, void *cuda_stream);

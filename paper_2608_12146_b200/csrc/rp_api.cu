@@ -265,11 +265,20 @@ static int window_load_impl(rp_ctx *c, const rp_config *cfg, const int32_t *leng
     free(edp); free(off); free(list);
     RP_TRY(st);
 
+    // Placement, projection and packing depend on nothing but the inputs: they are queued right
+    // behind the checks, so that the GPU works on them while the host waits for the verdict
+    // (rp_place_experts and rp_pack_rows then only hand the results over).
+    c->eager_place = (rp_launch_lpt(c) == RP_OK && rp_launch_project(c) == RP_OK);
+    c->eager_pack = (rp_launch_pack(c, 0) == RP_OK);
+    if (c->eager_pack)
+        RP_CUDA(cudaMemcpyAsync(c->h_pin + 10, c->d_pack_out, sizeof(int) * 4, cudaMemcpyDeviceToHost, c->stream));
+
     // verdict of the checks and the token total ride back in the pinned block
     RP_CUDA(cudaMemcpyAsync(c->h_pin + 8, c->d_counters + 7, sizeof(i64), cudaMemcpyDeviceToHost, c->stream));
     int sw[RP_SW_COUNT];
     RP_TRY(read_status(c, sw));
     if (sw[RP_SW_BAD_SAMPLE]) return RP_ERR_CONSERVATION;
+    memcpy(c->pack_out, c->h_pin + 10, sizeof(int) * 4);
 
     // fixed-point range of the score: s1 <= (2^8*C*L*k + (asum+bsum)*C) * sum t  must stay below 2^62
     const double total = (double)c->h_pin[8];
@@ -316,8 +325,11 @@ extern "C" int rp_place_experts(rp_ctx *c, int32_t *pi, int64_t *rank_load)
     if (!c) return RP_ERR_ARG;
     if (c->stage < 1) return RP_ERR_STATE;
     const RpDims &dm = c->dm;
-    RP_TRY(rp_launch_lpt(c));
-    RP_TRY(rp_launch_project(c));
+    if (!c->eager_place) {
+        RP_TRY(rp_launch_lpt(c));
+        RP_TRY(rp_launch_project(c));
+    }
+    c->eager_place = 0;               // a repeated call recomputes
     RP_TRY(copy_out(c, pi, c->d_pi, sizeof(int) * (size_t)dm.L * dm.E));
     RP_TRY(copy_out(c, rank_load, c->d_rank_load, sizeof(i64) * (size_t)dm.L * dm.P));
     // Host outputs are complete when the call returns; device outputs are ordered on the stream.
@@ -379,10 +391,14 @@ extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
     if (c->stage < 2) return RP_ERR_STATE;
     RpDims &dm = c->dm;
     c->best_ready = 0;
-    RP_TRY(rp_launch_pack(c, 0));
-    int *po = (int *)c->h_pin;
-    RP_CUDA(cudaMemcpyAsync(po, c->d_pack_out, sizeof(int) * 4, cudaMemcpyDeviceToHost, c->stream));
-    RP_CUDA(cudaStreamSynchronize(c->stream));
+    int *po = c->pack_out;
+    if (!c->eager_pack) {
+        RP_TRY(rp_launch_pack(c, 0));
+        RP_CUDA(cudaMemcpyAsync(c->h_pin + 10, c->d_pack_out, sizeof(int) * 4, cudaMemcpyDeviceToHost, c->stream));
+        RP_CUDA(cudaStreamSynchronize(c->stream));
+        memcpy(c->pack_out, c->h_pin + 10, sizeof(int) * 4);
+    }
+    c->eager_pack = 0;                // a repeated call recomputes
     if (po[3] || po[0] <= 0) return RP_ERR_INFEASIBLE;
     c->Rstar = po[0]; c->certified = po[1];
     dm.R = po[0]; dm.K = dm.R * dm.D; dm.RG = dm.R * dm.G;

@@ -145,6 +145,8 @@ struct rp_ctx {
     i64 *d_inc_score;          // [3]
     i64 *d_best_score;         // [3] full rescoring of the incumbent (validation)
     double *d_best_f64;        // [3] the same as the real-valued objective
+    int eager_place, eager_pack;   // rp_window_load already queued the placement / packing kernels behind its checks
+    int pack_out[4];           // R*, certified, R_lb, failure flag as read back with the load's verdict
     int best_ready;            // the incumbent has been validated and rescored since it last changed
     int best_verdict;          // RP_OK or RP_ERR_INVALID_PLAN of that validation
     // trace of the last rp_anneal call
