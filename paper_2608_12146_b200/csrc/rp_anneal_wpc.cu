@@ -33,6 +33,51 @@ struct ChainS {                 // bookkeeping of the chain within this level
     int has_snap;               // best_lay holds a layout that beats it
 };
 
+// Terminal state out of shared memory without waiting for it to land (the caller has fenced the
+// shared-memory writes for the bulk engine and synchronised the CTA).
+template <int NT, bool WS>
+__device__ __forceinline__ void rp_chain_store_async(const AnnealArgs &A, int j, const char *sm_blob, const int *Wsm, int tid)
+{
+    const RpDims &dm = A.dm;
+    const size_t wn = (size_t)dm.RG * dm.LP;
+    const bool w_bulk = WS && ((wn & 3) == 0);
+    if (tid == 0) {
+        rp_bulk_s2g(A.blob_dst + (size_t)j * A.bl.bytes, sm_blob, (u32)A.bl.bytes);
+        if (w_bulk) {
+            int *wd = A.W + (size_t)A.wloc_dst[j] * wn;
+            for (size_t off = 0; off < wn * 4; off += 32768) {
+                const u32 n = (u32)((wn * 4 - off) < 32768 ? (wn * 4 - off) : 32768);
+                rp_bulk_s2g((char *)wd + off, (const char *)Wsm + off, n);
+            }
+        }
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    }
+    if (WS && !w_bulk) {
+        int *wd = A.W + (size_t)A.wloc_dst[j] * wn;
+        for (size_t x = tid; x < wn; x += NT) wd[x] = Wsm[x];
+    }
+}
+
+// Tail of a chain CTA whose bulk stores are still in flight: publish the report, take a ticket,
+// wait until the stores have read shared memory (it is about to be reused or released), and let
+// the last arrival run the level barrier.
+__device__ __forceinline__ void rp_finish_level_async(const AnnealArgs &A, int tid, int nt, unsigned char *ws, size_t ws_bytes)
+{
+    __shared__ int is_last_a;
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const int ticket = atomicAdd(A.lo.done, 1);
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");      // this thread issued them
+        is_last_a = (ticket == (int)gridDim.x - 1);
+        if (is_last_a) *A.lo.done = 0;
+    }
+    __syncthreads();
+    if (!is_last_a) return;
+    __threadfence();
+    rp_level_end(A, tid, nt, ws, ws_bytes);
+}
+
 template <int NW, bool WS, int CH>
 __global__ void __launch_bounds__(NW * 32, 16 / NW)
 k_anneal_wpc(const AnnealArgs A)
@@ -380,8 +425,12 @@ k_anneal_wpc(const AnnealArgs A)
         }
     }
 
-    // ---- epilogue: terminal state and chain report ------------------------------------------
-    rp_chain_store<NT, WS>(A, j, sm_blob, Wsm, tid);
+    // ---- epilogue: chain report, then the terminal state ---------------------------------------
+    // The level barrier reads only the reports (and the layout snapshots), so those go out first
+    // with plain stores; the state itself leaves by asynchronous bulk copies that need not have
+    // landed before the ticket is taken (the next level starts after this grid has completed).
+    rp_fence_async_smem();                 // generic-proxy writes to shared memory -> visible to the bulk engine
+    __syncthreads();
     if (chain->has_snap) {
         unsigned short *row = A.lo.cand_layout + (size_t)j * dm.N;
         for (int x = tid; x < dm.N; x += NT) row[x] = best_lay[x];
@@ -399,8 +448,9 @@ k_anneal_wpc(const AnnealArgs A)
         A.digest[j] = chain->dig;
         atomicAdd((u64 *)&A.counters[0], (u64)A.steps);
     }
+    rp_chain_store_async<NT, WS>(A, j, sm_blob, Wsm, tid);
     asm volatile("griddepcontrol.launch_dependents;");     // the next level may start its own prologue
-    rp_finish_level(A, tid, NT, smraw, A.smem_bytes);
+    rp_finish_level_async(A, tid, NT, smraw, A.smem_bytes);
 }
 
 // Warps per chain: more warps score more candidates of a round at once (good when few chains
