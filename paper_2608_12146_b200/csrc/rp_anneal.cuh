@@ -186,6 +186,15 @@ __device__ __forceinline__ i64 warp_max_i64(i64 v)
     for (int o = 16; o; o >>= 1) { i64 x = __shfl_xor_sync(0xffffffffu, v, o); v = x > v ? x : v; }
     return v;
 }
+// Warp maximum of non-negative 64-bit values with two reduction instructions: the largest high
+// word, then the largest low word among the lanes that hold it.
+__device__ __forceinline__ i64 warp_max_nonneg_i64(i64 v)
+{
+    const u32 hi = (u32)((u64)v >> 32), lo = (u32)v;
+    const u32 mh = __reduce_max_sync(0xffffffffu, hi);
+    const u32 ml = __reduce_max_sync(0xffffffffu, hi == mh ? lo : 0u);
+    return (i64)(((u64)mh << 32) | ml);
+}
 __device__ __forceinline__ i64 warp_sum_i64(i64 v)
 {
     for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

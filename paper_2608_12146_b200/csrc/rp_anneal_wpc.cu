@@ -312,13 +312,13 @@ k_anneal_wpc(const AnnealArgs A)
                     if (fb & 1) {       // the previous maximum sat on a changed entry and fell: rescan
                         i64 v = 0;
                         for (int g = lane; g < dm.G; g += 32) if (g != g1 && g != g2 && U[g] > v) v = U[g];
-                        v = warp_max_i64(v);
+                        v = warp_max_nonneg_i64(v);
                         if (lane == 0 && v > n0) n0 = v;
                     }
                     if (fb & 2) {
                         i64 v = 0;
                         for (int rg = lane; rg < dm.RG; rg += 32) if (rg != rg1 && rg != rg2 && Jfx[rg] > v) v = Jfx[rg];
-                        v = warp_max_i64(v);
+                        v = warp_max_nonneg_i64(v);
                         if (lane == 0 && v > n2) n2 = v;
                     }
                     if (lane == 0) {
