@@ -330,6 +330,37 @@ def seeding_stages(rp, torch, name, dev, reps=3):
             "choice_width": 4, "n_proj": 8, "eta_q16": 1 << 16}
 
 
+def eval_stage(rp, torch, name, dev, reps=10):
+    """Context figure: full scoring of one population-sized batch of layouts (rp_eval_population,
+    device inputs and outputs): layouts/s and algorithmic bytes (N*2 + N*L*P*4 per layout) per second."""
+    import numpy as np
+    w = make_window(SPECS[name])
+    s = w.spec
+    t_dev = torch.from_numpy(w.lengths).to(dev)
+    a_dev = torch.from_numpy(w.demand).to(dev)
+    ctx = rp.rp_window_load(t_dev, a_dev, top_k=s.top_k, token_cap=s.token_cap, dp_width=s.dp_width,
+                            ep_width=s.ep_width, pop_size=s.pop_size, alpha=s.alpha, beta=s.beta, seed=s.anneal_seed)
+    rp.rp_place_experts(ctx)
+    rp.rp_pack_rows(ctx)
+    rp.rp_seed_population(ctx, 4)                  # distinct layouts, one per member
+    lays = torch.from_numpy(rp.rp_debug_dump(ctx, "POPULATION", (s.pop_size, s.n_samples), np.int32)).to(dev)
+    fx = torch.empty((s.pop_size, 3), dtype=torch.int64, device=dev)
+    f64 = torch.empty((s.pop_size, 3), dtype=torch.float64, device=dev)
+    for _ in range(3):
+        rp.rp_eval_population(ctx, lays, fx, f64)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        rp.rp_eval_population(ctx, lays, fx, f64)
+    e1.record()
+    e1.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    rp.rp_destroy(ctx)
+    byts = s.pop_size * (s.n_samples * 2 + s.n_samples * s.n_layers * s.ep_width * 4)
+    return {"workload": name, "layouts": s.pop_size, "ms": ms, "layouts_per_s": s.pop_size / ms * 1e3,
+            "algorithmic_gbs": byts / ms / 1e6}
+
+
 def run_cuda(args):
     import torch
     import paper_2608_12146_b200.binding as rp
@@ -369,6 +400,7 @@ def run_cuda(args):
             line["other_workloads"] = sweep
         if args.sweep and world == 1 and not args.pop and not args.levels:
             line["seeding_stages"] = seeding_stages(rp, torch, args.workload, dev)
+            line["eval_population"] = [eval_stage(rp, torch, n, dev) for n in ("medium", "large", "wide")]
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
