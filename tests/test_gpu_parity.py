@@ -428,6 +428,53 @@ def test_fuzz_random_small_windows():
         rp.rp_destroy(ctx)
 
 
+def test_fuzz_seeding_stages():
+    """Random shapes (one to six DP slots, one to all shards, 1..48 ranks, populations of 1..33,
+    choice widths 1..32, one to nine projections, zero to large eta): trial loop, pairing and
+    selection against the oracle, stage by stage."""
+    rng = np.random.default_rng(77)
+    done = 0
+    for trial in range(16):
+        P = int(rng.choice([1, 2, 3, 4, 8, 16, 48]))
+        E = P * int(rng.choice([1, 2]))
+        L = int(rng.integers(1, 6))
+        D = int(rng.choice([1, 2, 3, 4, 6]))
+        N = int(rng.integers(max(12, 4 * D), 140))
+        k = int(rng.choice([1, 2, 4]))
+        C = int(rng.choice([512, 3000, 8192]))
+        G = int(rng.integers(1, D + 1))
+        edp = None if G == D else [int(x) for x in rng.permutation(np.concatenate([np.arange(G), rng.integers(0, G, D - G)]))]
+        pop = int(rng.choice([1, 2, 7, 20, 33]))
+        spec = custom_spec(f"seedfuzz{trial}", N, L, E, k, C, D, P, pop, 0, data_seed=3000 + trial,
+                           anneal_seed=int(rng.integers(0, 2 ** 62)))
+        w = make_window(spec)
+        s = w.spec
+        min_rows = int(rng.integers(1, 4))
+        ref = oracle_front(w, edp, min_rows)
+        if ref["R"] == 0:
+            continue
+        ctx = load(w, pop=pop, edp=edp, min_rows=min_rows)
+        check_front(w, ctx, ref)
+        w1, w2 = int(rng.choice([1, 2, 5, 32])), int(rng.choice([1, 3, 32]))
+        n_proj, eta = int(rng.integers(1, 10)), int(rng.choice([0, 1 << 12, 1 << 16, 1 << 24]))
+        lays, ok = oracle.seed_trials(w.lengths, ref["seed"], ref["R"], s.token_cap, s.dp_width, pop, w1, s.anneal_seed)
+        assert rp.rp_seed_population(ctx, w1) == int(ok.sum())
+        assert (rp.rp_debug_dump(ctx, "POPULATION", (pop, s.n_samples), np.int32) == lays).all()
+        paired = oracle.edp_pair(ref["q"], lays, ref["R"], s.dp_width, w2, s.anneal_seed, edp)
+        assert rp.rp_pair_population(ctx, w2) == int((paired != lays).any(axis=1).sum())
+        assert (rp.rp_debug_dump(ctx, "POPULATION", (pop, s.n_samples), np.int32) == paired).all()
+        sc = oracle.eval_layouts(w.lengths, ref["q"], paired, ref["R"], s.token_cap, s.dp_width, edp, s.alpha, s.beta)["score"]
+        want = oracle.select_population(w.lengths, ref["q"], paired, sc, ref["R"], s.token_cap, s.dp_width, s.top_k, n_proj, eta,
+                                        s.anneal_seed, edp)
+        nd, order = rp.rp_select_population(ctx, n_proj, eta)
+        assert nd == want["n_distinct"] and (order == want["order"]).all()
+        assert (rp.rp_debug_dump(ctx, "POPULATION", (pop, s.n_samples), np.int32) == want["layouts"]).all()
+        check_anneal(w, ctx, ref, edp, pop, 2, 20, t_ratio=0.5, check_members=1, init=want["layouts"])
+        rp.rp_destroy(ctx)
+        done += 1
+    assert done >= 10
+
+
 def test_bad_inputs_are_host_side_errors():
     w = make_window("tiny")
     s = w.spec
