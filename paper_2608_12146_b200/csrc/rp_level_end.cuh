@@ -96,6 +96,28 @@ __device__ __forceinline__ void le_prefix_weights(const AnnealArgs &A, int tid, 
     }
 }
 
+// Lane holding the lexicographically smallest (v0, v1, v2) among the lanes with j != INT_MAX
+// (lowest j on ties), by reduction instructions: for each key the smallest high word, then the
+// smallest low word among the lanes still in the race.  Keys are non-negative.  Returns -1 when
+// no lane has a candidate.  All lanes must call.
+__device__ __forceinline__ int le_lexmin_lane(i64 v0, i64 v1, i64 v2, int j)
+{
+    bool alive = (j != 0x7fffffff);
+    const i64 key[3] = { v0, v1, v2 };
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+        const u32 hi = alive ? (u32)((u64)key[k] >> 32) : 0xffffffffu;
+        const u32 mh = __reduce_min_sync(0xffffffffu, hi);
+        alive = alive && (hi == mh);
+        const u32 lo = alive ? (u32)key[k] : 0xffffffffu;
+        const u32 ml = __reduce_min_sync(0xffffffffu, lo);
+        alive = alive && (lo == ml);
+    }
+    const int mj = (int)__reduce_min_sync(0xffffffffu, alive ? (unsigned)j : 0x7fffffffu);
+    const unsigned who = __ballot_sync(0xffffffffu, alive && j == mj);
+    return who ? __ffs(who) - 1 : -1;
+}
+
 // Called by all threads of one CTA (nt a multiple of 32, at most 1024).  `ws` is the CTA's
 // dynamic shared memory, free once the chain has been stored: the cumulative weights and the
 // replayed layout live there when they fit (global memory otherwise), which keeps the
@@ -140,25 +162,33 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
         const i64 e = rp_energy(t0, t1, t2);
         emin = e < emin ? e : emin;
     }
-    for (int o = 16; o; o >>= 1) { const i64 x = __shfl_xor_sync(0xffffffffu, emin, o); emin = x < emin ? x : emin; }
+    {   // warp minimum of the (non-negative) energies: smallest high word, then smallest low word among its holders
+        const u32 hi = (u32)((u64)emin >> 32), mh = __reduce_min_sync(0xffffffffu, hi);
+        const u32 ml = __reduce_min_sync(0xffffffffu, hi == mh ? (u32)emin : 0xffffffffu);
+        emin = (i64)(((u64)mh << 32) | ml);
+    }
     if (lane == 0) rmin[warp] = emin;
     if (__syncthreads_or(bj != 0x7fffffff)) {
-    for (int o = 16; o; o >>= 1) {
-        i64 o0 = __shfl_xor_sync(0xffffffffu, b0, o), o1 = __shfl_xor_sync(0xffffffffu, b1, o);
-        i64 o2 = __shfl_xor_sync(0xffffffffu, b2, o);
-        int oj = __shfl_xor_sync(0xffffffffu, bj, o);
-        const int on = __shfl_xor_sync(0xffffffffu, bn, o), oa = __shfl_xor_sync(0xffffffffu, ba, o);
-        bool take = rp_lex_less(o0, o1, o2, b0, b1, b2) || (o0 == b0 && o1 == b1 && o2 == b2 && oj < bj);
-        if (take) { b0 = o0; b1 = o1; b2 = o2; bj = oj; bn = on; ba = oa; }
+    {
+        const int src = le_lexmin_lane(b0, b1, b2, bj);         // this warp's best, handed to lane 0
+        if (src >= 0) {
+            b0 = __shfl_sync(0xffffffffu, b0, src); b1 = __shfl_sync(0xffffffffu, b1, src); b2 = __shfl_sync(0xffffffffu, b2, src);
+            bj = __shfl_sync(0xffffffffu, bj, src); bn = __shfl_sync(0xffffffffu, bn, src); ba = __shfl_sync(0xffffffffu, ba, src);
+        }
     }
     if (lane == 0) { r0[warp] = b0; r1[warp] = b1; r2[warp] = b2; rj[warp] = bj; rn[warp] = bn; ra[warp] = ba; }
     __syncthreads();
-    if (tid == 0) {
-        for (int w = 1; w < nwarps; ++w) {
-            bool take = rp_lex_less(r0[w], r1[w], r2[w], b0, b1, b2) ||
-                        (r0[w] == b0 && r1[w] == b1 && r2[w] == b2 && rj[w] < bj);
-            if (take) { b0 = r0[w]; b1 = r1[w]; b2 = r2[w]; bj = rj[w]; bn = rn[w]; ba = ra[w]; }
+    if (warp == 0) {                                            // the same over the warps' results
+        const bool has = lane < nwarps;
+        b0 = has ? r0[lane] : 0; b1 = has ? r1[lane] : 0; b2 = has ? r2[lane] : 0;
+        bj = has ? rj[lane] : 0x7fffffff; bn = has ? rn[lane] : 0; ba = has ? ra[lane] : 0;
+        const int src = le_lexmin_lane(b0, b1, b2, bj);
+        if (src >= 0) {
+            b0 = __shfl_sync(0xffffffffu, b0, src); b1 = __shfl_sync(0xffffffffu, b1, src); b2 = __shfl_sync(0xffffffffu, b2, src);
+            bj = __shfl_sync(0xffffffffu, bj, src); bn = __shfl_sync(0xffffffffu, bn, src); ba = __shfl_sync(0xffffffffu, ba, src);
         }
+    }
+    if (tid == 0) {
         win_j = bj; win_n = bn; win_a = ba;
         do_update = rp_lex_less(b0, b1, b2, i0, i1, i2);
         if (do_update) {
