@@ -46,7 +46,8 @@ __device__ __forceinline__ void le_weights(const i64 (&e)[U], i64 emin, u64 M, u
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const u64 cc = ((z[u] >> (32 - i)) & 1ull) ? c : (1ull << 63);
-            acc[u] = (__umul64hi(acc[u], cc) << 1) | ((acc[u] * cc) >> 63);
+            // (acc * cc) >> 63 = high word of (2*acc) * cc; acc = 2^63 (nothing applied yet) gives cc itself
+            acc[u] = (acc[u] >> 63) ? cc : __umul64hi(acc[u] << 1, cc);
         }
     }
 #pragma unroll
