@@ -342,6 +342,20 @@ int rp_anneal_smem_bytes(const rp_ctx *c, int *threads, size_t *bytes)
     return 0;
 }
 
+// Philox4x32-10 on the host (first output word): the resampling offset's random word depends only
+// on the seed and the level, so the level barrier does not have to compute it.
+static u32 host_philox_x(u32 c0, u32 c1, u32 c2, u32 c3, u32 k0, u32 k1)
+{
+    for (int r = 0; r < 10; ++r) {
+        const u64 p0 = (u64)0xD2511F53u * c0, p1 = (u64)0xCD9E8D57u * c2;
+        const u32 n0 = (u32)(p1 >> 32) ^ c1 ^ k0, n2 = (u32)(p0 >> 32) ^ c3 ^ k1;
+        c0 = n0; c1 = (u32)p1; c2 = n2; c3 = (u32)p0;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    return c0;
+}
+
 int rp_launch_anneal_level(rp_ctx *c, int level, int n_levels, const rp_anneal_params *prm, u64 rho_q32, u64 guide_q32)
 {
     AnnealArgs A;
@@ -354,6 +368,7 @@ int rp_launch_anneal_level(rp_ctx *c, int level, int n_levels, const rp_anneal_p
     A.level = level; A.steps = prm->steps_per_level; A.log_cap = c->log_cap;
     A.rho_q32 = rho_q32; A.guide_q32 = guide_q32;
     A.key0 = (u32)c->cfg.seed; A.key1 = (u32)(c->cfg.seed >> 32);
+    A.resample_x = host_philox_x(0u, (u32)level, 0u, 3u, A.key0, A.key1);
     A.term = c->d_term; A.best = c->d_best; A.best_step = c->d_best_step; A.best_nlog = c->d_best_nlog;
     A.digest = c->d_digest; A.log = c->d_log; A.counters = c->d_counters; A.status = c->d_status;
     A.tau = c->h_levels[level].tau;

@@ -40,6 +40,7 @@ struct AnnealArgs {
     unsigned smem_bytes;             // dynamic shared memory of the launch
     u64 tau, cq, rho_q32, guide_q32;
     u32 key0, key1;
+    u32 resample_x;                  // Philox(0, level, 0, 3).x, the word behind the resampling offset (computed on the host)
     i64 *term, *best;
     int *best_step, *best_nlog;
     u64 *digest;

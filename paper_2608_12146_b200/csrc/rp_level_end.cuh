@@ -268,8 +268,7 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
     else if (P <= 2 * nt) le_prefix_weights<2>(A, tid, nt, emin, M, F, rsum, &carry_s);
     else le_prefix_weights<4>(A, tid, nt, emin, M, F, rsum, &carry_s);
     const u64 Ftot = F[P - 1];
-    const uint4 xw = rp_philox(0u, (u32)A.level, 0u, 3u, A.key0, A.key1);
-    const u64 u0 = (u64)(((unsigned __int128)xw.x * Ftot) >> 32);
+    const u64 u0 = (u64)(((unsigned __int128)A.resample_x * Ftot) >> 32);
     int depth = 0;
     while ((1 << depth) < P) ++depth;
     constexpr int SU = 4;                       // searches per thread in flight
