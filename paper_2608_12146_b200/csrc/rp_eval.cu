@@ -75,12 +75,37 @@ k_eval(const unsigned short *__restrict__ cells, const int *__restrict__ t, cons
     for (int rg = blockIdx.y * nwarps + warp; rg < dm.RG; rg += gridDim.y * nwarps) {
         const int m0 = off[rg], m1 = off[rg + 1];
         int *wout = W_out ? W_out + ((size_t)lay * dm.RG + rg) * dm.LP : nullptr;
-        i64 es = rp_warp_layer_max_sum(dm, lane, [&](int x) {
-            int s = 0;
-            for (int m = m0; m < m1; ++m) s += __ldg(q + (size_t)members[m] * dm.LP + x);
-            if (wout) wout[x] = s;
-            return s;
-        });
+        i64 es;
+        if (dm.P <= 32 && (dm.P & (dm.P - 1)) == 0) {
+            // four strips of 32 columns at a time: four independent loads per member in flight, the
+            // busiest rank of a layer by segmented shuffles over the coalesced column order
+            es = 0;
+            for (int x0 = 0; x0 < dm.LP; x0 += 128) {
+                int acc[4] = { 0, 0, 0, 0 };
+#pragma unroll 2
+                for (int m = m0; m < m1; ++m) {
+                    const int *row = q + (size_t)members[m] * dm.LP + x0 + lane;
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) if (x0 + 32 * u + lane < dm.LP) acc[u] += __ldg(row + 32 * u);
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int x = x0 + 32 * u + lane;
+                    int v = (x < dm.LP) ? acc[u] : 0;
+                    if (wout && x < dm.LP) wout[x] = v;
+                    for (int o = dm.P >> 1; o; o >>= 1) v = max(v, __shfl_xor_sync(0xffffffffu, v, o));
+                    if ((lane & (dm.P - 1)) == 0 && x < dm.LP) es += v;
+                }
+            }
+            for (int o = 16; o; o >>= 1) es += __shfl_xor_sync(0xffffffffu, es, o);
+        } else {
+            es = rp_warp_layer_max_sum(dm, lane, [&](int x) {
+                int s = 0;
+                for (int m = m0; m < m1; ++m) s += __ldg(q + (size_t)members[m] * dm.LP + x);
+                if (wout) wout[x] = s;
+                return s;
+            });
+        }
         if (lane == 0) esum_lay[rg] = es;
     }
     __threadfence();
