@@ -386,7 +386,7 @@ k_anneal_wpc(const AnnealArgs A)
                         }
                         int snap = 0;
                         if (lane == 0) {
-                            const int c1 = m.c1, c2 = m.c2;
+                            const int c2 = m.c2;
                             const int k = kb + pos + my;
                             Esum[rg1] = e1; Afx[rg1] = A1; Jfx[rg1] = J1n;
                             if (touchW) { Esum[rg2] = e2; Afx[rg2] = A2; Jfx[rg2] = J2n; }

@@ -32,6 +32,9 @@ int rp_launch_cells_from_layouts(rp_ctx *c, const int *layouts, int n, unsigned 
 
 // grid = (layouts, splits): the CTAs of a layout share its row-shards (8 per CTA, one per warp);
 // the CTA that finishes last (atomic ticket) gathers the row-shard sums and scores the layout.
+// DEEP: eight members' loads in flight per pass (few layouts: latency matters); otherwise two
+// (many layouts: the CTAs in flight hide the latency and registers are better spent on occupancy).
+template <bool DEEP>
 __global__ void __launch_bounds__(EVAL_THREADS)
 k_eval(const unsigned short *__restrict__ cells, const int *__restrict__ t, const int *__restrict__ q,
        const int *__restrict__ edp, const int *__restrict__ dp_list, const int *__restrict__ dp_off,
@@ -82,11 +85,28 @@ k_eval(const unsigned short *__restrict__ cells, const int *__restrict__ t, cons
             es = 0;
             for (int x0 = 0; x0 < dm.LP; x0 += 128) {
                 int acc[4] = { 0, 0, 0, 0 };
-#pragma unroll 2
-                for (int m = m0; m < m1; ++m) {
-                    const int *row = q + (size_t)members[m] * dm.LP + x0 + lane;
+                if constexpr (DEEP) {
+                    for (int mb = m0; mb < m1; mb += 8) {      // eight members' loads in flight before any is added
+                        int v[8][4];
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) if (x0 + 32 * u + lane < dm.LP) acc[u] += __ldg(row + 32 * u);
+                        for (int e = 0; e < 8; ++e) {
+                            const bool on = mb + e < m1;
+                            const int *row = q + (size_t)(on ? members[mb + e] : 0) * dm.LP + x0 + lane;
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) v[e][u] = (on && x0 + 32 * u + lane < dm.LP) ? __ldg(row + 32 * u) : 0;
+                        }
+#pragma unroll
+                        for (int e = 0; e < 8; ++e)
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) acc[u] += v[e][u];
+                    }
+                } else {
+#pragma unroll 2
+                    for (int m = m0; m < m1; ++m) {
+                        const int *row = q + (size_t)members[m] * dm.LP + x0 + lane;
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) if (x0 + 32 * u + lane < dm.LP) acc[u] += __ldg(row + 32 * u);
+                    }
                 }
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
@@ -163,16 +183,23 @@ int rp_launch_eval(rp_ctx *c, const unsigned short *cells, int n, int *W_out, ch
     const RpDims &dm = c->dm;
     size_t smem = eval_smem_bytes(dm);
     if (smem > 220 * 1024) return RP_ERR_RANGE;
-    if (smem > 32 * 1024)
-        RP_CUDA(cudaFuncSetAttribute(k_eval, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    if (smem > 32 * 1024) {
+        RP_CUDA(cudaFuncSetAttribute(k_eval<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        RP_CUDA(cudaFuncSetAttribute(k_eval<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    }
     // few layouts: split each one's row-shards over several CTAs so the GPU is not left idle
     int splits = (2 * 148 + n - 1) / n;
     const int max_splits = (dm.RG + EVAL_THREADS / 32 - 1) / (EVAL_THREADS / 32);
     if (splits > max_splits) splits = max_splits;
     if (splits < 1) splits = 1;
-    k_eval<<<dim3(n, splits), EVAL_THREADS, smem, c->stream>>>(cells, c->d_t, c->d_q, c->d_edp, c->d_dp_list, c->d_dp_off,
-                                                              dm, c->bl, W_out, blob_out, score_out, f64_out,
-                                                              c->d_eval_Esum, c->d_eval_tickets);
+    if ((long long)n * splits <= 2 * 148)
+        k_eval<true><<<dim3(n, splits), EVAL_THREADS, smem, c->stream>>>(cells, c->d_t, c->d_q, c->d_edp, c->d_dp_list, c->d_dp_off,
+                                                                        dm, c->bl, W_out, blob_out, score_out, f64_out,
+                                                                        c->d_eval_Esum, c->d_eval_tickets);
+    else
+        k_eval<false><<<dim3(n, splits), EVAL_THREADS, smem, c->stream>>>(cells, c->d_t, c->d_q, c->d_edp, c->d_dp_list, c->d_dp_off,
+                                                                         dm, c->bl, W_out, blob_out, score_out, f64_out,
+                                                                         c->d_eval_Esum, c->d_eval_tickets);
     ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
     return RP_OK;
@@ -347,13 +374,13 @@ extern "C" int rp_diagnostics(rp_ctx *c, const int32_t *layout, rp_diag *out)
         const size_t smem = eval_smem_bytes(dm);
         if (smem > 220 * 1024) { st = RP_ERR_RANGE; break; }
         if (smem > 32 * 1024) {
-            e = cudaFuncSetAttribute(k_eval, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            e = cudaFuncSetAttribute(k_eval<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) break;
         }
         int splits = 2 * 148;
         const int max_splits = (dm.RG + EVAL_THREADS / 32 - 1) / (EVAL_THREADS / 32);
         if (splits > max_splits) splits = max_splits;
-        k_eval<<<dim3(1, splits), EVAL_THREADS, smem, c->stream>>>((const unsigned short *)(buf + off_cells), c->d_t, c->d_q,
+        k_eval<true><<<dim3(1, splits), EVAL_THREADS, smem, c->stream>>>((const unsigned short *)(buf + off_cells), c->d_t, c->d_q,
                                                                   c->d_edp, c->d_dp_list, c->d_dp_off, dm, c->bl,
                                                                   (int *)(buf + off_W), buf + off_blob, nullptr, nullptr,
                                                                   (i64 *)(buf + off_es), (int *)(buf + off_tk));
@@ -439,12 +466,12 @@ extern "C" int rp_eval_layouts_noalloc(rp_ctx *c, const int32_t *layouts, int32_
     const size_t smem = eval_smem_bytes(dm);
     if (smem > 220 * 1024) return RP_ERR_RANGE;
     if (smem > 32 * 1024)
-        RP_CUDA(cudaFuncSetAttribute(k_eval, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        RP_CUDA(cudaFuncSetAttribute(k_eval<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int splits = (2 * 148 + n - 1) / n;
     const int max_splits = (dm.RG + EVAL_THREADS / 32 - 1) / (EVAL_THREADS / 32);
     if (splits > max_splits) splits = max_splits;
     if (splits < 1) splits = 1;
-    k_eval<<<dim3(n, splits), EVAL_THREADS, smem, c->stream>>>(sc->cells, c->d_t, c->d_q, c->d_edp, c->d_dp_list, c->d_dp_off,
+    k_eval<false><<<dim3(n, splits), EVAL_THREADS, smem, c->stream>>>(sc->cells, c->d_t, c->d_q, c->d_edp, c->d_dp_list, c->d_dp_off,
                                                               dm, c->bl, nullptr, nullptr, (i64 *)score_fx, score_f64, sc->esum,
                                                               sc->tickets);
     ++g_rp_launches;
