@@ -428,6 +428,31 @@ def test_fuzz_random_small_windows():
         rp.rp_destroy(ctx)
 
 
+def test_repeated_front_end_calls_recompute():
+    """rp_window_load already queues placement and packing; a second rp_place_experts or
+    rp_pack_rows computes them again itself, and rp_best without a preceding rp_anneal validates
+    on its own: same results on every route."""
+    w = make_window(custom_spec("twice", 96, 5, 16, 2, 4096, 4, 4, 12, 400, data_seed=31))
+    edp = [0, 0, 1, 1]
+    ref = oracle_front(w, edp, 3)
+    ctx = load(w, pop=12, edp=edp, min_rows=3)
+    pi1, load1 = rp.rp_place_experts(ctx)
+    pi2, load2 = rp.rp_place_experts(ctx)
+    assert (pi1 == pi2).all() and (load1 == load2).all() and (pi1 == ref["pi"]).all()
+    r1 = rp.rp_pack_rows(ctx)
+    lay1, fx1, _ = rp.rp_best(ctx)                  # no rp_anneal yet: the seed, validated here
+    r2 = rp.rp_pack_rows(ctx)
+    lay2, fx2, _ = rp.rp_best(ctx)
+    assert r1 == r2 and r1[0] == ref["R"]
+    assert (lay1 == lay2).all() and (lay1 == ref["seed"]).all() and tuple(fx1) == tuple(fx2)
+    check_eval(w, ctx, ref, edp)
+    check_anneal(w, ctx, ref, edp, 12, 3, 40, t_ratio=0.5)
+    lay3, fx3, _ = rp.rp_best(ctx)                  # handed over by rp_anneal
+    lay4, fx4, _ = rp.rp_best(ctx)
+    assert (lay3 == lay4).all() and tuple(fx3) == tuple(fx4)
+    rp.rp_destroy(ctx)
+
+
 def test_fuzz_seeding_stages():
     """Random shapes (one to six DP slots, one to all shards, 1..48 ranks, populations of 1..33,
     choice widths 1..32, one to nine projections, zero to large eta): trial loop, pairing and
