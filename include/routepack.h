@@ -96,8 +96,9 @@ typedef struct {
  *   cuda_stream: a cudaStream_t (NULL = default stream).
  * The placement, projection and packing kernels depend on nothing but these inputs and are queued
  * on the stream right behind the checks, so the GPU is already working on them while the host
- * waits for the verdict; rp_place_experts and rp_pack_rows then hand their results over (and
- * compute them themselves when called again).
+ * waits for the verdict (packing, which reads only the lengths, on an internal side stream that
+ * forks from and joins the context's stream inside this call); rp_place_experts and
+ * rp_pack_rows then hand their results over (and compute them themselves when called again).
  * On failure *out is NULL. */
 int rp_window_load(rp_ctx **out, const rp_config *cfg, const int32_t *lengths,
                    const int32_t *demand, void *cuda_stream);

@@ -88,6 +88,39 @@ static void pin_give(void *p)
     g_pin_free.push_back(p);
 }
 
+// A side stream with two events, recycled across contexts of a device like the pinned blocks:
+// packing needs only the lengths, so it runs beside the check / placement / projection kernels.
+struct RpSide { int device; cudaStream_t stream; cudaEvent_t fork, join; };
+static std::vector<RpSide *> g_side_free;
+static RpSide *side_take(int device)
+{
+    {
+        std::lock_guard<std::mutex> lk(g_pin_mutex);
+        for (size_t x = 0; x < g_side_free.size(); ++x)
+            if (g_side_free[x]->device == device) {
+                RpSide *s = g_side_free[x];
+                g_side_free.erase(g_side_free.begin() + x);
+                return s;
+            }
+    }
+    RpSide *s = new RpSide;
+    s->device = device;
+    if (cudaStreamCreateWithFlags(&s->stream, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&s->fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&s->join, cudaEventDisableTiming) != cudaSuccess) {
+        cudaGetLastError();
+        delete s;
+        return nullptr;
+    }
+    return s;
+}
+static void side_give(RpSide *s)
+{
+    if (!s) return;
+    std::lock_guard<std::mutex> lk(g_pin_mutex);
+    g_side_free.push_back(s);
+}
+
 
 static bool is_device_ptr(const void *p)
 {
@@ -143,6 +176,7 @@ extern "C" void rp_destroy(rp_ctx *c)
     free_population(c); free_trace(c); free_eval(c);
     dev_free(c, c->own_t); dev_free(c, c->own_a); dev_free(c, c->d_load_slab); dev_free(c, c->d_static);
     pin_give(c->h_pin);
+    side_give((RpSide *)c->side);
     free(c->h_levels);
     free(c);
 }
@@ -268,8 +302,19 @@ static int window_load_impl(rp_ctx *c, const rp_config *cfg, const int32_t *leng
     // Placement, projection and packing depend on nothing but the inputs: they are queued right
     // behind the checks, so that the GPU works on them while the host waits for the verdict
     // (rp_place_experts and rp_pack_rows then only hand the results over).
+    // Packing reads only the lengths: it goes to a side stream that forks here and joins before the
+    // row count is read back.
+    RpSide *side = (RpSide *)c->side;
+    bool forked = false;
+    if (side && cudaEventRecord(side->fork, c->stream) == cudaSuccess &&
+        cudaStreamWaitEvent(side->stream, side->fork, 0) == cudaSuccess) {
+        c->eager_pack = (rp_launch_pack_on(c, side->stream) == RP_OK);
+        forked = (cudaEventRecord(side->join, side->stream) == cudaSuccess);
+        if (!forked) { cudaStreamSynchronize(side->stream); c->eager_pack = 0; }
+    }
     c->eager_place = (rp_launch_lpt(c) == RP_OK && rp_launch_project(c) == RP_OK);
-    c->eager_pack = (rp_launch_pack(c, 0) == RP_OK);
+    if (forked) RP_CUDA(cudaStreamWaitEvent(c->stream, side->join, 0));
+    else c->eager_pack = (rp_launch_pack(c, 0) == RP_OK);
     if (c->eager_pack)
         RP_CUDA(cudaMemcpyAsync(c->h_pin + 10, c->d_pack_out, sizeof(int) * 4, cudaMemcpyDeviceToHost, c->stream));
 
@@ -313,6 +358,7 @@ extern "C" int rp_window_load(rp_ctx **out, const rp_config *cfg, const int32_t 
     c->Ppop = cfg->pop_size;
     c->h_pin = (i64 *)pin_take();
     if (!c->h_pin) { free(c); return RP_ERR_CUDA; }
+    c->side = side_take(c->device);          // optional: without it everything runs on the one stream
     int st = window_load_impl(c, cfg, lengths, demand);
     if (st != RP_OK) { rp_destroy(c); return st; }
     c->stage = 1;

@@ -145,6 +145,7 @@ struct rp_ctx {
     i64 *d_inc_score;          // [3]
     i64 *d_best_score;         // [3] full rescoring of the incumbent (validation)
     double *d_best_f64;        // [3] the same as the real-valued objective
+    void *side;                // side stream + two events borrowed for the call that packs beside the placement (see RpSide)
     int eager_place, eager_pack;   // rp_window_load already queued the placement / packing kernels behind its checks
     int pack_out[4];           // R*, certified, R_lb, failure flag as read back with the load's verdict
     int best_ready;            // the incumbent has been validated and rescored since it last changed
@@ -184,6 +185,7 @@ int rp_launch_eval(rp_ctx *c, const unsigned short *cells, int n, int *W_out, ch
 int rp_launch_build_static(rp_ctx *c);
 int rp_launch_seed_trials(rp_ctx *c, int width, int *layouts, int *ok);
 int rp_launch_edp_pair(rp_ctx *c, const int *lay_in, int *lay_out, int *prof, int first, int count, int width);
+int rp_launch_pack_on(rp_ctx *c, cudaStream_t stream);
 int rp_launch_pick_best(rp_ctx *c, const i64 *scores, const int *layouts, int n, i64 *best_score_out);
 int rp_get_pool(int device, cudaMemPool_t *out);     // the library's stream-ordered pool of a device
 void rp_make_layouts(const RpDims &dm, RpBlob *bl, RpStatic *sl);

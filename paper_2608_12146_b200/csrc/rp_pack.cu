@@ -191,7 +191,9 @@ k_pack_ffd(RpDims dm, const int *__restrict__ t, int min_rows, u64 *__restrict__
     }
 }
 
-int rp_launch_pack(rp_ctx *c, int /*unused*/)
+int rp_launch_pack(rp_ctx *c, int /*unused*/) { return rp_launch_pack_on(c, c->stream); }
+
+int rp_launch_pack_on(rp_ctx *c, cudaStream_t stream)
 {
     const RpDims &dm = c->dm;
     int n_pow2 = 1;
@@ -205,7 +207,7 @@ int rp_launch_pack(rp_ctx *c, int /*unused*/)
         RP_CUDA(cudaFuncSetAttribute(k_pack_ffd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     // small windows: fewer warps make the block-wide barriers of the sort cheaper
     const int threads = n_pow2 >= PACK_THREADS ? PACK_THREADS : (n_pow2 < 256 ? 256 : n_pow2);
-    k_pack_ffd<<<1, threads, smem, c->stream>>>(dm, c->d_t, c->cfg.min_rows, keys_g, n_pow2, fill_g,
+    k_pack_ffd<<<1, threads, smem, stream>>>(dm, c->d_t, c->cfg.min_rows, keys_g, n_pow2, fill_g,
                                                     c->d_seed_layout, c->d_pack_out, c->d_order);
     ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
