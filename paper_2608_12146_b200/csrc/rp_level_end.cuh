@@ -60,7 +60,7 @@ __device__ __forceinline__ void le_weights(const i64 (&e)[U], i64 emin, u64 M, u
 // Inclusive prefix sums F[j] of the weights, U consecutive members per thread and round.
 template <int U>
 __device__ __forceinline__ void le_prefix_weights(const AnnealArgs &A, int tid, int nt, i64 emin, u64 M, u64 *F,
-                                                  u64 *rsum, u64 *carry_s)
+                                                  u64 *rsum, u64 *carry_s, bool have_e = false, i64 e_mine = 0)
 {
     const int lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
     const int P = A.Ppop;
@@ -71,8 +71,9 @@ __device__ __forceinline__ void le_prefix_weights(const AnnealArgs &A, int tid, 
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int j = j0 + u;
-            e[u] = (j < P) ? rp_energy(LE_LD(A.term[3 * (size_t)j]), LE_LD(A.term[3 * (size_t)j + 1]), LE_LD(A.term[3 * (size_t)j + 2]))
-                           : emin;
+            if (U == 1 && have_e) e[u] = (j < P) ? e_mine : emin;       // member tid's energy is still in a register
+            else e[u] = (j < P) ? rp_energy(LE_LD(A.term[3 * (size_t)j]), LE_LD(A.term[3 * (size_t)j + 1]), LE_LD(A.term[3 * (size_t)j + 2]))
+                                : emin;
         }
         le_weights<U>(e, emin, M, A.cq, w);
         u64 v = 0;
@@ -152,6 +153,8 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
     i64 b0 = i0, b1 = i1, b2 = i2;
     int bj = 0x7fffffff, bn = 0, ba = 0;
     i64 emin = 0x7fffffffffffffffll;         // smallest terminal energy, for the weights further down
+    i64 e_first = 0;                         // energy of member tid (all there is to weigh when P <= nt)
+    const int now0 = A.w_on_chip ? A.wloc_dst[0] : 0;      // which half of the cells this level worked in (needed at the end)
 #pragma unroll 2
     for (int j = tid; j < P; j += nt) {
         const i64 s0 = LE_LD(A.best[3 * (size_t)j]), s1 = LE_LD(A.best[3 * (size_t)j + 1]), s2 = LE_LD(A.best[3 * (size_t)j + 2]);
@@ -161,6 +164,7 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
             if (!O.cand_layout) { bn = LE_LD(A.best_nlog[j]); ba = A.anc[j]; }     // what the replay needs, fetched with the rest
         }
         const i64 e = rp_energy(t0, t1, t2);
+        if (j == tid) e_first = e;
         emin = e < emin ? e : emin;
     }
     {   // warp minimum of the (non-negative) energies: smallest high word, then smallest low word among its holders
@@ -264,7 +268,7 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
     if (tid == 0) carry_s = 0;
     __syncthreads();
     const u64 M = (u64)(emin > A.dm.SC ? emin : A.dm.SC);
-    if (P <= nt) le_prefix_weights<1>(A, tid, nt, emin, M, F, rsum, &carry_s);
+    if (P <= nt) le_prefix_weights<1>(A, tid, nt, emin, M, F, rsum, &carry_s, true, e_first);
     else if (P <= 2 * nt) le_prefix_weights<2>(A, tid, nt, emin, M, F, rsum, &carry_s);
     else le_prefix_weights<4>(A, tid, nt, emin, M, F, rsum, &carry_s);
     const u64 Ftot = F[P - 1];
@@ -325,7 +329,8 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
     int *freelist = isfree + 2 * P;        // [2P]  k-th free cell
     const int *now = A.wloc_dst;           // cells the terminal states of this level sit in
     if (A.w_on_chip) {      // W goes through shared memory every level anyway: alternate between the two halves
-        for (int m = tid; m < P; m += nt) O.wloc_out[m] = (now[m] >= P) ? m : P + m;
+        // every member sits in the same half (its own cell m or P + m)
+        for (int m = tid; m < P; m += nt) O.wloc_out[m] = (now0 >= P) ? m : P + m;
         return;
     }
     for (int a = tid; a < P; a += nt) kids[a] = 0;
