@@ -361,6 +361,31 @@ def eval_stage(rp, torch, name, dev, reps=10):
             "algorithmic_gbs": byts / ms / 1e6}
 
 
+def mechanism_diagnostics(rp, torch, name, dev):
+    """Context figure: the paper's mechanism diagnostics (global EP-rank CV before / after placement;
+    EP peak sum, tail peak, EP balance efficiency, attention proxy and joint cost of the length-only
+    seed against the annealed plan) on the named synthetic window."""
+    w = make_window(SPECS[name])
+    s = w.spec
+    t_dev = torch.from_numpy(w.lengths).to(dev)
+    a_dev = torch.from_numpy(w.demand).to(dev)
+    ctx = rp.rp_window_load(t_dev, a_dev, top_k=s.top_k, token_cap=s.token_cap, dp_width=s.dp_width,
+                            ep_width=s.ep_width, pop_size=s.pop_size, alpha=s.alpha, beta=s.beta, seed=s.anneal_seed)
+    rp.rp_place_experts(ctx)
+    rp.rp_pack_rows(ctx)
+    seed = rp.rp_diagnostics(ctx)
+    rp.rp_anneal(ctx, n_levels=s.n_levels, steps_per_level=s.steps_per_level, t0=s.t0, t_ratio=s.t_ratio,
+                 p_reloc=s.p_reloc, p_guide=s.p_guide, want_stats=False)
+    rp.rp_best(ctx)
+    best = rp.rp_diagnostics(ctx)
+    rp.rp_destroy(ctx)
+    rel = lambda k: (best[k] - seed[k]) / seed[k] if seed[k] else 0.0
+    return {"workload": name, "cv_identity": seed["cv_identity"], "cv_placed": seed["cv_placed"],
+            "seed": {k: seed[k] for k in ("s_ep", "t_ep", "eta_ep", "attention", "joint")},
+            "annealed": {k: best[k] for k in ("s_ep", "t_ep", "eta_ep", "attention", "joint")},
+            "change": {"s_ep": rel("s_ep"), "t_ep": rel("t_ep"), "attention": rel("attention"), "joint": rel("joint")}}
+
+
 def run_cuda(args):
     import torch
     import paper_2608_12146_b200.binding as rp
@@ -401,6 +426,7 @@ def run_cuda(args):
         if args.sweep and world == 1 and not args.pop and not args.levels:
             line["seeding_stages"] = seeding_stages(rp, torch, args.workload, dev)
             line["eval_population"] = [eval_stage(rp, torch, n, dev) for n in ("medium", "large", "wide")]
+            line["mechanism_diagnostics"] = [mechanism_diagnostics(rp, torch, n, dev) for n in ("medium", "large")]
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
