@@ -110,8 +110,8 @@ int rp_window_load(rp_ctx **out, const rp_config *cfg, const int32_t *lengths,
  * computes q[i][l][p].
  *   pi [L][E] int32 out, nullable: physical slot of logical expert e.
  *   rank_load [L][P] int64 out, nullable: aggregate load G[l][p] under pi.
- * Host outputs are complete on return; outputs in device memory (and the call itself when both
- * are NULL) are only ordered on the context's stream. */
+ * Outputs (host or device memory) are complete on return; with both NULL the call only queues
+ * its work on the context's stream. */
 int rp_place_experts(rp_ctx *ctx, int32_t *pi, int64_t *rank_load);
 
 /* Row count and seed population (Section 3.2; Algorithm 2, first line and last loop).
@@ -216,9 +216,8 @@ int rp_anneal(rp_ctx *ctx, const rp_anneal_params *params, rp_anneal_stats *stat
 /* Validate the incumbent (coverage, capacity, non-empty cells, cached score equals a full
  * rescoring, not worse than the seed) and return it.
  *   cell_of_sample [N] int32 out, nullable; score_fx [3], score_f64 [3] out, nullable.
- * RP_ERR_INVALID_PLAN when a check fails.  Host outputs are complete on return; outputs in
- * device memory are ordered on the context's stream.  Right after rp_anneal the checks are
- * already done and the call only hands the results over. */
+ * RP_ERR_INVALID_PLAN when a check fails.  Outputs are complete on return.  Right after
+ * rp_anneal the checks are already done and the call only hands the results over. */
 int rp_best(rp_ctx *ctx, int32_t *cell_of_sample, int64_t *score_fx, double *score_f64);
 
 /* Load-balance diagnostics of the paper's evaluation section for one layout (Eq. global-ep-cv,

@@ -378,9 +378,8 @@ extern "C" int rp_place_experts(rp_ctx *c, int32_t *pi, int64_t *rank_load)
     c->eager_place = 0;               // a repeated call recomputes
     RP_TRY(copy_out(c, pi, c->d_pi, sizeof(int) * (size_t)dm.L * dm.E));
     RP_TRY(copy_out(c, rank_load, c->d_rank_load, sizeof(i64) * (size_t)dm.L * dm.P));
-    // Host outputs are complete when the call returns; device outputs are ordered on the stream.
-    if ((pi && !is_device_ptr(pi)) || (rank_load && !is_device_ptr(rank_load)))
-        RP_CUDA(cudaStreamSynchronize(c->stream));
+    // Outputs are complete when the call returns (nothing to wait for when none was asked for).
+    if (pi || rank_load) RP_CUDA(cudaStreamSynchronize(c->stream));
     if (c->stage < 2) c->stage = 2;
     return RP_OK;
 }
@@ -856,9 +855,8 @@ extern "C" int rp_best(rp_ctx *c, int32_t *cell_of_sample, int64_t *score_fx, do
     RP_TRY(copy_out(c, cell_of_sample, c->d_inc_layout, sizeof(int) * (size_t)dm.N));
     RP_TRY(copy_out(c, score_fx, c->d_inc_score, sizeof(i64) * 3));
     RP_TRY(copy_out(c, score_f64, c->d_best_f64, sizeof(double) * 3));
-    const bool host_out = (cell_of_sample && !is_device_ptr(cell_of_sample)) || (score_fx && !is_device_ptr(score_fx)) ||
-                          (score_f64 && !is_device_ptr(score_f64));
-    if (fresh || host_out) RP_CUDA(cudaStreamSynchronize(c->stream));
+    // Outputs are complete when the call returns.
+    if (fresh || cell_of_sample || score_fx || score_f64) RP_CUDA(cudaStreamSynchronize(c->stream));
     if (fresh) { c->best_verdict = best_verdict(c, sw); c->best_ready = 1; }
     return c->best_verdict;
 }
