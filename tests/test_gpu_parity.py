@@ -4,6 +4,8 @@ Integers, indices, placements, layouts and the whole annealing trajectory must b
 the reported fp64 objective must agree with the oracle's real-valued evaluation to 1e-9
 relative (the tolerance the benchmark spec states).
 """
+import os
+
 import numpy as np
 import pytest
 
@@ -140,6 +142,34 @@ def test_device_integer_functions_bit_exact():
                         np.array([0, 1, 255, 256, 2 ** 32 - 1, 2 ** 32, 32 << 32, (32 << 32) - 1, 2 ** 40, 2 ** 63], np.uint64)])
     got = rp.rp_debug_exp2neg(z)
     assert got.tolist() == [oracle.exp2neg(int(v)) for v in z]
+
+
+def test_philox_against_the_curand_header(tmp_path):
+    """A third implementation: cuRAND's device function, compiled here with nvcc (skipped when the
+    toolkit is not on the machine), against the library's and the oracle's words."""
+    import ctypes
+    import shutil
+    import subprocess
+    nvcc = shutil.which("nvcc") or "/usr/local/cuda/bin/nvcc"
+    if not os.path.exists(nvcc):
+        pytest.skip("nvcc not available")
+    src = os.path.join(os.path.dirname(os.path.abspath(__file__)), "aux", "philox_curand.cu")
+    so = str(tmp_path / "philox_curand.so")
+    res = subprocess.run([nvcc, "-O2", "-gencode", "arch=compute_100a,code=sm_100a", "-Xcompiler", "-fPIC", "-shared",
+                          "-o", so, src], capture_output=True, text=True)
+    assert res.returncode == 0, res.stderr
+    lib = ctypes.CDLL(so)
+    rng = np.random.default_rng(12)
+    ctr = rng.integers(0, 2 ** 32, (512, 4), dtype=np.uint64).astype(np.uint32)
+    ctr[0] = 0
+    ctr[1] = 0xFFFFFFFF
+    key = np.array([0x243F6A88, 0x85A308D3], np.uint32)
+    out = np.zeros_like(ctr)
+    assert lib.curand_philox_host(ctr.ctypes.data_as(ctypes.c_void_p), ctypes.c_uint32(int(key[0])), ctypes.c_uint32(int(key[1])),
+                                  out.ctypes.data_as(ctypes.c_void_p), ctypes.c_int(len(ctr))) == 0
+    assert (rp.rp_debug_philox(ctr, key) == out).all()
+    for i in range(32):
+        assert (out[i] == oracle.philox4x32_10(ctr[i], key)).all()
 
 
 @pytest.mark.parametrize("name", ["tiny", "medium"])
