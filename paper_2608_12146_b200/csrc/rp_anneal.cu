@@ -80,13 +80,15 @@ k_anneal_level(const AnnealArgs A)
     const int j = blockIdx.x;
     const int src = A.anc[j];
     const bool identity_edp = (dm.G == dm.D);
-    int *Wj = A.W + (size_t)A.wloc_dst[j] * wn;
+    const int dst_cell = A.wloc_dst[j];
+    const int src_cell = rp_src_cell(A, src, j);
+    int *Wj = A.W + (size_t)dst_cell * wn;
     const bool vec = (dm.P >= 4) && (dm.P <= 128) && ((dm.P & (dm.P - 1)) == 0);
     const i64 aC = dm.asum * dm.C, bS = dm.bsum;
 
     if (tid == 0) chain->failed = 0;
-    const bool landed = rp_chain_load<NT, false>(A, src, j, sm_blob, sm_static, nullptr, mbar, tid);
-    if (tid == 0 && A.wloc_src[src] != A.wloc_dst[j])      // bytes of the W gather (counted here: off the level's tail)
+    const bool landed = rp_chain_load<NT, false>(A, src, j, sm_blob, sm_static, nullptr, mbar, tid, src_cell, dst_cell);
+    if (tid == 0 && src_cell != dst_cell)                  // bytes of the W gather (counted here: off the level's tail)
         atomicAdd((u64 *)&A.counters[5], (u64)2 * dm.RG * dm.LP * 4);
     if (!landed) chain->failed = 1;
     __syncthreads();

@@ -250,13 +250,21 @@ __device__ __forceinline__ void rp_fence_async_smem()
 // Shared-memory front of both chain kernels: [blob][static tables][W when it lives on chip].
 // The blob of the ancestor, the static block and (on chip) the ancestor's W arrive by bulk
 // copies on one mbarrier; W kept in global memory is copied by all threads.
+// Cell that holds the rank loads of ancestor `src` when this level starts.  With W on chip every
+// member works in its own cell m or P + m and all members sit in the same half, so the half of
+// this slot's own entry tells where the ancestor's is: no load that depends on `src`.
+__device__ __forceinline__ int rp_src_cell(const AnnealArgs &A, int src, int j)
+{
+    if (A.w_on_chip) return (A.wloc_src[j] >= A.Ppop) ? A.Ppop + src : src;
+    return A.wloc_src[src];
+}
+
 template <int NT, bool WS>
 __device__ __forceinline__ bool rp_chain_load(const AnnealArgs &A, int src, int j, char *sm_blob, char *sm_static,
-                                              int *Wsm, u64 *mbar, int tid)
+                                              int *Wsm, u64 *mbar, int tid, int src_cell, int dst_cell)
 {
     const RpDims &dm = A.dm;
     const size_t wn = (size_t)dm.RG * dm.LP;
-    const int src_cell = A.wloc_src[src], dst_cell = A.wloc_dst[j];
     const int *ws = A.W + (size_t)src_cell * wn;
     const bool w_bulk = WS && ((wn & 3) == 0);
     if (tid == 0) {

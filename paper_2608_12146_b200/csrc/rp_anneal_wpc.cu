@@ -138,12 +138,14 @@ k_anneal_wpc(const AnnealArgs A)
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const int src = A.anc[j];
-    int *Wj = WS ? Wsm : A.W + (size_t)A.wloc_dst[j] * wn;     // the previous level's barrier wrote wloc_dst
+    const int dst_cell = A.wloc_dst[j];                          // the previous level's barrier wrote it
+    const int src_cell = rp_src_cell(A, src, j);
+    int *Wj = WS ? Wsm : A.W + (size_t)dst_cell * wn;
 
     // ---- prologue: adopt the ancestor's terminal state -------------------------------
     if (tid == 0) chain->failed = 0;
-    const bool landed = rp_chain_load<NT, WS>(A, src, j, sm_blob, sm_static, Wsm, mbar, tid);
-    if (tid == 0 && A.wloc_src[src] != A.wloc_dst[j])      // bytes of the W gather (counted here: off the level's tail)
+    const bool landed = rp_chain_load<NT, WS>(A, src, j, sm_blob, sm_static, Wsm, mbar, tid, src_cell, dst_cell);
+    if (tid == 0 && src_cell != dst_cell)                  // bytes of the W gather (counted here: off the level's tail)
         atomicAdd((u64 *)&A.counters[5], (u64)2 * dm.RG * dm.LP * 4);
     if (!landed) chain->failed = 1;
     __syncthreads();
