@@ -141,6 +141,9 @@ k_anneal_wpc(const AnnealArgs A)
     const int dst_cell = A.wloc_dst[j];                          // the previous level's barrier wrote it
     const int src_cell = rp_src_cell(A, src, j);
     int *Wj = WS ? Wsm : A.W + (size_t)dst_cell * wn;
+    // the incumbent's score when the level starts (fetched now, beside the loads above; used below)
+    i64 inc0 = 0, inc1 = 0, inc2 = 0;
+    if (tid == 0) { inc0 = A.lo.inc_score[0]; inc1 = A.lo.inc_score[1]; inc2 = A.lo.inc_score[2]; }
 
     // ---- prologue: adopt the ancestor's terminal state -------------------------------
     if (tid == 0) chain->failed = 0;
@@ -161,7 +164,7 @@ k_anneal_wpc(const AnnealArgs A)
     if (tid == 0) {
         chain->B[0] = Sc[0]; chain->B[1] = Sc[1]; chain->B[2] = Sc[2];
         chain->dig = 0; chain->best_step = 0; chain->best_nlog = 0; chain->nlog = 0;
-        chain->I[0] = A.lo.inc_score[0]; chain->I[1] = A.lo.inc_score[1]; chain->I[2] = A.lo.inc_score[2];
+        chain->I[0] = inc0; chain->I[1] = inc1; chain->I[2] = inc2;
         chain->has_snap = 0;
     }
     __syncthreads();
