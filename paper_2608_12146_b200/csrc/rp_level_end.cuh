@@ -273,6 +273,11 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
     else le_prefix_weights<4>(A, tid, nt, emin, M, F, rsum, &carry_s);
     const u64 Ftot = F[P - 1];
     const u64 u0 = (u64)(((unsigned __int128)A.resample_x * Ftot) >> 32);
+    // The cell bookkeeping further down works in shared memory when 8*P ints fit: ancestors and
+    // current cells are staged beyond the cumulative weights while those are still in use.
+    const bool cells_on_chip = !A.w_on_chip && (size_t)P * 8 * sizeof(int) <= ws_bytes && F_on_chip;
+    int *anc_s = (int *)ws + 6 * (size_t)P, *now_s = anc_s + P;
+    if (cells_on_chip) for (int m = tid; m < P; m += nt) now_s[m] = A.wloc_dst[m];
     int depth = 0;
     while ((1 << depth) < P) ++depth;
     constexpr int SU = 4;                       // searches per thread in flight
@@ -314,6 +319,7 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
             const int m = base + u * nt + tid;
             if (m < P) {
                 O.anc_out[m] = lo[u];
+                if (cells_on_chip) anc_s[m] = lo[u];
                 if (O.tr_anc) O.tr_anc[(size_t)A.level * P + m] = lo[u];
             }
         }
@@ -323,55 +329,56 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
     // ---- W cells of the next level.  A member that is its ancestor's only child works on in the
     // ancestor's cell; children of an ancestor with several children each get a free cell and
     // copy.  Cells: 2*P of them; the ones no surviving ancestor holds are free.
-    int *kids = O.scratch;                 // [P]   children per ancestor
-    int *need = kids + P;                  // [P]   1 = this member needs a fresh cell -> exclusive ranks
-    int *isfree = need + P;                // [2P]  1 = free cell -> exclusive ranks
-    int *freelist = isfree + 2 * P;        // [2P]  k-th free cell
     const int *now = A.wloc_dst;           // cells the terminal states of this level sit in
     if (A.w_on_chip) {      // W goes through shared memory every level anyway: alternate between the two halves
         // every member sits in the same half (its own cell m or P + m)
         for (int m = tid; m < P; m += nt) O.wloc_out[m] = (now0 >= P) ? m : P + m;
         return;
     }
+    int *kids = cells_on_chip ? (int *)ws : O.scratch;     // [P]   children per ancestor
+    int *need = kids + P;                  // [P]   1 = this member needs a fresh cell -> exclusive ranks
+    int *isfree = need + P;                // [2P]  1 = free cell -> exclusive ranks
+    int *freelist = isfree + 2 * P;        // [2P]  k-th free cell
+    const int *anc_r = cells_on_chip ? anc_s : O.anc_out;
+    const int *now_r = cells_on_chip ? now_s : now;
     for (int a = tid; a < P; a += nt) kids[a] = 0;
     for (int c2 = tid; c2 < 2 * P; c2 += nt) isfree[c2] = 1;
     __syncthreads();
-    for (int m = tid; m < P; m += nt) atomicAdd(&kids[O.anc_out[m]], 1);
+    for (int m = tid; m < P; m += nt) atomicAdd(&kids[anc_r[m]], 1);
     __syncthreads();
-    for (int a = tid; a < P; a += nt) if (kids[a] >= 1) isfree[now[a]] = 0;
-    for (int m = tid; m < P; m += nt) need[m] = (kids[O.anc_out[m]] != 1);
+    for (int a = tid; a < P; a += nt) if (kids[a] >= 1) isfree[now_r[a]] = 0;
+    for (int m = tid; m < P; m += nt) need[m] = (kids[anc_r[m]] != 1);
     __syncthreads();
-    for (int pass = 0; pass < 2; ++pass) {          // exclusive prefix sums of need[P] and isfree[2P], in place
+    // exclusive prefix sums of need[P] and isfree[2P]: a thread scans its own consecutive chunk, one
+    // block-wide scan of the chunk totals joins them
+    for (int pass = 0; pass < 2; ++pass) {
         int *arr = pass ? isfree : need;
         const int n = pass ? 2 * P : P;
-        if (tid == 0) carry_s = 0;
+        const int chunk = (n + nt - 1) / nt;
+        const int x0 = min(n, tid * chunk), x1 = min(n, x0 + chunk);
+        int total = 0;
+        for (int x = x0; x < x1; ++x) total += arr[x];
+        int v = total;
+        for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += y; }
+        if (lane == 31) rj[warp] = v;
         __syncthreads();
-        for (int base = 0; base < n; base += nt) {
-            const int x = base + tid;
-            const int flag = (x < n) ? arr[x] : 0;
-            int v = flag;
-            for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += y; }
-            if (lane == 31) rj[warp] = v;
-            __syncthreads();
-            if (warp == 0) {
-                int s2 = (lane < nwarps) ? rj[lane] : 0;
-                for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, s2, o); if (lane >= o) s2 += y; }
-                rj[lane] = s2;
-            }
-            __syncthreads();
-            const int before = (int)carry_s + (warp ? rj[warp - 1] : 0);
-            if (x < n) {
-                const int rank = before + v - flag;          // exclusive
-                if (pass) { if (flag) freelist[rank] = x; }
-                else arr[x] = flag ? rank : -1;
-            }
-            __syncthreads();
-            if (tid == nt - 1) carry_s = (u64)(before + v);
-            __syncthreads();
+        if (warp == 0) {
+            int s2 = (lane < nwarps) ? rj[lane] : 0;
+            for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, s2, o); if (lane >= o) s2 += y; }
+            rj[lane] = s2;
         }
+        __syncthreads();
+        int rank = (warp ? rj[warp - 1] : 0) + v - total;          // exclusive rank of the chunk's first element
+        for (int x = x0; x < x1; ++x) {
+            const int flag = arr[x];
+            if (pass) { if (flag) freelist[rank] = x; }
+            else arr[x] = flag ? rank : -1;
+            rank += flag;
+        }
+        __syncthreads();
     }
     for (int m = tid; m < P; m += nt)
-        O.wloc_out[m] = (need[m] >= 0) ? freelist[need[m]] : now[O.anc_out[m]];
+        O.wloc_out[m] = (need[m] >= 0) ? freelist[need[m]] : now_r[anc_r[m]];
 }
 
 // Tail of a chain CTA: publish, take a ticket, and let the last arrival run the level barrier.
