@@ -10,19 +10,33 @@
 // Loads of values other CTAs wrote during this launch go to L2.
 #define LE_LD(x) __ldcg(&(x))
 
-// min(2^48 - 1, floor(Dd * 2^32 / M)) for 0 < M < 2^63.  A double-precision estimate is within
-// one of the quotient (it is below 2^48 and the estimate's relative error below 2^-50); the exact
-// 128-bit remainder then corrects it, so the result is the exact floor.
-__device__ __forceinline__ u64 le_scaled_quotient(u64 Dd, u64 M)
+// min(2^48 - 1, floor(Dd * 2^32 / M)) for 0 < M < 2^63, with rM = 2^32 / M in double precision
+// (the same M for every member of a level).  The estimate Dd * rM is within one of the quotient
+// (it is below 2^48 and the relative error of two roundings is below 2^-51); the exact 128-bit
+// remainder then corrects it, so the result is the exact floor.  No branches: members interleave.
+__device__ __forceinline__ u64 le_scaled_quotient(u64 Dd, u64 M, double rM)
 {
-    if ((Dd >> 16) >= M) return (1ull << 48) - 1;
-    u64 q = (u64)(((double)Dd * 4294967296.0) / (double)M);
+    const bool sat = (Dd >> 16) >= M;
+    u64 q = (u64)((double)Dd * rM);
     const u64 ph = __umul64hi(q, M), pl = q * M;
     const u64 nh = Dd >> 32, nl = Dd << 32;
     u64 rl = nl - pl, rh = nh - ph - (nl < pl ? 1ull : 0ull);        // remainder, signed 128-bit
-    for (int it = 0; it < 4 && (i64)rh < 0; ++it) { --q; const u64 t = rl + M; rh += (t < rl) ? 1ull : 0ull; rl = t; }
-    for (int it = 0; it < 4 && (rh != 0 || rl >= M); ++it) { ++q; rh -= (rl < M) ? 1ull : 0ull; rl -= M; }
-    return q;
+#pragma unroll
+    for (int it = 0; it < 2; ++it) {           // estimate too large: remainder negative
+        const bool neg = (i64)rh < 0;
+        const u64 t = rl + M;
+        q -= neg ? 1ull : 0ull;
+        rh += (neg && t < rl) ? 1ull : 0ull;
+        rl = neg ? t : rl;
+    }
+#pragma unroll
+    for (int it = 0; it < 2; ++it) {           // estimate too small: remainder at least M
+        const bool big = (rh != 0) || (rl >= M);
+        q += big ? 1ull : 0ull;
+        rh -= (big && rl < M) ? 1ull : 0ull;
+        rl -= big ? M : 0ull;
+    }
+    return sat ? (1ull << 48) - 1 : q;
 }
 
 // Boltzmann weights of U members at once (independent dependency chains interleave):
@@ -31,9 +45,10 @@ template <int U>
 __device__ __forceinline__ void le_weights(const i64 (&e)[U], i64 emin, u64 M, u64 cq, u64 (&w)[U])
 {
     u64 z[U], acc[U];
+    const double rM = 4294967296.0 / (double)M;
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-        const u64 eq = le_scaled_quotient((u64)(e[u] - emin), M);
+        const u64 eq = le_scaled_quotient((u64)(e[u] - emin), M, rM);
         const u64 zh = __umul64hi(eq, cq), zl = eq * cq;
         u64 zz = (zh >> 16) ? (1ull << 40) : ((zh << 48) | (zl >> 16));
         z[u] = zz > (1ull << 40) ? (1ull << 40) : zz;
