@@ -55,14 +55,22 @@ __device__ __forceinline__ void le_weights(const i64 (&e)[U], i64 emin, u64 M, u
         acc[u] = 1ull << 63;
     }
     // the fraction bits in the order of rp_exp2neg; a clear bit multiplies by one (2^63 in Q63), which is exact
-#pragma unroll 1
-    for (int i = 1; i <= 24; ++i) {
-        const u64 c = RP_EXP2_Q63[i - 1];
+    // (acc * cc) >> 63 = high word of (2*acc) * cc; acc = 2^63 (nothing applied yet) gives cc itself
+    if constexpr (U == 1) {          // one member per thread: a single dependent chain, unrolled (constants inline)
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const u64 cc = ((z[u] >> (32 - i)) & 1ull) ? c : (1ull << 63);
-            // (acc * cc) >> 63 = high word of (2*acc) * cc; acc = 2^63 (nothing applied yet) gives cc itself
-            acc[u] = (acc[u] >> 63) ? cc : __umul64hi(acc[u] << 1, cc);
+        for (int i = 1; i <= 24; ++i) {
+            const u64 cc = ((z[0] >> (32 - i)) & 1ull) ? RP_EXP2_Q63[i - 1] : (1ull << 63);
+            acc[0] = (acc[0] >> 63) ? cc : __umul64hi(acc[0] << 1, cc);
+        }
+    } else {
+#pragma unroll 1
+        for (int i = 1; i <= 24; ++i) {
+            const u64 c = RP_EXP2_Q63[i - 1];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const u64 cc = ((z[u] >> (32 - i)) & 1ull) ? c : (1ull << 63);
+                acc[u] = (acc[u] >> 63) ? cc : __umul64hi(acc[u] << 1, cc);
+            }
         }
     }
 #pragma unroll
