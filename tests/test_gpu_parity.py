@@ -458,6 +458,34 @@ def test_fuzz_random_small_windows():
         rp.rp_destroy(ctx)
 
 
+@pytest.mark.parametrize("name,pop", [("tiny", 8), ("medium", 256), ("medium", 100), ("large", 300)])
+def test_annealing_without_the_inspection_hook(name, pop):
+    """The per-level traces are an inspection hook: counters, final population, incumbent and
+    scores without them must be those of the traced run (itself checked against the oracle
+    elsewhere), over many levels, and again when rp_anneal continues from the population."""
+    w = make_window(name)
+    s = w.spec
+    outs = []
+    for trace in (True, False):
+        ctx = load(w, pop=pop)
+        rp.rp_debug_set_trace(ctx, trace)
+        rp.rp_place_experts(ctx)
+        rp.rp_pack_rows(ctx)
+        res = []
+        for levels, steps in ((12, 25), (5, 40)):
+            st = rp.rp_anneal(ctx, n_levels=levels, steps_per_level=steps, t0=s.t0, t_ratio=0.7, p_reloc=s.p_reloc, p_guide=s.p_guide)
+            layout, fx, _ = rp.rp_best(ctx)
+            res.append(([st.proposed, st.feasible, st.accepted, st.improved], layout.copy(), fx.copy(),
+                        rp.rp_debug_dump(ctx, "POPULATION", (pop, s.n_samples), np.int32),
+                        rp.rp_eval_population(ctx)[0]))
+        outs.append(res)
+        rp.rp_destroy(ctx)
+    for a, b in zip(*outs):
+        assert a[0] == b[0]
+        for x, y in zip(a[1:], b[1:]):
+            assert (x == y).all()
+
+
 def test_repeated_front_end_calls_recompute():
     """rp_window_load already queues placement and packing; a second rp_place_experts or
     rp_pack_rows computes them again itself, and rp_best without a preceding rp_anneal validates
