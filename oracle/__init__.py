@@ -43,6 +43,8 @@ def lib():
         _lib.orc_coassign_q20.restype = C.c_int64
         _lib.orc_accept_uphill.restype = C.c_int32
         _lib.orc_accept_uphill.argtypes = [C.c_int64, C.c_int64, C.c_int64, C.c_uint64, C.c_uint32]
+        _lib.orc_propose_once.restype = C.c_int32
+        _lib.orc_energy.restype = C.c_int64
     return _lib
 
 
@@ -294,6 +296,34 @@ def score_scale(C_cap: int) -> int:
 
 
 # ---- annealing --------------------------------------------------------------------------
+def energy(score) -> int:
+    """Scalar search energy of a score tuple (Eq. pa-energy), in score units."""
+    s = np.ascontiguousarray(score, np.int64)
+    return int(lib().orc_energy(_p(s)))
+
+
+def propose_once(lengths, q, layout, R: int, C_cap: int, D: int, A, B, rho_q32: int, guide_q32: int,
+                 edp_of_dp=None, alpha=(1.0, 1.0), beta=(0.0, 1.0)):
+    """One GuidedProposal draw (Section 4.1.2) on `layout` from the random words A[4], B[4].
+
+    Returns (move, feasible) with move = dict(reloc, i, i2, c1, c2)."""
+    t = _i32(lengths)
+    q = _i32(q)
+    lay = _i32(layout)
+    _, L, P = q.shape
+    edp = _edp(D, edp_of_dp)
+    G = int(edp.max()) + 1
+    al, be = _f64(alpha), _f64(beta)
+    Aw = np.ascontiguousarray(A, np.uint32)
+    Bw = np.ascontiguousarray(B, np.uint32)
+    mv = np.zeros(5, np.int32)
+    ok = lib().orc_propose_once(C.c_int32(t.shape[0]), C.c_int32(L), C.c_int32(P), C.c_int32(D), C.c_int32(G),
+                                C.c_int32(R), C.c_int32(C_cap), _p(edp), C.c_int32(al.shape[0]), _p(al), _p(be),
+                                _p(t), _p(q), _p(lay), _p(Aw), _p(Bw), C.c_uint64(rho_q32), C.c_uint64(guide_q32),
+                                _p(mv))
+    return dict(reloc=int(mv[0]), i=int(mv[1]), i2=int(mv[2]), c1=int(mv[3]), c2=int(mv[4])), bool(ok)
+
+
 def anneal(lengths, q, init_layouts, R: int, C_cap: int, D: int, *, n_levels: int, steps: int,
            t0: float, t_ratio: float, p_reloc: float, p_guide: float, seed: int,
            edp_of_dp=None, alpha=(1.0, 1.0), beta=(0.0, 1.0), full_rescore: bool = False,

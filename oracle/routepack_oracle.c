@@ -25,10 +25,14 @@
  * with ahat_s = round(alpha_s * 2^8), bhat_s = round(beta_s * 2^8).  orc_eval_f64 below
  * evaluates the paper's real-valued formulas directly, to show the two agree.
  *
- * Parity status of the pieces the paper leaves open (values it never prints): the
- * guided-proposal bias, the attention coefficients, the temperature schedule, the
- * relocation probability and the FixedRowFFD details are "parity unpinned" against the
- * paper; they are fixed by the readings listed beside each function.
+ * Parity status of the pieces the paper leaves open (values it never prints): the law
+ * of the guided-proposal bias (a tournament of two here), the attention coefficients, the
+ * temperature schedule, the relocation probability and the FixedRowFFD details are
+ * "parity unpinned" against the paper; they are fixed by the readings listed beside each
+ * function.  What the paper does fix about GuidedProposal (p_guide = 0.8, sources biased
+ * to a large J, targets to a small one, the attention straggler in proportion to its
+ * contribution, the other branch uniform) and the energy coefficients of Eq. pa-energy
+ * are pinned through orc_propose_once / orc_energy at the end of this file.
  */
 #include <stdint.h>
 #include <stdlib.h>
@@ -1355,3 +1359,31 @@ void orc_select_population(int32_t N, int32_t L, int32_t P, int32_t D, int32_t G
     *n_distinct = nd;
     free(old); free(canon); free(phi); free(rep); free(sel); free(mind); free(pen);
 }
+
+/* ------------------------------------------------------------------------------------ */
+/* Thin windows onto two internal functions, so that tests can pin them one call at a    */
+/* time (they add no arithmetic: the chain loop above calls the same propose() and       */
+/* energy()).                                                                            */
+/*   orc_propose_once: GuidedProposal (Section 4.1.2) on the state of `cell_of` with the */
+/*   given random words; move = {reloc, i, i2, c1, c2}; returns feasibility (0/1).       */
+/*   orc_energy: Eq. pa-energy of a score tuple.                                         */
+/* ------------------------------------------------------------------------------------ */
+int32_t orc_propose_once(int32_t N, int32_t L, int32_t P, int32_t D, int32_t G, int32_t R, int32_t C,
+                         const int32_t *edp_of_dp, int32_t S, const double *alpha, const double *beta,
+                         const int32_t *t, const int32_t *q, const int32_t *cell_of,
+                         const uint32_t A[4], const uint32_t B[4], uint64_t rho_q32, uint64_t guide_q32,
+                         int32_t move[5])
+{
+    orc_problem pb;
+    fill_problem(&pb, N, L, P, D, G, R, C, edp_of_dp, S, alpha, beta, t, q);
+    orc_state *st = state_new(&pb);
+    memcpy(st->cell_of, cell_of, sizeof(int32_t) * N);
+    evaluate(&pb, st);
+    orc_move mv = propose(&pb, st, A, B, rho_q32, guide_q32);
+    int32_t ok = feasible(&pb, st, &mv);
+    move[0] = mv.reloc; move[1] = mv.i; move[2] = mv.i2; move[3] = mv.c1; move[4] = mv.c2;
+    state_free(st);
+    return ok;
+}
+
+int64_t orc_energy(const int64_t s[3]) { return energy(s); }

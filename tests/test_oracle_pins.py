@@ -368,15 +368,34 @@ def fits(t, K, C):
     return go(0, [0] * K, 0)
 
 
+def ffd_plain(t, K, C):
+    """First-fit-decreasing into exactly K bins (Section 3.2 reading): the K longest samples open the
+    bins, every later one goes to the lowest bin it fits in; None when some sample fits nowhere."""
+    order = sorted(range(len(t)), key=lambda i: (-t[i], i))
+    if K > len(t):
+        return None
+    fill = [t[i] for i in order[:K]]
+    if any(f > C for f in fill):
+        return None
+    for i in order[K:]:
+        b = next((b for b in range(K) if fill[b] + t[i] <= C), None)
+        if b is None:
+            return None
+        fill[b] += t[i]
+    return fill
+
+
 def test_pack_ffd_properties_and_certificate():
     rng = np.random.default_rng(8)
     for trial in range(40):
         N, D, C = int(rng.integers(4, 12)), int(rng.choice([1, 2, 3])), 100
         t = rng.integers(5, 90, N).astype(np.int32)
         R, cert, cell = oracle.pack_ffd(t, C, D)
-        if R == 0:
-            assert all(not fits(t.tolist(), r * D, C) or r * D > N for r in range(1, N // D + 1)) or True
+        if R == 0:      # no row count packs: the plain first-fit-decreasing below fails for every one of them
+            assert all(ffd_plain(t.tolist(), r * D, C) is None for r in range(1, N // D + 1))
             continue
+        assert ffd_plain(t.tolist(), R * D, C) is not None
+        assert all(ffd_plain(t.tolist(), r * D, C) is None for r in range(max(1, -(-int(t.sum()) // (C * D))), R))
         K = R * D
         fill = np.bincount(cell, weights=t, minlength=K)
         assert K <= N and (fill <= C).all() and (np.bincount(cell, minlength=K) >= 1).all()
@@ -486,6 +505,195 @@ def test_annealing_keeps_the_feasible_set_and_never_regresses():
     assert tuple(again) == tuple(res["best_score"]) == inc[-1]
     # trajectory-best is never worse than the terminal state, and best_step = 0 means "start"
     assert all(tuple(b) <= tuple(t_) for b, t_ in zip(res["best"].reshape(-1, 3), res["term"].reshape(-1, 3)))
+
+
+# ----------------------------------------------------------------------------------------
+# GuidedProposal (Section 4.1.2) and the search energy (Eq. pa-energy)
+# ----------------------------------------------------------------------------------------
+def word_for(index, n):
+    """Smallest 32-bit word x with floor(x * n / 2^32) == index."""
+    return (index * 2 ** 32 + n - 1) // n
+
+
+def proposal_fixture(edp=None, seed=7, alpha=(1.0, 1.0), beta=(0.0, 1.0)):
+    """A heterogeneous window on 3 rows x 4 slots with, per cell, the row-shard cost J, its
+    attention part A and the cell's own attention cost, all in plain Python integers."""
+    w = make_window(custom_spec("prop", 48, 3, 8, 2, 2048, 4, 4, 4, 100, data_seed=seed, alpha=alpha, beta=beta))
+    s = w.spec
+    _, _, q = placed(w)
+    R, _, lay = oracle.pack_ffd(w.lengths, s.token_cap, s.dp_width, min_rows=3)
+    D, C = s.dp_width, s.token_cap
+    shard = list(range(D)) if edp is None else list(edp)
+    t = [int(x) for x in w.lengths]
+    ah = [int(math.floor(a * 256 + 0.5)) for a in alpha]
+    bh = [int(math.floor(b * 256 + 0.5)) for b in beta]
+    K = R * D
+    T = [sum(t[i] for i in range(len(t)) if lay[i] == c) for c in range(K)]
+    Q = [sum(t[i] ** 2 for i in range(len(t)) if lay[i] == c) for c in range(K)]
+    att = [sum(ah[x] * C * T[c] + bh[x] * Q[c] for x in range(len(ah))) for c in range(K)]
+    Jc, Ac = [0] * K, [0] * K
+    for c in range(K):
+        r, g = c // D, shard[c % D]
+        cells = [r * D + d for d in range(D) if shard[d] == g]
+        A = sum(max(ah[x] * C * T[k] + bh[x] * Q[k] for k in cells) for x in range(len(ah)))
+        Wsum = np.asarray(q, dtype=object)[[i for i in range(len(t)) if lay[i] in cells]].sum(axis=0)
+        Jc[c] = A + 256 * C * sum(int(max(row)) for row in Wsum)
+        Ac[c] = A
+    return dict(w=w, q=q, R=R, lay=lay, K=K, N=len(t), J=Jc, A=Ac, att=att, edp=edp, alpha=alpha, beta=beta)
+
+
+def propose(fx, A, B, rho=0.25, guide=0.8):
+    s = fx["w"].spec
+    return oracle.propose_once(fx["w"].lengths, fx["q"], fx["lay"], fx["R"], s.token_cap, s.dp_width, A, B,
+                               int(math.floor(rho * 2 ** 32)), int(math.floor(guide * 2 ** 32)), fx["edp"],
+                               fx["alpha"], fx["beta"])[0]
+
+
+def test_guided_proposal_thresholds_and_branches():
+    """Which word decides what: relocation iff A0 < rho*2^32, guided iff A1 < p_guide*2^32 (the
+    paper's 0.8), the uniform branch reads A2, A3 only, the guided branch takes its targets from B0, B1."""
+    fx = proposal_fixture()
+    N, K, lay = fx["N"], fx["K"], fx["lay"]
+    rho_q, guide_q = int(math.floor(0.25 * 2 ** 32)), int(math.floor(0.8 * 2 ** 32))
+    a2, a3, b0, b1 = word_for(5, N), word_for(17, N), word_for(30, N), word_for(41, N)
+    # uniform swap: sample pick(A2), partner pick(A3); the B words change nothing
+    for B in ([b0, b1, 0, 0], [1, 2 ** 32 - 1, 2 ** 31, 7]):
+        mv = propose(fx, [rho_q, guide_q, a2, a3], B)
+        assert mv == dict(reloc=0, i=5, i2=17, c1=int(lay[5]), c2=int(lay[17]))
+    # one below the relocation threshold: the same words now relocate sample 5 to cell pick(A3, K)
+    mv = propose(fx, [rho_q - 1, guide_q, a2, word_for(9, K)], [b0, b1, 0, 0])
+    assert mv == dict(reloc=1, i=5, i2=-1, c1=int(lay[5]), c2=9)
+    assert propose(fx, [rho_q, guide_q, a2, word_for(9, K)], [b0, b1, 0, 0])["reloc"] == 0
+    # one below the guide threshold: sources {pick(A2), pick(A3)}, targets {pick(B0), pick(B1)}
+    mv = propose(fx, [rho_q, guide_q - 1, a2, a3], [b0, b1, 2 ** 32 - 1, 0])
+    assert mv["reloc"] == 0 and mv["i"] in (5, 17) and mv["i2"] in (30, 41)
+    mv = propose(fx, [0, guide_q - 1, a2, a3], [word_for(2, K), word_for(10, K), 2 ** 32 - 1, 0])
+    assert mv["reloc"] == 1 and mv["i"] in (5, 17) and mv["c2"] in (2, 10) and mv["i2"] == -1
+    # rho = 0 never relocates, rho = 1 (threshold 2^32) always does; the same for p_guide
+    assert propose(fx, [0, 0, a2, a3], [b0, b1, 0, 0], rho=0.0, guide=0.0) == dict(reloc=0, i=5, i2=17, c1=int(lay[5]), c2=int(lay[17]))
+    assert propose(fx, [2 ** 32 - 1, 2 ** 32 - 1, a2, a3], [b0, b1, 2 ** 32 - 1, 0], rho=1.0, guide=1.0)["reloc"] == 1
+
+
+@pytest.mark.parametrize("edp", [None, [0, 0, 1, 1]])
+def test_guided_proposal_source_takes_the_larger_cost_and_target_the_smaller(edp):
+    """Section 4.1.2: the source is biased to a row-shard with a large J, the target to a small one.
+    Tournament of two on the row-shard cost (B2 = 2^32 - 1 keeps the attention key off): the larger
+    key wins the source, the smaller the target, the first candidate on ties."""
+    fx = proposal_fixture(edp)
+    N, K, lay, J = fx["N"], fx["K"], fx["lay"], fx["J"]
+    B2 = 2 ** 32 - 1
+    assert all(B2 * J[c] >= fx["A"][c] << 32 for c in range(K))          # the coin never picks the attention key
+    seen_first, seen_second = 0, 0
+    for sa in range(0, N, 5):
+        for sb in range(1, N, 7):
+            ja, jb = J[lay[sa]], J[lay[sb]]
+            src = sb if jb > ja else sa                                     # larger wins, tie -> first
+            for ta, tb in ((3, 40), (40, 3), (11, 29), (22, 22)):
+                want_t = tb if J[lay[tb]] < J[lay[ta]] else ta              # smaller wins, tie -> first
+                mv = propose(fx, [2 ** 32 - 1, 0, word_for(sa, N), word_for(sb, N)],
+                             [word_for(ta, N), word_for(tb, N), B2, 0])
+                assert (mv["i"], mv["i2"]) == (src, want_t)
+                assert (mv["c1"], mv["c2"]) == (int(lay[src]), int(lay[want_t]))
+            for ca, cb in ((0, K - 1), (K - 1, 0), (4, 4), (2, 7)):         # relocation: target cells
+                want_c = cb if J[cb] < J[ca] else ca
+                mv = propose(fx, [0, 0, word_for(sa, N), word_for(sb, N)], [word_for(ca, K), word_for(cb, K), B2, 0])
+                assert (mv["reloc"], mv["i"], mv["c2"]) == (1, src, want_c)
+            seen_first += src == sa and ja != jb
+            seen_second += src == sb
+    assert seen_first > 5 and seen_second > 5                               # both outcomes were exercised
+    # equal keys: two samples of one cell -> the first candidate
+    same = [i for i in range(N) if lay[i] == lay[0]]
+    assert len(same) >= 2
+    mv = propose(fx, [2 ** 32 - 1, 0, word_for(same[1], N), word_for(same[0], N)], [word_for(3, N), word_for(40, N), B2, 0])
+    assert mv["i"] == same[1]
+    mv = propose(fx, [2 ** 32 - 1, 0, word_for(3, N), word_for(40, N)], [word_for(same[1], N), word_for(same[0], N), B2, 0])
+    assert mv["i2"] == same[1]
+    twins = [(a, b) for a in range(K) for b in range(K) if a != b and J[a] == J[b]]      # cells of one row-shard
+    if twins:
+        ca, cb = twins[-1]
+        assert propose(fx, [0, 0, word_for(3, N), word_for(40, N)], [word_for(ca, K), word_for(cb, K), B2, 0])["c2"] == ca
+
+
+def test_guided_proposal_attention_key_coin():
+    """Section 4.1.2: the attention straggler is chosen in proportion to its contribution: the
+    cell-attention key replaces the row-shard cost iff B2 * J < A * 2^32 for the first source
+    candidate's row-shard (both sides of the boundary word), and then decides source and target."""
+    fx = proposal_fixture()
+    N, K, lay, J, A, att = fx["N"], fx["K"], fx["lay"], fx["J"], fx["A"], fx["att"]
+    # a pair of samples on which the two keys disagree
+    pair = next(((a, b) for a in range(N) for b in range(N)
+                 if (J[lay[b]] > J[lay[a]]) != (att[lay[b]] > att[lay[a]]) and att[lay[a]] != att[lay[b]]
+                 and J[lay[a]] != J[lay[b]]), None)
+    assert pair is not None
+    sa, sb = pair
+    tpair = next(((a, b) for a in range(N) for b in range(N)
+                  if (J[lay[b]] < J[lay[a]]) != (att[lay[b]] < att[lay[a]]) and att[lay[a]] != att[lay[b]]
+                  and J[lay[a]] != J[lay[b]]), None)
+    ta, tb = tpair
+    ca = lay[sa]
+    edge = -((-A[ca] << 32) // J[ca])              # smallest word with B2 * J >= A * 2^32
+    assert 0 < edge < 2 ** 32
+    by_J = (sb if J[lay[sb]] > J[lay[sa]] else sa, tb if J[lay[tb]] < J[lay[ta]] else ta)
+    by_att = (sb if att[lay[sb]] > att[lay[sa]] else sa, tb if att[lay[tb]] < att[lay[ta]] else ta)
+    assert by_J != by_att
+    words = [2 ** 32 - 1, 0, word_for(sa, N), word_for(sb, N)]
+    mv = propose(fx, words, [word_for(ta, N), word_for(tb, N), edge - 1, 0])
+    assert (mv["i"], mv["i2"]) == by_att
+    mv = propose(fx, words, [word_for(ta, N), word_for(tb, N), edge, 0])
+    assert (mv["i"], mv["i2"]) == by_J
+    # in proportion to its contribution: over uniform B2 the attention key is used with frequency A/J
+    rng = np.random.default_rng(4)
+    n = 4000
+    hits = sum(propose(fx, words, [word_for(ta, N), word_for(tb, N), int(x), 0])["i"] == by_att[0]
+               for x in rng.integers(0, 2 ** 32, n))
+    pr = A[ca] / J[ca]
+    assert abs(hits / n - pr) < 4 * math.sqrt(pr * (1 - pr) / n) + 1e-3
+
+
+def test_guided_proposal_statistics_over_philox_draws():
+    """Section 4.1.2 over the chain's own random words (Philox, purposes 0 and 1): 80 % of the
+    proposals are guided, a quarter are relocations, sources sit in costlier row-shards than the
+    average sample, targets in cheaper ones."""
+    fx = proposal_fixture(alpha=(0.0, 0.0), beta=(0.0, 0.0))       # no attention cost: the key is always J
+    N, K, lay, J = fx["N"], fx["K"], fx["lay"], fx["J"]
+    assert len(set(J)) > 4
+    n = 20000
+    key = np.array([0x1234, 0x9], np.uint32)
+    guided = reloc = larger = differ = 0
+    src_J, dst_J = 0, 0
+    for k in range(n):
+        A = oracle.philox4x32_10([k, 3, 1, 0], key)
+        B = oracle.philox4x32_10([k, 3, 1, 1], key)
+        mv = propose(fx, A, B)
+        sa, sb = int(A[2]) * N >> 32, int(A[3]) * N >> 32
+        reloc += mv["reloc"]
+        guided += int(A[1]) < int(math.floor(0.8 * 2 ** 32))
+        if J[lay[sa]] != J[lay[sb]]:
+            differ += 1
+            larger += J[lay[mv["i"]]] == max(J[lay[sa]], J[lay[sb]])
+        src_J += J[mv["c1"]]
+        dst_J += J[mv["c2"]]
+    sig = lambda p, m: 3.5 * math.sqrt(p * (1 - p) / m)
+    assert abs(guided / n - 0.8) < sig(0.8, n)
+    assert abs(reloc / n - 0.25) < sig(0.25, n)
+    # the source holds the larger cost always when guided, half of the time otherwise: 0.8 + 0.2/2
+    assert abs(larger / differ - 0.9) < sig(0.9, differ)
+    mean_J = sum(J[lay[i]] for i in range(N)) / N
+    assert src_J / n > mean_J > dst_J / n
+
+
+def test_energy_coefficients():
+    """Eq. pa-energy: E = s0 + 1e-6 * s1 + 1e-9 * s2, floored per term in integer units."""
+    s0 = 123456789012
+    assert oracle.energy([s0, 999999, 10 ** 9 - 1]) == s0
+    assert oracle.energy([s0, 1000000, 10 ** 9 - 1]) == s0 + 1
+    assert oracle.energy([s0, 999999, 10 ** 9]) == s0 + 1
+    assert oracle.energy([s0, 7 * 10 ** 6 + 5, 3 * 10 ** 9 + 999]) == s0 + 10
+    # equal s0: a difference of 10^6 in s1 weighs exactly what 10^9 in s2 does, and 1 in s0
+    assert oracle.energy([s0, 2 * 10 ** 6, 0]) == oracle.energy([s0, 0, 2 * 10 ** 9]) == oracle.energy([s0 + 2, 0, 0])
+    # and the chain ranks by it: at zero temperature a move that raises the energy is never kept
+    big = (2 ** 40, 5 * 10 ** 15, 3 * 10 ** 12)
+    assert oracle.energy(big) == 2 ** 40 + 5 * 10 ** 9 + 3000
 
 
 def test_zero_temperature_only_descends():
