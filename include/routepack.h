@@ -40,7 +40,7 @@ typedef enum {
     RP_ERR_RANGE = -5,         /* fixed-point range or on-chip memory budget exceeded       */
     RP_ERR_CUDA = -6,          /* a CUDA call failed; see rp_last_cuda_error()              */
     RP_ERR_STATE = -7,         /* call out of order                                         */
-    RP_ERR_TIMEOUT = -8,       /* reserved: a bounded device-side wait ran out              */
+    RP_ERR_TIMEOUT = -8,       /* rp_anneal: a bounded device-side wait ran out (see there) */
     RP_ERR_INVALID_PLAN = -9   /* rp_best: the incumbent failed validation                  */
 } rp_status;
 
@@ -81,7 +81,6 @@ typedef struct {
     int64_t proposed, feasible, accepted, improved;  /* summed over chains and levels       */
     double ms_chains;           /* device time of all levels (chain kernels incl. the level
                                    barrier that runs in their last CTA, and launch gaps)    */
-    double ms_barrier;          /* always 0: kept for layout compatibility                  */
     int64_t move_bytes;         /* algorithmic bytes of the feasible moves: rank-load slices
                                    and demand rows read, slices written on accept           */
     int64_t gather_bytes;       /* rank-load bytes read+written for members that resampling
@@ -210,11 +209,17 @@ int rp_eval_layouts_noalloc(rp_ctx *ctx, const int32_t *layouts, int32_t n, int6
  * current population; level indices of the random streams restart at 0 on each call.
  * Before it returns the call also validates and fully rescores its incumbent (the checks of
  * rp_best) in the same stream, so that a following rp_best has nothing left to compute.
- *   stats: HOST out, nullable. */
+ *   stats: HOST out, nullable.
+ * Every wait of a chain on its asynchronous copies is bounded.  If one runs out, that chain stores
+ * nothing, the level's barrier and all later levels are skipped, and the call returns
+ * RP_ERR_TIMEOUT with the device and the context intact but the population undefined: call
+ * rp_pack_rows again to start over from the seed, or rp_destroy. */
 int rp_anneal(rp_ctx *ctx, const rp_anneal_params *params, rp_anneal_stats *stats);
 
-/* Validate the incumbent (coverage, capacity, non-empty cells, cached score equals a full
- * rescoring, not worse than the seed) and return it.
+/* Validate(x*) and the non-regression assertion that close Algorithm 3 (Section 4.1.3: the
+ * returned plan is the archived incumbent, checked before it is handed to the trainer): coverage,
+ * capacity, non-empty cells, cached score equals a full rescoring, not worse than the best seed;
+ * then return it.
  *   cell_of_sample [N] int32 out, nullable; score_fx [3], score_f64 [3] out, nullable.
  * RP_ERR_INVALID_PLAN when a check fails.  Outputs are complete on return.  Right after
  * rp_anneal the checks are already done and the call only hands the results over. */
@@ -266,6 +271,17 @@ typedef enum {
     RP_DUMP_EVAL_W = 16      /* int32 [R][G][L][P] of layout `index` of the last
                                 rp_eval_population call with explicit layouts (n <= 64)    */
 } rp_dump_what;
+/* Knobs that steer the annealing kernels onto paths that full-size windows or failures reach,
+ * so that small tests can cover them; all 0 (off) by default.
+ *   RP_KNOB_BARRIER_WORKSPACE: shared-memory bytes (multiple of 16, >= 64) the level barrier may
+ *     use; a small value sends its cumulative weights, cell bookkeeping and incumbent replay
+ *     through their global-memory forms.
+ *   RP_KNOB_WAIT_POLLS: polls after which a chain's wait on its asynchronous copies gives up
+ *     (default 2^22).
+ *   RP_KNOB_STALL_ONE_CHAIN: chain 0 waits once more, after its copies have landed, on a barrier
+ *     phase that nothing completes: the wait runs out and rp_anneal returns RP_ERR_TIMEOUT. */
+typedef enum { RP_KNOB_BARRIER_WORKSPACE = 1, RP_KNOB_WAIT_POLLS = 2, RP_KNOB_STALL_ONE_CHAIN = 3 } rp_knob;
+int rp_debug_set_knob(rp_ctx *ctx, int knob, int64_t value);
 /* Per-level traces (RP_DUMP_TRACE_*) are recorded by rp_anneal calls made after
  * rp_debug_set_trace(ctx, 1); off by default (the copies cost a few microseconds per level). */
 int rp_debug_set_trace(rp_ctx *ctx, int on);

@@ -21,8 +21,9 @@
 //  * scoring a move is a data-parallel pass over two L*P slices.
 // Resampling is folded into the next level's prologue: slot j starts from the terminal
 // state of its ancestor in the other population buffer, so no separate gather pass runs.
-// Trajectory-best layouts are not copied: every accepted move is logged (8 bytes) and the
-// level barrier rebuilds the one winning layout from the chain's start layout and its log.
+// The trajectory-best layout of the cooperative kernel below is not copied: every accepted move
+// is logged (8 bytes) and the level barrier rebuilds the one winning layout from the chain's
+// start layout and its log (the warp-per-candidate kernel snapshots the layout instead).
 //
 // Algorithmic bytes per feasible move: reads 2 W slices + the moved samples' q rows
 // ((3 or 4) * L*P*4 bytes), writes 2 W slices when accepted.
@@ -86,14 +87,22 @@ k_anneal_level(const AnnealArgs A)
     const bool vec = (dm.P >= 4) && (dm.P <= 128) && ((dm.P & (dm.P - 1)) == 0);
     const i64 aC = dm.asum * dm.C, bS = dm.bsum;
 
-    if (tid == 0) chain->failed = 0;
-    const bool landed = rp_chain_load<NT, false>(A, src, j, sm_blob, sm_static, nullptr, mbar, tid, src_cell, dst_cell);
-    if (tid == 0 && src_cell != dst_cell)                  // bytes of the W gather (counted here: off the level's tail)
-        atomicAdd((u64 *)&A.counters[5], (u64)2 * dm.RG * dm.LP * 4);
-    if (!landed) chain->failed = 1;
+    // An earlier level of this call gave up on a wait: its barrier did not run, so the ancestor
+    // tables are stale.  Every later chain does nothing but take its ticket.
+    if (tid == 0) chain->failed = __ldcg(&A.status[RP_SW_TIMEOUT]) ? 2 : 0;
+    __syncthreads();
+    if (!chain->failed) {
+        const bool landed = rp_chain_load<NT, false>(A, src, j, sm_blob, sm_static, nullptr, mbar, tid, src_cell, dst_cell);
+        if (tid == 0 && src_cell != dst_cell)              // bytes of the W gather (counted here: off the level's tail)
+            atomicAdd((u64 *)&A.counters[5], (u64)2 * dm.RG * dm.LP * 4);
+        if (!landed) chain->failed = 1;
+    }
     __syncthreads();
     if (chain->failed) {
-        if (tid == 0) atomicExch(&A.status[RP_SW_TIMEOUT], 1);
+        // A bounded wait ran out (1), or an earlier level's did (2): raise the status word, store
+        // nothing, and still take the ticket so that the arrival counter stays consistent.
+        if (tid == 0 && chain->failed == 1) atomicExch(&A.status[RP_SW_TIMEOUT], 1);
+        rp_finish_level(A, tid, NT, smraw, A.smem_bytes);
         return;
     }
     for (int c = tid; c < dm.K; c += NT) {
@@ -317,7 +326,7 @@ k_anneal_level(const AnnealArgs A)
 }
 
 // Thread count and shared-memory plan of the chain kernels.  Windows with L*P <= 512 use the
-// warp-per-candidate kernel; larger ones the cooperative kernel with 256 threads.
+// warp-per-candidate kernel; larger ones the cooperative kernel with 128 threads.
 size_t rp_wpc_smem_bytes(const RpDims &dm, const RpBlob &bl, const RpStatic &sl, int nw, int *w_in_smem);
 int rp_wpc_warps(int pop_size);
 int rp_launch_anneal_wpc(rp_ctx *c, const AnnealArgs &A);
@@ -378,6 +387,9 @@ int rp_launch_anneal_level(rp_ctx *c, int level, int n_levels, const rp_anneal_p
     A.Ppop = c->Ppop;
     A.last = (level == n_levels - 1);
     A.w_on_chip = 0;
+    A.wait_polls = c->knob_wait_polls > 0 ? c->knob_wait_polls : (1 << 22);
+    A.stall_test = c->knob_stall;
+    A.le_ws_cap = (unsigned)c->knob_le_ws_cap;
     A.lo.done = c->d_done; A.lo.anc_out = c->d_anc_next; A.lo.F = c->d_F;
     A.lo.wloc_out = c->d_wloc; A.lo.scratch = c->d_le_scratch;   // the barrier rewrites the array the level read from
     A.lo.inc_layout = c->d_inc_layout; A.lo.inc_score = c->d_inc_score;

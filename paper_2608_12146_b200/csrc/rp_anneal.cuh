@@ -41,6 +41,10 @@ struct AnnealArgs {
     u64 tau, cq, rho_q32, guide_q32;
     u32 key0, key1;
     u32 resample_x;                  // Philox(0, level, 0, 3).x, the word behind the resampling offset (computed on the host)
+    int wait_polls;                  // limit of every bounded wait on a bulk-copy barrier (polls)
+    int stall_test;                  // inspection hook: after its loads have landed, chain 0 waits once more on a
+                                     // barrier phase that nothing completes, so that the wait runs out
+    unsigned le_ws_cap;              // inspection hook: shared-memory bytes the level barrier may use (0 = all)
     i64 *term, *best;
     int *best_step, *best_nlog;
     u64 *digest;
@@ -220,10 +224,10 @@ __device__ __forceinline__ void rp_bulk_g2s(void *smem_dst, const void *gmem_src
                  ::"r"(rp_smem_addr(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(rp_smem_addr(mbar)) : "memory");
 }
 // Bounded wait on a barrier phase; false when the limit ran out.
-__device__ __forceinline__ bool rp_mbar_wait(u64 *mbar, u32 parity)
+__device__ __forceinline__ bool rp_mbar_wait(u64 *mbar, u32 parity, int limit)
 {
     const u32 addr = rp_smem_addr(mbar);
-    for (int it = 0; it < (1 << 22); ++it) {
+    for (int it = 0; it < limit; ++it) {
         u32 done;
         asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
                      : "=r"(done) : "r"(addr), "r"(parity) : "memory");
@@ -291,7 +295,11 @@ __device__ __forceinline__ bool rp_chain_load(const AnnealArgs &A, int src, int 
         }
     }
     __syncthreads();                       // the barrier's initialisation is visible to every waiter
-    return rp_mbar_wait(mbar, 0);
+    bool ok = rp_mbar_wait(mbar, 0, A.wait_polls);
+    // Inspection hook: every copy has landed (phase 0 is complete); phase 1 is completed by nobody,
+    // so this second wait gives up after wait_polls polls and the chain takes the time-out path.
+    if (ok && A.stall_test && j == 0) ok = rp_mbar_wait(mbar, 1, A.wait_polls);
+    return ok;
 }
 
 template <int NT, bool WS>

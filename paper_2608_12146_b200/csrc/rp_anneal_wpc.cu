@@ -70,12 +70,15 @@ __device__ __forceinline__ void rp_finish_level_async(const AnnealArgs &A, int t
         const int ticket = atomicAdd(A.lo.done, 1);
         asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");      // this thread issued them
         is_last_a = (ticket == (int)gridDim.x - 1);
-        if (is_last_a) *A.lo.done = 0;
+        if (is_last_a) {
+            *A.lo.done = 0;
+            if (__ldcg(&A.status[RP_SW_TIMEOUT])) is_last_a = 0;            // some chain gave up: no barrier, the call fails
+        }
     }
     __syncthreads();
     if (!is_last_a) return;
     __threadfence();
-    rp_level_end(A, tid, nt, ws, ws_bytes);
+    rp_level_end(A, tid, nt, ws, rp_le_ws_bytes(A, ws_bytes));
 }
 
 template <int NW, bool WS, int CH>
@@ -143,17 +146,29 @@ k_anneal_wpc(const AnnealArgs A)
     int *Wj = WS ? Wsm : A.W + (size_t)dst_cell * wn;
     // the incumbent's score when the level starts (fetched now, beside the loads above; used below)
     i64 inc0 = 0, inc1 = 0, inc2 = 0;
-    if (tid == 0) { inc0 = A.lo.inc_score[0]; inc1 = A.lo.inc_score[1]; inc2 = A.lo.inc_score[2]; }
+    if (tid == 0) {
+        // An earlier level of this call gave up on a wait: its barrier did not run, so the ancestor
+        // tables are stale.  Every later chain does nothing but take its ticket.
+        chain->failed = __ldcg(&A.status[RP_SW_TIMEOUT]) ? 2 : 0;
+        inc0 = A.lo.inc_score[0]; inc1 = A.lo.inc_score[1]; inc2 = A.lo.inc_score[2];
+    }
+    __syncthreads();
 
     // ---- prologue: adopt the ancestor's terminal state -------------------------------
-    if (tid == 0) chain->failed = 0;
-    const bool landed = rp_chain_load<NT, WS>(A, src, j, sm_blob, sm_static, Wsm, mbar, tid, src_cell, dst_cell);
-    if (tid == 0 && src_cell != dst_cell)                  // bytes of the W gather (counted here: off the level's tail)
-        atomicAdd((u64 *)&A.counters[5], (u64)2 * dm.RG * dm.LP * 4);
-    if (!landed) chain->failed = 1;
+    if (!chain->failed) {
+        const bool landed = rp_chain_load<NT, WS>(A, src, j, sm_blob, sm_static, Wsm, mbar, tid, src_cell, dst_cell);
+        if (tid == 0 && src_cell != dst_cell)              // bytes of the W gather (counted here: off the level's tail)
+            atomicAdd((u64 *)&A.counters[5], (u64)2 * dm.RG * dm.LP * 4);
+        if (!landed) chain->failed = 1;
+    }
     __syncthreads();
-    if (chain->failed) {                 // a bulk copy never landed: report and leave
-        if (tid == 0) atomicExch(&A.status[RP_SW_TIMEOUT], 1);
+    if (chain->failed) {
+        // A bounded wait ran out (1), or an earlier level's did (2): raise the status word, store
+        // nothing, and still take the ticket so that the arrival counter stays consistent.  The
+        // copies this CTA issued have either landed or have been given wait_polls polls to do so.
+        if (tid == 0 && chain->failed == 1) atomicExch(&A.status[RP_SW_TIMEOUT], 1);
+        asm volatile("griddepcontrol.launch_dependents;");
+        rp_finish_level_async(A, tid, NT, smraw, A.smem_bytes);
         return;
     }
     for (int c = tid; c < dm.K; c += NT) {

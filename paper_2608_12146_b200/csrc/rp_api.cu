@@ -728,12 +728,13 @@ static void make_schedule(const rp_anneal_params *p, RpLevel *lv)
 static int launch_best_check(rp_ctx *c);
 static int best_verdict(const rp_ctx *c, const int *sw);
 
-__global__ void k_reset_anneal(i64 *__restrict__ counters, int *__restrict__ status, int *__restrict__ inc_slot)
+__global__ void k_reset_anneal(i64 *__restrict__ counters, int *__restrict__ status, int *__restrict__ inc_slot,
+                               int *__restrict__ done)
 {
     const int x = threadIdx.x;
     if (x < 8) counters[x] = 0;
     if (x < RP_SW_COUNT) status[x] = 0;
-    if (x == 0) *inc_slot = -1;
+    if (x == 0) { *inc_slot = -1; *done = 0; }
 }
 
 extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *stats)
@@ -769,7 +770,7 @@ extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *
         c->trace_levels = NL;
     }
     // counters and status words to zero, incumbent slot to -1 (the incumbent is in d_inc_layout)
-    k_reset_anneal<<<1, 32, 0, c->stream>>>(c->d_counters, c->d_status, c->d_inc_slot);
+    k_reset_anneal<<<1, 32, 0, c->stream>>>(c->d_counters, c->d_status, c->d_inc_slot, c->d_done);
     ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
 
@@ -801,12 +802,19 @@ extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *
     }
     if (st == RP_OK && e != cudaSuccess) { g_rp_last_cuda_error = (int)e; st = RP_ERR_CUDA; }
     RP_TRY(st);
-    if (sw[RP_SW_TIMEOUT]) return RP_ERR_TIMEOUT;         // a bounded device-side wait ran out
+    if (sw[RP_SW_TIMEOUT]) {
+        // A bounded device-side wait ran out: that level's barrier and every later level were
+        // skipped, so the population is not a population any more.  Back to "placed": only
+        // rp_pack_rows (which rebuilds it from the seed) and rp_destroy make sense now.
+        c->stage = 2;
+        c->best_ready = 0;
+        return RP_ERR_TIMEOUT;
+    }
     if (stats) {
         stats->proposed = cn[0]; stats->feasible = cn[1]; stats->accepted = cn[2]; stats->improved = cn[3];
         stats->move_bytes = cn[4]; stats->gather_bytes = cn[5];
         stats->kernel_launches = (int64_t)NL;
-        stats->ms_chains = ms_chains; stats->ms_barrier = 0.0;   // the barrier runs inside the chain kernels
+        stats->ms_chains = ms_chains;
     }
     c->best_verdict = best_verdict(c, sw);
     c->best_ready = 1;
@@ -874,6 +882,22 @@ __global__ void k_cell_stats(const unsigned short *__restrict__ cells, const int
         atomicAdd((u64 *)&T[c], (u64)t[i]);
         atomicAdd((u64 *)&Q[c], (u64)t[i] * (u64)t[i]);
         atomicAdd(&cnt[c], 1);
+    }
+}
+
+extern "C" int rp_debug_set_knob(rp_ctx *c, int knob, int64_t value)
+{
+    if (!c || value < 0) return RP_ERR_ARG;
+    switch (knob) {
+        case RP_KNOB_BARRIER_WORKSPACE:
+            if (value > (1 << 20) || (value & 15) || (value && value < 64)) return RP_ERR_ARG;
+            c->knob_le_ws_cap = (int)value; return RP_OK;
+        case RP_KNOB_WAIT_POLLS:
+            if (value > (1 << 22)) return RP_ERR_ARG;
+            c->knob_wait_polls = (int)value; return RP_OK;
+        case RP_KNOB_STALL_ONE_CHAIN:
+            c->knob_stall = value ? 1 : 0; return RP_OK;
+        default: return RP_ERR_ARG;
     }
 }
 

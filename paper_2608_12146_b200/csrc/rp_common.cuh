@@ -153,6 +153,7 @@ struct rp_ctx {
     // trace of the last rp_anneal call
     int trace_levels;
     int trace_on;              // keep per-level traces (inspection hook; off by default)
+    int knob_le_ws_cap, knob_wait_polls, knob_stall;   // inspection hooks (rp_debug_set_knob); 0 = off
     i64 *d_tr_term, *d_tr_best, *d_tr_inc;
     int *d_tr_best_step, *d_tr_anc;
     u64 *d_tr_digest;

@@ -439,6 +439,8 @@ extern "C" int rp_eval_layouts_noalloc(rp_ctx *c, const int32_t *layouts, int32_
     if (n > RP_NOALLOC_MAX_LAYOUTS || (long long)n * dm.N > RP_NOALLOC_MAX_CELLS ||
         (long long)n * dm.RG > RP_NOALLOC_MAX_ROWSHARDS)
         return RP_ERR_RANGE;                  // beyond the fixed scratch: use rp_eval_population
+    const size_t smem = eval_smem_bytes(dm);
+    if (smem > 220 * 1024) return RP_ERR_RANGE;   // nothing has been queued yet
     int cur = -1;
     RP_CUDA(cudaGetDevice(&cur));
     if (cur != c->device || cur < 0 || cur >= 64) return RP_ERR_STATE;
@@ -449,6 +451,7 @@ extern "C" int rp_eval_layouts_noalloc(rp_ctx *c, const int32_t *layouts, int32_
         cudaPointerAttributes at;
         if (cudaPointerGetAttributes(&at, ptrs[x]) != cudaSuccess) { cudaGetLastError(); return RP_ERR_ARG; }
         if (at.type != cudaMemoryTypeDevice && at.type != cudaMemoryTypeManaged) return RP_ERR_ARG;
+        if (at.type == cudaMemoryTypeDevice && at.device != c->device) return RP_ERR_ARG;    // another GPU's memory
     }
     if (!g_noalloc_addr[cur]) {               // set-up, once per device, with that device current
         void *p = nullptr;
@@ -463,8 +466,6 @@ extern "C" int rp_eval_layouts_noalloc(rp_ctx *c, const int32_t *layouts, int32_
     k_layouts_to_cells<<<(int)((total + 255) / 256), 256, 0, c->stream>>>(layouts, total, dm.K, sc->cells, c->d_status);
     ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
-    const size_t smem = eval_smem_bytes(dm);
-    if (smem > 220 * 1024) return RP_ERR_RANGE;
     if (smem > 32 * 1024)
         RP_CUDA(cudaFuncSetAttribute(k_eval<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int splits = (2 * 148 + n - 1) / n;

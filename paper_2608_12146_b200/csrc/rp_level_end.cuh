@@ -404,6 +404,14 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
         O.wloc_out[m] = (need[m] >= 0) ? freelist[need[m]] : now_r[anc_r[m]];
 }
 
+// Shared-memory bytes the level barrier works in: all of the CTA's dynamic shared memory, unless
+// the inspection hook caps it (which sends the cumulative weights, the replayed layout and the
+// cell bookkeeping through their global-memory forms on windows of any size).
+__device__ __forceinline__ size_t rp_le_ws_bytes(const AnnealArgs &A, size_t ws_bytes)
+{
+    return (A.le_ws_cap && A.le_ws_cap < ws_bytes) ? (size_t)A.le_ws_cap : ws_bytes;
+}
+
 // Tail of a chain CTA: publish, take a ticket, and let the last arrival run the level barrier.
 __device__ __forceinline__ void rp_finish_level(const AnnealArgs &A, int tid, int nt, unsigned char *ws, size_t ws_bytes)
 {
@@ -413,10 +421,13 @@ __device__ __forceinline__ void rp_finish_level(const AnnealArgs &A, int tid, in
     if (tid == 0) {
         const int ticket = atomicAdd(A.lo.done, 1);
         is_last = (ticket == (int)gridDim.x - 1);
-        if (is_last) *A.lo.done = 0;
+        if (is_last) {
+            *A.lo.done = 0;
+            if (__ldcg(&A.status[RP_SW_TIMEOUT])) is_last = 0;              // some chain gave up: no barrier, the call fails
+        }
     }
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    rp_level_end(A, tid, nt, ws, ws_bytes);
+    rp_level_end(A, tid, nt, ws, rp_le_ws_bytes(A, ws_bytes));
 }

@@ -70,17 +70,18 @@ def check_eval(w, ctx, ref, edp, n=6, seed=0):
         np.testing.assert_allclose(f64[j], real, rtol=F64_RTOL, atol=0)
 
 
-def check_anneal(w, ctx, ref, edp, pop, levels, steps, threads=8, t_ratio=None, check_members=3, init=None):
+def check_anneal(w, ctx, ref, edp, pop, levels, steps, threads=8, t_ratio=None, check_members=3, init=None, t0=None):
     s = w.spec
+    t0 = s.t0 if t0 is None else t0
     R, D = ref["R"], s.dp_width
     ratio = s.t_ratio if t_ratio is None else t_ratio
     if init is None:
         init = np.tile(ref["seed"], (pop, 1))
-    want = oracle.anneal(w.lengths, ref["q"], init, R, s.token_cap, D, n_levels=levels, steps=steps, t0=s.t0,
+    want = oracle.anneal(w.lengths, ref["q"], init, R, s.token_cap, D, n_levels=levels, steps=steps, t0=t0,
                          t_ratio=ratio, p_reloc=s.p_reloc, p_guide=s.p_guide, seed=s.anneal_seed,
                          edp_of_dp=edp, alpha=s.alpha, beta=s.beta, n_threads=threads)
     assert want["status"] == 0
-    stats = rp.rp_anneal(ctx, n_levels=levels, steps_per_level=steps, t0=s.t0, t_ratio=ratio,
+    stats = rp.rp_anneal(ctx, n_levels=levels, steps_per_level=steps, t0=t0, t_ratio=ratio,
                          p_reloc=s.p_reloc, p_guide=s.p_guide)
     got_counters = [stats.proposed, stats.feasible, stats.accepted, stats.improved]
     assert got_counters == want["counters"].tolist()
@@ -250,6 +251,82 @@ def test_large_windows_full_shapes_reduced_budget(name, pop, levels, steps):
     check_front(w, ctx, ref)
     check_eval(w, ctx, ref, None, n=2)
     check_anneal(w, ctx, ref, None, pop, levels, steps, check_members=2)
+    rp.rp_destroy(ctx)
+
+
+@pytest.mark.parametrize("name,pop,levels,steps,t0", [("large", 1024, 20, 250, None), ("heavy", 8192, 2, 1000, None),
+                                                      ("wide", 4096, 2, 250, 2e-5)])
+def test_large_windows_full_population(name, pop, levels, steps, t0, threads=16):
+    """The three big windows at the population the benchmark runs them at (large at its whole
+    budget, heavy and wide for two levels of their real step count), every trace against the
+    oracle: this is where the four-members-per-thread weights, the cumulative weights in global
+    memory, the off-chip cell bookkeeping and the multi-wave rank-load free list run.  (Wide starts
+    colder than its schedule does, so that already its first resampling replaces members.)"""
+    w = make_window(name)
+    assert pop == w.spec.pop_size and steps == w.spec.steps_per_level
+    ref = oracle_front(w)
+    ctx = load(w, pop=pop, device_inputs=True)
+    check_front(w, ctx, ref)
+    want, stats = check_anneal(w, ctx, ref, None, pop, levels, steps, threads=threads, check_members=2, t0=t0)
+    assert stats.accepted > pop            # the levels did move
+    if levels > 1:                          # resampling really replaced members and kept others
+        anc = want["anc"][0]
+        assert 1 < len(set(anc.tolist())) < pop
+    rp.rp_destroy(ctx)
+
+
+BARRIER_CASES = [
+    # name, N, L, E, k, C, D, P, edp, min_rows, pop   (first two: warp-per-candidate kernel; last two: cooperative kernel, L*P > 512)
+    ("ws_small", 96, 5, 16, 2, 4096, 4, 4, [0, 0, 1, 1], 3, 37),
+    ("ws_pow2", 130, 9, 40, 2, 8192, 5, 20, None, 3, 64),
+    ("ws_coop", 120, 20, 32, 2, 4096, 4, 32, None, 3, 40),
+    ("ws_coop_shared", 150, 17, 64, 2, 4096, 4, 32, [0, 1, 1, 0], 2, 130),
+]
+
+
+@pytest.mark.parametrize("spec", BARRIER_CASES, ids=[e[0] for e in BARRIER_CASES])
+@pytest.mark.parametrize("cap", [0, 64])
+def test_level_barrier_paths_on_small_windows(spec, cap):
+    """The level barrier with all of its shared memory (cap 0) and with next to none (cap 64: the
+    cumulative weights, the cell bookkeeping and the incumbent's replay go through global memory,
+    as they do for populations of thousands), on windows small enough for many levels; the
+    cooperative kernel is reached with L*P > 512."""
+    name, N, L, E, k, C, D, P, edp, min_rows, pop = spec
+    w = make_window(custom_spec(name, N, L, E, k, C, D, P, pop, 400, data_seed=len(name) * 11 + N))
+    ref = oracle_front(w, edp, min_rows)
+    ctx = load(w, pop=pop, edp=edp, min_rows=min_rows)
+    rp.rp_debug_set_knob(ctx, "BARRIER_WORKSPACE", cap)
+    check_front(w, ctx, ref)
+    want, stats = check_anneal(w, ctx, ref, edp, pop, 10, 40, t_ratio=0.6, check_members=2)
+    assert stats.accepted > 50 and stats.improved > 0
+    rp.rp_destroy(ctx)
+
+
+@pytest.mark.parametrize("spec", [BARRIER_CASES[0], BARRIER_CASES[2]], ids=["warp_per_candidate", "cooperative"])
+def test_a_wait_that_runs_out_is_reported_and_the_context_survives(spec):
+    """One chain waits on a barrier phase that nothing completes, with the poll limit cut to 10^4:
+    the wait gives up, the kernels return, rp_anneal reports RP_ERR_TIMEOUT, the calls that make no
+    sense afterwards are refused, and after rp_pack_rows the same context anneals again, bit for
+    bit as the oracle does.  Nothing traps, faults or spins without a limit."""
+    name, N, L, E, k, C, D, P, edp, min_rows, pop = spec
+    w = make_window(custom_spec(name, N, L, E, k, C, D, P, pop, 400, data_seed=len(name) * 11 + N))
+    s = w.spec
+    ref = oracle_front(w, edp, min_rows)
+    ctx = load(w, pop=pop, edp=edp, min_rows=min_rows)
+    check_front(w, ctx, ref)
+    rp.rp_debug_set_knob(ctx, "WAIT_POLLS", 10000)
+    rp.rp_debug_set_knob(ctx, "STALL_ONE_CHAIN", 1)
+    for _ in range(2):                      # the second call finds the arrival counter and the status words clean
+        with pytest.raises(rp.RpError) as e:
+            rp.rp_anneal(ctx, n_levels=4, steps_per_level=30, t0=s.t0, t_ratio=0.6, p_reloc=s.p_reloc, p_guide=s.p_guide)
+        assert e.value.status == -8
+        with pytest.raises(rp.RpError) as e:    # the population is gone: annealing on needs rp_pack_rows first
+            rp.rp_anneal(ctx, n_levels=1, steps_per_level=5, t0=s.t0, t_ratio=0.6, p_reloc=s.p_reloc, p_guide=s.p_guide)
+        assert e.value.status == -7
+        assert rp.rp_pack_rows(ctx) == (ref["R"], ref["cert"])
+    rp.rp_debug_set_knob(ctx, "STALL_ONE_CHAIN", 0)
+    rp.rp_debug_set_knob(ctx, "WAIT_POLLS", 0)
+    check_anneal(w, ctx, ref, edp, pop, 4, 30, t_ratio=0.6, check_members=1)
     rp.rp_destroy(ctx)
 
 
@@ -588,6 +665,16 @@ def test_bad_inputs_are_host_side_errors():
     with pytest.raises(rp.RpError) as e:
         rp.rp_window_load(w.lengths, w.demand, edp_of_dp=[0, 2], **kw)      # shard 1 unused
     assert e.value.status == -2
+    # rank loads are 32-bit: k * C * (DP slots of one shard) must stay below 2^31; the cap itself below 2^24
+    with pytest.raises(rp.RpError) as e:
+        rp.rp_window_load(w.lengths, w.demand, **dict(kw, top_k=64, token_cap=1 << 24, edp_of_dp=[0, 0]))
+    assert e.value.status == -5
+    with pytest.raises(rp.RpError) as e:
+        rp.rp_window_load(w.lengths, w.demand, **dict(kw, token_cap=(1 << 24) + 1))
+    assert e.value.status == -5
+    with pytest.raises(rp.RpError) as e:                                     # score range: (2^8*C*L*k + ...) * sum t >= 2^62
+        rp.rp_window_load(w.lengths, w.demand, **dict(kw, token_cap=1 << 24, alpha=(1e6,), beta=(0.0,)))
+    assert e.value.status == -5
     ctx = rp.rp_window_load(w.lengths, w.demand, **kw)
     with pytest.raises(rp.RpError) as e:
         rp.rp_pack_rows(ctx)                                                 # before rp_place_experts
