@@ -5,18 +5,21 @@ A "step" is one complete plan of one synthetic optimizer-step window: input chec
 aggregate demand, LPT placement, demand projection, row count + seed, population annealing
 over all temperature levels, validation and return of the best layout.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload medium] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload heavy] [--impl reference]
 
 Prints ONE JSON line.  `value` = replica-moves evaluated per second over the whole timed
 region (all stages, inputs resident in HBM); `e2e` = the same with host buffers in and out
 through the C ABI; `roofline` = the per-level chain kernel against the measured HBM peak;
-`cpu_baseline` = the C oracle on this machine's host cores.  With N > 1 every rank plans its own
-copy of the window (replicas only, no collective on the data path).
+`cpu_baseline` = the C oracle on this machine's host cores.  The headline workload is the largest
+window (heavy); `other_workloads` carries the same record for the other four windows.  With
+N > 1 every rank plans its own copy of the window (replicas only, no collective on the data path).
 """
 from __future__ import annotations
 
 import argparse
+import glob
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -34,9 +37,11 @@ from paper_2608_12146_b200.windows import SPECS, make_window
 METRIC = "annealing replica-moves evaluated/sec"
 UNIT = "moves/s"
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes (read + write) per launch of the chain kernel from the ncu captures summarised under
-# profiles/ (k_anneal_wpc_medium.txt); None where no full-size capture exists.
-NCU_DRAM_BYTES_PER_LAUNCH = {"medium": 6.5e6}
+# Bounded oracle samples (population, levels): the oracle scores every member of the initial
+# population from scratch and holds two rank-load tensors per member, so a sample keeps the window
+# and the steps per level and bounds the members and the levels.
+CPU_SAMPLE = {"tiny": (8, 20), "medium": (256, 20), "large": (1024, 4), "wide": (512, 2), "heavy": (2048, 2)}
+REF_SAMPLE = {"tiny": (8, 20), "medium": (256, 20), "large": (1024, 1), "wide": (128, 1), "heavy": (256, 1)}
 
 
 def hbm_peak():
@@ -49,34 +54,63 @@ def hbm_peak():
     return FALLBACK_HBM_GBS, "fallback"
 
 
+def profiled_traffic(kernel, workload):
+    """DRAM / L2 bytes per launch from the ncu summaries under profiles/: a summary that wants to be
+    used here carries one line `bench_traffic: {json}` naming its kernel, workload and population."""
+    for path in sorted(glob.glob(os.path.join(ROOT, "profiles", "*.txt"))):
+        try:
+            for line in open(path):
+                if not line.startswith("bench_traffic:"):
+                    continue
+                rec = json.loads(line[len("bench_traffic:"):])
+                if rec.get("kernel") == kernel and rec.get("workload") == workload:
+                    rec["file"] = os.path.relpath(path, ROOT)
+                    return rec
+        except Exception:
+            continue
+    return None
+
+
 def workload_config(spec, extra=None):
     cfg = {"workload": spec.name, "n_samples": spec.n_samples, "n_layers": spec.n_layers,
            "n_experts": spec.n_experts, "top_k": spec.top_k, "token_cap": spec.token_cap,
            "dp_shards": spec.dp_width, "ep_ranks": spec.ep_width, "population": spec.pop_size,
            "sweeps": spec.sweeps, "n_levels": spec.n_levels, "steps_per_level": spec.steps_per_level,
-           "l2": "flushed between steps (256 MiB write)"}
+           "l2": "flushed between steps (256 MiB written, then read back so that no dirty lines are left to evict)"}
     if extra:
         cfg.update(extra)
     return cfg
 
 
 # ---------------------------------------------------------------------------------------------
-# reference arm: the oracle on the host cores
+# the oracle on the host cores (reference arm and cpu_baseline)
 # ---------------------------------------------------------------------------------------------
-def oracle_sample(w, threads, budget_moves=3.0e6):
-    """Run the oracle on a bounded sample of the workload: the whole front end once, then
-    annealing at the full population for as many whole levels as fit the move budget."""
+def oracle_sample(w, threads, pop, levels):
+    """The oracle on a bounded sample of the workload: the whole front end once, then annealing
+    of `pop` members for `levels` whole temperature levels of the window's own step count."""
     import oracle
     s = w.spec
-    per_level = s.pop_size * s.steps_per_level
-    levels = int(max(1, min(s.n_levels, budget_moves // per_level)))
+    pop, levels = min(pop, s.pop_size), min(levels, s.n_levels)
     t0 = time.perf_counter()
-    res = oracle.plan(w, n_levels=levels, n_threads=threads, trace=False)
+    res = oracle.plan(w, pop_size=pop, n_levels=levels, n_threads=threads, trace=False)
     dt = time.perf_counter() - t0
     moves = int(res["counters"][0])
-    sample = (f"whole front end + {levels} of {s.n_levels} temperature levels at the full population "
-              f"({moves} replica-moves)")
+    sample = (f"whole front end + {levels} of {s.n_levels} temperature levels x {s.steps_per_level} steps for "
+              f"{pop} of {s.pop_size} members ({moves} replica-moves)")
     return moves, dt, sample
+
+
+def cpu_baseline(w, seconds):
+    import oracle
+    oracle.build()
+    threads = os.cpu_count() or 1
+    pop, levels = CPU_SAMPLE[w.spec.name]
+    m, d, reps = 0, 0.0, 0
+    while reps == 0 or (d < seconds and reps < 4096):
+        mi, di, sample = oracle_sample(w, threads, pop, levels)
+        m, d, reps = m + mi, d + di, reps + 1
+    return {"value": m / d, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"{reps} x ({sample})", "seconds": d}
 
 
 def run_reference(args):
@@ -88,22 +122,21 @@ def run_reference(args):
     spec = SPECS[args.workload]
     w = make_window(spec)
     threads = os.cpu_count() or 1
-    budget = {"tiny": 1e5, "medium": 3e6, "large": 6e6, "wide": 3e6, "heavy": 8e6}[spec.name]
-    for _ in range(args.warmup):
-        oracle_sample(w, threads, budget)
-    moves = 0
-    dt = 0.0
-    sample = ""
+    pop, levels = REF_SAMPLE[spec.name]
+    for _ in range(min(args.warmup, 2)):
+        oracle_sample(w, threads, pop, levels)
+    moves, dt, sample = 0, 0.0, ""
     for _ in range(args.steps):
-        m, d, sample = oracle_sample(w, threads, budget)
+        m, d, sample = oracle_sample(w, threads, pop, levels)
         moves += m
         dt += d
     value = moves / dt
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
-            "data": "synthetic", "config": workload_config(spec),
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "data": "synthetic", "config": workload_config(spec, {"parallelism": "1 gpu" if args.gpus == 1 else "replicas only"}),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                             "sample": f"each step: {sample}"},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
@@ -139,7 +172,7 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
             out = ""
-        sm, mx, reasons = [], [], set()
+        sm, mx, power, reasons = [], [], [], set()
         for line in out.splitlines():
             f = [x.strip() for x in line.split(",")]
             if len(f) < 9:
@@ -147,13 +180,14 @@ class ClockSampler:
             try:
                 sm.append(float(f[1]))
                 mx.append(float(f[2]))
+                power.append(float(f[3]))
             except ValueError:
                 continue
             for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm), "power_w_max": max(power) if power else None}
 
 
 def reduce_job(ms_local, moves_local, dist=None, device="cpu"):
@@ -171,7 +205,7 @@ def reduce_job(ms_local, moves_local, dist=None, device="cpu"):
     return float(tmax.item()), int(round(tsum.item()))
 
 
-def plan_once(rp, torch, w, t_in, a_in, outs, stream, want_stats=True):
+def plan_once(rp, w, t_in, a_in, outs, stream, stages=None):
     """One pass of the whole hot path through the C ABI; returns the annealing stats."""
     s = w.spec
     ctx = rp.rp_window_load(t_in, a_in, top_k=s.top_k, token_cap=s.token_cap, dp_width=s.dp_width,
@@ -180,14 +214,19 @@ def plan_once(rp, torch, w, t_in, a_in, outs, stream, want_stats=True):
     rp.rp_place_experts(ctx, outs["pi"], outs["rank_load"])
     rp.rp_pack_rows(ctx)
     stats = rp.rp_anneal(ctx, n_levels=s.n_levels, steps_per_level=s.steps_per_level, t0=s.t0,
-                         t_ratio=s.t_ratio, p_reloc=s.p_reloc, p_guide=s.p_guide, want_stats=want_stats)
+                         t_ratio=s.t_ratio, p_reloc=s.p_reloc, p_guide=s.p_guide, want_stats=True)
     rp.rp_best(ctx, outs["layout"], outs["score_fx"], outs["score_f64"])
+    if stages is not None:
+        for k, v in rp.rp_debug_stage_times(ctx).items():
+            if v is not None:
+                stages[k] = stages.get(k, 0.0) + v
     rp.rp_destroy(ctx)
     return stats
 
 
-def measure(rp, torch, args, name, steps, dist, dev, local, with_clocks, with_cpu):
-    """Time `steps` plans of the named workload on this rank; returns the pieces of the JSON line."""
+def measure(rp, torch, args, name, steps, min_seconds, dist, dev, local, cpu_seconds):
+    """Time plans of the named workload on this rank (exactly `steps` of them, or as many more as
+    `min_seconds` of timed region needs); returns the pieces of the JSON line."""
     spec = SPECS[name]
     overrides = {}
     if args.pop:
@@ -214,28 +253,32 @@ def measure(rp, torch, args, name, steps, dist, dev, local, with_clocks, with_cp
     outs_dev = outputs(device=dev)
     outs_host = {k: v.pin_memory() for k, v in outputs().items()}
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    flush_sink = torch.empty(1, dtype=torch.uint8, device=dev)
 
     def barrier():
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    def timed_loop(t_in, a_in, outs, n):
+    def timed_loop(t_in, a_in, outs, n, stages=None):
         """n plans, each timed with CUDA events on the launching stream; L2 flushed in between."""
-        acc = dict(ms=0.0, chain_ms=0.0, move_bytes=0, gather_bytes=0, feasible=0, accepted=0, chain_launches=0)
+        acc = dict(ms=0.0, chain_ms=0.0, move_bytes=0, gather_bytes=0, staging_bytes=0, feasible=0, accepted=0,
+                   chain_launches=0)
         barrier()
         wall0 = time.perf_counter()
         for _ in range(n):
             flush.fill_(1)
+            flush_sink.copy_(flush[:1] + flush.max())       # read pass: the cache is left with clean lines only
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(stream)
-            st = plan_once(rp, torch, w, t_in, a_in, outs, stream)
+            st = plan_once(rp, w, t_in, a_in, outs, stream, stages)
             e1.record(stream)
             e1.synchronize()
             acc["ms"] += e0.elapsed_time(e1)
             acc["chain_ms"] += st.ms_chains
             acc["move_bytes"] += st.move_bytes
             acc["gather_bytes"] += st.gather_bytes
+            acc["staging_bytes"] += st.staging_bytes
             acc["feasible"] += st.feasible
             acc["accepted"] += st.accepted
             acc["chain_launches"] += s.n_levels
@@ -243,61 +286,117 @@ def measure(rp, torch, args, name, steps, dist, dev, local, with_clocks, with_cp
         acc["wall"] = time.perf_counter() - wall0
         return acc
 
+    warm_ms = []
     for _ in range(args.warmup):
-        plan_once(rp, torch, w, t_dev, a_dev, outs_dev, stream)
-        plan_once(rp, torch, w, t_pin, a_pin, outs_host, stream)
-    clocks = None
-    if with_clocks:
-        vis = [x for x in os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",") if x]
-        sampler = ClockSampler(vis[local] if local < len(vis) else local)
-        sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        plan_once(rp, w, t_dev, a_dev, outs_dev, stream)
+        e1.record(stream)
+        e1.synchronize()
+        warm_ms.append(e0.elapsed_time(e1))
+        plan_once(rp, w, t_pin, a_pin, outs_host, stream)
+    if min_seconds:
+        steps = max(steps, int(math.ceil(min_seconds * 1e3 / max(min(warm_ms), 1e-3))))
+    vis = [x for x in os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",") if x]
+    sampler = ClockSampler(vis[local] if local < len(vis) else local)
+    sampler.start()
     launches0 = rp.rp_debug_launch_count()
     res = timed_loop(t_dev, a_dev, outs_dev, steps)
     launches = rp.rp_debug_launch_count() - launches0
-    if with_clocks:
-        clocks = sampler.stop()
+    clocks = sampler.stop()
     e2e = timed_loop(t_pin, a_pin, outs_host, steps)
+    # stage times of the front end: a few more plans with events around its kernels (outside the timed regions)
+    stages = {}
+    n_st = max(1, min(steps, 5))
+    rp.rp_debug_set_stage_timing(True)
+    timed_loop(t_dev, a_dev, outs_dev, n_st, stages)
+    rp.rp_debug_set_stage_timing(False)
+    stages = {k: v / n_st for k, v in stages.items()}
 
     ms, total_moves = reduce_job(res["ms"], moves_per_step * steps, dist, dev)
     ms_e2e, _ = reduce_job(e2e["ms"], moves_per_step * steps, dist, dev)
     world = 1 if dist is None else dist.get_world_size()
     peak, peak_kind = hbm_peak()
-    per_launch_s = res["chain_ms"] * 1e-3 / res["chain_launches"]
-    alg = (res["move_bytes"] + res["gather_bytes"]) / res["chain_launches"]
+    nl = res["chain_launches"]
+    per_launch_s = res["chain_ms"] * 1e-3 / nl
+    alg = (res["move_bytes"] + res["gather_bytes"]) / nl
     achieved = alg / per_launch_s / 1e9
     chain_kernel = "k_anneal_wpc" if s.n_layers * s.ep_width <= 512 else "k_anneal_level"
     roofline = {"bound": "hbm", "kernel": chain_kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_source": peak_kind, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(s.name),
-                "algorithmic_bytes_per_launch": alg,
-                "move_bytes_per_launch": res["move_bytes"] / res["chain_launches"],
-                "gather_bytes_per_launch": res["gather_bytes"] / res["chain_launches"],
-                "launch_ms": per_launch_s * 1e3, "share_of_step": res["chain_ms"] / res["ms"]}
+                "frac": achieved / peak, "peak_source": peak_kind, "served_by": "L2+HBM (algorithmic bytes; see dram)",
+                "traffic": None, "algorithmic_bytes_per_launch": alg,
+                "move_bytes_per_launch": res["move_bytes"] / nl, "gather_bytes_per_launch": res["gather_bytes"] / nl,
+                "staging_bytes_per_launch": res["staging_bytes"] / nl,
+                "launch_ms": per_launch_s * 1e3, "launches_per_step": s.n_levels, "share_of_step": res["chain_ms"] / res["ms"]}
+    prof = profiled_traffic(chain_kernel, s.name)
+    if prof:
+        scale = s.pop_size / float(prof["population"])
+        dram = prof["dram_bytes_per_launch"] * scale
+        roofline["traffic"] = dram
+        roofline["dram"] = {"source": prof["file"], "captured_population": prof["population"],
+                            "scaled_by_population": scale, "bytes_per_launch": dram,
+                            "hbm_frac": dram / per_launch_s / 1e9 / peak,
+                            "l2_bytes_per_launch": prof.get("lts_bytes_per_launch", 0) * scale or None,
+                            "captured_dram_gbs": prof.get("dram_gbs"), "captured_l2_gbs": prof.get("lts_gbs")}
+    n_le = s.n_samples * s.n_layers * s.n_experts * 4
+    n_lp = s.n_samples * s.n_layers * s.ep_width * 4
+    front = {}
+    for key, byts in (("check_reduce", n_le), ("projection", n_le + n_lp)):
+        if stages.get(key):
+            gbs = byts / stages[key] / 1e6
+            front[key] = {"ms": stages[key], "algorithmic_bytes": byts, "gbs": gbs, "frac_of_hbm_peak": gbs / peak}
     cpu = None
-    if with_cpu:
-        import oracle
-        oracle.build()
-        threads = os.cpu_count() or 1
-        budget = {"tiny": 1e5, "medium": 2e7, "large": 2e7, "wide": 6e6, "heavy": 2e7}[s.name]
-        oracle_sample(w, threads, min(budget, 1e6))           # warm the page cache and the thread pool
-        m, d, reps = 0, 0.0, 0
-        while d < 2.0 and reps < 64:                          # a few seconds of wall time on all cores
-            mi, di, sample = oracle_sample(w, threads, budget)
-            m, d, reps = m + mi, d + di, reps + 1
-        cpu = {"value": m / d, "unit": UNIT, "cores": threads, "kind": "oracle",
-               "sample": f"{reps} x ({sample})", "seconds": d}
+    if cpu_seconds:
+        cpu = cpu_baseline(w, cpu_seconds)
     h2d = int(w.lengths.nbytes + w.demand.nbytes)
     d2h = int(sum(v.numel() * v.element_size() for v in outs_host.values()))
     n_all = moves_per_step * steps
-    return {"value": total_moves / (ms * 1e-3), "ms_per_step": ms / steps,
+    stage_ms = {"anneal_levels": res["chain_ms"] / steps, "other": (res["ms"] - res["chain_ms"]) / steps}
+    stage_ms.update(stages)
+    return {"value": total_moves / (ms * 1e-3), "ms_per_step": ms / steps, "steps": steps,
             "config": workload_config(spec, {"parallelism": "replicas only" if world > 1 else "1 gpu"}),
             "plans_per_s": steps * world / (ms * 1e-3),
             "anneal_only_moves_per_s": n_all / (res["chain_ms"] * 1e-3),
             "feasible_fraction": res["feasible"] / n_all, "accepted_fraction": res["accepted"] / n_all,
-            "stage_ms_per_step": {"anneal_levels": res["chain_ms"] / steps, "other": (res["ms"] - res["chain_ms"]) / steps},
+            "stage_ms_per_step": stage_ms, "front_end": front,
             "roofline": roofline, "cpu_baseline": cpu,
             "e2e": {"value": total_moves / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / steps},
-            "gpu_launches": int(launches), "clocks": clocks, "wall_s": res["wall"]}
+            "gpu_launches": int(launches), "clocks": clocks, "timed_region_s": res["wall"]}
+
+
+def concurrent_plans(rp, torch, name, dev, n_ctx, reps):
+    """Context figure: plans per second with `n_ctx` windows planned at once on separate streams and
+    contexts (the ABI allows it); reported beside the single-plan latency, never instead of it."""
+    import threading
+    w = make_window(SPECS[name])
+    s = w.spec
+    t_dev = torch.from_numpy(w.lengths).to(dev)
+    a_dev = torch.from_numpy(w.demand).to(dev)
+    streams = [torch.cuda.Stream(device=dev) for _ in range(n_ctx)]
+
+    def worker(k, n):
+        torch.cuda.set_device(dev)
+        outs = dict(pi=torch.empty((s.n_layers, s.n_experts), dtype=torch.int32, device=dev),
+                    rank_load=torch.empty((s.n_layers, s.ep_width), dtype=torch.int64, device=dev),
+                    layout=torch.empty(s.n_samples, dtype=torch.int32, device=dev),
+                    score_fx=torch.empty(3, dtype=torch.int64, device=dev),
+                    score_f64=torch.empty(3, dtype=torch.float64, device=dev))
+        for _ in range(n):
+            plan_once(rp, w, t_dev, a_dev, outs, streams[k])
+
+    for n in (2, reps):                      # warm up, then time
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        th = [threading.Thread(target=worker, args=(k, n)) for k in range(n_ctx)]
+        for x in th:
+            x.start()
+        for x in th:
+            x.join()
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+    return {"workload": name, "concurrent_contexts": n_ctx, "plans": n_ctx * reps, "plans_per_s": n_ctx * reps / dt,
+            "timing": "wall clock around host threads, one stream and context each"}
 
 
 def seeding_stages(rp, torch, name, dev, reps=3):
@@ -330,10 +429,28 @@ def seeding_stages(rp, torch, name, dev, reps=3):
             "choice_width": 4, "n_proj": 8, "eta_q16": 1 << 16}
 
 
-def eval_stage(rp, torch, name, dev, reps=10):
-    """Context figure: full scoring of one population-sized batch of layouts (rp_eval_population,
-    device inputs and outputs): layouts/s and algorithmic bytes (N*2 + N*L*P*4 per layout) per second."""
-    import numpy as np
+def l2_copy_rate(torch, dev, mib=24, reps=50):
+    """Device-to-device copy of a buffer that stays in L2 (read + write bytes per second): the
+    denominator for kernels whose operands L2 serves."""
+    a = torch.empty(mib << 20, dtype=torch.uint8, device=dev)
+    b = torch.empty_like(a)
+    for _ in range(5):
+        b.copy_(a)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        b.copy_(a)
+    e1.record()
+    e1.synchronize()
+    return 2.0 * (mib << 20) * reps / (e0.elapsed_time(e1) * 1e-3) / 1e9
+
+
+def eval_stage(rp, torch, name, dev, l2_gbs, reps=10):
+    """Context figure: full scoring of one population-sized batch of distinct layouts
+    (rp_eval_population, device inputs and outputs).  The demand rows every layout gathers
+    (N*L*P*4 bytes per layout) are shared by all layouts and served by L2, so they are set against a
+    measured L2 copy rate; what must cross HBM is the assignment (N*2 bytes per layout) plus the
+    demand rows once, set against the measured HBM peak."""
     w = make_window(SPECS[name])
     s = w.spec
     t_dev = torch.from_numpy(w.lengths).to(dev)
@@ -356,9 +473,15 @@ def eval_stage(rp, torch, name, dev, reps=10):
     e1.synchronize()
     ms = e0.elapsed_time(e1) / reps
     rp.rp_destroy(ctx)
-    byts = s.pop_size * (s.n_samples * 2 + s.n_samples * s.n_layers * s.ep_width * 4)
+    peak, _ = hbm_peak()
+    q_bytes = s.n_samples * s.n_layers * s.ep_width * 4
+    gathered = s.pop_size * q_bytes
+    hbm_min = s.pop_size * s.n_samples * 4 + q_bytes          # int32 layouts in, demand rows once
     return {"workload": name, "layouts": s.pop_size, "ms": ms, "layouts_per_s": s.pop_size / ms * 1e3,
-            "algorithmic_gbs": byts / ms / 1e6}
+            "roofline": {"bound": "l2", "kernel": "k_eval", "achieved": gathered / ms / 1e6, "peak": l2_gbs, "unit": "GB/s",
+                         "frac": gathered / ms / 1e6 / l2_gbs, "peak_source": "L2-resident device copy measured in this run",
+                         "gathered_bytes_per_launch": gathered, "hbm_bytes_per_launch_min": hbm_min,
+                         "hbm_min_gbs": hbm_min / ms / 1e6, "hbm_min_frac": hbm_min / ms / 1e6 / peak}}
 
 
 def mechanism_diagnostics(rp, torch, name, dev):
@@ -403,29 +526,35 @@ def run_cuda(args):
     rp.lib()
     dev = torch.device("cuda", local)
 
-    main_res = measure(rp, torch, args, args.workload, args.steps, dist, dev, local, with_clocks=True,
-                       with_cpu=(world == 1 and rank == 0 and not args.no_cpu_baseline))
+    if args.eval_only:          # profiling aid: only the population-sized scoring batch of the named window
+        l2 = l2_copy_rate(torch, dev)
+        print(json.dumps(eval_stage(rp, torch, args.workload, dev, l2, reps=max(1, args.steps))))
+        return 0
+    main_cpu = 0 if (world > 1 or rank != 0 or args.no_cpu_baseline) else 12.0
+    main_res = measure(rp, torch, args, args.workload, args.steps, 0.0, dist, dev, local, main_cpu)
+    rp.rp_release_cached_memory()
     sweep = {}
+    extras = args.sweep and world == 1 and not args.pop and not args.levels
     if args.sweep and world == 1:
-        for name in SPECS:            # context beside the headline: the other windows, 3 plans each
+        for name in SPECS:            # the other windows: the same record, at least 1 s of timed region each
             if name == args.workload:
                 continue
-            r = measure(rp, torch, args, name, 3, None, dev, local, with_clocks=False, with_cpu=False)
-            sweep[name] = {"moves_per_s": r["value"], "plans_per_s": r["plans_per_s"], "ms_per_plan": r["ms_per_step"],
-                           "roofline_frac": r["roofline"]["frac"], "algorithmic_gbs": r["roofline"]["achieved"],
-                           "kernel": r["roofline"]["kernel"], "feasible_fraction": r["feasible_fraction"],
-                           "accepted_fraction": r["accepted_fraction"]}
+            sweep[name] = measure(rp, torch, args, name, 3, 1.0, None, dev, local, 0 if args.no_cpu_baseline else 4.0)
             rp.rp_release_cached_memory()
     if rank == 0:
-        line = {"metric": METRIC, "value": main_res.pop("value"), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        steps = main_res.pop("steps")
+        line = {"metric": METRIC, "value": main_res.pop("value"), "unit": UNIT, "n_gpus": world, "steps": steps,
                 "warmup": args.warmup, "ms_per_step": main_res.pop("ms_per_step"), "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic"}
         line.update(main_res)
         if sweep:
             line["other_workloads"] = sweep
-        if args.sweep and world == 1 and not args.pop and not args.levels:
-            line["seeding_stages"] = seeding_stages(rp, torch, args.workload, dev)
-            line["eval_population"] = [eval_stage(rp, torch, n, dev) for n in ("medium", "large", "wide")]
+        if extras:
+            l2 = l2_copy_rate(torch, dev)
+            line["l2_copy_gbs"] = l2
+            line["eval_population"] = [eval_stage(rp, torch, n, dev, l2) for n in ("medium", "large", "wide")]
+            line["concurrent_plans"] = [concurrent_plans(rp, torch, "medium", dev, n, 200) for n in (1, 2, 4)]
+            line["seeding_stages"] = seeding_stages(rp, torch, "medium", dev)
             line["mechanism_diagnostics"] = [mechanism_diagnostics(rp, torch, n, dev) for n in ("medium", "large")]
         print(json.dumps(line))
     if dist is not None:
@@ -436,13 +565,15 @@ def run_cuda(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=40)
-    ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--workload", default="medium", choices=list(SPECS))
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="heavy", choices=list(SPECS))
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", dest="sweep", action="store_false",
-                    help="skip the context sweep over the other four windows (3 plans each, N=1 only)")
+                    help="skip the records of the other four windows and the context figures (N=1 only)")
+    ap.add_argument("--eval-only", action="store_true",
+                    help="profiling aid: time only rp_eval_population on a population-sized batch of the workload")
     ap.add_argument("--pop", type=int, default=0, help="override the population size (profiling aid)")
     ap.add_argument("--levels", type=int, default=0, help="override the number of temperature levels (profiling aid)")
     args = ap.parse_args()

@@ -85,6 +85,9 @@ typedef struct {
                                    and demand rows read, slices written on accept           */
     int64_t gather_bytes;       /* rank-load bytes read+written for members that resampling
                                    replaced by another member's state                       */
+    int64_t staging_bytes;      /* rank-load bytes moved between global and shared memory for
+                                   members that kept their own state (windows whose rank loads
+                                   live on chip during a level); 0 otherwise                 */
     int64_t kernel_launches;    /* kernels this call launched                                */
 } rp_anneal_stats;
 
@@ -282,6 +285,15 @@ typedef enum {
  *     phase that nothing completes: the wait runs out and rp_anneal returns RP_ERR_TIMEOUT. */
 typedef enum { RP_KNOB_BARRIER_WORKSPACE = 1, RP_KNOB_WAIT_POLLS = 2, RP_KNOB_STALL_ONE_CHAIN = 3 } rp_knob;
 int rp_debug_set_knob(rp_ctx *ctx, int knob, int64_t value);
+/* Device time of the stages that have no statistics struct of their own.  After
+ * rp_debug_set_stage_timing(1) (process-wide; contexts loaded later record CUDA events around the
+ * kernels, a few microseconds of host time per call), rp_debug_stage_times synchronises the
+ * context's stream and fills ms[6], milliseconds, -1 where the stage has not run on this context:
+ *   [0] input checks + aggregate demand (K1)   [1] placement, Algorithm 1 (K2)   [2] projection (K3)
+ *   [3] row count + length-only seed (runs beside [0]-[2] on a side stream)
+ *   [4] seed evaluation and tables in rp_pack_rows   [5] validation + rescoring of the incumbent. */
+int rp_debug_set_stage_timing(int on);
+int rp_debug_stage_times(rp_ctx *ctx, double *ms);
 /* Per-level traces (RP_DUMP_TRACE_*) are recorded by rp_anneal calls made after
  * rp_debug_set_trace(ctx, 1); off by default (the copies cost a few microseconds per level). */
 int rp_debug_set_trace(rp_ctx *ctx, int on);

@@ -24,7 +24,7 @@ RP_OK = 0
 
 EXPORTS = ("rp_window_load", "rp_place_experts", "rp_pack_rows", "rp_seed_population", "rp_pair_population", "rp_select_population", "rp_eval_population", "rp_eval_layouts_noalloc", "rp_diagnostics", "rp_anneal",
            "rp_best", "rp_destroy", "rp_release_cached_memory", "rp_strerror", "rp_last_cuda_error", "rp_debug_dump",
-           "rp_debug_set_trace", "rp_debug_set_knob",
+           "rp_debug_set_trace", "rp_debug_set_knob", "rp_debug_set_stage_timing", "rp_debug_stage_times",
            "rp_debug_nl2", "rp_debug_exp2neg", "rp_debug_philox", "rp_debug_launch_count")
 
 
@@ -52,7 +52,8 @@ class rp_anneal_params(C.Structure):
 class rp_anneal_stats(C.Structure):
     _fields_ = [("proposed", C.c_int64), ("feasible", C.c_int64), ("accepted", C.c_int64),
                 ("improved", C.c_int64), ("ms_chains", C.c_double),
-                ("move_bytes", C.c_int64), ("gather_bytes", C.c_int64), ("kernel_launches", C.c_int64)]
+                ("move_bytes", C.c_int64), ("gather_bytes", C.c_int64), ("staging_bytes", C.c_int64),
+                ("kernel_launches", C.c_int64)]
 
 
 class rp_diag(C.Structure):
@@ -91,6 +92,8 @@ def lib():
         L.rp_debug_dump.argtypes = [C.c_void_p, C.c_int, C.c_int32, C.c_void_p, C.c_int64]
         L.rp_debug_set_trace.argtypes = [C.c_void_p, C.c_int]
         L.rp_debug_set_knob.argtypes = [C.c_void_p, C.c_int, C.c_int64]
+        L.rp_debug_set_stage_timing.argtypes = [C.c_int]
+        L.rp_debug_stage_times.argtypes = [C.c_void_p, C.c_void_p]
         L.rp_debug_nl2.argtypes = [C.c_void_p, C.c_void_p, C.c_int64]
         L.rp_debug_exp2neg.argtypes = [C.c_void_p, C.c_void_p, C.c_int64]
         L.rp_debug_philox.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64]
@@ -272,6 +275,20 @@ DUMP = dict(LAGG=1, Q=2, SEED_LAYOUT=3, POPULATION=4, W=5, CELL_T=6, CELL_Q=7, C
 
 def rp_debug_set_trace(ctx: Context, on: bool = True):
     _check(lib().rp_debug_set_trace(ctx.handle, int(on)), "rp_debug_set_trace")
+
+
+STAGES = ("check_reduce", "placement", "projection", "pack_rows", "seed_eval", "best_check")
+
+
+def rp_debug_set_stage_timing(on: bool = True):
+    _check(lib().rp_debug_set_stage_timing(int(on)), "rp_debug_set_stage_timing")
+
+
+def rp_debug_stage_times(ctx: Context) -> dict:
+    """Device milliseconds of the front-end stages of this context (None where a stage has not run)."""
+    ms = np.zeros(6, np.float64)
+    _check(lib().rp_debug_stage_times(ctx.handle, _ptr(ms)), "rp_debug_stage_times")
+    return {k: (float(v) if v >= 0 else None) for k, v in zip(STAGES, ms)}
 
 
 KNOB = dict(BARRIER_WORKSPACE=1, WAIT_POLLS=2, STALL_ONE_CHAIN=3)

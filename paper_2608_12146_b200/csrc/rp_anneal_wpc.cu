@@ -157,8 +157,12 @@ k_anneal_wpc(const AnnealArgs A)
     // ---- prologue: adopt the ancestor's terminal state -------------------------------
     if (!chain->failed) {
         const bool landed = rp_chain_load<NT, WS>(A, src, j, sm_blob, sm_static, Wsm, mbar, tid, src_cell, dst_cell);
-        if (tid == 0 && src_cell != dst_cell)              // bytes of the W gather (counted here: off the level's tail)
-            atomicAdd((u64 *)&A.counters[5], (u64)2 * dm.RG * dm.LP * 4);
+        // Bytes of the rank-load gather (counted here: off the level's tail): a copy made because
+        // resampling replaced this member by another one's state.  With the rank loads on chip
+        // every member's are staged in and out anyway; a member that kept its own state counts
+        // as staging, not as gather.
+        if (tid == 0 && src_cell != dst_cell)
+            atomicAdd((u64 *)&A.counters[(WS && src == j) ? 6 : 5], (u64)2 * dm.RG * dm.LP * 4);
         if (!landed) chain->failed = 1;
     }
     __syncthreads();

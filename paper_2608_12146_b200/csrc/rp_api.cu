@@ -122,6 +122,16 @@ static void side_give(RpSide *s)
 }
 
 
+// Optional stage timing: one flag for the process (a context only exists once rp_window_load has
+// already queued the front end), events per context.
+static int g_stage_timing = 0;
+static void stage_mark(rp_ctx *c, int which, cudaStream_t stream)
+{
+    if (!c->ev_stage[0]) return;
+    if (cudaEventRecord(c->ev_stage[which], stream) == cudaSuccess) c->ev_recorded |= 1u << which;
+    else cudaGetLastError();
+}
+
 static bool is_device_ptr(const void *p)
 {
     cudaPointerAttributes at;
@@ -176,6 +186,7 @@ extern "C" void rp_destroy(rp_ctx *c)
     free_population(c); free_trace(c); free_eval(c);
     dev_free(c, c->own_t); dev_free(c, c->own_a); dev_free(c, c->d_load_slab); dev_free(c, c->d_static);
     pin_give(c->h_pin);
+    for (int x = 0; x < RP_STAGE_EVENTS; ++x) if (c->ev_stage[x]) cudaEventDestroy(c->ev_stage[x]);
     side_give((RpSide *)c->side);
     free(c->h_levels);
     free(c);
@@ -286,7 +297,9 @@ static int window_load_impl(rp_ctx *c, const rp_config *cfg, const int32_t *leng
         // put in flight before the rest of the set-up
         if (cudaMemsetAsync(c->d_counters, 0, sizeof(i64) * 8, c->stream) != cudaSuccess) { st = RP_ERR_CUDA; break; }
         if ((st = reset_status(c)) != RP_OK) break;
+        stage_mark(c, RP_EV_K1_0, c->stream);
         if ((st = rp_launch_check_reduce(c)) != RP_OK) break;
+        stage_mark(c, RP_EV_K1_1, c->stream);
         // the EDP tables: one copy (pageable source: staged before the call returns)
         int *tab = (int *)malloc(sizeof(int) * n_tab);
         memcpy(tab, edp, sizeof(int) * D);
@@ -308,11 +321,17 @@ static int window_load_impl(rp_ctx *c, const rp_config *cfg, const int32_t *leng
     bool forked = false;
     if (side && cudaEventRecord(side->fork, c->stream) == cudaSuccess &&
         cudaStreamWaitEvent(side->stream, side->fork, 0) == cudaSuccess) {
+        stage_mark(c, RP_EV_PACK_0, side->stream);
         c->eager_pack = (rp_launch_pack_on(c, side->stream) == RP_OK);
+        stage_mark(c, RP_EV_PACK_1, side->stream);
         forked = (cudaEventRecord(side->join, side->stream) == cudaSuccess);
         if (!forked) { cudaStreamSynchronize(side->stream); c->eager_pack = 0; }
     }
-    c->eager_place = (rp_launch_lpt(c) == RP_OK && rp_launch_project(c) == RP_OK);
+    stage_mark(c, RP_EV_K2_0, c->stream);
+    c->eager_place = (rp_launch_lpt(c) == RP_OK);
+    stage_mark(c, RP_EV_K2_1, c->stream);
+    c->eager_place = c->eager_place && (rp_launch_project(c) == RP_OK);
+    stage_mark(c, RP_EV_K3_1, c->stream);
     if (forked) RP_CUDA(cudaStreamWaitEvent(c->stream, side->join, 0));
     else c->eager_pack = (rp_launch_pack(c, 0) == RP_OK);
     if (c->eager_pack)
@@ -359,6 +378,9 @@ extern "C" int rp_window_load(rp_ctx **out, const rp_config *cfg, const int32_t 
     c->h_pin = (i64 *)pin_take();
     if (!c->h_pin) { free(c); return RP_ERR_CUDA; }
     c->side = side_take(c->device);          // optional: without it everything runs on the one stream
+    if (g_stage_timing)
+        for (int x = 0; x < RP_STAGE_EVENTS; ++x)
+            if (cudaEventCreate(&c->ev_stage[x]) != cudaSuccess) { cudaGetLastError(); c->ev_stage[0] = nullptr; break; }
     int st = window_load_impl(c, cfg, lengths, demand);
     if (st != RP_OK) { rp_destroy(c); return st; }
     c->stage = 1;
@@ -485,6 +507,7 @@ extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
     // slots descend from slot 0
     dev_free(c, c->d_static); c->d_static = nullptr;
     RP_TRY(dev_alloc(c, &c->d_static, (size_t)c->sl.bytes));
+    stage_mark(c, RP_EV_SEED_0, c->stream);
     RP_TRY(rp_launch_build_static(c));
     RP_TRY(ensure_eval_scratch(c, 1, false));
     RP_TRY(rp_launch_cells_from_layouts(c, c->d_seed_layout, 1, c->d_eval_cells));
@@ -497,6 +520,7 @@ extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
         ++g_rp_launches;
         RP_CUDA(cudaGetLastError());
     }
+    stage_mark(c, RP_EV_SEED_1, c->stream);
     if (n_rows) *n_rows = c->Rstar;
     if (certified) *certified = c->certified;
     c->stage = 3;
@@ -812,7 +836,7 @@ extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *
     }
     if (stats) {
         stats->proposed = cn[0]; stats->feasible = cn[1]; stats->accepted = cn[2]; stats->improved = cn[3];
-        stats->move_bytes = cn[4]; stats->gather_bytes = cn[5];
+        stats->move_bytes = cn[4]; stats->gather_bytes = cn[5]; stats->staging_bytes = cn[6];
         stats->kernel_launches = (int64_t)NL;
         stats->ms_chains = ms_chains;
     }
@@ -826,10 +850,12 @@ extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *
 // incumbent; the three score tuples the verdict needs are queued into the pinned block.
 static int launch_best_check(rp_ctx *c)
 {
+    stage_mark(c, RP_EV_BEST_0, c->stream);
     RP_TRY(rp_launch_validate(c));
     RP_TRY(ensure_eval_scratch(c, 1, false));
     RP_TRY(rp_launch_cells_from_layouts(c, c->d_inc_layout, 1, c->d_eval_cells));
     RP_TRY(rp_launch_eval(c, c->d_eval_cells, 1, nullptr, nullptr, c->d_best_score, c->d_best_f64));
+    stage_mark(c, RP_EV_BEST_1, c->stream);
     RP_CUDA(cudaMemcpyAsync(c->h_pin + 16, c->d_inc_score, sizeof(i64) * 3, cudaMemcpyDeviceToHost, c->stream));
     RP_CUDA(cudaMemcpyAsync(c->h_pin + 19, c->d_best_score, sizeof(i64) * 3, cudaMemcpyDeviceToHost, c->stream));
     RP_CUDA(cudaMemcpyAsync(c->h_pin + 22, c->d_seed_score, sizeof(i64) * 3, cudaMemcpyDeviceToHost, c->stream));
@@ -883,6 +909,27 @@ __global__ void k_cell_stats(const unsigned short *__restrict__ cells, const int
         atomicAdd((u64 *)&Q[c], (u64)t[i] * (u64)t[i]);
         atomicAdd(&cnt[c], 1);
     }
+}
+
+extern "C" int rp_debug_set_stage_timing(int on) { g_stage_timing = on ? 1 : 0; return RP_OK; }
+
+extern "C" int rp_debug_stage_times(rp_ctx *c, double *ms)
+{
+    if (!c || !ms) return RP_ERR_ARG;
+    if (!c->ev_stage[0]) return RP_ERR_STATE;
+    RP_CUDA(cudaStreamSynchronize(c->stream));
+    static const int pairs[6][2] = { { RP_EV_K1_0, RP_EV_K1_1 }, { RP_EV_K2_0, RP_EV_K2_1 }, { RP_EV_K2_1, RP_EV_K3_1 },
+                                     { RP_EV_PACK_0, RP_EV_PACK_1 }, { RP_EV_SEED_0, RP_EV_SEED_1 }, { RP_EV_BEST_0, RP_EV_BEST_1 } };
+    for (int x = 0; x < 6; ++x) {
+        ms[x] = -1.0;
+        const unsigned need = (1u << pairs[x][0]) | (1u << pairs[x][1]);
+        if ((c->ev_recorded & need) != need) continue;
+        float t = 0.f;
+        if (cudaEventSynchronize(c->ev_stage[pairs[x][1]]) == cudaSuccess &&
+            cudaEventElapsedTime(&t, c->ev_stage[pairs[x][0]], c->ev_stage[pairs[x][1]]) == cudaSuccess) ms[x] = t;
+        else cudaGetLastError();
+    }
+    return RP_OK;
 }
 
 extern "C" int rp_debug_set_knob(rp_ctx *c, int knob, int64_t value)

@@ -84,6 +84,12 @@ struct RpPopBuf {
     char *blob;                // [P_pop][blob.bytes]
 };
 
+// Events of the optional stage timing: begin/end of the check+reduce, placement, projection and
+// packing kernels (rp_window_load), of the seed's evaluation and tables (rp_pack_rows) and of the
+// validation + rescoring of the incumbent.
+enum { RP_EV_K1_0, RP_EV_K1_1, RP_EV_K2_0, RP_EV_K2_1, RP_EV_K3_1, RP_EV_PACK_0, RP_EV_PACK_1, RP_EV_SEED_0, RP_EV_SEED_1,
+       RP_EV_BEST_0, RP_EV_BEST_1, RP_STAGE_EVENTS };
+
 struct rp_ctx {
     int device;
     cudaStream_t stream;
@@ -154,6 +160,8 @@ struct rp_ctx {
     int trace_levels;
     int trace_on;              // keep per-level traces (inspection hook; off by default)
     int knob_le_ws_cap, knob_wait_polls, knob_stall;   // inspection hooks (rp_debug_set_knob); 0 = off
+    cudaEvent_t ev_stage[RP_STAGE_EVENTS];             // stage timing (rp_debug_set_stage_timing); null when off
+    unsigned ev_recorded;                              // bit x: ev_stage[x] has been recorded
     i64 *d_tr_term, *d_tr_best, *d_tr_inc;
     int *d_tr_best_step, *d_tr_anc;
     u64 *d_tr_digest;

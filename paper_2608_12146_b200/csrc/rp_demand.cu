@@ -55,10 +55,120 @@ k_check_reduce(const int *__restrict__ a, const int *__restrict__ t, RpDims dm, 
     if (warp == 0 && lane == 0 && tsum > 0) atomicAdd((u64 *)t_sum, (u64)tsum);
 }
 
+// The same pass for rows that are whole multiples of 128 experts (512 bytes) on 16-byte aligned
+// tensors.  One CTA owns one layer and a range of samples: its warps take the samples round
+// robin, every lane reads 16 bytes of a row, the loads of several rows are issued before any is
+// consumed, and a row is summed exactly with two 32-bit warp reductions (low and high 16 bits of
+// the counts, neither of which can overflow for E <= 1024; a count outside [0, k*t_i] already
+// fails the row).  The warps' column sums meet in shared memory, so the CTA issues one atomic
+// per expert.
+#define K1V_ROWS_MIN 2
+template <int NQ>               // 16-byte pieces per lane and row = E / 128
+__global__ void __launch_bounds__(K1_WARPS * 32)
+k_check_reduce_vec(const int4 *__restrict__ a, const int *__restrict__ t, RpDims dm, int chunk,
+                   i64 *__restrict__ Lagg, int *__restrict__ status, i64 *__restrict__ t_sum)
+{
+    constexpr int K1V_ROWS = NQ == 1 ? 8 : (NQ == 2 ? 4 : K1V_ROWS_MIN);      // 128 bytes per lane in flight
+    extern __shared__ __align__(16) i64 colsum[];          // [K1_WARPS][E]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int l = blockIdx.x % dm.L;
+    const int i0 = (blockIdx.x / dm.L) * chunk;
+    const int i1 = min(dm.N, i0 + chunk);
+    const size_t row4 = (size_t)dm.E >> 2;            // 16-byte pieces per row
+    i64 tsum = 0;
+    bool bad = false;
+    i64 acc[NQ][4];
+#pragma unroll
+    for (int c = 0; c < NQ; ++c) { acc[c][0] = 0; acc[c][1] = 0; acc[c][2] = 0; acc[c][3] = 0; }
+    for (int ib = i0 + warp; ib < i1; ib += K1_WARPS * K1V_ROWS) {
+        int4 v[K1V_ROWS][NQ];
+        int ti[K1V_ROWS];
+#pragma unroll
+        for (int r = 0; r < K1V_ROWS; ++r) {
+            const int i = min(ib + r * K1_WARPS, i1 - 1);              // past the end: the last row again, not counted
+            const int4 *row = a + ((size_t)i * dm.L + l) * row4;
+#pragma unroll
+            for (int c = 0; c < NQ; ++c) v[r][c] = __ldcs(row + c * 32 + lane);     // read once: streaming
+            ti[r] = __ldg(t + i);
+        }
+#pragma unroll
+        for (int r = 0; r < K1V_ROWS; ++r) {
+            if (ib + r * K1_WARPS >= i1) break;
+            const i64 kt = (i64)dm.k * ti[r];
+            const unsigned ktu = kt < 0x7fffffffll ? (kt < 0 ? 0u : (unsigned)kt) : 0x7fffffffu;   // k*C < 2^31 for any window that loads
+            tsum += ti[r];
+            unsigned part = 0;                         // this lane's share of the row sum, at most k*t once nothing is out of range
+            bool out = false;
+#pragma unroll
+            for (int c = 0; c < NQ; ++c) {
+                const unsigned x0 = (unsigned)v[r][c].x, x1 = (unsigned)v[r][c].y, x2 = (unsigned)v[r][c].z, x3 = (unsigned)v[r][c].w;
+                // negative counts are huge as unsigned: one comparison covers both ends of [0, k*t]
+                out |= (x0 > ktu) | (x1 > ktu) | (x2 > ktu) | (x3 > ktu);
+                const unsigned s01 = x0 + x1, s23 = x2 + x3;               // each term below 2^31: no wrap
+                out |= (s01 > ktu) | (s23 > ktu);
+                const unsigned s4 = s01 + s23;
+                out |= (s4 > ktu);
+                part += out ? 0u : s4;
+                out |= (part > ktu);
+                acc[c][0] += v[r][c].x; acc[c][1] += v[r][c].y; acc[c][2] += v[r][c].z; acc[c][3] += v[r][c].w;
+            }
+            const unsigned slo = __reduce_add_sync(0xffffffffu, out ? 0u : (part & 0xffffu));
+            const unsigned shi = __reduce_add_sync(0xffffffffu, out ? 0u : (part >> 16));
+            const i64 rs = (i64)slo + ((i64)shi << 16);
+            bad |= __any_sync(0xffffffffu, out) || rs != kt || ti[r] < 1 || ti[r] > dm.C;
+        }
+    }
+#pragma unroll
+    for (int c = 0; c < NQ; ++c)
+#pragma unroll
+        for (int u = 0; u < 4; ++u) colsum[(size_t)warp * dm.E + (c * 32 + lane) * 4 + u] = acc[c][u];
+    __syncthreads();
+    for (int e = threadIdx.x; e < dm.E; e += K1_WARPS * 32) {
+        i64 sum = 0;
+#pragma unroll
+        for (int w = 0; w < K1_WARPS; ++w) sum += colsum[(size_t)w * dm.E + e];
+        if (sum) atomicAdd((u64 *)&Lagg[(size_t)l * dm.E + e], (u64)sum);
+    }
+    if (bad && lane == 0) atomicExch(&status[RP_SW_BAD_SAMPLE], 1);
+    if (l == 0 && lane == 0 && tsum > 0) atomicAdd((u64 *)t_sum, (u64)tsum);      // tokens of this warp's samples, once
+}
+
 int rp_launch_check_reduce(rp_ctx *c)
 {
     const RpDims &dm = c->dm;
     RP_CUDA(cudaMemsetAsync(c->d_Lagg, 0, sizeof(i64) * dm.L * dm.E, c->stream));
+    if (dm.E % 128 == 0 && dm.E <= 1024 && ((size_t)c->d_a & 15) == 0) {
+        // one CTA per (layer, range of samples): four CTAs per SM (one wave), at least 64 samples each
+        int splits = (4 * 148) / dm.L;
+        splits = splits < 1 ? 1 : splits;
+        int chunk = (dm.N + splits - 1) / splits;
+        chunk = chunk < K1_WARPS * 8 ? K1_WARPS * 8 : chunk;
+        splits = (dm.N + chunk - 1) / chunk;
+        const int grid = splits * dm.L;
+        const size_t smem = sizeof(i64) * K1_WARPS * dm.E;
+        const int4 *a4 = (const int4 *)c->d_a;
+#define K1V_CASE(NQ_)                                                                              \
+        do {                                                                                       \
+            if (smem > 32 * 1024)                                                                  \
+                RP_CUDA(cudaFuncSetAttribute(k_check_reduce_vec<NQ_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+            k_check_reduce_vec<NQ_><<<grid, K1_WARPS * 32, smem, c->stream>>>(a4, c->d_t, dm, chunk, c->d_Lagg, \
+                                                                             c->d_status, c->d_counters + 7); \
+        } while (0)
+        switch (dm.E / 128) {
+            case 1: K1V_CASE(1); break;
+            case 2: K1V_CASE(2); break;
+            case 3: K1V_CASE(3); break;
+            case 4: K1V_CASE(4); break;
+            case 5: K1V_CASE(5); break;
+            case 6: K1V_CASE(6); break;
+            case 7: K1V_CASE(7); break;
+            default: K1V_CASE(8); break;
+        }
+#undef K1V_CASE
+        ++g_rp_launches;
+        RP_CUDA(cudaGetLastError());
+        return RP_OK;
+    }
     // enough CTAs to fill the GPU on small windows, up to 32 samples per CTA on large ones
     int chunk = (dm.N + 2 * 148 - 1) / (2 * 148);
     chunk = chunk < 4 ? 4 : (chunk > K1_CHUNK_MAX ? K1_CHUNK_MAX : chunk);
@@ -222,9 +332,100 @@ k_project(const int *__restrict__ a, const int *__restrict__ inv, RpDims dm, int
     }
 }
 
+// The same projection for rows that are whole multiples of 128 experts on 16-byte aligned tensors
+// with at most 32 ranks.  One CTA owns one layer and a range of samples, so the layer's inverse
+// placement sits in registers (lane (p, part) keeps the PER slots it sums) and no table has to be
+// staged.  A warp stages K3V_ROWS rows at a time with 16-byte loads, all issued before any is
+// stored; the gather and the coalesced store of the P ranks follow row by row.
+#define K3V_ROWS 4
+template <int NQ, int PER>
+__global__ void __launch_bounds__(K3_WARPS * 32)
+k_project_vec(const int4 *__restrict__ a, const int *__restrict__ inv, RpDims dm, int chunk, int *__restrict__ q)
+{
+    extern __shared__ __align__(16) int smi[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int *rows_s = smi + (size_t)warp * K3V_ROWS * dm.E;
+    const int l = blockIdx.x % dm.L;
+    const int i0 = (blockIdx.x / dm.L) * chunk;
+    const int i1 = min(dm.N, i0 + chunk);
+    int parts = 1;
+    while (parts * 2 * dm.P <= 32) parts *= 2;
+    const int p = lane / parts, part = lane % parts;
+    int iv[PER];
+#pragma unroll
+    for (int x = 0; x < PER; ++x) iv[x] = (p < dm.P) ? __ldg(inv + (size_t)l * dm.E + p * dm.H + part + x * parts) : 0;
+    const size_t row4 = (size_t)dm.E >> 2;
+    for (int ib = i0 + warp; ib < i1; ib += K3_WARPS * K3V_ROWS) {
+        int4 v[K3V_ROWS][NQ];
+#pragma unroll
+        for (int u = 0; u < K3V_ROWS; ++u) {
+            const int i = min(ib + u * K3_WARPS, i1 - 1);
+#pragma unroll
+            for (int c = 0; c < NQ; ++c) v[u][c] = __ldcs(a + ((size_t)i * dm.L + l) * row4 + c * 32 + lane);
+        }
+#pragma unroll
+        for (int u = 0; u < K3V_ROWS; ++u)
+#pragma unroll
+            for (int c = 0; c < NQ; ++c) ((int4 *)(rows_s + (size_t)u * dm.E))[c * 32 + lane] = v[u][c];
+        __syncwarp();
+#pragma unroll
+        for (int u = 0; u < K3V_ROWS; ++u) {
+            const int i = ib + u * K3_WARPS;
+            if (i >= i1) break;
+            const int *row_s = rows_s + (size_t)u * dm.E;
+            int s = 0;
+#pragma unroll
+            for (int x = 0; x < PER; ++x) s += row_s[iv[x]];
+            for (int o = parts >> 1; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+            if (p < dm.P && part == 0) __stcs(q + ((size_t)i * dm.L + l) * dm.P + p, s);
+        }
+        __syncwarp();
+    }
+}
+
 int rp_launch_project(rp_ctx *c)
 {
     const RpDims &dm = c->dm;
+    {
+        int parts = 1;
+        while (parts * 2 * dm.P <= 32) parts *= 2;
+        const int per = dm.H / parts;
+        const bool per_ok = dm.H % parts == 0 && (per == 1 || per == 2 || per == 4 || per == 8 || per == 16);
+        const size_t smem_v = (size_t)K3_WARPS * K3V_ROWS * dm.E * sizeof(int);
+        if (dm.E % 128 == 0 && dm.E <= 512 && dm.P <= 32 && per_ok && ((size_t)c->d_a & 15) == 0) {
+            // one CTA per (layer, range of samples): about eight CTAs per SM, at least 32 samples each
+            int splits = (8 * 148 + dm.L - 1) / dm.L;
+            int chunk = (dm.N + splits - 1) / splits;
+            chunk = chunk < K3_WARPS * K3V_ROWS ? K3_WARPS * K3V_ROWS : chunk;
+            splits = (dm.N + chunk - 1) / chunk;
+            const int grid = splits * dm.L;
+#define K3V_LAUNCH(NQ_, PER_)                                                                                  \
+            do {                                                                                               \
+                if (smem_v > 32 * 1024)                                                                        \
+                    RP_CUDA(cudaFuncSetAttribute(k_project_vec<NQ_, PER_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_v)); \
+                k_project_vec<NQ_, PER_><<<grid, K3_WARPS * 32, smem_v, c->stream>>>((const int4 *)c->d_a, c->d_inv, dm, chunk, c->d_q); \
+            } while (0)
+#define K3V_CASE(NQ_)                                                                                          \
+            switch (per) {                                                                                     \
+                case 1: K3V_LAUNCH(NQ_, 1); break;                                                             \
+                case 2: K3V_LAUNCH(NQ_, 2); break;                                                             \
+                case 4: K3V_LAUNCH(NQ_, 4); break;                                                             \
+                case 8: K3V_LAUNCH(NQ_, 8); break;                                                             \
+                default: K3V_LAUNCH(NQ_, 16); break;                                                           \
+            }
+            switch (dm.E / 128) {
+                case 1: K3V_CASE(1); break;
+                case 2: K3V_CASE(2); break;
+                case 3: K3V_CASE(3); break;
+                default: K3V_CASE(4); break;
+            }
+#undef K3V_CASE
+#undef K3V_LAUNCH
+            ++g_rp_launches;
+            RP_CUDA(cudaGetLastError());
+            return RP_OK;
+        }
+    }
     size_t smem = (size_t)K3_WARPS * dm.E * sizeof(int);
     if ((size_t)(K3_WARPS + dm.L) * dm.E * sizeof(int) <= 96 * 1024) smem += (size_t)dm.L * dm.E * sizeof(int);
     if (smem > 32 * 1024)

@@ -720,6 +720,48 @@ def test_bad_inputs_are_host_side_errors():
     rp.rp_destroy(ctx)
 
 
+@pytest.mark.parametrize("E,P,N,L", [(128, 32, 70, 5), (256, 16, 37, 9), (384, 4, 33, 2), (1024, 8, 19, 3), (128, 1, 41, 3),
+                                     (128, 8, 100, 2), (512, 32, 35, 4), (256, 32, 300, 3), (128, 64, 50, 2)])
+def test_wide_expert_rows_front_end(E, P, N, L):
+    """Rows of whole multiples of 128 experts take the 16-byte-load forms of the check + reduce and
+    projection kernels (ragged sample counts: the last group of rows is partial): aggregate demand,
+    placement, rank demand and seed against the oracle, and every kind of bad input is still caught."""
+    w = make_window(custom_spec(f"rows{E}", N, L, E, 4, 4096, 2, P, 6, 100, data_seed=E + N))
+    s = w.spec
+    ref = oracle_front(w, None, 2)
+    for device_inputs in (False, True):
+        ctx = load(w, pop=6, min_rows=2, device_inputs=device_inputs)
+        check_front(w, ctx, ref)
+        check_eval(w, ctx, ref, None, n=2)
+        rp.rp_destroy(ctx)
+    kw = dict(top_k=s.top_k, token_cap=s.token_cap, dp_width=s.dp_width, ep_width=s.ep_width, pop_size=2)
+    for i, l, e in ((0, 0, 0), (N - 1, L - 1, E - 1), (N // 2, L // 2, 129 % E)):
+        bad = w.demand.copy()
+        bad[i, l, e] += 1                                   # row sum off by one
+        with pytest.raises(rp.RpError) as err:
+            rp.rp_window_load(w.lengths, bad, **kw)
+        assert err.value.status == -3
+        neg = w.demand.copy()                               # row sum right, one count negative
+        neg[i, l, e] -= neg[i, l, e] + 3
+        neg[i, l, (e + 5) % E] += w.demand[i, l, e] + 3
+        with pytest.raises(rp.RpError) as err:
+            rp.rp_window_load(w.lengths, neg, **kw)
+        assert err.value.status == -3
+        big = w.demand.copy()                               # sums right modulo 2^32, counts far out of range
+        big[i, l, e] += 2 ** 30
+        big[i, l, (e + 1) % E] += 2 ** 30
+        big[i, l, (e + 2) % E] += 2 ** 30
+        big[i, l, (e + 3) % E] += 2 ** 30
+        with pytest.raises(rp.RpError) as err:
+            rp.rp_window_load(w.lengths, big, **kw)
+        assert err.value.status == -3
+    long_ = w.lengths.copy()
+    long_[N - 1] = 0
+    with pytest.raises(rp.RpError) as err:
+        rp.rp_window_load(long_, w.demand, **kw)
+    assert err.value.status == -3
+
+
 def test_smallest_window_and_empty_moves():
     """N == D, one row, one sample per cell: every proposal is infeasible (same cell, or a
     relocation that would empty a cell, or a swap over the cap) or a legal swap."""
