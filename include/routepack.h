@@ -282,8 +282,12 @@ typedef enum {
  *   RP_KNOB_WAIT_POLLS: polls after which a chain's wait on its asynchronous copies gives up
  *     (default 2^22).
  *   RP_KNOB_STALL_ONE_CHAIN: chain 0 waits once more, after its copies have landed, on a barrier
- *     phase that nothing completes: the wait runs out and rp_anneal returns RP_ERR_TIMEOUT. */
-typedef enum { RP_KNOB_BARRIER_WORKSPACE = 1, RP_KNOB_WAIT_POLLS = 2, RP_KNOB_STALL_ONE_CHAIN = 3 } rp_knob;
+ *     phase that nothing completes: the wait runs out and rp_anneal returns RP_ERR_TIMEOUT.
+ *   RP_KNOB_RANK_LOAD_SLICES (set before rp_pack_rows): how windows with L*P > 512 keep the rank
+ *     loads of the population.  0 or 1 = shared slices with copy-on-write (the default), 2 = one
+ *     private cell per member, copied whole when resampling replaces the member. */
+typedef enum { RP_KNOB_BARRIER_WORKSPACE = 1, RP_KNOB_WAIT_POLLS = 2, RP_KNOB_STALL_ONE_CHAIN = 3,
+               RP_KNOB_RANK_LOAD_SLICES = 4 } rp_knob;
 int rp_debug_set_knob(rp_ctx *ctx, int knob, int64_t value);
 /* Device time of the stages that have no statistics struct of their own.  After
  * rp_debug_set_stage_timing(1) (process-wide; contexts loaded later record CUDA events around the

@@ -40,8 +40,8 @@ struct ChainB {                 // bookkeeping of the chain within this level
 // Cooperative chain kernel for bandwidth-bound windows (L*P > 512): all NT threads score one
 // candidate at a time (two L*P slices of W from global memory plus the moved samples' demand
 // rows, 16-byte loads); the leading warp rebuilds the score and decides.
-template <int NT>
-__global__ void __launch_bounds__(NT, 768 / NT)
+template <int NT, int MINB, bool SL>
+__global__ void __launch_bounds__(NT, MINB)
 k_anneal_level(const AnnealArgs A)
 {
     const RpDims &dm = A.dm;
@@ -59,6 +59,8 @@ k_anneal_level(const AnnealArgs A)
     ChainB *chain = (ChainB *)(recs + SPEC);
     u64 *mbar = (u64 *)(chain + 1);
     MoveS *mvs = (MoveS *)(mbar + 1);
+    int *spare = (int *)(mvs + SPEC);                       // [RG] slice mode: free slice set aside for each row-shard
+    unsigned char *own = (unsigned char *)(spare + (SL ? dm.RG : 0));   // [RG] this chain is the only holder of the row-shard's slice
 
     u64 *Q = (u64 *)(sm_blob + A.bl.off_Q);
     i64 *Esum = (i64 *)(sm_blob + A.bl.off_Esum);
@@ -69,6 +71,7 @@ k_anneal_level(const AnnealArgs A)
     int *T = (int *)(sm_blob + A.bl.off_T);
     int *cnt = (int *)(sm_blob + A.bl.off_cnt);
     unsigned short *cell_of = (unsigned short *)(sm_blob + A.bl.off_cell);
+    int *wtab = (int *)(sm_blob + (SL ? A.bl.off_wtab : 0));          // slice mode: row-shard -> slice of the pool
     const int *dpl = (const int *)(sm_static + A.sl.off_dpl);
     const int *dpo = (const int *)(sm_static + A.sl.off_dpo);
     const int *tt = A.sl.t_staged ? (const int *)(sm_static + A.sl.off_t) : A.t;
@@ -79,11 +82,14 @@ k_anneal_level(const AnnealArgs A)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int j = blockIdx.x;
-    const int src = A.anc[j];
+    // (clamped: after a level that gave up on a wait the table is stale, and the cell look-up below runs
+    // before this chain has seen the status word)
+    const int src = min(max(A.anc[j], 0), A.Ppop - 1);
     const bool identity_edp = (dm.G == dm.D);
-    const int dst_cell = A.wloc_dst[j];
-    const int src_cell = rp_src_cell(A, src, j);
+    const int dst_cell = SL ? 0 : A.wloc_dst[j];
+    const int src_cell = SL ? 0 : rp_src_cell(A, src, j);
     int *Wj = A.W + (size_t)dst_cell * wn;
+
     const bool vec = (dm.P >= 4) && (dm.P <= 128) && ((dm.P & (dm.P - 1)) == 0);
     const i64 aC = dm.asum * dm.C, bS = dm.bsum;
 
@@ -113,6 +119,18 @@ k_anneal_level(const AnnealArgs A)
     if (tid == 0) {
         chain->B[0] = Sc[0]; chain->B[1] = Sc[1]; chain->B[2] = Sc[2];
         chain->dig = 0; chain->best_step = 0; chain->best_nlog = 0; chain->nlog = 0;
+    }
+    if (SL) {
+        // A slice that only this member holds when the level starts is rewritten in place; a shared
+        // one is left at its first rewrite for this chain's spare slice of that row-shard (entry
+        // j*RG + rg of the free list, which holds at least RG slices per member).  Holder counts are
+        // only read here: nobody gains a slice during a level, and nobody who has left one reads it again.
+        const int n_free = A.wfree_head[1];
+        for (int rg = tid; rg < dm.RG; rg += NT) {
+            const bool mine = (__ldg(&A.wref[wtab[rg]]) == 1);
+            own[rg] = mine ? 1 : 0;
+            spare[rg] = mine ? -1 : ((size_t)j * dm.RG + rg < (size_t)n_free ? __ldg(&A.wfree[(size_t)j * dm.RG + rg]) : -1);
+        }
     }
     __syncthreads();
 
@@ -150,7 +168,8 @@ k_anneal_level(const AnnealArgs A)
                 if (touchW) {
                     const int *qi = A.q + (size_t)m.i * dm.LP;
                     const int *q2 = swap ? A.q + (size_t)m.i2 * dm.LP : nullptr;
-                    const int *w1 = Wj + (size_t)rg1 * dm.LP, *w2 = Wj + (size_t)rg2 * dm.LP;
+                    const int *w1 = SL ? A.W + (size_t)wtab[rg1] * dm.LP : Wj + (size_t)rg1 * dm.LP;
+                    const int *w2 = SL ? A.W + (size_t)wtab[rg2] * dm.LP : Wj + (size_t)rg2 * dm.LP;
                     const int P = dm.P, LP = dm.LP;
                     if (vec) {
                         RpSliceRegs<2> regs;
@@ -257,6 +276,18 @@ k_anneal_level(const AnnealArgs A)
                         if (touchW) n_bytes += (i64)((swap ? 4 : 3) + (acc ? 2 : 0)) * dm.LP * 4;
                         if (acc) {
                             ++n_acc;
+                            if (SL && touchW) {
+                                // Where the two rewritten slices go: in place when the slice is this chain's
+                                // own, else to the spare slice of that row-shard, which then is its own.
+                                const int both[2] = { rg1, rg2 };
+                                for (int x = 0; x < 2; ++x) {
+                                    const int rg = both[x];
+                                    if (own[rg]) continue;
+                                    if (spare[rg] >= 0) wtab[rg] = spare[rg];
+                                    else atomicExch(&A.status[RP_SW_POOL], 1);           // cannot happen: the list has a spare per row-shard
+                                    own[rg] = 1;
+                                }
+                            }
                             const int k = kb + ls;
                             cell_of[m.i] = (unsigned short)c2;
                             if (swap) cell_of[m.i2] = (unsigned short)c1;
@@ -291,7 +322,8 @@ k_anneal_level(const AnnealArgs A)
                 const int acc = chain->accept;
                 if (acc) {
                     if (touchW) {
-                        int *w1 = Wj + (size_t)rg1 * dm.LP, *w2 = Wj + (size_t)rg2 * dm.LP;
+                        int *w1 = SL ? A.W + (size_t)wtab[rg1] * dm.LP : Wj + (size_t)rg1 * dm.LP;
+                        int *w2 = SL ? A.W + (size_t)wtab[rg2] * dm.LP : Wj + (size_t)rg2 * dm.LP;
                         if (vec) {
                             for (int c = tid; c < (dm.LP >> 2); c += NT) {
                                 ((int4 *)w1)[c] = ((const int4 *)scratch)[c];
@@ -333,6 +365,92 @@ int rp_launch_anneal_wpc(rp_ctx *c, const AnnealArgs &A);
 
 static bool use_wpc(const RpDims &dm) { return dm.LP <= 512; }
 bool rp_uses_wpc(const RpDims &dm) { return use_wpc(dm); }
+// Rank loads in global memory are kept as shared slices (see AnnealArgs); the cooperative kernel
+// can also keep one private cell per member (inspection hook; slower wherever resampling replaces
+// many members, never faster).  Decided when the row count is known and kept in the dimensions.
+bool rp_uses_slices(const RpDims &dm) { return dm.slices != 0; }
+int rp_slice_mode(const RpDims &dm, int knob)
+{
+    if (use_wpc(dm)) return 0;
+    return knob == 2 ? 0 : 1;
+}
+
+// Blob and table layouts once the row count is known.  Whether the warp-per-candidate kernel keeps
+// the rank loads on chip depends on the blob's size, and the blob carries the slice table only when
+// they stay in global memory: lay out without the table first, then again if it is needed.
+void rp_decide_layouts(rp_ctx *c)
+{
+    RpDims &dm = c->dm;
+    dm.slices = 0;
+    rp_make_layouts(dm, &c->bl, &c->sl);
+    if (use_wpc(dm)) {
+        int ws = 0;
+        rp_wpc_smem_bytes(dm, c->bl, c->sl, rp_wpc_warps(c->Ppop), &ws);
+        dm.slices = ws ? 0 : 1;
+    } else {
+        dm.slices = rp_slice_mode(dm, c->knob_slices);
+    }
+    if (dm.slices) rp_make_layouts(dm, &c->bl, &c->sl);
+}
+
+// Slice bookkeeping between two levels: holders of every slice among the members that start the
+// next level (member m starts from the terminal table of anc[m]), then the list of free slices,
+// ascending within every block of SLICE_BLOCK slices and block after block in the order the blocks
+// arrive (so that a member's RG spares are a nearly contiguous piece of the pool).  The second
+// kernel leaves the counts at zero for the next round.
+#define SLICE_BLOCK 1024
+// After a level that gave up on a wait the ancestors were never written: both kernels then leave
+// everything as it is (the chains of the remaining levels do nothing either).  Indices are
+// checked before they are used, so that a broken table can only raise the status word.
+__global__ void k_slice_holders(const char *__restrict__ blobs, RpBlob bl, const int *__restrict__ anc, int RG, int P, int ns,
+                                int *__restrict__ ref, int *__restrict__ head, int *__restrict__ status)
+{
+    if (__ldcg(&status[RP_SW_TIMEOUT])) return;
+    const int a = anc[blockIdx.x];
+    if ((unsigned)a >= (unsigned)P) { if (threadIdx.x == 0) atomicExch(&status[RP_SW_POOL], 1); return; }
+    const int *tab = (const int *)(blobs + (size_t)a * bl.bytes + bl.off_wtab);
+    for (int rg = threadIdx.x; rg < RG; rg += blockDim.x) {
+        const int s = tab[rg];
+        if ((unsigned)s < (unsigned)ns) atomicAdd(&ref[s], 1);
+        else atomicExch(&status[RP_SW_POOL], 1);
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) { head[0] = 0; head[1] = 0; }
+}
+__global__ void __launch_bounds__(SLICE_BLOCK)
+k_slice_free_list(int *__restrict__ ref, int *__restrict__ holders, int n, int *__restrict__ list, int *__restrict__ head,
+                  const int *__restrict__ status)
+{
+    __shared__ int wsum[32];
+    __shared__ int base;
+    if (__ldcg(&status[RP_SW_TIMEOUT])) return;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int s = blockIdx.x * SLICE_BLOCK + threadIdx.x;
+    const int r = s < n ? ref[s] : 1;
+    if (s < n) { holders[s] = r; ref[s] = 0; }
+    const bool is_free = (r == 0);
+    const unsigned m = __ballot_sync(0xffffffffu, is_free);
+    if (lane == 0) wsum[warp] = __popc(m);
+    __syncthreads();
+    if (warp == 0) {
+        int w = wsum[lane];
+        for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, w, o); if (lane >= o) w += y; }
+        wsum[lane] = w;
+        if (lane == 31) base = w ? atomicAdd(&head[1], w) : 0;
+    }
+    __syncthreads();
+    if (is_free) list[base + (warp ? wsum[warp - 1] : 0) + __popc(m & ((1u << lane) - 1))] = s;
+}
+
+int rp_launch_slice_gc(rp_ctx *c)
+{
+    const int ns = 2 * c->Ppop * c->dm.RG, nb = (ns + SLICE_BLOCK - 1) / SLICE_BLOCK;
+    k_slice_holders<<<c->Ppop, 128, 0, c->stream>>>(c->buf[c->cur].blob, c->bl, c->d_anc, c->dm.RG, c->Ppop, ns, c->d_wcount,
+                                                    c->d_wfree_head, c->d_status);
+    k_slice_free_list<<<nb, SLICE_BLOCK, 0, c->stream>>>(c->d_wcount, c->d_wref, ns, c->d_wfree, c->d_wfree_head, c->d_status);
+    g_rp_launches += 2;
+    RP_CUDA(cudaGetLastError());
+    return RP_OK;
+}
 
 int rp_anneal_smem_bytes(const rp_ctx *c, int *threads, size_t *bytes)
 {
@@ -347,7 +465,7 @@ int rp_anneal_smem_bytes(const rp_ctx *c, int *threads, size_t *bytes)
     const int nt = 128;
     const size_t slice_pad = ((size_t)dm.LP + 3) & ~(size_t)3;
     size_t b = (size_t)c->bl.bytes + c->sl.bytes + sizeof(int) * 2 * slice_pad + sizeof(i64) * (3 * (size_t)dm.K + 2 * (nt / 32)) +
-               sizeof(StepRec) * SPEC + sizeof(ChainB) + sizeof(u64) + sizeof(MoveS) * SPEC;
+               sizeof(StepRec) * SPEC + sizeof(ChainB) + sizeof(u64) + sizeof(MoveS) * SPEC + (size_t)dm.RG * 5;
     *threads = nt;
     *bytes = (b + 15) & ~(size_t)15;
     return 0;
@@ -387,6 +505,9 @@ int rp_launch_anneal_level(rp_ctx *c, int level, int n_levels, const rp_anneal_p
     A.Ppop = c->Ppop;
     A.last = (level == n_levels - 1);
     A.w_on_chip = 0;
+    A.slices = rp_uses_slices(c->dm) ? 1 : 0;
+    A.wref = c->d_wref; A.wfree = c->d_wfree; A.wfree_head = c->d_wfree_head;
+    if (rp_uses_slices(c->dm)) RP_TRY(rp_launch_slice_gc(c));
     A.wait_polls = c->knob_wait_polls > 0 ? c->knob_wait_polls : (1 << 22);
     A.stall_test = c->knob_stall;
     A.le_ws_cap = (unsigned)c->knob_le_ws_cap;
@@ -402,9 +523,31 @@ int rp_launch_anneal_level(rp_ctx *c, int level, int n_levels, const rp_anneal_p
     rp_anneal_smem_bytes(c, &nt, &smem);
     if (smem > 220 * 1024) return RP_ERR_RANGE;
     A.smem_bytes = (unsigned)smem;
-    if (smem > 32 * 1024)
-        RP_CUDA(cudaFuncSetAttribute(k_anneal_level<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k_anneal_level<128><<<c->Ppop, 128, smem, c->stream>>>(A);
+#define COOP_LAUNCH(MINB_, SL_)                                                                                 \
+    do {                                                                                                     \
+        if (smem > 32 * 1024)                                                                                \
+            RP_CUDA(cudaFuncSetAttribute(k_anneal_level<128, MINB_, SL_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+        k_anneal_level<128, MINB_, SL_><<<c->Ppop, 128, smem, c->stream>>>(A);                               \
+    } while (0)
+    // Resident chains per SM: six (80 registers) keep the most bytes in flight; windows whose rank
+    // loads per member pass a megabyte run faster with five (their working set misses L2 either way,
+    // and fewer chains leave more of it to the demand rows).
+    int minb = ((size_t)c->dm.RG * c->dm.LP * sizeof(int) >= (1u << 20)) ? 5 : 6;
+    if (c->knob_exp >= 4 && c->knob_exp <= 6) minb = c->knob_exp;
+    if (A.slices) {
+        switch (minb) {
+            case 5: COOP_LAUNCH(5, true); break;
+            case 4: COOP_LAUNCH(4, true); break;
+            default: COOP_LAUNCH(6, true); break;
+        }
+    } else {
+        switch (minb) {
+            case 5: COOP_LAUNCH(5, false); break;
+            case 4: COOP_LAUNCH(4, false); break;
+            default: COOP_LAUNCH(6, false); break;
+        }
+    }
+#undef COOP_LAUNCH
     ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
     return RP_OK;

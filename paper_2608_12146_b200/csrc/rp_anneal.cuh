@@ -37,6 +37,14 @@ struct AnnealArgs {
     const int *anc;
     int level, steps, log_cap, Ppop, last;
     int w_on_chip;                   // W is staged in shared memory: every level moves it anyway
+    // Slice mode (rank loads too large for one cell copy per replaced member): W is a pool of
+    // 2*P_pop*RG slices of L*P ints, a member's blob carries the slice of each of its row-shards,
+    // and a child shares its ancestor's slices until it rewrites them (an accepted move rewrites
+    // whole slices anyway, so leaving a shared slice costs no copy).
+    int slices;
+    const int *wref;                 // [2*P_pop*RG] holders of each slice at the start of the level
+    const int *wfree;                // free slices in ascending order; member j's spares are entries j*RG .. j*RG+RG-1
+    const int *wfree_head;           // [1] entries in the list
     unsigned smem_bytes;             // dynamic shared memory of the launch
     u64 tau, cq, rho_q32, guide_q32;
     u32 key0, key1;
@@ -283,7 +291,7 @@ __device__ __forceinline__ bool rp_chain_load(const AnnealArgs &A, int src, int 
                 rp_bulk_g2s((char *)Wsm + off, (const char *)ws + off, n, mbar);
             }
     }
-    if (!w_bulk && (WS || src_cell != dst_cell)) {      // a sole child works on in its ancestor's cell
+    if (!w_bulk && !A.slices && (WS || src_cell != dst_cell)) {      // a sole child works on in its ancestor's cell
         int *wd = WS ? Wsm : A.W + (size_t)dst_cell * wn;
         if ((wn & 3) == 0) {
             const int4 *ws4 = (const int4 *)ws;

@@ -104,6 +104,11 @@ k_anneal_wpc(const AnnealArgs A)
     int *vote = (int *)(cand + SPEC);                                    // [NW] accept flags of a wave
     int *rnd = vote + NW;                                               // [0] feasible mask, [1] next position
     unsigned short *best_lay = (unsigned short *)(((size_t)(rnd + 2) + 15) & ~(size_t)15);   // [N] trajectory-best layout
+    // Rank loads in global memory are kept as shared slices (see AnnealArgs): a free slice set aside
+    // for each row-shard, and whether this chain is the only holder of the row-shard's slice.
+    constexpr bool SL = !WS;
+    int *spare = (int *)(((size_t)(best_lay + dm.N) + 15) & ~(size_t)15);                    // [RG]
+    unsigned char *own = (unsigned char *)(spare + (SL ? dm.RG : 0));                        // [RG]
 
     u64 *Q = (u64 *)(sm_blob + A.bl.off_Q);
     i64 *Esum = (i64 *)(sm_blob + A.bl.off_Esum);
@@ -114,6 +119,7 @@ k_anneal_wpc(const AnnealArgs A)
     int *T = (int *)(sm_blob + A.bl.off_T);
     int *cnt = (int *)(sm_blob + A.bl.off_cnt);
     unsigned short *cell_of = (unsigned short *)(sm_blob + A.bl.off_cell);
+    int *wtab = (int *)(sm_blob + (SL ? A.bl.off_wtab : 0));             // row-shard -> slice of the pool
     const int *dpl = (const int *)(sm_static + A.sl.off_dpl);
     const int *dpo = (const int *)(sm_static + A.sl.off_dpo);
     const int *tt = A.sl.t_staged ? (const int *)(sm_static + A.sl.off_t) : A.t;
@@ -140,10 +146,12 @@ k_anneal_wpc(const AnnealArgs A)
         if (tid < nb0) recs[tid] = rp_make_step_rec(A, (u32)tid, (u32)blockIdx.x);
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    const int src = A.anc[j];
-    const int dst_cell = A.wloc_dst[j];                          // the previous level's barrier wrote it
-    const int src_cell = rp_src_cell(A, src, j);
-    int *Wj = WS ? Wsm : A.W + (size_t)dst_cell * wn;
+    // (clamped: after a level that gave up on a wait the table is stale, and the cell look-up below runs
+    // before this chain has seen the status word)
+    const int src = min(max(A.anc[j], 0), A.Ppop - 1);
+    const int dst_cell = SL ? 0 : A.wloc_dst[j];                 // the previous level's barrier wrote it
+    const int src_cell = SL ? 0 : rp_src_cell(A, src, j);
+    int *Wj = WS ? Wsm : A.W;
     // the incumbent's score when the level starts (fetched now, beside the loads above; used below)
     i64 inc0 = 0, inc1 = 0, inc2 = 0;
     if (tid == 0) {
@@ -185,6 +193,17 @@ k_anneal_wpc(const AnnealArgs A)
         chain->dig = 0; chain->best_step = 0; chain->best_nlog = 0; chain->nlog = 0;
         chain->I[0] = inc0; chain->I[1] = inc1; chain->I[2] = inc2;
         chain->has_snap = 0;
+    }
+    if (SL) {
+        // A slice that only this member holds when the level starts is rewritten in place; a shared
+        // one is left at its first rewrite for this chain's spare slice of that row-shard (entry
+        // j*RG + rg of the free list, which holds at least RG slices per member).
+        const int n_free = A.wfree_head[1];
+        for (int rg = tid; rg < dm.RG; rg += NT) {
+            const bool mine = (__ldg(&A.wref[wtab[rg]]) == 1);
+            own[rg] = mine ? 1 : 0;
+            spare[rg] = mine ? -1 : ((size_t)j * dm.RG + rg < (size_t)n_free ? __ldg(&A.wfree[(size_t)j * dm.RG + rg]) : -1);
+        }
     }
     __syncthreads();
 
@@ -247,7 +266,7 @@ k_anneal_wpc(const AnnealArgs A)
                     touchW = (rg1 != rg2);
                     const int *qi = A.q + (size_t)m.i * dm.LP;
                     const int *q2 = swap ? A.q + (size_t)m.i2 * dm.LP : nullptr;
-                    const int *w1 = Wj + (size_t)rg1 * dm.LP, *w2 = Wj + (size_t)rg2 * dm.LP;
+                    const int *w1 = Wj + (size_t)(SL ? wtab[rg1] : rg1) * dm.LP, *w2 = Wj + (size_t)(SL ? wtab[rg2] : rg2) * dm.LP;
                     const int nchunks = dm.LP >> 2;
                     RpSliceRegs<CH> regs;
                     // (a) put the loads of the two slices and the demand rows in flight
@@ -398,7 +417,20 @@ k_anneal_wpc(const AnnealArgs A)
                     if (warp == win) {
                         const bool swap = !m.reloc;
                         if (touchW) {
-                            int *w1 = Wj + (size_t)rg1 * dm.LP, *w2 = Wj + (size_t)rg2 * dm.LP;
+                            if (SL) {      // where the two rewritten slices go: in place when they are this chain's own, else to the spares
+                                if (lane == 0) {
+                                    const int both[2] = { rg1, rg2 };
+                                    for (int x = 0; x < 2; ++x) {
+                                        const int rg = both[x];
+                                        if (own[rg]) continue;
+                                        if (spare[rg] >= 0) wtab[rg] = spare[rg];
+                                        else atomicExch(&A.status[RP_SW_POOL], 1);       // cannot happen: the list has a spare per row-shard
+                                        own[rg] = 1;
+                                    }
+                                }
+                                __syncwarp();
+                            }
+                            int *w1 = Wj + (size_t)(SL ? wtab[rg1] : rg1) * dm.LP, *w2 = Wj + (size_t)(SL ? wtab[rg2] : rg2) * dm.LP;
                             if (vec) {
                                 for (int c = lane; c < (dm.LP >> 2); c += 32) {
                                     ((int4 *)w1)[c] = ((const int4 *)my_s1)[c];
@@ -498,6 +530,7 @@ size_t rp_wpc_smem_bytes(const RpDims &dm, const RpBlob &bl, const RpStatic &sl,
     const size_t per_cta = (size_t)220 * 1024 / (16 / nw);
     *w_in_smem = (b + wbytes <= per_cta);
     if (*w_in_smem) b += wbytes;
+    else b += 16 + (size_t)dm.RG * 5;            // spare slices and ownership flags
     return (b + 15) & ~(size_t)15;
 }
 
@@ -534,6 +567,7 @@ int rp_launch_anneal_wpc(rp_ctx *c, const AnnealArgs &A0)
     const size_t smem = rp_wpc_smem_bytes(dm, c->bl, c->sl, nw, &ws);
     AnnealArgs A = A0;
     A.w_on_chip = ws;
+    A.slices = ws ? 0 : 1;
     A.smem_bytes = (unsigned)smem;
     if (smem > 220 * 1024) return RP_ERR_RANGE;
     const int chunks = ((dm.LP >> 2) + 31) / 32;

@@ -152,6 +152,7 @@ static void free_population(rp_ctx *c)
     dev_free(c, c->d_pop_slab); c->d_pop_slab = nullptr;           // every buffer below is a piece of it
     c->buf[0].blob = nullptr; c->buf[1].blob = nullptr;
     c->d_W = nullptr; c->d_wloc = nullptr; c->d_wloc_next = nullptr; c->d_le_scratch = nullptr;
+    c->d_wref = nullptr; c->d_wcount = nullptr; c->d_wfree = nullptr; c->d_wfree_head = nullptr;
     c->d_cand_layout = nullptr; c->d_inc_slot = nullptr;
     c->d_anc = nullptr; c->d_anc_next = nullptr; c->d_done = nullptr; c->d_term = nullptr; c->d_best = nullptr; c->d_best_step = nullptr;
     c->d_best_nlog = nullptr; c->d_digest = nullptr; c->d_F = nullptr;
@@ -235,7 +236,7 @@ static int window_load_impl(rp_ctx *c, const rp_config *cfg, const int32_t *leng
     }
     dm.N = N; dm.L = L; dm.E = E; dm.k = cfg->top_k; dm.C = cfg->token_cap; dm.D = D; dm.P = P; dm.G = G;
     dm.H = E / P; dm.S = cfg->n_stages;
-    dm.R = 0; dm.K = 0; dm.RG = 0; dm.LP = L * P;
+    dm.R = 0; dm.K = 0; dm.RG = 0; dm.LP = L * P; dm.slices = 0;
     dm.asum = 0; dm.bsum = 0;
     for (int s = 0; s < RP_MAX_STAGES; ++s) { dm.ahat[s] = 0; dm.bhat[s] = 0; }
     for (int s = 0; s < dm.S; ++s) {
@@ -378,6 +379,8 @@ extern "C" int rp_window_load(rp_ctx **out, const rp_config *cfg, const int32_t 
     c->h_pin = (i64 *)pin_take();
     if (!c->h_pin) { free(c); return RP_ERR_CUDA; }
     c->side = side_take(c->device);          // optional: without it everything runs on the one stream
+    { const char *e = getenv("RP_EXP"); c->knob_exp = e ? atoi(e) : 0; }
+    { const char *e = getenv("RP_SLICES"); c->knob_slices = e ? atoi(e) : 0; }
     if (g_stage_timing)
         for (int x = 0; x < RP_STAGE_EVENTS; ++x)
             if (cudaEventCreate(&c->ev_stage[x]) != cudaSuccess) { cudaGetLastError(); c->ev_stage[0] = nullptr; break; }
@@ -470,7 +473,7 @@ extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
     c->Rstar = po[0]; c->certified = po[1];
     dm.R = po[0]; dm.K = dm.R * dm.D; dm.RG = dm.R * dm.G;
     if (dm.K > 65535) return RP_ERR_RANGE;
-    rp_make_layouts(dm, &c->bl, &c->sl);
+    rp_decide_layouts(c);
     int nt; size_t smem;
     rp_anneal_smem_bytes(c, &nt, &smem);
     if (smem > 220 * 1024) return RP_ERR_RANGE;
@@ -488,6 +491,12 @@ extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
             slab.take(&c->d_wloc, P);
             slab.take(&c->d_wloc_next, P);
             slab.take(&c->d_le_scratch, 6 * P);
+            if (rp_uses_slices(c->dm)) {
+                slab.take(&c->d_wref, 2 * P * (size_t)dm.RG);
+                slab.take(&c->d_wcount, 2 * P * (size_t)dm.RG);
+                slab.take(&c->d_wfree, 2 * P * (size_t)dm.RG);
+                slab.take(&c->d_wfree_head, 2);
+            }
             slab.take(&c->d_inc_slot, 1);
             if (rp_uses_wpc(c->dm)) slab.take(&c->d_cand_layout, P * (size_t)c->dm.N);
             slab.take(&c->d_anc, P);
@@ -503,6 +512,7 @@ extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
         }
     }
     c->cur = 0;
+    if (c->d_wcount) RP_CUDA(cudaMemsetAsync(c->d_wcount, 0, sizeof(int) * 2 * P * (size_t)dm.RG, c->stream));
     // every member starts as the length-only seed: evaluate it once into slot 0 and let all
     // slots descend from slot 0
     dev_free(c, c->d_static); c->d_static = nullptr;
@@ -826,6 +836,7 @@ extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *
     }
     if (st == RP_OK && e != cudaSuccess) { g_rp_last_cuda_error = (int)e; st = RP_ERR_CUDA; }
     RP_TRY(st);
+    if (sw[RP_SW_POOL]) { c->stage = 2; c->best_ready = 0; return RP_ERR_STATE; }     // slice pool exhausted: an internal invariant broke
     if (sw[RP_SW_TIMEOUT]) {
         // A bounded device-side wait ran out: that level's barrier and every later level were
         // skipped, so the population is not a population any more.  Back to "placed": only
@@ -837,7 +848,7 @@ extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *
     if (stats) {
         stats->proposed = cn[0]; stats->feasible = cn[1]; stats->accepted = cn[2]; stats->improved = cn[3];
         stats->move_bytes = cn[4]; stats->gather_bytes = cn[5]; stats->staging_bytes = cn[6];
-        stats->kernel_launches = (int64_t)NL;
+        stats->kernel_launches = (int64_t)NL * (rp_uses_slices(c->dm) ? 3 : 1);
         stats->ms_chains = ms_chains;
     }
     c->best_verdict = best_verdict(c, sw);
@@ -944,8 +955,18 @@ extern "C" int rp_debug_set_knob(rp_ctx *c, int knob, int64_t value)
             c->knob_wait_polls = (int)value; return RP_OK;
         case RP_KNOB_STALL_ONE_CHAIN:
             c->knob_stall = value ? 1 : 0; return RP_OK;
+        case RP_KNOB_RANK_LOAD_SLICES:
+            if (value > 2) return RP_ERR_ARG;
+            c->knob_slices = (int)value; return RP_OK;
         default: return RP_ERR_ARG;
     }
+}
+
+__global__ void k_gather_slices(const int *__restrict__ W, const int *__restrict__ tab, int LP, int *__restrict__ out)
+{
+    const int rg = blockIdx.x;
+    const int *src = W + (size_t)tab[rg] * LP;
+    for (int x = threadIdx.x; x < LP; x += blockDim.x) out[(size_t)rg * LP + x] = src[x];
 }
 
 extern "C" int rp_debug_set_trace(rp_ctx *c, int on)
@@ -985,12 +1006,22 @@ extern "C" int rp_debug_dump(rp_ctx *c, int what, int32_t index, void *buf, int6
             src = tmp;
             break;
         }
-        case RP_DUMP_W: {
+        case RP_DUMP_W:
+            if (rp_uses_slices(dm)) {          // the member's slices, gathered through its table
+                need = sizeof(int) * (size_t)dm.RG * dm.LP;
+                if ((st = dev_alloc(c, (int **)&tmp, (size_t)dm.RG * dm.LP)) != RP_OK) return st;
+                k_gather_slices<<<dm.RG, 128, 0, c->stream>>>(c->d_W, (const int *)(c->buf[c->cur].blob + (size_t)member * c->bl.bytes + c->bl.off_wtab),
+                                                              dm.LP, (int *)tmp);
+                ++g_rp_launches;
+                src = tmp;
+                break;
+            }
+            {
             int cell = 0;
             RP_CUDA(cudaMemcpyAsync(&cell, c->d_wloc + member, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
             RP_CUDA(cudaStreamSynchronize(c->stream));
             src = c->d_W + (size_t)cell * dm.RG * dm.LP; need = sizeof(int) * (size_t)dm.RG * dm.LP; break;
-        }
+            }
         case RP_DUMP_ESUM: src = c->buf[c->cur].blob + (size_t)member * c->bl.bytes + c->bl.off_Esum; need = sizeof(i64) * dm.RG; break;
         case RP_DUMP_CELL_T: case RP_DUMP_CELL_Q: case RP_DUMP_CELL_CNT: {
             size_t K = dm.K;

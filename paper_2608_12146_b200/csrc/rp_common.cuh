@@ -40,6 +40,7 @@ extern long long g_rp_launches;
 struct RpDims {
     int N, L, E, k, C, D, P, G, H, S;   // H = E / P experts per rank, S = attention stages
     int R, K, RG, LP;                   // rows, cells R*D, row-shards R*G, L*P (set after packing)
+    int slices;                         // rank loads kept as shared slices (set after packing; see AnnealArgs)
     i64 ahat[RP_MAX_STAGES], bhat[RP_MAX_STAGES];
     i64 asum, bsum;                     // sums over stages (attention key of a cell)
     i64 SC;                             // 2^8 * C^2
@@ -65,6 +66,8 @@ struct RpBlob {
     int off_T;      // int [K]   token sum per cell
     int off_cnt;    // int [K]   samples per cell
     int off_cell;   // u16 [N]   sample -> cell
+    int off_wtab;   // int [RG]  slice of the rank-load pool that holds each row-shard (-1: windows whose rank loads
+                    //           sit in one cell per member, see rp_uses_slices)
     int bytes;
 };
 // Tables that are the same for every chain of a plan (one block in global memory).
@@ -126,6 +129,10 @@ struct rp_ctx {
     int *d_wloc;               // [P_pop] cell of each member's current W (read through d_anc)
     int *d_wloc_next;          // [P_pop] cell each member works in during the next level
     int *d_le_scratch;         // [6*P_pop] ints for the level barrier's cell bookkeeping
+    int *d_wref;               // [2*P_pop*RG] members that hold each slice when a level starts (slice mode)
+    int *d_wcount;             // [2*P_pop*RG] the same while it is being counted; zero between two counts
+    int *d_wfree;              // [2*P_pop*RG] slices nobody holds, handed out in this order during the level
+    int *d_wfree_head;         // [2] next free-list entry to hand out, entries in the list
     RpBlob bl;
     RpStatic sl;
     char *d_static;            // static tables block
@@ -159,6 +166,8 @@ struct rp_ctx {
     // trace of the last rp_anneal call
     int trace_levels;
     int trace_on;              // keep per-level traces (inspection hook; off by default)
+    int knob_exp;
+    int knob_slices;           // inspection hook: 0 = automatic, 1 = slices wherever the cooperative kernel runs, 2 = never
     int knob_le_ws_cap, knob_wait_polls, knob_stall;   // inspection hooks (rp_debug_set_knob); 0 = off
     cudaEvent_t ev_stage[RP_STAGE_EVENTS];             // stage timing (rp_debug_set_stage_timing); null when off
     unsigned ev_recorded;                              // bit x: ev_stage[x] has been recorded
@@ -180,7 +189,7 @@ struct rp_ctx {
     i64 *d_seed_score;         // [3] best score of the initial population
 };
 
-enum RpStatusWord { RP_SW_BAD_SAMPLE = 0, RP_SW_BAD_LAYOUT = 1, RP_SW_VALIDATE = 2, RP_SW_TIMEOUT = 3, RP_SW_COUNT = 8 };
+enum RpStatusWord { RP_SW_BAD_SAMPLE = 0, RP_SW_BAD_LAYOUT = 1, RP_SW_VALIDATE = 2, RP_SW_TIMEOUT = 3, RP_SW_POOL = 4, RP_SW_COUNT = 8 };
 
 // ---------------------------------------------------------------------------------------
 // launch wrappers (each returns an rp_status; none synchronises)
@@ -198,6 +207,10 @@ int rp_launch_pack_on(rp_ctx *c, cudaStream_t stream);
 int rp_launch_pick_best(rp_ctx *c, const i64 *scores, const int *layouts, int n, i64 *best_score_out);
 int rp_get_pool(int device, cudaMemPool_t *out);     // the library's stream-ordered pool of a device
 void rp_make_layouts(const RpDims &dm, RpBlob *bl, RpStatic *sl);
+bool rp_uses_slices(const RpDims &dm);
+int rp_slice_mode(const RpDims &dm, int knob);
+void rp_decide_layouts(rp_ctx *c);
+int rp_launch_slice_gc(rp_ctx *c);
 int rp_launch_cells_from_layouts(rp_ctx *c, const int *layouts, int n, unsigned short *cells);
 // Stream-ordered device memory from the device's pool (n elements of T; freed on the context's stream).
 template <class T>

@@ -155,6 +155,8 @@ k_eval(const unsigned short *__restrict__ cells, const int *__restrict__ t, cons
             ((i64 *)(b + bl.off_Jfx))[rg] = Afx[rg] + dm.EC * Esum[rg];
         }
         for (int g = tid; g < dm.G; g += EVAL_THREADS) ((i64 *)(b + bl.off_U))[g] = U[g];
+        if (bl.off_wtab >= 0)          // W_out holds layout `lay` as RG consecutive slices of the pool
+            for (int rg = tid; rg < dm.RG; rg += EVAL_THREADS) ((int *)(b + bl.off_wtab))[rg] = lay * dm.RG + rg;
         for (int i = tid; i < dm.N; i += EVAL_THREADS) ((unsigned short *)(b + bl.off_cell))[i] = cell_of[i];
         if (tid == 0) {
             i64 *S = (i64 *)(b + bl.off_S);
@@ -220,6 +222,8 @@ void rp_make_layouts(const RpDims &dm, RpBlob *bl, RpStatic *sl)
     bl->off_T = o;    o += 4 * dm.K;
     bl->off_cnt = o;  o += 4 * dm.K;
     bl->off_cell = o; o += 2 * dm.N;
+    bl->off_wtab = -1;
+    if (rp_uses_slices(dm)) { o = (o + 3) & ~3; bl->off_wtab = o; o += 4 * dm.RG; }
     bl->bytes = (o + 15) & ~15;
     sl->t_staged = dm.N <= 2048;
     o = 0;

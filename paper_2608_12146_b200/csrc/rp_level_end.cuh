@@ -298,7 +298,7 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
     const u64 u0 = (u64)(((unsigned __int128)A.resample_x * Ftot) >> 32);
     // The cell bookkeeping further down works in shared memory when 8*P ints fit: ancestors and
     // current cells are staged beyond the cumulative weights while those are still in use.
-    const bool cells_on_chip = !A.w_on_chip && (size_t)P * 8 * sizeof(int) <= ws_bytes && F_on_chip;
+    const bool cells_on_chip = !A.w_on_chip && !A.slices && (size_t)P * 8 * sizeof(int) <= ws_bytes && F_on_chip;
     int *anc_s = (int *)ws + 6 * (size_t)P, *now_s = anc_s + P;
     if (cells_on_chip) for (int m = tid; m < P; m += nt) now_s[m] = A.wloc_dst[m];
     int depth = 0;
@@ -352,6 +352,7 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
     // ---- W cells of the next level.  A member that is its ancestor's only child works on in the
     // ancestor's cell; children of an ancestor with several children each get a free cell and
     // copy.  Cells: 2*P of them; the ones no surviving ancestor holds are free.
+    if (A.slices) return;                  // slice mode: children share their ancestor's slices, nothing to assign
     const int *now = A.wloc_dst;           // cells the terminal states of this level sit in
     if (A.w_on_chip) {      // W goes through shared memory every level anyway: alternate between the two halves
         // every member sits in the same half (its own cell m or P + m)

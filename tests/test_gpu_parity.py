@@ -294,12 +294,28 @@ def test_level_barrier_paths_on_small_windows(spec, cap):
     name, N, L, E, k, C, D, P, edp, min_rows, pop = spec
     w = make_window(custom_spec(name, N, L, E, k, C, D, P, pop, 400, data_seed=len(name) * 11 + N))
     ref = oracle_front(w, edp, min_rows)
-    ctx = load(w, pop=pop, edp=edp, min_rows=min_rows)
-    rp.rp_debug_set_knob(ctx, "BARRIER_WORKSPACE", cap)
-    check_front(w, ctx, ref)
-    want, stats = check_anneal(w, ctx, ref, edp, pop, 10, 40, t_ratio=0.6, check_members=2)
-    assert stats.accepted > 50 and stats.improved > 0
-    rp.rp_destroy(ctx)
+    for slices in ((1, 2) if L * P > 512 else (0,)):       # cooperative kernel: rank loads as shared slices, and as cells
+        ctx = load(w, pop=pop, edp=edp, min_rows=min_rows)
+        rp.rp_debug_set_knob(ctx, "BARRIER_WORKSPACE", cap)
+        rp.rp_debug_set_knob(ctx, "RANK_LOAD_SLICES", slices)
+        check_front(w, ctx, ref)
+        want, stats = check_anneal(w, ctx, ref, edp, pop, 10, 40, t_ratio=0.6, check_members=2)
+        assert stats.accepted > 50 and stats.improved > 0
+        if slices == 1:
+            assert stats.gather_bytes == 0          # nothing is copied when members share slices
+            # resume: the tables survive between calls
+            s_ = w.spec
+            again = oracle.anneal(w.lengths, ref["q"], want["final_pop"], ref["R"], s_.token_cap, s_.dp_width, n_levels=3,
+                                  steps=30, t0=1e-4, t_ratio=0.5, p_reloc=0.5, p_guide=0.3, seed=s_.anneal_seed,
+                                  edp_of_dp=edp, alpha=s_.alpha, beta=s_.beta)
+            rp.rp_anneal(ctx, n_levels=3, steps_per_level=30, t0=1e-4, t_ratio=0.5, p_reloc=0.5, p_guide=0.3)
+            assert (rp.rp_debug_dump(ctx, "TRACE_TERM", (3, pop, 3), np.int64) == again["term"]).all()
+            assert (rp.rp_debug_dump(ctx, "POPULATION", (pop, s_.n_samples), np.int32) == again["final_pop"]).all()
+            G = 1 + (max(edp) if edp is not None else D - 1)
+            for j in (0, pop - 1):
+                ev = oracle.eval_layouts(w.lengths, ref["q"], again["final_pop"][j], ref["R"], s_.token_cap, D, edp, s_.alpha, s_.beta)
+                assert (rp.rp_debug_dump(ctx, "W", (ref["R"], G, L, P), np.int32, index=j) == ev["W"][0]).all()
+        rp.rp_destroy(ctx)
 
 
 @pytest.mark.parametrize("spec", [BARRIER_CASES[0], BARRIER_CASES[2]], ids=["warp_per_candidate", "cooperative"])
