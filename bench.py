@@ -205,12 +205,14 @@ def reduce_job(ms_local, moves_local, dist=None, device="cpu"):
     return float(tmax.item()), int(round(tsum.item()))
 
 
-def plan_once(rp, w, t_in, a_in, outs, stream, stages=None):
+def plan_once(rp, w, t_in, a_in, outs, stream, stages=None, knobs=None):
     """One pass of the whole hot path through the C ABI; returns the annealing stats."""
     s = w.spec
     ctx = rp.rp_window_load(t_in, a_in, top_k=s.top_k, token_cap=s.token_cap, dp_width=s.dp_width,
                             ep_width=s.ep_width, pop_size=s.pop_size, alpha=s.alpha, beta=s.beta,
                             seed=s.anneal_seed, stream=stream)
+    for k, v in (knobs or {}).items():
+        rp.rp_debug_set_knob(ctx, k, v)
     rp.rp_place_experts(ctx, outs["pi"], outs["rank_load"])
     rp.rp_pack_rows(ctx)
     stats = rp.rp_anneal(ctx, n_levels=s.n_levels, steps_per_level=s.steps_per_level, t0=s.t0,
@@ -281,7 +283,7 @@ def measure(rp, torch, args, name, steps, min_seconds, dist, dev, local, cpu_sec
             acc["staging_bytes"] += st.staging_bytes
             acc["feasible"] += st.feasible
             acc["accepted"] += st.accepted
-            acc["chain_launches"] += s.n_levels
+            acc["chain_launches"] += 1 if st.kernel_launches == 1 else s.n_levels
         barrier()
         acc["wall"] = time.perf_counter() - wall0
         return acc
@@ -327,7 +329,8 @@ def measure(rp, torch, args, name, steps, min_seconds, dist, dev, local, cpu_sec
                 "traffic": None, "algorithmic_bytes_per_launch": alg,
                 "move_bytes_per_launch": res["move_bytes"] / nl, "gather_bytes_per_launch": res["gather_bytes"] / nl,
                 "staging_bytes_per_launch": res["staging_bytes"] / nl,
-                "launch_ms": per_launch_s * 1e3, "launches_per_step": s.n_levels, "share_of_step": res["chain_ms"] / res["ms"]}
+                "launch_ms": per_launch_s * 1e3, "launches_per_step": nl / steps,
+                "levels_per_launch": s.n_levels * steps / nl, "share_of_step": res["chain_ms"] / res["ms"]}
     prof = profiled_traffic(chain_kernel, s.name)
     if prof:
         scale = s.pop_size / float(prof["population"])
@@ -399,6 +402,34 @@ def concurrent_plans(rp, torch, name, dev, n_ctx, reps):
             "timing": "wall clock around host threads, one stream and context each"}
 
 
+def one_launch_latency(rp, torch, name, dev, reps=200):
+    """Context figure: latency of a single plan when rp_anneal runs all levels in one launch (the
+    library does so by itself only up to 148 members, see RP_KNOB_LAUNCH_PER_LEVEL)."""
+    w = make_window(SPECS[name])
+    s = w.spec
+    stream = torch.cuda.current_stream()
+    t_dev = torch.from_numpy(w.lengths).to(dev)
+    a_dev = torch.from_numpy(w.demand).to(dev)
+    outs = dict(pi=torch.empty((s.n_layers, s.n_experts), dtype=torch.int32, device=dev),
+                rank_load=torch.empty((s.n_layers, s.ep_width), dtype=torch.int64, device=dev),
+                layout=torch.empty(s.n_samples, dtype=torch.int32, device=dev),
+                score_fx=torch.empty(3, dtype=torch.int64, device=dev),
+                score_f64=torch.empty(3, dtype=torch.float64, device=dev))
+    out = {"workload": name, "plans": reps}
+    for label, knob in (("launch_per_level", 1), ("one_launch", 2)):
+        for _ in range(5):
+            plan_once(rp, w, t_dev, a_dev, outs, stream, knobs={"LAUNCH_PER_LEVEL": knob})
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        chain = 0.0
+        for _ in range(reps):
+            chain += plan_once(rp, w, t_dev, a_dev, outs, stream, knobs={"LAUNCH_PER_LEVEL": knob}).ms_chains
+        e1.record(stream)
+        e1.synchronize()
+        out[label] = {"ms_per_plan": e0.elapsed_time(e1) / reps, "anneal_ms_per_plan": chain / reps}
+    return out
+
+
 def seeding_stages(rp, torch, name, dev, reps=3):
     """Context figure: device time of the optional seeding stages (trial loop, pairing, canonical
     map + quality-diversity selection) on the named window, mean over `reps` fresh contexts."""
@@ -429,27 +460,17 @@ def seeding_stages(rp, torch, name, dev, reps=3):
             "choice_width": 4, "n_proj": 8, "eta_q16": 1 << 16}
 
 
-def l2_copy_rate(torch, dev, mib=24, reps=50):
-    """Device-to-device copy of a buffer that stays in L2 (read + write bytes per second): the
-    denominator for kernels whose operands L2 serves."""
-    a = torch.empty(mib << 20, dtype=torch.uint8, device=dev)
-    b = torch.empty_like(a)
-    for _ in range(5):
-        b.copy_(a)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(reps):
-        b.copy_(a)
-    e1.record()
-    e1.synchronize()
-    return 2.0 * (mib << 20) * reps / (e0.elapsed_time(e1) * 1e-3) / 1e9
+def l2_read_rate(rp, mib=32, reps=50):
+    """Read bandwidth of a buffer that stays in L2 (every thread of a full grid sums it with 16-byte
+    loads): the denominator for kernels whose operands L2 serves."""
+    return rp.rp_debug_l2_read_rate(mib << 20, reps)
 
 
 def eval_stage(rp, torch, name, dev, l2_gbs, reps=10):
     """Context figure: full scoring of one population-sized batch of distinct layouts
     (rp_eval_population, device inputs and outputs).  The demand rows every layout gathers
     (N*L*P*4 bytes per layout) are shared by all layouts and served by L2, so they are set against a
-    measured L2 copy rate; what must cross HBM is the assignment (N*2 bytes per layout) plus the
+    measured L2 read rate; what must cross HBM is the assignment (N*2 bytes per layout) plus the
     demand rows once, set against the measured HBM peak."""
     w = make_window(SPECS[name])
     s = w.spec
@@ -479,7 +500,7 @@ def eval_stage(rp, torch, name, dev, l2_gbs, reps=10):
     hbm_min = s.pop_size * s.n_samples * 4 + q_bytes          # int32 layouts in, demand rows once
     return {"workload": name, "layouts": s.pop_size, "ms": ms, "layouts_per_s": s.pop_size / ms * 1e3,
             "roofline": {"bound": "l2", "kernel": "k_eval", "achieved": gathered / ms / 1e6, "peak": l2_gbs, "unit": "GB/s",
-                         "frac": gathered / ms / 1e6 / l2_gbs, "peak_source": "L2-resident device copy measured in this run",
+                         "frac": gathered / ms / 1e6 / l2_gbs, "peak_source": "read rate of a 32 MiB L2-resident buffer measured in this run (rp_debug_l2_read_rate)",
                          "gathered_bytes_per_launch": gathered, "hbm_bytes_per_launch_min": hbm_min,
                          "hbm_min_gbs": hbm_min / ms / 1e6, "hbm_min_frac": hbm_min / ms / 1e6 / peak}}
 
@@ -527,7 +548,7 @@ def run_cuda(args):
     dev = torch.device("cuda", local)
 
     if args.eval_only:          # profiling aid: only the population-sized scoring batch of the named window
-        l2 = l2_copy_rate(torch, dev)
+        l2 = l2_read_rate(rp)
         print(json.dumps(eval_stage(rp, torch, args.workload, dev, l2, reps=max(1, args.steps))))
         return 0
     main_cpu = 0 if (world > 1 or rank != 0 or args.no_cpu_baseline) else 12.0
@@ -550,10 +571,11 @@ def run_cuda(args):
         if sweep:
             line["other_workloads"] = sweep
         if extras:
-            l2 = l2_copy_rate(torch, dev)
-            line["l2_copy_gbs"] = l2
+            l2 = l2_read_rate(rp)
+            line["l2_read_gbs"] = l2
             line["eval_population"] = [eval_stage(rp, torch, n, dev, l2) for n in ("medium", "large", "wide")]
             line["concurrent_plans"] = [concurrent_plans(rp, torch, "medium", dev, n, 200) for n in (1, 2, 4)]
+            line["single_plan_latency"] = [one_launch_latency(rp, torch, n, dev) for n in ("tiny", "medium")]
             line["seeding_stages"] = seeding_stages(rp, torch, "medium", dev)
             line["mechanism_diagnostics"] = [mechanism_diagnostics(rp, torch, n, dev) for n in ("medium", "large")]
         print(json.dumps(line))

@@ -280,14 +280,20 @@ typedef enum {
  *     use; a small value sends its cumulative weights, cell bookkeeping and incumbent replay
  *     through their global-memory forms.
  *   RP_KNOB_WAIT_POLLS: polls after which a chain's wait on its asynchronous copies gives up
- *     (default 2^22).
+ *     (default 2^22); a chain's wait for the other chains of a launch that runs all levels then
+ *     gives up after that many microseconds (default 2 s + 50 us per step of a level).
  *   RP_KNOB_STALL_ONE_CHAIN: chain 0 waits once more, after its copies have landed, on a barrier
  *     phase that nothing completes: the wait runs out and rp_anneal returns RP_ERR_TIMEOUT.
+ *   RP_KNOB_LAUNCH_PER_LEVEL: how rp_anneal launches windows whose chains can all be resident at
+ *     once (rank loads on chip, at most 256 members).  0 = automatic: one launch for all levels up
+ *     to 148 members, one launch per level above (two windows planned at once on two streams then
+ *     still share the GPU); 1 = always one launch per level; 2 = one launch for all levels
+ *     wherever possible (lowest latency of a single plan).
  *   RP_KNOB_RANK_LOAD_SLICES (set before rp_pack_rows): how windows with L*P > 512 keep the rank
  *     loads of the population.  0 or 1 = shared slices with copy-on-write (the default), 2 = one
  *     private cell per member, copied whole when resampling replaces the member. */
 typedef enum { RP_KNOB_BARRIER_WORKSPACE = 1, RP_KNOB_WAIT_POLLS = 2, RP_KNOB_STALL_ONE_CHAIN = 3,
-               RP_KNOB_RANK_LOAD_SLICES = 4 } rp_knob;
+               RP_KNOB_RANK_LOAD_SLICES = 4, RP_KNOB_LAUNCH_PER_LEVEL = 5 } rp_knob;
 int rp_debug_set_knob(rp_ctx *ctx, int knob, int64_t value);
 /* Device time of the stages that have no statistics struct of their own.  After
  * rp_debug_set_stage_timing(1) (process-wide; contexts loaded later record CUDA events around the
@@ -310,6 +316,11 @@ int rp_debug_nl2(const uint32_t *x, uint64_t *out, int64_t n);
 int rp_debug_exp2neg(const uint64_t *z, uint64_t *out, int64_t n);
 /* out[i][0..3] = Philox4x32-10(counter ctr[i][0..3], key) on the device. */
 int rp_debug_philox(const uint32_t *ctr, const uint32_t key[2], uint32_t *out, int64_t n);
+/* Read bandwidth, in GB/s, of a zeroed buffer of `bytes` (1 MiB .. 2 GiB) that every thread of a
+ * full grid sums `reps` times over with 16-byte loads: with a buffer that fits L2 this is the
+ * measured L2 read rate that kernels whose operands L2 serves are set against.  Allocates and
+ * frees its own buffer; runs on the default stream of the current device. */
+int rp_debug_l2_read_rate(int64_t bytes, int32_t reps, double *gb_per_s);
 /* Number of kernels this library has launched in this process so far. */
 int64_t rp_debug_launch_count(void);
 

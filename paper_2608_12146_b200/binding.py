@@ -25,7 +25,7 @@ RP_OK = 0
 EXPORTS = ("rp_window_load", "rp_place_experts", "rp_pack_rows", "rp_seed_population", "rp_pair_population", "rp_select_population", "rp_eval_population", "rp_eval_layouts_noalloc", "rp_diagnostics", "rp_anneal",
            "rp_best", "rp_destroy", "rp_release_cached_memory", "rp_strerror", "rp_last_cuda_error", "rp_debug_dump",
            "rp_debug_set_trace", "rp_debug_set_knob", "rp_debug_set_stage_timing", "rp_debug_stage_times",
-           "rp_debug_nl2", "rp_debug_exp2neg", "rp_debug_philox", "rp_debug_launch_count")
+           "rp_debug_nl2", "rp_debug_exp2neg", "rp_debug_philox", "rp_debug_launch_count", "rp_debug_l2_read_rate")
 
 
 class RpError(RuntimeError):
@@ -98,6 +98,7 @@ def lib():
         L.rp_debug_exp2neg.argtypes = [C.c_void_p, C.c_void_p, C.c_int64]
         L.rp_debug_philox.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64]
         L.rp_debug_launch_count.restype = C.c_int64
+        L.rp_debug_l2_read_rate.argtypes = [C.c_int64, C.c_int32, C.POINTER(C.c_double)]
         _lib = L
     return _lib
 
@@ -291,7 +292,7 @@ def rp_debug_stage_times(ctx: Context) -> dict:
     return {k: (float(v) if v >= 0 else None) for k, v in zip(STAGES, ms)}
 
 
-KNOB = dict(BARRIER_WORKSPACE=1, WAIT_POLLS=2, STALL_ONE_CHAIN=3, RANK_LOAD_SLICES=4)
+KNOB = dict(BARRIER_WORKSPACE=1, WAIT_POLLS=2, STALL_ONE_CHAIN=3, RANK_LOAD_SLICES=4, LAUNCH_PER_LEVEL=5)
 
 
 def rp_debug_set_knob(ctx: Context, knob: str, value: int):
@@ -316,6 +317,13 @@ def rp_debug_exp2neg(z) -> np.ndarray:
     out = np.empty(z.shape, np.uint64)
     _check(lib().rp_debug_exp2neg(_ptr(z), _ptr(out), z.size), "rp_debug_exp2neg")
     return out
+
+
+def rp_debug_l2_read_rate(nbytes: int = 32 << 20, reps: int = 50) -> float:
+    """Measured read bandwidth (GB/s) of a buffer of `nbytes` that stays in L2."""
+    out = C.c_double(0.0)
+    _check(lib().rp_debug_l2_read_rate(nbytes, reps, C.byref(out)), "rp_debug_l2_read_rate")
+    return float(out.value)
 
 
 def rp_debug_launch_count() -> int:

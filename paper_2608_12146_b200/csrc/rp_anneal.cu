@@ -140,7 +140,7 @@ k_anneal_level(const AnnealArgs A)
 
     for (int kb = 0; kb < A.steps; kb += SPEC) {
         const int nb = min(SPEC, A.steps - kb);
-        if (tid < nb) recs[tid] = rp_make_step_rec(A, (u32)(kb + tid), (u32)j);
+        if (tid < nb) recs[tid] = rp_make_step_rec(A, A.level, A.tau, (u32)(kb + tid), (u32)j);
         __syncthreads();
         int pos = 0;
         while (pos < nb) {
@@ -485,9 +485,10 @@ static u32 host_philox_x(u32 c0, u32 c1, u32 c2, u32 c3, u32 k0, u32 k1)
     return c0;
 }
 
-int rp_launch_anneal_level(rp_ctx *c, int level, int n_levels, const rp_anneal_params *prm, u64 rho_q32, u64 guide_q32)
+int rp_launch_anneal_wpc_all(rp_ctx *c, const AnnealArgs &A, int *done);
+
+static void fill_args(rp_ctx *c, int level, int n_levels, const rp_anneal_params *prm, u64 rho_q32, u64 guide_q32, AnnealArgs &A)
 {
-    AnnealArgs A;
     A.dm = c->dm; A.bl = c->bl; A.sl = c->sl;
     A.t = c->d_t; A.q = c->d_q; A.static_blk = c->d_static;
     const RpPopBuf &s = c->buf[c->cur], &d = c->buf[1 - c->cur];
@@ -507,7 +508,6 @@ int rp_launch_anneal_level(rp_ctx *c, int level, int n_levels, const rp_anneal_p
     A.w_on_chip = 0;
     A.slices = rp_uses_slices(c->dm) ? 1 : 0;
     A.wref = c->d_wref; A.wfree = c->d_wfree; A.wfree_head = c->d_wfree_head;
-    if (rp_uses_slices(c->dm)) RP_TRY(rp_launch_slice_gc(c));
     A.wait_polls = c->knob_wait_polls > 0 ? c->knob_wait_polls : (1 << 22);
     A.stall_test = c->knob_stall;
     A.le_ws_cap = (unsigned)c->knob_le_ws_cap;
@@ -518,6 +518,56 @@ int rp_launch_anneal_level(rp_ctx *c, int level, int n_levels, const rp_anneal_p
     A.lo.inc_slot = c->d_inc_slot;
     A.lo.tr_term = c->d_tr_term; A.lo.tr_best = c->d_tr_best; A.lo.tr_inc = c->d_tr_inc;
     A.lo.tr_best_step = c->d_tr_best_step; A.lo.tr_anc = c->d_tr_anc; A.lo.tr_digest = c->d_tr_digest;
+    A.n_levels = n_levels; A.cur0 = c->cur;
+    A.levels = (const RpLevelDev *)c->d_levels;
+    A.blob_b0 = c->buf[0].blob; A.blob_b1 = c->buf[1].blob;
+    A.sync = c->d_sync;
+    A.lo.anc_cur = c->d_anc;
+    A.bar_timeout_ns = c->knob_wait_polls > 0 ? (u64)c->knob_wait_polls * 1000ull
+                                               : 2000000000ull + (u64)prm->steps_per_level * 50000ull;
+}
+
+// The levels' schedule integers for the launch that runs all levels (with the random word behind
+// each resampling offset, which depends only on the seed and the level).
+int rp_upload_levels(rp_ctx *c, int n_levels)
+{
+    if (n_levels > c->levels_dev_cap) {
+        dev_free(c, c->d_levels); c->d_levels = nullptr; c->levels_dev_cap = 0;
+        RpLevelDev *d = nullptr;
+        RP_TRY(dev_alloc(c, &d, (size_t)n_levels));
+        c->d_levels = d; c->levels_dev_cap = n_levels;
+    }
+    RpLevelDev *h = (RpLevelDev *)malloc(sizeof(RpLevelDev) * n_levels);
+    const u32 k0 = (u32)c->cfg.seed, k1 = (u32)(c->cfg.seed >> 32);
+    for (int n = 0; n < n_levels; ++n) {
+        h[n].tau = c->h_levels[n].tau; h[n].cq = c->h_levels[n].cq;
+        h[n].resample_x = host_philox_x(0u, (u32)n, 0u, 3u, k0, k1); h[n].pad = 0;
+    }
+    const cudaError_t e = cudaMemcpyAsync(c->d_levels, h, sizeof(RpLevelDev) * n_levels, cudaMemcpyHostToDevice, c->stream);
+    free(h);            // pageable source: staged before the call returned
+    if (e != cudaSuccess) { g_rp_last_cuda_error = (int)e; return RP_ERR_CUDA; }
+    return RP_OK;
+}
+
+// Every level of the call in one launch, when the window allows it (*done = 1); see rp_anneal_wpc.cu.
+int rp_launch_anneal_all(rp_ctx *c, int n_levels, const rp_anneal_params *prm, u64 rho_q32, u64 guide_q32, int *done)
+{
+    *done = 0;
+    // Automatic: only populations of at most one chain per SM, so that a second window planned at
+    // the same time on another stream still finds room (a launch whose chains wait for one another
+    // needs all of them resident at once, and two such launches do not share the SMs).
+    const bool wanted = c->knob_level_launches == 2 || (c->knob_level_launches == 0 && c->Ppop <= 148);
+    if (!use_wpc(c->dm) || !wanted || !c->d_levels) return RP_OK;
+    AnnealArgs A;
+    fill_args(c, 0, n_levels, prm, rho_q32, guide_q32, A);
+    return rp_launch_anneal_wpc_all(c, A, done);
+}
+
+int rp_launch_anneal_level(rp_ctx *c, int level, int n_levels, const rp_anneal_params *prm, u64 rho_q32, u64 guide_q32)
+{
+    AnnealArgs A;
+    fill_args(c, level, n_levels, prm, rho_q32, guide_q32, A);
+    if (rp_uses_slices(c->dm)) RP_TRY(rp_launch_slice_gc(c));
     if (use_wpc(c->dm)) return rp_launch_anneal_wpc(c, A);
     int nt; size_t smem;
     rp_anneal_smem_bytes(c, &nt, &smem);
@@ -533,7 +583,6 @@ int rp_launch_anneal_level(rp_ctx *c, int level, int n_levels, const rp_anneal_p
     // loads per member pass a megabyte run faster with five (their working set misses L2 either way,
     // and fewer chains leave more of it to the demand rows).
     int minb = ((size_t)c->dm.RG * c->dm.LP * sizeof(int) >= (1u << 20)) ? 5 : 6;
-    if (c->knob_exp >= 4 && c->knob_exp <= 6) minb = c->knob_exp;
     if (A.slices) {
         switch (minb) {
             case 5: COOP_LAUNCH(5, true); break;

@@ -19,10 +19,13 @@ struct LevelOut {
     // among the writers: the row of the current incumbent's slot is never overwritten unnoticed.
     unsigned short *cand_layout;   // [P_pop][N]
     int *inc_slot;                 // slot whose row holds the incumbent, -1 = inc_layout is current
+    int *anc_cur;                  // the ancestor table the call started from (one launch for all levels: both are set at the end)
     i64 *tr_term, *tr_best, *tr_inc;     // trace (nullable)
     int *tr_best_step, *tr_anc;
     u64 *tr_digest;
 };
+
+struct RpLevelDev { u64 tau, cq; u32 resample_x, pad; };   // per-level schedule integers on the device
 
 struct AnnealArgs {
     RpDims dm;
@@ -49,6 +52,14 @@ struct AnnealArgs {
     u64 tau, cq, rho_q32, guide_q32;
     u32 key0, key1;
     u32 resample_x;                  // Philox(0, level, 0, 3).x, the word behind the resampling offset (computed on the host)
+    // One launch for all levels (every chain resident at once): the levels' schedule, the two blob
+    // buffers by name, which of them the call starts from, the arrival counter and the time a chain
+    // may wait for the others.
+    int n_levels, cur0;
+    const RpLevelDev *levels;
+    char *blob_b0, *blob_b1;
+    int *sync;
+    u64 bar_timeout_ns;
     int wait_polls;                  // limit of every bounded wait on a bulk-copy barrier (polls)
     int stall_test;                  // inspection hook: after its loads have landed, chain 0 waits once more on a
                                      // barrier phase that nothing completes, so that the wait runs out
@@ -76,12 +87,12 @@ struct MoveS { int reloc, i, i2, c1, c2; };
 // Purposes: 0 = proposal words A, 1 = proposal words B, 2 = accept word.
 // The uniform branch is stored as a tournament between a candidate and itself, so that the
 // proposal rule below needs no branch on it.
-__device__ __forceinline__ StepRec rp_make_step_rec(const AnnealArgs &A, u32 k, u32 j)
+__device__ __forceinline__ StepRec rp_make_step_rec(const AnnealArgs &A, int level, u64 tau, u32 k, u32 j)
 {
     const RpDims &dm = A.dm;
-    const uint4 a = rp_philox(k, (u32)A.level, j, 0u, A.key0, A.key1);
-    const uint4 b = rp_philox(k, (u32)A.level, j, 1u, A.key0, A.key1);
-    const uint4 xw = rp_philox(k, (u32)A.level, j, 2u, A.key0, A.key1);
+    const uint4 a = rp_philox(k, (u32)level, j, 0u, A.key0, A.key1);
+    const uint4 b = rp_philox(k, (u32)level, j, 1u, A.key0, A.key1);
+    const uint4 xw = rp_philox(k, (u32)level, j, 2u, A.key0, A.key1);
     const bool reloc = (u64)a.x < A.rho_q32, guided = (u64)a.y < A.guide_q32;
     StepRec r;
     r.i0 = rp_pick(a.z, dm.N);
@@ -96,7 +107,7 @@ __device__ __forceinline__ StepRec rp_make_step_rec(const AnnealArgs &A, u32 k, 
     }
     r.bz = b.z;
     const u64 nl = rp_nl2(xw.x);
-    const u64 hi = __umul64hi(A.tau, nl), lo = A.tau * nl;
+    const u64 hi = __umul64hi(tau, nl), lo = tau * nl;
     const bool sat = (hi >> 30) != 0;
     r.thr = (hi << 32) | (lo >> 32);
     r.flags = (reloc ? 1u : 0u) | (guided ? 2u : 0u) | (sat ? 4u : 0u);

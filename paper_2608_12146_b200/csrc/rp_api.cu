@@ -154,6 +154,7 @@ static void free_population(rp_ctx *c)
     c->d_W = nullptr; c->d_wloc = nullptr; c->d_wloc_next = nullptr; c->d_le_scratch = nullptr;
     c->d_wref = nullptr; c->d_wcount = nullptr; c->d_wfree = nullptr; c->d_wfree_head = nullptr;
     c->d_cand_layout = nullptr; c->d_inc_slot = nullptr;
+    c->d_sync = nullptr;
     c->d_anc = nullptr; c->d_anc_next = nullptr; c->d_done = nullptr; c->d_term = nullptr; c->d_best = nullptr; c->d_best_step = nullptr;
     c->d_best_nlog = nullptr; c->d_digest = nullptr; c->d_F = nullptr;
     dev_free(c, c->d_sel_dist); c->d_sel_dist = nullptr;
@@ -185,7 +186,7 @@ extern "C" void rp_destroy(rp_ctx *c)
     if (!c) return;
     cudaStreamSynchronize(c->stream);
     free_population(c); free_trace(c); free_eval(c);
-    dev_free(c, c->own_t); dev_free(c, c->own_a); dev_free(c, c->d_load_slab); dev_free(c, c->d_static);
+    dev_free(c, c->own_t); dev_free(c, c->own_a); dev_free(c, c->d_load_slab); dev_free(c, c->d_static); dev_free(c, c->d_levels);
     pin_give(c->h_pin);
     for (int x = 0; x < RP_STAGE_EVENTS; ++x) if (c->ev_stage[x]) cudaEventDestroy(c->ev_stage[x]);
     side_give((RpSide *)c->side);
@@ -379,8 +380,6 @@ extern "C" int rp_window_load(rp_ctx **out, const rp_config *cfg, const int32_t 
     c->h_pin = (i64 *)pin_take();
     if (!c->h_pin) { free(c); return RP_ERR_CUDA; }
     c->side = side_take(c->device);          // optional: without it everything runs on the one stream
-    { const char *e = getenv("RP_EXP"); c->knob_exp = e ? atoi(e) : 0; }
-    { const char *e = getenv("RP_SLICES"); c->knob_slices = e ? atoi(e) : 0; }
     if (g_stage_timing)
         for (int x = 0; x < RP_STAGE_EVENTS; ++x)
             if (cudaEventCreate(&c->ev_stage[x]) != cudaSuccess) { cudaGetLastError(); c->ev_stage[0] = nullptr; break; }
@@ -502,11 +501,12 @@ extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
             slab.take(&c->d_anc, P);
             slab.take(&c->d_anc_next, P);
             slab.take(&c->d_done, 1);
-            slab.take(&c->d_term, P * 3);
-            slab.take(&c->d_best, P * 3);
-            slab.take(&c->d_best_step, P);
-            slab.take(&c->d_best_nlog, P);
-            slab.take(&c->d_digest, P);
+            slab.take(&c->d_sync, P + 1);                // arrival counter, then one state-complete flag per member
+            slab.take(&c->d_term, 2 * P * 3);            // reports: two sets, taken in turn by the launch that runs all levels
+            slab.take(&c->d_best, 2 * P * 3);
+            slab.take(&c->d_best_step, 2 * P);
+            slab.take(&c->d_best_nlog, 2 * P);
+            slab.take(&c->d_digest, 2 * P);
             slab.take(&c->d_F, P);
             if (pass == 0) { RP_TRY(dev_alloc(c, &c->d_pop_slab, slab.off)); slab.base = c->d_pop_slab; }
         }
@@ -763,12 +763,13 @@ static int launch_best_check(rp_ctx *c);
 static int best_verdict(const rp_ctx *c, const int *sw);
 
 __global__ void k_reset_anneal(i64 *__restrict__ counters, int *__restrict__ status, int *__restrict__ inc_slot,
-                               int *__restrict__ done)
+                               int *__restrict__ done, int *__restrict__ sync, int n_sync)
 {
     const int x = threadIdx.x;
     if (x < 8) counters[x] = 0;
     if (x < RP_SW_COUNT) status[x] = 0;
     if (x == 0) { *inc_slot = -1; *done = 0; }
+    for (int y = x; y < n_sync; y += blockDim.x) sync[y] = 0;
 }
 
 extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *stats)
@@ -804,7 +805,7 @@ extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *
         c->trace_levels = NL;
     }
     // counters and status words to zero, incumbent slot to -1 (the incumbent is in d_inc_layout)
-    k_reset_anneal<<<1, 32, 0, c->stream>>>(c->d_counters, c->d_status, c->d_inc_slot, c->d_done);
+    k_reset_anneal<<<1, 256, 0, c->stream>>>(c->d_counters, c->d_status, c->d_inc_slot, c->d_done, c->d_sync, c->Ppop + 1);
     ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
 
@@ -812,8 +813,13 @@ extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *
     if (stats) for (int x = 0; x < 2; ++x) RP_CUDA(cudaEventCreate(&ev[x]));
     float ms_chains = 0.f;
     int st = RP_OK;
+    // One launch for all levels where every chain can be resident at once, else one launch per level.
+    int all_in_one = 0;
+    if (rp_uses_wpc(c->dm) && c->knob_level_launches != 1) st = rp_upload_levels(c, NL);
     if (stats) cudaEventRecord(ev[0], c->stream);
-    for (int n = 0; n < NL && st == RP_OK; ++n) {
+    if (st == RP_OK) st = rp_launch_anneal_all(c, NL, p, rho_q32, guide_q32, &all_in_one);
+    if (all_in_one) c->cur = (c->cur + NL) & 1;       // the kernel has left both ancestor tables and both cell tables current
+    for (int n = 0; n < NL && st == RP_OK && !all_in_one; ++n) {
         st = rp_launch_anneal_level(c, n, NL, p, rho_q32, guide_q32);
         c->cur = 1 - c->cur;          // the terminal states are the next level's sources
         { int *sw = c->d_anc; c->d_anc = c->d_anc_next; c->d_anc_next = sw; }
@@ -848,7 +854,7 @@ extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *
     if (stats) {
         stats->proposed = cn[0]; stats->feasible = cn[1]; stats->accepted = cn[2]; stats->improved = cn[3];
         stats->move_bytes = cn[4]; stats->gather_bytes = cn[5]; stats->staging_bytes = cn[6];
-        stats->kernel_launches = (int64_t)NL * (rp_uses_slices(c->dm) ? 3 : 1);
+        stats->kernel_launches = all_in_one ? 1 : (int64_t)NL * (rp_uses_slices(c->dm) ? 3 : 1);
         stats->ms_chains = ms_chains;
     }
     c->best_verdict = best_verdict(c, sw);
@@ -955,6 +961,9 @@ extern "C" int rp_debug_set_knob(rp_ctx *c, int knob, int64_t value)
             c->knob_wait_polls = (int)value; return RP_OK;
         case RP_KNOB_STALL_ONE_CHAIN:
             c->knob_stall = value ? 1 : 0; return RP_OK;
+        case RP_KNOB_LAUNCH_PER_LEVEL:
+            if (value > 2) return RP_ERR_ARG;
+            c->knob_level_launches = (int)value; return RP_OK;
         case RP_KNOB_RANK_LOAD_SLICES:
             if (value > 2) return RP_ERR_ARG;
             c->knob_slices = (int)value; return RP_OK;
@@ -1077,6 +1086,50 @@ __global__ void k_dbg_philox(const u32 *ctr, u32 k0, u32 k1, u32 *out, long long
         uint4 r = rp_philox(ctr[4 * i], ctr[4 * i + 1], ctr[4 * i + 2], ctr[4 * i + 3], k0, k1);
         out[4 * i] = r.x; out[4 * i + 1] = r.y; out[4 * i + 2] = r.z; out[4 * i + 3] = r.w;
     }
+}
+
+// Read bandwidth of a buffer that stays in L2: every thread sums 16-byte pieces of it, the whole
+// buffer `reps` times over; the figure is the denominator for kernels whose operands L2 serves.
+__global__ void k_dbg_l2_read(const int4 *__restrict__ buf, long long n4, int reps, int *__restrict__ sink)
+{
+    int acc = 0;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (int r = 0; r < reps; ++r)
+        for (long long x = (long long)blockIdx.x * blockDim.x + threadIdx.x; x < n4; x += stride) {
+            const int4 v = __ldcg(buf + x);
+            acc += v.x ^ v.y ^ v.z ^ v.w;
+        }
+    if (acc == 0x7fffffff) *sink = acc;          // never true for the zeroed buffer: keeps the loads alive
+}
+
+extern "C" int rp_debug_l2_read_rate(int64_t bytes, int32_t reps, double *gb_per_s)
+{
+    if (!gb_per_s || bytes < (1 << 20) || bytes > (1ll << 31) || reps < 1 || reps > 10000) return RP_ERR_ARG;
+    int4 *buf = nullptr;
+    int *sink = nullptr;
+    RP_CUDA(cudaMalloc((void **)&buf, (size_t)bytes));
+    if (cudaMalloc((void **)&sink, sizeof(int)) != cudaSuccess) { cudaFree(buf); return RP_ERR_CUDA; }
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    cudaError_t e = cudaMemset(buf, 0, (size_t)bytes);
+    if (e == cudaSuccess) e = cudaEventCreate(&e0);
+    if (e == cudaSuccess) e = cudaEventCreate(&e1);
+    float ms = 0.f;
+    if (e == cudaSuccess) {
+        const long long n4 = bytes / 16;
+        k_dbg_l2_read<<<148 * 8, 256>>>(buf, n4, 2, sink);              // warm the cache
+        cudaEventRecord(e0);
+        k_dbg_l2_read<<<148 * 8, 256>>>(buf, n4, reps, sink);
+        cudaEventRecord(e1);
+        g_rp_launches += 2;
+        e = cudaEventSynchronize(e1);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+    }
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    cudaFree(buf); cudaFree(sink);
+    if (e != cudaSuccess) { g_rp_last_cuda_error = (int)e; return RP_ERR_CUDA; }
+    *gb_per_s = (double)bytes * reps / (ms * 1e-3) / 1e9;
+    return RP_OK;
 }
 
 template <class TI, class TO, class F>

@@ -140,6 +140,9 @@ struct rp_ctx {
     int *d_anc;                // [P_pop] which member of buf[cur] each slot continues from
     int *d_anc_next;           // [P_pop] written by the level barrier, swapped with d_anc
     int *d_done;               // arrival counter of the chain CTAs
+    int *d_sync;               // arrival counter of the launch that runs all levels
+    void *d_levels;            // per-level schedule integers on the device (RpLevelDev), levels_dev_cap of them
+    int levels_dev_cap;
     // per-level results
     i64 *d_term;               // [P_pop][3]
     i64 *d_best;               // [P_pop][3]
@@ -166,7 +169,7 @@ struct rp_ctx {
     // trace of the last rp_anneal call
     int trace_levels;
     int trace_on;              // keep per-level traces (inspection hook; off by default)
-    int knob_exp;
+    int knob_level_launches;   // 0 = automatic, 1 = one launch per level, 2 = one launch for all levels wherever possible
     int knob_slices;           // inspection hook: 0 = automatic, 1 = slices wherever the cooperative kernel runs, 2 = never
     int knob_le_ws_cap, knob_wait_polls, knob_stall;   // inspection hooks (rp_debug_set_knob); 0 = off
     cudaEvent_t ev_stage[RP_STAGE_EVENTS];             // stage timing (rp_debug_set_stage_timing); null when off
@@ -243,6 +246,8 @@ int rp_launch_select(rp_ctx *c, int *lay, int *out, const i64 *score, int n_proj
                      int *n_distinct, i64 *dist);
 bool rp_uses_wpc(const RpDims &dm);
 int rp_launch_anneal_level(rp_ctx *c, int level, int n_levels, const rp_anneal_params *prm, u64 rho_q32, u64 guide_q32);
+int rp_launch_anneal_all(rp_ctx *c, int n_levels, const rp_anneal_params *prm, u64 rho_q32, u64 guide_q32, int *done);
+int rp_upload_levels(rp_ctx *c, int n_levels);
 int rp_launch_validate(rp_ctx *c);
 int rp_anneal_smem_bytes(const rp_ctx *c, int *threads, size_t *bytes);
 

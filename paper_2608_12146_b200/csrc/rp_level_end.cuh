@@ -82,11 +82,10 @@ __device__ __forceinline__ void le_weights(const i64 (&e)[U], i64 emin, u64 M, u
 
 // Inclusive prefix sums F[j] of the weights, U consecutive members per thread and round.
 template <int U>
-__device__ __forceinline__ void le_prefix_weights(const AnnealArgs &A, int tid, int nt, i64 emin, u64 M, u64 *F,
+__device__ __forceinline__ void le_prefix_weights(int P, const i64 *term, u64 cq, int tid, int nt, i64 emin, u64 M, u64 *F,
                                                   u64 *rsum, u64 *carry_s, bool have_e = false, i64 e_mine = 0)
 {
     const int lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
-    const int P = A.Ppop;
     for (int base = 0; base < P; base += nt * U) {
         const int j0 = base + tid * U;
         i64 e[U];
@@ -95,10 +94,10 @@ __device__ __forceinline__ void le_prefix_weights(const AnnealArgs &A, int tid, 
         for (int u = 0; u < U; ++u) {
             const int j = j0 + u;
             if (U == 1 && have_e) e[u] = (j < P) ? e_mine : emin;       // member tid's energy is still in a register
-            else e[u] = (j < P) ? rp_energy(LE_LD(A.term[3 * (size_t)j]), LE_LD(A.term[3 * (size_t)j + 1]), LE_LD(A.term[3 * (size_t)j + 2]))
+            else e[u] = (j < P) ? rp_energy(LE_LD(term[3 * (size_t)j]), LE_LD(term[3 * (size_t)j + 1]), LE_LD(term[3 * (size_t)j + 2]))
                                 : emin;
         }
-        le_weights<U>(e, emin, M, A.cq, w);
+        le_weights<U>(e, emin, M, cq, w);
         u64 v = 0;
 #pragma unroll
         for (int u = 0; u < U; ++u) { if (j0 + u >= P) w[u] = 0; v += w[u]; w[u] = v; }     // thread-local inclusive sums
@@ -291,9 +290,9 @@ __device__ __forceinline__ void rp_level_end(const AnnealArgs &A, int tid, int n
     if (tid == 0) carry_s = 0;
     __syncthreads();
     const u64 M = (u64)(emin > A.dm.SC ? emin : A.dm.SC);
-    if (P <= nt) le_prefix_weights<1>(A, tid, nt, emin, M, F, rsum, &carry_s, true, e_first);
-    else if (P <= 2 * nt) le_prefix_weights<2>(A, tid, nt, emin, M, F, rsum, &carry_s);
-    else le_prefix_weights<4>(A, tid, nt, emin, M, F, rsum, &carry_s);
+    if (P <= nt) le_prefix_weights<1>(P, A.term, A.cq, tid, nt, emin, M, F, rsum, &carry_s, true, e_first);
+    else if (P <= 2 * nt) le_prefix_weights<2>(P, A.term, A.cq, tid, nt, emin, M, F, rsum, &carry_s);
+    else le_prefix_weights<4>(P, A.term, A.cq, tid, nt, emin, M, F, rsum, &carry_s);
     const u64 Ftot = F[P - 1];
     const u64 u0 = (u64)(((unsigned __int128)A.resample_x * Ftot) >> 32);
     // The cell bookkeeping further down works in shared memory when 8*P ints fit: ancestors and

@@ -173,13 +173,16 @@ def test_philox_against_the_curand_header(tmp_path):
         assert (out[i] == oracle.philox4x32_10(ctr[i], key)).all()
 
 
+@pytest.mark.parametrize("per_level", [2, 1], ids=["one_launch", "launch_per_level"])
 @pytest.mark.parametrize("name", ["tiny", "medium"])
-def test_named_window_full_budget(name):
-    """The two windows the oracle finishes in seconds, at their full population and sweeps."""
+def test_named_window_full_budget(name, per_level):
+    """The two windows the oracle finishes in seconds, at their full population and sweeps: all
+    levels in one launch (every chain is resident at once), and one launch per level."""
     w = make_window(name)
     s = w.spec
     ref = oracle_front(w)
     ctx = load(w, device_inputs=(name == "medium"))
+    rp.rp_debug_set_knob(ctx, "LAUNCH_PER_LEVEL", per_level)
     check_front(w, ctx, ref)
     check_eval(w, ctx, ref, None)
     check_anneal(w, ctx, ref, None, s.pop_size, s.n_levels, s.steps_per_level)
@@ -213,6 +216,39 @@ def test_edge_shapes(spec):
     check_eval(w, ctx, ref, edp)
     want, stats = check_anneal(w, ctx, ref, edp, 24, 8, 50, t_ratio=0.6)
     assert stats.accepted > 50
+    rp.rp_destroy(ctx)
+
+
+@pytest.mark.parametrize("per_level", [2, 1], ids=["one_launch", "launch_per_level"])
+def test_resampling_under_selection_pressure_small_population(per_level):
+    """A cold schedule on a window whose samples really differ: resampling replaces many members
+    every level, so chains adopt other members' states (and others keep theirs on chip when all
+    levels run in one launch); several rp_anneal calls in a row continue from one another."""
+    w = make_window(custom_spec("pressure", 140, 6, 32, 2, 4096, 4, 8, 100, 400, data_seed=321))
+    s = w.spec
+    edp = [0, 1, 1, 0]
+    ref = oracle_front(w, edp, 3)
+    ctx = load(w, pop=100, edp=edp, min_rows=3)
+    rp.rp_debug_set_knob(ctx, "LAUNCH_PER_LEVEL", per_level)
+    check_front(w, ctx, ref)
+    want, stats = check_anneal(w, ctx, ref, edp, 100, 12, 60, t_ratio=0.5, t0=2e-5, check_members=3)
+    anc = want["anc"]
+    assert any(len(set(a.tolist())) < 60 for a in anc) and stats.gather_bytes > 0
+    again = oracle.anneal(w.lengths, ref["q"], want["final_pop"], ref["R"], s.token_cap, s.dp_width, n_levels=5,
+                          steps=33, t0=1e-5, t_ratio=0.7, p_reloc=0.4, p_guide=0.8, seed=s.anneal_seed,
+                          edp_of_dp=edp, alpha=s.alpha, beta=s.beta)
+    rp.rp_anneal(ctx, n_levels=5, steps_per_level=33, t0=1e-5, t_ratio=0.7, p_reloc=0.4, p_guide=0.8)
+    assert (rp.rp_debug_dump(ctx, "TRACE_TERM", (5, 100, 3), np.int64) == again["term"]).all()
+    assert (rp.rp_debug_dump(ctx, "TRACE_ANC", (4, 100), np.int32) == again["anc"]).all()
+    assert (rp.rp_debug_dump(ctx, "POPULATION", (100, s.n_samples), np.int32) == again["final_pop"]).all()
+    layout, fx, _ = rp.rp_best(ctx)
+    best = min((tuple(want["best_score"]), 0), (tuple(again["best_score"]), 1))
+    assert tuple(fx) == best[0]
+    assert (layout == (want, again)[best[1]]["best_layout"]).all()
+    G = 2
+    for j in (0, 57, 99):
+        ev = oracle.eval_layouts(w.lengths, ref["q"], again["final_pop"][j], ref["R"], s.token_cap, s.dp_width, edp, s.alpha, s.beta)
+        assert (rp.rp_debug_dump(ctx, "W", (ref["R"], G, s.n_layers, s.ep_width), np.int32, index=j) == ev["W"][0]).all()
     rp.rp_destroy(ctx)
 
 
@@ -297,6 +333,7 @@ def test_level_barrier_paths_on_small_windows(spec, cap):
     for slices in ((1, 2) if L * P > 512 else (0,)):       # cooperative kernel: rank loads as shared slices, and as cells
         ctx = load(w, pop=pop, edp=edp, min_rows=min_rows)
         rp.rp_debug_set_knob(ctx, "BARRIER_WORKSPACE", cap)
+        rp.rp_debug_set_knob(ctx, "LAUNCH_PER_LEVEL", 1)    # the barrier in question is the one between launches
         rp.rp_debug_set_knob(ctx, "RANK_LOAD_SLICES", slices)
         check_front(w, ctx, ref)
         want, stats = check_anneal(w, ctx, ref, edp, pop, 10, 40, t_ratio=0.6, check_members=2)
