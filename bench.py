@@ -456,8 +456,21 @@ def seeding_stages(rp, torch, name, dev, reps=3):
             if key == "select_population":
                 n_distinct = int(out[0])
         rp.rp_destroy(ctx)
+    # Algorithm 2 as one call: M candidates (here as many as members), selected down to the population
+    ctx = rp.rp_window_load(t_dev, a_dev, top_k=s.top_k, token_cap=s.token_cap, dp_width=s.dp_width,
+                            ep_width=s.ep_width, pop_size=s.pop_size, alpha=s.alpha, beta=s.beta, seed=s.anneal_seed)
+    rp.rp_place_experts(ctx)
+    rp.rp_pack_rows(ctx)
+    m_cand = min(s.pop_size, 256)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    nd_all, _ = rp.rp_init_population(ctx, m_cand, 4, 8, 1 << 16)
+    e1.record()
+    e1.synchronize()
+    rp.rp_destroy(ctx)
     return {"workload": name, "ms": ms, "n_distinct": n_distinct, "population": s.pop_size,
-            "choice_width": 4, "n_proj": 8, "eta_q16": 1 << 16}
+            "choice_width": 4, "n_proj": 8, "eta_q16": 1 << 16,
+            "init_population": {"candidates": m_cand, "n_distinct": nd_all, "ms": e0.elapsed_time(e1)}}
 
 
 def l2_read_rate(rp, mib=32, reps=50):
@@ -576,7 +589,7 @@ def run_cuda(args):
             line["eval_population"] = [eval_stage(rp, torch, n, dev, l2) for n in ("medium", "large", "wide")]
             line["concurrent_plans"] = [concurrent_plans(rp, torch, "medium", dev, n, 200) for n in (1, 2, 4)]
             line["single_plan_latency"] = [one_launch_latency(rp, torch, n, dev) for n in ("tiny", "medium")]
-            line["seeding_stages"] = seeding_stages(rp, torch, "medium", dev)
+            line["seeding_stages"] = [seeding_stages(rp, torch, n, dev, reps=(3 if n == "medium" else 1)) for n in ("medium", "heavy")]
             line["mechanism_diagnostics"] = [mechanism_diagnostics(rp, torch, n, dev) for n in ("medium", "large")]
         print(json.dumps(line))
     if dist is not None:

@@ -175,6 +175,22 @@ int rp_pair_population(rp_ctx *ctx, int32_t choice_width, int32_t *n_changed);
  *   former member index of every new member (nullable). */
 int rp_select_population(rp_ctx *ctx, int32_t n_proj, int64_t eta_q16, int32_t *n_distinct, int32_t *order);
 
+/* Algorithm 2 as one operation (Section 4.1.1, all lines): M = n_candidates fixed-row candidates,
+ *   candidate 0 = x_length (the length-only seed),
+ *   candidate 1 = x_paired = the lower-scoring of x_length and EDPAwarePair(x_length) (x_length on ties),
+ *   candidate t >= 2 = EDPAwarePair(trial t), trial t = WindowShuffle -> RandomizedBestFit with the
+ *     random streams of member t of rp_seed_population / rp_pair_population (a trial with no feasible
+ *     cell falls back to the length-only seed before it is paired),
+ * then CanonicalMap over all M and QualityDiversitySelect as in rp_select_population; population
+ * member m becomes the (m mod n_distinct)-th selected plan.  Between rp_pack_rows and rp_anneal;
+ * replaces whatever the population held.  The incumbent becomes the best member.
+ *   n_candidates in [2, 65536] (may be smaller or larger than the population); choice_width in
+ *   [1, 32]; n_proj in [1, 64]; eta_q16 >= 0.  n_distinct: HOST out (nullable); picked: HOST out
+ *   [P_pop], candidate index of every member (nullable).
+ * Cost grows with the square of the number of distinct candidates (see rp_select_population). */
+int rp_init_population(rp_ctx *ctx, int32_t n_candidates, int32_t choice_width, int32_t n_proj, int64_t eta_q16,
+                       int32_t *n_distinct, int32_t *picked);
+
 /* Full evaluation of layouts (Section 3.4-3.5: Eqs. cell-token-statistics,
  * stage-aware-attention, row-expert-load, row-expert-cost, lexicographic-score).
  *   layouts [n][N] int32 cell ids, or NULL to score the current population (n = pop_size).

@@ -22,7 +22,7 @@ STATUS_NAMES = {0: "RP_OK", -1: "RP_ERR_ARG", -2: "RP_ERR_SHAPE", -3: "RP_ERR_CO
                 -8: "RP_ERR_TIMEOUT", -9: "RP_ERR_INVALID_PLAN"}
 RP_OK = 0
 
-EXPORTS = ("rp_window_load", "rp_place_experts", "rp_pack_rows", "rp_seed_population", "rp_pair_population", "rp_select_population", "rp_eval_population", "rp_eval_layouts_noalloc", "rp_diagnostics", "rp_anneal",
+EXPORTS = ("rp_window_load", "rp_place_experts", "rp_pack_rows", "rp_seed_population", "rp_pair_population", "rp_select_population", "rp_init_population", "rp_eval_population", "rp_eval_layouts_noalloc", "rp_diagnostics", "rp_anneal",
            "rp_best", "rp_destroy", "rp_release_cached_memory", "rp_strerror", "rp_last_cuda_error", "rp_debug_dump",
            "rp_debug_set_trace", "rp_debug_set_knob", "rp_debug_set_stage_timing", "rp_debug_stage_times",
            "rp_debug_nl2", "rp_debug_exp2neg", "rp_debug_philox", "rp_debug_launch_count", "rp_debug_l2_read_rate")
@@ -84,6 +84,7 @@ def lib():
         L.rp_seed_population.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_int32)]
         L.rp_pair_population.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_int32)]
         L.rp_select_population.argtypes = [C.c_void_p, C.c_int32, C.c_int64, C.POINTER(C.c_int32), C.c_void_p]
+        L.rp_init_population.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int64, C.POINTER(C.c_int32), C.c_void_p]
         L.rp_eval_population.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
         L.rp_eval_layouts_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
         L.rp_diagnostics.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(rp_diag)]
@@ -208,6 +209,15 @@ def rp_select_population(ctx: Context, n_proj: int = 8, eta_q16: int = 1 << 16):
     order = np.zeros(ctx.cfg.pop_size, np.int32)
     _check(lib().rp_select_population(ctx.handle, n_proj, eta_q16, C.byref(nd), _ptr(order)), "rp_select_population")
     return int(nd.value), order
+
+
+def rp_init_population(ctx: Context, n_candidates: int, choice_width: int = 4, n_proj: int = 8, eta_q16: int = 1 << 16):
+    """Algorithm 2 over n_candidates fixed-row candidates; returns (n_distinct, picked [P_pop])."""
+    nd = C.c_int32(0)
+    picked = np.zeros(ctx.cfg.pop_size, np.int32)
+    _check(lib().rp_init_population(ctx.handle, n_candidates, choice_width, n_proj, eta_q16, C.byref(nd), _ptr(picked)),
+           "rp_init_population")
+    return int(nd.value), picked
 
 
 def rp_eval_population(ctx: Context, layouts=None, score_fx=None, score_f64=None):

@@ -454,6 +454,8 @@ __global__ void k_init_population(int P, int N, int *__restrict__ anc, int *__re
     if (x == 0) *done = 0;
 }
 
+static int build_population(rp_ctx *c);
+
 extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
 {
     if (!c) return RP_ERR_ARG;
@@ -472,6 +474,18 @@ extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
     c->Rstar = po[0]; c->certified = po[1];
     dm.R = po[0]; dm.K = dm.R * dm.D; dm.RG = dm.R * dm.G;
     if (dm.K > 65535) return RP_ERR_RANGE;
+    RP_TRY(build_population(c));
+    if (n_rows) *n_rows = c->Rstar;
+    if (certified) *certified = c->certified;
+    c->stage = 3;
+    return RP_OK;
+}
+
+// Buffers of a population of c->Ppop members for the row count in c->dm, every member a copy of the
+// length-only seed (evaluated once into slot 0, which all slots descend from); the seed is the incumbent.
+static int build_population(rp_ctx *c)
+{
+    RpDims &dm = c->dm;
     rp_decide_layouts(c);
     int nt; size_t smem;
     rp_anneal_smem_bytes(c, &nt, &smem);
@@ -531,9 +545,6 @@ extern "C" int rp_pack_rows(rp_ctx *c, int32_t *n_rows, int32_t *certified)
         RP_CUDA(cudaGetLastError());
     }
     stage_mark(c, RP_EV_SEED_1, c->stream);
-    if (n_rows) *n_rows = c->Rstar;
-    if (certified) *certified = c->certified;
-    c->stage = 3;
     return RP_OK;
 }
 
@@ -736,6 +747,106 @@ extern "C" int rp_select_population(rp_ctx *c, int32_t n_proj, int64_t eta_q16, 
     free(h);
     dev_free(c, lay); dev_free(c, out); dev_free(c, d_order); dev_free(c, d_nd);
     if (!c->trace_on) { dev_free(c, c->d_sel_dist); c->d_sel_dist = nullptr; }      // kept for inspection only
+    if (e != cudaSuccess) { g_rp_last_cuda_error = (int)e; return RP_ERR_CUDA; }
+    return st;
+}
+
+// Candidate 1 of Algorithm 2: the better of the length-only seed and its pairing (the seed on ties).
+__global__ void k_keep_better_of_seed(const int *__restrict__ seed_layout, const i64 *__restrict__ seed_score,
+                                      int *__restrict__ lay1, const i64 *__restrict__ score1, int N)
+{
+    const bool paired_wins = rp_lex_less(score1[0], score1[1], score1[2], seed_score[0], seed_score[1], seed_score[2]);
+    if (paired_wins) return;
+    for (int i = threadIdx.x; i < N; i += blockDim.x) lay1[i] = seed_layout[i];
+}
+__global__ void k_pick_rows(int N, const int *__restrict__ pick, const int *__restrict__ lay, int *__restrict__ out)
+{
+    const int *src = lay + (size_t)pick[blockIdx.x] * N;
+    for (int i = threadIdx.x; i < N; i += blockDim.x) out[(size_t)blockIdx.x * N + i] = src[i];
+}
+
+// Algorithm 2 as one operation over M candidates: x_length, x_paired = min_Score{x_length,
+// EDPAwarePair(x_length)}, M - 2 trials (WindowShuffle -> RandomizedBestFit -> EDPAwarePair),
+// CanonicalMap over all of them and QualityDiversitySelect down to the population, repeated
+// cyclically when fewer distinct plans exist.  The candidates are worked on as a population of M
+// members of their own; the population proper is rebuilt from the selected ones afterwards.
+extern "C" int rp_init_population(rp_ctx *c, int32_t n_candidates, int32_t choice_width, int32_t n_proj, int64_t eta_q16,
+                                  int32_t *n_distinct, int32_t *picked)
+{
+    if (!c) return RP_ERR_ARG;
+    if (c->stage != 3) return RP_ERR_STATE;
+    if (n_candidates < 2 || n_candidates > (1 << 16) || choice_width < 1 || choice_width > 32) return RP_ERR_ARG;
+    if (n_proj < 1 || n_proj > 64 || eta_q16 < 0 || eta_q16 > ((int64_t)1 << 40)) return RP_ERR_ARG;
+    const RpDims &dm = c->dm;
+    if (dm.K > 2048) return RP_ERR_RANGE;
+    if ((double)dm.C * dm.C * dm.D * 65536.0 >= 9.0e18) return RP_ERR_RANGE;
+    const int P = c->Ppop, M = n_candidates;
+    int *lay = nullptr, *out = nullptr, *sel = nullptr, *ok = nullptr, *prof = nullptr, *d_order = nullptr, *d_nd = nullptr;
+    int *fin = nullptr, *d_pick = nullptr;
+    i64 *dist = nullptr;
+    int *h = (int *)malloc(sizeof(int) * ((size_t)M + 1 + P));
+    int st = RP_OK;
+    cudaError_t e = cudaSuccess;
+    // the candidates as a population of their own
+    c->Ppop = M;
+    st = build_population(c);
+    do {
+        if (st != RP_OK) break;
+        if ((st = dev_alloc(c, &lay, (size_t)M * dm.N)) != RP_OK) break;
+        if ((st = dev_alloc(c, &out, (size_t)M * dm.N)) != RP_OK) break;
+        if ((st = dev_alloc(c, &sel, (size_t)M * dm.N)) != RP_OK) break;
+        if ((st = dev_alloc(c, &ok, M)) != RP_OK) break;
+        if ((st = dev_alloc(c, &d_order, M)) != RP_OK) break;
+        if ((st = dev_alloc(c, &d_nd, 1)) != RP_OK) break;
+        if ((st = dev_alloc(c, &dist, (size_t)M * M)) != RP_OK) break;
+        const int batch = M - 1 < 1024 ? M - 1 : 1024;
+        if ((st = dev_alloc(c, &prof, (size_t)batch * dm.K * dm.LP)) != RP_OK) break;
+        // trials 2 .. M-1; candidates 0 and 1 start as the length-only seed
+        if ((st = rp_launch_seed_trials(c, choice_width, lay, ok)) != RP_OK) break;
+        if ((e = cudaMemcpyAsync(lay + dm.N, c->d_seed_layout, sizeof(int) * dm.N, cudaMemcpyDeviceToDevice, c->stream)) != cudaSuccess) break;
+        // pairing of every candidate but x_length
+        if ((e = cudaMemcpyAsync(out, lay, sizeof(int) * dm.N, cudaMemcpyDeviceToDevice, c->stream)) != cudaSuccess) break;
+        for (int first = 1; st == RP_OK && first < M; first += batch)
+            st = rp_launch_edp_pair(c, lay, out, prof, first, M - first < batch ? M - first : batch, choice_width);
+        if (st != RP_OK) break;
+        // x_paired: the pairing of the seed only if it scores lower
+        if ((st = ensure_eval_scratch(c, (size_t)M, false)) != RP_OK) break;
+        if ((st = rp_launch_cells_from_layouts(c, out + dm.N, 1, c->d_eval_cells)) != RP_OK) break;
+        if ((st = rp_launch_eval(c, c->d_eval_cells, 1, nullptr, nullptr, c->d_eval_score, nullptr)) != RP_OK) break;
+        k_keep_better_of_seed<<<1, 256, 0, c->stream>>>(c->d_seed_layout, c->d_seed_score, out + dm.N, c->d_eval_score, dm.N);
+        ++g_rp_launches;
+        // all candidates scored and installed, then the selection over them
+        if ((st = install_population(c, out)) != RP_OK) break;
+        if ((st = rp_launch_select(c, out, sel, c->d_eval_score, n_proj, eta_q16, d_order, d_nd, dist)) != RP_OK) break;
+        if ((e = cudaMemcpyAsync(h, d_order, sizeof(int) * M, cudaMemcpyDeviceToHost, c->stream)) != cudaSuccess) break;
+        if ((e = cudaMemcpyAsync(h + M, d_nd, sizeof(int), cudaMemcpyDeviceToHost, c->stream)) != cudaSuccess) break;
+        if ((e = cudaStreamSynchronize(c->stream)) != cudaSuccess) break;
+        const int nd = h[M];
+        if (nd < 1) { st = RP_ERR_STATE; break; }
+        int *pick = h + M + 1;
+        for (int m = 0; m < P; ++m) pick[m] = h[m % nd];         // the selection order, repeated cyclically
+        if ((st = dev_alloc(c, &fin, (size_t)P * dm.N)) != RP_OK) break;
+        if ((st = dev_alloc(c, &d_pick, P)) != RP_OK) break;
+        if ((e = cudaMemcpyAsync(d_pick, pick, sizeof(int) * P, cudaMemcpyHostToDevice, c->stream)) != cudaSuccess) break;
+        k_pick_rows<<<P, 256, 0, c->stream>>>(dm.N, d_pick, out, fin);
+        ++g_rp_launches;
+        if ((e = cudaStreamSynchronize(c->stream)) != cudaSuccess) break;      // `pick` is pageable memory
+        // the population proper
+        c->Ppop = P;
+        if ((st = build_population(c)) != RP_OK) break;
+        if ((st = install_population(c, fin)) != RP_OK) break;
+        if ((e = cudaStreamSynchronize(c->stream)) != cudaSuccess) break;
+        if (n_distinct) *n_distinct = nd;
+        if (picked) memcpy(picked, pick, sizeof(int) * P);
+    } while (0);
+    dev_free(c, lay); dev_free(c, out); dev_free(c, sel); dev_free(c, ok); dev_free(c, prof); dev_free(c, d_order); dev_free(c, d_nd);
+    dev_free(c, dist); dev_free(c, fin); dev_free(c, d_pick);
+    free(h);
+    if (c->Ppop != P) {                      // failed half way: back to a seed population of the right size
+        c->Ppop = P;
+        const int st2 = build_population(c);
+        if (st == RP_OK && e == cudaSuccess) st = st2;
+    }
     if (e != cudaSuccess) { g_rp_last_cuda_error = (int)e; return RP_ERR_CUDA; }
     return st;
 }

@@ -551,6 +551,66 @@ def test_canonical_map_and_quality_diversity_selection(case, eta):
     rp.rp_destroy(ctx)
 
 
+def oracle_init_population(w, ref, edp, M, pop, width, n_proj, eta):
+    """Algorithm 2 over M candidates, composed from the oracle's stages: x_length, x_paired, M - 2
+    trials (shuffle -> best fit -> pairing), CanonicalMap + QualityDiversitySelect, cyclic fill."""
+    s = w.spec
+    R, D = ref["R"], s.dp_width
+    lays, _ = oracle.seed_trials(w.lengths, ref["seed"], R, s.token_cap, D, M, width, s.anneal_seed)
+    lays[1] = ref["seed"]                                  # candidate 1 starts as the length-only seed too
+    cand = oracle.edp_pair(ref["q"], lays, R, D, width, s.anneal_seed, edp)
+    score = lambda l: oracle.eval_layouts(w.lengths, ref["q"], l, R, s.token_cap, D, edp, s.alpha, s.beta)["score"]
+    if not tuple(score(cand[1])[0]) < tuple(score(ref["seed"])[0]):
+        cand[1] = ref["seed"]                              # x_paired = min_Score{x_length, pairing of x_length}
+    sel = oracle.select_population(w.lengths, ref["q"], cand, score(cand), R, s.token_cap, D, s.top_k, n_proj, eta,
+                                   s.anneal_seed, edp)
+    nd = sel["n_distinct"]
+    picked = np.array([sel["order"][m % nd] for m in range(pop)], np.int32)
+    return nd, picked, cand[picked]
+
+
+@pytest.mark.parametrize("case,M,pop", [("shared", 60, 24), ("shared", 10, 24), ("interleaved", 33, 33), ("medium", 80, 48),
+                                        ("identity", 2, 5), ("copies", 40, 16)])
+def test_algorithm_2_as_one_call(case, M, pop):
+    """rp_init_population against the composition of the oracle's stages: how many candidates are
+    distinct, which candidate every member is, the members' layouts and scores, the incumbent, and
+    the annealing that starts from them; with fewer, as many and more candidates than members."""
+    edp, min_rows, width, n_proj, eta = None, 3, 3, 6, 1 << 16
+    if case == "medium":
+        w = make_window("medium")
+        min_rows = 0
+    elif case in ("shared", "copies"):
+        w = make_window(custom_spec("a2_shared", 96, 5, 16, 2, 4096, 4, 4, pop, 400, data_seed=45))
+        edp = [0, 0, 1, 1]
+        if case == "copies":
+            width = 1                                       # no randomness: few distinct candidates
+    elif case == "interleaved":
+        w = make_window(custom_spec("a2_inter", 120, 7, 24, 3, 4096, 6, 6, pop, 400, data_seed=46))
+        edp, min_rows = [0, 1, 2, 0, 1, 2], 2
+    else:
+        w = make_window(custom_spec("a2_ident", 77, 3, 12, 2, 3000, 3, 3, pop, 400, data_seed=48))
+        min_rows = 4
+    s = w.spec
+    ref = oracle_front(w, edp, min_rows)
+    ctx = load(w, pop=pop, edp=edp, min_rows=min_rows)
+    check_front(w, ctx, ref)
+    nd_want, picked_want, lays_want = oracle_init_population(w, ref, edp, M, pop, width, n_proj, eta)
+    nd, picked = rp.rp_init_population(ctx, M, width, n_proj, eta)
+    assert nd == nd_want and (picked == picked_want).all()
+    if case == "copies":
+        assert nd < M
+    got = rp.rp_debug_dump(ctx, "POPULATION", (pop, s.n_samples), np.int32)
+    assert (got == lays_want).all()
+    ev = oracle.eval_layouts(w.lengths, ref["q"], lays_want, ref["R"], s.token_cap, s.dp_width, edp, s.alpha, s.beta)
+    fx, _ = rp.rp_eval_population(ctx)
+    assert (fx == ev["score"]).all()
+    best = min(range(pop), key=lambda j: (tuple(ev["score"][j]), j))
+    layout, bfx, _ = rp.rp_best(ctx)
+    assert (layout == lays_want[best]).all() and tuple(bfx) == tuple(ev["score"][best])
+    check_anneal(w, ctx, ref, edp, pop, 3, 40, t_ratio=0.5, check_members=2, init=lays_want)
+    rp.rp_destroy(ctx)
+
+
 def test_fuzz_random_small_windows():
     """Random shapes and search parameters (rank counts 1..48 including non powers of two, shared
     and interleaved shards, swap-only and relocation-only proposals, unguided and fully guided,
@@ -737,13 +797,15 @@ def test_bad_inputs_are_host_side_errors():
         rp.rp_anneal(ctx, n_levels=1, steps_per_level=1, t0=1e-3, t_ratio=0.5, p_reloc=0.2, p_guide=0.8)
     assert e.value.status == -7
     for call in (lambda: rp.rp_seed_population(ctx, 4), lambda: rp.rp_pair_population(ctx, 4),
-                 lambda: rp.rp_select_population(ctx, 4, 1 << 16)):
+                 lambda: rp.rp_select_population(ctx, 4, 1 << 16), lambda: rp.rp_init_population(ctx, 8)):
         with pytest.raises(rp.RpError) as e:
             call()                                                           # before rp_pack_rows
         assert e.value.status == -7
     R, _ = rp.rp_pack_rows(ctx)
     for call in (lambda: rp.rp_seed_population(ctx, 0), lambda: rp.rp_pair_population(ctx, 33),
-                 lambda: rp.rp_select_population(ctx, 0, 1 << 16), lambda: rp.rp_select_population(ctx, 4, -1)):
+                 lambda: rp.rp_select_population(ctx, 0, 1 << 16), lambda: rp.rp_select_population(ctx, 4, -1),
+                 lambda: rp.rp_init_population(ctx, 1), lambda: rp.rp_init_population(ctx, 8, 0),
+                 lambda: rp.rp_init_population(ctx, 8, 4, 65), lambda: rp.rp_init_population(ctx, 8, 4, 8, -1)):
         with pytest.raises(rp.RpError) as e:
             call()
         assert e.value.status == -1
