@@ -430,7 +430,7 @@ def one_launch_latency(rp, torch, name, dev, reps=200):
     return out
 
 
-def seeding_stages(rp, torch, name, dev, reps=3):
+def seeding_stages(rp, torch, name, dev, reps=3, per_stage=True):
     """Context figure: device time of the optional seeding stages (trial loop, pairing, canonical
     map + quality-diversity selection) on the named window, mean over `reps` fresh contexts."""
     w = make_window(SPECS[name])
@@ -439,7 +439,7 @@ def seeding_stages(rp, torch, name, dev, reps=3):
     a_dev = torch.from_numpy(w.demand).to(dev)
     ms = {"seed_population": 0.0, "pair_population": 0.0, "select_population": 0.0}
     n_distinct = 0
-    for _ in range(reps):
+    for _ in range(reps if per_stage else 0):      # (the selection grows with the square of the population: not on the big windows)
         ctx = rp.rp_window_load(t_dev, a_dev, top_k=s.top_k, token_cap=s.token_cap, dp_width=s.dp_width,
                                 ep_width=s.ep_width, pop_size=s.pop_size, alpha=s.alpha, beta=s.beta, seed=s.anneal_seed)
         rp.rp_place_experts(ctx)
@@ -468,7 +468,7 @@ def seeding_stages(rp, torch, name, dev, reps=3):
     e1.record()
     e1.synchronize()
     rp.rp_destroy(ctx)
-    return {"workload": name, "ms": ms, "n_distinct": n_distinct, "population": s.pop_size,
+    return {"workload": name, "ms": ms if per_stage else None, "n_distinct": n_distinct, "population": s.pop_size,
             "choice_width": 4, "n_proj": 8, "eta_q16": 1 << 16,
             "init_population": {"candidates": m_cand, "n_distinct": nd_all, "ms": e0.elapsed_time(e1)}}
 
@@ -589,7 +589,7 @@ def run_cuda(args):
             line["eval_population"] = [eval_stage(rp, torch, n, dev, l2) for n in ("medium", "large", "wide")]
             line["concurrent_plans"] = [concurrent_plans(rp, torch, "medium", dev, n, 200) for n in (1, 2, 4)]
             line["single_plan_latency"] = [one_launch_latency(rp, torch, n, dev) for n in ("tiny", "medium")]
-            line["seeding_stages"] = [seeding_stages(rp, torch, n, dev, reps=(3 if n == "medium" else 1)) for n in ("medium", "heavy")]
+            line["seeding_stages"] = [seeding_stages(rp, torch, "medium", dev), seeding_stages(rp, torch, "heavy", dev, per_stage=False)]
             line["mechanism_diagnostics"] = [mechanism_diagnostics(rp, torch, n, dev) for n in ("medium", "large")]
         print(json.dumps(line))
     if dist is not None:

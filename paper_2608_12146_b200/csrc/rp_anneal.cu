@@ -40,7 +40,7 @@ struct ChainB {                 // bookkeeping of the chain within this level
 // Cooperative chain kernel for bandwidth-bound windows (L*P > 512): all NT threads score one
 // candidate at a time (two L*P slices of W from global memory plus the moved samples' demand
 // rows, 16-byte loads); the leading warp rebuilds the score and decides.
-template <int NT, int MINB, bool SL>
+template <int NT, int MINB, bool SL, bool ALIAS>
 __global__ void __launch_bounds__(NT, MINB)
 k_anneal_level(const AnnealArgs A)
 {
@@ -51,10 +51,14 @@ k_anneal_level(const AnnealArgs A)
     char *sm_blob = (char *)smraw;
     char *sm_static = sm_blob + A.bl.bytes;
     int *scratch = (int *)(sm_static + A.sl.bytes);
+    // Per-cell caches of the proposal keys (attention cost of the cell, cost and attention part of its
+    // row-shard).  With one cell per row-shard (every DP slot its own shard) they equal the row-shard
+    // arrays of the blob; ALIAS then uses those arrays themselves and keeps no copy (chosen where the
+    // shared memory saved lets one more chain be resident per SM).
     i64 *attkey = (i64 *)(scratch + 2 * slice_pad);
     i64 *Jcell = attkey + dm.K;
     i64 *Acell = Jcell + dm.K;
-    i64 *red = Acell + dm.K;
+    i64 *red = ALIAS ? attkey : Acell + dm.K;
     StepRec *recs = (StepRec *)(red + 2 * (NT / 32));
     ChainB *chain = (ChainB *)(recs + SPEC);
     u64 *mbar = (u64 *)(chain + 1);
@@ -71,6 +75,7 @@ k_anneal_level(const AnnealArgs A)
     int *T = (int *)(sm_blob + A.bl.off_T);
     int *cnt = (int *)(sm_blob + A.bl.off_cnt);
     unsigned short *cell_of = (unsigned short *)(sm_blob + A.bl.off_cell);
+    if (ALIAS) { attkey = Afx; Jcell = Jfx; Acell = Afx; }
     int *wtab = (int *)(sm_blob + (SL ? A.bl.off_wtab : 0));          // slice mode: row-shard -> slice of the pool
     const int *dpl = (const int *)(sm_static + A.sl.off_dpl);
     const int *dpo = (const int *)(sm_static + A.sl.off_dpo);
@@ -111,11 +116,12 @@ k_anneal_level(const AnnealArgs A)
         rp_finish_level(A, tid, NT, smraw, A.smem_bytes);
         return;
     }
-    for (int c = tid; c < dm.K; c += NT) {
-        attkey[c] = aC * (i64)T[c] + bS * (i64)Q[c];
-        Jcell[c] = Jfx[rg_of[c]];
-        Acell[c] = Afx[rg_of[c]];
-    }
+    if (!ALIAS)
+        for (int c = tid; c < dm.K; c += NT) {
+            attkey[c] = aC * (i64)T[c] + bS * (i64)Q[c];
+            Jcell[c] = Jfx[rg_of[c]];
+            Acell[c] = Afx[rg_of[c]];
+        }
     if (tid == 0) {
         chain->B[0] = Sc[0]; chain->B[1] = Sc[1]; chain->B[2] = Sc[2];
         chain->dig = 0; chain->best_step = 0; chain->best_nlog = 0; chain->nlog = 0;
@@ -292,11 +298,12 @@ k_anneal_level(const AnnealArgs A)
                             cell_of[m.i] = (unsigned short)c2;
                             if (swap) cell_of[m.i2] = (unsigned short)c1;
                             T[c1] = (int)Ta; Q[c1] = (u64)Qa; T[c2] = (int)Tb; Q[c2] = (u64)Qb;
-                            attkey[c1] = aC * Ta + bS * Qa; attkey[c2] = aC * Tb + bS * Qb;
+                            if (!ALIAS) { attkey[c1] = aC * Ta + bS * Qa; attkey[c2] = aC * Tb + bS * Qb; }
                             if (!swap) { cnt[c1] -= 1; cnt[c2] += 1; }
                             Esum[rg1] = e1; Afx[rg1] = A1; Jfx[rg1] = J1n;
                             if (touchW) { Esum[rg2] = e2; Afx[rg2] = A2; Jfx[rg2] = J2n; }
-                            if (identity_edp) { Jcell[c1] = J1n; Acell[c1] = A1; Jcell[c2] = J2n; Acell[c2] = A2; }
+                            if (ALIAS) { }
+                            else if (identity_edp) { Jcell[c1] = J1n; Acell[c1] = A1; Jcell[c2] = J2n; Acell[c2] = A2; }
                             else {
                                 for (int x = dpo[g1]; x < dpo[g1 + 1]; ++x) { const int c = rowbase[c1] + dpl[x]; Jcell[c] = J1n; Acell[c] = A1; }
                                 for (int x = dpo[g2]; x < dpo[g2 + 1]; ++x) { const int c = rowbase[c2] + dpl[x]; Jcell[c] = J2n; Acell[c] = A2; }
@@ -452,6 +459,14 @@ int rp_launch_slice_gc(rp_ctx *c)
     return RP_OK;
 }
 
+// Resident chains per SM of the cooperative kernel: six (80 registers) keep the most bytes in
+// flight; windows whose rank loads per member pass a megabyte run faster with five (96 registers,
+// no spills; their working set misses L2 either way).
+static int rp_coop_chains_per_sm(const RpDims &dm)
+{
+    return ((size_t)dm.RG * dm.LP * sizeof(int) >= (1u << 20)) ? 5 : 6;
+}
+
 int rp_anneal_smem_bytes(const rp_ctx *c, int *threads, size_t *bytes)
 {
     const RpDims &dm = c->dm;
@@ -466,9 +481,16 @@ int rp_anneal_smem_bytes(const rp_ctx *c, int *threads, size_t *bytes)
     const size_t slice_pad = ((size_t)dm.LP + 3) & ~(size_t)3;
     size_t b = (size_t)c->bl.bytes + c->sl.bytes + sizeof(int) * 2 * slice_pad + sizeof(i64) * (3 * (size_t)dm.K + 2 * (nt / 32)) +
                sizeof(StepRec) * SPEC + sizeof(ChainB) + sizeof(u64) + sizeof(MoveS) * SPEC + (size_t)dm.RG * 5;
+    b = (b + 15) & ~(size_t)15;
+    // Without the per-cell key caches (possible with one cell per row-shard): taken when it lets
+    // more chains be resident per SM than the registers allow anyway.
+    const size_t b_alias = b - sizeof(i64) * 3 * (size_t)dm.K;
+    const int minb = rp_coop_chains_per_sm(dm);
+    const size_t room = 227 * 1024;
+    const bool alias = (dm.G == dm.D) && (room / (b + 1024) < (size_t)minb) && (room / (b_alias + 1024) > room / (b + 1024));
     *threads = nt;
-    *bytes = (b + 15) & ~(size_t)15;
-    return 0;
+    *bytes = alias ? b_alias : b;
+    return alias ? 2 : 0;
 }
 
 // Philox4x32-10 on the host (first output word): the resampling offset's random word depends only
@@ -570,32 +592,25 @@ int rp_launch_anneal_level(rp_ctx *c, int level, int n_levels, const rp_anneal_p
     if (rp_uses_slices(c->dm)) RP_TRY(rp_launch_slice_gc(c));
     if (use_wpc(c->dm)) return rp_launch_anneal_wpc(c, A);
     int nt; size_t smem;
-    rp_anneal_smem_bytes(c, &nt, &smem);
+    const bool alias = rp_anneal_smem_bytes(c, &nt, &smem) == 2;
     if (smem > 220 * 1024) return RP_ERR_RANGE;
     A.smem_bytes = (unsigned)smem;
-#define COOP_LAUNCH(MINB_, SL_)                                                                                 \
+#define COOP_LAUNCH(MINB_, SL_, ID_)                                                                                 \
     do {                                                                                                     \
         if (smem > 32 * 1024)                                                                                \
-            RP_CUDA(cudaFuncSetAttribute(k_anneal_level<128, MINB_, SL_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
-        k_anneal_level<128, MINB_, SL_><<<c->Ppop, 128, smem, c->stream>>>(A);                               \
+            RP_CUDA(cudaFuncSetAttribute(k_anneal_level<128, MINB_, SL_, ID_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+        k_anneal_level<128, MINB_, SL_, ID_><<<c->Ppop, 128, smem, c->stream>>>(A);                          \
     } while (0)
-    // Resident chains per SM: six (80 registers) keep the most bytes in flight; windows whose rank
-    // loads per member pass a megabyte run faster with five (their working set misses L2 either way,
-    // and fewer chains leave more of it to the demand rows).
-    int minb = ((size_t)c->dm.RG * c->dm.LP * sizeof(int) >= (1u << 20)) ? 5 : 6;
-    if (A.slices) {
-        switch (minb) {
-            case 5: COOP_LAUNCH(5, true); break;
-            case 4: COOP_LAUNCH(4, true); break;
-            default: COOP_LAUNCH(6, true); break;
-        }
-    } else {
-        switch (minb) {
-            case 5: COOP_LAUNCH(5, false); break;
-            case 4: COOP_LAUNCH(4, false); break;
-            default: COOP_LAUNCH(6, false); break;
-        }
+    const int minb = rp_coop_chains_per_sm(c->dm);
+#define COOP_PICK(SL_, ID_)                                  \
+    switch (minb) {                                          \
+        case 5: COOP_LAUNCH(5, SL_, ID_); break;             \
+        case 4: COOP_LAUNCH(4, SL_, ID_); break;             \
+        default: COOP_LAUNCH(6, SL_, ID_); break;            \
     }
+    if (A.slices) { if (alias) { COOP_PICK(true, true) } else { COOP_PICK(true, false) } }
+    else { if (alias) { COOP_PICK(false, true) } else { COOP_PICK(false, false) } }
+#undef COOP_PICK
 #undef COOP_LAUNCH
     ++g_rp_launches;
     RP_CUDA(cudaGetLastError());
