@@ -368,9 +368,10 @@ def measure(rp, torch, args, name, steps, min_seconds, dist, dev, local, cpu_sec
             "gpu_launches": int(launches), "clocks": clocks, "timed_region_s": res["wall"]}
 
 
-def concurrent_plans(rp, torch, name, dev, n_ctx, reps):
+def concurrent_plans(rp, torch, name, dev, n_ctx, reps, per_level=1):
     """Context figure: plans per second with `n_ctx` windows planned at once on separate streams and
-    contexts (the ABI allows it); reported beside the single-plan latency, never instead of it."""
+    contexts (the ABI allows it), with one launch per level (which lets the windows share the SMs) or
+    the default single launch; reported beside the single-plan latency, never instead of it."""
     import threading
     w = make_window(SPECS[name])
     s = w.spec
@@ -386,7 +387,7 @@ def concurrent_plans(rp, torch, name, dev, n_ctx, reps):
                     score_fx=torch.empty(3, dtype=torch.int64, device=dev),
                     score_f64=torch.empty(3, dtype=torch.float64, device=dev))
         for _ in range(n):
-            plan_once(rp, w, t_dev, a_dev, outs, streams[k])
+            plan_once(rp, w, t_dev, a_dev, outs, streams[k], knobs={"LAUNCH_PER_LEVEL": per_level})
 
     for n in (2, reps):                      # warm up, then time
         torch.cuda.synchronize()
@@ -398,7 +399,8 @@ def concurrent_plans(rp, torch, name, dev, n_ctx, reps):
             x.join()
         torch.cuda.synchronize()
         dt = time.perf_counter() - t0
-    return {"workload": name, "concurrent_contexts": n_ctx, "plans": n_ctx * reps, "plans_per_s": n_ctx * reps / dt,
+    return {"workload": name, "concurrent_contexts": n_ctx, "launch_per_level": per_level, "plans": n_ctx * reps,
+            "plans_per_s": n_ctx * reps / dt,
             "timing": "wall clock around host threads, one stream and context each"}
 
 
@@ -587,7 +589,7 @@ def run_cuda(args):
             l2 = l2_read_rate(rp)
             line["l2_read_gbs"] = l2
             line["eval_population"] = [eval_stage(rp, torch, n, dev, l2) for n in ("medium", "large", "wide")]
-            line["concurrent_plans"] = [concurrent_plans(rp, torch, "medium", dev, n, 200) for n in (1, 2, 4)]
+            line["concurrent_plans"] = [concurrent_plans(rp, torch, "medium", dev, n, 200, pl) for pl in (1, 0) for n in (1, 2, 4)]
             line["single_plan_latency"] = [one_launch_latency(rp, torch, n, dev) for n in ("tiny", "medium")]
             line["seeding_stages"] = [seeding_stages(rp, torch, "medium", dev), seeding_stages(rp, torch, "heavy", dev, per_stage=False)]
             line["mechanism_diagnostics"] = [mechanism_diagnostics(rp, torch, n, dev) for n in ("medium", "large")]

@@ -301,10 +301,9 @@ typedef enum {
  *   RP_KNOB_STALL_ONE_CHAIN: chain 0 waits once more, after its copies have landed, on a barrier
  *     phase that nothing completes: the wait runs out and rp_anneal returns RP_ERR_TIMEOUT.
  *   RP_KNOB_LAUNCH_PER_LEVEL: how rp_anneal launches windows whose chains can all be resident at
- *     once (rank loads on chip, at most 256 members).  0 = automatic: one launch for all levels up
- *     to 148 members, one launch per level above (two windows planned at once on two streams then
- *     still share the GPU); 1 = always one launch per level; 2 = one launch for all levels
- *     wherever possible (lowest latency of a single plan).
+ *     once (rank loads on chip, at most 256 members).  0 or 2 = one launch for all levels (lowest
+ *     latency of a single plan); 1 = one launch per level (two windows planned at once on two
+ *     streams then share the GPU, which two launches of the first kind cannot).
  *   RP_KNOB_RANK_LOAD_SLICES (set before rp_pack_rows): how windows with L*P > 512 keep the rank
  *     loads of the population.  0 or 1 = shared slices with copy-on-write (the default), 2 = one
  *     private cell per member, copied whole when resampling replaces the member. */

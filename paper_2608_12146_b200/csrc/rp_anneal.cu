@@ -575,10 +575,10 @@ int rp_upload_levels(rp_ctx *c, int n_levels)
 int rp_launch_anneal_all(rp_ctx *c, int n_levels, const rp_anneal_params *prm, u64 rho_q32, u64 guide_q32, int *done)
 {
     *done = 0;
-    // Automatic: only populations of at most one chain per SM, so that a second window planned at
-    // the same time on another stream still finds room (a launch whose chains wait for one another
-    // needs all of them resident at once, and two such launches do not share the SMs).
-    const bool wanted = c->knob_level_launches == 2 || (c->knob_level_launches == 0 && c->Ppop <= 148);
+    // Automatic: wherever it is possible (lowest latency of a plan).  A launch whose chains wait for
+    // one another needs all of them resident at once, so two such launches do not share the SMs: a
+    // caller that plans several windows at once on separate streams asks for one launch per level.
+    const bool wanted = c->knob_level_launches != 1;
     if (!use_wpc(c->dm) || !wanted || !c->d_levels) return RP_OK;
     AnnealArgs A;
     fill_args(c, 0, n_levels, prm, rho_q32, guide_q32, A);

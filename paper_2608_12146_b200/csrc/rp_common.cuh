@@ -169,7 +169,7 @@ struct rp_ctx {
     // trace of the last rp_anneal call
     int trace_levels;
     int trace_on;              // keep per-level traces (inspection hook; off by default)
-    int knob_level_launches;   // 0 = automatic, 1 = one launch per level, 2 = one launch for all levels wherever possible
+    int knob_level_launches;   // 1 = one launch per level even where one launch for all levels is possible
     int knob_slices;           // inspection hook: 0 = automatic, 1 = slices wherever the cooperative kernel runs, 2 = never
     int knob_le_ws_cap, knob_wait_polls, knob_stall;   // inspection hooks (rp_debug_set_knob); 0 = off
     cudaEvent_t ev_stage[RP_STAGE_EVENTS];             // stage timing (rp_debug_set_stage_timing); null when off
