@@ -231,7 +231,7 @@ def test_resampling_under_selection_pressure_small_population(per_level):
     ctx = load(w, pop=100, edp=edp, min_rows=3)
     rp.rp_debug_set_knob(ctx, "LAUNCH_PER_LEVEL", per_level)
     check_front(w, ctx, ref)
-    want, stats = check_anneal(w, ctx, ref, edp, 100, 12, 60, t_ratio=0.5, t0=2e-5, check_members=3)
+    want, stats = check_anneal(w, ctx, ref, edp, 100, 12, 300, t_ratio=0.5, t0=2e-5, check_members=3)    # 300 steps: two batches of step records
     anc = want["anc"]
     assert any(len(set(a.tolist())) < 60 for a in anc) and stats.gather_bytes > 0
     again = oracle.anneal(w.lengths, ref["q"], want["final_pop"], ref["R"], s.token_cap, s.dp_width, n_levels=5,
