@@ -133,10 +133,102 @@ k_check_reduce_vec(const int4 *__restrict__ a, const int *__restrict__ t, RpDims
     if (l == 0 && lane == 0 && tsum > 0) atomicAdd((u64 *)t_sum, (u64)tsum);      // tokens of this warp's samples, once
 }
 
+// The same pass as one sequential stream.  A CTA owns a range of samples, i.e. one contiguous
+// piece of the tensor; warp w of its NW warps owns the layers w, w + NW, ... (LW of them: L = NW*LW),
+// so that the warps of a CTA together read whole samples front to back while every warp keeps the
+// column sums of its own layers in registers.  SPI samples are in flight per warp at a time.
+template <int NQ, int LW, int NW, int SPI>
+__global__ void __launch_bounds__(NW * 32)
+k_check_reduce_seq(const int4 *__restrict__ a, const int *__restrict__ t, RpDims dm, int chunk,
+                   i64 *__restrict__ Lagg, int *__restrict__ status, i64 *__restrict__ t_sum)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int i0 = blockIdx.x * chunk;
+    const int i1 = min(dm.N, i0 + chunk);
+    const size_t row4 = (size_t)dm.E >> 2;
+    i64 acc[LW][NQ][4];
+#pragma unroll
+    for (int li = 0; li < LW; ++li)
+#pragma unroll
+        for (int c = 0; c < NQ; ++c) { acc[li][c][0] = 0; acc[li][c][1] = 0; acc[li][c][2] = 0; acc[li][c][3] = 0; }
+    i64 tsum = 0;
+    bool bad = false;
+    for (int ib = i0; ib < i1; ib += SPI) {
+        int4 v[SPI][LW][NQ];
+        int ti[SPI];
+#pragma unroll
+        for (int s = 0; s < SPI; ++s) {
+            const int i = min(ib + s, i1 - 1);                       // past the end: the last sample again, not counted
+            ti[s] = __ldg(t + i);
+#pragma unroll
+            for (int li = 0; li < LW; ++li) {
+                const int4 *row = a + ((size_t)i * dm.L + warp + li * NW) * row4;
+#pragma unroll
+                for (int c = 0; c < NQ; ++c) v[s][li][c] = __ldcs(row + c * 32 + lane);
+            }
+        }
+#pragma unroll
+        for (int s = 0; s < SPI; ++s) {
+            if (ib + s >= i1) break;
+            const i64 kt = (i64)dm.k * ti[s];
+            const unsigned ktu = kt < 0x7fffffffll ? (kt < 0 ? 0u : (unsigned)kt) : 0x7fffffffu;
+            if (warp == 0) tsum += ti[s];
+            bad |= ti[s] < 1 || ti[s] > dm.C;
+#pragma unroll
+            for (int li = 0; li < LW; ++li) {
+                unsigned part = 0;
+                bool out = false;
+#pragma unroll
+                for (int c = 0; c < NQ; ++c) {
+                    const int4 x = v[s][li][c];
+                    const unsigned x0 = (unsigned)x.x, x1 = (unsigned)x.y, x2 = (unsigned)x.z, x3 = (unsigned)x.w;
+                    out |= (x0 > ktu) | (x1 > ktu) | (x2 > ktu) | (x3 > ktu);
+                    const unsigned s01 = x0 + x1, s23 = x2 + x3;
+                    out |= (s01 > ktu) | (s23 > ktu);
+                    const unsigned s4 = s01 + s23;
+                    out |= (s4 > ktu);
+                    part += out ? 0u : s4;
+                    out |= (part > ktu);
+                    acc[li][c][0] += x.x; acc[li][c][1] += x.y; acc[li][c][2] += x.z; acc[li][c][3] += x.w;
+                }
+                const unsigned slo = __reduce_add_sync(0xffffffffu, out ? 0u : (part & 0xffffu));
+                const unsigned shi = __reduce_add_sync(0xffffffffu, out ? 0u : (part >> 16));
+                bad |= __any_sync(0xffffffffu, out) || ((i64)slo + ((i64)shi << 16)) != kt;
+            }
+        }
+    }
+#pragma unroll
+    for (int li = 0; li < LW; ++li)
+#pragma unroll
+        for (int c = 0; c < NQ; ++c)
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (acc[li][c][u]) atomicAdd((u64 *)&Lagg[(size_t)(warp + li * NW) * dm.E + (c * 32 + lane) * 4 + u], (u64)acc[li][c][u]);
+    if (bad && lane == 0) atomicExch(&status[RP_SW_BAD_SAMPLE], 1);
+    if (warp == 0 && lane == 0 && tsum > 0) atomicAdd((u64 *)t_sum, (u64)tsum);
+}
+
+template <int NQ, int LW, int NW, int SPI>
+static int launch_check_reduce_seq(rp_ctx *c)
+{
+    const RpDims &dm = c->dm;
+    int chunk = (dm.N + 2 * 148 - 1) / (2 * 148);           // two CTAs per SM: enough bytes in flight, few enough atomics
+    chunk = chunk < SPI ? SPI : chunk;
+    const int grid = (dm.N + chunk - 1) / chunk;
+    k_check_reduce_seq<NQ, LW, NW, SPI><<<grid, NW * 32, 0, c->stream>>>((const int4 *)c->d_a, c->d_t, dm, chunk, c->d_Lagg,
+                                                                       c->d_status, c->d_counters + 7);
+    ++g_rp_launches;
+    RP_CUDA(cudaGetLastError());
+    return RP_OK;
+}
+
 int rp_launch_check_reduce(rp_ctx *c)
 {
     const RpDims &dm = c->dm;
     RP_CUDA(cudaMemsetAsync(c->d_Lagg, 0, sizeof(i64) * dm.L * dm.E, c->stream));
+    // The sequential form where it measured faster (512-byte rows, 32 layers: one atomic per expert,
+    // layer and CTA is then the smaller part of the time; on wider or fewer rows the form below wins).
+    if (((size_t)c->d_a & 15) == 0 && dm.N >= 2 * 148 && dm.E == 128 && dm.L == 32) return launch_check_reduce_seq<1, 2, 16, 4>(c);
     if (dm.E % 128 == 0 && dm.E <= 1024 && ((size_t)c->d_a & 15) == 0) {
         // one CTA per (layer, range of samples): four CTAs per SM (one wave), at least 64 samples each
         int splits = (4 * 148) / dm.L;

@@ -836,10 +836,12 @@ def test_bad_inputs_are_host_side_errors():
 
 
 @pytest.mark.parametrize("E,P,N,L", [(128, 32, 70, 5), (256, 16, 37, 9), (384, 4, 33, 2), (1024, 8, 19, 3), (128, 1, 41, 3),
-                                     (128, 8, 100, 2), (512, 32, 35, 4), (256, 32, 300, 3), (128, 64, 50, 2)])
+                                     (128, 8, 100, 2), (512, 32, 35, 4), (256, 32, 300, 3), (128, 64, 50, 2),
+                                     (128, 32, 301, 32), (128, 4, 296, 32), (256, 16, 297, 48)])
 def test_wide_expert_rows_front_end(E, P, N, L):
     """Rows of whole multiples of 128 experts take the 16-byte-load forms of the check + reduce and
-    projection kernels (ragged sample counts: the last group of rows is partial): aggregate demand,
+    projection kernels (ragged sample counts: the last group of rows is partial; two shapes with 32 layers
+    of 128 experts take the sequential-stream form of the check + reduce): aggregate demand,
     placement, rank demand and seed against the oracle, and every kind of bad input is still caught."""
     w = make_window(custom_spec(f"rows{E}", N, L, E, 4, 4096, 2, P, 6, 100, data_seed=E + N))
     s = w.spec
