@@ -6,9 +6,10 @@
 // Mapping.  One CTA runs one chain for all K steps of a level.  The chain's small state
 // (assignment, cell statistics, per-row-shard costs, shard work) lives in shared memory.
 // Its rank-load tensor W[R][G][L][P] lives in shared memory too when it fits beside a
-// second CTA on the SM (small windows: the chain is latency-bound), else in global memory
-// (L2/HBM; large windows: the chain is bandwidth-bound and many CTAs per SM hide latency).
-// The sample demand rows q[i][L][P] are shared by all chains and stay L2-resident.
+// second CTA on the SM (small windows), else in global memory as slices of L*P ints that a
+// member shares with its ancestor until it rewrites them (see AnnealArgs; many CTAs per SM
+// hide the latency of L2 and HBM).  The sample demand rows q[i][L][P] are shared by all
+// chains and stay L2-resident.
 //
 // A chain is a sequential process, but three things about it are not:
 //  * every random number is a pure function of (step, level, slot), so the proposal words

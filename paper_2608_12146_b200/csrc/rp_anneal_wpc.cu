@@ -14,6 +14,11 @@
 // by its warp straight from its registers, and everything speculated after it is discarded
 // and redone; if none is accepted the next NW follow.  This is step-for-step the sequential
 // chain of Algorithm 3: a later step is only ever scored against the state it would have seen.
+//
+// Launched once per level (the last CTA to finish runs the level barrier, rp_level_end), or, where
+// the rank loads are on chip and every chain is resident at once, once for all levels (PERSIST):
+// then the chains meet at an arrival counter after every level, each CTA works out the barrier
+// for itself from the reports of all, and a chain that is its own ancestor keeps its state on chip.
 #include <string.h>
 
 #include "rp_level_end.cuh"
