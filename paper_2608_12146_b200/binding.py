@@ -302,7 +302,8 @@ def rp_debug_stage_times(ctx: Context) -> dict:
     return {k: (float(v) if v >= 0 else None) for k, v in zip(STAGES, ms)}
 
 
-KNOB = dict(BARRIER_WORKSPACE=1, WAIT_POLLS=2, STALL_ONE_CHAIN=3, RANK_LOAD_SLICES=4, LAUNCH_PER_LEVEL=5)
+KNOB = dict(BARRIER_WORKSPACE=1, WAIT_POLLS=2, STALL_ONE_CHAIN=3, RANK_LOAD_SLICES=4, LAUNCH_PER_LEVEL=5,
+            CHAIN_KERNEL=6)
 
 
 def rp_debug_set_knob(ctx: Context, knob: str, value: int):

@@ -36,6 +36,8 @@ struct ChainB {                 // bookkeeping of the chain within this level
     int best_step, best_nlog, nlog, failed;
     unsigned fmask;
     int accept;
+    i64 n_feas, n_acc, n_imp, n_bytes;      // counters of the level
+    int mt[SPEC][2];                        // lengths of the samples each feasible proposal moves
 };
 
 // Cooperative chain kernel for bandwidth-bound windows (L*P > 512): all NT threads score one
@@ -126,6 +128,7 @@ k_anneal_level(const AnnealArgs A)
     if (tid == 0) {
         chain->B[0] = Sc[0]; chain->B[1] = Sc[1]; chain->B[2] = Sc[2];
         chain->dig = 0; chain->best_step = 0; chain->best_nlog = 0; chain->nlog = 0;
+        chain->n_feas = 0; chain->n_acc = 0; chain->n_imp = 0; chain->n_bytes = 0;
     }
     if (SL) {
         // A slice that only this member holds when the level starts is rewritten in place; a shared
@@ -143,7 +146,6 @@ k_anneal_level(const AnnealArgs A)
 
     uint2 *logj = A.log + (size_t)j * A.log_cap;
     const RpChainView view = { cell_of, T, cnt, tt, attkey, Jcell, Acell };
-    i64 n_feas = 0, n_acc = 0, n_imp = 0, n_bytes = 0;          // thread 0
 
     for (int kb = 0; kb < A.steps; kb += SPEC) {
         const int nb = min(SPEC, A.steps - kb);
@@ -155,8 +157,9 @@ k_anneal_level(const AnnealArgs A)
                 bool ok = false;
                 if (lane >= pos && lane < nb) {
                     MoveS m;
-                    ok = rp_propose(dm, view, recs[lane], m);
-                    if (ok) mvs[lane] = m;
+                    int ti, t2;
+                    ok = rp_propose_len(dm, view, recs[lane], m, ti, t2);
+                    if (ok) { mvs[lane] = m; chain->mt[lane][0] = ti; chain->mt[lane][1] = t2; }
                 }
                 const unsigned fm = __ballot_sync(0xffffffffu, ok);
                 if (lane == 0) { chain->fmask = fm; chain->accept = 0; }
@@ -224,7 +227,7 @@ k_anneal_level(const AnnealArgs A)
                     int fb0 = 0, fb2 = 0;
                     if (lane == 0) {
                         const i64 S0 = Sc[0], S1 = Sc[1], S2 = Sc[2];
-                        const i64 ti = tt[m.i], t2 = swap ? tt[m.i2] : 0;
+                        const i64 ti = chain->mt[ls][0], t2 = chain->mt[ls][1];
                         Ta = (i64)T[c1] - ti + t2; Qa = (i64)Q[c1] - ti * ti + t2 * t2;
                         Tb = (i64)T[c2] + ti - t2; Qb = (i64)Q[c2] + ti * ti - t2 * t2;
                         if (!touchW) { e1 = Esum[rg1]; e2 = e1; }
@@ -279,10 +282,10 @@ k_anneal_level(const AnnealArgs A)
                                 acc = (bh >> 31) ? true : ((u64)(en - Ecur) < ((bh << 32) | (bl >> 32)));
                             }
                         }
-                        ++n_feas;
-                        if (touchW) n_bytes += (i64)((swap ? 4 : 3) + (acc ? 2 : 0)) * dm.LP * 4;
+                        chain->n_feas += 1;
+                        if (touchW) chain->n_bytes += (i64)((swap ? 4 : 3) + (acc ? 2 : 0)) * dm.LP * 4;
                         if (acc) {
-                            ++n_acc;
+                            chain->n_acc += 1;
                             if (SL && touchW) {
                                 // Where the two rewritten slices go: in place when the slice is this chain's
                                 // own, else to the spare slice of that row-shard, which then is its own.
@@ -320,7 +323,7 @@ k_anneal_level(const AnnealArgs A)
                             if (rp_lex_less(n0, n1, n2, chain->B[0], chain->B[1], chain->B[2])) {
                                 chain->B[0] = n0; chain->B[1] = n1; chain->B[2] = n2;
                                 chain->best_step = k + 1; chain->best_nlog = nlog;
-                                ++n_imp;
+                                chain->n_imp += 1;
                             }
                         }
                         chain->accept = acc;
@@ -357,10 +360,10 @@ k_anneal_level(const AnnealArgs A)
         A.best_nlog[j] = chain->best_nlog;
         A.digest[j] = chain->dig;
         atomicAdd((u64 *)&A.counters[0], (u64)A.steps);
-        atomicAdd((u64 *)&A.counters[1], (u64)n_feas);
-        atomicAdd((u64 *)&A.counters[2], (u64)n_acc);
-        atomicAdd((u64 *)&A.counters[3], (u64)n_imp);
-        atomicAdd((u64 *)&A.counters[4], (u64)n_bytes);
+        atomicAdd((u64 *)&A.counters[1], (u64)chain->n_feas);
+        atomicAdd((u64 *)&A.counters[2], (u64)chain->n_acc);
+        atomicAdd((u64 *)&A.counters[3], (u64)chain->n_imp);
+        atomicAdd((u64 *)&A.counters[4], (u64)chain->n_bytes);
     }
     rp_finish_level(A, tid, NT, smraw, A.smem_bytes);
 }
@@ -509,6 +512,7 @@ static u32 host_philox_x(u32 c0, u32 c1, u32 c2, u32 c3, u32 k0, u32 k1)
 }
 
 int rp_launch_anneal_wpc_all(rp_ctx *c, const AnnealArgs &A, int *done);
+int rp_launch_anneal_warp(rp_ctx *c, AnnealArgs &A);
 
 static void fill_args(rp_ctx *c, int level, int n_levels, const rp_anneal_params *prm, u64 rho_q32, u64 guide_q32, AnnealArgs &A)
 {
@@ -592,6 +596,7 @@ int rp_launch_anneal_level(rp_ctx *c, int level, int n_levels, const rp_anneal_p
     fill_args(c, level, n_levels, prm, rho_q32, guide_q32, A);
     if (rp_uses_slices(c->dm)) RP_TRY(rp_launch_slice_gc(c));
     if (use_wpc(c->dm)) return rp_launch_anneal_wpc(c, A);
+    if (rp_uses_warp_chains(c)) return rp_launch_anneal_warp(c, A);
     int nt; size_t smem;
     const bool alias = rp_anneal_smem_bytes(c, &nt, &smem) == 2;
     if (smem > 220 * 1024) return RP_ERR_RANGE;

@@ -155,6 +155,35 @@ __device__ __forceinline__ bool rp_propose(const RpDims &dm, const RpChainView &
     return (v.T[m.c1] - ti + t2 <= dm.C) && (v.T[m.c2] - t2 + ti <= dm.C);
 }
 
+// The same rule, also handing back the lengths of the moved samples (the decision needs them again,
+// and for long windows they come from global memory).
+__device__ __forceinline__ bool rp_propose_len(const RpDims &dm, const RpChainView &v, const StepRec &r, MoveS &m, int &ti_out, int &t2_out)
+{
+    const bool reloc = r.flags & 1u;
+    const int ca = v.cell_of[r.i0], cb = v.cell_of[r.i1];
+    const int xa = reloc ? r.i2 : (int)v.cell_of[r.i2];
+    const int xb = reloc ? r.i3 : (int)v.cell_of[r.i3];
+    const u64 Ja = (u64)v.Jcell[ca], Aa = (u64)v.Acell[ca];
+    const u64 lh = __umul64hi((u64)r.bz, Ja), ll = (u64)r.bz * Ja;
+    const u64 rh = Aa >> 32, rl = Aa << 32;
+    const bool use_att = (lh < rh) || (lh == rh && ll < rl);
+    const i64 *key = use_att ? v.attkey : v.Jcell;
+    const i64 ka = key[ca], kb = key[cb], ta = key[xa], tb = key[xb];
+    const bool src_b = kb > ka, dst_b = tb < ta;
+    m.reloc = reloc;
+    m.i = src_b ? r.i1 : r.i0;
+    m.c1 = src_b ? cb : ca;
+    m.c2 = dst_b ? xb : xa;
+    m.i2 = reloc ? -1 : (dst_b ? r.i3 : r.i2);
+    if (m.c1 == m.c2) return false;
+    const int ti = v.tt[m.i];
+    ti_out = ti; t2_out = 0;
+    if (reloc) return (v.cnt[m.c1] > 1) && (v.T[m.c2] + ti <= dm.C);
+    const int t2 = v.tt[m.i2];
+    t2_out = t2;
+    return (v.T[m.c1] - ti + t2 <= dm.C) && (v.T[m.c2] - t2 + ti <= dm.C);
+}
+
 __device__ __forceinline__ int max4(const int4 &v) { return max(max(v.x, v.y), max(v.z, v.w)); }
 
 // Tentative rank loads of the two touched row-shards, W1' = W1 - d and W2' = W2 + d with

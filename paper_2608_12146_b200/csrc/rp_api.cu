@@ -965,7 +965,7 @@ extern "C" int rp_anneal(rp_ctx *c, const rp_anneal_params *p, rp_anneal_stats *
     if (stats) {
         stats->proposed = cn[0]; stats->feasible = cn[1]; stats->accepted = cn[2]; stats->improved = cn[3];
         stats->move_bytes = cn[4]; stats->gather_bytes = cn[5]; stats->staging_bytes = cn[6];
-        stats->kernel_launches = all_in_one ? 1 : (int64_t)NL * (rp_uses_slices(c->dm) ? 3 : 1);
+        stats->kernel_launches = all_in_one ? 1 : (int64_t)NL * ((rp_uses_slices(c->dm) ? 3 : 1) + (rp_uses_warp_chains(c) ? 1 : 0));
         stats->ms_chains = ms_chains;
     }
     c->best_verdict = best_verdict(c, sw);
@@ -1078,6 +1078,9 @@ extern "C" int rp_debug_set_knob(rp_ctx *c, int knob, int64_t value)
         case RP_KNOB_RANK_LOAD_SLICES:
             if (value > 2) return RP_ERR_ARG;
             c->knob_slices = (int)value; return RP_OK;
+        case RP_KNOB_CHAIN_KERNEL:
+            if (value > 3) return RP_ERR_ARG;
+            c->knob_chain_kernel = (int)value; return RP_OK;
         default: return RP_ERR_ARG;
     }
 }

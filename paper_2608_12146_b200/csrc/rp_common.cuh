@@ -170,6 +170,7 @@ struct rp_ctx {
     int trace_levels;
     int trace_on;              // keep per-level traces (inspection hook; off by default)
     int knob_level_launches;   // 1 = one launch per level even where one launch for all levels is possible
+    int knob_chain_kernel;     // 1 = 128 threads per chain, 2 = one warp per chain, wherever the window allows both
     int knob_slices;           // inspection hook: 0 = automatic, 1 = slices wherever the cooperative kernel runs, 2 = never
     int knob_le_ws_cap, knob_wait_polls, knob_stall;   // inspection hooks (rp_debug_set_knob); 0 = off
     cudaEvent_t ev_stage[RP_STAGE_EVENTS];             // stage timing (rp_debug_set_stage_timing); null when off
@@ -245,6 +246,7 @@ struct RpSlab {
 int rp_launch_select(rp_ctx *c, int *lay, int *out, const i64 *score, int n_proj, i64 eta_q16, int *order,
                      int *n_distinct, i64 *dist);
 bool rp_uses_wpc(const RpDims &dm);
+bool rp_uses_warp_chains(const rp_ctx *c);
 int rp_launch_anneal_level(rp_ctx *c, int level, int n_levels, const rp_anneal_params *prm, u64 rho_q32, u64 guide_q32);
 int rp_launch_anneal_all(rp_ctx *c, int n_levels, const rp_anneal_params *prm, u64 rho_q32, u64 guide_q32, int *done);
 int rp_upload_levels(rp_ctx *c, int n_levels);

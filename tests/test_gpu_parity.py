@@ -355,6 +355,49 @@ def test_level_barrier_paths_on_small_windows(spec, cap):
         rp.rp_destroy(ctx)
 
 
+WARP_CHAIN_CASES = [
+    # name, N, L, E, k, C, D, P, edp, min_rows, pop: windows with 512 < L*P <= 1024 for the warp-per-chain kernel
+    ("wc_ragged", 120, 20, 32, 2, 4096, 4, 32, None, 3, 40),            # 160 chunks of 16 bytes: 5 per lane
+    ("wc_shared", 151, 17, 64, 2, 4096, 4, 32, [0, 1, 1, 0], 2, 130),   # two DP slots per shard, odd sample count
+    ("wc_p4", 140, 200, 16, 2, 4096, 4, 4, None, 3, 33),                # one lane per layer
+    ("wc_p128", 100, 8, 128, 2, 4096, 3, 128, None, 2, 50),             # a whole warp per layer, L*P = 1024
+    ("wc_cells", 700, 16, 64, 2, 8192, 64, 64, None, 5, 24),            # 320 cells: the assignment stays in global memory
+]
+
+
+@pytest.mark.parametrize("spec", WARP_CHAIN_CASES, ids=[e[0] for e in WARP_CHAIN_CASES])
+@pytest.mark.parametrize("kernel", [2, 3])
+def test_warp_per_chain_kernel_on_small_windows(spec, kernel):
+    """The chain kernel that full-size windows with thousands of chains use (one warp per chain),
+    forced onto small windows: the assignment as bytes in shared memory (2, where a cell fits a
+    byte) and as the blob's array in global memory (3), ragged chunk counts, one to 32 lanes per
+    layer, shared shards; the level barrier as a launch of its own, with all of its shared
+    memory and with next to none; a second rp_anneal call that resumes from the tables."""
+    name, N, L, E, k, C, D, P, edp, min_rows, pop = spec
+    w = make_window(custom_spec(name, N, L, E, k, C, D, P, pop, 400, data_seed=len(name) * 13 + N))
+    ref = oracle_front(w, edp, min_rows)
+    for cap in (0, 64):
+        ctx = load(w, pop=pop, edp=edp, min_rows=min_rows)
+        rp.rp_debug_set_knob(ctx, "CHAIN_KERNEL", kernel)
+        rp.rp_debug_set_knob(ctx, "BARRIER_WORKSPACE", cap)
+        check_front(w, ctx, ref)
+        want, stats = check_anneal(w, ctx, ref, edp, pop, 8, 40, t_ratio=0.6, check_members=2)
+        assert stats.accepted > 50 and stats.improved > 0
+        assert stats.gather_bytes == 0 and stats.kernel_launches == 8 * 4       # bookkeeping (2), chains, barrier
+        s_ = w.spec
+        again = oracle.anneal(w.lengths, ref["q"], want["final_pop"], ref["R"], s_.token_cap, s_.dp_width, n_levels=3,
+                              steps=30, t0=1e-4, t_ratio=0.5, p_reloc=0.5, p_guide=0.3, seed=s_.anneal_seed,
+                              edp_of_dp=edp, alpha=s_.alpha, beta=s_.beta)
+        rp.rp_anneal(ctx, n_levels=3, steps_per_level=30, t0=1e-4, t_ratio=0.5, p_reloc=0.5, p_guide=0.3)
+        assert (rp.rp_debug_dump(ctx, "TRACE_TERM", (3, pop, 3), np.int64) == again["term"]).all()
+        assert (rp.rp_debug_dump(ctx, "POPULATION", (pop, s_.n_samples), np.int32) == again["final_pop"]).all()
+        G = 1 + (max(edp) if edp is not None else D - 1)
+        for j in (0, pop - 1):
+            ev = oracle.eval_layouts(w.lengths, ref["q"], again["final_pop"][j], ref["R"], s_.token_cap, D, edp, s_.alpha, s_.beta)
+            assert (rp.rp_debug_dump(ctx, "W", (ref["R"], G, L, P), np.int32, index=j) == ev["W"][0]).all()
+        rp.rp_destroy(ctx)
+
+
 @pytest.mark.parametrize("spec", [BARRIER_CASES[0], BARRIER_CASES[2]], ids=["warp_per_candidate", "cooperative"])
 def test_a_wait_that_runs_out_is_reported_and_the_context_survives(spec):
     """One chain waits on a barrier phase that nothing completes, with the poll limit cut to 10^4:
