@@ -310,8 +310,7 @@ typedef enum {
  *   RP_KNOB_CHAIN_KERNEL: which chain kernel windows with 512 < L*P <= 1024 and shared slices
  *     use.  0 = by population (one warp per chain when the chains outnumber what the 128-thread
  *     kernel keeps resident, else 128 threads per chain), 1 = always 128 threads per chain,
- *     2 = always one warp per chain, 3 = one warp per chain that keeps the assignment in global
- *     memory (as windows with more than 256 cells do) instead of shared memory. */
+ *     2 = always one warp per chain. */
 typedef enum { RP_KNOB_BARRIER_WORKSPACE = 1, RP_KNOB_WAIT_POLLS = 2, RP_KNOB_STALL_ONE_CHAIN = 3,
                RP_KNOB_RANK_LOAD_SLICES = 4, RP_KNOB_LAUNCH_PER_LEVEL = 5, RP_KNOB_CHAIN_KERNEL = 6 } rp_knob;
 int rp_debug_set_knob(rp_ctx *ctx, int knob, int64_t value);

@@ -1,32 +1,31 @@
-// Chain kernel of the population annealing for windows with thousands of chains and slices of
-// 512 < L*P <= 1024 ints (at most 256 cells): "warp per chain".
+// Chain kernel of the population annealing for windows with more chains than the 128-thread
+// kernel keeps resident and slices of 512 < L*P <= 1024 ints: "warp per chain".
 //
-// A chain of Algorithm 3 is latency-bound: a step is a proposal, two dependent trips to L2 or HBM
-// for the touched rank-load slices, an exact rescoring in 64-bit integers and a decision, each
-// waiting for the one before.  What raises the throughput of a level is therefore the number of
-// chains an SM keeps in flight, and that is set by what one chain occupies.  Here a chain is a
-// single warp: the two tentative slices of a candidate (2 * L*P ints, 8 chunks of 16 bytes per
-// lane and slice) are reduced as they arrive and kept nowhere (an accepted move builds them once
-// more from L2 and stores them); the assignment is kept as one byte per sample; the chain's
-// state arrives and leaves with plain loads and stores.  Fourteen
-// chains are resident per SM (against six CTAs of 128 threads in the cooperative kernel), no
-// block-wide barrier is left in the step loop, and nothing in the kernel waits on another CTA:
-// the level barrier (incumbent, weights, ancestors) is a launch of its own behind it.
-//
-// The steps are the same as in the other two chain kernels: the random words and accept
-// thresholds of the next 32 steps one step per lane; proposals and feasibility of those steps
-// against the current state one step per lane; feasible candidates scored in step order by the
-// whole warp; speculation redone after an acceptance.  Rank loads are slices of the pool shared
-// copy-on-write with the ancestor (see AnnealArgs).
+// A chain of Algorithm 3 is a sequence of dependent rounds (proposal, the touched rank-load
+// slices and demand rows from L2 or HBM, exact rescoring in 64-bit integers, decision), so the
+// throughput of a level is the number of chains an SM keeps in flight over the latency of a round.
+// Here a chain is a single warp with about 23 KB of shared memory, nine to an SM:
+//  * the two demand rows and two slices of a candidate (4 * L*P ints) arrive in shared memory by
+//    four bulk asynchronous copies on one mbarrier (bounded wait): one trip to memory per
+//    candidate and no registers held while it lasts; lane 0 rebuilds the part of the score that
+//    needs only the cell statistics in the meantime;
+//  * the busiest rank of every layer is found with a lane per layer (no shuffles), an accepted
+//    move is stored straight from the staged copies, and the slices of the candidate that
+//    follows are prefetched into L2 while this one is decided;
+//  * the random words of the next 32 steps, the cells of their candidate samples and those
+//    samples' lengths are fetched once per batch, one step per lane, and kept in registers; an
+//    accepted move patches the cached cells, so a proposal reads shared memory only;
+//  * the assignment itself stays in the chain's blob in global memory (written on acceptance,
+//    read once per batch), the chain's small arrays arrive and leave with plain loads and stores,
+//    and the level barrier (incumbent, weights, ancestors) is a launch of its own behind the chains.
+// Step for step this is the sequential chain: proposals are evaluated against the current state,
+// feasible ones are scored in step order, and the speculation is redone after an acceptance.
+// Rank loads are slices of the pool shared copy-on-write with the ancestor (see AnnealArgs).
 #include <algorithm>
 
 #include "rp_level_end.cuh"
 
-#define WARP_CHAINS_PER_SM 14            // assignment in shared memory
-#define WARP_CHAINS_PER_SM_CG 16         // assignment in global memory
-#define WARP_CHK 8                      // 16-byte chunks per lane and slice
-#define WARP_PREFETCH 1                 // the next candidate's slices are prefetched into L2
-#define WARP_PART 2                     // of which so many are in flight at once
+#define WARP_CHAINS_PER_SM 9            // resident chains the register budget is set for
 
 struct CandW { MoveS m; int ti, t2, pad; };          // a feasible proposal and the lengths of the moved samples
 struct ChainW {                                      // bookkeeping of the chain within this level
@@ -37,16 +36,15 @@ struct ChainW {                                      // bookkeeping of the chain
 };
 
 // Shared-memory plan of one chain: the blob's arrays up to the assignment at their blob offsets,
-// then the assignment as bytes, the slice table, the static tables, and the kernel's own arrays.
+// then the slice table, the static tables, the kernel's own arrays and the staging area.
 struct RpWarpLayout {
-    int off_cell8, off_wtab, off_static, off_keys, off_recs, off_cand, off_chain, off_spare, off_own, bytes;
+    int off_wtab, off_static, off_keys, off_recs, off_cand, off_chain, off_spare, off_own, off_mbar, off_stage, bytes;
 };
 
-static RpWarpLayout rp_warp_layout(const RpDims &dm, const RpBlob &bl, const RpStatic &sl, bool identity, bool cells_global)
+static RpWarpLayout rp_warp_layout(const RpDims &dm, const RpBlob &bl, const RpStatic &sl, bool identity)
 {
     RpWarpLayout w;
     size_t o = ((size_t)bl.off_cell + 15) & ~(size_t)15;
-    w.off_cell8 = (int)o;  o += cells_global ? 0 : (((size_t)dm.N + 15) & ~(size_t)15);
     w.off_wtab = (int)o;   o += ((size_t)4 * dm.RG + 15) & ~(size_t)15;
     w.off_static = (int)o; o += sl.bytes;
     w.off_keys = (int)o;   o += identity ? 0 : (size_t)3 * 8 * dm.K;
@@ -55,36 +53,29 @@ static RpWarpLayout rp_warp_layout(const RpDims &dm, const RpBlob &bl, const RpS
     w.off_chain = (int)o;  o += sizeof(ChainW);
     w.off_spare = (int)o;  o += (size_t)4 * dm.RG;
     w.off_own = (int)o;    o += dm.RG;
+    o = (o + 15) & ~(size_t)15;
+    w.off_mbar = (int)o;   o += 16;
+    o = (o + 127) & ~(size_t)127;
+    w.off_stage = (int)o;  o += (size_t)4 * 4 * dm.LP;          // two demand rows and two slices of a candidate
     w.bytes = (int)((o + 15) & ~(size_t)15);
     return w;
 }
 
-// The assignment of the chain: one byte per sample in shared memory, or (CG) the 16-bit array of
-// the chain's blob in global memory, read and written through L2 (more chains then fit an SM).
-template <bool CG>
-__device__ __forceinline__ int rp_cell_rd(const void *cells, int i)
-{
-    if (CG) return (int)__ldcg((const unsigned short *)cells + i);
-    return (int)((const unsigned char *)cells)[i];
-}
-template <bool CG>
-__device__ __forceinline__ void rp_cell_wr(void *cells, int i, int c)
-{
-    if (CG) ((unsigned short *)cells)[i] = (unsigned short)c;
-    else ((unsigned char *)cells)[i] = (unsigned char)c;
-}
+// What a lane keeps about the step it proposes for: the candidate indices of the step record with
+// the cells of the candidate samples (kept in step with the accepted moves) and their lengths.
+struct StepRegs {
+    u32 flags, bz;
+    int i[4];               // samples; for a relocation i[2], i[3] are target cells
+    int c[4];               // cell of sample i[x] (i[2], i[3] themselves for a relocation)
+    int t[4];               // length of sample i[x] (unused for relocation targets)
+};
 
-// GuidedProposal + feasibility of one step (the rule of rp_propose, on the chain's assignment), also
-// handing back the lengths of the moved samples, which the decision needs again.
-template <bool CG>
-__device__ __forceinline__ bool rp_propose_bytes(const RpDims &dm, const void *cell8, const int *T, const int *cnt,
-                                                 const int *__restrict__ tt, const i64 *attkey, const i64 *Jcell, const i64 *Acell,
-                                                 const StepRec &r, CandW &cd)
+// GuidedProposal + feasibility of one step (the rule of rp_propose) from the lane's registers.
+__device__ __forceinline__ bool rp_propose_regs(const RpDims &dm, const StepRegs &r, const int *T, const int *cnt,
+                                                const i64 *attkey, const i64 *Jcell, const i64 *Acell, CandW &cd)
 {
     const bool reloc = r.flags & 1u;
-    const int ca = rp_cell_rd<CG>(cell8, r.i0), cb = rp_cell_rd<CG>(cell8, r.i1);
-    const int xa = reloc ? r.i2 : rp_cell_rd<CG>(cell8, r.i2);
-    const int xb = reloc ? r.i3 : rp_cell_rd<CG>(cell8, r.i3);
+    const int ca = r.c[0], cb = r.c[1], xa = r.c[2], xb = r.c[3];
     const u64 Ja = (u64)Jcell[ca], Aa = (u64)Acell[ca];
     const u64 lh = __umul64hi((u64)r.bz, Ja), ll = (u64)r.bz * Ja;
     const u64 rh = Aa >> 32, rl = Aa << 32;
@@ -94,79 +85,71 @@ __device__ __forceinline__ bool rp_propose_bytes(const RpDims &dm, const void *c
     const bool src_b = kb > ka, dst_b = tb < ta;
     MoveS &m = cd.m;
     m.reloc = reloc;
-    m.i = src_b ? r.i1 : r.i0;
+    m.i = src_b ? r.i[1] : r.i[0];
     m.c1 = src_b ? cb : ca;
     m.c2 = dst_b ? xb : xa;
-    m.i2 = reloc ? -1 : (dst_b ? r.i3 : r.i2);
+    m.i2 = reloc ? -1 : (dst_b ? r.i[3] : r.i[2]);
+    const int ti = src_b ? r.t[1] : r.t[0];
+    const int t2 = reloc ? 0 : (dst_b ? r.t[3] : r.t[2]);
+    cd.ti = ti; cd.t2 = t2; cd.pad = 0;
     if (m.c1 == m.c2) return false;
-    const int ti = __ldg(tt + m.i);
-    cd.ti = ti; cd.t2 = 0; cd.pad = 0;
     if (reloc) return (cnt[m.c1] > 1) && (T[m.c2] + ti <= dm.C);
-    const int t2 = __ldg(tt + m.i2);
-    cd.t2 = t2;
     return (T[m.c1] - ti + t2 <= dm.C) && (T[m.c2] - t2 + ti <= dm.C);
 }
 
-// Half `h` of the pass over the two touched slices: this lane's chunks of W1' = W1 - d and
-// W2' = W2 + d with d = q[i] - q[i2] (relocation: d = q[i]), all loads in flight before any is
-// used.  COMMIT = false adds the busiest rank of every layer to p1, p2 (e1, e2 when the sums need
-// 64 bits); COMMIT = true stores the two slices to o1, o2 instead.
-template <bool COMMIT>
-__device__ __forceinline__ void rp_warp_half(int h, int lane, int nchunks, int lpl, bool sum32, const int4 *__restrict__ qi,
-                                             const int4 *__restrict__ q2, const int4 *w1, const int4 *w2, int4 *o1, int4 *o2,
-                                             int &p1, int &p2, i64 &e1, i64 &e2)
+// Scoring pass over a candidate whose two demand rows and two slices have been staged in shared
+// memory: W1' = W1 - d and W2' = W2 + d with d = q[i] - q[i2] (relocation: d = q[i]).  A lane takes
+// whole layers (layer = lane, lane + 32, ...), so the busiest rank of a layer needs no shuffles;
+// the lanes of a quarter warp start at different chunks of their layers, which keeps the 16-byte
+// reads off each other's banks.  cpl = 16-byte chunks per layer (a power of two).  Returns the
+// two sums over layers of the busiest ranks.
+__device__ __forceinline__ void rp_warp_staged_score(int lane, int L, int cpl, bool sum32, bool swap, const int4 *s_qi,
+                                                     const int4 *s_q2, const int4 *s_w1, const int4 *s_w2, i64 &e1, i64 &e2)
 {
-    constexpr int H = WARP_PART;
-    int4 d[H], a[H], b[H];
-    // (the swap / relocation branch stays outside the loops: a branch between two loads would make
-    // the second wait for the first)
-    if (q2) {
-        int4 o[H];
-#pragma unroll
-        for (int u = 0; u < H; ++u) {
-            const int c = (h * H + u) * 32 + lane;
-            if (h * H + u < WARP_CHK && c < nchunks) { d[u] = __ldg(qi + c); o[u] = __ldg(q2 + c); a[u] = w1[c]; b[u] = w2[c]; }
-        }
-#pragma unroll
-        for (int u = 0; u < H; ++u) {
-            const int c = (h * H + u) * 32 + lane;
-            if (h * H + u < WARP_CHK && c < nchunks) { d[u].x -= o[u].x; d[u].y -= o[u].y; d[u].z -= o[u].z; d[u].w -= o[u].w; }
-        }
-    } else {
-#pragma unroll
-        for (int u = 0; u < H; ++u) {
-            const int c = (h * H + u) * 32 + lane;
-            if (h * H + u < WARP_CHK && c < nchunks) { d[u] = __ldg(qi + c); a[u] = w1[c]; b[u] = w2[c]; }
-        }
-    }
-#pragma unroll
-    for (int u = 0; u < H; ++u) {
-        const int c = (h * H + u) * 32 + lane;
+    int p1 = 0, p2 = 0;
+    for (int ly = lane; ly < L; ly += 32) {
+        const int base = ly * cpl;
         int m1 = 0, m2 = 0;
-        if (h * H + u >= WARP_CHK) continue;
-        if (c < nchunks) {
-            const int4 v1 = make_int4(a[u].x - d[u].x, a[u].y - d[u].y, a[u].z - d[u].z, a[u].w - d[u].w);
-            const int4 v2 = make_int4(b[u].x + d[u].x, b[u].y + d[u].y, b[u].z + d[u].z, b[u].w + d[u].w);
-            if (COMMIT) { o1[c] = v1; o2[c] = v2; }
-            else { m1 = max4(v1); m2 = max4(v2); }
+#pragma unroll 4
+        for (int k = 0; k < cpl; ++k) {
+            const int c = base + ((k + lane) & (cpl - 1));
+            int4 d = s_qi[c];
+            if (swap) { const int4 o = s_q2[c]; d.x -= o.x; d.y -= o.y; d.z -= o.z; d.w -= o.w; }
+            const int4 a = s_w1[c], b = s_w2[c];
+            m1 = max(m1, max(max(a.x - d.x, a.y - d.y), max(a.z - d.z, a.w - d.w)));
+            m2 = max(m2, max(max(b.x + d.x, b.y + d.y), max(b.z + d.z, b.w + d.w)));
         }
-        if (!COMMIT) {
-            for (int o = lpl >> 1; o; o >>= 1) {          // busiest rank of the layer
-                m1 = max(m1, __shfl_xor_sync(0xffffffffu, m1, o));
-                m2 = max(m2, __shfl_xor_sync(0xffffffffu, m2, o));
-            }
-            if ((lane & (lpl - 1)) == 0 && c < nchunks) {
-                if (sum32) { p1 += m1; p2 += m2; }
-                else { e1 += m1; e2 += m2; }
-            }
-        }
+        if (sum32) { p1 += m1; p2 += m2; }
+        else { e1 += m1; e2 += m2; }
+    }
+    if (sum32) {
+        e1 = (i64)__reduce_add_sync(0xffffffffu, (unsigned)p1);
+        e2 = (i64)__reduce_add_sync(0xffffffffu, (unsigned)p2);
+    } else {
+        e1 = warp_sum_i64(e1);
+        e2 = warp_sum_i64(e2);
+    }
+}
+
+// An accepted move: the two new slices straight from the staged copies to where they now live,
+// consecutive lanes storing consecutive 16-byte chunks.
+__device__ __forceinline__ void rp_warp_staged_commit(int lane, int nchunks, bool swap, const int4 *s_qi, const int4 *s_q2,
+                                                      const int4 *s_w1, const int4 *s_w2, int4 *o1, int4 *o2)
+{
+#pragma unroll 4
+    for (int c = lane; c < nchunks; c += 32) {
+        int4 d = s_qi[c];
+        if (swap) { const int4 o = s_q2[c]; d.x -= o.x; d.y -= o.y; d.z -= o.z; d.w -= o.w; }
+        const int4 a = s_w1[c], b = s_w2[c];
+        o1[c] = make_int4(a.x - d.x, a.y - d.y, a.z - d.z, a.w - d.w);
+        o2[c] = make_int4(b.x + d.x, b.y + d.y, b.z + d.z, b.w + d.w);
     }
 }
 
 // ID: every DP slot is its own shard, so a cell is a row-shard and the per-cell proposal keys are
 // the row-shard arrays of the blob themselves.
-template <bool ID, bool CG>
-__global__ void __launch_bounds__(32, CG ? WARP_CHAINS_PER_SM_CG : WARP_CHAINS_PER_SM)
+template <bool ID>
+__global__ void __launch_bounds__(32, WARP_CHAINS_PER_SM)
 k_anneal_warp(const AnnealArgs A, const RpWarpLayout wl)
 {
     const RpDims &dm = A.dm;
@@ -180,7 +163,6 @@ k_anneal_warp(const AnnealArgs A, const RpWarpLayout wl)
     i64 *Sc = (i64 *)(sm + A.bl.off_S);                              // S0, S1, S2, energy
     int *T = (int *)(sm + A.bl.off_T);
     int *cnt = (int *)(sm + A.bl.off_cnt);
-    void *cell8 = CG ? (void *)(A.blob_dst + (size_t)blockIdx.x * A.bl.bytes + A.bl.off_cell) : (void *)(sm + wl.off_cell8);
     int *wtab = (int *)(sm + wl.off_wtab);
     char *sm_static = sm + wl.off_static;
     i64 *attkey = ID ? Afx : (i64 *)(sm + wl.off_keys);
@@ -191,6 +173,8 @@ k_anneal_warp(const AnnealArgs A, const RpWarpLayout wl)
     ChainW *chain = (ChainW *)(sm + wl.off_chain);
     int *spare = (int *)(sm + wl.off_spare);
     unsigned char *own = (unsigned char *)(sm + wl.off_own);
+    u64 *mbar = (u64 *)(sm + wl.off_mbar);
+    int4 *s_qi = (int4 *)(sm + wl.off_stage), *s_q2 = s_qi + (dm.LP >> 2), *s_w1 = s_q2 + (dm.LP >> 2), *s_w2 = s_w1 + (dm.LP >> 2);
     const int *dpl = (const int *)(sm_static + A.sl.off_dpl);
     const int *dpo = (const int *)(sm_static + A.sl.off_dpo);
     const unsigned short *rg_of = (const unsigned short *)(sm_static + A.sl.off_rg);
@@ -202,8 +186,12 @@ k_anneal_warp(const AnnealArgs A, const RpWarpLayout wl)
     const int j = blockIdx.x;
     if (__ldcg(&A.status[RP_SW_TIMEOUT])) return;                  // the call has failed already: nothing to do
     const int src = min(max(A.anc[j], 0), A.Ppop - 1);
-    const int LP = dm.LP, nchunks = LP >> 2, lpl = dm.P >> 2;      // lanes that share a layer
+    const int LP = dm.LP, nchunks = LP >> 2, cpl = dm.P >> 2;      // 16-byte chunks per slice and per layer
     const bool sum32 = (i64)dm.L * dm.k * dm.C * ((dm.D + dm.G - 1) / dm.G) < (1ll << 31);
+    // The chain's assignment: the 16-bit array of its blob, read and written through L2.
+    unsigned short *cells = (unsigned short *)(A.blob_dst + (size_t)j * A.bl.bytes + A.bl.off_cell);
+    u32 phase = 0;
+    if (lane == 0) rp_mbar_init(mbar, 1);
 
     // ---- prologue: the ancestor's terminal state --------------------------------------------
     {
@@ -212,12 +200,8 @@ k_anneal_warp(const AnnealArgs A, const RpWarpLayout wl)
         for (int x = lane; x < nh; x += 32) ((int *)sm)[x] = __ldg((const int *)bsrc + x);
         const unsigned short *cs = (const unsigned short *)(bsrc + A.bl.off_cell);
         const int n4 = dm.N >> 2;
-        for (int x = lane; x < n4; x += 32) {
-            const uint2 v = __ldg((const uint2 *)cs + x);
-            if (CG) ((uint2 *)cell8)[x] = v;
-            else ((u32 *)cell8)[x] = (v.x & 0xffu) | ((v.x >> 16) << 8) | ((v.y & 0xffu) << 16) | ((v.y >> 16) << 24);
-        }
-        for (int i = (n4 << 2) + lane; i < dm.N; i += 32) rp_cell_wr<CG>(cell8, i, (int)__ldg(cs + i));
+        for (int x = lane; x < n4; x += 32) ((uint2 *)cells)[x] = __ldg((const uint2 *)cs + x);
+        for (int i = (n4 << 2) + lane; i < dm.N; i += 32) cells[i] = __ldg(cs + i);
         const int *ts = (const int *)(bsrc + A.bl.off_wtab);
         for (int rg = lane; rg < dm.RG; rg += 32) wtab[rg] = __ldg(ts + rg);
         const int nsb = A.sl.bytes >> 2;
@@ -248,10 +232,26 @@ k_anneal_warp(const AnnealArgs A, const RpWarpLayout wl)
     }
     __syncwarp();
 
-
     for (int kb = 0; kb < A.steps; kb += SPEC) {
         const int nb = min(SPEC, A.steps - kb);
-        if (lane < nb) recs[lane] = rp_make_step_rec(A, A.level, A.tau, (u32)(kb + lane), (u32)j);
+        // ---- the next 32 steps, one per lane: random words, candidate cells and lengths -------
+        StepRegs sr;
+        sr.flags = 0; sr.bz = 0;
+#pragma unroll
+        for (int x = 0; x < 4; ++x) { sr.i[x] = -1; sr.c[x] = 0; sr.t[x] = 0; }
+        if (lane < nb) {
+            const StepRec r = rp_make_step_rec(A, A.level, A.tau, (u32)(kb + lane), (u32)j);
+            recs[lane] = r;
+            const bool rl = r.flags & 1u;
+            sr.flags = r.flags; sr.bz = r.bz;
+            sr.i[0] = r.i0; sr.i[1] = r.i1; sr.i[2] = r.i2; sr.i[3] = r.i3;
+            sr.c[0] = (int)__ldcg(cells + r.i0); sr.c[1] = (int)__ldcg(cells + r.i1);
+            sr.c[2] = rl ? r.i2 : (int)__ldcg(cells + r.i2);
+            sr.c[3] = rl ? r.i3 : (int)__ldcg(cells + r.i3);
+            sr.t[0] = __ldg(A.t + r.i0); sr.t[1] = __ldg(A.t + r.i1);
+            sr.t[2] = rl ? 0 : __ldg(A.t + r.i2);
+            sr.t[3] = rl ? 0 : __ldg(A.t + r.i3);
+        }
         __syncwarp();
         int pos = 0;
         while (pos < nb) {
@@ -259,7 +259,7 @@ k_anneal_warp(const AnnealArgs A, const RpWarpLayout wl)
             bool ok = false;
             if (lane >= pos && lane < nb) {
                 CandW cd;
-                ok = rp_propose_bytes<CG>(dm, cell8, T, cnt, A.t, attkey, Jcell, Acell, recs[lane], cd);
+                ok = rp_propose_regs(dm, sr, T, cnt, attkey, Jcell, Acell, cd);
                 if (ok) cand[lane] = cd;
             }
             unsigned fmask = __ballot_sync(0xffffffffu, ok);
@@ -270,12 +270,25 @@ k_anneal_warp(const AnnealArgs A, const RpWarpLayout wl)
                 fmask &= fmask - 1;
                 const MoveS m = cand[ls].m;
                 const bool swap = !m.reloc;
-                const int rg1 = rg_of[m.c1], rg2 = rg_of[m.c2];
+                const int c1 = m.c1, c2 = m.c2;
+                const int rg1 = rg_of[c1], rg2 = rg_of[c2];
+                const int g1 = g_of[c1], g2 = g_of[c2];
                 const bool touchW = (rg1 != rg2);
-#if WARP_PREFETCH
+                const int4 *w1 = (const int4 *)(A.W + (size_t)wtab[rg1] * LP);
+                const int4 *w2 = (const int4 *)(A.W + (size_t)wtab[rg2] * LP);
+                if (touchW && lane == 0) {
+                    // the candidate's rows and slices into shared memory: one trip, nothing in registers
+                    const u32 bytes = (u32)LP * 4u;
+                    rp_fence_async_smem();          // the previous candidate's reads of the staging area come first
+                    rp_mbar_expect_tx(mbar, (swap ? 4u : 3u) * bytes);
+                    rp_bulk_g2s(s_qi, A.q + (size_t)m.i * LP, bytes, mbar);
+                    if (swap) rp_bulk_g2s(s_q2, A.q + (size_t)m.i2 * LP, bytes, mbar);
+                    rp_bulk_g2s(s_w1, w1, bytes, mbar);
+                    rp_bulk_g2s(s_w2, w2, bytes, mbar);
+                }
                 if (fmask) {
                     // The candidate after this one is scored if this one is rejected: start its two slices on
-                    // their way from HBM to L2 now, one 128-byte line per lane and slice (no registers held).
+                    // their way from HBM to L2 now, one 128-byte line per lane and slice.
                     const int ln = __ffs(fmask) - 1;
                     const int ra = rg_of[cand[ln].m.c1], rb = rg_of[cand[ln].m.c2];
                     if (ra != rb && lane * 32 < LP) {
@@ -284,47 +297,52 @@ k_anneal_warp(const AnnealArgs A, const RpWarpLayout wl)
                         asm volatile("prefetch.global.L2 [%0];" ::"l"(pb));
                     }
                 }
-#endif
-                i64 e1 = 0, e2 = 0;
-                const int4 *qi = (const int4 *)(A.q + (size_t)m.i * LP);
-                const int4 *q2 = swap ? (const int4 *)(A.q + (size_t)m.i2 * LP) : nullptr;
-                const int4 *w1 = (const int4 *)(A.W + (size_t)wtab[rg1] * LP);
-                const int4 *w2 = (const int4 *)(A.W + (size_t)wtab[rg2] * LP);
-                if (touchW) {
-                    int p1 = 0, p2 = 0;
-#pragma unroll
-                    for (int h = 0; h < (WARP_CHK + WARP_PART - 1) / WARP_PART; ++h)
-                        rp_warp_half<false>(h, lane, nchunks, lpl, sum32, qi, q2, w1, w2, nullptr, nullptr, p1, p2, e1, e2);
-                    if (sum32) {
-                        e1 = (i64)__reduce_add_sync(0xffffffffu, (unsigned)p1);
-                        e2 = (i64)__reduce_add_sync(0xffffffffu, (unsigned)p2);
-                    } else {
-                        e1 = warp_sum_i64(e1);
-                        e2 = warp_sum_i64(e2);
-                    }
-                }
-                // exact new score and the Metropolis decision, lane 0
-                const int c1 = m.c1, c2 = m.c2;
-                const int g1 = g_of[c1], g2 = g_of[c2];
-                i64 n0 = 0, n1 = 0, n2 = 0, A1 = 0, A2 = 0, J1n = 0, J2n = 0, U1n = 0, U2n = 0;
-                i64 Ta = 0, Qa = 0, Tb = 0, Qb = 0;
-                int fb0 = 0, fb2 = 0;
+                // ---- lane 0, while the copies are on their way: the part of the new score that needs
+                // only the cell statistics, and the accept bound
+                i64 S0 = 0, S1 = 0, S2 = 0, Ecur = 0, Ta = 0, Qa = 0, Tb = 0, Qb = 0, A1 = 0, A2 = 0;
+                i64 J1o = 0, J2o = 0, U1o = 0, U2o = 0;
+                u64 bound = 0;                      // accept when the energy rises by less than this
+                bool always = false;                // the bound does not fit 64 bits, or the threshold is saturated
                 if (lane == 0) {
-                    const i64 S0 = Sc[0], S1 = Sc[1], S2 = Sc[2];
+                    S0 = Sc[0]; S1 = Sc[1]; S2 = Sc[2]; Ecur = Sc[3];
                     const i64 ti = cand[ls].ti, t2 = cand[ls].t2;
                     Ta = (i64)T[c1] - ti + t2; Qa = (i64)Q[c1] - ti * ti + t2 * t2;
                     Tb = (i64)T[c2] + ti - t2; Qb = (i64)Q[c2] + ti * ti - t2 * t2;
-                    if (!touchW) { e1 = Esum[rg1]; e2 = e1; }
                     const i64 aC = dm.asum * dm.C, bS = dm.bsum;
                     if (ID) { A1 = aC * Ta + bS * Qa; A2 = aC * Tb + bS * Qb; }
                     else {
                         A1 = rp_attention(dm, st, dpl, dpo, rowbase[c1] / dm.D, g1, c1, Ta, Qa, c2, Tb, Qb);
                         A2 = touchW ? rp_attention(dm, st, dpl, dpo, rowbase[c2] / dm.D, g2, c1, Ta, Qa, c2, Tb, Qb) : A1;
                     }
-                    const i64 J1o = Jfx[rg1], J2o = Jfx[rg2];
+                    J1o = Jfx[rg1]; J2o = Jfx[rg2];
+                    U1o = U[g1]; U2o = U[g2];
+                    const StepRec rr = recs[ls];
+                    const u64 M = (u64)(Ecur > dm.SC ? Ecur : dm.SC);
+                    const u64 bh = __umul64hi(rr.thr, M), bl = rr.thr * M;
+                    always = (rr.flags & 4u) || (bh >> 31);
+                    bound = (bh << 32) | (bl >> 32);
+                }
+                i64 e1 = 0, e2 = 0;
+                if (touchW) {
+                    bool landed = rp_mbar_wait(mbar, phase, A.wait_polls);
+                    phase ^= 1u;
+                    // Inspection hook: chain 0 waits once more, on a phase that nothing completes.
+                    if (landed && A.stall_test && j == 0) landed = rp_mbar_wait(mbar, phase, A.wait_polls);
+                    if (!__all_sync(0xffffffffu, landed)) {
+                        // The bounded wait ran out: raise the status word and leave without storing anything (the
+                        // level barrier and every later level then do nothing, and rp_anneal reports the time-out).
+                        if (lane == 0) atomicExch(&A.status[RP_SW_TIMEOUT], 1);
+                        return;
+                    }
+                    rp_warp_staged_score(lane, dm.L, cpl, sum32, swap, s_qi, s_q2, s_w1, s_w2, e1, e2);
+                }
+                // ---- exact new score and the Metropolis decision, lane 0 ---------------------------------
+                i64 n0 = 0, n1 = 0, n2 = 0, J1n = 0, J2n = 0, U1n = 0, U2n = 0;
+                int fb0 = 0, fb2 = 0;
+                if (lane == 0) {
+                    if (!touchW) { e1 = Esum[rg1]; e2 = e1; }
                     J1n = A1 + dm.EC * e1; J2n = touchW ? A2 + dm.EC * e2 : J1n;
                     const i64 dJ1 = J1n - J1o, dJ2 = touchW ? J2n - J2o : 0;
-                    const i64 U1o = U[g1], U2o = U[g2];
                     if (g1 == g2) { U1n = U1o + dJ1 + dJ2; U2n = U1n; }
                     else { U1n = U1o + dJ1; U2n = U2o + dJ2; }
                     n1 = S1 + dJ1 + dJ2;
@@ -356,18 +374,8 @@ k_anneal_warp(const AnnealArgs A, const RpWarpLayout wl)
                 }
                 int acc_i = 0;
                 if (lane == 0) {
-                    const StepRec rr = recs[ls];
-                    const i64 Ecur = Sc[3];
-                    bool acc = rp_lex_less(n0, n1, n2, Sc[0], Sc[1], Sc[2]);
                     const i64 en = rp_energy(n0, n1, n2);
-                    if (!acc) {
-                        if (en <= Ecur || (rr.flags & 4u)) acc = true;
-                        else {
-                            const u64 M = (u64)(Ecur > dm.SC ? Ecur : dm.SC);
-                            const u64 bh = __umul64hi(rr.thr, M), bl = rr.thr * M;
-                            acc = (bh >> 31) ? true : ((u64)(en - Ecur) < ((bh << 32) | (bl >> 32)));
-                        }
-                    }
+                    const bool acc = rp_lex_less(n0, n1, n2, S0, S1, S2) || en <= Ecur || always || (u64)(en - Ecur) < bound;
                     chain->n_feas += 1;
                     if (touchW) chain->n_bytes += (i64)((swap ? 4 : 3) + (acc ? 2 : 0)) * LP * 4;
                     if (acc) {
@@ -385,8 +393,8 @@ k_anneal_warp(const AnnealArgs A, const RpWarpLayout wl)
                             }
                         }
                         const int k = kb + ls;
-                        rp_cell_wr<CG>(cell8, m.i, c2);
-                        if (swap) rp_cell_wr<CG>(cell8, m.i2, c1);
+                        cells[m.i] = (unsigned short)c2;
+                        if (swap) cells[m.i2] = (unsigned short)c1;
                         T[c1] = (int)Ta; Q[c1] = (u64)Qa; T[c2] = (int)Tb; Q[c2] = (u64)Qb;
                         if (!swap) { cnt[c1] -= 1; cnt[c2] += 1; }
                         Esum[rg1] = e1; Afx[rg1] = A1; Jfx[rg1] = J1n;
@@ -416,22 +424,29 @@ k_anneal_warp(const AnnealArgs A, const RpWarpLayout wl)
                 __syncwarp();                                               // lane 0's updates (slice table included) are visible
                 if (acc_i) {
                     if (touchW) {
-                        // The two slices are built once more (their sources are in L2 now) and stored
-                        // where the slice table points after lane 0's update: in place or to the spares.
+                        // the two new slices, stored where the slice table points after lane 0's update
                         int4 *o1 = (int4 *)(A.W + (size_t)wtab[rg1] * LP);
                         int4 *o2 = (int4 *)(A.W + (size_t)wtab[rg2] * LP);
-                        int p1 = 0, p2 = 0;
-                        i64 x1 = 0, x2 = 0;
-#pragma unroll
-                        for (int h = 0; h < (WARP_CHK + WARP_PART - 1) / WARP_PART; ++h)
-                            rp_warp_half<true>(h, lane, nchunks, lpl, sum32, qi, q2, w1, w2, o1, o2, p1, p2, x1, x2);
+                        rp_warp_staged_commit(lane, nchunks, swap, s_qi, s_q2, s_w1, s_w2, o1, o2);
+                        // these stores are read again by bulk copies: order them before the asynchronous proxy
+                        asm volatile("fence.proxy.async.global;" ::: "memory");
                     }
+                    // the cached cells of the steps still to come follow the move
+                    const bool rl = sr.flags & 1u;
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) {
+                        if (x >= 2 && rl) continue;
+                        if (sr.i[x] == m.i) sr.c[x] = c2;
+                        else if (swap && sr.i[x] == m.i2) sr.c[x] = c1;
+                    }
+                    __syncwarp();               // the staged copies have been read: the next candidate may overwrite them
                     next_pos = ls + 1;
                     fmask = 0;
                 }
             }
             pos = next_pos;
         }
+        __syncwarp();                           // lane 0's stores to the assignment come before the next batch's reads
     }
     __syncwarp();
 
@@ -440,15 +455,6 @@ k_anneal_warp(const AnnealArgs A, const RpWarpLayout wl)
         char *bdst = A.blob_dst + (size_t)j * A.bl.bytes;
         const int nh = A.bl.off_cell >> 2;
         for (int x = lane; x < nh; x += 32) ((int *)bdst)[x] = ((const int *)sm)[x];
-        if (!CG) {
-            unsigned short *cd = (unsigned short *)(bdst + A.bl.off_cell);
-            const int n4 = dm.N >> 2;
-            for (int x = lane; x < n4; x += 32) {
-                const u32 v = ((const u32 *)cell8)[x];
-                ((uint2 *)cd)[x] = make_uint2((v & 0xffu) | (((v >> 8) & 0xffu) << 16), ((v >> 16) & 0xffu) | ((v >> 24) << 16));
-            }
-            for (int i = (n4 << 2) + lane; i < dm.N; i += 32) cd[i] = (unsigned short)rp_cell_rd<false>(cell8, i);
-        }
         int *td = (int *)(bdst + A.bl.off_wtab);
         for (int rg = lane; rg < dm.RG; rg += 32) td[rg] = wtab[rg];
     }
@@ -475,44 +481,38 @@ k_level_end(const AnnealArgs A)
     rp_level_end(A, threadIdx.x, LEVEL_END_THREADS, smraw, rp_le_ws_bytes(A, A.smem_bytes));
 }
 
-// Windows the warp-per-chain kernel takes: slices in the pool, 16-byte chunks of L*P <= 1024 ints
-// with a power-of-two rank count, and more chains than the 128-thread kernel keeps resident (6 per
-// SM; fewer chains run faster with 128 threads each).
-// The assignment stays in shared memory, a byte per sample, wherever a cell fits a byte (faster:
-// proposals read it four times per step); else the chain works on its blob's 16-bit array in L2.
-static bool rp_warp_cells_global(const rp_ctx *c)
-{
-    return c->knob_chain_kernel == 3 || c->dm.K > 256;
-}
+// Windows the warp-per-chain kernel takes: slices in the pool, whole 16-byte chunks of L*P <= 1024
+// ints with a power-of-two rank count, and more chains than the 128-thread kernel keeps resident
+// (6 per SM; fewer chains finish sooner with 128 threads each).
 bool rp_uses_warp_chains(const rp_ctx *c)
 {
     const RpDims &dm = c->dm;
-    if (rp_uses_wpc(dm) || !rp_uses_slices(dm) || c->knob_stall) return false;
+    if (rp_uses_wpc(dm) || !rp_uses_slices(dm)) return false;
     const bool vec = (dm.P >= 4) && (dm.P <= 128) && ((dm.P & (dm.P - 1)) == 0);
-    if (!vec || dm.LP > WARP_CHK * 32 * 4) return false;
+    if (!vec || dm.LP > 1024) return false;
     if (c->knob_chain_kernel == 1) return false;
-    if (c->knob_chain_kernel < 2 && c->Ppop <= 148 * 6) return false;
-    const RpWarpLayout wl = rp_warp_layout(dm, c->bl, c->sl, dm.G == dm.D, rp_warp_cells_global(c));
+    if (c->knob_chain_kernel != 2 && c->Ppop <= 148 * 6) return false;
+    const RpWarpLayout wl = rp_warp_layout(dm, c->bl, c->sl, dm.G == dm.D);
     return wl.bytes <= 96 * 1024;
 }
 
-template <bool ID, bool CG>
+template <bool ID>
 static int launch_warp(rp_ctx *c, const AnnealArgs &A, const RpWarpLayout &wl)
 {
     if (wl.bytes > 32 * 1024)
-        RP_CUDA(cudaFuncSetAttribute(k_anneal_warp<ID, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize, wl.bytes));
-    k_anneal_warp<ID, CG><<<c->Ppop, 32, wl.bytes, c->stream>>>(A, wl);
+        RP_CUDA(cudaFuncSetAttribute(k_anneal_warp<ID>, cudaFuncAttributeMaxDynamicSharedMemorySize, wl.bytes));
+    k_anneal_warp<ID><<<c->Ppop, 32, wl.bytes, c->stream>>>(A, wl);
     RP_CUDA(cudaGetLastError());
     return RP_OK;
 }
 
 int rp_launch_anneal_warp(rp_ctx *c, AnnealArgs &A)
 {
-    const bool identity = (c->dm.G == c->dm.D), cg = rp_warp_cells_global(c);
-    const RpWarpLayout wl = rp_warp_layout(c->dm, c->bl, c->sl, identity, cg);
+    const bool identity = (c->dm.G == c->dm.D);
+    const RpWarpLayout wl = rp_warp_layout(c->dm, c->bl, c->sl, identity);
     A.smem_bytes = (unsigned)wl.bytes;
-    if (identity) { if (cg) RP_TRY((launch_warp<true, true>(c, A, wl))); else RP_TRY((launch_warp<true, false>(c, A, wl))); }
-    else { if (cg) RP_TRY((launch_warp<false, true>(c, A, wl))); else RP_TRY((launch_warp<false, false>(c, A, wl))); }
+    if (identity) RP_TRY(launch_warp<true>(c, A, wl));
+    else RP_TRY(launch_warp<false>(c, A, wl));
     // workspace of the barrier: cumulative weights and the replayed layout on chip where they fit
     size_t ws = 2 * std::max((size_t)c->Ppop * 8, (size_t)c->dm.N * 2);
     ws = std::min(std::max(ws, (size_t)16 * 1024), (size_t)200 * 1024);

@@ -1079,7 +1079,7 @@ extern "C" int rp_debug_set_knob(rp_ctx *c, int knob, int64_t value)
             if (value > 2) return RP_ERR_ARG;
             c->knob_slices = (int)value; return RP_OK;
         case RP_KNOB_CHAIN_KERNEL:
-            if (value > 3) return RP_ERR_ARG;
+            if (value > 2) return RP_ERR_ARG;
             c->knob_chain_kernel = (int)value; return RP_OK;
         default: return RP_ERR_ARG;
     }

@@ -361,18 +361,18 @@ WARP_CHAIN_CASES = [
     ("wc_shared", 151, 17, 64, 2, 4096, 4, 32, [0, 1, 1, 0], 2, 130),   # two DP slots per shard, odd sample count
     ("wc_p4", 140, 200, 16, 2, 4096, 4, 4, None, 3, 33),                # one lane per layer
     ("wc_p128", 100, 8, 128, 2, 4096, 3, 128, None, 2, 50),             # a whole warp per layer, L*P = 1024
-    ("wc_cells", 700, 16, 64, 2, 8192, 64, 64, None, 5, 24),            # 320 cells: the assignment stays in global memory
+    ("wc_cells", 700, 16, 64, 2, 8192, 64, 64, None, 5, 24),            # 320 cells
 ]
 
 
 @pytest.mark.parametrize("spec", WARP_CHAIN_CASES, ids=[e[0] for e in WARP_CHAIN_CASES])
-@pytest.mark.parametrize("kernel", [2, 3])
-def test_warp_per_chain_kernel_on_small_windows(spec, kernel):
+def test_warp_per_chain_kernel_on_small_windows(spec):
     """The chain kernel that full-size windows with thousands of chains use (one warp per chain),
-    forced onto small windows: the assignment as bytes in shared memory (2, where a cell fits a
-    byte) and as the blob's array in global memory (3), ragged chunk counts, one to 32 lanes per
-    layer, shared shards; the level barrier as a launch of its own, with all of its shared
-    memory and with next to none; a second rp_anneal call that resumes from the tables."""
+    forced onto small windows: ragged chunk counts, one to 32 chunks per layer, fewer layers than
+    lanes and more, shared shards, more than 256 cells; the level barrier as a launch of its own,
+    with all of its shared memory and with next to none; a second rp_anneal call that resumes
+    from the tables."""
+    kernel = 2
     name, N, L, E, k, C, D, P, edp, min_rows, pop = spec
     w = make_window(custom_spec(name, N, L, E, k, C, D, P, pop, 400, data_seed=len(name) * 13 + N))
     ref = oracle_front(w, edp, min_rows)
@@ -398,7 +398,8 @@ def test_warp_per_chain_kernel_on_small_windows(spec, kernel):
         rp.rp_destroy(ctx)
 
 
-@pytest.mark.parametrize("spec", [BARRIER_CASES[0], BARRIER_CASES[2]], ids=["warp_per_candidate", "cooperative"])
+@pytest.mark.parametrize("spec", [BARRIER_CASES[0], BARRIER_CASES[2], WARP_CHAIN_CASES[0]],
+                         ids=["warp_per_candidate", "cooperative", "warp_per_chain"])
 def test_a_wait_that_runs_out_is_reported_and_the_context_survives(spec):
     """One chain waits on a barrier phase that nothing completes, with the poll limit cut to 10^4:
     the wait gives up, the kernels return, rp_anneal reports RP_ERR_TIMEOUT, the calls that make no
@@ -410,6 +411,8 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_survives(spec):
     ref = oracle_front(w, edp, min_rows)
     ctx = load(w, pop=pop, edp=edp, min_rows=min_rows)
     check_front(w, ctx, ref)
+    if name.startswith("wc_"):
+        rp.rp_debug_set_knob(ctx, "CHAIN_KERNEL", 2)
     rp.rp_debug_set_knob(ctx, "WAIT_POLLS", 10000)
     rp.rp_debug_set_knob(ctx, "STALL_ONE_CHAIN", 1)
     for _ in range(2):                      # the second call finds the arrival counter and the status words clean
