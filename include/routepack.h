@@ -307,10 +307,10 @@ typedef enum {
  *   RP_KNOB_RANK_LOAD_SLICES (set before rp_pack_rows): how windows with L*P > 512 keep the rank
  *     loads of the population.  0 or 1 = shared slices with copy-on-write (the default), 2 = one
  *     private cell per member, copied whole when resampling replaces the member.
- *   RP_KNOB_CHAIN_KERNEL: which chain kernel windows with 512 < L*P <= 1024 and shared slices
- *     use.  0 = by population (one warp per chain when the chains outnumber what the 128-thread
- *     kernel keeps resident, else 128 threads per chain), 1 = always 128 threads per chain,
- *     2 = always one warp per chain. */
+ *   RP_KNOB_CHAIN_KERNEL: which chain kernel windows use whose rank loads live in the slice pool
+ *     (not on chip).  0 = one warp per chain, except for windows with L*P <= 512 and at most 592
+ *     members, which finish sooner with several warps per chain; 1 = always several warps per
+ *     chain; 2 = always one warp per chain. */
 typedef enum { RP_KNOB_BARRIER_WORKSPACE = 1, RP_KNOB_WAIT_POLLS = 2, RP_KNOB_STALL_ONE_CHAIN = 3,
                RP_KNOB_RANK_LOAD_SLICES = 4, RP_KNOB_LAUNCH_PER_LEVEL = 5, RP_KNOB_CHAIN_KERNEL = 6 } rp_knob;
 int rp_debug_set_knob(rp_ctx *ctx, int knob, int64_t value);

@@ -541,7 +541,7 @@ static void fill_args(rp_ctx *c, int level, int n_levels, const rp_anneal_params
     A.lo.done = c->d_done; A.lo.anc_out = c->d_anc_next; A.lo.F = c->d_F;
     A.lo.wloc_out = c->d_wloc; A.lo.scratch = c->d_le_scratch;   // the barrier rewrites the array the level read from
     A.lo.inc_layout = c->d_inc_layout; A.lo.inc_score = c->d_inc_score;
-    A.lo.cand_layout = use_wpc(c->dm) ? c->d_cand_layout : nullptr;
+    A.lo.cand_layout = (use_wpc(c->dm) && !rp_uses_warp_chains(c)) ? c->d_cand_layout : nullptr;
     A.lo.inc_slot = c->d_inc_slot;
     A.lo.tr_term = c->d_tr_term; A.lo.tr_best = c->d_tr_best; A.lo.tr_inc = c->d_tr_inc;
     A.lo.tr_best_step = c->d_tr_best_step; A.lo.tr_anc = c->d_tr_anc; A.lo.tr_digest = c->d_tr_digest;
@@ -595,8 +595,8 @@ int rp_launch_anneal_level(rp_ctx *c, int level, int n_levels, const rp_anneal_p
     AnnealArgs A;
     fill_args(c, level, n_levels, prm, rho_q32, guide_q32, A);
     if (rp_uses_slices(c->dm)) RP_TRY(rp_launch_slice_gc(c));
-    if (use_wpc(c->dm)) return rp_launch_anneal_wpc(c, A);
     if (rp_uses_warp_chains(c)) return rp_launch_anneal_warp(c, A);
+    if (use_wpc(c->dm)) return rp_launch_anneal_wpc(c, A);
     int nt; size_t smem;
     const bool alias = rp_anneal_smem_bytes(c, &nt, &smem) == 2;
     if (smem > 220 * 1024) return RP_ERR_RANGE;

@@ -1,10 +1,10 @@
-// Chain kernel of the population annealing for windows with more chains than the 128-thread
-// kernel keeps resident and slices of 512 < L*P <= 1024 ints: "warp per chain".
+// Chain kernel of the population annealing for windows whose rank loads live in the slice pool
+// and whose chains outnumber what the multi-warp kernels keep resident: "warp per chain".
 //
 // A chain of Algorithm 3 is a sequence of dependent rounds (proposal, the touched rank-load
 // slices and demand rows from L2 or HBM, exact rescoring in 64-bit integers, decision), so the
 // throughput of a level is the number of chains an SM keeps in flight over the latency of a round.
-// Here a chain is a single warp with about 23 KB of shared memory, nine to an SM:
+// Here a chain is a single warp (on the largest window: 23 KB of shared memory, nine to an SM):
 //  * the two demand rows and two slices of a candidate (4 * L*P ints) arrive in shared memory by
 //    four bulk asynchronous copies on one mbarrier (bounded wait): one trip to memory per
 //    candidate and no registers held while it lasts; lane 0 rebuilds the part of the score that
@@ -291,10 +291,12 @@ k_anneal_warp(const AnnealArgs A, const RpWarpLayout wl)
                     // their way from HBM to L2 now, one 128-byte line per lane and slice.
                     const int ln = __ffs(fmask) - 1;
                     const int ra = rg_of[cand[ln].m.c1], rb = rg_of[cand[ln].m.c2];
-                    if (ra != rb && lane * 32 < LP) {
-                        const int *pa = A.W + (size_t)wtab[ra] * LP + lane * 32, *pb = A.W + (size_t)wtab[rb] * LP + lane * 32;
-                        asm volatile("prefetch.global.L2 [%0];" ::"l"(pa));
-                        asm volatile("prefetch.global.L2 [%0];" ::"l"(pb));
+                    if (ra != rb) {
+                        const int *pa = A.W + (size_t)wtab[ra] * LP, *pb = A.W + (size_t)wtab[rb] * LP;
+                        for (int x = lane * 32; x < LP; x += 1024) {
+                            asm volatile("prefetch.global.L2 [%0];" ::"l"(pa + x));
+                            asm volatile("prefetch.global.L2 [%0];" ::"l"(pb + x));
+                        }
                     }
                 }
                 // ---- lane 0, while the copies are on their way: the part of the new score that needs
@@ -481,19 +483,21 @@ k_level_end(const AnnealArgs A)
     rp_level_end(A, threadIdx.x, LEVEL_END_THREADS, smraw, rp_le_ws_bytes(A, A.smem_bytes));
 }
 
-// Windows the warp-per-chain kernel takes: slices in the pool, whole 16-byte chunks of L*P <= 1024
-// ints with a power-of-two rank count, and more chains than the 128-thread kernel keeps resident
-// (6 per SM; fewer chains finish sooner with 128 threads each).
+// Windows the warp-per-chain kernel takes: rank loads as slices of the pool, layers of whole
+// 16-byte chunks (a power-of-two rank count of 4 to 128) and a chain that fits shared memory at
+// least twice per SM.  Where L*P <= 512 the warp-per-candidate kernel is the alternative: it
+// finishes a level sooner as long as all of its chains are resident at once (four per SM).
+#define WARP_MIN_CHAINS (148 * 4)
 bool rp_uses_warp_chains(const rp_ctx *c)
 {
     const RpDims &dm = c->dm;
-    if (rp_uses_wpc(dm) || !rp_uses_slices(dm)) return false;
+    if (!rp_uses_slices(dm)) return false;
     const bool vec = (dm.P >= 4) && (dm.P <= 128) && ((dm.P & (dm.P - 1)) == 0);
-    if (!vec || dm.LP > 1024) return false;
+    if (!vec) return false;
     if (c->knob_chain_kernel == 1) return false;
-    if (c->knob_chain_kernel != 2 && c->Ppop <= 148 * 6) return false;
+    if (c->knob_chain_kernel != 2 && rp_uses_wpc(dm) && c->Ppop <= WARP_MIN_CHAINS) return false;
     const RpWarpLayout wl = rp_warp_layout(dm, c->bl, c->sl, dm.G == dm.D);
-    return wl.bytes <= 96 * 1024;
+    return wl.bytes <= 100 * 1024;
 }
 
 template <bool ID>

@@ -276,14 +276,17 @@ def test_three_attention_stages_and_resume():
     rp.rp_destroy(ctx)
 
 
+@pytest.mark.parametrize("kernel", [1, 2], ids=["several_warps_per_chain", "warp_per_chain"])
 @pytest.mark.parametrize("name,pop,levels,steps", [("large", 96, 3, 60), ("wide", 48, 2, 40), ("heavy", 64, 2, 80)])
-def test_large_windows_full_shapes_reduced_budget(name, pop, levels, steps):
+def test_large_windows_full_shapes_reduced_budget(name, pop, levels, steps, kernel):
     """Full N, L, E, P, C, D of the three big windows (so the kernels run in the launch
     configuration of the full-size runs), with a population and step budget the oracle finishes
-    quickly; every trajectory is still compared bit for bit."""
+    quickly, on both chain kernels that take such windows; every trajectory is still compared bit
+    for bit."""
     w = make_window(name)
     ref = oracle_front(w)
     ctx = load(w, pop=pop, device_inputs=True)
+    rp.rp_debug_set_knob(ctx, "CHAIN_KERNEL", kernel)
     check_front(w, ctx, ref)
     check_eval(w, ctx, ref, None, n=2)
     check_anneal(w, ctx, ref, None, pop, levels, steps, check_members=2)
@@ -335,6 +338,7 @@ def test_level_barrier_paths_on_small_windows(spec, cap):
         rp.rp_debug_set_knob(ctx, "BARRIER_WORKSPACE", cap)
         rp.rp_debug_set_knob(ctx, "LAUNCH_PER_LEVEL", 1)    # the barrier in question is the one between launches
         rp.rp_debug_set_knob(ctx, "RANK_LOAD_SLICES", slices)
+        rp.rp_debug_set_knob(ctx, "CHAIN_KERNEL", 1)        # (L*P > 512: the 128-thread kernel, not one warp per chain)
         check_front(w, ctx, ref)
         want, stats = check_anneal(w, ctx, ref, edp, pop, 10, 40, t_ratio=0.6, check_members=2)
         assert stats.accepted > 50 and stats.improved > 0
@@ -411,8 +415,7 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_survives(spec):
     ref = oracle_front(w, edp, min_rows)
     ctx = load(w, pop=pop, edp=edp, min_rows=min_rows)
     check_front(w, ctx, ref)
-    if name.startswith("wc_"):
-        rp.rp_debug_set_knob(ctx, "CHAIN_KERNEL", 2)
+    rp.rp_debug_set_knob(ctx, "CHAIN_KERNEL", 2 if name.startswith("wc_") else 1)
     rp.rp_debug_set_knob(ctx, "WAIT_POLLS", 10000)
     rp.rp_debug_set_knob(ctx, "STALL_ONE_CHAIN", 1)
     for _ in range(2):                      # the second call finds the arrival counter and the status words clean
@@ -691,6 +694,43 @@ def test_fuzz_random_small_windows():
         check_front(w, ctx, ref)
         levels, steps = int(rng.integers(1, 5)), int(rng.choice([1, 7, 33, 130]))
         check_anneal(w, ctx, ref, edp, pop, levels, steps, t_ratio=float(rng.choice([0.3, 0.7, 1.0])), check_members=1)
+        rp.rp_destroy(ctx)
+
+
+def test_fuzz_warp_per_chain_kernel():
+    """Random windows whose rank loads live in the slice pool (L*P of 600 to 2000 with 4 to 64
+    ranks), random shard maps, attention stages, proposal mixes and schedules, on the
+    warp-per-chain kernel: every trajectory against the oracle."""
+    rng = np.random.default_rng(77)
+    for trial in range(12):
+        P = int(rng.choice([4, 8, 16, 32, 64]))
+        L = int(rng.integers(600 // P + 1, 2000 // P + 1))
+        H = int(rng.choice([1, 2]))
+        E = P * H
+        D = int(rng.choice([1, 2, 3, 4, 6]))
+        N = int(rng.integers(max(16, 4 * D), 140))
+        k = int(rng.choice([1, 2, 4]))
+        C = int(rng.choice([3000, 8192]))
+        G = int(rng.integers(1, D + 1))
+        edp = None if G == D else [int(x) for x in rng.permutation(np.concatenate([np.arange(G), rng.integers(0, G, D - G)]))]
+        S = int(rng.integers(1, 4))
+        alpha = tuple(float(x) for x in np.round(rng.uniform(0, 3, S) * 256) / 256)
+        beta = tuple(float(x) for x in np.round(rng.uniform(0, 3, S) * 256) / 256)
+        pop = int(rng.choice([1, 3, 9, 40]))
+        spec = custom_spec(f"wfuzz{trial}", N, L, E, k, C, D, P, pop, 0, data_seed=3000 + trial, alpha=alpha, beta=beta,
+                           p_reloc=float(rng.choice([0.0, 0.25, 0.6, 1.0])), p_guide=float(rng.choice([0.0, 0.5, 0.8, 1.0])),
+                           t0=float(rng.choice([1e-5, 1e-3, 5e-2])), anneal_seed=int(rng.integers(0, 2 ** 62)))
+        w = make_window(spec)
+        min_rows = int(rng.integers(1, 4))
+        ref = oracle_front(w, edp, min_rows)
+        if ref["R"] == 0:
+            continue
+        ctx = load(w, pop=pop, edp=edp, min_rows=min_rows)
+        rp.rp_debug_set_knob(ctx, "CHAIN_KERNEL", 2)
+        check_front(w, ctx, ref)
+        levels, steps = int(rng.integers(1, 5)), int(rng.choice([1, 7, 33, 70]))
+        _, stats = check_anneal(w, ctx, ref, edp, pop, levels, steps, t_ratio=float(rng.choice([0.3, 0.7, 1.0])), check_members=1)
+        assert stats.kernel_launches == levels * 4
         rp.rp_destroy(ctx)
 
 
