@@ -103,14 +103,16 @@ __device__ __forceinline__ bool rp_propose_regs(const RpDims &dm, const StepRegs
 // the lanes of a quarter warp start at different chunks of their layers, which keeps the 16-byte
 // reads off each other's banks.  cpl = 16-byte chunks per layer (a power of two).  Returns the
 // two sums over layers of the busiest ranks.
-__device__ __forceinline__ void rp_warp_staged_score(int lane, int L, int cpl, bool sum32, bool swap, const int4 *s_qi,
-                                                     const int4 *s_q2, const int4 *s_w1, const int4 *s_w2, i64 &e1, i64 &e2)
+template <int CPL>      // chunks per layer when known at compile time (the loop over them is then unrolled), else 0
+__device__ __forceinline__ void rp_warp_staged_score_t(int lane, int L, int cpl_rt, bool sum32, bool swap, const int4 *s_qi,
+                                                       const int4 *s_q2, const int4 *s_w1, const int4 *s_w2, i64 &e1, i64 &e2)
 {
+    const int cpl = CPL ? CPL : cpl_rt;
     int p1 = 0, p2 = 0;
     for (int ly = lane; ly < L; ly += 32) {
         const int base = ly * cpl;
         int m1 = 0, m2 = 0;
-#pragma unroll 4
+#pragma unroll (CPL ? CPL : 4)
         for (int k = 0; k < cpl; ++k) {
             const int c = base + ((k + lane) & (cpl - 1));
             int4 d = s_qi[c];
@@ -129,6 +131,13 @@ __device__ __forceinline__ void rp_warp_staged_score(int lane, int L, int cpl, b
         e1 = warp_sum_i64(e1);
         e2 = warp_sum_i64(e2);
     }
+}
+
+__device__ __forceinline__ void rp_warp_staged_score(int lane, int L, int cpl, bool sum32, bool swap, const int4 *s_qi,
+                                                     const int4 *s_q2, const int4 *s_w1, const int4 *s_w2, i64 &e1, i64 &e2)
+{
+    if (cpl == 8) rp_warp_staged_score_t<8>(lane, L, cpl, sum32, swap, s_qi, s_q2, s_w1, s_w2, e1, e2);
+    else rp_warp_staged_score_t<0>(lane, L, cpl, sum32, swap, s_qi, s_q2, s_w1, s_w2, e1, e2);
 }
 
 // An accepted move: the two new slices straight from the staged copies to where they now live,
@@ -279,7 +288,8 @@ k_anneal_warp(const AnnealArgs A, const RpWarpLayout wl)
                 if (touchW && lane == 0) {
                     // the candidate's rows and slices into shared memory: one trip, nothing in registers
                     const u32 bytes = (u32)LP * 4u;
-                    rp_fence_async_smem();          // the previous candidate's reads of the staging area come first
+                    // (the previous candidate's reads of the staging area are complete: their values were used
+                    // before the warp-wide barrier that precedes this point)
                     rp_mbar_expect_tx(mbar, (swap ? 4u : 3u) * bytes);
                     rp_bulk_g2s(s_qi, A.q + (size_t)m.i * LP, bytes, mbar);
                     if (swap) rp_bulk_g2s(s_q2, A.q + (size_t)m.i2 * LP, bytes, mbar);
