@@ -215,6 +215,8 @@ def plan_once(rp, w, t_in, a_in, outs, stream, stages=None, knobs=None):
         rp.rp_debug_set_knob(ctx, k, v)
     rp.rp_place_experts(ctx, outs["pi"], outs["rank_load"])
     rp.rp_pack_rows(ctx)
+    if stages is not None:
+        stages["chain_kernel"] = rp.rp_debug_chain_kernel(ctx)
     stats = rp.rp_anneal(ctx, n_levels=s.n_levels, steps_per_level=s.steps_per_level, t0=s.t0,
                          t_ratio=s.t_ratio, p_reloc=s.p_reloc, p_guide=s.p_guide, want_stats=True)
     rp.rp_best(ctx, outs["layout"], outs["score_fx"], outs["score_f64"])
@@ -313,6 +315,7 @@ def measure(rp, torch, args, name, steps, min_seconds, dist, dev, local, cpu_sec
     rp.rp_debug_set_stage_timing(True)
     timed_loop(t_dev, a_dev, outs_dev, n_st, stages)
     rp.rp_debug_set_stage_timing(False)
+    chain_kernel = stages.pop("chain_kernel")
     stages = {k: v / n_st for k, v in stages.items()}
 
     ms, total_moves = reduce_job(res["ms"], moves_per_step * steps, dist, dev)
@@ -323,7 +326,6 @@ def measure(rp, torch, args, name, steps, min_seconds, dist, dev, local, cpu_sec
     per_launch_s = res["chain_ms"] * 1e-3 / nl
     alg = (res["move_bytes"] + res["gather_bytes"]) / nl
     achieved = alg / per_launch_s / 1e9
-    chain_kernel = "k_anneal_wpc" if s.n_layers * s.ep_width <= 512 else "k_anneal_level"
     roofline = {"bound": "hbm", "kernel": chain_kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_source": peak_kind, "served_by": "L2+HBM (algorithmic bytes; see dram)",
                 "traffic": None, "algorithmic_bytes_per_launch": alg,

@@ -340,6 +340,10 @@ int rp_debug_philox(const uint32_t *ctr, const uint32_t key[2], uint32_t *out, i
  * measured L2 read rate that kernels whose operands L2 serves are set against.  Allocates and
  * frees its own buffer; runs on the default stream of the current device. */
 int rp_debug_l2_read_rate(int64_t bytes, int32_t reps, double *gb_per_s);
+/* Which chain kernel rp_anneal runs for this context (valid after rp_pack_rows; inspection only):
+ * 0 = warp per candidate (k_anneal_wpc), 1 = 128 threads per chain (k_anneal_level), 2 = warp per
+ * chain (k_anneal_warp). */
+int rp_debug_chain_kernel(rp_ctx *ctx, int32_t *which);
 /* Number of kernels this library has launched in this process so far. */
 int64_t rp_debug_launch_count(void);
 

@@ -25,7 +25,8 @@ RP_OK = 0
 EXPORTS = ("rp_window_load", "rp_place_experts", "rp_pack_rows", "rp_seed_population", "rp_pair_population", "rp_select_population", "rp_init_population", "rp_eval_population", "rp_eval_layouts_noalloc", "rp_diagnostics", "rp_anneal",
            "rp_best", "rp_destroy", "rp_release_cached_memory", "rp_strerror", "rp_last_cuda_error", "rp_debug_dump",
            "rp_debug_set_trace", "rp_debug_set_knob", "rp_debug_set_stage_timing", "rp_debug_stage_times",
-           "rp_debug_nl2", "rp_debug_exp2neg", "rp_debug_philox", "rp_debug_launch_count", "rp_debug_l2_read_rate")
+           "rp_debug_nl2", "rp_debug_exp2neg", "rp_debug_philox", "rp_debug_launch_count", "rp_debug_l2_read_rate",
+           "rp_debug_chain_kernel")
 
 
 class RpError(RuntimeError):
@@ -100,6 +101,7 @@ def lib():
         L.rp_debug_philox.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64]
         L.rp_debug_launch_count.restype = C.c_int64
         L.rp_debug_l2_read_rate.argtypes = [C.c_int64, C.c_int32, C.POINTER(C.c_double)]
+        L.rp_debug_chain_kernel.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
         _lib = L
     return _lib
 
@@ -335,6 +337,16 @@ def rp_debug_l2_read_rate(nbytes: int = 32 << 20, reps: int = 50) -> float:
     out = C.c_double(0.0)
     _check(lib().rp_debug_l2_read_rate(nbytes, reps, C.byref(out)), "rp_debug_l2_read_rate")
     return float(out.value)
+
+
+CHAIN_KERNELS = ("k_anneal_wpc", "k_anneal_level", "k_anneal_warp")
+
+
+def rp_debug_chain_kernel(ctx: Context) -> str:
+    """Name of the chain kernel rp_anneal runs for this context (after rp_pack_rows)."""
+    out = C.c_int32(-1)
+    _check(lib().rp_debug_chain_kernel(ctx.handle, C.byref(out)), "rp_debug_chain_kernel")
+    return CHAIN_KERNELS[out.value]
 
 
 def rp_debug_launch_count() -> int:

@@ -9,9 +9,8 @@
 //    four bulk asynchronous copies on one mbarrier (bounded wait): one trip to memory per
 //    candidate and no registers held while it lasts; lane 0 rebuilds the part of the score that
 //    needs only the cell statistics in the meantime;
-//  * the busiest rank of every layer is found with a lane per layer (no shuffles), an accepted
-//    move is stored straight from the staged copies, and the slices of the candidate that
-//    follows are prefetched into L2 while this one is decided;
+//  * the busiest rank of every layer is found with a lane per layer (no shuffles), and an accepted
+//    move is stored straight from the staged copies;
 //  * the random words of the next 32 steps, the cells of their candidate samples and those
 //    samples' lengths are fetched once per batch, one step per lane, and kept in registers; an
 //    accepted move patches the cached cells, so a proposal reads shared memory only;
@@ -137,6 +136,7 @@ __device__ __forceinline__ void rp_warp_staged_score(int lane, int L, int cpl, b
                                                      const int4 *s_q2, const int4 *s_w1, const int4 *s_w2, i64 &e1, i64 &e2)
 {
     if (cpl == 8) rp_warp_staged_score_t<8>(lane, L, cpl, sum32, swap, s_qi, s_q2, s_w1, s_w2, e1, e2);
+    else if (cpl == 4) rp_warp_staged_score_t<4>(lane, L, cpl, sum32, swap, s_qi, s_q2, s_w1, s_w2, e1, e2);
     else rp_warp_staged_score_t<0>(lane, L, cpl, sum32, swap, s_qi, s_q2, s_w1, s_w2, e1, e2);
 }
 
@@ -295,19 +295,6 @@ k_anneal_warp(const AnnealArgs A, const RpWarpLayout wl)
                     if (swap) rp_bulk_g2s(s_q2, A.q + (size_t)m.i2 * LP, bytes, mbar);
                     rp_bulk_g2s(s_w1, w1, bytes, mbar);
                     rp_bulk_g2s(s_w2, w2, bytes, mbar);
-                }
-                if (fmask) {
-                    // The candidate after this one is scored if this one is rejected: start its two slices on
-                    // their way from HBM to L2 now, one 128-byte line per lane and slice.
-                    const int ln = __ffs(fmask) - 1;
-                    const int ra = rg_of[cand[ln].m.c1], rb = rg_of[cand[ln].m.c2];
-                    if (ra != rb) {
-                        const int *pa = A.W + (size_t)wtab[ra] * LP, *pb = A.W + (size_t)wtab[rb] * LP;
-                        for (int x = lane * 32; x < LP; x += 1024) {
-                            asm volatile("prefetch.global.L2 [%0];" ::"l"(pa + x));
-                            asm volatile("prefetch.global.L2 [%0];" ::"l"(pb + x));
-                        }
-                    }
                 }
                 // ---- lane 0, while the copies are on their way: the part of the new score that needs
                 // only the cell statistics, and the accept bound

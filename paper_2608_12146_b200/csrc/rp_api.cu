@@ -1216,6 +1216,14 @@ __global__ void k_dbg_l2_read(const int4 *__restrict__ buf, long long n4, int re
     if (acc == 0x7fffffff) *sink = acc;          // never true for the zeroed buffer: keeps the loads alive
 }
 
+extern "C" int rp_debug_chain_kernel(rp_ctx *c, int32_t *which)
+{
+    if (!c || !which) return RP_ERR_ARG;
+    if (c->stage < 3) return RP_ERR_STATE;
+    *which = rp_uses_warp_chains(c) ? 2 : (rp_uses_wpc(c->dm) ? 0 : 1);
+    return RP_OK;
+}
+
 extern "C" int rp_debug_l2_read_rate(int64_t bytes, int32_t reps, double *gb_per_s)
 {
     if (!gb_per_s || bytes < (1 << 20) || bytes > (1ll << 31) || reps < 1 || reps > 10000) return RP_ERR_ARG;
