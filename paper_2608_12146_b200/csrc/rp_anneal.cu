@@ -7,9 +7,15 @@
 // (assignment, cell statistics, per-row-shard costs, shard work) lives in shared memory.
 // Its rank-load tensor W[R][G][L][P] lives in shared memory too when it fits beside a
 // second CTA on the SM (small windows), else in global memory as slices of L*P ints that a
-// member shares with its ancestor until it rewrites them (see AnnealArgs; many CTAs per SM
-// hide the latency of L2 and HBM).  The sample demand rows q[i][L][P] are shared by all
-// chains and stay L2-resident.
+// member shares with its ancestor until it rewrites them (see AnnealArgs).  The sample demand
+// rows q[i][L][P] are shared by all chains and stay L2-resident.
+//
+// Three chain kernels: warp per candidate (rp_anneal_wpc.cu: rank loads on chip, or L*P <= 512
+// with at most 592 members), warp per chain (rp_anneal_warp.cu: every other window whose rank
+// loads are slices of the pool and whose ranks are a power of two from 4 to 128), and the
+// 128-thread kernel of this file for what is left (other rank counts, chains too large for the
+// staging area of the warp-per-chain kernel, private rank-load cells) and for comparison
+// (RP_KNOB_CHAIN_KERNEL).
 //
 // A chain is a sequential process, but three things about it are not:
 //  * every random number is a pure function of (step, level, slot), so the proposal words
@@ -22,9 +28,9 @@
 //  * scoring a move is a data-parallel pass over two L*P slices.
 // Resampling is folded into the next level's prologue: slot j starts from the terminal
 // state of its ancestor in the other population buffer, so no separate gather pass runs.
-// The trajectory-best layout of the cooperative kernel below is not copied: every accepted move
-// is logged (8 bytes) and the level barrier rebuilds the one winning layout from the chain's
-// start layout and its log (the warp-per-candidate kernel snapshots the layout instead).
+// The trajectory-best layout of the kernel below (and of the warp-per-chain kernel) is not copied:
+// every accepted move is logged (8 bytes) and the level barrier rebuilds the one winning layout from
+// the chain's start layout and its log (the warp-per-candidate kernel snapshots the layout instead).
 //
 // Algorithmic bytes per feasible move: reads 2 W slices + the moved samples' q rows
 // ((3 or 4) * L*P*4 bytes), writes 2 W slices when accepted.
@@ -40,9 +46,9 @@ struct ChainB {                 // bookkeeping of the chain within this level
     int mt[SPEC][2];                        // lengths of the samples each feasible proposal moves
 };
 
-// Cooperative chain kernel for bandwidth-bound windows (L*P > 512): all NT threads score one
-// candidate at a time (two L*P slices of W from global memory plus the moved samples' demand
-// rows, 16-byte loads); the leading warp rebuilds the score and decides.
+// Chain kernel with NT threads per chain: all of them score one candidate at a time (two L*P
+// slices of W from global memory plus the moved samples' demand rows, 16-byte loads into
+// registers); the leading warp rebuilds the score and decides.
 template <int NT, int MINB, bool SL, bool ALIAS>
 __global__ void __launch_bounds__(NT, MINB)
 k_anneal_level(const AnnealArgs A)
@@ -369,14 +375,15 @@ k_anneal_level(const AnnealArgs A)
 }
 
 // Thread count and shared-memory plan of the chain kernels.  Windows with L*P <= 512 use the
-// warp-per-candidate kernel; larger ones the cooperative kernel with 128 threads.
+// warp-per-candidate kernel; larger ones the kernel above with 128 threads (unless the
+// warp-per-chain kernel takes the window, see rp_launch_anneal_level).
 size_t rp_wpc_smem_bytes(const RpDims &dm, const RpBlob &bl, const RpStatic &sl, int nw, int *w_in_smem);
 int rp_wpc_warps(int pop_size);
 int rp_launch_anneal_wpc(rp_ctx *c, const AnnealArgs &A);
 
 static bool use_wpc(const RpDims &dm) { return dm.LP <= 512; }
 bool rp_uses_wpc(const RpDims &dm) { return use_wpc(dm); }
-// Rank loads in global memory are kept as shared slices (see AnnealArgs); the cooperative kernel
+// Rank loads in global memory are kept as shared slices (see AnnealArgs); the 128-thread kernel
 // can also keep one private cell per member (inspection hook; slower wherever resampling replaces
 // many members, never faster).  Decided when the row count is known and kept in the dimensions.
 bool rp_uses_slices(const RpDims &dm) { return dm.slices != 0; }
@@ -463,7 +470,7 @@ int rp_launch_slice_gc(rp_ctx *c)
     return RP_OK;
 }
 
-// Resident chains per SM of the cooperative kernel: six (80 registers) keep the most bytes in
+// Resident chains per SM of the 128-thread kernel: six (80 registers) keep the most bytes in
 // flight; windows whose rank loads per member pass a megabyte run faster with five (96 registers,
 // no spills; their working set misses L2 either way).
 static int rp_coop_chains_per_sm(const RpDims &dm)

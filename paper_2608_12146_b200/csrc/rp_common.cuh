@@ -171,7 +171,7 @@ struct rp_ctx {
     int trace_on;              // keep per-level traces (inspection hook; off by default)
     int knob_level_launches;   // 1 = one launch per level even where one launch for all levels is possible
     int knob_chain_kernel;     // 1 = 128 threads per chain, 2 = one warp per chain, wherever the window allows both
-    int knob_slices;           // inspection hook: 0 = automatic, 1 = slices wherever the cooperative kernel runs, 2 = never
+    int knob_slices;           // inspection hook: 0 = automatic, 1 = slices wherever L*P > 512, 2 = never
     int knob_le_ws_cap, knob_wait_polls, knob_stall;   // inspection hooks (rp_debug_set_knob); 0 = off
     cudaEvent_t ev_stage[RP_STAGE_EVENTS];             // stage timing (rp_debug_set_stage_timing); null when off
     unsigned ev_recorded;                              // bit x: ev_stage[x] has been recorded
