@@ -324,6 +324,9 @@ k_anneal_warp(const AnnealArgs A, const RpWarpLayout wl)
                 i64 e1 = 0, e2 = 0;
                 if (touchW) {
                     bool landed = rp_mbar_wait(mbar, phase, A.wait_polls);
+                    // (once more before giving up, so that a copy still in flight has had twice the limit to land
+                    // before this chain's shared memory is handed to another one)
+                    if (!landed) landed = rp_mbar_wait(mbar, phase, A.wait_polls);
                     phase ^= 1u;
                     // Inspection hook: chain 0 waits once more, on a phase that nothing completes.
                     if (landed && A.stall_test && j == 0) landed = rp_mbar_wait(mbar, phase, A.wait_polls);
