@@ -592,6 +592,8 @@ def run_cuda(args):
             line["l2_read_gbs"] = l2
             line["eval_population"] = [eval_stage(rp, torch, n, dev, l2) for n in ("medium", "large", "wide")]
             line["concurrent_plans"] = [concurrent_plans(rp, torch, "medium", dev, n, 200, pl) for pl in (1, 0) for n in (1, 2, 4)]
+            # large: one warp per chain and 7 warps per SM for a single window, so several windows fit the SMs at once
+            line["concurrent_plans"] += [concurrent_plans(rp, torch, "large", dev, n, 60, 0) for n in (1, 2, 4)]
             line["single_plan_latency"] = [one_launch_latency(rp, torch, n, dev) for n in ("tiny", "medium")]
             line["seeding_stages"] = [seeding_stages(rp, torch, "medium", dev), seeding_stages(rp, torch, "heavy", dev, per_stage=False)]
             line["mechanism_diagnostics"] = [mechanism_diagnostics(rp, torch, n, dev) for n in ("medium", "large")]
