@@ -359,6 +359,29 @@ def test_level_barrier_paths_on_small_windows(spec, cap):
         rp.rp_destroy(ctx)
 
 
+OTHER_RANK_CASES = [
+    # name, N, L, E, k, C, D, P, edp, min_rows, pop: L*P > 512 with rank counts that are not a power of two from 4 to 128
+    ("ranks_48", 100, 12, 48, 2, 4096, 4, 48, None, 3, 30),
+    ("ranks_2", 90, 300, 4, 2, 4096, 3, 2, [0, 1, 0], 2, 21),
+    ("ranks_3", 64, 180, 6, 1, 3000, 2, 3, None, 4, 9),
+]
+
+
+@pytest.mark.parametrize("spec", OTHER_RANK_CASES, ids=[e[0] for e in OTHER_RANK_CASES])
+def test_slice_pool_windows_with_other_rank_counts(spec):
+    """Windows whose rank loads live in the slice pool but whose rank count the warp-per-chain
+    kernel does not take (its layers must be whole 16-byte chunks): the 128-thread kernel runs them
+    by default, with its element-wise scoring loop."""
+    name, N, L, E, k, C, D, P, edp, min_rows, pop = spec
+    w = make_window(custom_spec(name, N, L, E, k, C, D, P, pop, 400, data_seed=len(name) * 17 + N))
+    ref = oracle_front(w, edp, min_rows)
+    ctx = load(w, pop=pop, edp=edp, min_rows=min_rows)
+    check_front(w, ctx, ref)
+    want, stats = check_anneal(w, ctx, ref, edp, pop, 6, 40, t_ratio=0.6, check_members=2)
+    assert stats.accepted > 0 and stats.kernel_launches == 6 * 3
+    rp.rp_destroy(ctx)
+
+
 WARP_CHAIN_CASES = [
     # name, N, L, E, k, C, D, P, edp, min_rows, pop: windows with 512 < L*P <= 1024 for the warp-per-chain kernel
     ("wc_ragged", 120, 20, 32, 2, 4096, 4, 32, None, 3, 40),            # 160 chunks of 16 bytes: 5 per lane
