@@ -25,6 +25,7 @@
 #include "rp_level_end.cuh"
 
 #define WARP_CHAINS_PER_SM 9            // resident chains the register budget is set for
+#define WARP_SMEM_OPTIN (208 * 1024)    // dynamic shared memory these kernels may ask for (227 KB per CTA on sm_100a, less their static arrays)
 
 struct CandW { MoveS m; int ti, t2, pad; };          // a feasible proposal and the lengths of the moved samples
 struct ChainW {                                      // bookkeeping of the chain within this level
@@ -503,8 +504,9 @@ bool rp_uses_warp_chains(const rp_ctx *c)
 template <bool ID>
 static int launch_warp(rp_ctx *c, const AnnealArgs &A, const RpWarpLayout &wl)
 {
-    if (wl.bytes > 32 * 1024)
-        RP_CUDA(cudaFuncSetAttribute(k_anneal_warp<ID>, cudaFuncAttributeMaxDynamicSharedMemorySize, wl.bytes));
+    // (always the same value, above anything a launch asks for: contexts that plan different
+    // windows at once on different host threads then never lower each other's limit)
+    RP_CUDA(cudaFuncSetAttribute(k_anneal_warp<ID>, cudaFuncAttributeMaxDynamicSharedMemorySize, WARP_SMEM_OPTIN));
     k_anneal_warp<ID><<<c->Ppop, 32, wl.bytes, c->stream>>>(A, wl);
     RP_CUDA(cudaGetLastError());
     return RP_OK;
@@ -523,8 +525,7 @@ int rp_launch_anneal_warp(rp_ctx *c, AnnealArgs &A)
     ws = (ws + 15) & ~(size_t)15;
     AnnealArgs B = A;
     B.smem_bytes = (unsigned)ws;
-    if (ws > 32 * 1024)
-        RP_CUDA(cudaFuncSetAttribute(k_level_end, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ws));
+    RP_CUDA(cudaFuncSetAttribute(k_level_end, cudaFuncAttributeMaxDynamicSharedMemorySize, WARP_SMEM_OPTIN));
     k_level_end<<<1, LEVEL_END_THREADS, ws, c->stream>>>(B);
     g_rp_launches += 2;
     RP_CUDA(cudaGetLastError());
