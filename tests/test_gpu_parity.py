@@ -757,6 +757,56 @@ def test_fuzz_warp_per_chain_kernel():
         rp.rp_destroy(ctx)
 
 
+def test_windows_planned_at_once_on_separate_streams():
+    """Three different windows (a warp-per-chain one with more than 32 KB of shared memory per
+    chain, a second warp-per-chain one, and one whose rank loads live on chip) planned at the same
+    time by three host threads, each on its own stream and context, several plans each: every
+    plan equals the oracle's, so nothing process-wide (shared-memory limits of the kernels, memory
+    pools, launch counters) is upset by another context."""
+    import threading
+    import torch
+    cases = [("conc_a", 90, 40, 32, 2, 4096, 4, 32, None, 3, 37),        # L*P = 1280
+             ("conc_b", 120, 20, 32, 2, 4096, 4, 32, [0, 1, 1, 0], 3, 25),
+             ("conc_c", 96, 5, 16, 2, 4096, 4, 4, None, 3, 40)]
+    jobs = []
+    for name, N, L, E, k, C, D, P, edp, min_rows, pop in cases:
+        w = make_window(custom_spec(name, N, L, E, k, C, D, P, pop, 400, data_seed=len(name) * 19 + N))
+        s = w.spec
+        ref = oracle_front(w, edp, min_rows)
+        want = oracle.anneal(w.lengths, ref["q"], np.tile(ref["seed"], (pop, 1)), ref["R"], s.token_cap, D, n_levels=6, steps=40,
+                             t0=s.t0, t_ratio=0.6, p_reloc=s.p_reloc, p_guide=s.p_guide, seed=s.anneal_seed, edp_of_dp=edp,
+                             alpha=s.alpha, beta=s.beta)
+        jobs.append((w, edp, min_rows, pop, want))
+    errors = []
+
+    def worker(job):
+        try:
+            w, edp, min_rows, pop, want = job
+            s = w.spec
+            stream = torch.cuda.Stream()
+            for _ in range(6):
+                ctx = rp.rp_window_load(w.lengths, w.demand, top_k=s.top_k, token_cap=s.token_cap, dp_width=s.dp_width,
+                                        ep_width=s.ep_width, pop_size=pop, edp_of_dp=edp, alpha=s.alpha, beta=s.beta,
+                                        min_rows=min_rows, seed=s.anneal_seed, stream=stream)
+                rp.rp_place_experts(ctx)
+                rp.rp_pack_rows(ctx)
+                st = rp.rp_anneal(ctx, n_levels=6, steps_per_level=40, t0=s.t0, t_ratio=0.6, p_reloc=s.p_reloc, p_guide=s.p_guide)
+                layout, fx, _ = rp.rp_best(ctx)
+                assert [st.proposed, st.feasible, st.accepted, st.improved] == want["counters"].tolist()
+                assert (layout == want["best_layout"]).all() and (fx == want["best_score"]).all()
+                assert (rp.rp_debug_dump(ctx, "POPULATION", (pop, s.n_samples), np.int32) == want["final_pop"]).all()
+                rp.rp_destroy(ctx)
+        except Exception as e:          # reported by the main thread
+            errors.append(repr(e))
+
+    threads = [threading.Thread(target=worker, args=(j,)) for j in jobs]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+
+
 @pytest.mark.parametrize("name,pop", [("tiny", 8), ("medium", 256), ("medium", 100), ("large", 300)])
 def test_annealing_without_the_inspection_hook(name, pop):
     """The per-level traces are an inspection hook: counters, final population, incumbent and
