@@ -215,21 +215,32 @@ __device__ __forceinline__ i64 sel_both(const int *__restrict__ list, const int 
 }
 
 __global__ void __launch_bounds__(SEL_THREADS)
-k_sel_dist(RpDims dm, int Ppop, int n_proj, const int *__restrict__ rep, SelBuf B, i64 *__restrict__ dist)
+k_sel_dist(RpDims dm, int Ppop, int n_proj, const int *__restrict__ rep, SelBuf B, i64 *__restrict__ dist, int cells_by_table)
 {
     const int a = blockIdx.x, b = blockIdx.y;
     if (b <= a) { if (a == b && threadIdx.x == 0) dist[(size_t)a * Ppop + a] = 0; return; }
     if (!rep[a] || !rep[b]) return;
     __shared__ i64 acc[3];
     __shared__ int tab[SEL_TABLE];                 // row-by-row contingency counts when R*R fits
+    extern __shared__ int ctab[];                  // cell-by-cell contingency counts when K*K ints fit (cells_by_table)
     const int tid = threadIdx.x;
     const int N = dm.N, K = dm.K, R = dm.R, D = dm.D;
     const bool rows_by_table = R * R <= SEL_TABLE;
     if (tid < 3) acc[tid] = 0;
     if (rows_by_table) for (int x = tid; x < R * R; x += SEL_THREADS) tab[x] = 0;
+    if (cells_by_table) for (int x = tid; x < K * K; x += SEL_THREADS) ctab[x] = 0;
     __syncthreads();
     const int *la = B.lay + (size_t)a * N, *lb = B.lay + (size_t)b * N;
-    i64 bc = sel_both(B.clist + (size_t)a * N, B.cstart + (size_t)a * (K + 1), K, lb, 1, tid);
+    i64 bc = 0;
+    if (cells_by_table) {
+        // pairs in the same cell of both plans = sum over (cell of a, cell of b) of C(count, 2): N counts
+        // instead of one look-up per pair of a cell's samples (cells of hundreds of samples)
+        for (int i = tid; i < N; i += SEL_THREADS) atomicAdd(&ctab[la[i] * K + lb[i]], 1);
+        __syncthreads();
+        for (int x = tid; x < K * K; x += SEL_THREADS) { const i64 n = ctab[x]; bc += n * (n - 1) / 2; }
+    } else {
+        bc = sel_both(B.clist + (size_t)a * N, B.cstart + (size_t)a * (K + 1), K, lb, 1, tid);
+    }
     i64 br = 0;
     if (rows_by_table) {
         // pairs in the same row of both plans = sum over (row of a, row of b) of C(count, 2)
@@ -391,7 +402,14 @@ int rp_launch_select(rp_ctx *c, int *lay, int *out, const i64 *score, int n_proj
             e = cudaMemsetAsync(dist, 0, sizeof(i64) * P * P, c->stream);
         }
         if (e == cudaSuccess) {
-            k_sel_dist<<<dim3((unsigned)P, (unsigned)P), SEL_THREADS, 0, c->stream>>>(dm, (int)P, n_proj, rep, B, dist);
+            // cell-by-cell counts in shared memory where they fit twice per SM beside the row table
+            const size_t ctab_bytes = sizeof(int) * (size_t)dm.K * dm.K;
+            const int cells_by_table = ctab_bytes <= 80 * 1024;
+            if (cells_by_table && ctab_bytes > 24 * 1024)
+                e = cudaFuncSetAttribute(k_sel_dist, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024);
+            if (e == cudaSuccess)
+                k_sel_dist<<<dim3((unsigned)P, (unsigned)P), SEL_THREADS, cells_by_table ? ctab_bytes : 0, c->stream>>>(
+                    dm, (int)P, n_proj, rep, B, dist, cells_by_table);
             k_sel_greedy<<<1, GREEDY_THREADS, 0, c->stream>>>((int)P, rep, score, dist, eta_q16, mind, pen, order, n_distinct);
             k_sel_fill<<<(int)P, 256, 0, c->stream>>>(dm.N, order, lay, out);
             g_rp_launches += 6;
