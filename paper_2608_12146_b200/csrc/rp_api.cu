@@ -602,23 +602,38 @@ extern "C" int rp_eval_population(rp_ctx *c, const int32_t *layouts, int32_t n, 
 // from scratch and the incumbent becomes the best of them.
 // Scores `lay` [P_pop][N] from scratch, makes it the population (member m owns rank-load cell m)
 // and makes the best member the incumbent (lowest index on ties).
-static int install_population(rp_ctx *c, const int *lay)
+// Members n_distinct, n_distinct + 1, ... repeat the first n_distinct layouts in turn: member m descends
+// from member m mod n_distinct (whose state it reads when the first level starts) and works in a
+// rank-load cell of the other half, as the members of a freshly built population do.
+__global__ void k_descend_cyclic(int P, int nd, int *__restrict__ anc, int *__restrict__ wloc, int *__restrict__ wloc_next)
+{
+    const int m = blockIdx.x * blockDim.x + threadIdx.x;
+    if (m < P) { anc[m] = m % nd; wloc[m] = m % nd; wloc_next[m] = P + m; }
+}
+
+// n_distinct > 0: rows n_distinct .. P_pop-1 of `lay` repeat the first n_distinct rows cyclically, so
+// only those are scored and every other member descends from its original (no state is copied).
+static int install_population(rp_ctx *c, const int *lay, int n_distinct = 0)
 {
     const size_t P = (size_t)c->Ppop;
+    const size_t ne = (n_distinct > 0 && (size_t)n_distinct < P) ? (size_t)n_distinct : P;
     c->best_ready = 0;
     i64 *best = nullptr;
     RP_TRY(dev_alloc(c, &best, 3));
-    int st = ensure_eval_scratch(c, P, false);
-    if (st == RP_OK) st = rp_launch_cells_from_layouts(c, lay, (int)P, c->d_eval_cells);
+    int st = ensure_eval_scratch(c, ne, false);
+    if (st == RP_OK) st = rp_launch_cells_from_layouts(c, lay, (int)ne, c->d_eval_cells);
     c->cur = 0;
-    if (st == RP_OK) st = rp_launch_eval(c, c->d_eval_cells, (int)P, c->d_W, c->buf[0].blob, c->d_eval_score, nullptr);
-    if (st == RP_OK) {
+    if (st == RP_OK) st = rp_launch_eval(c, c->d_eval_cells, (int)ne, c->d_W, c->buf[0].blob, c->d_eval_score, nullptr);
+    if (st == RP_OK && ne == P) {
         k_iota<<<(int)((P + 255) / 256), 256, 0, c->stream>>>(c->d_wloc, (int)P, 0);
         k_iota<<<(int)((P + 255) / 256), 256, 0, c->stream>>>(c->d_wloc_next, (int)P, 0);
         k_iota<<<(int)((P + 255) / 256), 256, 0, c->stream>>>(c->d_anc, (int)P, 0);
         g_rp_launches += 3;
+    } else if (st == RP_OK) {
+        k_descend_cyclic<<<(int)((P + 255) / 256), 256, 0, c->stream>>>((int)P, (int)ne, c->d_anc, c->d_wloc, c->d_wloc_next);
+        ++g_rp_launches;
     }
-    if (st == RP_OK) st = rp_launch_pick_best(c, c->d_eval_score, lay, (int)P, best);
+    if (st == RP_OK) st = rp_launch_pick_best(c, c->d_eval_score, lay, (int)ne, best);
     cudaError_t e = cudaSuccess;
     if (st == RP_OK) e = cudaMemcpyAsync(c->d_seed_score, best, sizeof(i64) * 3, cudaMemcpyDeviceToDevice, c->stream);
     dev_free(c, best);
@@ -834,7 +849,7 @@ extern "C" int rp_init_population(rp_ctx *c, int32_t n_candidates, int32_t choic
         // the population proper
         c->Ppop = P;
         if ((st = build_population(c)) != RP_OK) break;
-        if ((st = install_population(c, fin)) != RP_OK) break;
+        if ((st = install_population(c, fin, nd)) != RP_OK) break;          // rows nd.. repeat the first nd
         if ((e = cudaStreamSynchronize(c->stream)) != cudaSuccess) break;
         if (n_distinct) *n_distinct = nd;
         if (picked) memcpy(picked, pick, sizeof(int) * P);

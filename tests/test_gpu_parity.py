@@ -642,7 +642,7 @@ def oracle_init_population(w, ref, edp, M, pop, width, n_proj, eta):
 
 
 @pytest.mark.parametrize("case,M,pop", [("shared", 60, 24), ("shared", 10, 24), ("interleaved", 33, 33), ("medium", 80, 48),
-                                        ("identity", 2, 5), ("copies", 40, 16)])
+                                        ("identity", 2, 5), ("copies", 40, 16), ("slices", 12, 40), ("slices_shared", 9, 30)])
 def test_algorithm_2_as_one_call(case, M, pop):
     """rp_init_population against the composition of the oracle's stages: how many candidates are
     distinct, which candidate every member is, the members' layouts and scores, the incumbent, and
@@ -659,6 +659,11 @@ def test_algorithm_2_as_one_call(case, M, pop):
     elif case == "interleaved":
         w = make_window(custom_spec("a2_inter", 120, 7, 24, 3, 4096, 6, 6, pop, 400, data_seed=46))
         edp, min_rows = [0, 1, 2, 0, 1, 2], 2
+    elif case in ("slices", "slices_shared"):
+        # rank loads in the slice pool, fewer candidates than members: the repeated members share
+        # their original's slices until they rewrite them
+        w = make_window(custom_spec("a2_slices", 120, 20, 32, 2, 4096, 4, 32, pop, 400, data_seed=47))
+        edp = [0, 1, 1, 0] if case == "slices_shared" else None
     else:
         w = make_window(custom_spec("a2_ident", 77, 3, 12, 2, 3000, 3, 3, pop, 400, data_seed=48))
         min_rows = 4
