@@ -618,7 +618,6 @@ int rp_launch_anneal_level(rp_ctx *c, int level, int n_levels, const rp_anneal_p
 #define COOP_PICK(SL_, ID_)                                  \
     switch (minb) {                                          \
         case 5: COOP_LAUNCH(5, SL_, ID_); break;             \
-        case 4: COOP_LAUNCH(4, SL_, ID_); break;             \
         default: COOP_LAUNCH(6, SL_, ID_); break;            \
     }
     if (A.slices) { if (alias) { COOP_PICK(true, true) } else { COOP_PICK(true, false) } }
