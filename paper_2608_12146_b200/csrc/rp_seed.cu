@@ -10,10 +10,14 @@
 
 #define SEED_WARPS 4
 
+// Warp minimum of 64-bit keys with two reduction instructions: the smallest high word, then the
+// smallest low word among the lanes that hold it.
 __device__ __forceinline__ u64 warp_min_u64(u64 v)
 {
-    for (int o = 16; o; o >>= 1) { const u64 x = __shfl_xor_sync(0xffffffffu, v, o); v = x < v ? x : v; }
-    return v;
+    const u32 hi = (u32)(v >> 32), lo = (u32)v;
+    const u32 mh = __reduce_min_sync(0xffffffffu, hi);
+    const u32 ml = __reduce_min_sync(0xffffffffu, hi == mh ? lo : 0xffffffffu);
+    return ((u64)mh << 32) | ml;
 }
 
 __global__ void __launch_bounds__(SEED_WARPS * 32)
