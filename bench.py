@@ -590,6 +590,12 @@ def run_cuda(args):
         if extras:
             l2 = l2_read_rate(rp)
             line["l2_read_gbs"] = l2
+            # the chain kernels' L2 traffic (ncu capture) against the L2 read rate measured in this run
+            for rec in [line] + list((line.get("other_workloads") or {}).values()):
+                dram = rec["roofline"].get("dram")
+                if dram and dram.get("l2_bytes_per_launch"):
+                    dram["l2_gbs"] = dram["l2_bytes_per_launch"] / (rec["roofline"]["launch_ms"] * 1e-3) / 1e9
+                    dram["l2_frac_of_measured_read_rate"] = dram["l2_gbs"] / l2
             line["eval_population"] = [eval_stage(rp, torch, n, dev, l2) for n in ("medium", "large", "wide")]
             line["concurrent_plans"] = [concurrent_plans(rp, torch, "medium", dev, n, 200, pl) for pl in (1, 0) for n in (1, 2, 4)]
             # large: one warp per chain and 7 warps per SM for a single window, so several windows fit the SMs at once
